@@ -1,0 +1,487 @@
+"""CPU oracle for the streaming decoder step.  TEST INFRASTRUCTURE ONLY.
+
+Plain, slow, float64 numpy restatement of what the per-chunk decoder step
+computes.  Only the tests, the smoke check and the benchmark's cpu-baseline /
+reference legs may import this module; the product path (the CUDA library and
+its Python binding) never does, and shares no code, table or constant with it.
+
+Two independent formulations are given for every pipeline:
+
+* ``*_offline``  - the plain definition: the causal network evaluated over the
+  whole concatenated input, with the chunk boundaries known (they only matter
+  for attention: every frame of a chunk sees its whole chunk plus at most W
+  carried frames before the chunk start).
+* ``*Stream``    - chunk-by-chunk evaluation with explicit carries that are
+  updated by "concatenate, compute, keep the last rows" (the stock discipline
+  the paper's Eq. 4 replaces by an in-place write), or, for the KV carry,
+  optionally by an in-place ring (``carry="ring"``), whose equality with the
+  concatenating form is the content of Eq. 4.
+
+The paper (a runtime-systems paper) fixes the streaming semantics - carried
+state per solver step and layer (Section 3.1, product clock "solver step x mel
+frame"), retention capped after inference (Section 3.1, envelope vs attended
+extent), in-place carry (Section 3.2, Eq. 4), admission f <= f_chunk - but not
+the layer arithmetic, which is fixed by the benchmark configurations and the
+readings listed in the design notes.  Pins: see tests/test_oracle_*.py.
+Whole-configuration outputs have no value printed in the paper: parity
+unpinned against the paper for those; they are pinned by closed forms, brute
+force, library special cases and the streamed == offline invariant.
+
+Precision: all arithmetic in float64.  For ``precision == "bf16"`` the values
+are additionally rounded (round-to-nearest-even to 8 significant bits) at the
+declared storage points: weight matrices, the input-projection operand
+[x_s | mu], every stored residual-stream activation h, the normalised
+activation u, q, k, v, the unnormalised softmax numerators (the row sum uses
+the unrounded ones) and the attention output o.  Biases, the timestep bias
+tau, the Euler state x_s and all accumulations stay unrounded.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------------------------
+# scalar helpers
+# --------------------------------------------------------------------------------------------
+
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """Round float64 values to the nearest bfloat16 (8-bit significand, ties to
+    even), returned as float64.  Exponent range is not clamped (values here
+    are O(1))."""
+    x = np.asarray(x, dtype=np.float64)
+    m, e = np.frexp(x)                       # x = m * 2**e, 0.5 <= |m| < 1
+    return np.ldexp(np.rint(m * 256.0), e - 8)
+
+
+def silu(z: np.ndarray) -> np.ndarray:
+    return z / (1.0 + np.exp(-z))
+
+
+def rmsnorm(h: np.ndarray, eps: float) -> np.ndarray:
+    """Parameter-free RMS normalisation over the channel axis."""
+    return h / np.sqrt(np.mean(h * h, axis=-1, keepdims=True) + eps)
+
+
+def timestep_embedding(t: float, C: int) -> np.ndarray:
+    """emb[i] = sin(1000 t w_i), emb[C/2+i] = cos(1000 t w_i), w_i = 10000^(-i/(C/2))."""
+    half = C // 2
+    i = np.arange(half, dtype=np.float64)
+    w = 10000.0 ** (-i / half)
+    return np.concatenate([np.sin(1000.0 * t * w), np.cos(1000.0 * t * w)])
+
+
+def shift_rows(x: np.ndarray, delta: int, left: Optional[np.ndarray] = None) -> np.ndarray:
+    """Row i of the result is row i-delta of x; rows before the start come from
+    `left` (its last rows) or are zero."""
+    F = x.shape[0]
+    if left is None:
+        left = np.zeros((delta, x.shape[1]))
+    ext = np.concatenate([left[left.shape[0] - delta:], x], axis=0) if delta else x
+    return ext[:F]
+
+
+def causal_conv_k3(x: np.ndarray, W: np.ndarray, d: int,
+                   left: Optional[np.ndarray] = None) -> np.ndarray:
+    """y[i] = sum_{j=0..2} x[i-(2-j)d] @ W[j]  (cross-correlation, tap 2 = current
+    frame); frames before the start are `left` (shape [2d, C_in]) or zeros."""
+    if left is None:
+        left = np.zeros((2 * d, x.shape[1]))
+    y = np.zeros((x.shape[0], W.shape[2]))
+    for j in range(3):
+        y += shift_rows(x, (2 - j) * d, left) @ W[j]
+    return y
+
+
+# --------------------------------------------------------------------------------------------
+# weights
+# --------------------------------------------------------------------------------------------
+
+def parse_blob(cfg, blob: np.ndarray) -> Dict[str, np.ndarray]:
+    """Split the canonical flat float32 blob into named float64 tensors.  In bf16
+    precision the matrices are rounded to bf16; biases are not."""
+    blob = np.asarray(blob, dtype=np.float32)
+    W: Dict[str, np.ndarray] = {}
+    pos = 0
+    bf = cfg.precision == "bf16"
+
+    def take(name, shape, is_bias=False):
+        nonlocal pos
+        n = int(np.prod(shape))
+        a = blob[pos:pos + n].astype(np.float64).reshape(shape)
+        pos += n
+        W[name] = round_bf16(a) if (bf and not is_bias) else a
+
+    C = cfg.hidden
+    if cfg.pipeline == "conv":
+        for l in range(len(cfg.dilations)):
+            take(f"conv{l}.W", (3, C, C))
+            take(f"conv{l}.b", (C,), True)
+    elif cfg.pipeline == "flow":
+        m = cfg.mel_dim
+        take("in.W", (2 * m, C))
+        take("in.b", (C,), True)
+        l = 0
+        for g in range(max(cfg.n_attn_layers, 1)):
+            for _ in range(cfg.conv_per_attn):
+                take(f"conv{l}.W", (3, C, C))
+                take(f"conv{l}.b", (C,), True)
+                take(f"conv{l}.P", (C, C))
+                l += 1
+            if cfg.n_attn_layers:
+                for nm in ("Wq", "Wk", "Wv", "Wo"):
+                    take(f"attn{g}.{nm}", (C, C))
+                for nm in ("bq", "bk", "bv", "bo"):
+                    take(f"attn{g}.{nm}", (C,), True)
+        take("out.W", (C, m))
+        take("out.b", (m,), True)
+    elif cfg.pipeline == "vocoder":
+        ch = cfg.up_channels
+        take("pre.W", (3, cfg.mel_dim, ch[0]))
+        take("pre.b", (ch[0],), True)
+        for q, s in enumerate(cfg.up_strides):
+            take(f"up{q}.Wt", (2 * s, ch[q], ch[q + 1]))
+            take(f"up{q}.bt", (ch[q + 1],), True)
+            for r in range(len(cfg.res_dilations)):
+                take(f"up{q}.res{r}.W", (3, ch[q + 1], ch[q + 1]))
+                take(f"up{q}.res{r}.b", (ch[q + 1],), True)
+        take("head.W", (3, ch[-1], cfg.n_fft + 2))
+        take("head.b", (cfg.n_fft + 2,), True)
+    else:
+        raise ValueError(cfg.pipeline)
+    if pos != blob.size:
+        raise ValueError(f"weight blob has {blob.size} floats, layout needs {pos}")
+    return W
+
+
+def tau_table(cfg, W) -> np.ndarray:
+    """tau[s][l] = emb(s / n_steps) @ P_l : the per-step, per-block timestep bias."""
+    n, L, C = cfg.n_steps, len(cfg.dilations), cfg.hidden
+    tau = np.zeros((n, L, C))
+    for s in range(n):
+        e = timestep_embedding(s / n, C)
+        for l in range(L):
+            tau[s, l] = e @ W[f"conv{l}.P"]
+    return tau
+
+
+# --------------------------------------------------------------------------------------------
+# conv stack (tiny causal conv stream)
+# --------------------------------------------------------------------------------------------
+
+def conv_stack_offline(cfg, blob, x: np.ndarray) -> np.ndarray:
+    """y = block_L(...block_1(x)),  block: h <- h + SiLU(conv_k3,d(h) + b)."""
+    W = parse_blob(cfg, blob)
+    h = np.asarray(x, dtype=np.float64)
+    for l, d in enumerate(cfg.dilations):
+        h = h + silu(causal_conv_k3(h, W[f"conv{l}.W"], d) + W[f"conv{l}.b"])
+    return h.astype(np.float32)
+
+
+class ConvStackStream:
+    """Chunk-by-chunk conv stack; carry per block = last 2d input frames."""
+
+    def __init__(self, cfg, blob):
+        self.cfg = cfg
+        self.W = parse_blob(cfg, blob)
+        self.carry = [np.zeros((2 * d, cfg.hidden)) for d in cfg.dilations]
+
+    def decode_chunk(self, x: np.ndarray) -> np.ndarray:
+        h = np.asarray(x, dtype=np.float64)
+        assert 1 <= h.shape[0] <= self.cfg.f_chunk
+        for l, d in enumerate(self.cfg.dilations):
+            left = self.carry[l]
+            self.carry[l] = np.concatenate([left, h], axis=0)[-2 * d:]
+            h = h + silu(causal_conv_k3(h, self.W[f"conv{l}.W"], d, left) + self.W[f"conv{l}.b"])
+        return h.astype(np.float32)
+
+
+# --------------------------------------------------------------------------------------------
+# flow decoder
+# --------------------------------------------------------------------------------------------
+
+def _attend(cfg, q, k, v, rb):
+    """All rows of q attend to all rows of k/v (one chunk against its key set).
+    Per head: e = exp(s - max s), o = (rb(e) @ v) / sum(e)."""
+    H, dh = cfg.n_heads, cfg.head_dim
+    o = np.zeros_like(q)
+    for eta in range(H):
+        sl = slice(eta * dh, (eta + 1) * dh)
+        s = (q[:, sl] @ k[:, sl].T) / math.sqrt(dh)
+        e = np.exp(s - s.max(axis=1, keepdims=True))
+        o[:, sl] = (rb(e) @ v[:, sl]) / e.sum(axis=1, keepdims=True)
+    return rb(o)
+
+
+def _layer_plan(cfg):
+    """[('conv', l, d) ... ('attn', g)] in execution order."""
+    plan, l = [], 0
+    for g in range(max(cfg.n_attn_layers, 1)):
+        for _ in range(cfg.conv_per_attn):
+            plan.append(("conv", l, cfg.dilations[l]))
+            l += 1
+        if cfg.n_attn_layers:
+            plan.append(("attn", g, 0))
+    return plan
+
+
+def flow_offline(cfg, blob, feats: np.ndarray, boundaries: Sequence[int]) -> np.ndarray:
+    """Offline causal run over the concatenated input.  feats[:, :mel] is the
+    conditioning mu, feats[:, mel:] the initial noise x_0.  For s in 0..n-1:
+    h = [x_s | mu] W_in + b_in; conv blocks h <- h + SiLU(conv(h) + b + tau_{s,l});
+    attention h <- h + attn(rmsnorm(h)) W_o + b_o with keys
+    K(i) = { j : max(0, B_c(i) - W) <= j < B_{c(i)+1} };
+    v = rmsnorm(h) W_out + b_out;  x_{s+1} = x_s + v / n.  Output x_n."""
+    W = parse_blob(cfg, blob)
+    rb = round_bf16 if cfg.precision == "bf16" else (lambda a: a)
+    m, n = cfg.mel_dim, cfg.n_steps
+    feats = np.asarray(feats, dtype=np.float64)
+    mu, x = feats[:, :m], feats[:, m:].copy()
+    F = feats.shape[0]
+    assert boundaries[0] == 0 and boundaries[-1] == F
+    tau = tau_table(cfg, W)
+    plan = _layer_plan(cfg)
+    for s in range(n):
+        h = rb(rb(np.concatenate([x, mu], axis=1)) @ W["in.W"] + W["in.b"])
+        for kind, idx, d in plan:
+            if kind == "conv":
+                z = causal_conv_k3(h, W[f"conv{idx}.W"], d) + W[f"conv{idx}.b"] + tau[s, idx]
+                h = rb(h + silu(z))
+            else:
+                u = rb(rmsnorm(h, cfg.rms_eps))
+                q = rb(u @ W[f"attn{idx}.Wq"] + W[f"attn{idx}.bq"])
+                k = rb(u @ W[f"attn{idx}.Wk"] + W[f"attn{idx}.bk"])
+                v = rb(u @ W[f"attn{idx}.Wv"] + W[f"attn{idx}.bv"])
+                o = np.zeros_like(q)
+                for c in range(len(boundaries) - 1):
+                    lo, hi = boundaries[c], boundaries[c + 1]
+                    k0 = max(0, lo - cfg.kv_cap)
+                    o[lo:hi] = _attend(cfg, q[lo:hi], k[k0:hi], v[k0:hi], rb)
+                h = rb(h + o @ W[f"attn{idx}.Wo"] + W[f"attn{idx}.bo"])
+        vel = rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]
+        x = x + vel / n
+    return x.astype(np.float32)
+
+
+class KVRing:
+    """In-place KV carry: fixed storage of W + f_chunk rows, written at the head;
+    the attended rows are the last min(filled, W) + T rows ending at the head
+    (Eq. 4's discipline: same values as concatenate-then-truncate, constant
+    storage)."""
+
+    def __init__(self, cap: int, f_chunk: int, C: int):
+        self.cap, self.size = cap, cap + f_chunk
+        self.k = np.zeros((self.size, C))
+        self.v = np.zeros((self.size, C))
+        self.head = 0          # next row to write
+        self.filled = 0        # carried rows (<= cap)
+
+    def append_and_view(self, k, v):
+        T = k.shape[0]
+        idx = (self.head + np.arange(T)) % self.size
+        self.k[idx], self.v[idx] = k, v
+        L = self.filled + T
+        rows = (self.head + T - L + np.arange(L)) % self.size
+        self.head = (self.head + T) % self.size
+        self.filled = min(self.cap, L)
+        return self.k[rows], self.v[rows]
+
+
+class FlowStream:
+    """Chunk-by-chunk flow decoder.  State per Euler step s: per conv block the
+    last 2d block-input frames; per attention layer the keys/values of the last
+    <= W frames (empty at stream start)."""
+
+    def __init__(self, cfg, blob, carry: str = "concat"):
+        self.cfg = cfg
+        self.W = parse_blob(cfg, blob)
+        self.tau = tau_table(cfg, self.W)
+        self.plan = _layer_plan(cfg)
+        self.ring = carry == "ring"
+        C, n = cfg.hidden, cfg.n_steps
+        self.halo = [[np.zeros((2 * d, C)) for d in cfg.dilations] for _ in range(n)]
+        if self.ring:
+            self.kv = [[KVRing(cfg.kv_cap, cfg.f_chunk, C) for _ in range(cfg.n_attn_layers)]
+                       for _ in range(n)]
+        else:
+            self.kv = [[(np.zeros((0, C)), np.zeros((0, C))) for _ in range(cfg.n_attn_layers)]
+                       for _ in range(n)]
+        self.kv_len_seen: List[int] = []
+
+    def decode_chunk(self, feats: np.ndarray) -> np.ndarray:
+        cfg, W = self.cfg, self.W
+        rb = round_bf16 if cfg.precision == "bf16" else (lambda a: a)
+        feats = np.asarray(feats, dtype=np.float64)
+        T = feats.shape[0]
+        assert 1 <= T <= cfg.f_chunk
+        m, n = cfg.mel_dim, cfg.n_steps
+        mu, x = feats[:, :m], feats[:, m:].copy()
+        for s in range(n):
+            h = rb(rb(np.concatenate([x, mu], axis=1)) @ W["in.W"] + W["in.b"])
+            for kind, idx, d in self.plan:
+                if kind == "conv":
+                    left = self.halo[s][idx]
+                    self.halo[s][idx] = np.concatenate([left, h], axis=0)[-2 * d:]
+                    z = (causal_conv_k3(h, W[f"conv{idx}.W"], d, left)
+                         + W[f"conv{idx}.b"] + self.tau[s, idx])
+                    h = rb(h + silu(z))
+                else:
+                    u = rb(rmsnorm(h, cfg.rms_eps))
+                    q = rb(u @ W[f"attn{idx}.Wq"] + W[f"attn{idx}.bq"])
+                    k = rb(u @ W[f"attn{idx}.Wk"] + W[f"attn{idx}.bk"])
+                    v = rb(u @ W[f"attn{idx}.Wv"] + W[f"attn{idx}.bv"])
+                    if self.ring:
+                        if s == 0 and idx == 0:
+                            self.kv_len_seen.append(self.kv[s][idx].filled)
+                        k_all, v_all = self.kv[s][idx].append_and_view(k, v)
+                    else:
+                        kc, vc = self.kv[s][idx]
+                        if s == 0 and idx == 0:
+                            self.kv_len_seen.append(kc.shape[0])
+                        k_all = np.concatenate([kc, k], axis=0)
+                        v_all = np.concatenate([vc, v], axis=0)
+                        self.kv[s][idx] = (k_all[-cfg.kv_cap:], v_all[-cfg.kv_cap:])
+                    o = _attend(cfg, q, k_all, v_all, rb)
+                    h = rb(h + o @ W[f"attn{idx}.Wo"] + W[f"attn{idx}.bo"])
+            vel = rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]
+            x = x + vel / n
+        return x.astype(np.float32)
+
+
+# --------------------------------------------------------------------------------------------
+# vocoder tail: upsampler + head + iSTFT / overlap-add
+# --------------------------------------------------------------------------------------------
+
+def conv_transpose_causal(x: np.ndarray, Wt: np.ndarray, b: np.ndarray, stride: int,
+                          prev: Optional[np.ndarray] = None) -> np.ndarray:
+    """y[stride*n + r] = b + x[n] @ Wt[r] + x[n-1] @ Wt[r+stride], r in [0, stride);
+    x[-1] = prev (zeros at stream start).  This is ConvTranspose1d(stride, kernel
+    2*stride) with the trailing `stride` outputs deferred to the next frame."""
+    F = x.shape[0]
+    if prev is None:
+        prev = np.zeros((1, x.shape[1]))
+    xm1 = np.concatenate([prev.reshape(1, -1), x], axis=0)[:F]
+    y = np.zeros((F, stride, Wt.shape[2]))
+    for r in range(stride):
+        y[:, r, :] = b + x @ Wt[r] + xm1 @ Wt[r + stride]
+    return y.reshape(F * stride, Wt.shape[2])
+
+
+def hann_periodic(N: int) -> np.ndarray:
+    return 0.5 - 0.5 * np.cos(2.0 * np.pi * np.arange(N) / N)
+
+
+def frame_signal(z: np.ndarray, n_fft: int, clamp: float) -> np.ndarray:
+    """Head output z [M, n_fft+2] -> per-frame real signal xi [M, n_fft].
+    Channels [0, n_fft/2] are log-magnitudes (clamped from above), the rest are
+    phases; X_f = exp(m_f)(cos phi_f + i sin phi_f); inverse real DFT with 1/N
+    scaling, imaginary parts of the DC and Nyquist bins ignored."""
+    nb = n_fft // 2 + 1
+    mag = np.exp(np.minimum(z[:, :nb], clamp))
+    re, im = mag * np.cos(z[:, nb:]), mag * np.sin(z[:, nb:])
+    kap = np.arange(n_fft)
+    xi = re[:, 0:1] + re[:, nb - 1:nb] * ((-1.0) ** kap)[None, :]
+    for f in range(1, nb - 1):
+        ang = 2.0 * np.pi * f * kap / n_fft
+        xi = xi + 2.0 * (re[:, f:f + 1] * np.cos(ang)[None, :] - im[:, f:f + 1] * np.sin(ang)[None, :])
+    return xi / n_fft
+
+
+def ola_norm(n_fft: int, hop: int) -> float:
+    """Steady-state overlap-add envelope sum_j w[j*hop]^2 (1.5 for periodic Hann, hop N/4)."""
+    w = hann_periodic(n_fft)
+    return float(sum(w[j] ** 2 for j in range(0, n_fft, hop)))
+
+
+def overlap_add(xi: np.ndarray, n_fft: int, hop: int, tail: Optional[np.ndarray] = None):
+    """pcm[n] = (1/norm) sum_m w[n - hop m] xi_m[n - hop m]; returns the hop*M
+    finalised samples and the (n_fft - hop)-sample unnormalised tail to carry."""
+    M = xi.shape[0]
+    w = hann_periodic(n_fft)
+    acc = np.zeros(hop * M + n_fft - hop)
+    if tail is not None:
+        acc[:n_fft - hop] += tail
+    for mfr in range(M):
+        acc[hop * mfr: hop * mfr + n_fft] += w * xi[mfr]
+    return acc[:hop * M] / ola_norm(n_fft, hop), acc[hop * M:]
+
+
+def vocoder_offline(cfg, blob, mel: np.ndarray) -> np.ndarray:
+    W = parse_blob(cfg, blob)
+    a = causal_conv_k3(np.asarray(mel, dtype=np.float64), W["pre.W"], 1) + W["pre.b"]
+    for q, s in enumerate(cfg.up_strides):
+        a = conv_transpose_causal(a, W[f"up{q}.Wt"], W[f"up{q}.bt"], s)
+        for r, d in enumerate(cfg.res_dilations):
+            a = a + silu(causal_conv_k3(a, W[f"up{q}.res{r}.W"], d) + W[f"up{q}.res{r}.b"])
+    z = causal_conv_k3(silu(a), W["head.W"], 1) + W["head.b"]
+    xi = frame_signal(z, cfg.n_fft, cfg.logmag_clamp)
+    pcm, _ = overlap_add(xi, cfg.n_fft, cfg.hop)
+    return pcm.astype(np.float32)
+
+
+class VocoderStream:
+    """Chunk-by-chunk vocoder tail.  Carries: last 2 mel frames, last input frame
+    of each transposed conv, last 2d input frames of each residual block, last 2
+    frames before the head, and the n_fft - hop overlap-add partial sums."""
+
+    def __init__(self, cfg, blob):
+        self.cfg = cfg
+        self.W = parse_blob(cfg, blob)
+        ch = cfg.up_channels
+        self.c_pre = np.zeros((2, cfg.mel_dim))
+        self.c_up = [np.zeros((1, ch[q])) for q in range(len(cfg.up_strides))]
+        self.c_res = [[np.zeros((2 * d, ch[q + 1])) for d in cfg.res_dilations]
+                      for q in range(len(cfg.up_strides))]
+        self.c_head = np.zeros((2, ch[-1]))
+        self.tail = np.zeros(cfg.n_fft - cfg.hop)
+
+    def decode_chunk(self, mel: np.ndarray) -> np.ndarray:
+        cfg, W = self.cfg, self.W
+        x = np.asarray(mel, dtype=np.float64)
+        assert 1 <= x.shape[0] <= cfg.f_chunk
+        left, self.c_pre = self.c_pre, np.concatenate([self.c_pre, x], axis=0)[-2:]
+        a = causal_conv_k3(x, W["pre.W"], 1, left) + W["pre.b"]
+        for q, s in enumerate(cfg.up_strides):
+            prev, self.c_up[q] = self.c_up[q], a[-1:].copy()
+            a = conv_transpose_causal(a, W[f"up{q}.Wt"], W[f"up{q}.bt"], s, prev)
+            for r, d in enumerate(cfg.res_dilations):
+                left = self.c_res[q][r]
+                self.c_res[q][r] = np.concatenate([left, a], axis=0)[-2 * d:]
+                a = a + silu(causal_conv_k3(a, W[f"up{q}.res{r}.W"], d, left) + W[f"up{q}.res{r}.b"])
+        g = silu(a)
+        left, self.c_head = self.c_head, np.concatenate([self.c_head, g], axis=0)[-2:]
+        z = causal_conv_k3(g, W["head.W"], 1, left) + W["head.b"]
+        xi = frame_signal(z, cfg.n_fft, cfg.logmag_clamp)
+        pcm, self.tail = overlap_add(xi, cfg.n_fft, cfg.hop, self.tail)
+        return pcm.astype(np.float32)
+
+
+# --------------------------------------------------------------------------------------------
+# drivers
+# --------------------------------------------------------------------------------------------
+
+def make_stream(cfg, blob, **kw):
+    if cfg.pipeline == "conv":
+        return ConvStackStream(cfg, blob)
+    if cfg.pipeline == "flow":
+        return FlowStream(cfg, blob, **kw)
+    if cfg.pipeline == "vocoder":
+        return VocoderStream(cfg, blob)
+    raise ValueError(cfg.pipeline)
+
+
+def run_offline(cfg, blob, feats, boundaries) -> np.ndarray:
+    if cfg.pipeline == "conv":
+        return conv_stack_offline(cfg, blob, feats)
+    if cfg.pipeline == "flow":
+        return flow_offline(cfg, blob, feats, boundaries)
+    return vocoder_offline(cfg, blob, feats)
+
+
+def run_stream(cfg, blob, feats, boundaries, **kw) -> np.ndarray:
+    st = make_stream(cfg, blob, **kw)
+    outs = [st.decode_chunk(feats[boundaries[c]:boundaries[c + 1]])
+            for c in range(len(boundaries) - 1)]
+    return np.concatenate(outs, axis=0)
