@@ -1,0 +1,175 @@
+/*
+ * dc.h - C ABI of the streaming decoder step (one GPU, sm_100a).
+ *
+ * One call of dc_decode_chunk / dc_decode_batch runs the whole per-chunk decoder
+ * step on the device: for the flow decoder the input projection, the causal
+ * conv residual blocks and chunk-causal attention over [carried state | new
+ * chunk], repeated for every Euler step, with the Euler update; for the
+ * vocoder tail the transposed-conv upsampler, the magnitude/phase head and the
+ * inverse STFT with overlap-add.  All state that crosses chunks (conv left
+ * context, key/value carry, overlap-add tail) lives in device buffers that are
+ * allocated once per stream, keep their address for the stream's lifetime and
+ * are read and written in place (paper Section 3.2, "State Rule", Eq. 4: the
+ * carry is written into existing storage and its pointer stays constant; the
+ * retained extent is capped after inference, Section 3.1 "Two extents").
+ *
+ * Conventions
+ *   - All matrices are row-major, one frame per row, channels contiguous.
+ *   - "dev" pointers are device pointers valid on the model's device, "host"
+ *     pointers are ordinary host pointers.  The library never takes ownership
+ *     of a caller buffer.
+ *   - Every function returns a dc_status; nothing throws or aborts.  Argument
+ *     and admission checks run before any state is touched (fail closed, paper
+ *     Section 3.3 admission clauses; the admission predicate is
+ *     1 <= n_frames <= f_chunk, Section 3.1).
+ *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and is asynchronous unless
+ *     stated otherwise.  A model owns one set of scratch buffers: all decode
+ *     calls on streams of one model must be ordered on the device (use one
+ *     CUDA stream, or synchronise between calls).
+ *   - There is no CPU fallback: without a usable sm_100 device every call that
+ *     needs the device fails with DC_ERR_CUDA.
+ */
+#ifndef DC_H_
+#define DC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dc_model  dc_model;   /* immutable after creation: packed weights, constant tables */
+typedef struct dc_stream dc_stream;  /* mutable: every carry of one audio stream                   */
+
+typedef enum dc_status {
+  DC_OK = 0,
+  DC_ERR_ARG = 1,      /* null pointer, bad size, bad batch                                  */
+  DC_ERR_CONFIG = 2,   /* configuration outside what the kernels support                     */
+  DC_ERR_FRAMES = 3,   /* admission predicate violated: n_frames < 1 or n_frames > f_chunk   */
+  DC_ERR_OOM = 4,      /* device or host allocation failed                                   */
+  DC_ERR_CUDA = 5,     /* a CUDA call failed (see dc_last_error)                             */
+  DC_ERR_TIMEOUT = 6,  /* a bounded device-side wait gave up; the stream is poisoned         */
+  DC_ERR_STATE = 7     /* closed or poisoned stream, or streams of different models          */
+} dc_status;
+
+enum { DC_PIPE_CONV = 1, DC_PIPE_FLOW = 2, DC_PIPE_VOCODER = 3 };
+enum { DC_F32 = 0, DC_BF16 = 1 };   /* DC_BF16: bf16 storage and operands, fp32 accumulation */
+
+#define DC_MAX_CONV 32
+#define DC_MAX_UP 4
+#define DC_MAX_RES 4
+
+/* Plain-data description of the network.  Unused fields are zero.
+ *   DC_PIPE_CONV    : hidden, n_conv, dilations[]           (fp32)
+ *   DC_PIPE_FLOW    : hidden, n_conv, dilations[], n_attn, n_heads, head_dim, kv_cap,
+ *                     n_steps, mel_dim                       (bf16)
+ *   DC_PIPE_VOCODER : mel_dim, n_up, up_strides[], up_channels[n_up+1], n_res,
+ *                     res_dilations[], n_fft, hop, logmag_clamp   (fp32)
+ * The flow decoder runs n_conv / n_attn conv blocks, then one attention layer,
+ * repeated n_attn times (n_attn = 0: conv blocks only). */
+typedef struct dc_config {
+  uint32_t size;                 /* sizeof(dc_config), for versioning                        */
+  int32_t  pipeline;             /* DC_PIPE_*                                                */
+  int32_t  precision;            /* DC_F32 | DC_BF16                                         */
+  int32_t  hidden;               /* C                                                        */
+  int32_t  n_conv;               /* causal conv residual blocks (k = 3)                      */
+  int32_t  dilations[DC_MAX_CONV];
+  int32_t  n_attn, n_heads, head_dim;
+  int32_t  kv_cap;               /* W: carried key/value frames per (step, layer)            */
+  int32_t  n_steps;              /* Euler steps per chunk                                    */
+  int32_t  f_chunk;              /* largest admitted n_frames                                */
+  int32_t  mel_dim;
+  int32_t  n_up;
+  int32_t  up_strides[DC_MAX_UP];
+  int32_t  up_channels[DC_MAX_UP + 1];
+  int32_t  n_res;
+  int32_t  res_dilations[DC_MAX_RES];
+  int32_t  n_fft, hop;
+  float    rms_eps;
+  float    logmag_clamp;
+  int32_t  max_batch;            /* most streams one dc_decode_batch call may carry (>= 1)   */
+} dc_config;
+
+/* Number of floats of the canonical weight blob for this configuration, 0 if the
+ * configuration is invalid.  Blob order (all matrices [C_in][C_out], conv and
+ * transposed-conv weights tap-major [tap][C_in][C_out], tap 2 of a conv = current
+ * frame):
+ *   conv    : per block W[3][C][C], b[C]
+ *   flow    : W_in[2 mel][C], b_in[C]; per group: per conv block W[3][C][C], b[C],
+ *             P[C][C] (timestep bias tau = emb(t_s) P); then W_q, W_k, W_v, W_o [C][C],
+ *             b_q, b_k, b_v, b_o [C]; finally W_out[C][mel], b_out[mel]
+ *   vocoder : W_pre[3][mel][C0], b; per stage Wt[2 stride][C_in][C_out], b, per residual
+ *             block W[3][C_out][C_out], b; W_head[3][C_last][n_fft+2], b. */
+size_t dc_weights_count(const dc_config* cfg);
+
+/* Builds a model on the current CUDA device: validates cfg, converts and packs
+ * the weights (bf16 round-to-nearest-even for DC_BF16), precomputes the constant
+ * tables (per-step timestep bias, synthesis window) and allocates the scratch
+ * buffers for max_batch streams.  weights_host: n_floats floats in the canonical
+ * order; the caller may free it on return.  Synchronous.  (Device-resident
+ * constants: paper Section 3.1, "constant has a trivial clock".) */
+dc_status dc_create(const float* weights_host, size_t n_floats, const dc_config* cfg, dc_model** out);
+
+/* Frees a model.  All its streams must be closed first (else DC_ERR_STATE). */
+dc_status dc_destroy(dc_model* model);
+
+/* Allocates and zeroes every carry of one stream (conv left context per (step,
+ * block), key/value ring per (step, attention layer), vocoder left contexts,
+ * overlap-add tail).  The buffers never move until dc_stream_close (paper
+ * Section 3.2: pointer constancy over the stream lifetime).  Synchronous. */
+dc_status dc_stream_open(dc_model* model, dc_stream** out);
+
+/* Turn boundary: writes the base state (zeros, empty key/value carry) into the
+ * existing buffers, on cuda_stream; addresses do not change (Section 3.2). */
+dc_status dc_stream_reset(dc_stream* stream, void* cuda_stream);
+
+dc_status dc_stream_close(dc_stream* stream);
+
+/* One chunk of one stream.
+ *   feats_dev : device fp32 [n_frames][F_in]; F_in = hidden (conv), 2*mel_dim (flow:
+ *               cols [0,mel) conditioning, [mel,2 mel) initial noise), mel_dim (vocoder)
+ *   out_dev   : device fp32; conv: [n_frames][hidden]; flow: [n_frames][mel_dim];
+ *               vocoder: n_frames * prod(up_strides) * hop PCM samples
+ *   n_out     : host pointer (may be NULL) receiving the number of floats written
+ * Fails with DC_ERR_FRAMES unless 1 <= n_frames <= f_chunk; a failed call leaves
+ * the stream untouched.  Allocates nothing. */
+dc_status dc_decode_chunk(dc_stream* stream, const float* feats_dev, int n_frames,
+                          float* out_dev, int* n_out, void* cuda_stream);
+
+/* One chunk for each of n distinct streams of one model (n <= max_batch) in one
+ * pass; stream i consumes n_frames[i] frames from feats_dev[i] and writes
+ * out_dev[i].  feats_dev, n_frames and out_dev are HOST arrays (of device
+ * pointers / ints).  Results are bitwise identical to n single dc_decode_chunk
+ * calls.  (Multi-session serving over shared weights with per-session state:
+ * paper Section 3.4, last paragraph, and Section 4.3 "Serving capacity".)  Flow pipeline only. */
+dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
+                          const float* const* feats_dev, const int* n_frames,
+                          float* const* out_dev, void* cuda_stream);
+
+/* Convenience for callers with host buffers: copies feats_host to the device,
+ * decodes, copies the result back and synchronises cuda_stream.  Uses staging
+ * buffers owned by the stream (allocated at dc_stream_open). */
+dc_status dc_decode_chunk_host(dc_stream* stream, const float* feats_host, int n_frames,
+                               float* out_host, int* n_out, void* cuda_stream);
+
+/* Device addresses and byte sizes of the stream's carry buffers, for pointer
+ * constancy checks: writes up to max_entries (address, bytes) pairs into out and
+ * the number of buffers into n_entries. */
+dc_status dc_stream_carry_info(const dc_stream* stream, uint64_t* out, int max_entries, int* n_entries);
+
+/* counters[0] chunks decoded, [1] frames decoded, [2] calls rejected (DC_ERR_FRAMES),
+ * [3] calls rejected (other argument/state errors), [4] device timeouts,
+ * [5] kernel launches issued, [6] streams open, [7] reserved. */
+dc_status dc_get_counters(const dc_model* model, uint64_t counters[8]);
+
+const char* dc_status_str(dc_status s);
+
+/* Text of the last CUDA or validation error on the calling thread ("" if none). */
+const char* dc_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* DC_H_ */

@@ -1,0 +1,212 @@
+"""ctypes binding with the same names as include/dc.h."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libdc.so")
+_lib = None
+
+DC_MAX_CONV, DC_MAX_UP, DC_MAX_RES = 32, 4, 4
+PIPE = {"conv": 1, "flow": 2, "vocoder": 3}
+PREC = {"f32": 0, "bf16": 1}
+STATUS = {0: "DC_OK", 1: "DC_ERR_ARG", 2: "DC_ERR_CONFIG", 3: "DC_ERR_FRAMES", 4: "DC_ERR_OOM",
+          5: "DC_ERR_CUDA", 6: "DC_ERR_TIMEOUT", 7: "DC_ERR_STATE"}
+
+EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_stream_reset",
+           "dc_stream_close", "dc_decode_chunk", "dc_decode_batch", "dc_decode_chunk_host",
+           "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error"]
+
+
+class dc_config(C.Structure):
+    _fields_ = [("size", C.c_uint32), ("pipeline", C.c_int32), ("precision", C.c_int32),
+                ("hidden", C.c_int32), ("n_conv", C.c_int32), ("dilations", C.c_int32 * DC_MAX_CONV),
+                ("n_attn", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("kv_cap", C.c_int32), ("n_steps", C.c_int32), ("f_chunk", C.c_int32),
+                ("mel_dim", C.c_int32), ("n_up", C.c_int32), ("up_strides", C.c_int32 * DC_MAX_UP),
+                ("up_channels", C.c_int32 * (DC_MAX_UP + 1)), ("n_res", C.c_int32),
+                ("res_dilations", C.c_int32 * DC_MAX_RES), ("n_fft", C.c_int32), ("hop", C.c_int32),
+                ("rms_eps", C.c_float), ("logmag_clamp", C.c_float), ("max_batch", C.c_int32)]
+
+
+class DCError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = load_library().dc_last_error().decode()
+        super().__init__(f"{where}: {STATUS.get(status, status)} {msg}")
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Loads libdc.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2609_35115_b200.build`")
+    lib = C.CDLL(_LIB_PATH)
+    vp, cp = C.c_void_p, C.POINTER
+    lib.dc_weights_count.restype = C.c_size_t
+    lib.dc_weights_count.argtypes = [cp(dc_config)]
+    lib.dc_create.argtypes = [vp, C.c_size_t, cp(dc_config), cp(vp)]
+    lib.dc_destroy.argtypes = [vp]
+    lib.dc_stream_open.argtypes = [vp, cp(vp)]
+    lib.dc_stream_reset.argtypes = [vp, vp]
+    lib.dc_stream_close.argtypes = [vp]
+    lib.dc_decode_chunk.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
+    lib.dc_decode_batch.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
+    lib.dc_decode_chunk_host.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
+    lib.dc_stream_carry_info.argtypes = [vp, cp(C.c_uint64), C.c_int, cp(C.c_int)]
+    lib.dc_get_counters.argtypes = [vp, cp(C.c_uint64)]
+    lib.dc_status_str.restype = C.c_char_p
+    lib.dc_status_str.argtypes = [C.c_int]
+    lib.dc_last_error.restype = C.c_char_p
+    lib.dc_last_error.argtypes = []
+    for fn in EXPORTS:
+        if fn not in ("dc_weights_count", "dc_status_str", "dc_last_error"):
+            getattr(lib, fn).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def make_config(cfg, max_batch: int = 1) -> dc_config:
+    """dc_workloads.DCConfig (or any object with the same attributes) -> dc_config."""
+    c = dc_config()
+    c.size = C.sizeof(dc_config)
+    c.pipeline = PIPE[cfg.pipeline]
+    c.precision = PREC[cfg.precision]
+    c.hidden = cfg.hidden
+    c.n_conv = len(cfg.dilations)
+    for i, d in enumerate(cfg.dilations):
+        c.dilations[i] = d
+    c.n_attn, c.n_heads, c.head_dim, c.kv_cap = cfg.n_attn_layers, cfg.n_heads, cfg.head_dim, cfg.kv_cap
+    c.n_steps, c.f_chunk, c.mel_dim = cfg.n_steps, cfg.f_chunk, cfg.mel_dim
+    if cfg.pipeline == "vocoder":
+        c.n_up = len(cfg.up_strides)
+        for i, s in enumerate(cfg.up_strides):
+            c.up_strides[i] = s
+        for i, ch in enumerate(cfg.up_channels):
+            c.up_channels[i] = ch
+        c.n_res = len(cfg.res_dilations)
+        for i, d in enumerate(cfg.res_dilations):
+            c.res_dilations[i] = d
+        c.n_fft, c.hop = cfg.n_fft, cfg.hop
+    c.rms_eps, c.logmag_clamp = cfg.rms_eps, cfg.logmag_clamp
+    c.max_batch = max_batch
+    return c
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise DCError(status, where)
+
+
+def _cuda_stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+class Model:
+    """dc_create / dc_destroy."""
+
+    def __init__(self, cfg, weights: np.ndarray, max_batch: int = 1):
+        self.lib = load_library()
+        self.cfg = cfg
+        self.c_cfg = make_config(cfg, max_batch)
+        w = np.ascontiguousarray(weights, dtype=np.float32)
+        self.handle = C.c_void_p()
+        _check(self.lib.dc_create(w.ctypes.data, w.size, C.byref(self.c_cfg), C.byref(self.handle)), "dc_create")
+        self.out_per_frame = cfg.out_per_frame
+        self.in_dim = cfg.in_dim
+
+    def weights_count(self) -> int:
+        return self.lib.dc_weights_count(C.byref(self.c_cfg))
+
+    def open_stream(self) -> "Stream":
+        return Stream(self)
+
+    def counters(self) -> List[int]:
+        out = (C.c_uint64 * 8)()
+        _check(self.lib.dc_get_counters(self.handle, out), "dc_get_counters")
+        return list(out)
+
+    def destroy(self):
+        if self.handle:
+            _check(self.lib.dc_destroy(self.handle), "dc_destroy")
+            self.handle = C.c_void_p()
+
+
+class Stream:
+    """dc_stream_open / dc_decode_chunk / dc_stream_reset / dc_stream_close."""
+
+    def __init__(self, model: Model):
+        self.model = model
+        self.lib = model.lib
+        self.handle = C.c_void_p()
+        _check(self.lib.dc_stream_open(model.handle, C.byref(self.handle)), "dc_stream_open")
+
+    def decode_chunk(self, feats, out=None, stream=None):
+        """feats: CUDA float32 tensor [T, in_dim]; returns a CUDA float32 tensor."""
+        import torch
+        assert feats.is_cuda and feats.dtype == torch.float32 and feats.is_contiguous()
+        T = feats.shape[0]
+        if out is None:
+            n = max(T, 0) * self.model.out_per_frame
+            out = torch.empty(max(n, 1), dtype=torch.float32, device=feats.device)
+        n_out = C.c_int(0)
+        st = self.lib.dc_decode_chunk(self.handle, feats.data_ptr(), T, out.data_ptr(), C.byref(n_out),
+                                      _cuda_stream_handle(stream))
+        _check(st, "dc_decode_chunk")
+        res = out[: n_out.value]
+        if self.model.cfg.pipeline != "vocoder":
+            res = res.view(T, -1)
+        return res
+
+    def decode_chunk_host(self, feats_host, out_host, stream=None) -> int:
+        """feats_host / out_host: CPU float32 tensors (pinned for true async copies)."""
+        T = feats_host.shape[0]
+        n_out = C.c_int(0)
+        st = self.lib.dc_decode_chunk_host(self.handle, feats_host.data_ptr(), T, out_host.data_ptr(),
+                                           C.byref(n_out), _cuda_stream_handle(stream))
+        _check(st, "dc_decode_chunk_host")
+        return n_out.value
+
+    def decode_raw(self, feats_ptr: int, T: int, out_ptr: int, stream=None) -> int:
+        """Unchecked pass-through (used by the error-path tests)."""
+        n_out = C.c_int(0)
+        return self.lib.dc_decode_chunk(self.handle, feats_ptr, T, out_ptr, C.byref(n_out),
+                                        _cuda_stream_handle(stream))
+
+    def carry_info(self):
+        buf = (C.c_uint64 * 256)()
+        n = C.c_int(0)
+        _check(self.lib.dc_stream_carry_info(self.handle, buf, 128, C.byref(n)), "dc_stream_carry_info")
+        return [(buf[2 * i], buf[2 * i + 1]) for i in range(min(n.value, 128))]
+
+    def reset(self, stream=None):
+        _check(self.lib.dc_stream_reset(self.handle, _cuda_stream_handle(stream)), "dc_stream_reset")
+
+    def close(self):
+        if self.handle:
+            _check(self.lib.dc_stream_close(self.handle), "dc_stream_close")
+            self.handle = C.c_void_p()
+
+
+def decode_batch(model: Model, streams: Sequence[Stream], feats: Sequence, outs: Sequence, stream=None):
+    """dc_decode_batch: one chunk for each stream; feats[i] CUDA float32 [T_i, in_dim]."""
+    n = len(streams)
+    hs = (C.c_void_p * n)(*[s.handle for s in streams])
+    fp = (C.c_void_p * n)(*[f.data_ptr() for f in feats])
+    op = (C.c_void_p * n)(*[o.data_ptr() for o in outs])
+    nf = (C.c_int * n)(*[f.shape[0] for f in feats])
+    _check(model.lib.dc_decode_batch(model.handle, n, hs, fp, nf, op, _cuda_stream_handle(stream)),
+           "dc_decode_batch")

@@ -1,0 +1,538 @@
+// C ABI of the streaming decoder step: model / stream lifetime, admission checks and the host
+// side of one chunk step.  Every step of the path runs in the kernels; this file only validates,
+// sizes the address-stable state and enqueues launches.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <atomic>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "dc_internal.h"
+
+namespace dc {
+
+static thread_local std::string g_last_error;
+
+void set_error(const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  g_last_error = buf;
+}
+
+#define DC_CUDA(expr)                                                                    \
+  do {                                                                                   \
+    cudaError_t e__ = (expr);                                                            \
+    if (e__ != cudaSuccess) {                                                            \
+      dc::set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), __FILE__, __LINE__); \
+      return e__ == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;                \
+    }                                                                                    \
+  } while (0)
+
+static int pow2_ceil(int v) {
+  int p = 1;
+  while (p < v) p <<= 1;
+  return p;
+}
+
+// One fp32 layer of the conv pipeline / vocoder tail.
+struct F32Layer {
+  int    kind;        // 0 conv k3, 1 transposed conv, 2 head + iSTFT
+  int    C_in, C_out;
+  int    dil;         // conv dilation
+  int    stride;      // transposed conv stride
+  int    rate_in;     // input frames of this layer per chunk frame
+  int    halo;        // left-context frames it reads
+  int    residual_silu, post_silu;
+  size_t w_off, b_off;  // float offsets in the blob
+  int    ring_cap;    // rows of its input ring
+};
+
+}  // namespace dc
+
+using dc::DevBuf;
+using dc::F32Layer;
+
+struct dc_model {
+  dc_config cfg;
+  int       device = 0;
+  float*    d_w = nullptr;   // fp32 pipelines: the blob on the device
+  std::vector<F32Layer> layers;
+  int       out_per_frame = 0;
+  int       in_dim = 0;
+  dc::FlowModel* flow = nullptr;
+  std::atomic<uint64_t> counters[8];
+  std::atomic<int> open_streams{0};
+  std::mutex mu;
+  std::vector<dc_stream*> all_streams;   // host structs live until dc_destroy, so a closed handle stays detectable
+};
+
+struct dc_stream {
+  dc_model* model = nullptr;
+  bool      closed = false, poisoned = false;
+  long long frames_total = 0;
+  long long chunks = 0;
+  std::vector<DevBuf> f32_rings;   // input ring of each fp32 layer
+  float*    tails = nullptr;       // [2][12] overlap-add tails (ping-pong)
+  dc::FlowState* flow = nullptr;
+  float*    stage_in = nullptr;    // device staging of dc_decode_chunk_host
+  float*    stage_out = nullptr;
+};
+
+// ---------------------------------------------------------------------------------------------
+// configuration
+// ---------------------------------------------------------------------------------------------
+
+static bool config_ok(const dc_config* c, const char** why) {
+#define BAD(msg) do { *why = msg; return false; } while (0)
+  if (!c) BAD("null config");
+  if (c->size != sizeof(dc_config)) BAD("dc_config.size mismatch");
+  if (c->f_chunk < 1 || c->f_chunk > 4096) BAD("f_chunk out of range");
+  if (c->max_batch < 1 || c->max_batch > 1024) BAD("max_batch out of range");
+  if (c->pipeline == DC_PIPE_CONV) {
+    if (c->precision != DC_F32) BAD("conv pipeline is fp32");
+    if (c->hidden < 4 || c->hidden % 4) BAD("hidden must be a multiple of 4");
+    if (c->n_conv < 1 || c->n_conv > DC_MAX_CONV) BAD("n_conv out of range");
+    for (int l = 0; l < c->n_conv; ++l)
+      if (c->dilations[l] < 1 || c->dilations[l] > 64) BAD("dilation out of range");
+  } else if (c->pipeline == DC_PIPE_FLOW) {
+    if (c->precision != DC_BF16) BAD("flow pipeline is bf16");
+    if (c->hidden < 64 || c->hidden % 64 || c->hidden > 2048) BAD("hidden must be a multiple of 64");
+    if (c->n_conv < 1 || c->n_conv > DC_MAX_CONV) BAD("n_conv out of range");
+    for (int l = 0; l < c->n_conv; ++l)
+      if (c->dilations[l] < 1 || c->dilations[l] > 4) BAD("flow conv dilation must be 1..4");
+    if (c->n_attn < 0 || (c->n_attn > 0 && c->n_conv % c->n_attn)) BAD("n_conv must be a multiple of n_attn");
+    if (c->n_attn > 0) {
+      if (c->head_dim != 32 && c->head_dim != 64) BAD("head_dim must be 32 or 64");
+      if (c->n_heads * c->head_dim != c->hidden) BAD("n_heads * head_dim != hidden");
+      if (c->kv_cap < 1 || c->kv_cap > 4096) BAD("kv_cap out of range");
+    }
+    if (c->n_steps < 1 || c->n_steps > 64) BAD("n_steps out of range");
+    if (c->mel_dim < 16 || c->mel_dim % 16 || c->mel_dim > 128) BAD("mel_dim must be a multiple of 16, <= 128");
+    if (c->f_chunk > 56) BAD("flow f_chunk must be <= 56");
+  } else if (c->pipeline == DC_PIPE_VOCODER) {
+    if (c->precision != DC_F32) BAD("vocoder pipeline is fp32");
+    if (c->mel_dim < 4 || c->mel_dim % 4) BAD("mel_dim must be a multiple of 4");
+    if (c->n_up < 1 || c->n_up > DC_MAX_UP) BAD("n_up out of range");
+    int up = 1;
+    for (int q = 0; q < c->n_up; ++q) {
+      if (c->up_strides[q] < 1 || c->up_strides[q] > 16) BAD("stride out of range");
+      up *= c->up_strides[q];
+    }
+    if (up < 3) BAD("total upsampling must be >= 3");
+    for (int q = 0; q <= c->n_up; ++q)
+      if (c->up_channels[q] < 4 || c->up_channels[q] % 4) BAD("channels must be multiples of 4");
+    if (c->n_res < 0 || c->n_res > DC_MAX_RES) BAD("n_res out of range");
+    for (int r = 0; r < c->n_res; ++r)
+      if (c->res_dilations[r] < 1 || c->res_dilations[r] > 64) BAD("dilation out of range");
+    if (c->n_fft != 16 || c->hop != 4) BAD("only n_fft = 16, hop = 4 is built");
+    if ((long long)c->f_chunk * up > (1 << 20)) BAD("chunk too long");
+  } else {
+    BAD("unknown pipeline");
+  }
+#undef BAD
+  return true;
+}
+
+extern "C" size_t dc_weights_count(const dc_config* c) {
+  const char* why = "";
+  if (!config_ok(c, &why)) return 0;
+  size_t n = 0;
+  const size_t C = (size_t)c->hidden;
+  if (c->pipeline == DC_PIPE_CONV) {
+    n = (size_t)c->n_conv * (3 * C * C + C);
+  } else if (c->pipeline == DC_PIPE_FLOW) {
+    const size_t m = (size_t)c->mel_dim;
+    n = 2 * m * C + C + (size_t)c->n_conv * (3 * C * C + C + C * C) + (size_t)c->n_attn * (4 * C * C + 4 * C) + C * m + m;
+  } else {
+    n = 3 * (size_t)c->mel_dim * c->up_channels[0] + c->up_channels[0];
+    for (int q = 0; q < c->n_up; ++q) {
+      const size_t ci = c->up_channels[q], co = c->up_channels[q + 1];
+      n += 2 * (size_t)c->up_strides[q] * ci * co + co + (size_t)c->n_res * (3 * co * co + co);
+    }
+    n += 3 * (size_t)c->up_channels[c->n_up] * (c->n_fft + 2) + (c->n_fft + 2);
+  }
+  return n;
+}
+
+static void build_f32_layers(dc_model* m) {
+  const dc_config& c = m->cfg;
+  size_t off = 0;
+  auto add = [&](int kind, int ci, int co, int dil, int stride, int rate_in, int halo, int res, size_t wsz) {
+    F32Layer L{};
+    L.kind = kind; L.C_in = ci; L.C_out = co; L.dil = dil; L.stride = stride;
+    L.rate_in = rate_in; L.halo = halo; L.residual_silu = res; L.post_silu = 0;
+    L.w_off = off; off += wsz;
+    L.b_off = off; off += (size_t)co;
+    L.ring_cap = dc::pow2_ceil(c.f_chunk * rate_in + halo);
+    m->layers.push_back(L);
+  };
+  if (c.pipeline == DC_PIPE_CONV) {
+    const int C = c.hidden;
+    for (int l = 0; l < c.n_conv; ++l) add(0, C, C, c.dilations[l], 1, 1, 2 * c.dilations[l], 1, (size_t)3 * C * C);
+    m->in_dim = C;
+    m->out_per_frame = C;
+  } else {
+    int rate = 1;
+    add(0, c.mel_dim, c.up_channels[0], 1, 1, rate, 2, 0, (size_t)3 * c.mel_dim * c.up_channels[0]);
+    for (int q = 0; q < c.n_up; ++q) {
+      const int ci = c.up_channels[q], co = c.up_channels[q + 1], s = c.up_strides[q];
+      add(1, ci, co, 1, s, rate, 1, 0, (size_t)2 * s * ci * co);
+      rate *= s;
+      for (int r = 0; r < c.n_res; ++r)
+        add(0, co, co, c.res_dilations[r], 1, rate, 2 * c.res_dilations[r], 1, (size_t)3 * co * co);
+    }
+    m->layers.back().post_silu = 1;   // only the head reads it, and the head wants SiLU(a)
+    add(2, c.up_channels[c.n_up], c.n_fft + 2, 1, 1, rate, 2, 0, (size_t)3 * c.up_channels[c.n_up] * (c.n_fft + 2));
+    m->in_dim = c.mel_dim;
+    m->out_per_frame = rate * c.hop;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// lifetime
+// ---------------------------------------------------------------------------------------------
+
+extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config* cfg, dc_model** out) {
+  if (!out) return DC_ERR_ARG;
+  *out = nullptr;
+  const char* why = "";
+  if (!config_ok(cfg, &why)) {
+    dc::set_error("invalid configuration: %s", why);
+    return DC_ERR_CONFIG;
+  }
+  if (!w || n_floats != dc_weights_count(cfg)) {
+    dc::set_error("weight blob has %zu floats, configuration needs %zu", n_floats, dc_weights_count(cfg));
+    return DC_ERR_ARG;
+  }
+  int dev = 0;
+  DC_CUDA(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  DC_CUDA(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) {
+    dc::set_error("device %d is sm_%d%d; this library is built for sm_100a only", dev, prop.major, prop.minor);
+    return DC_ERR_CUDA;
+  }
+  dc_model* m = new (std::nothrow) dc_model();
+  if (!m) return DC_ERR_OOM;
+  m->cfg = *cfg;
+  m->device = dev;
+  for (auto& c : m->counters) c = 0;
+  dc_status st = DC_OK;
+  if (cfg->pipeline == DC_PIPE_FLOW) {
+    st = dc::flow_model_create(*cfg, w, &m->flow);
+    m->in_dim = 2 * cfg->mel_dim;
+    m->out_per_frame = cfg->mel_dim;
+  } else {
+    build_f32_layers(m);
+    cudaError_t e = cudaMalloc(&m->d_w, n_floats * sizeof(float));
+    if (e == cudaSuccess) e = cudaMemcpy(m->d_w, w, n_floats * sizeof(float), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = dc::prepare_f32_constants();
+    if (e != cudaSuccess) {
+      dc::set_error("weight upload failed: %s", cudaGetErrorString(e));
+      st = e == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;
+    }
+  }
+  if (st != DC_OK) {
+    if (m->d_w) cudaFree(m->d_w);
+    delete m;
+    return st;
+  }
+  *out = m;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_destroy(dc_model* m) {
+  if (!m) return DC_ERR_ARG;
+  if (m->open_streams.load() != 0) {
+    dc::set_error("dc_destroy: %d streams still open", m->open_streams.load());
+    return DC_ERR_STATE;
+  }
+  if (m->flow) dc::flow_model_destroy(m->flow);
+  if (m->d_w) cudaFree(m->d_w);
+  for (dc_stream* s : m->all_streams) delete s;
+  delete m;
+  return DC_OK;
+}
+
+static void free_stream_buffers(dc_stream* s) {
+  for (auto& b : s->f32_rings)
+    if (b.p) cudaFree(b.p);
+  s->f32_rings.clear();
+  if (s->tails) cudaFree(s->tails);
+  if (s->flow) dc::flow_state_close(s->flow);
+  if (s->stage_in) cudaFree(s->stage_in);
+  if (s->stage_out) cudaFree(s->stage_out);
+  s->tails = nullptr;
+  s->flow = nullptr;
+  s->stage_in = s->stage_out = nullptr;
+}
+
+extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
+  if (!m || !out) return DC_ERR_ARG;
+  *out = nullptr;
+  dc_stream* s = new (std::nothrow) dc_stream();
+  if (!s) return DC_ERR_OOM;
+  s->model = m;
+  cudaError_t e = cudaSuccess;
+  dc_status st = DC_OK;
+  if (m->flow) {
+    st = dc::flow_state_open(m->flow, &s->flow);
+  } else {
+    for (const F32Layer& L : m->layers) {
+      DevBuf b{nullptr, (size_t)L.ring_cap * L.C_in * sizeof(float)};
+      e = cudaMalloc(&b.p, b.bytes);
+      if (e != cudaSuccess) break;
+      s->f32_rings.push_back(b);
+      e = cudaMemset(b.p, 0, b.bytes);
+      if (e != cudaSuccess) break;
+    }
+    if (e == cudaSuccess && m->cfg.pipeline == DC_PIPE_VOCODER) {
+      e = cudaMalloc(&s->tails, 2 * 12 * sizeof(float));
+      if (e == cudaSuccess) e = cudaMemset(s->tails, 0, 2 * 12 * sizeof(float));
+    }
+  }
+  if (e == cudaSuccess && st == DC_OK) {
+    e = cudaMalloc(&s->stage_in, (size_t)m->cfg.f_chunk * m->in_dim * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(&s->stage_out, (size_t)m->cfg.f_chunk * m->out_per_frame * sizeof(float));
+  }
+  if (e != cudaSuccess) {
+    dc::set_error("stream allocation failed: %s", cudaGetErrorString(e));
+    st = e == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;
+  }
+  if (st != DC_OK) {
+    free_stream_buffers(s);
+    delete s;
+    return st;
+  }
+  {
+    std::lock_guard<std::mutex> lk(m->mu);
+    m->all_streams.push_back(s);
+  }
+  m->open_streams++;
+  m->counters[6]++;
+  *out = s;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_stream_reset(dc_stream* s, void* cuda_stream) {
+  if (!s || s->closed) return DC_ERR_STATE;
+  cudaStream_t cs = (cudaStream_t)cuda_stream;
+  if (s->flow) {
+    dc_status st = dc::flow_state_reset(s->model->flow, s->flow, cs);
+    if (st != DC_OK) return st;
+  } else {
+    for (auto& b : s->f32_rings) DC_CUDA(cudaMemsetAsync(b.p, 0, b.bytes, cs));
+    if (s->tails) DC_CUDA(cudaMemsetAsync(s->tails, 0, 2 * 12 * sizeof(float), cs));
+  }
+  s->frames_total = 0;
+  s->chunks = 0;
+  s->poisoned = false;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_stream_close(dc_stream* s) {
+  if (!s) return DC_ERR_ARG;
+  if (s->closed) return DC_ERR_STATE;
+  cudaDeviceSynchronize();
+  s->closed = true;
+  s->model->open_streams--;
+  s->model->counters[6]--;
+  free_stream_buffers(s);
+  return DC_OK;
+}
+
+extern "C" dc_status dc_stream_carry_info(const dc_stream* s, uint64_t* out, int max_entries, int* n_entries) {
+  if (!s || !out || !n_entries || max_entries < 0) return DC_ERR_ARG;
+  if (s->closed) return DC_ERR_STATE;
+  std::vector<DevBuf> bufs;
+  if (s->flow) {
+    bufs.resize(64);
+    int n = 0;
+    dc::flow_state_buffers(s->flow, bufs.data(), 64, &n);
+    bufs.resize(n);
+  } else {
+    bufs = s->f32_rings;
+    if (s->tails) bufs.push_back(DevBuf{s->tails, 2 * 12 * sizeof(float)});
+  }
+  *n_entries = (int)bufs.size();
+  for (int i = 0; i < (int)bufs.size() && i < max_entries; ++i) {
+    out[2 * i] = (uint64_t)(uintptr_t)bufs[i].p;
+    out[2 * i + 1] = (uint64_t)bufs[i].bytes;
+  }
+  return DC_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// the chunk step
+// ---------------------------------------------------------------------------------------------
+
+static dc_status decode_f32(dc_stream* s, const float* feats, int T, float* out, cudaStream_t cs, int* launches) {
+  dc_model* m = s->model;
+  const int nL = (int)m->layers.size();
+  for (int l = 0; l < nL; ++l) {
+    const F32Layer& L = m->layers[l];
+    const long long pos = s->frames_total * L.rate_in;
+    const int Tin = T * L.rate_in;
+    float* ring = (float*)s->f32_rings[l].p;
+    if (L.kind == 2) {
+      dc::HeadIstftF32 h{};
+      h.in_ring = ring; h.in_mask = L.ring_cap - 1; h.pos = pos; h.T = Tin; h.C = L.C_in;
+      h.W = m->d_w + L.w_off; h.bias = m->d_w + L.b_off; h.clamp = m->cfg.logmag_clamp;
+      h.tail_in = s->tails + 12 * (s->chunks & 1);
+      h.tail_out = s->tails + 12 * ((s->chunks + 1) & 1);
+      h.pcm = out;
+      dc::launch_head_istft_f32(h, cs);
+    } else {
+      dc::TapConvF32 p{};
+      p.in_ring = ring; p.in_mask = L.ring_cap - 1; p.pos_in = pos; p.T_in = Tin; p.C_in = L.C_in;
+      if (l == 0) { p.in_direct = feats; p.save_ring = ring; p.save_rows = L.halo; }
+      if (L.kind == 0) {
+        p.n_taps = 3; p.shift[0] = 2 * L.dil; p.shift[1] = L.dil; p.shift[2] = 0; p.n_phase = 1;
+        p.w_tap_stride = (long long)L.C_in * L.C_out; p.w_phase_stride = 0;
+      } else {
+        p.n_taps = 2; p.shift[0] = 0; p.shift[1] = 1; p.shift[2] = 0; p.n_phase = L.stride;
+        p.w_tap_stride = (long long)L.stride * L.C_in * L.C_out; p.w_phase_stride = (long long)L.C_in * L.C_out;
+      }
+      p.W = m->d_w + L.w_off; p.bias = m->d_w + L.b_off; p.C_out = L.C_out;
+      p.residual_silu = L.residual_silu; p.post_silu = L.post_silu;
+      if (l + 1 < nL) {
+        p.out_ring = (float*)s->f32_rings[l + 1].p; p.out_mask = m->layers[l + 1].ring_cap - 1;
+      } else {
+        p.out_direct = out; p.pos_out = pos * p.n_phase;
+      }
+      dc::launch_tapconv_f32(p, cs);
+    }
+    ++*launches;
+  }
+  DC_CUDA(cudaGetLastError());
+  return DC_OK;
+}
+
+static dc_status admit(dc_stream* s, const float* feats, int T, float* out) {
+  if (!s) return DC_ERR_ARG;
+  if (s->closed || s->poisoned) return DC_ERR_STATE;
+  if (!feats || !out) {
+    s->model->counters[3]++;
+    return DC_ERR_ARG;
+  }
+  if (T < 1 || T > s->model->cfg.f_chunk) {
+    s->model->counters[2]++;
+    dc::set_error("n_frames = %d violates 1 <= n_frames <= f_chunk = %d", T, s->model->cfg.f_chunk);
+    return DC_ERR_FRAMES;
+  }
+  return DC_OK;
+}
+
+extern "C" dc_status dc_decode_chunk(dc_stream* s, const float* feats, int T, float* out, int* n_out, void* cuda_stream) {
+  dc_status st = admit(s, feats, T, out);
+  if (st != DC_OK) return st;
+  dc_model* m = s->model;
+  cudaStream_t cs = (cudaStream_t)cuda_stream;
+  int launches = 0;
+  if (m->flow) {
+    st = dc::flow_decode(m->flow, 1, &s->flow, &feats, &T, &out, cs, &launches);
+  } else {
+    st = decode_f32(s, feats, T, out, cs, &launches);
+  }
+  m->counters[5] += (uint64_t)launches;
+  if (st != DC_OK) {
+    s->poisoned = true;
+    return st;
+  }
+  s->frames_total += T;
+  s->chunks += 1;
+  m->counters[0] += 1;
+  m->counters[1] += (uint64_t)T;
+  if (n_out) *n_out = T * m->out_per_frame;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* streams, const float* const* feats,
+                                     const int* n_frames, float* const* out, void* cuda_stream) {
+  if (!m || !streams || !feats || !n_frames || !out) return DC_ERR_ARG;
+  if (!m->flow) {
+    dc::set_error("dc_decode_batch serves the flow pipeline only");
+    return DC_ERR_CONFIG;
+  }
+  if (n < 1 || n > m->cfg.max_batch) {
+    m->counters[3]++;
+    dc::set_error("batch of %d streams, max_batch = %d", n, m->cfg.max_batch);
+    return DC_ERR_ARG;
+  }
+  std::vector<dc::FlowState*> states((size_t)n);
+  for (int i = 0; i < n; ++i) {
+    dc_status st = admit(streams[i], feats[i], n_frames[i], out[i]);
+    if (st != DC_OK) return st;
+    if (streams[i]->model != m) {
+      m->counters[3]++;
+      return DC_ERR_STATE;
+    }
+    for (int j = 0; j < i; ++j)
+      if (streams[j] == streams[i]) {
+        m->counters[3]++;
+        dc::set_error("stream %d appears twice in the batch", i);
+        return DC_ERR_ARG;
+      }
+    states[(size_t)i] = streams[i]->flow;
+  }
+  int launches = 0;
+  dc_status st = dc::flow_decode(m->flow, n, states.data(), feats, n_frames, out, (cudaStream_t)cuda_stream, &launches);
+  m->counters[5] += (uint64_t)launches;
+  if (st != DC_OK) {
+    for (int i = 0; i < n; ++i) streams[i]->poisoned = true;
+    return st;
+  }
+  for (int i = 0; i < n; ++i) {
+    streams[i]->frames_total += n_frames[i];
+    streams[i]->chunks += 1;
+    m->counters[1] += (uint64_t)n_frames[i];
+  }
+  m->counters[0] += (uint64_t)n;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_decode_chunk_host(dc_stream* s, const float* feats_host, int T, float* out_host, int* n_out,
+                                          void* cuda_stream) {
+  dc_status st = admit(s, feats_host, T, out_host);
+  if (st != DC_OK) return st;
+  dc_model* m = s->model;
+  cudaStream_t cs = (cudaStream_t)cuda_stream;
+  DC_CUDA(cudaMemcpyAsync(s->stage_in, feats_host, (size_t)T * m->in_dim * sizeof(float), cudaMemcpyHostToDevice, cs));
+  int n = 0;
+  st = dc_decode_chunk(s, s->stage_in, T, s->stage_out, &n, cuda_stream);
+  if (st != DC_OK) return st;
+  DC_CUDA(cudaMemcpyAsync(out_host, s->stage_out, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, cs));
+  DC_CUDA(cudaStreamSynchronize(cs));
+  if (n_out) *n_out = n;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_get_counters(const dc_model* m, uint64_t counters[8]) {
+  if (!m || !counters) return DC_ERR_ARG;
+  for (int i = 0; i < 8; ++i) counters[i] = m->counters[i].load();
+  return DC_OK;
+}
+
+extern "C" const char* dc_status_str(dc_status s) {
+  switch (s) {
+    case DC_OK: return "DC_OK";
+    case DC_ERR_ARG: return "DC_ERR_ARG";
+    case DC_ERR_CONFIG: return "DC_ERR_CONFIG";
+    case DC_ERR_FRAMES: return "DC_ERR_FRAMES";
+    case DC_ERR_OOM: return "DC_ERR_OOM";
+    case DC_ERR_CUDA: return "DC_ERR_CUDA";
+    case DC_ERR_TIMEOUT: return "DC_ERR_TIMEOUT";
+    case DC_ERR_STATE: return "DC_ERR_STATE";
+  }
+  return "DC_ERR_UNKNOWN";
+}
+
+extern "C" const char* dc_last_error(void) { return dc::g_last_error.c_str(); }

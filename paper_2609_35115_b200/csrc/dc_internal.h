@@ -1,0 +1,91 @@
+// Internal declarations shared by the translation units of libdc (not installed).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "dc.h"
+
+namespace dc {
+
+// ---------------------------------------------------------------------------------------------
+// fp32 tap convolution over ring buffers (conv pipeline and vocoder tail)
+// ---------------------------------------------------------------------------------------------
+// A layer reads frames by logical index t (frames since stream start at that layer's rate).
+// Frame t lives in row (t & mask) of a power-of-two ring; frames t >= pos_in may instead come
+// from a plain [T_in][C_in] array (`in_direct`, the caller's chunk).  Rings start zeroed, so
+// t < 0 reads the causal zero padding.  Nothing is ever concatenated or moved: the left context
+// of the next chunk is simply the rows already in the ring.
+struct TapConvF32 {
+  const float* in_ring;
+  int          in_mask;
+  const float* in_direct;     // may be null
+  long long    pos_in;        // logical index of the first new input frame
+  int          T_in;          // new input frames in this call
+  int          C_in;
+  int          n_taps;        // 3 (conv) or 2 (transposed conv phases)
+  int          shift[3];      // tap j reads frame t - shift[j]
+  int          n_phase;       // output frame index = n_phase * t + phase
+  const float* W;             // weights of (phase p, tap j) at W + p*w_phase_stride + j*w_tap_stride, [C_in][C_out]
+  long long    w_tap_stride;
+  long long    w_phase_stride;
+  const float* bias;          // [C_out]
+  int          C_out;
+  int          residual_silu; // out = in[t] + SiLU(acc + bias)   (needs C_in == C_out, n_phase == 1)
+  int          post_silu;     // out = SiLU(out)
+  float*       out_ring;      // row (t_out & out_mask)
+  int          out_mask;
+  float*       out_direct;    // or plain [T_out][C_out] rows (t_out - pos_out)
+  long long    pos_out;
+  float*       save_ring;     // if set: copy the last save_rows rows of in_direct into the input ring
+  int          save_rows;
+};
+
+void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st);
+
+// Head conv (k = 3, input already SiLU-activated) + magnitude/phase -> inverse real DFT (n_fft = 16)
+// -> synthesis window -> overlap-add (hop 4) with the 12-sample tail carried across chunks.
+struct HeadIstftF32 {
+  const float* in_ring;       // [cap][C]
+  int          in_mask;
+  long long    pos;           // logical index of the first new frame
+  int          T;             // new frames (>= 3)
+  int          C;
+  const float* W;             // [3][C][18]
+  const float* bias;          // [18]
+  float        clamp;         // upper clamp of the log-magnitude
+  const float* tail_in;       // [12] unnormalised partial sums of samples hop*pos .. +11
+  float*       tail_out;      // [12] the same for the next chunk (a different buffer)
+  float*       pcm;           // [4*T]
+};
+
+void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st);
+
+// Uploads the constant tables of the head kernel (DFT twiddles, periodic Hann window) to the
+// current device.  Synchronous; called from dc_create, never from a decode call.
+cudaError_t prepare_f32_constants();
+
+// ---------------------------------------------------------------------------------------------
+// bf16 flow decoder (dc_flow.cu)
+// ---------------------------------------------------------------------------------------------
+struct DevBuf {
+  void*  p;
+  size_t bytes;
+};
+
+struct FlowModel;    // packed bf16 weights, tensor maps, timestep-bias table, scratch for max_batch streams
+struct FlowState;    // carries of one stream
+
+void set_error(const char* fmt, ...);
+
+dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** out);
+void      flow_model_destroy(FlowModel* m);
+dc_status flow_state_open(FlowModel* m, FlowState** out);
+void      flow_state_buffers(const FlowState* s, DevBuf* out, int max_entries, int* n);
+dc_status flow_state_reset(FlowModel* m, FlowState* s, cudaStream_t st);
+void      flow_state_close(FlowState* s);
+// One chunk for each of n streams.  Returns the number of kernel launches through *launches.
+dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats_dev,
+                      const int* n_frames, float* const* out_dev, cudaStream_t st, int* launches);
+
+}  // namespace dc

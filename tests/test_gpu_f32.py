@@ -1,0 +1,165 @@
+"""GPU parity of the fp32 pipelines (tiny causal conv stream, vocoder tail) against the oracle,
+through the C ABI.  Tolerance: max |err| / RMS(ref) <= 1e-4."""
+import hashlib
+
+import numpy as np
+import pytest
+import torch
+
+import dc_workloads as wl
+from oracle import dc_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+
+
+@pytest.fixture(scope="module")
+def dc():
+    import paper_2609_35115_b200 as dc
+    dc.load_library()
+    return dc
+
+
+def _util():
+    from tests import gpu_util
+    return gpu_util
+
+
+def test_cfg1_streamed_matches_offline_oracle(dc):
+    gu = _util()
+    w = wl.make_workload(wl.CONFIGS["cfg1"])
+    s = w.streams[0]
+    ref = orc.run_offline(w.cfg, w.weights, s.feats, s.boundaries)
+    m = dc.Model(w.cfg, w.weights)
+    got = gu.run_gpu_stream(m, s.feats, s.boundaries)
+    assert got.shape == ref.shape
+    assert gu.rel_err(got, ref) <= TOL_F32
+    # ragged partition incl. chunks shorter than the conv left context
+    ragged = [0, 1, 2, 5, 21, 22, 38, 39, 55, 71, 87, 103, 119, 128]
+    got2 = gu.run_gpu_stream(m, s.feats, ragged)
+    assert gu.rel_err(got2, ref) <= TOL_F32
+    # bitwise reproducible run to run
+    got3 = gu.run_gpu_stream(m, s.feats, s.boundaries)
+    assert hashlib.sha256(got.tobytes()).hexdigest() == hashlib.sha256(got3.tobytes()).hexdigest()
+    m.destroy()
+
+
+def test_conv_stack_nonzero_bias_large_dilation(dc):
+    gu = _util()
+    cfg = wl.CONFIGS["cfg1"].replace(name="conv_b", hidden=72, dilations=(1, 3, 9), f_chunk=40, n_chunks=6,
+                                     seed=21, bias_std=0.3)
+    bnd = [0, 40, 41, 60, 100, 117, 157]
+    w = wl.make_workload(cfg, boundaries=[bnd])
+    s = w.streams[0]
+    ref = orc.run_offline(cfg, w.weights, s.feats, bnd)
+    m = dc.Model(cfg, w.weights)
+    assert gu.rel_err(gu.run_gpu_stream(m, s.feats, bnd), ref) <= TOL_F32
+    m.destroy()
+
+
+def test_tiny_vocoder_ragged_chunks(dc):
+    gu = _util()
+    cfg = wl.tiny_vocoder()
+    bnd = [0, 1, 2, 7, 8, 13, 18, 20]
+    w = wl.make_workload(cfg, boundaries=[bnd])
+    s = w.streams[0]
+    ref = orc.vocoder_offline(cfg, w.weights, s.feats)
+    m = dc.Model(cfg, w.weights)
+    got = gu.run_gpu_stream(m, s.feats, bnd)
+    assert got.shape == ref.shape
+    assert gu.rel_err(got, ref) <= TOL_F32
+    m.destroy()
+
+
+def test_cfg4_vocoder_tail_full(dc):
+    gu = _util()
+    cfg = wl.CONFIGS["cfg4"]
+    w = wl.make_workload(cfg)
+    s = w.streams[0]
+    ref = orc.run_stream(cfg, w.weights, s.feats, s.boundaries)
+    m = dc.Model(cfg, w.weights)
+    got = gu.run_gpu_stream(m, s.feats, s.boundaries)
+    assert got.shape == (cfg.n_chunks * 24000,)
+    assert gu.rel_err(got, ref) <= TOL_F32
+    # per chunk, too
+    for c in (0, 1, 57, 199):
+        assert gu.rel_err(got[c * 24000:(c + 1) * 24000], ref[c * 24000:(c + 1) * 24000]) <= TOL_F32
+    got2 = gu.run_gpu_stream(m, s.feats, s.boundaries)
+    assert np.array_equal(got, got2)
+    m.destroy()
+
+
+def test_vocoder_reset_and_pointer_constancy(dc):
+    gu = _util()
+    cfg = wl.tiny_vocoder()
+    w = wl.make_workload(cfg)
+    s = w.streams[0]
+    m = dc.Model(cfg, w.weights)
+    st = m.open_stream()
+    before = st.carry_info()
+    a = gu.run_gpu_stream(m, s.feats, s.boundaries, stream=st)
+    assert st.carry_info() == before           # carries never move while the stream lives
+    st.reset()
+    assert st.carry_info() == before           # ... nor at a turn boundary
+    b = gu.run_gpu_stream(m, s.feats, s.boundaries, stream=st)
+    assert np.array_equal(a, b)                # reset writes the base state in place
+    st.close()
+    m.destroy()
+
+
+def test_admission_and_error_paths(dc):
+    cfg = wl.CONFIGS["cfg1"]
+    w = wl.make_workload(cfg)
+    m = dc.Model(cfg, w.weights)
+    st = m.open_stream()
+    x = torch.zeros(17, 64, device="cuda")
+    y = torch.zeros(17, 64, device="cuda")
+    good = torch.from_numpy(w.streams[0].feats[:16]).cuda()
+    ref1 = st.decode_chunk(good).clone()
+    # admission predicate: 1 <= n_frames <= f_chunk; a refused call must not touch the stream
+    assert st.decode_raw(x.data_ptr(), 17, y.data_ptr()) == 3
+    assert st.decode_raw(x.data_ptr(), 0, y.data_ptr()) == 3
+    assert st.decode_raw(0, 4, y.data_ptr()) == 1
+    assert st.decode_raw(x.data_ptr(), 4, 0) == 1
+    nxt = torch.from_numpy(w.streams[0].feats[16:32]).cuda()
+    got2 = st.decode_chunk(nxt).clone()
+    ref = orc.run_offline(cfg, w.weights, w.streams[0].feats[:32], [0, 32])
+    torch.cuda.synchronize()
+    from tests import gpu_util as gu
+    assert gu.rel_err(torch.cat([ref1, got2]).cpu().numpy(), ref) <= TOL_F32
+    c = m.counters()
+    assert c[0] == 2 and c[1] == 32 and c[2] == 2 and c[3] == 2 and c[5] == 4
+    # a model with open streams cannot be destroyed; a closed stream refuses work
+    with pytest.raises(dc.DCError):
+        m.destroy()
+    h = st.handle
+    st.close()
+    st.handle = h
+    assert st.decode_raw(x.data_ptr(), 4, y.data_ptr()) == 7
+    st.handle = None
+    # bad configuration / blob size fail closed
+    with pytest.raises(dc.DCError):
+        dc.Model(cfg, w.weights[:-1])
+    with pytest.raises(dc.DCError):
+        dc.Model(cfg.replace(hidden=63), w.weights)
+    m.destroy()
+
+
+def test_host_buffer_entry_point(dc):
+    gu = _util()
+    cfg = wl.CONFIGS["cfg1"]
+    w = wl.make_workload(cfg)
+    s = w.streams[0]
+    m = dc.Model(cfg, w.weights)
+    st = m.open_stream()
+    fin = torch.from_numpy(s.feats).pin_memory()
+    fout = torch.empty(s.feats.shape[0], 64).pin_memory()
+    for c in range(len(s.boundaries) - 1):
+        lo, hi = s.boundaries[c], s.boundaries[c + 1]
+        n = st.decode_chunk_host(fin[lo:hi], fout[lo:hi])
+        assert n == (hi - lo) * 64
+    ref = orc.run_offline(cfg, w.weights, s.feats, s.boundaries)
+    assert gu.rel_err(fout.numpy(), ref) <= TOL_F32
+    st.close()
+    m.destroy()
