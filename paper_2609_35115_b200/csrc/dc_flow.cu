@@ -1,11 +1,976 @@
-// placeholder until the bf16 flow decoder lands
+// bf16 flow decoder: host engine + kernels.
+//
+// Data layout.  Up to max_batch streams are served by one pass.  Every activation matrix is a
+// bf16 row-major [GUARD + 64*slots][C] array: stream slot i owns the 64-row block starting at
+// row GUARD + 64 i, whose rows 0..7 hold the conv left context (the last 8 block-input frames of
+// the previous chunk, copied in from the stream's carry by the producing epilogue) and rows
+// 8..8+T-1 the T <= 56 frames of the chunk.  A tap of a dilated conv is then a plain row shift
+// of the whole matrix, so the k = 3 conv is three accumulating UMMA passes whose A tiles are TMA
+// boxes at row offsets -2d, -d, 0.  One CTA computes a 128 x BN output tile (two slots).
+//
+// GEMM kernel: warp 0 = TMA producer, warp 1 = UMMA issuer (accumulator in tensor memory),
+// warps 2..5 = epilogue (one TMEM lane = one output row per thread).  The epilogues fuse bias,
+// timestep bias, SiLU, residual, the carry update of the next conv block, the in-place append of
+// K/V rows to the stream's ring, and the Euler update.
+#include <cuda.h>
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
 #include "dc_internal.h"
+#include "dc_ptx.cuh"
+
 namespace dc {
-dc_status flow_model_create(const dc_config&, const float*, FlowModel**) { set_error("flow decoder not built"); return DC_ERR_CONFIG; }
-void flow_model_destroy(FlowModel*) {}
-dc_status flow_state_open(FlowModel*, FlowState**) { return DC_ERR_CONFIG; }
-void flow_state_buffers(const FlowState*, DevBuf*, int, int* n) { *n = 0; }
-dc_status flow_state_reset(FlowModel*, FlowState*, cudaStream_t) { return DC_ERR_CONFIG; }
-void flow_state_close(FlowState*) {}
-dc_status flow_decode(FlowModel*, int, FlowState* const*, const float* const*, const int*, float* const*, cudaStream_t, int*) { return DC_ERR_CONFIG; }
+
+namespace {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int GUARD = 8;        // zero rows in front of every activation matrix (tap shifts never go negative)
+constexpr int SLOT_ROWS = 64;   // rows per stream slot: 8 left-context rows + up to 56 chunk rows
+constexpr int HALO = 8;         // carried frames per (step, conv block); dilation <= 4 reads at most 8 back
+constexpr int TILE_M = 128;
+constexpr int KBLK = 64;        // bf16 elements per 128-byte swizzled smem row
+constexpr int STAGES = 4;
+constexpr int A_BYTES = TILE_M * 128;
+constexpr int MAX_BN = 128;
+constexpr int GEMM_THREADS = 192;
+constexpr int MAX_SLOTS_PER_SET = 64;
+
+enum GemmMode { MODE_INPROJ = 0, MODE_CONV = 1, MODE_QKV = 2, MODE_OPROJ = 3, MODE_OUT = 4 };
+
+struct SlotInfo {
+  int          T;         // frames presented by this stream in this call
+  int          kv_head;   // ring row that receives the chunk's first K/V row
+  int          kv_len;    // carried K/V rows attended (<= kv_cap), before this chunk
+  int          pad;
+  const float* feats;     // [T][2 mel]
+  float*       out;       // [T][mel]
+  bf16*        halo;      // stream carry: [n_steps][n_conv][8][C]
+  bf16*        kv;        // stream carry: [n_steps][n_attn][2][Rk][C]
+};
+
+struct SlotSet {
+  int      first, count;
+  SlotInfo s[MAX_SLOTS_PER_SET];
+};
+
+struct GemmParams {
+  int          mode;
+  int          BN;              // output columns per CTA (multiple of 16, <= 128)
+  int          n_slots;
+  int          n_kblocks;       // total 64-wide reduction blocks (= taps * kb_per_tap)
+  int          kb_per_tap;
+  int          shift[3];        // row shift of tap j
+  const float* bias;            // [N]
+  const float* tau;             // [N] or null
+  const bf16*  resid;           // residual source matrix (same row layout) or null
+  bf16*        out;             // output activation matrix or null
+  int          ld;              // row stride (elements) of resid / out / q
+  const SlotInfo* slots;
+  long long    halo_off;        // element offset of the next conv's carry inside SlotInfo::halo, or -1
+  bf16*        q_out;           // MODE_QKV
+  long long    kv_off;          // element offset of this (step, layer)'s K ring inside SlotInfo::kv
+  int          Rk;              // ring rows
+  int          C;
+  float*       xstate;          // MODE_OUT: fp32 Euler state [rows][mel]
+  bf16*        ain;             // MODE_OUT: next step's input-projection operand [GUARD+rows][ld_ain]
+  int          ld_ain;
+  float        inv_n;
+  int          last_step;
+  int          mel;
+  int*         err;
+};
+
+__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
+
+__device__ __forceinline__ void load16_bf16(const bf16* p, float* v) {
+  const uint4 a = *reinterpret_cast<const uint4*>(p);
+  const uint4 b = *reinterpret_cast<const uint4*>(p + 8);
+  const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
 }
+__device__ __forceinline__ void pack16_bf16(const float* v, uint4& a, uint4& b) {
+  uint32_t w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    w[i] = *reinterpret_cast<const uint32_t*>(&h);
+  }
+  a = make_uint4(w[0], w[1], w[2], w[3]);
+  b = make_uint4(w[4], w[5], w[6], w[7]);
+}
+__device__ __forceinline__ void store16(bf16* p, const uint4& a, const uint4& b) {
+  *reinterpret_cast<uint4*>(p) = a;
+  *reinterpret_cast<uint4*>(p + 8) = b;
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + STAGES * A_BYTES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(sB + STAGES * MAX_BN * 128);
+  uint64_t* empty = full + STAGES;
+  uint64_t* accum = empty + STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+  int* s_fail = reinterpret_cast<int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * TILE_M, n0 = blockIdx.y * p.BN;
+  const uint32_t b_bytes = (uint32_t)p.BN * 128u;
+  const uint32_t tmem_cols = p.BN <= 32 ? 32u : (p.BN <= 64 ? 64u : 128u);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) {
+      ptx::mbar_init(&full[i], 1);
+      ptx::mbar_init(&empty[i], 1);
+    }
+    ptx::mbar_init(accum, 1);
+    *s_fail = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) ptx::tmem_alloc(tmem_slot, tmem_cols);
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      ptx::prefetch_tmap(&tmA);
+      ptx::prefetch_tmap(&tmB);
+      for (int kb = 0; kb < p.n_kblocks; ++kb) {
+        const int st = kb % STAGES;
+        if (kb >= STAGES && !ptx::mbar_wait(&empty[st], ((kb / STAGES) - 1) & 1)) {
+          atomicExch(p.err, 1);
+          *s_fail = 1;
+          break;
+        }
+        const int tap = kb / p.kb_per_tap;
+        const int cb = kb - tap * p.kb_per_tap;
+        ptx::mbar_expect_tx(&full[st], (uint32_t)A_BYTES + b_bytes);
+        ptx::tma_load_2d(sA + st * A_BYTES, &tmA, cb * KBLK, GUARD + m0 - p.shift[tap], &full[st]);
+        ptx::tma_load_2d(sB + st * MAX_BN * 128, &tmB, kb * KBLK, n0, &full[st]);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.BN, 0, 0);
+      bool ok = true;
+      for (int kb = 0; kb < p.n_kblocks && ok; ++kb) {
+        const int st = kb % STAGES;
+        if (!ptx::mbar_wait(&full[st], (kb / STAGES) & 1)) {
+          atomicExch(p.err, 2);
+          *s_fail = 1;
+          ok = false;
+          break;
+        }
+        ptx::tc_fence_after();
+        const uint32_t a0 = ptx::smem_u32(sA + st * A_BYTES), b0 = ptx::smem_u32(sB + st * MAX_BN * 128);
+#pragma unroll
+        for (int k = 0; k < KBLK / 16; ++k)
+          ptx::umma_bf16(tmem_base, ptx::umma_desc_sw128(a0 + k * 32), ptx::umma_desc_sw128(b0 + k * 32), idesc,
+                         (kb | k) != 0);
+        ptx::umma_commit(&empty[st]);
+      }
+      ptx::umma_commit(accum);   // arrives when every UMMA above has finished (also on the failure path)
+    }
+  } else {
+    // ---------------- epilogue: 4 warps, thread <-> output row ----------------
+    const bool got = ptx::mbar_wait(accum, 0);
+    ptx::tc_fence_after();
+    if (!got) atomicExch(p.err, 3);
+    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    const int r = m0 + q * 32 + lane;             // row in slot layout (without GUARD)
+    const int slot = r / SLOT_ROWS, rho = r % SLOT_ROWS;
+    const bool slot_ok = slot < p.n_slots && got && *s_fail == 0;
+    const SlotInfo si = slot_ok ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr};
+    const int f = rho - HALO;
+    const bool is_halo = slot_ok && rho < HALO;
+    const bool is_chunk = slot_ok && f >= 0 && f < si.T;
+    const long long grow = (long long)(GUARD + r);
+    const bool do_halo = p.halo_off >= 0;
+    bf16* carry = do_halo && slot_ok ? si.halo + p.halo_off : nullptr;
+    const int new_row = rho - si.T;               // carry row this thread's value moves to
+    const bool carry_wr = do_halo && (is_halo || is_chunk) && new_row >= 0 && new_row < HALO;
+
+    for (int c0 = 0; c0 < p.BN; c0 += 16) {
+      float acc[16];
+      ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
+      const int n = n0 + c0;
+      float y[16];
+      if (p.mode == MODE_OUT) {
+        if (is_chunk) {
+          float* xs = p.xstate + (long long)r * p.mel + n;
+          float xv[16];
+#pragma unroll
+          for (int i = 0; i < 16; i += 4) {
+            const float4 t = *reinterpret_cast<const float4*>(xs + i);
+            xv[i] = t.x; xv[i + 1] = t.y; xv[i + 2] = t.z; xv[i + 3] = t.w;
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) xv[i] = xv[i] + (acc[i] + p.bias[n + i]) * p.inv_n;
+#pragma unroll
+          for (int i = 0; i < 16; i += 4)
+            *reinterpret_cast<float4*>(xs + i) = make_float4(xv[i], xv[i + 1], xv[i + 2], xv[i + 3]);
+          uint4 a, b;
+          pack16_bf16(xv, a, b);
+          store16(p.ain + grow * p.ld_ain + n, a, b);
+          if (p.last_step) {
+            float* o = si.out + (long long)f * p.mel + n;
+#pragma unroll
+            for (int i = 0; i < 16; i += 4)
+              *reinterpret_cast<float4*>(o + i) = make_float4(xv[i], xv[i + 1], xv[i + 2], xv[i + 3]);
+          }
+        }
+        continue;
+      }
+#pragma unroll
+      for (int i = 0; i < 16; ++i) y[i] = acc[i] + p.bias[n + i];
+      if (p.mode == MODE_QKV) {
+        if (is_chunk) {
+          uint4 a, b;
+          pack16_bf16(y, a, b);
+          const int which = n / p.C, col = n - which * p.C;
+          if (which == 0) {
+            store16(p.q_out + grow * p.ld + col, a, b);
+          } else {
+            int row = si.kv_head + f;
+            if (row >= p.Rk) row -= p.Rk;
+            store16(si.kv + p.kv_off + (long long)(which - 1) * p.Rk * p.C + (long long)row * p.C + col, a, b);
+          }
+        }
+        continue;
+      }
+      if (p.mode == MODE_CONV || p.mode == MODE_OPROJ) {
+        float x[16];
+        if (is_chunk) {
+          load16_bf16(p.resid + grow * p.ld + n, x);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) x[i] = 0.f;
+        }
+        if (p.mode == MODE_CONV) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) y[i] = x[i] + silu_f(y[i] + p.tau[n + i]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) y[i] = x[i] + y[i];
+        }
+      }
+      uint4 va, vb;
+      pack16_bf16(y, va, vb);
+      if (is_chunk) store16(p.out + grow * p.ld + n, va, vb);
+      if (do_halo) {
+        // left context of the next conv block: hand the carried rows to the consumer, then shift
+        // the carry by T frames ([old carry | chunk] -> last 8 rows), all inside this CTA
+        if (is_halo) {
+          va = *reinterpret_cast<const uint4*>(carry + rho * p.C + n);
+          vb = *reinterpret_cast<const uint4*>(carry + rho * p.C + n + 8);
+          store16(p.out + grow * p.ld + n, va, vb);
+        }
+        ptx::named_bar_sync(1, 128);
+        if (carry_wr) store16(carry + new_row * p.C + n, va, vb);
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) ptx::tmem_dealloc(tmem_base, tmem_cols);
+}
+
+// ---- small kernels ---------------------------------------------------------------------------
+
+__global__ void set_slots_kernel(const SlotSet set, SlotInfo* dst) {
+  const int i = threadIdx.x;
+  if (i < set.count) dst[set.first + i] = set.s[i];
+}
+
+// feats [T][2 mel] -> Euler state x_0 (fp32) and the bf16 input-projection operand [x_0 | mu].
+__global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, bf16* ain, int ld_ain) {
+  const SlotInfo si = slots[blockIdx.x];
+  for (int i = threadIdx.x; i < si.T * mel; i += blockDim.x) {
+    const int f = i / mel, c = i - f * mel;
+    const long long r = (long long)blockIdx.x * SLOT_ROWS + HALO + f;
+    const float mu = si.feats[(long long)f * 2 * mel + c];
+    const float x0 = si.feats[(long long)f * 2 * mel + mel + c];
+    xstate[r * mel + c] = x0;
+    ain[(GUARD + r) * ld_ain + c] = __float2bfloat16_rn(x0);
+    ain[(GUARD + r) * ld_ain + mel + c] = __float2bfloat16_rn(mu);
+  }
+}
+
+// u = bf16(x * rsqrt(mean(x^2) + eps)), one warp per chunk row.
+__global__ void flow_rmsnorm_kernel(const SlotInfo* slots, int n_slots, const bf16* x, bf16* u, int C, float eps) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  const int slot = warp / SLOT_ROWS, rho = warp % SLOT_ROWS;
+  if (slot >= n_slots) return;
+  const int f = rho - HALO;
+  if (f < 0 || f >= slots[slot].T) return;
+  const long long off = (long long)(GUARD + warp) * C;
+  float ss = 0.f;
+  for (int c = lane * 8; c < C; c += 256) {
+    const uint4 v = *reinterpret_cast<const uint4*>(x + off + c);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
+      ss = fmaf(a, a, ss);
+      ss = fmaf(b, b, ss);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float rs = rsqrtf(ss / (float)C + eps);
+  for (int c = lane * 8; c < C; c += 256) {
+    const uint4 v = *reinterpret_cast<const uint4*>(x + off + c);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(w[i] << 16) * rs, __uint_as_float(w[i] & 0xFFFF0000u) * rs);
+      o[i] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(u + off + c) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+
+// ---- chunk-causal attention with the K/V carry ---------------------------------------------------
+// One CTA per (stream slot, head).  Queries: the T chunk frames (padded to the 128 UMMA rows).
+// Keys/values: the kv_len carried frames followed by the chunk's own T frames, read in place
+// from the stream's ring with 128-bit loads (the ring may wrap; nothing is compacted or copied
+// in global memory).  Two passes over the keys in blocks of 128, both on tcgen05:
+//   pass 1: S = Q K^T per block -> row maximum;
+//   pass 2: S again, e = exp(scale (S - max)), row sum from the unrounded e, P = bf16(e) written to
+//           shared memory as the A operand of O += P V (V is the MN-major B operand).
+// One thread owns one query row (= one TMEM lane), so the softmax needs no cross-thread traffic.
+constexpr int ATT_THREADS = 128;
+constexpr int ATT_KB = 128;     // keys per block
+constexpr int ATT_TMEM_COLS = 512;  // S double buffer (2 x 128) + O (64)
+
+struct AttnParams {
+  const SlotInfo* slots;
+  const bf16*     q;          // [GUARD + rows][ld]
+  bf16*           o;          // [GUARD + rows][ld]
+  int             ld;
+  int             dh;         // 32 or 64 (smem rows are padded to 64 columns)
+  long long       kv_off;     // element offset of this (step, layer)'s K ring inside SlotInfo::kv
+  int             Rk, C;
+  int             kv_rows_max;  // smem rows reserved for K and for V (multiple of 128)
+  float           scale_log2e;  // log2(e) / sqrt(dh)
+  int*            err;
+};
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(dst)), "l"(src) : "memory");
+}
+
+__global__ void __launch_bounds__(ATT_THREADS, 1) flow_attn_kernel(const AttnParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;                       // [128][128 B]
+  uint8_t* sP = sQ + 128 * 128;             // 2 tiles of [128][128 B]
+  uint8_t* sK = sP + 2 * 128 * 128;         // [kv_rows_max][128 B]
+  uint8_t* sV = sK + (size_t)p.kv_rows_max * 128;
+  uint64_t* bar_s = reinterpret_cast<uint64_t*>(sV + (size_t)p.kv_rows_max * 128);   // [2]
+  uint64_t* bar_pv = bar_s + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_pv + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int slot = blockIdx.x, head = blockIdx.y;
+  const SlotInfo si = p.slots[slot];
+  const int T = si.T, L = si.kv_len + T;
+  const int nkb = (L + ATT_KB - 1) / ATT_KB;
+  const int chunks = p.dh >> 3;             // 16-byte chunks per head row
+
+  if (tid == 0) {
+    ptx::mbar_init(&bar_s[0], 1);
+    ptx::mbar_init(&bar_s[1], 1);
+    ptx::mbar_init(bar_pv, 1);
+    ptx::fence_barrier_init();
+  }
+  __syncwarp();
+  if (warp == 0) ptx::tmem_alloc(tmem_slot, ATT_TMEM_COLS);
+
+  // ---- stage Q, K, V into 128-byte-swizzled shared memory ----
+  {
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    const bf16* qbase = p.q + (long long)(GUARD + slot * SLOT_ROWS + HALO) * p.ld + head * p.dh;
+    for (int i = tid; i < 128 * 8; i += ATT_THREADS) {
+      const int row = i >> 3, j = i & 7;
+      uint8_t* dst = sQ + row * 128 + ((j ^ (row & 7)) << 4);
+      if (row < T && j < chunks) cp_async16(dst, qbase + (long long)row * p.ld + j * 8);
+      else *reinterpret_cast<uint4*>(dst) = zero;
+    }
+    const bf16* kbase = si.kv + p.kv_off + head * p.dh;
+    const bf16* vbase = kbase + (long long)p.Rk * p.C;
+    int start = si.kv_head - si.kv_len;
+    if (start < 0) start += p.Rk;
+    for (int i = tid; i < nkb * ATT_KB * 8; i += ATT_THREADS) {
+      const int row = i >> 3, j = i & 7;
+      const int off = row * 128 + ((j ^ (row & 7)) << 4);
+      if (row < L && j < chunks) {
+        int rr = start + row;
+        if (rr >= p.Rk) rr -= p.Rk;
+        cp_async16(sK + off, kbase + (long long)rr * p.C + j * 8);
+        cp_async16(sV + off, vbase + (long long)rr * p.C + j * 8);
+      } else {
+        *reinterpret_cast<uint4*>(sK + off) = zero;
+        *reinterpret_cast<uint4*>(sV + off) = zero;
+      }
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    ptx::fence_proxy_async_smem();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+  const uint32_t idesc_s = ptx::umma_idesc_bf16(128, ATT_KB, 0, 0);
+  const uint32_t idesc_pv = ptx::umma_idesc_bf16(128, 64, 0, 1);   // B = V, MN-major
+  const uint32_t q_addr = ptx::smem_u32(sQ), k_addr = ptx::smem_u32(sK), v_addr = ptx::smem_u32(sV), p_addr = ptx::smem_u32(sP);
+
+  auto issue_s = [&](int kb) {   // S[kb & 1] = Q K_kb^T
+    const uint32_t d = tmem_base + (uint32_t)((kb & 1) * ATT_KB);
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      ptx::umma_bf16(d, ptx::umma_desc_sw128(q_addr + k * 32), ptx::umma_desc_sw128(k_addr + kb * ATT_KB * 128 + k * 32),
+                     idesc_s, k != 0);
+    ptx::umma_commit(&bar_s[kb & 1]);
+  };
+
+  bool ok = true;
+  uint32_t n_s[2] = {0u, 0u};    // completed waits per S buffer (phase parity)
+  float mrow = -INFINITY;
+  // ---- pass 1: row maximum ----
+  if (tid == 0) issue_s(0);
+  for (int kb = 0; kb < nkb; ++kb) {
+    if (tid == 0 && kb + 1 < nkb) issue_s(kb + 1);
+    const int b = kb & 1;
+    if (ok && !ptx::mbar_wait(&bar_s[b], n_s[b] & 1)) { ok = false; atomicExch(p.err, 4); }
+    ++n_s[b];
+    ptx::tc_fence_after();
+    const int valid = L - kb * ATT_KB;
+    for (int c0 = 0; c0 < ATT_KB; c0 += 16) {
+      float v[16];
+      ptx::tmem_ld16(lane_addr + (uint32_t)(b * ATT_KB + c0), v);
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        if (c0 + i < valid) mrow = fmaxf(mrow, v[i]);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+  }
+  // ---- pass 2: numerators, row sum, O += P V ----
+  float lsum = 0.f;
+  uint32_t n_pv = 0;
+  const float mscaled = mrow * p.scale_log2e;
+  if (tid == 0) issue_s(0);
+  for (int kb = 0; kb < nkb; ++kb) {
+    if (tid == 0 && kb + 1 < nkb) issue_s(kb + 1);
+    const int b = kb & 1;
+    if (ok && !ptx::mbar_wait(&bar_s[b], n_s[b] & 1)) { ok = false; atomicExch(p.err, 5); }
+    ++n_s[b];
+    if (kb > 0) {   // the previous P V must have consumed the P tile before it is overwritten
+      if (ok && !ptx::mbar_wait(bar_pv, n_pv & 1)) { ok = false; atomicExch(p.err, 6); }
+      ++n_pv;
+    }
+    ptx::tc_fence_after();
+    const int valid = L - kb * ATT_KB;
+    for (int c0 = 0; c0 < ATT_KB; c0 += 16) {
+      float v[16];
+      ptx::tmem_ld16(lane_addr + (uint32_t)(b * ATT_KB + c0), v);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const float e = (c0 + i < valid) ? exp2f(fmaf(v[i], p.scale_log2e, -mscaled)) : 0.f;
+        lsum += e;
+        v[i] = e;
+      }
+      uint4 a, bq;
+      pack16_bf16(v, a, bq);
+      // key columns c0..c0+15 -> tile c0/64, 16-byte chunks (c0 % 64)/8 and +1 of row `tid`
+      uint8_t* prow = sP + (c0 >> 6) * (128 * 128) + tid * 128;
+      const int j0 = (c0 & 63) >> 3;
+      *reinterpret_cast<uint4*>(prow + (((j0) ^ (tid & 7)) << 4)) = a;
+      *reinterpret_cast<uint4*>(prow + (((j0 + 1) ^ (tid & 7)) << 4)) = bq;
+    }
+    ptx::fence_proxy_async_smem();
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      ptx::tc_fence_after();
+      const int ksteps = valid >= ATT_KB ? ATT_KB / 16 : (valid + 15) / 16;
+      const uint32_t d = tmem_base + 2 * ATT_KB;
+      for (int k = 0; k < ksteps; ++k)
+        ptx::umma_bf16(d, ptx::umma_desc_sw128(p_addr + (k >> 2) * (128 * 128) + (k & 3) * 32),
+                       ptx::umma_desc_sw128(v_addr + (kb * ATT_KB + k * 16) * 128), idesc_pv, (kb | k) != 0);
+      ptx::umma_commit(bar_pv);
+    }
+  }
+  if (ok && !ptx::mbar_wait(bar_pv, n_pv & 1)) { ok = false; atomicExch(p.err, 7); }
+  ptx::tc_fence_after();
+  {
+    const float inv = 1.0f / lsum;
+    bf16* orow = p.o + (long long)(GUARD + slot * SLOT_ROWS + HALO + tid) * p.ld + head * p.dh;
+    for (int c0 = 0; c0 < p.dh; c0 += 16) {
+      float v[16];
+      ptx::tmem_ld16(lane_addr + (uint32_t)(2 * ATT_KB + c0), v);
+      if (tid < T && ok) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] *= inv;
+        uint4 a, bq;
+        pack16_bf16(v, a, bq);
+        store16(orow + c0, a, bq);
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 0) ptx::tmem_dealloc(tmem_base, ATT_TMEM_COLS);
+}
+
+// ---- host helpers ----------------------------------------------------------------------------
+
+uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+float bf16_to_f32(uint16_t h) {
+  uint32_t u = (uint32_t)h << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return f;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+// bf16 row-major [rows][cols] matrix, tiles of box_rows x 64 columns, 128-byte swizzle.
+bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstr[1] = {cols * sizeof(bf16)};
+  cuuint32_t box[2] = {(cuuint32_t)KBLK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr size_t GEMM_SMEM = 1024 + STAGES * A_BYTES + STAGES * MAX_BN * 128 + 256;
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// engine
+// ---------------------------------------------------------------------------------------------
+
+struct FlowModel {
+  dc_config cfg;
+  int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0, kv_rows_max = 0;
+  size_t attn_smem = 0;
+  bf16 *Xa = nullptr, *Xb = nullptr, *U = nullptr, *Q = nullptr, *O = nullptr, *Ain = nullptr;
+  float* xstate = nullptr;
+  bf16*  wts = nullptr;
+  float* fconst = nullptr;   // biases and the timestep-bias table
+  SlotInfo* d_slots = nullptr;
+  int*   d_err = nullptr;
+  CUtensorMap tmAin, tmXa, tmXb, tmU, tmO, tmWin, tmWout;
+  std::vector<CUtensorMap> tmWconv, tmWqkv, tmWo;
+  // float offsets into fconst
+  size_t o_bin = 0, o_bout = 0, o_tau = 0;
+  std::vector<size_t> o_bconv, o_bqkv, o_bo;
+  std::vector<void*> allocs;
+};
+
+struct FlowState {
+  FlowModel* m = nullptr;
+  bf16* halo = nullptr;
+  bf16* kv = nullptr;
+  size_t halo_bytes = 0, kv_bytes = 0;
+  long long frames = 0;     // frames appended so far (drives ring head and carried length)
+};
+
+namespace {
+
+template <typename T>
+cudaError_t dalloc(FlowModel* m, T** p, size_t n, bool zero = true) {
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T));
+  if (e != cudaSuccess) return e;
+  m->allocs.push_back(*p);
+  return zero ? cudaMemset(*p, 0, n * sizeof(T)) : cudaSuccess;
+}
+
+// transposes a [K][N] fp32 matrix into bf16 [N][ldk] (K-major rows), zero padded
+void pack_wt(std::vector<uint16_t>& dst, size_t off, const float* W, int K, int N, int ldk) {
+  for (int n = 0; n < N; ++n)
+    for (int k = 0; k < K; ++k) dst[off + (size_t)n * ldk + k] = f32_to_bf16_rne(W[(size_t)k * N + n]);
+}
+
+}  // namespace
+
+void flow_model_destroy(FlowModel* m) {
+  if (!m) return;
+  for (void* p : m->allocs) cudaFree(p);
+  delete m;
+}
+
+dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** out) {
+  FlowModel* m = new (std::nothrow) FlowModel();
+  if (!m) return DC_ERR_OOM;
+  m->cfg = cfg;
+  const int C = m->C = cfg.hidden, mel = m->mel = cfg.mel_dim;
+  m->Kin = ((2 * mel + KBLK - 1) / KBLK) * KBLK;
+  m->S = cfg.max_batch;
+  m->rows = ((m->S * SLOT_ROWS + TILE_M - 1) / TILE_M) * TILE_M;
+  m->Rk = cfg.kv_cap + cfg.f_chunk;
+  m->cpa = cfg.n_attn > 0 ? cfg.n_conv / cfg.n_attn : cfg.n_conv;
+  m->kv_rows_max = ((m->Rk + ATT_KB - 1) / ATT_KB) * ATT_KB;
+  m->attn_smem = 1024 + 3 * 128 * 128 + 2 * (size_t)m->kv_rows_max * 128 + 64;
+  if (cfg.n_attn > 0 && m->attn_smem > 227 * 1024) {
+    set_error("kv_cap + f_chunk = %d key rows do not fit the attention kernel's shared memory", m->Rk);
+    delete m;
+    return DC_ERR_CONFIG;
+  }
+  const int nL = cfg.n_conv, nA = cfg.n_attn, nS = cfg.n_steps;
+  const size_t R = (size_t)GUARD + m->rows;
+
+  // ---- pack weights: every matrix transposed to [N][K] so that both UMMA operands are K-major
+  size_t wn = (size_t)C * m->Kin + (size_t)nL * C * 3 * C + (size_t)nA * (3 * (size_t)C * C + (size_t)C * C) + (size_t)mel * C;
+  std::vector<uint16_t> hw(wn, 0);
+  size_t fn = (size_t)C + (size_t)nL * C + (size_t)nA * 4 * C + mel + (size_t)nS * nL * C;
+  std::vector<float> hf(fn, 0.f);
+  std::vector<size_t> w_conv(nL), w_qkv(nA), w_o(nA);
+  size_t wo = 0, fo = 0, src = 0;
+  const size_t w_in = wo;
+  pack_wt(hw, wo, w + src, 2 * mel, C, m->Kin);
+  wo += (size_t)C * m->Kin;
+  src += (size_t)2 * mel * C;
+  m->o_bin = fo;
+  memcpy(&hf[fo], w + src, C * sizeof(float));
+  fo += C;
+  src += C;
+  std::vector<const float*> Pmat(nL);
+  m->o_bconv.resize(nL);
+  m->o_bqkv.resize(nA);
+  m->o_bo.resize(nA);
+  int l = 0;
+  const int n_groups = nA > 0 ? nA : 1;
+  for (int g = 0; g < n_groups; ++g) {
+    for (int j = 0; j < m->cpa; ++j, ++l) {
+      w_conv[l] = wo;
+      // blob W[tap][c_in][c_out] is one [3C][C] matrix with k = tap*C + c_in
+      pack_wt(hw, wo, w + src, 3 * C, C, 3 * C);
+      wo += (size_t)C * 3 * C;
+      src += (size_t)3 * C * C;
+      m->o_bconv[l] = fo;
+      memcpy(&hf[fo], w + src, C * sizeof(float));
+      fo += C;
+      src += C;
+      Pmat[l] = w + src;
+      src += (size_t)C * C;
+    }
+    if (nA > 0) {
+      w_qkv[g] = wo;
+      for (int t = 0; t < 3; ++t) {
+        pack_wt(hw, wo, w + src, C, C, C);
+        wo += (size_t)C * C;
+        src += (size_t)C * C;
+      }
+      w_o[g] = wo;
+      pack_wt(hw, wo, w + src, C, C, C);
+      wo += (size_t)C * C;
+      src += (size_t)C * C;
+      m->o_bqkv[g] = fo;
+      memcpy(&hf[fo], w + src, 3 * (size_t)C * sizeof(float));
+      fo += 3 * (size_t)C;
+      src += 3 * (size_t)C;
+      m->o_bo[g] = fo;
+      memcpy(&hf[fo], w + src, C * sizeof(float));
+      fo += C;
+      src += C;
+    }
+  }
+  const size_t w_out = wo;
+  pack_wt(hw, wo, w + src, C, mel, C);
+  wo += (size_t)mel * C;
+  src += (size_t)C * mel;
+  m->o_bout = fo;
+  memcpy(&hf[fo], w + src, mel * sizeof(float));
+  fo += mel;
+  src += mel;
+  // timestep-bias table tau[s][l][:] = emb(s / n) @ bf16(P_l), evaluated once in double
+  m->o_tau = fo;
+  {
+    const int half = C / 2;
+    std::vector<double> emb(C);
+    for (int s = 0; s < nS; ++s) {
+      const double t = (double)s / nS;
+      for (int i = 0; i < half; ++i) {
+        const double om = pow(10000.0, -(double)i / half);
+        emb[i] = sin(1000.0 * t * om);
+        emb[half + i] = cos(1000.0 * t * om);
+      }
+      for (int ll = 0; ll < nL; ++ll) {
+        std::vector<double> acc(C, 0.0);
+        for (int k = 0; k < C; ++k) {
+          const double e = emb[k];
+          const float* prow = Pmat[ll] + (size_t)k * C;
+          for (int n = 0; n < C; ++n) acc[n] += e * (double)bf16_to_f32(f32_to_bf16_rne(prow[n]));
+        }
+        for (int n = 0; n < C; ++n) hf[fo + ((size_t)s * nL + ll) * C + n] = (float)acc[n];
+      }
+    }
+    fo += (size_t)nS * nL * C;
+  }
+
+  cudaError_t e = cudaSuccess;
+  auto chk = [&](cudaError_t x) { if (e == cudaSuccess) e = x; };
+  chk(dalloc(m, &m->wts, wn, false));
+  chk(dalloc(m, &m->fconst, fn, false));
+  chk(dalloc(m, &m->Xa, R * C));
+  chk(dalloc(m, &m->Xb, R * C));
+  chk(dalloc(m, &m->U, R * C));
+  chk(dalloc(m, &m->Q, R * C));
+  chk(dalloc(m, &m->O, R * C));
+  chk(dalloc(m, &m->Ain, R * m->Kin));
+  chk(dalloc(m, &m->xstate, (size_t)m->rows * mel));
+  chk(dalloc(m, &m->d_slots, (size_t)m->S));
+  chk(dalloc(m, &m->d_err, 1));
+  if (e == cudaSuccess) chk(cudaMemcpy(m->wts, hw.data(), wn * sizeof(uint16_t), cudaMemcpyHostToDevice));
+  if (e == cudaSuccess) chk(cudaMemcpy(m->fconst, hf.data(), fn * sizeof(float), cudaMemcpyHostToDevice));
+  if (e == cudaSuccess)
+    chk(cudaFuncSetAttribute(flow_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
+  if (e == cudaSuccess && cfg.n_attn > 0)
+    chk(cudaFuncSetAttribute(flow_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m->attn_smem));
+  if (e != cudaSuccess) {
+    set_error("flow model allocation failed: %s", cudaGetErrorString(e));
+    flow_model_destroy(m);
+    return e == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;
+  }
+
+  bool ok = true;
+  ok &= make_tmap(&m->tmAin, m->Ain, R, m->Kin, TILE_M);
+  ok &= make_tmap(&m->tmXa, m->Xa, R, C, TILE_M);
+  ok &= make_tmap(&m->tmXb, m->Xb, R, C, TILE_M);
+  ok &= make_tmap(&m->tmU, m->U, R, C, TILE_M);
+  ok &= make_tmap(&m->tmO, m->O, R, C, TILE_M);
+  ok &= make_tmap(&m->tmWin, m->wts + w_in, C, m->Kin, 64);
+  ok &= make_tmap(&m->tmWout, m->wts + w_out, mel, C, mel);
+  m->tmWconv.resize(nL);
+  m->tmWqkv.resize(nA);
+  m->tmWo.resize(nA);
+  for (int i = 0; i < nL; ++i) ok &= make_tmap(&m->tmWconv[i], m->wts + w_conv[i], C, 3 * C, 64);
+  for (int i = 0; i < nA; ++i) {
+    ok &= make_tmap(&m->tmWqkv[i], m->wts + w_qkv[i], 3 * C, C, 64);
+    ok &= make_tmap(&m->tmWo[i], m->wts + w_o[i], C, C, 64);
+  }
+  if (!ok) {
+    set_error("cuTensorMapEncodeTiled failed or is unavailable");
+    flow_model_destroy(m);
+    return DC_ERR_CUDA;
+  }
+  *out = m;
+  return DC_OK;
+}
+
+dc_status flow_state_open(FlowModel* m, FlowState** out) {
+  FlowState* s = new (std::nothrow) FlowState();
+  if (!s) return DC_ERR_OOM;
+  s->m = m;
+  const dc_config& c = m->cfg;
+  s->halo_bytes = (size_t)c.n_steps * c.n_conv * HALO * m->C * sizeof(bf16);
+  s->kv_bytes = (size_t)c.n_steps * c.n_attn * 2 * m->Rk * m->C * sizeof(bf16);
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s->halo), s->halo_bytes);
+  if (e == cudaSuccess) e = cudaMemset(s->halo, 0, s->halo_bytes);
+  if (e == cudaSuccess && s->kv_bytes) {
+    e = cudaMalloc(reinterpret_cast<void**>(&s->kv), s->kv_bytes);
+    if (e == cudaSuccess) e = cudaMemset(s->kv, 0, s->kv_bytes);
+  }
+  if (e != cudaSuccess) {
+    set_error("flow stream allocation failed: %s", cudaGetErrorString(e));
+    flow_state_close(s);
+    return e == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;
+  }
+  *out = s;
+  return DC_OK;
+}
+
+void flow_state_buffers(const FlowState* s, DevBuf* out, int max_entries, int* n) {
+  int k = 0;
+  if (k < max_entries) out[k++] = DevBuf{s->halo, s->halo_bytes};
+  if (s->kv && k < max_entries) out[k++] = DevBuf{s->kv, s->kv_bytes};
+  *n = k;
+}
+
+dc_status flow_state_reset(FlowModel*, FlowState* s, cudaStream_t st) {
+  // base state: zero left context, empty K/V carry (stale ring rows are never attended)
+  if (cudaMemsetAsync(s->halo, 0, s->halo_bytes, st) != cudaSuccess) return DC_ERR_CUDA;
+  s->frames = 0;
+  return DC_OK;
+}
+
+void flow_state_close(FlowState* s) {
+  if (!s) return;
+  if (s->halo) cudaFree(s->halo);
+  if (s->kv) cudaFree(s->kv);
+  delete s;
+}
+
+void launch_flow_attention(FlowModel* m, int n, int step, int layer, cudaStream_t st);
+
+dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats, const int* T,
+                      float* const* outp, cudaStream_t st, int* launches) {
+  const dc_config& c = m->cfg;
+  const int C = m->C, mel = m->mel;
+  // ---- per-call slot table (passed by value through a kernel, so nothing is staged or allocated)
+  for (int first = 0; first < n; first += MAX_SLOTS_PER_SET) {
+    SlotSet set;
+    set.first = first;
+    set.count = n - first < MAX_SLOTS_PER_SET ? n - first : MAX_SLOTS_PER_SET;
+    for (int i = 0; i < set.count; ++i) {
+      FlowState* s = states[first + i];
+      SlotInfo& si = set.s[i];
+      si.T = T[first + i];
+      si.kv_head = (int)(s->frames % m->Rk);
+      si.kv_len = (int)(s->frames < c.kv_cap ? s->frames : c.kv_cap);
+      si.pad = 0;
+      si.feats = feats[first + i];
+      si.out = outp[first + i];
+      si.halo = s->halo;
+      si.kv = s->kv;
+    }
+    set_slots_kernel<<<1, MAX_SLOTS_PER_SET, 0, st>>>(set, m->d_slots);
+    ++*launches;
+  }
+  flow_prep_kernel<<<n, 128, 0, st>>>(m->d_slots, mel, m->xstate, m->Ain, m->Kin);
+  ++*launches;
+
+  const int m_tiles = (n * SLOT_ROWS + TILE_M - 1) / TILE_M;
+  auto gemm = [&](const CUtensorMap& tA, const CUtensorMap& tB, GemmParams& p, int N) {
+    p.n_slots = n;
+    p.slots = m->d_slots;
+    p.ld = C;
+    p.C = C;
+    p.Rk = m->Rk;
+    p.err = m->d_err;
+    dim3 grid(m_tiles, N / p.BN);
+    flow_gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(tA, tB, p);
+    ++*launches;
+  };
+  auto rmsnorm = [&](const bf16* x) {
+    const int warps = n * SLOT_ROWS;
+    flow_rmsnorm_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(m->d_slots, n, x, m->U, C, c.rms_eps);
+    ++*launches;
+  };
+  const float* fc = m->fconst;
+  const long long halo_stride = (long long)HALO * C;
+
+  for (int s = 0; s < c.n_steps; ++s) {
+    bf16* X = m->Xa;                 // current residual stream
+    bf16* Y = m->Xb;
+    const CUtensorMap* tX = &m->tmXa;
+    const CUtensorMap* tY = &m->tmXb;
+    auto swap = [&]() { std::swap(X, Y); std::swap(tX, tY); };
+    {
+      GemmParams p{};
+      p.mode = MODE_INPROJ; p.BN = 64; p.n_kblocks = m->Kin / KBLK; p.kb_per_tap = p.n_kblocks;
+      p.bias = fc + m->o_bin; p.out = X;
+      p.halo_off = ((long long)s * c.n_conv + 0) * halo_stride;
+      gemm(m->tmAin, m->tmWin, p, C);
+    }
+    int l = 0;
+    const int n_groups = c.n_attn > 0 ? c.n_attn : 1;
+    for (int g = 0; g < n_groups; ++g) {
+      for (int j = 0; j < m->cpa; ++j, ++l) {
+        const int d = c.dilations[l];
+        GemmParams p{};
+        p.mode = MODE_CONV; p.BN = 64; p.kb_per_tap = C / KBLK; p.n_kblocks = 3 * p.kb_per_tap;
+        p.shift[0] = 2 * d; p.shift[1] = d; p.shift[2] = 0;
+        p.bias = fc + m->o_bconv[l]; p.tau = fc + m->o_tau + ((size_t)s * c.n_conv + l) * C;
+        p.resid = X; p.out = Y;
+        const bool next_is_conv = (j + 1 < m->cpa);
+        p.halo_off = next_is_conv ? ((long long)s * c.n_conv + l + 1) * halo_stride : -1;
+        gemm(*tX, m->tmWconv[l], p, C);
+        swap();
+      }
+      if (c.n_attn > 0) {
+        rmsnorm(X);
+        {
+          GemmParams p{};
+          p.mode = MODE_QKV; p.BN = 64; p.n_kblocks = C / KBLK; p.kb_per_tap = p.n_kblocks;
+          p.bias = fc + m->o_bqkv[g]; p.q_out = m->Q; p.halo_off = -1;
+          p.kv_off = ((long long)s * c.n_attn + g) * 2 * m->Rk * C;
+          gemm(m->tmU, m->tmWqkv[g], p, 3 * C);
+        }
+        launch_flow_attention(m, n, s, g, st);
+        ++*launches;
+        {
+          GemmParams p{};
+          p.mode = MODE_OPROJ; p.BN = 64; p.n_kblocks = C / KBLK; p.kb_per_tap = p.n_kblocks;
+          p.bias = fc + m->o_bo[g]; p.resid = X; p.out = Y;
+          p.halo_off = (l < c.n_conv) ? ((long long)s * c.n_conv + l) * halo_stride : -1;
+          gemm(m->tmO, m->tmWo[g], p, C);
+          swap();
+        }
+      }
+    }
+    rmsnorm(X);
+    {
+      GemmParams p{};
+      p.mode = MODE_OUT; p.BN = mel; p.n_kblocks = C / KBLK; p.kb_per_tap = p.n_kblocks;
+      p.bias = fc + m->o_bout; p.halo_off = -1;
+      p.xstate = m->xstate; p.ain = m->Ain; p.ld_ain = m->Kin; p.inv_n = 1.0f / c.n_steps;
+      p.last_step = (s == c.n_steps - 1); p.mel = mel;
+      gemm(m->tmU, m->tmWout, p, mel);
+    }
+  }
+  if (cudaGetLastError() != cudaSuccess) {
+    set_error("flow decode launch failed");
+    return DC_ERR_CUDA;
+  }
+  for (int i = 0; i < n; ++i) states[i]->frames += T[i];
+  return DC_OK;
+}
+
+void launch_flow_attention(FlowModel* m, int n, int step, int layer, cudaStream_t st) {
+  const dc_config& c = m->cfg;
+  AttnParams p{};
+  p.slots = m->d_slots; p.q = m->Q; p.o = m->O; p.ld = m->C; p.dh = c.head_dim;
+  p.kv_off = ((long long)step * c.n_attn + layer) * 2 * m->Rk * m->C;
+  p.Rk = m->Rk; p.C = m->C; p.kv_rows_max = m->kv_rows_max;
+  p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
+  p.err = m->d_err;
+  flow_attn_kernel<<<dim3(n, c.n_heads), ATT_THREADS, m->attn_smem, st>>>(p);
+}
+
+}  // namespace dc

@@ -1,0 +1,112 @@
+"""GPU parity of the bf16 flow decoder (conv blocks + chunk-causal attention + Euler steps)
+against the bf16-mirrored oracle, through the C ABI.  Tolerance: max |err| / RMS(ref) <= 2e-2."""
+import numpy as np
+import pytest
+import torch
+
+import dc_workloads as wl
+from oracle import dc_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+RAGGED = [0, 3, 13, 14, 24, 31, 41, 51, 52, 62, 72, 80]      # T in {1,3,7,8,10}; wraps the K/V ring
+
+
+@pytest.fixture(scope="module")
+def dc():
+    import paper_2609_35115_b200 as dc
+    dc.load_library()
+    return dc
+
+
+def _gu():
+    from tests import gpu_util
+    return gpu_util
+
+
+def _parity(dc, cfg, boundaries=None, tol=TOL_BF16):
+    gu = _gu()
+    w = wl.make_workload(cfg, boundaries=[boundaries] if boundaries else None)
+    s = w.streams[0]
+    ref = orc.run_stream(cfg, w.weights, s.feats, s.boundaries)
+    m = dc.Model(cfg, w.weights)
+    got = gu.run_gpu_stream(m, s.feats, s.boundaries)
+    err = gu.rel_err(got, ref)
+    got2 = gu.run_gpu_stream(m, s.feats, s.boundaries)
+    m.destroy()
+    assert got.shape == ref.shape
+    assert np.isfinite(got).all()
+    assert err <= tol, f"{cfg.name}: max|err|/rms = {err}"
+    assert np.array_equal(got, got2), "not bitwise reproducible run to run"
+    return err
+
+
+def test_flow_conv_only_gemm_path(dc):
+    # no attention: input projection, conv blocks with carried left context, Euler epilogue
+    _parity(dc, wl.tiny_flow(name="tiny_conv_only", n_attn_layers=0, n_heads=0, head_dim=0, kv_cap=0,
+                             dilations=(1, 2, 4)), RAGGED)
+
+
+def test_flow_tiny_with_attention_ragged(dc):
+    _parity(dc, wl.tiny_flow(), RAGGED)
+
+
+def test_flow_tiny_head_dim_64_full_chunks(dc):
+    _parity(dc, wl.tiny_flow(name="tiny_h64", hidden=128, n_heads=2, head_dim=64, kv_cap=150, f_chunk=50,
+                             n_chunks=6, dilations=(1, 2, 4, 1), n_steps=2))
+
+
+def test_cfg2_small_flow_decoder(dc):
+    _parity(dc, wl.CONFIGS["cfg2"])
+
+
+def test_cfg3_token2wav_sized_flow_decoder(dc):
+    # 30 chunks: passes the K/V cap (512 frames after 11 chunks) and wraps the 562-row ring
+    _parity(dc, wl.CONFIGS["cfg3"].replace(n_chunks=30))
+
+
+def test_batched_streams_match_oracle_and_single_stream_bytes(dc):
+    gu = _gu()
+    cfg = wl.tiny_flow(name="tiny_batch", n_streams=5, n_chunks=5)
+    w = wl.make_workload(cfg)
+    m = dc.Model(cfg, w.weights, max_batch=5)
+    single = [gu.run_gpu_stream(m, s.feats, s.boundaries) for s in w.streams]
+    streams = [m.open_stream() for _ in w.streams]
+    feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+    outs = [torch.empty(s.feats.shape[0], cfg.mel_dim, device="cuda") for s in w.streams]
+    for r in range(cfg.n_chunks):
+        fs, os_, ss = [], [], []
+        for i, s in enumerate(w.streams):
+            lo, hi = s.boundaries[r], s.boundaries[r + 1]
+            fs.append(feats[i][lo:hi])
+            os_.append(outs[i][lo:hi])
+            ss.append(streams[i])
+        dc.decode_batch(m, ss, fs, os_)
+    torch.cuda.synchronize()
+    for i, s in enumerate(w.streams):
+        got = outs[i].cpu().numpy()
+        ref = orc.run_stream(cfg, w.weights, s.feats, s.boundaries)
+        assert gu.rel_err(got, ref) <= TOL_BF16
+        assert np.array_equal(got, single[i]), "batched result differs from the single-stream bytes"
+    for st in streams:
+        st.close()
+    m.destroy()
+
+
+def test_flow_reset_and_pointer_constancy(dc):
+    gu = _gu()
+    cfg = wl.tiny_flow()
+    w = wl.make_workload(cfg)
+    s = w.streams[0]
+    m = dc.Model(cfg, w.weights)
+    st = m.open_stream()
+    before = st.carry_info()
+    assert len(before) == 2
+    a = gu.run_gpu_stream(m, s.feats, s.boundaries, stream=st)
+    assert st.carry_info() == before
+    st.reset()
+    b = gu.run_gpu_stream(m, s.feats, s.boundaries, stream=st)
+    assert st.carry_info() == before and np.array_equal(a, b)
+    st.close()
+    m.destroy()
