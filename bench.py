@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the streaming decoder step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg3|cfg2|cfg4|cfg1]
+    python bench.py --impl reference ...        # the CPU oracle, timed on the host cores
+
+A step is one pass of the whole per-chunk hot path over one batch of synthetic input: for the
+multi-stream workload (default, cfg5) one dc_decode_batch call that advances each of the 32
+streams by one 50-frame chunk (= 1 s of audio per stream); for the single-stream workloads one
+dc_decode_chunk call.  Prints ONE JSON line on rank 0.
+
+Multi-GPU: the path does not shard (a stream is strictly sequential), so --gpus N runs N
+independent replicas, one process per GPU, each with its own streams ("replicas only"); the only
+cross-rank traffic is the barrier and the max-over-ranks of the timing.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import dc_workloads as wl  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# FP32 FFMA peak of the part: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (no measured figure exists)
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+HISTORY_CHUNKS = 12      # untimed stream history so that the K/V carry sits at its cap (steady state)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists for that workload)
+NCU_TRAFFIC_BYTES = {"cfg5": None, "cfg3": None, "cfg2": None, "cfg4": None, "cfg1": None}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+def describe(cfg) -> str:
+    if cfg.pipeline == "flow":
+        return (f"{cfg.name}: {cfg.n_streams} stream(s) x flow decoder C={cfg.hidden}, {len(cfg.dilations)} conv blocks, "
+                f"{cfg.n_attn_layers} attention layers ({cfg.n_heads}x{cfg.head_dim}, KV cap {cfg.kv_cap}), "
+                f"{cfg.n_steps} Euler steps, {cfg.f_chunk}-frame chunks, bf16 / fp32 accumulate")
+    if cfg.pipeline == "vocoder":
+        return (f"{cfg.name}: vocoder tail mel {cfg.mel_dim} -> strides {cfg.up_strides} channels {cfg.up_channels} "
+                f"-> head -> iSTFT n_fft {cfg.n_fft} hop {cfg.hop}, {cfg.f_chunk}-frame chunks, fp32")
+    return f"{cfg.name}: causal conv stream C={cfg.hidden} dilations {cfg.dilations}, {cfg.f_chunk}-frame chunks, fp32"
+
+
+def units_per_chunk(cfg):
+    """(metric, unit, units one chunk of one stream is worth)."""
+    if cfg.pipeline == "conv":
+        return "streamed_frames_per_second", "frames/s", float(cfg.f_chunk)
+    return "streamed_audio_seconds_per_second", "audio-s/s", cfg.f_chunk / 50.0   # 50 frames = 1 s of 24 kHz audio
+
+
+def flops_per_launch(cfg, cls: str, n_streams: int) -> float:
+    """Algorithmic FLOPs of one launch of a kernel class (valid rows only)."""
+    rows = n_streams * cfg.f_chunk
+    C = cfg.hidden
+    if cls == "gemm_conv":
+        return 2.0 * rows * C * 3 * C
+    if cls == "attention":
+        L = cfg.kv_cap + cfg.f_chunk
+        return 2.0 * 2.0 * rows * L * C
+    return 0.0
+
+
+def attention_bytes_per_launch(cfg, n_streams: int) -> float:
+    """K and V rows of the attended window (bf16) + Q read + O write."""
+    L = cfg.kv_cap + cfg.f_chunk
+    return n_streams * (2.0 * L * cfg.hidden * 2 + 2.0 * cfg.f_chunk * cfg.hidden * 2)
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(cfg, weights, feats, n_chunks: int):
+    """Times the oracle as it stands on n_chunks chunks of one stream; returns seconds."""
+    from oracle import dc_oracle as orc
+    st = orc.make_stream(cfg, weights)
+    t0 = time.perf_counter()
+    for c in range(n_chunks):
+        st.decode_chunk(feats[c * cfg.f_chunk:(c + 1) * cfg.f_chunk])
+    return time.perf_counter() - t0
+
+
+def run_reference(args, cfg):
+    """--impl reference: the CPU oracle, one chunk of one stream per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import dc_oracle as orc
+    metric, unit, per_chunk = units_per_chunk(cfg)
+    rng = np.random.default_rng(cfg.seed)
+    weights = wl.make_weights(cfg, rng)
+    total = args.warmup + args.steps
+    feats = rng.standard_normal((total * cfg.f_chunk, cfg.in_dim), dtype=np.float32)
+    st = orc.make_stream(cfg, weights)
+    for c in range(args.warmup):
+        st.decode_chunk(feats[c * cfg.f_chunk:(c + 1) * cfg.f_chunk])
+    t0 = time.perf_counter()
+    for c in range(args.warmup, total):
+        st.decode_chunk(feats[c * cfg.f_chunk:(c + 1) * cfg.f_chunk])
+    dt = time.perf_counter() - t0
+    value = per_chunk * args.steps / dt
+    cores = cpu_threads()
+    sample = f"one chunk of one stream per step ({args.steps} steps after {args.warmup} warm-up chunks, carry growing from empty)"
+    print(json.dumps({
+        "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": describe(cfg), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg5", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--history", type=int, default=None,
+                    help="untimed chunks decoded per stream before warm-up (default: enough to fill the K/V carry)")
+    args = ap.parse_args()
+    cfg = wl.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import paper_2609_35115_b200 as dc
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decoder step has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dc.load_library()
+
+    metric, unit, per_chunk = units_per_chunk(cfg)
+    S, T = cfg.n_streams, cfg.f_chunk
+    W, K = max(args.warmup, 3), args.steps
+    history = HISTORY_CHUNKS if cfg.pipeline == "flow" else 2
+    if args.history is not None:
+        history = args.history
+    rounds = history + W + K
+    rng = np.random.default_rng(cfg.seed + 1000 * rank)
+    weights = wl.make_weights(cfg, np.random.default_rng(cfg.seed))
+    model = dc.Model(cfg, weights, max_batch=S)
+    streams = [model.open_stream() for _ in range(S)]
+    feats_h = torch.from_numpy(rng.standard_normal((rounds, S, T, cfg.in_dim), dtype=np.float32))
+    feats_d = feats_h.cuda()
+    out_d = torch.empty(S, T * cfg.out_per_frame, device="cuda")
+    batched = cfg.pipeline == "flow" and S > 1
+
+    def step(r):
+        if batched:
+            dc.decode_batch(model, streams, [feats_d[r, i] for i in range(S)], [out_d[i] for i in range(S)])
+        else:
+            for i in range(S):
+                streams[i].decode_chunk(feats_d[r, i], out=out_d[i])
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for r in range(history + W):
+        step(r)
+    sync_all()
+    sampler = ClockSampler(local)
+    sampler.start()
+    c0 = model.counters()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    evs[0].record()
+    for k in range(K):
+        step(history + W + k)
+        evs[k + 1].record()
+    torch.cuda.synchronize()
+    total_ms = evs[0].elapsed_time(evs[K])
+    clocks = sampler.stop()
+    c1 = model.counters()
+    step_ms = sorted(evs[k].elapsed_time(evs[k + 1]) for k in range(K))
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    value = world * S * K * per_chunk / (total_ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry points (H2D + decode + D2H + sync per step) ----
+    fin = [feats_h[r].pin_memory() for r in range(history + W, rounds)]
+    fout = torch.empty(S, T * cfg.out_per_frame).pin_memory()
+    e2e_warm = min(3, K)
+    def e2e_step(k):
+        if batched:
+            dc.decode_batch_host(model, streams, [fin[k][i] for i in range(S)], [fout[i] for i in range(S)])
+        else:
+            for i in range(S):
+                streams[i].decode_chunk_host(fin[k][i], fout[i])
+    for k in range(e2e_warm):
+        e2e_step(k)
+    sync_all()
+    t0 = time.perf_counter()
+    for k in range(K):
+        e2e_step(k)
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * S * K * per_chunk / e2e_s
+
+    # ---- per-kernel-class device time (separate profiled pass; events between launches slow the step) ----
+    pk, how = peaks()
+    nprof = min(K, 3)
+    model.profile_begin(1 << 15)
+    for k in range(nprof):
+        step(history + W + k)
+    ms, nl = model.profile_end()
+    tot = sum(ms.values()) or 1.0
+    kernels = {k: {"launches_per_step": nl[k] // nprof, "ms_per_step": ms[k] / nprof, "share": ms[k] / tot}
+               for k in ms if nl[k]}
+    dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    avg_s = 1e-3 * ms[dom] / nl[dom]
+    if dom in ("gemm_conv",):
+        fl = flops_per_launch(cfg, dom, S)
+        roof = {"kernel": "flow_gemm_kernel (conv blocks)", "bound": "tensor", "achieved": fl / avg_s / 1e12,
+                "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "peak_kind": f"bf16 sustained, {how}"}
+    elif dom == "attention":
+        by = attention_bytes_per_launch(cfg, S)
+        roof = {"kernel": "flow_attn_kernel", "bound": "hbm", "achieved": by / avg_s / 1e9, "peak": pk["hbm_gbs"],
+                "unit": "GB/s", "peak_kind": f"copy bandwidth, {how}"}
+    elif dom == "tapconv_f32":
+        fl_chunk = {"cfg4": 1.73e9, "cfg1": 0.79e6}.get(cfg.name, 0.0)
+        roof = {"kernel": "tapconv_f32_kernel", "bound": "alu", "achieved": fl_chunk / (1e-3 * ms[dom] / nprof) / 1e12,
+                "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s", "peak_kind": "FP32 FFMA, derived: 148 SM x 128 x 2 x 1.965 GHz"}
+    else:
+        roof = {"kernel": dom, "bound": "hbm", "achieved": None, "peak": pk["hbm_gbs"], "unit": "GB/s", "peak_kind": how}
+    roof["frac"] = (roof["achieved"] / roof["peak"]) if roof["achieved"] else None
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(cfg.name)
+    roof["avg_launch_us"] = 1e6 * avg_s
+    if "attention" in kernels and dom != "attention":
+        a_s = 1e-3 * ms["attention"] / nl["attention"]
+        roof["attention_hbm_gbs"] = attention_bytes_per_launch(cfg, S) / a_s / 1e9
+        roof["attention_hbm_frac"] = roof["attention_hbm_gbs"] / pk["hbm_gbs"]
+
+    # ---- the oracle on the host cores (rank 0, N = 1 only), bounded sample ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_c = {"cfg5": 40, "cfg3": 40, "cfg2": 40, "cfg4": 200, "cfg1": 8}[cfg.name]
+        f = feats_h[:, 0].reshape(-1, cfg.in_dim).numpy()
+        n_c = min(n_c, f.shape[0] // T)
+        dt = time_oracle(cfg, weights, f, n_c)
+        cpu = {"value": n_c * per_chunk / dt, "unit": unit, "cores": cpu_threads(), "kind": "oracle",
+               "sample": f"first {n_c} chunks of stream 0 (carry growing from empty), {dt:.1f} s"}
+
+    if rank == 0:
+        ws = (S * (cfg.n_steps * cfg.n_attn_layers * 2 * (cfg.kv_cap + T) * cfg.hidden * 2) / 1e6) if cfg.pipeline == "flow" else 0
+        line = {
+            "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if cfg.precision == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": describe(cfg), "streams_per_gpu": S, "frames_per_chunk": T,
+                       "history_chunks": history, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                       "l2": (f"K/V carries {ws:.0f} MB > 126 MB L2, streamed from HBM every step" if ws > 126 else
+                              "working set fits L2; inputs differ every step, no flush"),
+                       "inputs": "N(0,1) features, N(0,1/fan_in) weights, seeded"},
+            "latency_us": {"p50": 1e3 * step_ms[len(step_ms) // 2], "p95": 1e3 * step_ms[min(len(step_ms) - 1, int(0.95 * len(step_ms)))],
+                           "per": "step (one chunk of every stream)"},
+            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": S * T * cfg.in_dim * 4,
+                    "d2h_bytes_per_step": S * T * cfg.out_per_frame * 4, "ms_per_step": 1e3 * e2e_s / K},
+            "gpu_launches": int(c1[5] - c0[5]),
+            "clocks": clocks,
+            "roofline": roof,
+            "kernels": kernels,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    for s_ in streams:
+        s_.close()
+    model.destroy()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

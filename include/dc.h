@@ -154,6 +154,26 @@ dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
 dc_status dc_decode_chunk_host(dc_stream* stream, const float* feats_host, int n_frames,
                                float* out_host, int* n_out, void* cuda_stream);
 
+/* dc_decode_batch for callers with host buffers: feats_host[i] / out_host[i] are host
+ * pointers (pinned memory makes the copies asynchronous).  Copies every stream's chunk to
+ * its staging buffer, decodes the batch, copies the results back and synchronises
+ * cuda_stream. */
+dc_status dc_decode_batch_host(dc_model* model, int n, dc_stream* const* streams,
+                               const float* const* feats_host, const int* n_frames,
+                               float* const* out_host, void* cuda_stream);
+
+/* Per-kernel-class device timing, for roofline reports (the paper's
+ * measurement model, Section 2.2, Eq. 1: stage time vs its roofline bound).  Between
+ * dc_profile_begin and dc_profile_end every kernel launch of decode calls on this model is
+ * bracketed by CUDA events on the launching stream (this slows the step down: never report
+ * throughput from a profiled pass).  dc_profile_end synchronises the device and returns, per
+ * class, the summed milliseconds and the launch count.  Classes: 0 conv GEMM, 1 other GEMMs
+ * (input/QKV/output projections), 2 attention, 3 RMS norm, 4 slot table + input prep,
+ * 5 fp32 tap convolution, 6 fp32 head + inverse STFT.
+ * max_launches bounds the event pool allocated by dc_profile_begin. */
+dc_status dc_profile_begin(dc_model* model, int max_launches);
+dc_status dc_profile_end(dc_model* model, double ms[8], uint64_t launches[8]);
+
 /* Device addresses and byte sizes of the stream's carry buffers, for pointer
  * constancy checks: writes up to max_entries (address, bytes) pairs into out and
  * the number of buffers into n_entries. */

@@ -19,7 +19,8 @@ STATUS = {0: "DC_OK", 1: "DC_ERR_ARG", 2: "DC_ERR_CONFIG", 3: "DC_ERR_FRAMES", 4
 
 EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_stream_reset",
            "dc_stream_close", "dc_decode_chunk", "dc_decode_batch", "dc_decode_chunk_host",
-           "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error"]
+           "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error",
+           "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end"]
 
 
 class dc_config(C.Structure):
@@ -63,6 +64,9 @@ def load_library():
     lib.dc_decode_chunk.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
     lib.dc_decode_batch.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
     lib.dc_decode_chunk_host.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
+    lib.dc_decode_batch_host.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
+    lib.dc_profile_begin.argtypes = [vp, C.c_int]
+    lib.dc_profile_end.argtypes = [vp, cp(C.c_double), cp(C.c_uint64)]
     lib.dc_stream_carry_info.argtypes = [vp, cp(C.c_uint64), C.c_int, cp(C.c_int)]
     lib.dc_get_counters.argtypes = [vp, cp(C.c_uint64)]
     lib.dc_status_str.restype = C.c_char_p
@@ -139,6 +143,17 @@ class Model:
         _check(self.lib.dc_get_counters(self.handle, out), "dc_get_counters")
         return list(out)
 
+    def profile_begin(self, max_launches: int = 1 << 16):
+        _check(self.lib.dc_profile_begin(self.handle, max_launches), "dc_profile_begin")
+
+    def profile_end(self):
+        """Returns ({class: ms}, {class: launches}) summed since profile_begin."""
+        ms = (C.c_double * 8)()
+        n = (C.c_uint64 * 8)()
+        _check(self.lib.dc_profile_end(self.handle, ms, n), "dc_profile_end")
+        names = ["gemm_conv", "gemm_proj", "attention", "rmsnorm", "prep", "tapconv_f32", "head_istft_f32"]
+        return ({k: ms[i] for i, k in enumerate(names)}, {k: n[i] for i, k in enumerate(names)})
+
     def destroy(self):
         if self.handle:
             _check(self.lib.dc_destroy(self.handle), "dc_destroy")
@@ -199,6 +214,17 @@ class Stream:
         if self.handle:
             _check(self.lib.dc_stream_close(self.handle), "dc_stream_close")
             self.handle = C.c_void_p()
+
+
+def decode_batch_host(model: Model, streams: Sequence[Stream], feats_host: Sequence, outs_host: Sequence, stream=None):
+    """dc_decode_batch_host: feats_host[i] / outs_host[i] are CPU float32 tensors (ideally pinned)."""
+    n = len(streams)
+    hs = (C.c_void_p * n)(*[s.handle for s in streams])
+    fp = (C.c_void_p * n)(*[f.data_ptr() for f in feats_host])
+    op = (C.c_void_p * n)(*[o.data_ptr() for o in outs_host])
+    nf = (C.c_int * n)(*[f.shape[0] for f in feats_host])
+    _check(model.lib.dc_decode_batch_host(model.handle, n, hs, fp, nf, op, _cuda_stream_handle(stream)),
+           "dc_decode_batch_host")
 
 
 def decode_batch(model: Model, streams: Sequence[Stream], feats: Sequence, outs: Sequence, stream=None):

@@ -71,6 +71,7 @@ struct dc_model {
   std::atomic<uint64_t> counters[8];
   std::atomic<int> open_streams{0};
   std::mutex mu;
+  dc::Profiler prof;
   std::vector<dc_stream*> all_streams;   // host structs live until dc_destroy, so a closed handle stays detectable
 };
 
@@ -389,6 +390,7 @@ static dc_status decode_f32(dc_stream* s, const float* feats, int T, float* out,
       h.tail_in = s->tails + 12 * (s->chunks & 1);
       h.tail_out = s->tails + 12 * ((s->chunks + 1) & 1);
       h.pcm = out;
+      dc::ProfScope ps(&m->prof, 6, cs);
       dc::launch_head_istft_f32(h, cs);
     } else {
       dc::TapConvF32 p{};
@@ -408,6 +410,7 @@ static dc_status decode_f32(dc_stream* s, const float* feats, int T, float* out,
       } else {
         p.out_direct = out; p.pos_out = pos * p.n_phase;
       }
+      dc::ProfScope ps(&m->prof, 5, cs);
       dc::launch_tapconv_f32(p, cs);
     }
     ++*launches;
@@ -512,6 +515,67 @@ extern "C" dc_status dc_decode_chunk_host(dc_stream* s, const float* feats_host,
   DC_CUDA(cudaMemcpyAsync(out_host, s->stage_out, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaStreamSynchronize(cs));
   if (n_out) *n_out = n;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* streams, const float* const* feats_host,
+                                          const int* n_frames, float* const* out_host, void* cuda_stream) {
+  if (!m || !streams || !feats_host || !n_frames || !out_host) return DC_ERR_ARG;
+  if (n < 1 || n > m->cfg.max_batch) return DC_ERR_ARG;
+  cudaStream_t cs = (cudaStream_t)cuda_stream;
+  std::vector<const float*> fin((size_t)n);
+  std::vector<float*> fout((size_t)n);
+  for (int i = 0; i < n; ++i) {
+    dc_status st = admit(streams[i], feats_host[i], n_frames[i], out_host[i]);
+    if (st != DC_OK) return st;
+    fin[(size_t)i] = streams[i]->stage_in;
+    fout[(size_t)i] = streams[i]->stage_out;
+  }
+  for (int i = 0; i < n; ++i)
+    DC_CUDA(cudaMemcpyAsync(streams[i]->stage_in, feats_host[i], (size_t)n_frames[i] * m->in_dim * sizeof(float),
+                            cudaMemcpyHostToDevice, cs));
+  dc_status st = dc_decode_batch(m, n, streams, fin.data(), n_frames, fout.data(), cuda_stream);
+  if (st != DC_OK) return st;
+  for (int i = 0; i < n; ++i)
+    DC_CUDA(cudaMemcpyAsync(out_host[i], streams[i]->stage_out, (size_t)n_frames[i] * m->out_per_frame * sizeof(float),
+                            cudaMemcpyDeviceToHost, cs));
+  DC_CUDA(cudaStreamSynchronize(cs));
+  return DC_OK;
+}
+
+extern "C" dc_status dc_profile_begin(dc_model* m, int max_launches) {
+  if (!m || max_launches < 1 || max_launches > (1 << 20)) return DC_ERR_ARG;
+  dc::Profiler& p = m->prof;
+  if (p.on) return DC_ERR_STATE;
+  p.ev = new (std::nothrow) cudaEvent_t[2 * (size_t)max_launches];
+  p.cls = new (std::nothrow) int[(size_t)max_launches];
+  if (!p.ev || !p.cls) return DC_ERR_OOM;
+  for (int i = 0; i < 2 * max_launches; ++i) DC_CUDA(cudaEventCreate(&p.ev[i]));
+  p.cap = max_launches;
+  p.used = 0;
+  p.on = true;
+  if (m->flow) dc::flow_set_profiler(m->flow, &p);
+  return DC_OK;
+}
+
+extern "C" dc_status dc_profile_end(dc_model* m, double ms[8], uint64_t launches[8]) {
+  if (!m || !ms || !launches) return DC_ERR_ARG;
+  dc::Profiler& p = m->prof;
+  if (!p.on) return DC_ERR_STATE;
+  p.on = false;
+  if (m->flow) dc::flow_set_profiler(m->flow, nullptr);
+  DC_CUDA(cudaDeviceSynchronize());
+  for (int i = 0; i < 8; ++i) { ms[i] = 0.0; launches[i] = 0; }
+  for (int i = 0; i < p.used; ++i) {
+    float t = 0.f;
+    DC_CUDA(cudaEventElapsedTime(&t, p.ev[2 * i], p.ev[2 * i + 1]));
+    ms[p.cls[i] & 7] += (double)t;
+    launches[p.cls[i] & 7] += 1;
+  }
+  for (int i = 0; i < 2 * p.cap; ++i) cudaEventDestroy(p.ev[i]);
+  delete[] p.ev;
+  delete[] p.cls;
+  p.ev = nullptr; p.cls = nullptr; p.cap = p.used = 0;
   return DC_OK;
 }
 

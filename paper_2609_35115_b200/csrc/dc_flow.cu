@@ -610,6 +610,7 @@ struct FlowModel {
   size_t o_bin = 0, o_bout = 0, o_tau = 0;
   std::vector<size_t> o_bconv, o_bqkv, o_bo;
   std::vector<void*> allocs;
+  Profiler* prof = nullptr;
 };
 
 struct FlowState {
@@ -848,6 +849,10 @@ void flow_state_close(FlowState* s) {
 
 void launch_flow_attention(FlowModel* m, int n, int step, int layer, cudaStream_t st);
 
+void flow_set_profiler(FlowModel* m, Profiler* prof) { m->prof = prof; }
+
+
+
 dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats, const int* T,
                       float* const* outp, cudaStream_t st, int* launches) {
   const dc_config& c = m->cfg;
@@ -869,10 +874,16 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       si.halo = s->halo;
       si.kv = s->kv;
     }
-    set_slots_kernel<<<1, MAX_SLOTS_PER_SET, 0, st>>>(set, m->d_slots);
+    {
+      ProfScope ps(m->prof, 4, st);
+      set_slots_kernel<<<1, MAX_SLOTS_PER_SET, 0, st>>>(set, m->d_slots);
+    }
     ++*launches;
   }
-  flow_prep_kernel<<<n, 128, 0, st>>>(m->d_slots, mel, m->xstate, m->Ain, m->Kin);
+  {
+    ProfScope ps(m->prof, 4, st);
+    flow_prep_kernel<<<n, 128, 0, st>>>(m->d_slots, mel, m->xstate, m->Ain, m->Kin);
+  }
   ++*launches;
 
   const int m_tiles = (n * SLOT_ROWS + TILE_M - 1) / TILE_M;
@@ -884,11 +895,13 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
     p.Rk = m->Rk;
     p.err = m->d_err;
     dim3 grid(m_tiles, N / p.BN);
+    ProfScope ps(m->prof, p.mode == MODE_CONV ? 0 : 1, st);
     flow_gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(tA, tB, p);
     ++*launches;
   };
   auto rmsnorm = [&](const bf16* x) {
     const int warps = n * SLOT_ROWS;
+    ProfScope ps(m->prof, 3, st);
     flow_rmsnorm_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(m->d_slots, n, x, m->U, C, c.rms_eps);
     ++*launches;
   };
@@ -970,6 +983,7 @@ void launch_flow_attention(FlowModel* m, int n, int step, int layer, cudaStream_
   p.Rk = m->Rk; p.C = m->C; p.kv_rows_max = m->kv_rows_max;
   p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
   p.err = m->d_err;
+  ProfScope ps(m->prof, 2, st);
   flow_attn_kernel<<<dim3(n, c.n_heads), ATT_THREADS, m->attn_smem, st>>>(p);
 }
 

@@ -88,4 +88,30 @@ void      flow_state_close(FlowState* s);
 dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats_dev,
                       const int* n_frames, float* const* out_dev, cudaStream_t st, int* launches);
 
+// Event-bracketed launches while profiling is on (see dc_profile_begin in dc.h).
+struct Profiler {
+  bool on = false;
+  int  used = 0, cap = 0;
+  cudaEvent_t* ev = nullptr;     // 2 per launch
+  int*         cls = nullptr;
+};
+void flow_set_profiler(FlowModel* m, Profiler* prof);
+
+// Brackets one launch with events when profiling is on.
+struct ProfScope {
+  Profiler*    p;
+  cudaStream_t st;
+  int          idx = -1;
+  ProfScope(Profiler* prof, int cls, cudaStream_t s) : p(prof), st(s) {
+    if (p && p->on && p->used < p->cap) {
+      idx = p->used++;
+      p->cls[idx] = cls;
+      cudaEventRecord(p->ev[2 * idx], st);
+    }
+  }
+  ~ProfScope() {
+    if (idx >= 0) cudaEventRecord(p->ev[2 * idx + 1], st);
+  }
+};
+
 }  // namespace dc

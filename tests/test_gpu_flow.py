@@ -110,3 +110,42 @@ def test_flow_reset_and_pointer_constancy(dc):
     assert st.carry_info() == before and np.array_equal(a, b)
     st.close()
     m.destroy()
+
+
+def test_cfg5_multi_stream_serving_full_size(dc):
+    """32 staggered streams x 100 chunks through dc_decode_batch (the launch configuration the
+    benchmark times).  Sampled streams are checked against the oracle; every stream is checked
+    against the property that batching does not change the bytes (prefix of 12 chunks)."""
+    gu = _gu()
+    cfg = wl.CONFIGS["cfg5"]
+    w = wl.make_workload(cfg)
+    S = cfg.n_streams
+    assert len({s.boundaries[1] for s in w.streams}) > 8          # offsets really are staggered
+    m = dc.Model(cfg, w.weights, max_batch=S)
+    streams = [m.open_stream() for _ in range(S)]
+    feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+    outs = [torch.empty(s.feats.shape[0], cfg.mel_dim, device="cuda") for s in w.streams]
+    for r in range(cfg.n_chunks):
+        fs = [feats[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
+        os_ = [outs[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
+        dc.decode_batch(m, streams, fs, os_)
+    torch.cuda.synchronize()
+    for st in streams:
+        st.close()
+    got = [o.cpu().numpy() for o in outs]
+    assert all(np.isfinite(g).all() for g in got)
+    # (a) one stream against the oracle over all 100 chunks, another over its first 14 chunks
+    s7 = w.streams[7]
+    ref = orc.run_stream(cfg, w.weights, s7.feats, s7.boundaries)
+    assert gu.rel_err(got[7], ref) <= TOL_BF16
+    s20 = w.streams[20]
+    b = s20.boundaries[:15]
+    ref = orc.run_stream(cfg, w.weights, s20.feats[:b[-1]], b)
+    assert gu.rel_err(got[20][:b[-1]], ref) <= TOL_BF16
+    # (b) batching never changes a stream's bytes
+    for i in (0, 13, 31):
+        si = w.streams[i]
+        b = si.boundaries[:13]
+        single = gu.run_gpu_stream(m, si.feats[:b[-1]], b)
+        assert np.array_equal(single, got[i][:b[-1]])
+    m.destroy()
