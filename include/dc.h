@@ -174,6 +174,39 @@ dc_status dc_decode_batch_host(dc_model* model, int n, dc_stream* const* streams
 dc_status dc_profile_begin(dc_model* model, int max_launches);
 dc_status dc_profile_end(dc_model* model, double ms[8], uint64_t launches[8]);
 
+/* (The paper has no counterpart for this entry point; it exists for callers that cannot
+ * allocate device memory.)
+ *
+ * Some callers of this library run where cudaMalloc is off limits: inside a region whose memory
+ * budget is fixed up front, in a process that must not disturb another allocator's pool, or in a
+ * real-time audio callback where an allocation's unbounded latency is unacceptable.  dc_create
+ * and dc_stream_open allocate, so those callers cannot use the stream API.  For them this one call
+ * runs the causal conv residual stack (the DC_PIPE_CONV network: n_conv blocks of
+ * h <- h + SiLU(conv_k3,dilation(h) + b)) over ONE whole sequence with zero left context, and
+ * keeps the activations that pass between blocks in a fixed array that is part of the library
+ * image instead of in allocated buffers.  The call allocates nothing: no cudaMalloc, no cudaFree,
+ * no allocating library routine.
+ *
+ *   weights_dev : DEVICE pointer, canonical conv blob (per block W[3][C][C], b[C]), fp32
+ *   dilations   : HOST array of n_conv dilations (each >= 1)
+ *   x_dev       : DEVICE fp32 [n_frames][hidden] input;  y_dev: DEVICE fp32 [n_frames][hidden] output
+ *
+ * Limit: the scratch array holds DC_NOALLOC_SCRATCH_FLOATS floats (2 MiB; every GPU that loads
+ * the library carries it until the process exits).  A call needs 2 * P * hidden floats, where P
+ * is the smallest power of two >= n_frames + 2 * max(dilations); larger requests are refused
+ * with DC_ERR_ARG and a message (dc_last_error) that states the need and the limit.  hidden must
+ * be a multiple of 4.
+ *
+ * The first call on a device looks up the array's device address (a synchronous runtime query,
+ * made with that device current); make that first call outside any stream capture.  All calls on
+ * a device share the one array, which still holds the previous call's values: the call itself
+ * clears the rows that must read as zero, and two calls that overlap on the GPU (issued on
+ * different CUDA streams without ordering) race on it - order them.  Work is enqueued on
+ * cuda_stream; the result is ready when that stream reaches the end of the call's work. */
+#define DC_NOALLOC_SCRATCH_FLOATS (1u << 19)
+dc_status dc_conv_stack_noalloc(const float* weights_dev, int hidden, int n_conv, const int* dilations,
+                                const float* x_dev, int n_frames, float* y_dev, void* cuda_stream);
+
 /* Device addresses and byte sizes of the stream's carry buffers, for pointer
  * constancy checks: writes up to max_entries (address, bytes) pairs into out and
  * the number of buffers into n_entries. */

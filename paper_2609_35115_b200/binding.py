@@ -20,7 +20,7 @@ STATUS = {0: "DC_OK", 1: "DC_ERR_ARG", 2: "DC_ERR_CONFIG", 3: "DC_ERR_FRAMES", 4
 EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_stream_reset",
            "dc_stream_close", "dc_decode_chunk", "dc_decode_batch", "dc_decode_chunk_host",
            "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error",
-           "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end"]
+           "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end", "dc_conv_stack_noalloc"]
 
 
 class dc_config(C.Structure):
@@ -67,6 +67,7 @@ def load_library():
     lib.dc_decode_batch_host.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
     lib.dc_profile_begin.argtypes = [vp, C.c_int]
     lib.dc_profile_end.argtypes = [vp, cp(C.c_double), cp(C.c_uint64)]
+    lib.dc_conv_stack_noalloc.argtypes = [vp, C.c_int, C.c_int, cp(C.c_int), vp, C.c_int, vp, vp]
     lib.dc_stream_carry_info.argtypes = [vp, cp(C.c_uint64), C.c_int, cp(C.c_int)]
     lib.dc_get_counters.argtypes = [vp, cp(C.c_uint64)]
     lib.dc_status_str.restype = C.c_char_p
@@ -236,3 +237,16 @@ def decode_batch(model: Model, streams: Sequence[Stream], feats: Sequence, outs:
     nf = (C.c_int * n)(*[f.shape[0] for f in feats])
     _check(model.lib.dc_decode_batch(model.handle, n, hs, fp, nf, op, _cuda_stream_handle(stream)),
            "dc_decode_batch")
+
+
+NOALLOC_SCRATCH_FLOATS = 1 << 19
+
+
+def conv_stack_noalloc(weights_dev, hidden: int, dilations: Sequence[int], x, y, stream=None) -> int:
+    """dc_conv_stack_noalloc: the conv residual stack over one whole sequence, for callers that
+    must not allocate device memory.  weights_dev, x, y are CUDA float32 tensors the caller owns;
+    returns the dc_status (0 = DC_OK) so that refusals can be inspected."""
+    lib = load_library()
+    d = (C.c_int * len(dilations))(*dilations)
+    return lib.dc_conv_stack_noalloc(weights_dev.data_ptr(), hidden, len(dilations), d, x.data_ptr(),
+                                     x.shape[0], y.data_ptr(), _cuda_stream_handle(stream))

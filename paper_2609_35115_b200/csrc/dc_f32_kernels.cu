@@ -6,6 +6,8 @@
 
 #include <math.h>
 
+#include <mutex>
+
 namespace dc {
 
 namespace {
@@ -242,3 +244,119 @@ void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st) {
 }
 
 }  // namespace dc
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free conv stack (see dc.h).  The activations between blocks live in this array,
+// which is part of the library image.  In host code `g_noalloc_scratch` is only a handle for the
+// runtime's symbol lookup, never an address to hand to a kernel; the device address comes from
+// cudaGetSymbolAddress, once per device.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) float g_noalloc_scratch[DC_NOALLOC_SCRATCH_FLOATS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float*     g_noalloc_ptr[kMaxDevices] = {nullptr};
+std::mutex g_noalloc_mu;
+
+// Device address of the scratch array on the current device (looked up on first use).
+dc_status noalloc_scratch(float** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    dc::set_error("dc_conv_stack_noalloc: cannot identify the current device (%s)", cudaGetErrorString(e));
+    return DC_ERR_CUDA;
+  }
+  std::lock_guard<std::mutex> lk(g_noalloc_mu);
+  if (g_noalloc_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess || p == nullptr) {
+      dc::set_error("dc_conv_stack_noalloc: cudaGetSymbolAddress failed on device %d: %s", dev, cudaGetErrorString(e));
+      return DC_ERR_CUDA;
+    }
+    g_noalloc_ptr[dev] = static_cast<float*>(p);
+  }
+  *out = g_noalloc_ptr[dev];
+  return DC_OK;
+}
+}  // namespace
+
+extern "C" dc_status dc_conv_stack_noalloc(const float* weights_dev, int hidden, int n_conv, const int* dilations,
+                                           const float* x_dev, int n_frames, float* y_dev, void* cuda_stream) {
+  if (!weights_dev || !dilations || !x_dev || !y_dev) {
+    dc::set_error("dc_conv_stack_noalloc: null pointer argument");
+    return DC_ERR_ARG;
+  }
+  if (hidden < 4 || hidden % 4 || n_conv < 1 || n_conv > DC_MAX_CONV || n_frames < 1) {
+    dc::set_error("dc_conv_stack_noalloc: need hidden %% 4 == 0, 1 <= n_conv <= %d, n_frames >= 1", DC_MAX_CONV);
+    return DC_ERR_ARG;
+  }
+  int dmax = 0;
+  for (int l = 0; l < n_conv; ++l) {
+    if (dilations[l] < 1 || dilations[l] > 4096) {
+      dc::set_error("dc_conv_stack_noalloc: dilation %d out of range", dilations[l]);
+      return DC_ERR_ARG;
+    }
+    dmax = dilations[l] > dmax ? dilations[l] : dmax;
+  }
+  const long long halo = 2ll * dmax;
+  long long cap = 1;
+  while (cap < (long long)n_frames + halo) cap <<= 1;
+  const long long need = 2 * cap * hidden;
+  if (need > (long long)DC_NOALLOC_SCRATCH_FLOATS) {
+    dc::set_error("dc_conv_stack_noalloc: %d frames x %d channels with dilation %d need %lld scratch floats, "
+                  "the built-in array holds %u", n_frames, hidden, dmax, need, DC_NOALLOC_SCRATCH_FLOATS);
+    return DC_ERR_ARG;
+  }
+  float* scratch = nullptr;
+  dc_status st = noalloc_scratch(&scratch);
+  if (st != DC_OK) return st;
+  cudaStream_t cs = (cudaStream_t)cuda_stream;
+  float* region[2] = {scratch, scratch + cap * hidden};
+  // The array keeps the previous call's values.  Rows [cap - halo, cap) of both regions are the
+  // frames "before the start" that every block reads as its left context: they must be zero.
+  for (int r = 0; r < 2; ++r) {
+    cudaError_t e = cudaMemsetAsync(region[r] + (cap - halo) * hidden, 0, (size_t)(halo * hidden) * sizeof(float), cs);
+    if (e != cudaSuccess) {
+      dc::set_error("dc_conv_stack_noalloc: clearing the left context failed: %s", cudaGetErrorString(e));
+      return DC_ERR_CUDA;
+    }
+  }
+  size_t woff = 0;
+  for (int l = 0; l < n_conv; ++l) {
+    dc::TapConvF32 p{};
+    // block l reads region[l & 1] (block 0: the caller's x, whose left context is the zeroed rows
+    // of region[0]) and writes region[(l + 1) & 1] (last block: the caller's y)
+    p.in_ring = region[l & 1];
+    p.in_mask = (int)cap - 1;
+    p.in_direct = (l == 0) ? x_dev : nullptr;
+    p.pos_in = 0;
+    p.T_in = n_frames;
+    p.C_in = hidden;
+    p.n_taps = 3;
+    p.shift[0] = 2 * dilations[l]; p.shift[1] = dilations[l]; p.shift[2] = 0;
+    p.n_phase = 1;
+    p.W = weights_dev + woff;
+    p.w_tap_stride = (long long)hidden * hidden;
+    p.w_phase_stride = 0;
+    woff += (size_t)3 * hidden * hidden;
+    p.bias = weights_dev + woff;
+    woff += (size_t)hidden;
+    p.C_out = hidden;
+    p.residual_silu = 1;
+    if (l + 1 < n_conv) {
+      p.out_ring = region[(l + 1) & 1];
+      p.out_mask = (int)cap - 1;
+    } else {
+      p.out_direct = y_dev;
+      p.pos_out = 0;
+    }
+    dc::launch_tapconv_f32(p, cs);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    dc::set_error("dc_conv_stack_noalloc: launch failed: %s", cudaGetErrorString(e));
+    return DC_ERR_CUDA;
+  }
+  return DC_OK;
+}
