@@ -15,6 +15,7 @@
 #include <cuda.h>
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -35,10 +36,13 @@ constexpr int SLOT_ROWS = 64;   // rows per stream slot: 8 left-context rows + u
 constexpr int HALO = 8;         // carried frames per (step, conv block); dilation <= 4 reads at most 8 back
 constexpr int TILE_M = 128;
 constexpr int KBLK = 64;        // bf16 elements per 128-byte swizzled smem row
-constexpr int STAGES = 4;
-constexpr int A_BYTES = TILE_M * 128;
+constexpr int MAX_STAGES = 8;
+constexpr int GEMM_TILE_SMEM = 200 * 1024;   // bytes of operand stages per CTA
+constexpr int A_ROWS = TILE_M + HALO;  // the A tile carries 8 extra leading rows so that all taps read it
+constexpr int A_BYTES = A_ROWS * 128;
 constexpr int MAX_BN = 128;
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 352;      // warp 0 TMA (A), warp 1 UMMA, warp 2 TMA (B), warps 3..10 epilogue
+constexpr int EPI_THREADS = 256;
 constexpr int MAX_SLOTS_PER_SET = 64;
 
 enum GemmMode { MODE_INPROJ = 0, MODE_CONV = 1, MODE_QKV = 2, MODE_OPROJ = 3, MODE_OUT = 4 };
@@ -62,10 +66,11 @@ struct SlotSet {
 struct GemmParams {
   int          mode;
   int          BN;              // output columns per CTA (multiple of 16, <= 128)
+  int          n_stages;        // TMA pipeline depth (<= MAX_STAGES, n_stages * stage bytes <= GEMM_TILE_SMEM)
   int          n_slots;
-  int          n_kblocks;       // total 64-wide reduction blocks (= taps * kb_per_tap)
-  int          kb_per_tap;
-  int          shift[3];        // row shift of tap j
+  int          n_kblocks;       // 64-wide channel blocks of the A matrix (one pipeline stage each)
+  int          taps;            // 1, or 3 for the conv blocks (weights: K index = tap * 64 * n_kblocks + channel)
+  int          shift[3];        // row shift of tap j (0..8)
   const float* bias;            // [N]
   const float* tau;             // [N] or null
   const bf16*  resid;           // residual source matrix (same row layout) or null
@@ -84,9 +89,10 @@ struct GemmParams {
   int          last_step;
   int          mel;
   int*         err;
+  int          dbg;
 };
 
-__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
+__device__ __forceinline__ float silu_f(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
 __device__ __forceinline__ void load16_bf16(const bf16* p, float* v) {
   const uint4 a = *reinterpret_cast<const uint4*>(p);
@@ -117,22 +123,39 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sA = smem;
-  uint8_t* sB = smem + STAGES * A_BYTES;
-  uint64_t* full = reinterpret_cast<uint64_t*>(sB + STAGES * MAX_BN * 128);
-  uint64_t* empty = full + STAGES;
-  uint64_t* accum = empty + STAGES;
+  // stage = [A tile 136 x 128 B | one B tile BN x 128 B per tap]; all tile sizes are multiples of
+  // 1024 B.  The A tile starts 8 rows above the output tile: tap j reads it from row 8 - shift[j],
+  // so one load serves all taps.
+  const uint32_t b_bytes = (uint32_t)p.BN * 128u;
+  const uint32_t b_tile = (b_bytes + 1023u) & ~1023u;
+  const uint32_t stage_bytes = (uint32_t)A_BYTES + (uint32_t)p.taps * b_tile;
+  const int STAGES = p.n_stages;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + GEMM_TILE_SMEM);
+  uint64_t* empty = full + MAX_STAGES;
+  uint64_t* accum = empty + MAX_STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
   int* s_fail = reinterpret_cast<int*>(tmem_slot + 1);
+  float* s_bias = reinterpret_cast<float*>(s_fail + 1);
+  float* s_tau = s_bias + MAX_BN;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * TILE_M, n0 = blockIdx.y * p.BN;
-  const uint32_t b_bytes = (uint32_t)p.BN * 128u;
+#ifdef DC_TIMING
+  const bool tm = blockIdx.x == 1 && blockIdx.y == 1 && p.mode == MODE_CONV;
+  long long t_start = 0;
+  if (tm) t_start = clock64();
+  __shared__ long long s_t[8];
+  __shared__ long long s_k[32];
+  __shared__ long long s_p[32];
+#define DC_T(idx) do { if (tm) s_t[idx] = clock64() - t_start; } while (0)
+#else
+#define DC_T(tag) do {} while (0)
+#endif
   const uint32_t tmem_cols = p.BN <= 32 ? 32u : (p.BN <= 64 ? 64u : 128u);
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
-      ptx::mbar_init(&full[i], 1);
+      ptx::mbar_init(&full[i], 2);   // one arrival per producer thread
       ptx::mbar_init(&empty[i], 1);
     }
     ptx::mbar_init(accum, 1);
@@ -144,24 +167,35 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) DC_T(0);
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 2) {
+    // two producer threads, one per tensor map: warp 0 streams the A tiles, warp 2 the weight tiles
     if (lane == 0) {
-      ptx::prefetch_tmap(&tmA);
-      ptx::prefetch_tmap(&tmB);
+      const bool is_a = warp == 0;
       for (int kb = 0; kb < p.n_kblocks; ++kb) {
         const int st = kb % STAGES;
+#ifdef DC_TIMING
+        if ((p.dbg & 4) && kb >= STAGES) break;
+#endif
         if (kb >= STAGES && !ptx::mbar_wait(&empty[st], ((kb / STAGES) - 1) & 1)) {
           atomicExch(p.err, 1);
           *s_fail = 1;
           break;
         }
-        const int tap = kb / p.kb_per_tap;
-        const int cb = kb - tap * p.kb_per_tap;
-        ptx::mbar_expect_tx(&full[st], (uint32_t)A_BYTES + b_bytes);
-        ptx::tma_load_2d(sA + st * A_BYTES, &tmA, cb * KBLK, GUARD + m0 - p.shift[tap], &full[st]);
-        ptx::tma_load_2d(sB + st * MAX_BN * 128, &tmB, kb * KBLK, n0, &full[st]);
+#ifdef DC_TIMING
+        if (tm && kb < 32 && is_a) s_p[kb] = clock64() - t_start;
+#endif
+        if (is_a) {
+          ptx::mbar_expect_tx(&full[st], (uint32_t)A_BYTES);
+          ptx::tma_load_2d(smem + st * stage_bytes, &tmA, kb * KBLK, GUARD + m0 - HALO, &full[st]);
+        } else {
+          ptx::mbar_expect_tx(&full[st], (uint32_t)p.taps * b_bytes);
+          for (int j = 0; j < p.taps; ++j)
+            ptx::tma_load_2d(smem + st * stage_bytes + A_BYTES + j * b_tile, &tmB, (j * p.n_kblocks + kb) * KBLK, n0, &full[st]);
+        }
       }
+      if (is_a) DC_T(1);
     }
   } else if (warp == 1) {
     if (lane == 0) {
@@ -169,46 +203,103 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       bool ok = true;
       for (int kb = 0; kb < p.n_kblocks && ok; ++kb) {
         const int st = kb % STAGES;
+#ifdef DC_TIMING
+        if ((p.dbg & 4) && kb >= STAGES) goto skip_wait;
+#endif
         if (!ptx::mbar_wait(&full[st], (kb / STAGES) & 1)) {
           atomicExch(p.err, 2);
           *s_fail = 1;
           ok = false;
           break;
         }
+#ifdef DC_TIMING
+      skip_wait:
+#endif
         ptx::tc_fence_after();
-        const uint32_t a0 = ptx::smem_u32(sA + st * A_BYTES), b0 = ptx::smem_u32(sB + st * MAX_BN * 128);
+        if (kb == 0) DC_T(2);
+#ifdef DC_TIMING
+        if (tm && kb < 32) s_k[kb] = clock64() - t_start;
+#endif
+        const uint32_t a0 = ptx::smem_u32(smem + st * stage_bytes), b0 = a0 + A_BYTES;
+        for (int j = 0; j < p.taps; ++j) {
+          // descriptors differ only in the 16-byte-unit start address (low bits): +2 per 32-byte K step
+          const uint64_t da = ptx::umma_desc_sw128(a0 + (uint32_t)(HALO - p.shift[j]) * 128u);
+          const uint64_t db = ptx::umma_desc_sw128(b0 + (uint32_t)j * b_tile);
 #pragma unroll
-        for (int k = 0; k < KBLK / 16; ++k)
-          ptx::umma_bf16(tmem_base, ptx::umma_desc_sw128(a0 + k * 32), ptx::umma_desc_sw128(b0 + k * 32), idesc,
-                         (kb | k) != 0);
+          for (int k = 0; k < KBLK / 16; ++k) {
+#ifdef DC_TIMING
+            if ((p.dbg & 1) && k != 0) continue;
+            if ((p.dbg & 2) && (k != 0 || j != 0)) continue;
+#endif
+            ptx::umma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | j | k) != 0);
+          }
+        }
         ptx::umma_commit(&empty[st]);
       }
+      DC_T(3);
       ptx::umma_commit(accum);   // arrives when every UMMA above has finished (also on the failure path)
     }
   } else {
-    // ---------------- epilogue: 4 warps, thread <-> output row ----------------
-    const bool got = ptx::mbar_wait(accum, 0);
-    ptx::tc_fence_after();
-    if (!got) atomicExch(p.err, 3);
+    // ---------------- epilogue: 8 warps; a thread owns one output row and every other 16-column chunk ----------------
+    // Everything that does not depend on the accumulator is fetched while the main loop runs:
+    // per-column constants go to shared memory, the thread's residual row (or, for a left-context
+    // row, the carried row) goes to registers.
+    const int et = threadIdx.x - 96;
+    if (et < p.BN) {   // BN <= 128 < EPI_THREADS
+      s_bias[et] = p.bias[n0 + et];
+      s_tau[et] = p.tau != nullptr ? p.tau[n0 + et] : 0.f;
+    }
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    const int half = (warp - 3) >> 2;             // which chunks of the row: chunk index & 1 == half
     const int r = m0 + q * 32 + lane;             // row in slot layout (without GUARD)
     const int slot = r / SLOT_ROWS, rho = r % SLOT_ROWS;
-    const bool slot_ok = slot < p.n_slots && got && *s_fail == 0;
-    const SlotInfo si = slot_ok ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr};
+    const bool in_range = slot < p.n_slots;
+    const SlotInfo si = in_range ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr};
     const int f = rho - HALO;
+    const bool do_halo = p.halo_off >= 0;
+    const bool has_resid = p.mode == MODE_CONV || p.mode == MODE_OPROJ;
+    const long long grow = (long long)(GUARD + r);
+    bf16* carry = do_halo && in_range ? si.halo + p.halo_off : nullptr;
+    // pre[2k], pre[2k+1]: the 16 bf16 of this thread's k-th chunk (columns n0 + 16 (2k + half) ..)
+    uint4 pre[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) pre[j] = make_uint4(0u, 0u, 0u, 0u);
+    {
+      const bf16* src = nullptr;
+      if (in_range && f >= 0 && f < si.T && has_resid) src = p.resid + grow * p.ld + n0;
+      else if (in_range && rho < HALO && do_halo) src = carry + rho * p.C + n0;
+      if (src != nullptr) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          pre[2 * k] = *reinterpret_cast<const uint4*>(src + 16 * (2 * k + half));
+          pre[2 * k + 1] = *reinterpret_cast<const uint4*>(src + 16 * (2 * k + half) + 8);
+        }
+      }
+    }
+    // constants visible to all epilogue threads; every read of the carry has been performed
+    // before any thread below overwrites carry rows
+    ptx::named_bar_sync(1, EPI_THREADS);
+
+    const bool got = ptx::mbar_wait_relaxed(accum, 0);
+    ptx::tc_fence_after();
+    if (threadIdx.x == 96) DC_T(4);
+    if (!got) atomicExch(p.err, 3);
+    const bool slot_ok = in_range && got && *s_fail == 0;
     const bool is_halo = slot_ok && rho < HALO;
     const bool is_chunk = slot_ok && f >= 0 && f < si.T;
-    const long long grow = (long long)(GUARD + r);
-    const bool do_halo = p.halo_off >= 0;
-    bf16* carry = do_halo && slot_ok ? si.halo + p.halo_off : nullptr;
     const int new_row = rho - si.T;               // carry row this thread's value moves to
     const bool carry_wr = do_halo && (is_halo || is_chunk) && new_row >= 0 && new_row < HALO;
 
-    for (int c0 = 0; c0 < p.BN; c0 += 16) {
+#pragma unroll
+    for (int kk = 0; kk < MAX_BN / 32; ++kk) {
+      const int ch = 2 * kk + half;
+      const int c0 = ch * 16;
+      if (c0 >= p.BN) break;
       float acc[16];
       ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
       const int n = n0 + c0;
-      float y[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) acc[i] += s_bias[c0 + i];
       if (p.mode == MODE_OUT) {
         if (is_chunk) {
           float* xs = p.xstate + (long long)r * p.mel + n;
@@ -219,7 +310,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             xv[i] = t.x; xv[i + 1] = t.y; xv[i + 2] = t.z; xv[i + 3] = t.w;
           }
 #pragma unroll
-          for (int i = 0; i < 16; ++i) xv[i] = xv[i] + (acc[i] + p.bias[n + i]) * p.inv_n;
+          for (int i = 0; i < 16; ++i) xv[i] = xv[i] + acc[i] * p.inv_n;
 #pragma unroll
           for (int i = 0; i < 16; i += 4)
             *reinterpret_cast<float4*>(xs + i) = make_float4(xv[i], xv[i + 1], xv[i + 2], xv[i + 3]);
@@ -235,12 +326,10 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         continue;
       }
-#pragma unroll
-      for (int i = 0; i < 16; ++i) y[i] = acc[i] + p.bias[n + i];
       if (p.mode == MODE_QKV) {
         if (is_chunk) {
           uint4 a, b;
-          pack16_bf16(y, a, b);
+          pack16_bf16(acc, a, b);
           const int which = n / p.C, col = n - which * p.C;
           if (which == 0) {
             store16(p.q_out + grow * p.ld + col, a, b);
@@ -252,41 +341,51 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         continue;
       }
-      if (p.mode == MODE_CONV || p.mode == MODE_OPROJ) {
-        float x[16];
-        if (is_chunk) {
-          load16_bf16(p.resid + grow * p.ld + n, x);
-        } else {
+      // modes with a bf16 activation output: INPROJ, CONV, OPROJ (BN <= 64, so kk < 2)
+      uint4 va = pre[(2 * kk) & 3], vb = pre[(2 * kk + 1) & 3];
+      if (!is_halo) {
+        if (has_resid) {
+          const uint32_t w[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+          if (p.mode == MODE_CONV) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) x[i] = 0.f;
+            for (int i = 0; i < 8; ++i) {
+              acc[2 * i] = __uint_as_float(w[i] << 16) + silu_f(acc[2 * i] + s_tau[c0 + 2 * i]);
+              acc[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u) + silu_f(acc[2 * i + 1] + s_tau[c0 + 2 * i + 1]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              acc[2 * i] += __uint_as_float(w[i] << 16);
+              acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+            }
+          }
         }
-        if (p.mode == MODE_CONV) {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) y[i] = x[i] + silu_f(y[i] + p.tau[n + i]);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) y[i] = x[i] + y[i];
-        }
+        pack16_bf16(acc, va, vb);
       }
-      uint4 va, vb;
-      pack16_bf16(y, va, vb);
-      if (is_chunk) store16(p.out + grow * p.ld + n, va, vb);
-      if (do_halo) {
-        // left context of the next conv block: hand the carried rows to the consumer, then shift
-        // the carry by T frames ([old carry | chunk] -> last 8 rows), all inside this CTA
-        if (is_halo) {
-          va = *reinterpret_cast<const uint4*>(carry + rho * p.C + n);
-          vb = *reinterpret_cast<const uint4*>(carry + rho * p.C + n + 8);
-          store16(p.out + grow * p.ld + n, va, vb);
-        }
-        ptx::named_bar_sync(1, 128);
-        if (carry_wr) store16(carry + new_row * p.C + n, va, vb);
-      }
+      // chunk rows store y; left-context rows hand the carried rows to the consumer of `out`
+      if (is_chunk || (is_halo && do_halo)) store16(p.out + grow * p.ld + n, va, vb);
+      // shift the carry by T frames: [old carry | chunk] -> its last 8 rows
+      if (carry_wr) store16(carry + new_row * p.C + n, va, vb);
+      if (threadIdx.x == 96 && kk == 0) DC_T(6);
+      if (threadIdx.x == 96 && kk == 1) DC_T(7);
     }
   }
+  if (threadIdx.x == 96) DC_T(5);
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 1) ptx::tmem_dealloc(tmem_base, tmem_cols);
+#ifdef DC_TIMING
+  if (tm && threadIdx.x == 0)
+    printf("T setup %lld tma_issued %lld first_full %lld mma_issued %lld accum_ready %lld ch0 %lld ch1 %lld epi_done %lld end %lld\n", s_t[0], s_t[1],
+           s_t[2], s_t[3], s_t[4], s_t[6], s_t[7], s_t[5], clock64() - t_start);
+  if (tm && threadIdx.x == 0) {
+    printf("K full:");
+    for (int i = 0; i < p.n_kblocks && i < 32; ++i) printf(" %lld", s_k[i]);
+    printf("\nK prod:");
+    for (int i = 0; i < p.n_kblocks && i < 32; ++i) printf(" %lld", s_p[i]);
+    printf("\n");
+  }
+#endif
 }
 
 // ---- small kernels ---------------------------------------------------------------------------
@@ -586,7 +685,7 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, u
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr size_t GEMM_SMEM = 1024 + STAGES * A_BYTES + STAGES * MAX_BN * 128 + 256;
+constexpr size_t GEMM_SMEM = 1024 + GEMM_TILE_SMEM + 2 * MAX_STAGES * 8 + 8 + 8 + 2 * MAX_BN * 4 + 64;
 
 }  // namespace
 
@@ -780,11 +879,11 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   }
 
   bool ok = true;
-  ok &= make_tmap(&m->tmAin, m->Ain, R, m->Kin, TILE_M);
-  ok &= make_tmap(&m->tmXa, m->Xa, R, C, TILE_M);
-  ok &= make_tmap(&m->tmXb, m->Xb, R, C, TILE_M);
-  ok &= make_tmap(&m->tmU, m->U, R, C, TILE_M);
-  ok &= make_tmap(&m->tmO, m->O, R, C, TILE_M);
+  ok &= make_tmap(&m->tmAin, m->Ain, R, m->Kin, A_ROWS);
+  ok &= make_tmap(&m->tmXa, m->Xa, R, C, A_ROWS);
+  ok &= make_tmap(&m->tmXb, m->Xb, R, C, A_ROWS);
+  ok &= make_tmap(&m->tmU, m->U, R, C, A_ROWS);
+  ok &= make_tmap(&m->tmO, m->O, R, C, A_ROWS);
   ok &= make_tmap(&m->tmWin, m->wts + w_in, C, m->Kin, 64);
   ok &= make_tmap(&m->tmWout, m->wts + w_out, mel, C, mel);
   m->tmWconv.resize(nL);
@@ -894,6 +993,14 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
     p.C = C;
     p.Rk = m->Rk;
     p.err = m->d_err;
+    {
+      const int stage_bytes = A_BYTES + p.taps * ((p.BN * 128 + 1023) & ~1023);
+      p.n_stages = std::min(MAX_STAGES, GEMM_TILE_SMEM / stage_bytes);
+      const char* d = getenv("DC_GEMM_DBG");
+      p.dbg = d ? atoi(d) : 0;
+      const char* e = getenv("DC_GEMM_STAGES");   // experiments only
+      if (e && atoi(e) >= 1 && atoi(e) < p.n_stages) p.n_stages = atoi(e);
+    }
     dim3 grid(m_tiles, N / p.BN);
     ProfScope ps(m->prof, p.mode == MODE_CONV ? 0 : 1, st);
     flow_gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(tA, tB, p);
@@ -916,7 +1023,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
     auto swap = [&]() { std::swap(X, Y); std::swap(tX, tY); };
     {
       GemmParams p{};
-      p.mode = MODE_INPROJ; p.BN = 64; p.n_kblocks = m->Kin / KBLK; p.kb_per_tap = p.n_kblocks;
+      p.mode = MODE_INPROJ; p.BN = 64; p.n_kblocks = m->Kin / KBLK; p.taps = 1;
       p.bias = fc + m->o_bin; p.out = X;
       p.halo_off = ((long long)s * c.n_conv + 0) * halo_stride;
       gemm(m->tmAin, m->tmWin, p, C);
@@ -927,7 +1034,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       for (int j = 0; j < m->cpa; ++j, ++l) {
         const int d = c.dilations[l];
         GemmParams p{};
-        p.mode = MODE_CONV; p.BN = 64; p.kb_per_tap = C / KBLK; p.n_kblocks = 3 * p.kb_per_tap;
+        p.mode = MODE_CONV; p.BN = 64; p.n_kblocks = C / KBLK; p.taps = 3;
         p.shift[0] = 2 * d; p.shift[1] = d; p.shift[2] = 0;
         p.bias = fc + m->o_bconv[l]; p.tau = fc + m->o_tau + ((size_t)s * c.n_conv + l) * C;
         p.resid = X; p.out = Y;
@@ -940,7 +1047,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
         rmsnorm(X);
         {
           GemmParams p{};
-          p.mode = MODE_QKV; p.BN = 64; p.n_kblocks = C / KBLK; p.kb_per_tap = p.n_kblocks;
+          p.mode = MODE_QKV; p.BN = 64; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bqkv[g]; p.q_out = m->Q; p.halo_off = -1;
           p.kv_off = ((long long)s * c.n_attn + g) * 2 * m->Rk * C;
           gemm(m->tmU, m->tmWqkv[g], p, 3 * C);
@@ -949,7 +1056,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
         ++*launches;
         {
           GemmParams p{};
-          p.mode = MODE_OPROJ; p.BN = 64; p.n_kblocks = C / KBLK; p.kb_per_tap = p.n_kblocks;
+          p.mode = MODE_OPROJ; p.BN = 64; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bo[g]; p.resid = X; p.out = Y;
           p.halo_off = (l < c.n_conv) ? ((long long)s * c.n_conv + l) * halo_stride : -1;
           gemm(m->tmO, m->tmWo[g], p, C);
@@ -960,7 +1067,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
     rmsnorm(X);
     {
       GemmParams p{};
-      p.mode = MODE_OUT; p.BN = mel; p.n_kblocks = C / KBLK; p.kb_per_tap = p.n_kblocks;
+      p.mode = MODE_OUT; p.BN = mel; p.n_kblocks = C / KBLK; p.taps = 1;
       p.bias = fc + m->o_bout; p.halo_off = -1;
       p.xstate = m->xstate; p.ain = m->Ain; p.ld_ain = m->Kin; p.inv_n = 1.0f / c.n_steps;
       p.last_step = (s == c.n_steps - 1); p.mel = mel;

@@ -49,6 +49,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return false;
 }
 
+// Same bound, but the waiter sleeps between polls: for the many threads that wait for a whole
+// main loop, so that their polling does not compete with the issuing warps for issue slots and
+// shared-memory bandwidth.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kMaxPolls; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(100);
+  }
+  return false;
+}
+
 // ---- fences -----------------------------------------------------------------------------------
 // generic-proxy smem writes -> visible to the async proxy (UMMA / TMA reads)
 __device__ __forceinline__ void fence_proxy_async_smem() {
