@@ -446,17 +446,28 @@ __global__ void flow_rmsnorm_kernel(const SlotInfo* slots, int n_slots, const bf
 
 
 // ---- chunk-causal attention with the K/V carry ---------------------------------------------------
-// One CTA per (stream slot, head).  Queries: the T chunk frames (padded to the 128 UMMA rows).
-// Keys/values: the kv_len carried frames followed by the chunk's own T frames, read in place
-// from the stream's ring with 128-bit loads (the ring may wrap; nothing is compacted or copied
-// in global memory).  Two passes over the keys in blocks of 128, both on tcgen05:
-//   pass 1: S = Q K^T per block -> row maximum;
-//   pass 2: S again, e = exp(scale (S - max)), row sum from the unrounded e, P = bf16(e) written to
-//           shared memory as the A operand of O += P V (V is the MN-major B operand).
-// One thread owns one query row (= one TMEM lane), so the softmax needs no cross-thread traffic.
-constexpr int ATT_THREADS = 128;
-constexpr int ATT_KB = 128;     // keys per block
-constexpr int ATT_TMEM_COLS = 512;  // S double buffer (2 x 128) + O (64)
+// One CTA per (stream slot, head), two CTAs per SM.  Queries: the T <= 56 chunk frames (rows 0..63
+// of the 128 UMMA rows; rows 64..127 are never read back).  Keys/values: the kv_len carried frames
+// followed by the chunk's own T frames, streamed in place from the stream's ring in blocks of 128
+// keys with 128-bit cp.async loads (the ring may wrap; nothing is compacted or copied in global
+// memory) through a two-stage shared-memory ring.
+//
+// Warp roles (8 warps): warps 0,1,4,5 = softmax (thread = (query row, half of the block's 128 key
+// columns)); warp 3 = UMMA issuer; warps 2,6,7 = K/V/Q loaders.
+// Per key block: S = Q K^T on tcgen05 (accumulator in TMEM) -> the softmax threads read their
+// columns, e = exp2(scale*S - m) with a running reference m that is only raised when the block
+// maximum exceeds it by more than 2^8 (then O and the row sum are rescaled once), row sum from the
+// unrounded e, P = bf16(e) into shared memory -> O += P V on tcgen05 (V is the MN-major operand).
+constexpr int ATT_THREADS = 256;
+constexpr int ATT_KB = 128;             // keys per block
+constexpr int ATT_STAGES = 2;
+constexpr int ATT_TMEM_COLS = 256;      // S (128 columns) + O (64 columns); two CTAs share the SM's 512
+constexpr int ATT_LOADERS = 96;
+constexpr int ATT_Q_BYTES = 64 * 128;   // 64 query rows; the UMMA's rows 64..127 alias the P region
+constexpr int ATT_P_BYTES = 2 * 64 * 128;
+constexpr int ATT_STAGE_BYTES = 2 * ATT_KB * 128;   // K block + V block
+constexpr size_t ATT_SMEM = 1024 + ATT_Q_BYTES + ATT_P_BYTES + ATT_STAGES * ATT_STAGE_BYTES + 1024;
+constexpr float ATT_RESCALE_LOG2 = 8.0f;
 
 struct AttnParams {
   const SlotInfo* slots;
@@ -466,7 +477,6 @@ struct AttnParams {
   int             dh;         // 32 or 64 (smem rows are padded to 64 columns)
   long long       kv_off;     // element offset of this (step, layer)'s K ring inside SlotInfo::kv
   int             Rk, C;
-  int             kv_rows_max;  // smem rows reserved for K and for V (multiple of 128)
   float           scale_log2e;  // log2(e) / sqrt(dh)
   int*            err;
 };
@@ -475,18 +485,21 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(dst)), "l"(src) : "memory");
 }
 
-__global__ void __launch_bounds__(ATT_THREADS, 1) flow_attn_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;                       // [128][128 B]
-  uint8_t* sP = sQ + 128 * 128;             // 2 tiles of [128][128 B]
-  uint8_t* sK = sP + 2 * 128 * 128;         // [kv_rows_max][128 B]
-  uint8_t* sV = sK + (size_t)p.kv_rows_max * 128;
-  uint64_t* bar_s = reinterpret_cast<uint64_t*>(sV + (size_t)p.kv_rows_max * 128);   // [2]
-  uint64_t* bar_pv = bar_s + 2;
+  uint8_t* sQ = smem;
+  uint8_t* sP = sQ + ATT_Q_BYTES;                    // tile t (keys 64 t .. 64 t + 63 of the block) at + 8192 t
+  uint8_t* ring = sP + ATT_P_BYTES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(ring + ATT_STAGES * ATT_STAGE_BYTES);   // [ATT_STAGES]
+  uint64_t* empty = full + ATT_STAGES;
+  uint64_t* bar_s = empty + ATT_STAGES;
+  uint64_t* bar_p = bar_s + 1;
+  uint64_t* bar_pv = bar_p + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_pv + 1);
+  float* s_x = reinterpret_cast<float*>(tmem_slot + 2);   // [2][64] exchange between the two column halves
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int slot = blockIdx.x, head = blockIdx.y;
   const SlotInfo si = p.slots[slot];
   const int T = si.T, L = si.kv_len + T;
@@ -494,19 +507,27 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) flow_attn_kernel(const AttnPar
   const int chunks = p.dh >> 3;             // 16-byte chunks per head row
 
   if (tid == 0) {
-    ptx::mbar_init(&bar_s[0], 1);
-    ptx::mbar_init(&bar_s[1], 1);
+    for (int i = 0; i < ATT_STAGES; ++i) {
+      ptx::mbar_init(&full[i], ATT_LOADERS);
+      ptx::mbar_init(&empty[i], 1);
+    }
+    ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_p, 128);
     ptx::mbar_init(bar_pv, 1);
     ptx::fence_barrier_init();
   }
-  __syncwarp();
-  if (warp == 0) ptx::tmem_alloc(tmem_slot, ATT_TMEM_COLS);
+  if (warp == 3) ptx::tmem_alloc(tmem_slot, ATT_TMEM_COLS);
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
 
-  // ---- stage Q, K, V into 128-byte-swizzled shared memory ----
-  {
+  if (warp == 2 || warp >= 6) {
+    // ---------------- loaders ----------------
+    const int lt = (warp == 2 ? 0 : (warp - 5) * 32) + lane;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
     const bf16* qbase = p.q + (long long)(GUARD + slot * SLOT_ROWS + HALO) * p.ld + head * p.dh;
-    for (int i = tid; i < 128 * 8; i += ATT_THREADS) {
+    for (int i = lt; i < 64 * 8; i += ATT_LOADERS) {
       const int row = i >> 3, j = i & 7;
       uint8_t* dst = sQ + row * 128 + ((j ^ (row & 7)) << 4);
       if (row < T && j < chunks) cp_async16(dst, qbase + (long long)row * p.ld + j * 8);
@@ -516,129 +537,154 @@ __global__ void __launch_bounds__(ATT_THREADS, 1) flow_attn_kernel(const AttnPar
     const bf16* vbase = kbase + (long long)p.Rk * p.C;
     int start = si.kv_head - si.kv_len;
     if (start < 0) start += p.Rk;
-    for (int i = tid; i < nkb * ATT_KB * 8; i += ATT_THREADS) {
-      const int row = i >> 3, j = i & 7;
-      const int off = row * 128 + ((j ^ (row & 7)) << 4);
-      if (row < L && j < chunks) {
-        int rr = start + row;
-        if (rr >= p.Rk) rr -= p.Rk;
-        cp_async16(sK + off, kbase + (long long)rr * p.C + j * 8);
-        cp_async16(sV + off, vbase + (long long)rr * p.C + j * 8);
-      } else {
-        *reinterpret_cast<uint4*>(sK + off) = zero;
-        *reinterpret_cast<uint4*>(sV + off) = zero;
+    bool ok = true;
+    for (int b = 0; b < nkb; ++b) {
+      const int st = b % ATT_STAGES;
+      if (b >= 1) {   // the previous block has been issued a whole iteration ago: publish it
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        ptx::fence_proxy_async_smem();
+        ptx::mbar_arrive(&full[(b - 1) % ATT_STAGES]);
+      }
+      if (b >= ATT_STAGES && ok && !ptx::mbar_wait_relaxed(&empty[st], ((b / ATT_STAGES) - 1) & 1)) {
+        ok = false;
+        atomicExch(p.err, 4);
+      }
+      uint8_t* sK = ring + st * ATT_STAGE_BYTES;
+      uint8_t* sV = sK + ATT_KB * 128;
+      for (int i = lt; i < ATT_KB * 8; i += ATT_LOADERS) {
+        const int row = i >> 3, j = i & 7;
+        const int key = b * ATT_KB + row;
+        const int off = row * 128 + ((j ^ (row & 7)) << 4);
+        if (key < L && j < chunks) {
+          int rr = start + key;
+          if (rr >= p.Rk) rr -= p.Rk;
+          cp_async16(sK + off, kbase + (long long)rr * p.C + j * 8);
+          cp_async16(sV + off, vbase + (long long)rr * p.C + j * 8);
+        } else {
+          *reinterpret_cast<uint4*>(sK + off) = zero;
+          *reinterpret_cast<uint4*>(sV + off) = zero;   // 0 * garbage must not poison O
+        }
       }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     ptx::fence_proxy_async_smem();
-  }
-  ptx::tc_fence_before();
-  __syncthreads();
-  ptx::tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
-  const uint32_t idesc_s = ptx::umma_idesc_bf16(128, ATT_KB, 0, 0);
-  const uint32_t idesc_pv = ptx::umma_idesc_bf16(128, 64, 0, 1);   // B = V, MN-major
-  const uint32_t q_addr = ptx::smem_u32(sQ), k_addr = ptx::smem_u32(sK), v_addr = ptx::smem_u32(sV), p_addr = ptx::smem_u32(sP);
-
-  auto issue_s = [&](int kb) {   // S[kb & 1] = Q K_kb^T
-    const uint32_t d = tmem_base + (uint32_t)((kb & 1) * ATT_KB);
+    ptx::mbar_arrive(&full[(nkb - 1) % ATT_STAGES]);
+  } else if (warp == 3) {
+    // ---------------- UMMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc_s = ptx::umma_idesc_bf16(128, ATT_KB, 0, 0);
+      const uint32_t idesc_pv = ptx::umma_idesc_bf16(128, 64, 0, 1);   // B = V, MN-major
+      const uint64_t dq = ptx::umma_desc_sw128(ptx::smem_u32(sQ));
+      const uint64_t dp = ptx::umma_desc_sw128(ptx::smem_u32(sP));
+      bool ok = true;
+      for (int b = 0; b < nkb; ++b) {
+        const int st = b % ATT_STAGES;
+        if (ok && !ptx::mbar_wait(&full[st], (b / ATT_STAGES) & 1)) { ok = false; atomicExch(p.err, 5); }
+        ptx::tc_fence_after();
+        const uint64_t dk = ptx::umma_desc_sw128(ptx::smem_u32(ring + st * ATT_STAGE_BYTES));
+        const uint64_t dv = ptx::umma_desc_sw128(ptx::smem_u32(ring + st * ATT_STAGE_BYTES + ATT_KB * 128));
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
-      ptx::umma_bf16(d, ptx::umma_desc_sw128(q_addr + k * 32), ptx::umma_desc_sw128(k_addr + kb * ATT_KB * 128 + k * 32),
-                     idesc_s, k != 0);
-    ptx::umma_commit(&bar_s[kb & 1]);
-  };
-
-  bool ok = true;
-  uint32_t n_s[2] = {0u, 0u};    // completed waits per S buffer (phase parity)
-  float mrow = -INFINITY;
-  // ---- pass 1: row maximum ----
-  if (tid == 0) issue_s(0);
-  for (int kb = 0; kb < nkb; ++kb) {
-    if (tid == 0 && kb + 1 < nkb) issue_s(kb + 1);
-    const int b = kb & 1;
-    if (ok && !ptx::mbar_wait(&bar_s[b], n_s[b] & 1)) { ok = false; atomicExch(p.err, 4); }
-    ++n_s[b];
-    ptx::tc_fence_after();
-    const int valid = L - kb * ATT_KB;
-    for (int c0 = 0; c0 < ATT_KB; c0 += 16) {
-      float v[16];
-      ptx::tmem_ld16(lane_addr + (uint32_t)(b * ATT_KB + c0), v);
-#pragma unroll
-      for (int i = 0; i < 16; ++i)
-        if (c0 + i < valid) mrow = fmaxf(mrow, v[i]);
-    }
-    ptx::tc_fence_before();
-    __syncthreads();
-    ptx::tc_fence_after();
-  }
-  // ---- pass 2: numerators, row sum, O += P V ----
-  float lsum = 0.f;
-  uint32_t n_pv = 0;
-  const float mscaled = mrow * p.scale_log2e;
-  if (tid == 0) issue_s(0);
-  for (int kb = 0; kb < nkb; ++kb) {
-    if (tid == 0 && kb + 1 < nkb) issue_s(kb + 1);
-    const int b = kb & 1;
-    if (ok && !ptx::mbar_wait(&bar_s[b], n_s[b] & 1)) { ok = false; atomicExch(p.err, 5); }
-    ++n_s[b];
-    if (kb > 0) {   // the previous P V must have consumed the P tile before it is overwritten
-      if (ok && !ptx::mbar_wait(bar_pv, n_pv & 1)) { ok = false; atomicExch(p.err, 6); }
-      ++n_pv;
-    }
-    ptx::tc_fence_after();
-    const int valid = L - kb * ATT_KB;
-    for (int c0 = 0; c0 < ATT_KB; c0 += 16) {
-      float v[16];
-      ptx::tmem_ld16(lane_addr + (uint32_t)(b * ATT_KB + c0), v);
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const float e = (c0 + i < valid) ? exp2f(fmaf(v[i], p.scale_log2e, -mscaled)) : 0.f;
-        lsum += e;
-        v[i] = e;
+        for (int k = 0; k < 4; ++k) ptx::umma_bf16(tmem_base, dq + 2 * k, dk + 2 * k, idesc_s, k != 0);
+        ptx::umma_commit(bar_s);
+        if (ok && !ptx::mbar_wait(bar_p, b & 1)) { ok = false; atomicExch(p.err, 6); }
+        ptx::tc_fence_after();
+        const int valid = L - b * ATT_KB;
+        const int ksteps = valid >= ATT_KB ? ATT_KB / 16 : (valid + 15) / 16;
+        for (int k = 0; k < ksteps; ++k)   // P tile k/4 (8 KB apart), 32-byte K steps; V: 16 key rows = 2 KB per step
+          ptx::umma_bf16(tmem_base + ATT_KB, dp + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
+                         idesc_pv, (b | k) != 0);
+        ptx::umma_commit(&empty[st]);
+        ptx::umma_commit(bar_pv);
       }
-      uint4 a, bq;
-      pack16_bf16(v, a, bq);
-      // key columns c0..c0+15 -> tile c0/64, 16-byte chunks (c0 % 64)/8 and +1 of row `tid`
-      uint8_t* prow = sP + (c0 >> 6) * (128 * 128) + tid * 128;
-      const int j0 = (c0 & 63) >> 3;
-      *reinterpret_cast<uint4*>(prow + (((j0) ^ (tid & 7)) << 4)) = a;
-      *reinterpret_cast<uint4*>(prow + (((j0 + 1) ^ (tid & 7)) << 4)) = bq;
     }
-    ptx::fence_proxy_async_smem();
-    ptx::tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
+  } else {
+    // ---------------- softmax: warps 0,1,4,5 ----------------
+    const int quarter = warp & 1;               // TMEM lanes 32*quarter .. (warp % 4 == quarter)
+    const int half = warp >> 2;                 // key columns 64*half .. of each block
+    const int row = quarter * 32 + lane;        // query row
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    bool ok = true;
+    float m_ref = -INFINITY, lsum = 0.f;
+    for (int b = 0; b < nkb; ++b) {
+      if (ok && !ptx::mbar_wait(bar_s, b & 1)) { ok = false; atomicExch(p.err, 7); }
       ptx::tc_fence_after();
-      const int ksteps = valid >= ATT_KB ? ATT_KB / 16 : (valid + 15) / 16;
-      const uint32_t d = tmem_base + 2 * ATT_KB;
-      for (int k = 0; k < ksteps; ++k)
-        ptx::umma_bf16(d, ptx::umma_desc_sw128(p_addr + (k >> 2) * (128 * 128) + (k & 3) * 32),
-                       ptx::umma_desc_sw128(v_addr + (kb * ATT_KB + k * 16) * 128), idesc_pv, (kb | k) != 0);
-      ptx::umma_commit(bar_pv);
-    }
-  }
-  if (ok && !ptx::mbar_wait(bar_pv, n_pv & 1)) { ok = false; atomicExch(p.err, 7); }
-  ptx::tc_fence_after();
-  {
-    const float inv = 1.0f / lsum;
-    bf16* orow = p.o + (long long)(GUARD + slot * SLOT_ROWS + HALO + tid) * p.ld + head * p.dh;
-    for (int c0 = 0; c0 < p.dh; c0 += 16) {
-      float v[16];
-      ptx::tmem_ld16(lane_addr + (uint32_t)(2 * ATT_KB + c0), v);
-      if (tid < T && ok) {
+      const int valid = L - b * ATT_KB - half * 64;   // columns of this half that are real keys
+      float v[64];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] *= inv;
+      for (int c = 0; c < 4; ++c) ptx::tmem_ld16(lane_addr + (uint32_t)(half * 64 + c * 16), v + 16 * c);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 64; ++i) {
+        v[i] = (i < valid) ? v[i] * p.scale_log2e : -INFINITY;
+        mx = fmaxf(mx, v[i]);
+      }
+      s_x[half * 64 + row] = mx;
+      ptx::named_bar_sync(2, 128);
+      mx = fmaxf(s_x[row], s_x[64 + row]);
+      if (b > 0) {   // P V of the previous block must be done: P tile free, O quiescent
+        if (ok && !ptx::mbar_wait(bar_pv, (b - 1) & 1)) { ok = false; atomicExch(p.err, 8); }
+        ptx::tc_fence_after();
+      }
+      if (b == 0) {
+        m_ref = mx;
+      } else {
+        const bool need = mx > m_ref + ATT_RESCALE_LOG2;
+        if (__any_sync(0xffffffffu, need)) {
+          const float alpha = need ? exp2f(m_ref - mx) : 1.0f;
+          if (need) m_ref = mx;
+          lsum *= alpha;
+          const int ncol = p.dh >> 1;             // O columns owned by this half
+          for (int c = 0; c < ncol; c += 16) {
+            float o16[16];
+            const uint32_t addr = lane_addr + (uint32_t)(ATT_KB + half * ncol + c);
+            ptx::tmem_ld16(addr, o16);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o16[i] *= alpha;
+            ptx::tmem_st16(addr, o16);
+          }
+        }
+      }
+      uint8_t* prow = sP + half * 8192 + row * 128;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float e[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          e[i] = exp2f(v[16 * c + i] - m_ref);
+          lsum += e[i];
+        }
         uint4 a, bq;
-        pack16_bf16(v, a, bq);
-        store16(orow + c0, a, bq);
+        pack16_bf16(e, a, bq);
+        *reinterpret_cast<uint4*>(prow + (((2 * c) ^ (row & 7)) << 4)) = a;
+        *reinterpret_cast<uint4*>(prow + (((2 * c + 1) ^ (row & 7)) << 4)) = bq;
+      }
+      ptx::fence_proxy_async_smem();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(bar_p);
+    }
+    if (ok && !ptx::mbar_wait(bar_pv, (nkb - 1) & 1)) { ok = false; atomicExch(p.err, 9); }
+    ptx::tc_fence_after();
+    ptx::named_bar_sync(2, 128);       // every thread is past its last read of s_x
+    s_x[half * 64 + row] = lsum;
+    ptx::named_bar_sync(2, 128);
+    const float inv = 1.0f / (s_x[row] + s_x[64 + row]);
+    const int ncol = p.dh >> 1;
+    bf16* orow = p.o + (long long)(GUARD + slot * SLOT_ROWS + HALO + row) * p.ld + head * p.dh + half * ncol;
+    for (int c = 0; c < ncol; c += 16) {
+      float o16[16];
+      ptx::tmem_ld16(lane_addr + (uint32_t)(ATT_KB + half * ncol + c), o16);
+      if (row < T && ok) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) o16[i] *= inv;
+        uint4 a, bq;
+        pack16_bf16(o16, a, bq);
+        store16(orow + c, a, bq);
       }
     }
   }
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 0) ptx::tmem_dealloc(tmem_base, ATT_TMEM_COLS);
+  if (warp == 3) ptx::tmem_dealloc(tmem_base, ATT_TMEM_COLS);
 }
 
 // ---- host helpers ----------------------------------------------------------------------------
@@ -695,8 +741,7 @@ constexpr size_t GEMM_SMEM = 1024 + GEMM_TILE_SMEM + 2 * MAX_STAGES * 8 + 8 + 8 
 
 struct FlowModel {
   dc_config cfg;
-  int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0, kv_rows_max = 0;
-  size_t attn_smem = 0;
+  int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0;
   bf16 *Xa = nullptr, *Xb = nullptr, *U = nullptr, *Q = nullptr, *O = nullptr, *Ain = nullptr;
   float* xstate = nullptr;
   bf16*  wts = nullptr;
@@ -754,13 +799,6 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   m->rows = ((m->S * SLOT_ROWS + TILE_M - 1) / TILE_M) * TILE_M;
   m->Rk = cfg.kv_cap + cfg.f_chunk;
   m->cpa = cfg.n_attn > 0 ? cfg.n_conv / cfg.n_attn : cfg.n_conv;
-  m->kv_rows_max = ((m->Rk + ATT_KB - 1) / ATT_KB) * ATT_KB;
-  m->attn_smem = 1024 + 3 * 128 * 128 + 2 * (size_t)m->kv_rows_max * 128 + 64;
-  if (cfg.n_attn > 0 && m->attn_smem > 227 * 1024) {
-    set_error("kv_cap + f_chunk = %d key rows do not fit the attention kernel's shared memory", m->Rk);
-    delete m;
-    return DC_ERR_CONFIG;
-  }
   const int nL = cfg.n_conv, nA = cfg.n_attn, nS = cfg.n_steps;
   const size_t R = (size_t)GUARD + m->rows;
 
@@ -871,7 +909,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   if (e == cudaSuccess)
     chk(cudaFuncSetAttribute(flow_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
   if (e == cudaSuccess && cfg.n_attn > 0)
-    chk(cudaFuncSetAttribute(flow_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m->attn_smem));
+    chk(cudaFuncSetAttribute(flow_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATT_SMEM));
   if (e != cudaSuccess) {
     set_error("flow model allocation failed: %s", cudaGetErrorString(e));
     flow_model_destroy(m);
@@ -1087,11 +1125,11 @@ void launch_flow_attention(FlowModel* m, int n, int step, int layer, cudaStream_
   AttnParams p{};
   p.slots = m->d_slots; p.q = m->Q; p.o = m->O; p.ld = m->C; p.dh = c.head_dim;
   p.kv_off = ((long long)step * c.n_attn + layer) * 2 * m->Rk * m->C;
-  p.Rk = m->Rk; p.C = m->C; p.kv_rows_max = m->kv_rows_max;
+  p.Rk = m->Rk; p.C = m->C;
   p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
   p.err = m->d_err;
   ProfScope ps(m->prof, 2, st);
-  flow_attn_kernel<<<dim3(n, c.n_heads), ATT_THREADS, m->attn_smem, st>>>(p);
+  flow_attn_kernel<<<dim3(n, c.n_heads), ATT_THREADS, ATT_SMEM, st>>>(p);
 }
 
 }  // namespace dc
