@@ -19,7 +19,9 @@
 #include <string.h>
 
 #include <algorithm>
+#include <map>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "dc_internal.h"
@@ -37,10 +39,11 @@ constexpr int HALO = 8;         // carried frames per (step, conv block); dilati
 constexpr int TILE_M = 128;
 constexpr int KBLK = 64;        // bf16 elements per 128-byte swizzled smem row
 constexpr int MAX_STAGES = 8;
-constexpr int GEMM_TILE_SMEM = 200 * 1024;   // bytes of operand stages per CTA
+constexpr int GEMM_TILE_SMEM = 88 * 1024;    // operand stages per CTA: small enough for two CTAs per SM, so that
+                                             // the next kernel's prologue and weight prefetch overlap this one's tail
 constexpr int A_ROWS = TILE_M + HALO;  // the A tile carries 8 extra leading rows so that all taps read it
 constexpr int A_BYTES = A_ROWS * 128;
-constexpr int MAX_BN = 128;
+constexpr int MAX_BN = 192;
 constexpr int GEMM_THREADS = 352;      // warp 0 TMA (A), warp 1 UMMA, warp 2 TMA (B), warps 3..10 epilogue
 constexpr int EPI_THREADS = 256;
 constexpr int MAX_SLOTS_PER_SET = 64;
@@ -119,7 +122,7 @@ __device__ __forceinline__ void store16(bf16* p, const uint4& a, const uint4& b)
   *reinterpret_cast<uint4*>(p + 8) = b;
 }
 
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
 flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -130,7 +133,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t b_tile = (b_bytes + 1023u) & ~1023u;
   const uint32_t stage_bytes = (uint32_t)A_BYTES + (uint32_t)p.taps * b_tile;
   const int STAGES = p.n_stages;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + GEMM_TILE_SMEM);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * stage_bytes);
   uint64_t* empty = full + MAX_STAGES;
   uint64_t* accum = empty + MAX_STAGES;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
@@ -151,7 +154,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #else
 #define DC_T(tag) do {} while (0)
 #endif
-  const uint32_t tmem_cols = p.BN <= 32 ? 32u : (p.BN <= 64 ? 64u : 128u);
+  const uint32_t tmem_cols = p.BN <= 32 ? 32u : (p.BN <= 64 ? 64u : (p.BN <= 128 ? 128u : 256u));
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
@@ -168,76 +171,101 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   if (threadIdx.x == 0) DC_T(0);
+  ptx::pdl_launch();   // the next kernel may start its prologue and its weight prefetch now
 
   if (warp == 0 || warp == 2) {
-    // two producer threads, one per tensor map: warp 0 streams the A tiles, warp 2 the weight tiles
-    if (lane == 0) {
+    // two producer threads, one per tensor map: warp 0 streams the A tiles, warp 2 the weight tiles.
+    // The loops keep their state in registers (no division, no parameter reloads): a single thread
+    // issues every copy, so its instruction count is what bounds the fill rate.
+    {
+      const uint32_t on = lane == 0;   // the whole warp runs the loop, lane 0 issues
       const bool is_a = warp == 0;
-      for (int kb = 0; kb < p.n_kblocks; ++kb) {
-        const int st = kb % STAGES;
-#ifdef DC_TIMING
-        if ((p.dbg & 4) && kb >= STAGES) break;
-#endif
-        if (kb >= STAGES && !ptx::mbar_wait(&empty[st], ((kb / STAGES) - 1) & 1)) {
+      const int nkb = p.n_kblocks, taps = p.taps;
+      const int ya = GUARD + m0 - HALO;
+      const uint32_t tx_bytes = is_a ? (uint32_t)A_BYTES : (uint32_t)taps * b_bytes;
+      uint8_t* dst = smem + (is_a ? 0 : A_BYTES);
+      int st = 0;
+      uint32_t phase = 1;          // parity of the "empty" phase to wait for (first pass: no wait)
+      int x = 0;
+      if (is_a) ptx::pdl_wait();   // activations come from the previous kernel; weights do not
+      for (int kb = 0; kb < nkb; ++kb) {
+        if (kb >= STAGES && !ptx::mbar_wait(&empty[st], phase)) {
           atomicExch(p.err, 1);
           *s_fail = 1;
           break;
         }
 #ifdef DC_TIMING
-        if (tm && kb < 32 && is_a) s_p[kb] = clock64() - t_start;
+        if (tm && kb < 32 && is_a && on) s_p[kb] = clock64() - t_start;
 #endif
+        ptx::mbar_expect_tx_if(on, &full[st], tx_bytes);
         if (is_a) {
-          ptx::mbar_expect_tx(&full[st], (uint32_t)A_BYTES);
-          ptx::tma_load_2d(smem + st * stage_bytes, &tmA, kb * KBLK, GUARD + m0 - HALO, &full[st]);
+          ptx::tma_load_2d_if(on, dst, &tmA, x, ya, &full[st]);
         } else {
-          ptx::mbar_expect_tx(&full[st], (uint32_t)p.taps * b_bytes);
-          for (int j = 0; j < p.taps; ++j)
-            ptx::tma_load_2d(smem + st * stage_bytes + A_BYTES + j * b_tile, &tmB, (j * p.n_kblocks + kb) * KBLK, n0, &full[st]);
-        }
-      }
-      if (is_a) DC_T(1);
-    }
-  } else if (warp == 1) {
-    if (lane == 0) {
-      const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.BN, 0, 0);
-      bool ok = true;
-      for (int kb = 0; kb < p.n_kblocks && ok; ++kb) {
-        const int st = kb % STAGES;
-#ifdef DC_TIMING
-        if ((p.dbg & 4) && kb >= STAGES) goto skip_wait;
-#endif
-        if (!ptx::mbar_wait(&full[st], (kb / STAGES) & 1)) {
-          atomicExch(p.err, 2);
-          *s_fail = 1;
-          ok = false;
-          break;
-        }
-#ifdef DC_TIMING
-      skip_wait:
-#endif
-        ptx::tc_fence_after();
-        if (kb == 0) DC_T(2);
-#ifdef DC_TIMING
-        if (tm && kb < 32) s_k[kb] = clock64() - t_start;
-#endif
-        const uint32_t a0 = ptx::smem_u32(smem + st * stage_bytes), b0 = a0 + A_BYTES;
-        for (int j = 0; j < p.taps; ++j) {
-          // descriptors differ only in the 16-byte-unit start address (low bits): +2 per 32-byte K step
-          const uint64_t da = ptx::umma_desc_sw128(a0 + (uint32_t)(HALO - p.shift[j]) * 128u);
-          const uint64_t db = ptx::umma_desc_sw128(b0 + (uint32_t)j * b_tile);
-#pragma unroll
-          for (int k = 0; k < KBLK / 16; ++k) {
-#ifdef DC_TIMING
-            if ((p.dbg & 1) && k != 0) continue;
-            if ((p.dbg & 2) && (k != 0 || j != 0)) continue;
-#endif
-            ptx::umma_bf16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | j | k) != 0);
+          ptx::tma_load_2d_if(on, dst, &tmB, x, n0, &full[st]);
+          if (taps == 3) {
+            ptx::tma_load_2d_if(on, dst + b_tile, &tmB, x + nkb * KBLK, n0, &full[st]);
+            ptx::tma_load_2d_if(on, dst + 2 * b_tile, &tmB, x + 2 * nkb * KBLK, n0, &full[st]);
           }
         }
-        ptx::umma_commit(&empty[st]);
+        x += KBLK;
+        dst += stage_bytes;
+        if (++st == STAGES) {
+          st = 0;
+          dst -= (size_t)STAGES * stage_bytes;
+          phase ^= 1;
+        }
       }
-      DC_T(3);
-      ptx::umma_commit(accum);   // arrives when every UMMA above has finished (also on the failure path)
+      if (is_a && on) DC_T(1);
+    }
+  } else if (warp == 1) {
+    {
+      const uint32_t on = lane == 0;
+      const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.BN, 0, 0);
+      const int nkb = p.n_kblocks, taps = p.taps;
+      // descriptor start addresses are in 16-byte units: +2 per 32-byte K step
+      const uint64_t d_a0 = ptx::umma_desc_sw128(ptx::smem_u32(smem));
+      const uint32_t stage16 = stage_bytes >> 4, b16 = b_tile >> 4, ab16 = A_BYTES >> 4;
+      const uint32_t o0 = (uint32_t)(HALO - p.shift[0]) * 8u, o1 = (uint32_t)(HALO - p.shift[1]) * 8u,
+                     o2 = (uint32_t)(HALO - p.shift[2]) * 8u;   // row offset of tap j: rows * 128 B / 16
+      int st = 0;
+      uint32_t phase = 0, acc = 0;
+      uint64_t d_st = d_a0;
+      for (int kb = 0; kb < nkb; ++kb) {
+        if (!ptx::mbar_wait(&full[st], phase)) {
+          atomicExch(p.err, 2);
+          *s_fail = 1;
+          break;
+        }
+        ptx::tc_fence_after();
+        if (kb == 0 && on) DC_T(2);
+#ifdef DC_TIMING
+        if (tm && kb < 32 && on) s_k[kb] = clock64() - t_start;
+#endif
+        const uint64_t da = d_st, db = d_st + ab16;
+        if (taps == 3) {
+          ptx::umma_bf16_if(on, tmem_base, da + o0, db, idesc, acc);
+#pragma unroll
+          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, tmem_base, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, tmem_base, da + (o1 + 2 * k), db + (b16 + 2 * k), idesc, 1);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, tmem_base, da + (o2 + 2 * k), db + (2 * b16 + 2 * k), idesc, 1);
+        } else {
+          ptx::umma_bf16_if(on, tmem_base, da + o0, db, idesc, acc);
+#pragma unroll
+          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, tmem_base, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
+        }
+        acc = 1;
+        ptx::umma_commit_if(on, &empty[st]);
+        d_st += stage16;
+        if (++st == STAGES) {
+          st = 0;
+          d_st = d_a0;
+          phase ^= 1;
+        }
+      }
+      if (on) DC_T(3);
+      ptx::umma_commit_if(on, accum);   // arrives when every UMMA above has finished (also on the failure path)
     }
   } else {
     // ---------------- epilogue: 8 warps; a thread owns one output row and every other 16-column chunk ----------------
@@ -245,10 +273,11 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // per-column constants go to shared memory, the thread's residual row (or, for a left-context
     // row, the carried row) goes to registers.
     const int et = threadIdx.x - 96;
-    if (et < p.BN) {   // BN <= 128 < EPI_THREADS
+    if (et < p.BN) {   // BN <= 192 < EPI_THREADS
       s_bias[et] = p.bias[n0 + et];
       s_tau[et] = p.tau != nullptr ? p.tau[n0 + et] : 0.f;
     }
+    ptx::pdl_wait();                              // slot table, residual and carry rows are upstream data
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int half = (warp - 3) >> 2;             // which chunks of the row: chunk index & 1 == half
     const int r = m0 + q * 32 + lane;             // row in slot layout (without GUARD)
@@ -391,12 +420,15 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // ---- small kernels ---------------------------------------------------------------------------
 
 __global__ void set_slots_kernel(const SlotSet set, SlotInfo* dst) {
+  ptx::pdl_launch();
   const int i = threadIdx.x;
   if (i < set.count) dst[set.first + i] = set.s[i];
 }
 
 // feats [T][2 mel] -> Euler state x_0 (fp32) and the bf16 input-projection operand [x_0 | mu].
 __global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, bf16* ain, int ld_ain) {
+  ptx::pdl_launch();
+  ptx::pdl_wait();
   const SlotInfo si = slots[blockIdx.x];
   for (int i = threadIdx.x; i < si.T * mel; i += blockDim.x) {
     const int f = i / mel, c = i - f * mel;
@@ -411,6 +443,8 @@ __global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, 
 
 // u = bf16(x * rsqrt(mean(x^2) + eps)), one warp per chunk row.
 __global__ void flow_rmsnorm_kernel(const SlotInfo* slots, int n_slots, const bf16* x, bf16* u, int C, float eps) {
+  ptx::pdl_launch();
+  ptx::pdl_wait();
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   const int slot = warp / SLOT_ROWS, rho = warp % SLOT_ROWS;
   if (slot >= n_slots) return;
@@ -501,9 +535,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int slot = blockIdx.x, head = blockIdx.y;
-  const SlotInfo si = p.slots[slot];
-  const int T = si.T, L = si.kv_len + T;
-  const int nkb = (L + ATT_KB - 1) / ATT_KB;
   const int chunks = p.dh >> 3;             // 16-byte chunks per head row
 
   if (tid == 0) {
@@ -521,6 +552,11 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  ptx::pdl_launch();
+  ptx::pdl_wait();      // the slot table, Q and the appended K/V rows come from earlier kernels
+  const SlotInfo si = p.slots[slot];
+  const int T = si.T, L = si.kv_len + T;
+  const int nkb = (L + ATT_KB - 1) / ATT_KB;
 
   if (warp == 2 || warp >= 6) {
     // ---------------- loaders ----------------
@@ -739,6 +775,14 @@ constexpr size_t GEMM_SMEM = 1024 + GEMM_TILE_SMEM + 2 * MAX_STAGES * 8 + 8 + 8 
 // engine
 // ---------------------------------------------------------------------------------------------
 
+struct GraphEntry {
+  cudaGraph_t     graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  cudaGraphNode_t set_node = nullptr;
+  int             launches = 0;
+  bool            pdl = false;
+};
+
 struct FlowModel {
   dc_config cfg;
   int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0;
@@ -755,6 +799,12 @@ struct FlowModel {
   std::vector<size_t> o_bconv, o_bqkv, o_bo;
   std::vector<void*> allocs;
   Profiler* prof = nullptr;
+  // launch plumbing
+  bool pdl = true;                       // programmatic dependent launch between the step's kernels
+  int  dbg = 0;
+  cudaStream_t cap_stream = nullptr;     // used only to capture graphs at create
+  std::map<int, GraphEntry> graphs;      // batch size -> captured chunk step
+  std::vector<SlotSet> sets;
 };
 
 struct FlowState {
@@ -783,8 +833,17 @@ void pack_wt(std::vector<uint16_t>& dst, size_t off, const float* W, int K, int 
 
 }  // namespace
 
+namespace {
+bool build_graph(FlowModel* m, int n);
+}
+
 void flow_model_destroy(FlowModel* m) {
   if (!m) return;
+  for (auto& kv : m->graphs) {
+    if (kv.second.exec) cudaGraphExecDestroy(kv.second.exec);
+    if (kv.second.graph) cudaGraphDestroy(kv.second.graph);
+  }
+  if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
   for (void* p : m->allocs) cudaFree(p);
   delete m;
 }
@@ -929,13 +988,31 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   m->tmWo.resize(nA);
   for (int i = 0; i < nL; ++i) ok &= make_tmap(&m->tmWconv[i], m->wts + w_conv[i], C, 3 * C, 64);
   for (int i = 0; i < nA; ++i) {
-    ok &= make_tmap(&m->tmWqkv[i], m->wts + w_qkv[i], 3 * C, C, 64);
+    ok &= make_tmap(&m->tmWqkv[i], m->wts + w_qkv[i], 3 * C, C, 192);
     ok &= make_tmap(&m->tmWo[i], m->wts + w_o[i], C, C, 64);
   }
   if (!ok) {
     set_error("cuTensorMapEncodeTiled failed or is unavailable");
     flow_model_destroy(m);
     return DC_ERR_CUDA;
+  }
+  m->sets.resize((size_t)(m->S + MAX_SLOTS_PER_SET - 1) / MAX_SLOTS_PER_SET);
+  {
+    const char* e = getenv("DC_NO_PDL");        // experiments only
+    m->pdl = !(e && atoi(e));
+    const char* d = getenv("DC_GEMM_DBG");
+    m->dbg = d ? atoi(d) : 0;
+    const char* g = getenv("DC_NO_GRAPH");
+    if (!(g && atoi(g)) && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) == cudaSuccess) {
+      // the two batch sizes that matter are captured now, so that no decode call ever builds a graph:
+      // a single stream, and the full batch
+      const bool g1 = build_graph(m, 1);
+      const bool gs = m->S > 1 ? build_graph(m, m->S) : g1;
+      if (getenv("DC_VERBOSE"))
+        fprintf(stderr, "[dc] graphs: n=1 %s, n=%d %s, pdl %d/%d\n", g1 ? "ok" : "none", m->S, gs ? "ok" : "none",
+                g1 ? (int)m->graphs[1].pdl : -1, gs ? (int)m->graphs[m->S].pdl : -1);
+    }
+    cudaGetLastError();
   }
   *out = m;
   return DC_OK;
@@ -984,44 +1061,50 @@ void flow_state_close(FlowState* s) {
   delete s;
 }
 
-void launch_flow_attention(FlowModel* m, int n, int step, int layer, cudaStream_t st);
 
 void flow_set_profiler(FlowModel* m, Profiler* prof) { m->prof = prof; }
 
 
 
-dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats, const int* T,
-                      float* const* outp, cudaStream_t st, int* launches) {
+namespace {
+
+// Launch helper: optional programmatic-dependent-launch attribute, optional event bracketing.
+struct LaunchCtx {
+  cudaStream_t st;
+  bool         pdl;
+  Profiler*    prof;
+  int          launches = 0;
+  cudaError_t  err = cudaSuccess;
+};
+
+template <typename... KArgs, typename... Args>
+void launch(LaunchCtx& lc, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, bool pdl_ok, int cls, Args&&... args) {
+  ProfScope ps(lc.prof, cls, lc.st);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = lc.st;
+  cudaLaunchAttribute attr[1];
+  if (lc.pdl && pdl_ok) {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+  if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+  ++lc.launches;
+}
+
+// Issues every kernel of one chunk step for n slots (the slot table is uploaded by the first
+// kernel(s) from `sets`).
+void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchCtx& lc) {
   const dc_config& c = m->cfg;
   const int C = m->C, mel = m->mel;
-  // ---- per-call slot table (passed by value through a kernel, so nothing is staged or allocated)
-  for (int first = 0; first < n; first += MAX_SLOTS_PER_SET) {
-    SlotSet set;
-    set.first = first;
-    set.count = n - first < MAX_SLOTS_PER_SET ? n - first : MAX_SLOTS_PER_SET;
-    for (int i = 0; i < set.count; ++i) {
-      FlowState* s = states[first + i];
-      SlotInfo& si = set.s[i];
-      si.T = T[first + i];
-      si.kv_head = (int)(s->frames % m->Rk);
-      si.kv_len = (int)(s->frames < c.kv_cap ? s->frames : c.kv_cap);
-      si.pad = 0;
-      si.feats = feats[first + i];
-      si.out = outp[first + i];
-      si.halo = s->halo;
-      si.kv = s->kv;
-    }
-    {
-      ProfScope ps(m->prof, 4, st);
-      set_slots_kernel<<<1, MAX_SLOTS_PER_SET, 0, st>>>(set, m->d_slots);
-    }
-    ++*launches;
-  }
-  {
-    ProfScope ps(m->prof, 4, st);
-    flow_prep_kernel<<<n, 128, 0, st>>>(m->d_slots, mel, m->xstate, m->Ain, m->Kin);
-  }
-  ++*launches;
+  for (int i = 0; i < n_sets; ++i)   // not a programmatic launch: it overwrites the table the previous chunk still reads
+    launch(lc, set_slots_kernel, dim3(1), dim3(MAX_SLOTS_PER_SET), 0, false, 4, sets[i], m->d_slots);
+  launch(lc, flow_prep_kernel, dim3(n), dim3(128), 0, true, 4, (const SlotInfo*)m->d_slots, mel, m->xstate, m->Ain, m->Kin);
 
   const int m_tiles = (n * SLOT_ROWS + TILE_M - 1) / TILE_M;
   auto gemm = [&](const CUtensorMap& tA, const CUtensorMap& tB, GemmParams& p, int N) {
@@ -1031,24 +1114,24 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
     p.C = C;
     p.Rk = m->Rk;
     p.err = m->d_err;
-    {
-      const int stage_bytes = A_BYTES + p.taps * ((p.BN * 128 + 1023) & ~1023);
-      p.n_stages = std::min(MAX_STAGES, GEMM_TILE_SMEM / stage_bytes);
-      const char* d = getenv("DC_GEMM_DBG");
-      p.dbg = d ? atoi(d) : 0;
-      const char* e = getenv("DC_GEMM_STAGES");   // experiments only
-      if (e && atoi(e) >= 1 && atoi(e) < p.n_stages) p.n_stages = atoi(e);
-    }
-    dim3 grid(m_tiles, N / p.BN);
-    ProfScope ps(m->prof, p.mode == MODE_CONV ? 0 : 1, st);
-    flow_gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(tA, tB, p);
-    ++*launches;
+    const int stage_bytes = A_BYTES + p.taps * ((p.BN * 128 + 1023) & ~1023);
+    p.n_stages = std::min(MAX_STAGES, GEMM_TILE_SMEM / stage_bytes);
+    p.dbg = m->dbg;
+    launch(lc, flow_gemm_kernel, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), GEMM_SMEM, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
   };
   auto rmsnorm = [&](const bf16* x) {
     const int warps = n * SLOT_ROWS;
-    ProfScope ps(m->prof, 3, st);
-    flow_rmsnorm_kernel<<<(warps * 32 + 255) / 256, 256, 0, st>>>(m->d_slots, n, x, m->U, C, c.rms_eps);
-    ++*launches;
+    launch(lc, flow_rmsnorm_kernel, dim3((warps * 32 + 255) / 256), dim3(256), 0, true, 3, (const SlotInfo*)m->d_slots, n, x, m->U, C,
+           c.rms_eps);
+  };
+  auto attention = [&](int step, int layer) {
+    AttnParams p{};
+    p.slots = m->d_slots; p.q = m->Q; p.o = m->O; p.ld = C; p.dh = c.head_dim;
+    p.kv_off = ((long long)step * c.n_attn + layer) * 2 * m->Rk * C;
+    p.Rk = m->Rk; p.C = C;
+    p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
+    p.err = m->d_err;
+    launch(lc, flow_attn_kernel, dim3(n, c.n_heads), dim3(ATT_THREADS), ATT_SMEM, true, 2, p);
   };
   const float* fc = m->fconst;
   const long long halo_stride = (long long)HALO * C;
@@ -1085,13 +1168,12 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
         rmsnorm(X);
         {
           GemmParams p{};
-          p.mode = MODE_QKV; p.BN = 64; p.n_kblocks = C / KBLK; p.taps = 1;
+          p.mode = MODE_QKV; p.BN = 192; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bqkv[g]; p.q_out = m->Q; p.halo_off = -1;
           p.kv_off = ((long long)s * c.n_attn + g) * 2 * m->Rk * C;
           gemm(m->tmU, m->tmWqkv[g], p, 3 * C);
         }
-        launch_flow_attention(m, n, s, g, st);
-        ++*launches;
+        attention(s, g);
         {
           GemmParams p{};
           p.mode = MODE_OPROJ; p.BN = 64; p.n_kblocks = C / KBLK; p.taps = 1;
@@ -1112,24 +1194,112 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       gemm(m->tmU, m->tmWout, p, mel);
     }
   }
-  if (cudaGetLastError() != cudaSuccess) {
-    set_error("flow decode launch failed");
-    return DC_ERR_CUDA;
+}
+
+// One captured graph per batch size: the whole chunk step becomes a single graph launch; only the
+// slot-table node's by-value argument changes from call to call.
+bool build_graph(FlowModel* m, int n) {
+  if (n > MAX_SLOTS_PER_SET || m->cap_stream == nullptr) return false;
+  for (int use_pdl = m->pdl ? 1 : 0; use_pdl >= 0; --use_pdl) {
+    SlotSet dummy{};
+    dummy.first = 0;
+    dummy.count = 0;
+    cudaGraph_t graph = nullptr;
+    if (cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    LaunchCtx lc{m->cap_stream, use_pdl != 0, nullptr};
+    enqueue_chunk(m, n, &dummy, 1, lc);
+    cudaError_t e = cudaStreamEndCapture(m->cap_stream, &graph);
+    if (e != cudaSuccess || lc.err != cudaSuccess || graph == nullptr) {
+      cudaGetLastError();
+      if (graph) cudaGraphDestroy(graph);
+      continue;
+    }
+    GraphEntry ge{};
+    size_t n_nodes = 0;
+    cudaGraphGetNodes(graph, nullptr, &n_nodes);
+    std::vector<cudaGraphNode_t> nodes(n_nodes);
+    cudaGraphGetNodes(graph, nodes.data(), &n_nodes);
+    for (cudaGraphNode_t nd : nodes) {
+      cudaGraphNodeType ty;
+      if (cudaGraphNodeGetType(nd, &ty) != cudaSuccess || ty != cudaGraphNodeTypeKernel) continue;
+      cudaKernelNodeParams kp{};
+      if (cudaGraphKernelNodeGetParams(nd, &kp) == cudaSuccess && kp.func == (void*)set_slots_kernel) ge.set_node = nd;
+    }
+    e = cudaGraphInstantiate(&ge.exec, graph, 0);
+    if (e != cudaSuccess || ge.set_node == nullptr) {
+      cudaGetLastError();
+      if (ge.exec) cudaGraphExecDestroy(ge.exec);
+      cudaGraphDestroy(graph);
+      continue;
+    }
+    ge.graph = graph;
+    ge.launches = lc.launches;
+    ge.pdl = use_pdl != 0;
+    m->graphs[n] = ge;
+    return true;
+  }
+  return false;
+}
+
+}  // namespace
+
+dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats, const int* T,
+                      float* const* outp, cudaStream_t st, int* launches) {
+  const dc_config& c = m->cfg;
+  // ---- per-call slot table (passed by value through a kernel, so nothing is staged or allocated)
+  const int n_sets = (n + MAX_SLOTS_PER_SET - 1) / MAX_SLOTS_PER_SET;
+  std::vector<SlotSet>& sets = m->sets;   // sized at create
+  for (int k = 0; k < n_sets; ++k) {
+    SlotSet& set = sets[(size_t)k];
+    set.first = k * MAX_SLOTS_PER_SET;
+    set.count = n - set.first < MAX_SLOTS_PER_SET ? n - set.first : MAX_SLOTS_PER_SET;
+    for (int i = 0; i < set.count; ++i) {
+      FlowState* s = states[set.first + i];
+      SlotInfo& si = set.s[i];
+      si.T = T[set.first + i];
+      si.kv_head = (int)(s->frames % m->Rk);
+      si.kv_len = (int)(s->frames < c.kv_cap ? s->frames : c.kv_cap);
+      si.pad = 0;
+      si.feats = feats[set.first + i];
+      si.out = outp[set.first + i];
+      si.halo = s->halo;
+      si.kv = s->kv;
+    }
+  }
+  const bool profiling = m->prof != nullptr && m->prof->on;
+  auto it = m->graphs.find(n);
+  if (!profiling && it != m->graphs.end()) {
+    // one launch for the whole chunk step
+    GraphEntry& ge = it->second;
+    void* args[2] = {&sets[0], &m->d_slots};
+    cudaKernelNodeParams kp{};
+    kp.func = (void*)set_slots_kernel;
+    kp.gridDim = dim3(1);
+    kp.blockDim = dim3(MAX_SLOTS_PER_SET);
+    kp.sharedMemBytes = 0;
+    kp.kernelParams = args;
+    kp.extra = nullptr;
+    cudaError_t e = cudaGraphExecKernelNodeSetParams(ge.exec, ge.set_node, &kp);
+    if (e == cudaSuccess) e = cudaGraphLaunch(ge.exec, st);
+    if (e != cudaSuccess) {
+      set_error("flow decode graph launch failed: %s", cudaGetErrorString(e));
+      return DC_ERR_CUDA;
+    }
+    *launches += ge.launches;
+  } else {
+    LaunchCtx lc{st, m->pdl && !profiling, m->prof};
+    enqueue_chunk(m, n, sets.data(), n_sets, lc);
+    *launches += lc.launches;
+    if (lc.err != cudaSuccess || cudaGetLastError() != cudaSuccess) {
+      set_error("flow decode launch failed: %s", cudaGetErrorString(lc.err));
+      return DC_ERR_CUDA;
+    }
   }
   for (int i = 0; i < n; ++i) states[i]->frames += T[i];
   return DC_OK;
-}
-
-void launch_flow_attention(FlowModel* m, int n, int step, int layer, cudaStream_t st) {
-  const dc_config& c = m->cfg;
-  AttnParams p{};
-  p.slots = m->d_slots; p.q = m->Q; p.o = m->O; p.ld = m->C; p.dh = c.head_dim;
-  p.kv_off = ((long long)step * c.n_attn + layer) * 2 * m->Rk * m->C;
-  p.Rk = m->Rk; p.C = m->C;
-  p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
-  p.err = m->d_err;
-  ProfScope ps(m->prof, 2, st);
-  flow_attn_kernel<<<dim3(n, c.n_heads), ATT_THREADS, ATT_SMEM, st>>>(p);
 }
 
 }  // namespace dc
