@@ -496,7 +496,8 @@ constexpr int ATT_THREADS = 256;
 constexpr int ATT_KB = 128;             // keys per block
 constexpr int ATT_STAGES = 2;
 constexpr int ATT_TMEM_COLS = 256;      // S (128 columns) + O (64 columns); two CTAs share the SM's 512
-constexpr int ATT_LOADERS = 96;
+constexpr int ATT_K_LOADERS = 64;       // warps 2 and 6: Q, then the K blocks
+constexpr int ATT_V_LOADERS = 32;       // warp 7: the V blocks
 constexpr int ATT_Q_BYTES = 64 * 128;   // 64 query rows; the UMMA's rows 64..127 alias the P region
 constexpr int ATT_P_BYTES = 2 * 64 * 128;
 constexpr int ATT_STAGE_BYTES = 2 * ATT_KB * 128;   // K block + V block
@@ -515,6 +516,12 @@ struct AttnParams {
   int*            err;
 };
 
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(dst)), "l"(src) : "memory");
 }
@@ -525,26 +532,42 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   uint8_t* sQ = smem;
   uint8_t* sP = sQ + ATT_Q_BYTES;                    // tile t (keys 64 t .. 64 t + 63 of the block) at + 8192 t
   uint8_t* ring = sP + ATT_P_BYTES;
-  uint64_t* full = reinterpret_cast<uint64_t*>(ring + ATT_STAGES * ATT_STAGE_BYTES);   // [ATT_STAGES]
-  uint64_t* empty = full + ATT_STAGES;
-  uint64_t* bar_s = empty + ATT_STAGES;
+  // K and V have their own two-stage rings: a K stage is free as soon as S of its block has been
+  // computed, long before the V stage of the same block (free after P V), so K runs further ahead.
+  uint64_t* full_k = reinterpret_cast<uint64_t*>(ring + ATT_STAGES * ATT_STAGE_BYTES);   // [ATT_STAGES] each
+  uint64_t* empty_k = full_k + ATT_STAGES;
+  uint64_t* full_v = empty_k + ATT_STAGES;
+  uint64_t* empty_v = full_v + ATT_STAGES;
+  uint64_t* bar_s = empty_v + ATT_STAGES;
   uint64_t* bar_p = bar_s + 1;
   uint64_t* bar_pv = bar_p + 1;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_pv + 1);
+  uint64_t* bar_sfree = bar_pv + 1;     // every softmax thread has copied its S columns to registers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_sfree + 1);
   float* s_x = reinterpret_cast<float*>(tmem_slot + 2);   // [2][64] exchange between the two column halves
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int slot = blockIdx.x, head = blockIdx.y;
   const int chunks = p.dh >> 3;             // 16-byte chunks per head row
+#ifdef DC_TIMING
+  __shared__ long long a_t[64];
+  const bool atm = blockIdx.x == 3 && blockIdx.y == 2;
+  const long long a_start = clock64();
+#define DC_AT(i) do { if (atm) a_t[i] = clock64() - a_start; } while (0)
+#else
+#define DC_AT(i) do {} while (0)
+#endif
 
   if (tid == 0) {
     for (int i = 0; i < ATT_STAGES; ++i) {
-      ptx::mbar_init(&full[i], ATT_LOADERS);
-      ptx::mbar_init(&empty[i], 1);
+      ptx::mbar_init(&full_k[i], ATT_K_LOADERS);
+      ptx::mbar_init(&empty_k[i], 1);
+      ptx::mbar_init(&full_v[i], ATT_V_LOADERS);
+      ptx::mbar_init(&empty_v[i], 1);
     }
     ptx::mbar_init(bar_s, 1);
     ptx::mbar_init(bar_p, 128);
     ptx::mbar_init(bar_pv, 1);
+    ptx::mbar_init(bar_sfree, 128);
     ptx::fence_barrier_init();
   }
   if (warp == 3) ptx::tmem_alloc(tmem_slot, ATT_TMEM_COLS);
@@ -560,17 +583,22 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
 
   if (warp == 2 || warp >= 6) {
     // ---------------- loaders ----------------
-    const int lt = (warp == 2 ? 0 : (warp - 5) * 32) + lane;
+    const bool is_k = warp != 7;
+    const int nl = is_k ? ATT_K_LOADERS : ATT_V_LOADERS;
+    const int lt = (warp == 6 ? 32 : 0) + lane;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-    const bf16* qbase = p.q + (long long)(GUARD + slot * SLOT_ROWS + HALO) * p.ld + head * p.dh;
-    for (int i = lt; i < 64 * 8; i += ATT_LOADERS) {
-      const int row = i >> 3, j = i & 7;
-      uint8_t* dst = sQ + row * 128 + ((j ^ (row & 7)) << 4);
-      if (row < T && j < chunks) cp_async16(dst, qbase + (long long)row * p.ld + j * 8);
-      else *reinterpret_cast<uint4*>(dst) = zero;
+    if (is_k) {
+      const bf16* qbase = p.q + (long long)(GUARD + slot * SLOT_ROWS + HALO) * p.ld + head * p.dh;
+      for (int i = lt; i < 64 * 8; i += nl) {
+        const int row = i >> 3, j = i & 7;
+        uint8_t* dst = sQ + row * 128 + ((j ^ (row & 7)) << 4);
+        if (row < T && j < chunks) cp_async16(dst, qbase + (long long)row * p.ld + j * 8);
+        else *reinterpret_cast<uint4*>(dst) = zero;
+      }
     }
-    const bf16* kbase = si.kv + p.kv_off + head * p.dh;
-    const bf16* vbase = kbase + (long long)p.Rk * p.C;
+    const bf16* src0 = si.kv + p.kv_off + head * p.dh + (is_k ? 0 : (long long)p.Rk * p.C);
+    uint64_t* full = is_k ? full_k : full_v;
+    uint64_t* empty = is_k ? empty_k : empty_v;
     int start = si.kv_head - si.kv_len;
     if (start < 0) start += p.Rk;
     bool ok = true;
@@ -580,31 +608,31 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         asm volatile("cp.async.wait_all;" ::: "memory");
         ptx::fence_proxy_async_smem();
         ptx::mbar_arrive(&full[(b - 1) % ATT_STAGES]);
+        if (lt == 0 && is_k && b - 1 < 8) DC_AT(8 + b - 1);     // block b-1 landed
       }
       if (b >= ATT_STAGES && ok && !ptx::mbar_wait_relaxed(&empty[st], ((b / ATT_STAGES) - 1) & 1)) {
         ok = false;
         atomicExch(p.err, 4);
       }
-      uint8_t* sK = ring + st * ATT_STAGE_BYTES;
-      uint8_t* sV = sK + ATT_KB * 128;
-      for (int i = lt; i < ATT_KB * 8; i += ATT_LOADERS) {
+      uint8_t* dstb = ring + st * ATT_STAGE_BYTES + (is_k ? 0 : ATT_KB * 128);
+      if (lt == 0 && is_k && b < 8) DC_AT(b);                    // block b load issue starts
+      for (int i = lt; i < ATT_KB * 8; i += nl) {
         const int row = i >> 3, j = i & 7;
         const int key = b * ATT_KB + row;
         const int off = row * 128 + ((j ^ (row & 7)) << 4);
         if (key < L && j < chunks) {
           int rr = start + key;
           if (rr >= p.Rk) rr -= p.Rk;
-          cp_async16(sK + off, kbase + (long long)rr * p.C + j * 8);
-          cp_async16(sV + off, vbase + (long long)rr * p.C + j * 8);
+          cp_async16(dstb + off, src0 + (long long)rr * p.C + j * 8);
         } else {
-          *reinterpret_cast<uint4*>(sK + off) = zero;
-          *reinterpret_cast<uint4*>(sV + off) = zero;   // 0 * garbage must not poison O
+          *reinterpret_cast<uint4*>(dstb + off) = zero;   // for V: 0 * garbage must not poison O
         }
       }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     ptx::fence_proxy_async_smem();
     ptx::mbar_arrive(&full[(nkb - 1) % ATT_STAGES]);
+    if (lt == 0 && is_k && nkb - 1 < 8) DC_AT(8 + nkb - 1);
   } else if (warp == 3) {
     // ---------------- UMMA issuer ----------------
     if (lane == 0) {
@@ -613,24 +641,39 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       const uint64_t dq = ptx::umma_desc_sw128(ptx::smem_u32(sQ));
       const uint64_t dp = ptx::umma_desc_sw128(ptx::smem_u32(sP));
       bool ok = true;
-      for (int b = 0; b < nkb; ++b) {
+      // S(b+1) is issued as soon as the softmax threads have copied S(b) out of tensor memory, i.e.
+      // before P(b) exists: the tensor pipe computes the next block's scores while the softmax of
+      // this block runs, and P V follows when P is ready.
+      auto issue_s = [&](int b) {
         const int st = b % ATT_STAGES;
-        if (ok && !ptx::mbar_wait(&full[st], (b / ATT_STAGES) & 1)) { ok = false; atomicExch(p.err, 5); }
+        if (ok && !ptx::mbar_wait(&full_k[st], (b / ATT_STAGES) & 1)) { ok = false; atomicExch(p.err, 5); }
         ptx::tc_fence_after();
         const uint64_t dk = ptx::umma_desc_sw128(ptx::smem_u32(ring + st * ATT_STAGE_BYTES));
-        const uint64_t dv = ptx::umma_desc_sw128(ptx::smem_u32(ring + st * ATT_STAGE_BYTES + ATT_KB * 128));
 #pragma unroll
         for (int k = 0; k < 4; ++k) ptx::umma_bf16(tmem_base, dq + 2 * k, dk + 2 * k, idesc_s, k != 0);
         ptx::umma_commit(bar_s);
+        ptx::umma_commit(&empty_k[st]);                  // the K stage is free once S(b) has been computed
+        if (b < 8) DC_AT(16 + b);                        // S(b) issued
+      };
+      issue_s(0);
+      for (int b = 0; b < nkb; ++b) {
+        const int st = b % ATT_STAGES;
+        if (b + 1 < nkb) {
+          if (ok && !ptx::mbar_wait(bar_sfree, b & 1)) { ok = false; atomicExch(p.err, 10); }
+          issue_s(b + 1);
+        }
         if (ok && !ptx::mbar_wait(bar_p, b & 1)) { ok = false; atomicExch(p.err, 6); }
+        if (ok && !ptx::mbar_wait(&full_v[st], (b / ATT_STAGES) & 1)) { ok = false; atomicExch(p.err, 11); }
         ptx::tc_fence_after();
+        const uint64_t dv = ptx::umma_desc_sw128(ptx::smem_u32(ring + st * ATT_STAGE_BYTES + ATT_KB * 128));
         const int valid = L - b * ATT_KB;
         const int ksteps = valid >= ATT_KB ? ATT_KB / 16 : (valid + 15) / 16;
         for (int k = 0; k < ksteps; ++k)   // P tile k/4 (8 KB apart), 32-byte K steps; V: 16 key rows = 2 KB per step
           ptx::umma_bf16(tmem_base + ATT_KB, dp + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
                          idesc_pv, (b | k) != 0);
-        ptx::umma_commit(&empty[st]);
+        ptx::umma_commit(&empty_v[st]);
         ptx::umma_commit(bar_pv);
+        if (b < 8) DC_AT(24 + b);                        // PV(b) issued
       }
     }
   } else {
@@ -644,17 +687,22 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     for (int b = 0; b < nkb; ++b) {
       if (ok && !ptx::mbar_wait(bar_s, b & 1)) { ok = false; atomicExch(p.err, 7); }
       ptx::tc_fence_after();
+      if (tid == 0 && b < 8) DC_AT(32 + b);              // S(b) ready
       const int valid = L - b * ATT_KB - half * 64;   // columns of this half that are real keys
       float v[64];
 #pragma unroll
       for (int c = 0; c < 4; ++c) ptx::tmem_ld16(lane_addr + (uint32_t)(half * 64 + c * 16), v + 16 * c);
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(bar_sfree);               // S(b) is in registers: the next block's scores may overwrite it
+      if (valid < 64) {                          // only the last block has padded key columns
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (i >= valid) v[i] = -INFINITY;
+      }
       float mx = -INFINITY;
 #pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        v[i] = (i < valid) ? v[i] * p.scale_log2e : -INFINITY;
-        mx = fmaxf(mx, v[i]);
-      }
-      s_x[half * 64 + row] = mx;
+      for (int i = 0; i < 64; ++i) mx = fmaxf(mx, v[i]);
+      s_x[half * 64 + row] = mx * p.scale_log2e;
       ptx::named_bar_sync(2, 128);
       mx = fmaxf(s_x[row], s_x[64 + row]);
       if (b > 0) {   // P V of the previous block must be done: P tile free, O quiescent
@@ -686,7 +734,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         float e[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          e[i] = exp2f(v[16 * c + i] - m_ref);
+          e[i] = ex2_approx(fmaf(v[16 * c + i], p.scale_log2e, -m_ref));
           lsum += e[i];
         }
         uint4 a, bq;
@@ -697,6 +745,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       ptx::fence_proxy_async_smem();
       ptx::tc_fence_before();
       ptx::mbar_arrive(bar_p);
+      if (tid == 0 && b < 8) DC_AT(40 + b);              // P(b) written
     }
     if (ok && !ptx::mbar_wait(bar_pv, (nkb - 1) & 1)) { ok = false; atomicExch(p.err, 9); }
     ptx::tc_fence_after();
@@ -721,6 +770,23 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 3) ptx::tmem_dealloc(tmem_base, ATT_TMEM_COLS);
+#ifdef DC_TIMING
+  if (atm && tid == 0) {
+    printf("ATT nkb %d end %lld\n load_issue:", nkb, clock64() - a_start);
+    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[i]);
+    printf("\n landed:");
+    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[8 + i]);
+    printf("\n S_issued:");
+    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[16 + i]);
+    printf("\n S_ready:");
+    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[32 + i]);
+    printf("\n P_written:");
+    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[40 + i]);
+    printf("\n PV_issued:");
+    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[24 + i]);
+    printf("\n");
+  }
+#endif
 }
 
 // ---- host helpers ----------------------------------------------------------------------------
