@@ -3,19 +3,18 @@
 // fused head conv + inverse STFT + overlap-add kernel.  fp32 parity (max err <= 1e-4 of RMS) rules
 // out single-pass TF32, so these run on the FP32 pipe.
 #include "dc_internal.h"
+#include "dc_ptx.cuh"
 
 #include <math.h>
 
 #include <mutex>
+#include <utility>
 
 namespace dc {
 
 namespace {
 
-constexpr int BM = 64;   // frames per CTA tile
-constexpr int BN = 64;   // output channels per CTA tile
 constexpr int BK = 16;   // reduction slice
-constexpr int NT = 256;  // threads: 16 x 16, each a 4 x 4 micro tile
 
 __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z)); }
 
@@ -24,22 +23,62 @@ __device__ __forceinline__ const float* in_row_ptr(const TapConvF32& p, long lon
   return p.in_ring + (long long)((int)(t & (long long)p.in_mask)) * p.C_in;
 }
 
-__global__ void __launch_bounds__(NT) tapconv_f32_kernel(const TapConvF32 p) {
-  __shared__ __align__(16) float As[2][BK][BM + 4];
-  __shared__ __align__(16) float Bs[2][BK][BN];
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros (out-of-range rows / columns).
+__device__ __forceinline__ void cp_async16_zfill(void* dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src),
+               "r"(src_bytes)
+               : "memory");
+}
 
-  const int tid = threadIdx.x;
-  const int tx = tid & 15, ty = tid >> 4;
+// One CTA computes a BM x BN tile of one phase.  A group of BM*BN/16 threads (each a 4 x 4 micro
+// tile) accumulates a share of the reduction; KS such groups split the reduction steps among
+// themselves (step kb belongs to group kb % KS) and their partial tiles are summed through shared
+// memory in a fixed order, so the result does not depend on timing.  The vocoder's early layers
+// have few frames and long reductions: without the split most SMs would hold a single warp.
+// Operands stream through a 4-stage cp.async ring per group (a reduction step is far cheaper than
+// one L2 round trip, so three steps are kept in flight).
+constexpr int F32_STAGES = 4;
+
+template <int BM, int BN>
+struct TapTile {
+  static constexpr int NTG = BM * BN / 16;                 // threads per group
+  static constexpr int LDA = BK + 4;                       // row stride of the A tile (floats)
+  static constexpr int STAGE_FLOATS = BM * LDA + BK * BN;  // one stage of one group
+  static constexpr int GROUP_FLOATS = F32_STAGES * STAGE_FLOATS;
+};
+
+template <int BM, int BN>
+__global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p_in, const int KS) {
+  using TT = TapTile<BM, BN>;
+  ptx::pdl_launch();
+  ptx::pdl_wait();          // the call record and the input ring come from earlier kernels
+  TapConvF32 p = p_in;
+  if (p.call != nullptr) {
+    const F32Call c = *p.call;
+    p.T_in = c.T * p.rate_in;
+    p.pos_in = c.frames * p.rate_in;
+    p.pos_out = p.pos_in * p.n_phase;
+    p.in_direct = p.first_layer ? c.feats : nullptr;
+    p.out_direct = p.last_layer ? c.out : nullptr;
+  }
+  if ((int)blockIdx.x * BM >= p.T_in) return;   // the grid is sized for the longest chunk
+  constexpr int NTG = TT::NTG;
+  constexpr int TX = BN / 4;              // threads along the channel axis
+  constexpr int NA = BM * 4 / NTG;        // 16-byte copies of the A tile per thread
+  constexpr int NB = BN * 4 / NTG;        // 16-byte copies of the B tile per thread
+  constexpr int LDA = TT::LDA;
+  extern __shared__ __align__(16) float f32_smem[];
+
+  const int grp = threadIdx.x / NTG;      // reduction group
+  const int tid = threadIdx.x - grp * NTG;
+  float* gbase = f32_smem + grp * TT::GROUP_FLOATS;
+  const int tx = tid % TX, ty = tid / TX;
   const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, phase = blockIdx.z;
-
-  const int a_row = tid >> 2, a_k = (tid & 3) * 4;     // A tile: 64 rows x 16 k, one float4 per thread
-  const int b_k = tid >> 4, b_n = (tid & 15) * 4;      // B tile: 16 k x 64 n
-  const bool a_ok = (m0 + a_row) < p.T_in;
-  const long long t_row = p.pos_in + m0 + a_row;
   const float* Wp = p.W + (long long)phase * p.w_phase_stride;
 
   const int kb_per_tap = (p.C_in + BK - 1) / BK;
   const int nkb = p.n_taps * kb_per_tap;
+  const int my_steps = (nkb - grp + KS - 1) / KS;   // steps grp, grp + KS, ...
 
   float acc[4][4];
 #pragma unroll
@@ -47,46 +86,79 @@ __global__ void __launch_bounds__(NT) tapconv_f32_kernel(const TapConvF32 p) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-  float4 ra, rb;
-  auto gload = [&](int kb) {
-    const int tap = kb / kb_per_tap;
-    const int c0 = (kb - tap * kb_per_tap) * BK;
-    ra = make_float4(0.f, 0.f, 0.f, 0.f);
-    rb = ra;
-    if (a_ok && c0 + a_k < p.C_in)
-      ra = *reinterpret_cast<const float4*>(in_row_ptr(p, t_row - p.shift[tap]) + c0 + a_k);
-    if (c0 + b_k < p.C_in && n0 + b_n < p.C_out)
-      rb = *reinterpret_cast<const float4*>(Wp + (long long)tap * p.w_tap_stride +
-                                            (long long)(c0 + b_k) * p.C_out + n0 + b_n);
-  };
-  auto sstore = [&](int buf) {
-    As[buf][a_k + 0][a_row] = ra.x;
-    As[buf][a_k + 1][a_row] = ra.y;
-    As[buf][a_k + 2][a_row] = ra.z;
-    As[buf][a_k + 3][a_row] = ra.w;
-    *reinterpret_cast<float4*>(&Bs[buf][b_k][b_n]) = rb;
+  auto issue = [&](int s) {   // s-th step of this group
+    if (s < my_steps) {
+      const int kb = grp + s * KS;
+      float* As = gbase + (s % F32_STAGES) * TT::STAGE_FLOATS;   // [BM][LDA]
+      float* Bs = As + BM * LDA;                                  // [BK][BN]
+      const int tap = kb / kb_per_tap;
+      const int c0 = (kb - tap * kb_per_tap) * BK;
+#pragma unroll
+      for (int u = 0; u < NA; ++u) {
+        const int i = tid + u * NTG;
+        const int row = i >> 2, kq = (i & 3) * 4;      // A tile: BM rows x 16 k
+        const bool ok = m0 + row < p.T_in && c0 + kq < p.C_in;
+        const float* src = ok ? in_row_ptr(p, p.pos_in + m0 + row - p.shift[tap]) + c0 + kq : p.W;
+        cp_async16_zfill(As + row * LDA + kq, src, ok ? 16 : 0);
+      }
+#pragma unroll
+      for (int u = 0; u < NB; ++u) {
+        const int i = tid + u * NTG;
+        const int k = i / TX, nq = (i % TX) * 4;       // B tile: 16 k x BN n
+        const bool ok = c0 + k < p.C_in && n0 + nq < p.C_out;
+        const float* src = ok ? Wp + (long long)tap * p.w_tap_stride + (long long)(c0 + k) * p.C_out + n0 + nq : p.W;
+        cp_async16_zfill(Bs + k * BN + nq, src, ok ? 16 : 0);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");   // an (empty) group per step keeps the count uniform
   };
 
-  gload(0);
-  sstore(0);
-  __syncthreads();
-  for (int kb = 0; kb < nkb; ++kb) {
-    const int cur = kb & 1;
-    if (kb + 1 < nkb) gload(kb + 1);
 #pragma unroll
-    for (int k = 0; k < BK; ++k) {
-      const float4 a = *reinterpret_cast<const float4*>(&As[cur][k][ty * 4]);
-      const float4 b = *reinterpret_cast<const float4*>(&Bs[cur][k][tx * 4]);
-      const float av[4] = {a.x, a.y, a.z, a.w};
-      const float bv[4] = {b.x, b.y, b.z, b.w};
+  for (int s = 0; s < F32_STAGES - 1; ++s) issue(s);
+  for (int s = 0; s < my_steps; ++s) {
+    asm volatile("cp.async.wait_group %0;" ::"n"(F32_STAGES - 2) : "memory");   // step s has landed
+    asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "r"(NTG) : "memory");       // for the whole group; step s-1's buffer is free
+    issue(s + F32_STAGES - 1);
+    const float* As = gbase + (s % F32_STAGES) * TT::STAGE_FLOATS;
+    const float* Bs = As + BM * LDA;
+#pragma unroll
+    for (int k4 = 0; k4 < BK; k4 += 4) {
+      float4 a[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4*>(As + (ty * 4 + i) * LDA + k4);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        const float4 b = *reinterpret_cast<const float4*>(Bs + (k4 + kk) * BN + tx * 4);
+        const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float av = kk == 0 ? a[i].x : (kk == 1 ? a[i].y : (kk == 2 ? a[i].z : a[i].w));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av, bv[j], acc[i][j]);
+        }
+      }
+    }
+  }
+
+  if (KS > 1) {
+    // fixed-order sum of the groups' partial tiles: group g parks its tile in its own (now idle)
+    // operand ring, group 0 adds them in the order 1, 2, ...
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncthreads();
+    if (grp > 0) {
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        *reinterpret_cast<float4*>(gbase + (tid * 4 + i) * 4) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
     }
-    if (kb + 1 < nkb) {
-      sstore(cur ^ 1);
-      __syncthreads();
+    __syncthreads();
+    if (grp > 0) return;
+    for (int g = 1; g < KS; ++g) {
+      const float* src = f32_smem + g * TT::GROUP_FLOATS;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float4 v = *reinterpret_cast<const float4*>(src + (tid * 4 + i) * 4);
+        acc[i][0] += v.x; acc[i][1] += v.y; acc[i][2] += v.z; acc[i][3] += v.w;
+      }
     }
   }
 
@@ -118,7 +190,7 @@ __global__ void __launch_bounds__(NT) tapconv_f32_kernel(const TapConvF32 p) {
   if (p.save_ring != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
     const int first = p.T_in > p.save_rows ? p.T_in - p.save_rows : 0;
     const int c4 = p.C_in >> 2;
-    for (int i = tid; i < (p.T_in - first) * c4; i += NT) {
+    for (int i = tid; i < (p.T_in - first) * c4; i += NTG) {
       const int r = first + i / c4, c = (i - (i / c4) * c4) * 4;
       const float4 v = *reinterpret_cast<const float4*>(p.in_direct + (long long)r * p.C_in + c);
       *reinterpret_cast<float4*>(p.save_ring + (long long)((int)((p.pos_in + r) & (long long)p.in_mask)) * p.C_in + c) = v;
@@ -136,8 +208,20 @@ __constant__ float c_cos16[16];  // cos(2 pi j / 16)
 __constant__ float c_sin16[16];
 __constant__ float c_hann16[16];
 
-__global__ void __launch_bounds__(HT) head_istft_f32_kernel(const HeadIstftF32 p) {
+__global__ void __launch_bounds__(HT) head_istft_f32_kernel(const HeadIstftF32 p_in) {
   extern __shared__ __align__(16) float smem[];
+  ptx::pdl_launch();
+  ptx::pdl_wait();
+  HeadIstftF32 p = p_in;
+  if (p.call != nullptr) {
+    const F32Call c = *p.call;
+    p.T = c.T * p.rate_in;
+    p.pos = c.frames * p.rate_in;
+    p.tail_in = p.tails + 12 * c.parity;
+    p.tail_out = p.tails + 12 * (c.parity ^ 1);
+    p.pcm = c.out;
+  }
+  if ((int)blockIdx.x * HF >= p.T) return;
   float* Ws = smem;                              // [3*C][NH]
   float* g = smem + 3 * p.C * NH;                // [HT][NFFT] windowed frame signals
   const int tid = threadIdx.x;
@@ -218,9 +302,65 @@ __global__ void __launch_bounds__(HT) head_istft_f32_kernel(const HeadIstftF32 p
 
 }  // namespace
 
-void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st) {
-  dim3 grid((p.T_in + BM - 1) / BM, (p.C_out + BN - 1) / BN, p.n_phase);
-  tapconv_f32_kernel<<<grid, NT, 0, st>>>(p);
+namespace {
+__global__ void set_f32_call_kernel(const F32Call v, F32Call* dst) {
+  ptx::pdl_launch();
+  if (threadIdx.x == 0) *dst = v;
+}
+
+template <typename... KArgs, typename... Args>
+void launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  if (pdl) {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+template <int BM, int BN>
+void launch_tile(const TapConvF32& p, int KS, int T_grid, cudaStream_t st, bool pdl) {
+  using TT = TapTile<BM, BN>;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !attr_set[dev]) {   // opt in to > 48 KB of dynamic shared memory, once per device
+    const int want = 8 * TT::GROUP_FLOATS * 4;
+    cudaFuncSetAttribute(tapconv_f32_kernel<BM, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, want > 227 * 1024 ? 227 * 1024 : want);
+    attr_set[dev] = true;
+  }
+  dim3 grid((T_grid + BM - 1) / BM, (p.C_out + BN - 1) / BN, p.n_phase);
+  launch_ex(tapconv_f32_kernel<BM, BN>, grid, dim3(KS * TT::NTG), (size_t)KS * TT::GROUP_FLOATS * sizeof(float), st, pdl, p, KS);
+}
+}  // namespace
+
+const void* set_f32_call_func() { return (const void*)set_f32_call_kernel; }
+
+void launch_set_f32_call(const F32Call& v, F32Call* dst, cudaStream_t st) {
+  set_f32_call_kernel<<<1, 32, 0, st>>>(v, dst);
+}
+
+void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st, int T_grid, bool pdl) {
+  if (T_grid < 0) T_grid = p.T_in;
+  const int nkb = p.n_taps * ((p.C_in + BK - 1) / BK);
+  const long long ctas64 = (long long)((T_grid + 63) / 64) * ((p.C_out + 63) / 64) * p.n_phase;
+  if (ctas64 >= 296) {
+    launch_tile<64, 64>(p, 1, T_grid, st, pdl);
+  } else {
+    // few tiles: small tiles, and split the reduction inside the CTA until the GPU holds about
+    // 1200 warps (8 per SM), keeping at least 4 steps per group; at most 8 groups (512 threads)
+    const long long ctas32 = (long long)((T_grid + 31) / 32) * ((p.C_out + 31) / 32) * p.n_phase;
+    int KS = 1;
+    while (KS < 8 && ctas32 * 2 * KS < 1200 && nkb / (2 * KS) >= 4) KS *= 2;
+    launch_tile<32, 32>(p, KS, T_grid, st, pdl);
+  }
 }
 
 cudaError_t prepare_f32_constants() {
@@ -237,10 +377,11 @@ cudaError_t prepare_f32_constants() {
   return e;
 }
 
-void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st) {
+void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st, int T_grid, bool pdl) {
+  if (T_grid < 0) T_grid = p.T;
   const size_t smem = (size_t)(3 * p.C * NH + HT * NFFT) * sizeof(float);
-  const int grid = (p.T + HF - 1) / HF;
-  head_istft_f32_kernel<<<grid, HT, smem, st>>>(p);
+  const int grid = (T_grid + HF - 1) / HF;
+  launch_ex(head_istft_f32_kernel, dim3(grid), dim3(HT), smem, st, pdl, p);
 }
 
 }  // namespace dc

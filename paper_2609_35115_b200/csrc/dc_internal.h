@@ -16,7 +16,22 @@ namespace dc {
 // from a plain [T_in][C_in] array (`in_direct`, the caller's chunk).  Rings start zeroed, so
 // t < 0 reads the causal zero padding.  Nothing is ever concatenated or moved: the left context
 // of the next chunk is simply the rows already in the ring.
+// Per-call values of the fp32 pipelines, kept in device memory so that a captured graph of the
+// chunk step stays valid from call to call: a tiny kernel rewrites this record (its by-value
+// argument is the only thing that changes in the graph) and every layer kernel derives its frame
+// counts, ring positions and the caller's pointers from it.
+struct F32Call {
+  long long    frames;     // frames decoded by the stream before this call
+  int          T;          // frames presented by this call
+  int          parity;     // which overlap-add tail buffer holds the previous call's tail
+  const float* feats;      // caller's chunk
+  float*       out;        // caller's output
+};
+
 struct TapConvF32 {
+  const F32Call* call;     // if set: T_in, pos_in, pos_out, in_direct, out_direct come from *call
+  int          rate_in;    // ... scaled by this layer's frames per chunk frame
+  int          first_layer, last_layer;
   const float* in_ring;
   int          in_mask;
   const float* in_direct;     // may be null
@@ -41,11 +56,17 @@ struct TapConvF32 {
   int          save_rows;
 };
 
-void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st);
+// T_grid: frames the grid is sized for (p.T_in, or the largest T_in when p.call is set).
+void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st, int T_grid = -1, bool pdl = false);
+void launch_set_f32_call(const F32Call& v, F32Call* dst, cudaStream_t st);
+const void* set_f32_call_func();
 
 // Head conv (k = 3, input already SiLU-activated) + magnitude/phase -> inverse real DFT (n_fft = 16)
 // -> synthesis window -> overlap-add (hop 4) with the 12-sample tail carried across chunks.
 struct HeadIstftF32 {
+  const F32Call* call;        // if set: pos, T, tails and pcm come from *call
+  int          rate_in;
+  float*       tails;         // [2][12] ping-pong pair (used with call)
   const float* in_ring;       // [cap][C]
   int          in_mask;
   long long    pos;           // logical index of the first new frame
@@ -59,7 +80,7 @@ struct HeadIstftF32 {
   float*       pcm;           // [4*T]
 };
 
-void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st);
+void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st, int T_grid = -1, bool pdl = false);
 
 // Uploads the constant tables of the head kernel (DFT twiddles, periodic Hann window) to the
 // current device.  Synchronous; called from dc_create, never from a decode call.

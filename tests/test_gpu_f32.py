@@ -129,7 +129,7 @@ def test_admission_and_error_paths(dc):
     from tests import gpu_util as gu
     assert gu.rel_err(torch.cat([ref1, got2]).cpu().numpy(), ref) <= TOL_F32
     c = m.counters()
-    assert c[0] == 2 and c[1] == 32 and c[2] == 2 and c[3] == 2 and c[5] == 4
+    assert c[0] == 2 and c[1] == 32 and c[2] == 2 and c[3] == 2 and c[5] == 6   # per chunk: call record + 2 conv blocks
     # a model with open streams cannot be destroyed; a closed stream refuses work
     with pytest.raises(dc.DCError):
         m.destroy()
