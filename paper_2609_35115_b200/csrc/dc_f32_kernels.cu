@@ -6,6 +6,7 @@
 #include "dc_ptx.cuh"
 
 #include <math.h>
+#include <stdio.h>
 
 #include <mutex>
 #include <utility>
@@ -18,9 +19,11 @@ constexpr int BK = 16;   // reduction slice
 
 __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z)); }
 
-__device__ __forceinline__ const float* in_row_ptr(const TapConvF32& p, long long t) {
-  if (p.in_direct != nullptr && t >= p.pos_in) return p.in_direct + (t - p.pos_in) * p.C_in;
-  return p.in_ring + (long long)((int)(t & (long long)p.in_mask)) * p.C_in;
+// Row of logical frame t: the caller's chunk for new frames of the first layer, else the ring.
+__device__ __forceinline__ const float* in_row_ptr(const float* in_direct, long long pos_in, const float* in_ring, int in_mask,
+                                                   int C_in, long long t) {
+  if (in_direct != nullptr && t >= pos_in) return in_direct + (t - pos_in) * C_in;
+  return in_ring + (long long)((int)(t & (long long)in_mask)) * C_in;
 }
 
 // 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros (out-of-range rows / columns).
@@ -48,20 +51,27 @@ struct TapTile {
 };
 
 template <int BM, int BN>
-__global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p_in, const int KS) {
+__global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, const int KS) {
   using TT = TapTile<BM, BN>;
   ptx::pdl_launch();
   ptx::pdl_wait();          // the call record and the input ring come from earlier kernels
-  TapConvF32 p = p_in;
+  // per-call values: by value, or from the device-side call record (captured graphs)
+  int T_in = p.T_in;
+  long long pos_in = p.pos_in, pos_out = p.pos_out;
+  const float* in_direct = p.in_direct;
+  float* out_direct = p.out_direct;
   if (p.call != nullptr) {
     const F32Call c = *p.call;
-    p.T_in = c.T * p.rate_in;
-    p.pos_in = c.frames * p.rate_in;
-    p.pos_out = p.pos_in * p.n_phase;
-    p.in_direct = p.first_layer ? c.feats : nullptr;
-    p.out_direct = p.last_layer ? c.out : nullptr;
+    T_in = c.T * p.rate_in;
+    pos_in = c.frames * p.rate_in;
+    pos_out = pos_in * p.n_phase;
+    in_direct = p.first_layer ? c.feats : nullptr;
+    out_direct = p.last_layer ? c.out : nullptr;
   }
-  if ((int)blockIdx.x * BM >= p.T_in) return;   // the grid is sized for the longest chunk
+  if ((int)blockIdx.x * BM >= T_in) return;   // the grid is sized for the longest chunk
+  const float* in_ring = p.in_ring;
+  const int in_mask = p.in_mask, C_in = p.C_in, C_out = p.C_out;
+  const int sh0 = p.shift[0], sh1 = p.shift[1], sh2 = p.shift[2];
   constexpr int NTG = TT::NTG;
   constexpr int TX = BN / 4;              // threads along the channel axis
   constexpr int NA = BM * 4 / NTG;        // 16-byte copies of the A tile per thread
@@ -76,7 +86,7 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p_in,
   const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, phase = blockIdx.z;
   const float* Wp = p.W + (long long)phase * p.w_phase_stride;
 
-  const int kb_per_tap = (p.C_in + BK - 1) / BK;
+  const int kb_per_tap = (C_in + BK - 1) / BK;
   const int nkb = p.n_taps * kb_per_tap;
   const int my_steps = (nkb - grp + KS - 1) / KS;   // steps grp, grp + KS, ...
 
@@ -85,6 +95,37 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p_in,
   for (int i = 0; i < 4; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  // Per-thread copy descriptors, hoisted out of the step loop: the source row of every A copy for
+  // each tap, and the base of every B copy.
+  const float* a_src[NA][3];
+  bool a_ok[NA];
+  int a_dst[NA], a_kq[NA];
+#pragma unroll
+  for (int u = 0; u < NA; ++u) {
+    const int i = tid + u * NTG;
+    const int row = i >> 2;
+    a_kq[u] = (i & 3) * 4;                                // A tile: BM rows x 16 k
+    a_ok[u] = m0 + row < T_in;
+    a_dst[u] = row * LDA + a_kq[u];
+    const long long t = pos_in + m0 + row;
+    a_src[u][0] = in_row_ptr(in_direct, pos_in, in_ring, in_mask, C_in, t - sh0) + a_kq[u];
+    a_src[u][1] = in_row_ptr(in_direct, pos_in, in_ring, in_mask, C_in, t - sh1) + a_kq[u];
+    a_src[u][2] = in_row_ptr(in_direct, pos_in, in_ring, in_mask, C_in, t - sh2) + a_kq[u];
+  }
+  const float* b_src[NB];
+  bool b_ok[NB];
+  int b_dst[NB], b_k[NB];
+#pragma unroll
+  for (int u = 0; u < NB; ++u) {
+    const int i = tid + u * NTG;
+    b_k[u] = i / TX;                                      // B tile: 16 k x BN n
+    const int nq = (i % TX) * 4;
+    b_ok[u] = n0 + nq < C_out;
+    b_dst[u] = b_k[u] * BN + nq;
+    b_src[u] = Wp + (long long)b_k[u] * C_out + n0 + nq;
+  }
+  const long long w_tap = p.w_tap_stride;
 
   auto issue = [&](int s) {   // s-th step of this group
     if (s < my_steps) {
@@ -95,27 +136,31 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p_in,
       const int c0 = (kb - tap * kb_per_tap) * BK;
 #pragma unroll
       for (int u = 0; u < NA; ++u) {
-        const int i = tid + u * NTG;
-        const int row = i >> 2, kq = (i & 3) * 4;      // A tile: BM rows x 16 k
-        const bool ok = m0 + row < p.T_in && c0 + kq < p.C_in;
-        const float* src = ok ? in_row_ptr(p, p.pos_in + m0 + row - p.shift[tap]) + c0 + kq : p.W;
-        cp_async16_zfill(As + row * LDA + kq, src, ok ? 16 : 0);
+        const bool ok = a_ok[u] && c0 + a_kq[u] < C_in;
+        const float* src = (tap == 0 ? a_src[u][0] : (tap == 1 ? a_src[u][1] : a_src[u][2])) + c0;
+        cp_async16_zfill(As + a_dst[u], ok ? src : p.W, ok ? 16 : 0);
       }
+      const long long boff = (long long)tap * w_tap + (long long)c0 * C_out;
 #pragma unroll
       for (int u = 0; u < NB; ++u) {
-        const int i = tid + u * NTG;
-        const int k = i / TX, nq = (i % TX) * 4;       // B tile: 16 k x BN n
-        const bool ok = c0 + k < p.C_in && n0 + nq < p.C_out;
-        const float* src = ok ? Wp + (long long)tap * p.w_tap_stride + (long long)(c0 + k) * p.C_out + n0 + nq : p.W;
-        cp_async16_zfill(Bs + k * BN + nq, src, ok ? 16 : 0);
+        const bool ok = b_ok[u] && c0 + b_k[u] < C_in;
+        cp_async16_zfill(Bs + b_dst[u], ok ? b_src[u] + boff : p.W, ok ? 16 : 0);
       }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");   // an (empty) group per step keeps the count uniform
   };
 
+#ifdef DC_TIMING
+  __shared__ long long f_t[40];
+  const bool ftm = blockIdx.x == 0 && blockIdx.y == 1 && blockIdx.z == 0 && threadIdx.x == 0;
+  const long long f0 = clock64();
+#endif
 #pragma unroll
   for (int s = 0; s < F32_STAGES - 1; ++s) issue(s);
   for (int s = 0; s < my_steps; ++s) {
+#ifdef DC_TIMING
+    if (ftm && s < 32) f_t[s] = clock64() - f0;
+#endif
     asm volatile("cp.async.wait_group %0;" ::"n"(F32_STAGES - 2) : "memory");   // step s has landed
     asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "r"(NTG) : "memory");       // for the whole group; step s-1's buffer is free
     issue(s + F32_STAGES - 1);
@@ -140,6 +185,13 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p_in,
     }
   }
 
+#ifdef DC_TIMING
+  if (ftm) {
+    printf("F32 grid (%d,%d,%d) KS %d steps %d loop_end %lld:", gridDim.x, gridDim.y, gridDim.z, KS, my_steps, clock64() - f0);
+    for (int i = 0; i < my_steps && i < 32; ++i) printf(" %lld", f_t[i]);
+    printf("\n");
+  }
+#endif
   if (KS > 1) {
     // fixed-order sum of the groups' partial tiles: group g parks its tile in its own (now idle)
     // operand ring, group 0 adds them in the order 1, 2, ...
@@ -163,23 +215,23 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p_in,
   }
 
   const int n = n0 + tx * 4;
-  if (n < p.C_out) {
+  if (n < C_out) {
     const float4 bias = *reinterpret_cast<const float4*>(p.bias + n);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int row = m0 + ty * 4 + i;
-      if (row >= p.T_in) continue;
-      const long long t_in = p.pos_in + row;
+      if (row >= T_in) continue;
+      const long long t_in = pos_in + row;
       float4 v = make_float4(acc[i][0] + bias.x, acc[i][1] + bias.y, acc[i][2] + bias.z, acc[i][3] + bias.w);
       if (p.residual_silu) {
-        const float4 x = *reinterpret_cast<const float4*>(in_row_ptr(p, t_in) + n);
+        const float4 x = *reinterpret_cast<const float4*>(in_row_ptr(in_direct, pos_in, in_ring, in_mask, C_in, t_in) + n);
         v = make_float4(x.x + silu_f(v.x), x.y + silu_f(v.y), x.z + silu_f(v.z), x.w + silu_f(v.w));
       }
       if (p.post_silu) v = make_float4(silu_f(v.x), silu_f(v.y), silu_f(v.z), silu_f(v.w));
       const long long t_out = (long long)p.n_phase * t_in + phase;
-      float* dst = (p.out_direct != nullptr)
-                       ? p.out_direct + (t_out - p.pos_out) * p.C_out + n
-                       : p.out_ring + (long long)((int)(t_out & (long long)p.out_mask)) * p.C_out + n;
+      float* dst = (out_direct != nullptr)
+                       ? out_direct + (t_out - pos_out) * C_out + n
+                       : p.out_ring + (long long)((int)(t_out & (long long)p.out_mask)) * C_out + n;
       *reinterpret_cast<float4*>(dst) = v;
     }
   }
@@ -188,12 +240,12 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p_in,
   // caller's chunk, written into ring rows that no CTA of this launch reads (distinct logical
   // frames map to distinct rows because the ring holds f_chunk + halo frames).
   if (p.save_ring != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
-    const int first = p.T_in > p.save_rows ? p.T_in - p.save_rows : 0;
-    const int c4 = p.C_in >> 2;
-    for (int i = tid; i < (p.T_in - first) * c4; i += NTG) {
+    const int first = T_in > p.save_rows ? T_in - p.save_rows : 0;
+    const int c4 = C_in >> 2;
+    for (int i = tid; i < (T_in - first) * c4; i += NTG) {
       const int r = first + i / c4, c = (i - (i / c4) * c4) * 4;
-      const float4 v = *reinterpret_cast<const float4*>(p.in_direct + (long long)r * p.C_in + c);
-      *reinterpret_cast<float4*>(p.save_ring + (long long)((int)((p.pos_in + r) & (long long)p.in_mask)) * p.C_in + c) = v;
+      const float4 v = *reinterpret_cast<const float4*>(in_direct + (long long)r * C_in + c);
+      *reinterpret_cast<float4*>(p.save_ring + (long long)((int)((pos_in + r) & (long long)in_mask)) * C_in + c) = v;
     }
   }
 }
