@@ -130,6 +130,22 @@ def attention_bytes_per_launch(cfg, n_streams: int) -> float:
     return n_streams * (2.0 * L * cfg.hidden * 2 + 2.0 * cfg.f_chunk * cfg.hidden * 2)
 
 
+def max_over_ranks(value: float, world: int, device: str = "cuda") -> float:
+    """Max of a per-rank scalar over all ranks (the replicas only meet here and at the barrier)."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(world: int, streams_per_rank: int, steps: int, per_chunk: float, seconds: float) -> float:
+    """Whole-job units per second: every rank advances its own streams by `steps` chunks (weak scaling)."""
+    return world * streams_per_rank * steps * per_chunk / seconds
+
+
 def cpu_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -255,12 +271,8 @@ def main():
     clocks = sampler.stop()
     c1 = model.counters()
     step_ms = sorted(evs[k].elapsed_time(evs[k + 1]) for k in range(K))
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    value = world * S * K * per_chunk / (total_ms * 1e-3)
+    total_ms = max_over_ranks(total_ms, world)
+    value = aggregate_throughput(world, S, K, per_chunk, total_ms * 1e-3)
 
     # ---- end to end through the host-buffer entry points (H2D + decode + D2H + sync per step) ----
     fin = [feats_h[r].pin_memory() for r in range(history + W, rounds)]
@@ -279,12 +291,8 @@ def main():
     for k in range(K):
         e2e_step(k)
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * S * K * per_chunk / e2e_s
+    e2e_s = max_over_ranks(e2e_s, world)
+    e2e_value = aggregate_throughput(world, S, K, per_chunk, e2e_s)
 
     # ---- per-kernel-class device time (separate profiled pass; events between launches slow the step) ----
     pk, how = peaks()

@@ -150,7 +150,8 @@ dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
 
 /* Convenience for callers with host buffers: copies feats_host to the device,
  * decodes, copies the result back and synchronises cuda_stream.  Uses staging
- * buffers owned by the stream (allocated at dc_stream_open). */
+ * buffers owned by the stream (allocated at dc_stream_open).  Returns DC_ERR_TIMEOUT
+ * (and poisons the stream until dc_stream_reset) if a bounded device-side wait gave up. */
 dc_status dc_decode_chunk_host(dc_stream* stream, const float* feats_host, int n_frames,
                                float* out_host, int* n_out, void* cuda_stream);
 
@@ -213,7 +214,8 @@ dc_status dc_conv_stack_noalloc(const float* weights_dev, int hidden, int n_conv
 dc_status dc_stream_carry_info(const dc_stream* stream, uint64_t* out, int max_entries, int* n_entries);
 
 /* counters[0] chunks decoded, [1] frames decoded, [2] calls rejected (DC_ERR_FRAMES),
- * [3] calls rejected (other argument/state errors), [4] device timeouts,
+ * [3] calls rejected (other argument/state errors), [4] device timeouts (this call reads the
+ * device-side error word synchronously, so it also reports timeouts of asynchronous decode calls),
  * [5] kernel launches issued, [6] streams open, [7] reserved. */
 dc_status dc_get_counters(const dc_model* model, uint64_t counters[8]);
 

@@ -606,6 +606,15 @@ extern "C" dc_status dc_decode_chunk_host(dc_stream* s, const float* feats_host,
   if (st != DC_OK) return st;
   DC_CUDA(cudaMemcpyAsync(out_host, s->stage_out, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaStreamSynchronize(cs));
+  if (m->flow) {
+    const int code = dc::flow_take_device_error(m->flow);
+    if (code != 0) {   // a bounded device-side wait gave up: the chunk's result is not valid
+      m->counters[4]++;
+      s->poisoned = true;
+      dc::set_error("device-side wait timed out (code %d)", code);
+      return DC_ERR_TIMEOUT;
+    }
+  }
   if (n_out) *n_out = n;
   return DC_OK;
 }
@@ -632,6 +641,15 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
     DC_CUDA(cudaMemcpyAsync(out_host[i], streams[i]->stage_out, (size_t)n_frames[i] * m->out_per_frame * sizeof(float),
                             cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaStreamSynchronize(cs));
+  {
+    const int code = dc::flow_take_device_error(m->flow);
+    if (code != 0) {
+      m->counters[4]++;
+      for (int i = 0; i < n; ++i) streams[i]->poisoned = true;
+      dc::set_error("device-side wait timed out (code %d)", code);
+      return DC_ERR_TIMEOUT;
+    }
+  }
   return DC_OK;
 }
 
@@ -673,6 +691,10 @@ extern "C" dc_status dc_profile_end(dc_model* m, double ms[8], uint64_t launches
 
 extern "C" dc_status dc_get_counters(const dc_model* m, uint64_t counters[8]) {
   if (!m || !counters) return DC_ERR_ARG;
+  if (m->flow) {   // synchronous read of the device error word (asynchronous decode calls cannot see it)
+    const int code = dc::flow_take_device_error(m->flow);
+    if (code > 0) const_cast<dc_model*>(m)->counters[4]++;
+  }
   for (int i = 0; i < 8; ++i) counters[i] = m->counters[i].load();
   return DC_OK;
 }

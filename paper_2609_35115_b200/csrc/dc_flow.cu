@@ -1131,6 +1131,13 @@ dc_status flow_state_reset(FlowModel*, FlowState* s, cudaStream_t st) {
   return DC_OK;
 }
 
+int flow_take_device_error(FlowModel* m) {
+  int v = 0;
+  if (cudaMemcpy(&v, m->d_err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  if (v != 0) cudaMemset(m->d_err, 0, sizeof(int));
+  return v;
+}
+
 void flow_state_close(FlowState* s) {
   if (!s) return;
   if (s->halo) cudaFree(s->halo);
