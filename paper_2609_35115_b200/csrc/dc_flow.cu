@@ -308,8 +308,10 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (src != nullptr) {
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
-          pre[2 * k] = *reinterpret_cast<const uint4*>(src + 16 * (2 * k + half));
-          pre[2 * k + 1] = *reinterpret_cast<const uint4*>(src + 16 * (2 * k + half) + 8);
+          if (16 * (2 * k + half) < p.BN) {
+            pre[2 * k] = *reinterpret_cast<const uint4*>(src + 16 * (2 * k + half));
+            pre[2 * k + 1] = *reinterpret_cast<const uint4*>(src + 16 * (2 * k + half) + 8);
+          }
         }
       }
     }
@@ -869,8 +871,11 @@ struct FlowModel {
   float* fconst = nullptr;   // biases and the timestep-bias table
   SlotInfo* d_slots = nullptr;
   int*   d_err = nullptr;
-  CUtensorMap tmAin, tmXa, tmXb, tmU, tmO, tmWin, tmWout;
-  std::vector<CUtensorMap> tmWconv, tmWqkv, tmWo;
+  CUtensorMap tmAin, tmXa, tmXb, tmU, tmO;
+  // weight maps in three tile-width variants v (box rows = N tile): v = 0 wide (64 / 192 / mel), for full
+  // batches; v = 1, 2 narrower (32, 16 / 96, 48 / 16), so that a small batch still spreads over many SMs
+  CUtensorMap tmWin[3], tmWout[3];
+  std::vector<CUtensorMap> tmWconv[3], tmWqkv[3], tmWo[3];
   // float offsets into fconst
   size_t o_bin = 0, o_bout = 0, o_tau = 0;
   std::vector<size_t> o_bconv, o_bqkv, o_bo;
@@ -1058,15 +1063,18 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   ok &= make_tmap(&m->tmXb, m->Xb, R, C, A_ROWS);
   ok &= make_tmap(&m->tmU, m->U, R, C, A_ROWS);
   ok &= make_tmap(&m->tmO, m->O, R, C, A_ROWS);
-  ok &= make_tmap(&m->tmWin, m->wts + w_in, C, m->Kin, 64);
-  ok &= make_tmap(&m->tmWout, m->wts + w_out, mel, C, mel);
-  m->tmWconv.resize(nL);
-  m->tmWqkv.resize(nA);
-  m->tmWo.resize(nA);
-  for (int i = 0; i < nL; ++i) ok &= make_tmap(&m->tmWconv[i], m->wts + w_conv[i], C, 3 * C, 64);
-  for (int i = 0; i < nA; ++i) {
-    ok &= make_tmap(&m->tmWqkv[i], m->wts + w_qkv[i], 3 * C, C, 192);
-    ok &= make_tmap(&m->tmWo[i], m->wts + w_o[i], C, C, 64);
+  for (int v = 0; v < 3; ++v) {
+    const int bn = 64 >> v, bq = 192 >> v, bo = v == 0 ? mel : 16;
+    ok &= make_tmap(&m->tmWin[v], m->wts + w_in, C, m->Kin, bn);
+    ok &= make_tmap(&m->tmWout[v], m->wts + w_out, mel, C, bo);
+    m->tmWconv[v].resize(nL);
+    m->tmWqkv[v].resize(nA);
+    m->tmWo[v].resize(nA);
+    for (int i = 0; i < nL; ++i) ok &= make_tmap(&m->tmWconv[v][i], m->wts + w_conv[i], C, 3 * C, bn);
+    for (int i = 0; i < nA; ++i) {
+      ok &= make_tmap(&m->tmWqkv[v][i], m->wts + w_qkv[i], 3 * C, C, bq);
+      ok &= make_tmap(&m->tmWo[v][i], m->wts + w_o[i], C, C, bn);
+    }
   }
   if (!ok) {
     set_error("cuTensorMapEncodeTiled failed or is unavailable");
@@ -1191,6 +1199,10 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
   launch(lc, flow_prep_kernel, dim3(n), dim3(128), 0, true, 4, (const SlotInfo*)m->d_slots, mel, m->xstate, m->Ain, m->Kin);
 
   const int m_tiles = (n * SLOT_ROWS + TILE_M - 1) / TILE_M;
+  // N-tile variant: the widest whose C-wide GEMMs still give about 96 CTAs, else the narrowest
+  int v = 0;
+  while (v < 2 && m_tiles * (C / (64 >> v)) < 96) ++v;
+  const int bn = 64 >> v, bq = 192 >> v, bo = v == 0 ? mel : 16;
   auto gemm = [&](const CUtensorMap& tA, const CUtensorMap& tB, GemmParams& p, int N) {
     p.n_slots = n;
     p.slots = m->d_slots;
@@ -1228,10 +1240,10 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     auto swap = [&]() { std::swap(X, Y); std::swap(tX, tY); };
     {
       GemmParams p{};
-      p.mode = MODE_INPROJ; p.BN = 64; p.n_kblocks = m->Kin / KBLK; p.taps = 1;
+      p.mode = MODE_INPROJ; p.BN = bn; p.n_kblocks = m->Kin / KBLK; p.taps = 1;
       p.bias = fc + m->o_bin; p.out = X;
       p.halo_off = ((long long)s * c.n_conv + 0) * halo_stride;
-      gemm(m->tmAin, m->tmWin, p, C);
+      gemm(m->tmAin, m->tmWin[v], p, C);
     }
     int l = 0;
     const int n_groups = c.n_attn > 0 ? c.n_attn : 1;
@@ -1239,31 +1251,31 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       for (int j = 0; j < m->cpa; ++j, ++l) {
         const int d = c.dilations[l];
         GemmParams p{};
-        p.mode = MODE_CONV; p.BN = 64; p.n_kblocks = C / KBLK; p.taps = 3;
+        p.mode = MODE_CONV; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 3;
         p.shift[0] = 2 * d; p.shift[1] = d; p.shift[2] = 0;
         p.bias = fc + m->o_bconv[l]; p.tau = fc + m->o_tau + ((size_t)s * c.n_conv + l) * C;
         p.resid = X; p.out = Y;
         const bool next_is_conv = (j + 1 < m->cpa);
         p.halo_off = next_is_conv ? ((long long)s * c.n_conv + l + 1) * halo_stride : -1;
-        gemm(*tX, m->tmWconv[l], p, C);
+        gemm(*tX, m->tmWconv[v][l], p, C);
         swap();
       }
       if (c.n_attn > 0) {
         rmsnorm(X);
         {
           GemmParams p{};
-          p.mode = MODE_QKV; p.BN = 192; p.n_kblocks = C / KBLK; p.taps = 1;
+          p.mode = MODE_QKV; p.BN = bq; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bqkv[g]; p.q_out = m->Q; p.halo_off = -1;
           p.kv_off = ((long long)s * c.n_attn + g) * 2 * m->Rk * C;
-          gemm(m->tmU, m->tmWqkv[g], p, 3 * C);
+          gemm(m->tmU, m->tmWqkv[v][g], p, 3 * C);
         }
         attention(s, g);
         {
           GemmParams p{};
-          p.mode = MODE_OPROJ; p.BN = 64; p.n_kblocks = C / KBLK; p.taps = 1;
+          p.mode = MODE_OPROJ; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bo[g]; p.resid = X; p.out = Y;
           p.halo_off = (l < c.n_conv) ? ((long long)s * c.n_conv + l) * halo_stride : -1;
-          gemm(m->tmO, m->tmWo[g], p, C);
+          gemm(m->tmO, m->tmWo[v][g], p, C);
           swap();
         }
       }
@@ -1271,11 +1283,11 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     rmsnorm(X);
     {
       GemmParams p{};
-      p.mode = MODE_OUT; p.BN = mel; p.n_kblocks = C / KBLK; p.taps = 1;
+      p.mode = MODE_OUT; p.BN = bo; p.n_kblocks = C / KBLK; p.taps = 1;
       p.bias = fc + m->o_bout; p.halo_off = -1;
       p.xstate = m->xstate; p.ain = m->Ain; p.ld_ain = m->Kin; p.inv_n = 1.0f / c.n_steps;
       p.last_step = (s == c.n_steps - 1); p.mel = mel;
-      gemm(m->tmU, m->tmWout, p, mel);
+      gemm(m->tmU, m->tmWout[v], p, mel);
     }
   }
 }
