@@ -44,7 +44,7 @@ constexpr int GEMM_TILE_SMEM = 88 * 1024;    // operand stages per CTA: small en
 constexpr int A_ROWS = TILE_M + HALO;  // the A tile carries 8 extra leading rows so that all taps read it
 constexpr int A_BYTES = A_ROWS * 128;
 constexpr int MAX_BN = 192;
-constexpr int GEMM_THREADS = 352;      // warp 0 TMA (A), warp 1 UMMA, warp 2 TMA (B), warps 3..10 epilogue
+constexpr int GEMM_THREADS = 384;      // warp 0 TMA (A), warps 1 and 3 UMMA issuers, warp 2 TMA (B), warps 4..11 epilogue
 constexpr int EPI_THREADS = 256;
 constexpr int MAX_SLOTS_PER_SET = 64;
 
@@ -69,6 +69,7 @@ struct SlotSet {
 struct GemmParams {
   int          mode;
   int          BN;              // output columns per CTA (multiple of 16, <= 128)
+  int          n_issuers;       // 1 or 2 UMMA-issuing threads (2: even / odd reduction blocks, own accumulators)
   int          n_stages;        // TMA pipeline depth (<= MAX_STAGES, n_stages * stage bytes <= GEMM_TILE_SMEM)
   int          n_slots;
   int          n_kblocks;       // 64-wide channel blocks of the A matrix (one pipeline stage each)
@@ -152,7 +153,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * TILE_M, n0 = blockIdx.y * p.BN;
 #ifdef DC_TIMING
-  const bool tm = blockIdx.x == 1 && blockIdx.y == 1 && p.mode == MODE_CONV;
+  const bool tm = blockIdx.x == 0 && blockIdx.y == 1 && p.mode == MODE_CONV;
   long long t_start = 0;
   if (tm) t_start = clock64();
   __shared__ long long s_t[8];
@@ -162,14 +163,17 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #else
 #define DC_T(tag) do {} while (0)
 #endif
-  const uint32_t tmem_cols = p.BN <= 32 ? 32u : (p.BN <= 64 ? 64u : (p.BN <= 128 ? 128u : 256u));
+  // second issuer's accumulator sits acc2_off columns after the first
+  const uint32_t acc2_off = p.BN <= 32 ? 32u : 64u;
+  const uint32_t need_cols = p.n_issuers == 2 ? 2u * acc2_off : (uint32_t)p.BN;
+  const uint32_t tmem_cols = need_cols <= 32 ? 32u : (need_cols <= 64 ? 64u : (need_cols <= 128 ? 128u : 256u));
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
       ptx::mbar_init(&full[i], 2);   // one arrival per producer thread
       ptx::mbar_init(&empty[i], 1);
     }
-    ptx::mbar_init(accum, 1);
+    ptx::mbar_init(accum, (uint32_t)p.n_issuers);
     *s_fail = 0;
     ptx::fence_barrier_init();
   }
@@ -198,7 +202,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (is_a) ptx::pdl_wait();   // activations come from the previous kernel; weights do not
       for (int kb = 0; kb < nkb; ++kb) {
         if (kb >= STAGES && !ptx::mbar_wait(&empty[st], phase)) {
-          atomicExch(p.err, 1);
+          atomicCAS(p.err, 0, 1 | (is_a ? 0 : 0x10) | (p.mode << 8) | (kb << 12) | ((int)blockIdx.x << 20));
           *s_fail = 1;
           break;
         }
@@ -225,22 +229,26 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       if (is_a && on) DC_T(1);
     }
-  } else if (warp == 1) {
-    {
+  } else if (warp == 1 || warp == 3) {
+    // UMMA issuers.  A single thread spends about 100 cycles per tcgen05.mma it issues, more than a
+    // narrow UMMA takes to execute, so two warps issue alternate reduction blocks into accumulators
+    // of their own; the epilogue adds the two in a fixed order.
+    const int me = warp >> 1;                     // 0 or 1
+    if (me < p.n_issuers) {
       const uint32_t on = lane == 0;
       const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.BN, 0, 0);
-      const int nkb = p.n_kblocks, taps = p.taps;
+      const int nkb = p.n_kblocks, taps = p.taps, step = p.n_issuers;
+      const uint32_t d_acc = tmem_base + (uint32_t)me * acc2_off;
       // descriptor start addresses are in 16-byte units: +2 per 32-byte K step
       const uint64_t d_a0 = ptx::umma_desc_sw128(ptx::smem_u32(smem));
       const uint32_t stage16 = stage_bytes >> 4, b16 = b_tile >> 4, ab16 = A_BYTES >> 4;
       const uint32_t o0 = (uint32_t)(HALO - p.shift[0]) * 8u, o1 = (uint32_t)(HALO - p.shift[1]) * 8u,
                      o2 = (uint32_t)(HALO - p.shift[2]) * 8u;   // row offset of tap j: rows * 128 B / 16
-      int st = 0;
-      uint32_t phase = 0, acc = 0;
-      uint64_t d_st = d_a0;
-      for (int kb = 0; kb < nkb; ++kb) {
-        if (!ptx::mbar_wait(&full[st], phase)) {
-          atomicExch(p.err, 2);
+      uint32_t acc = 0;
+      for (int kb = me; kb < nkb; kb += step) {
+        const int st = kb % STAGES;
+        if (!ptx::mbar_wait(&full[st], (uint32_t)(kb / STAGES) & 1u)) {
+          atomicCAS(p.err, 0, 2 | (me << 4) | (p.mode << 8) | (kb << 12) | ((int)blockIdx.x << 20));
           *s_fail = 1;
           break;
         }
@@ -249,30 +257,24 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #ifdef DC_TIMING
         if (tm && kb < 32 && on) s_k[kb] = clock64() - t_start;
 #endif
-        const uint64_t da = d_st, db = d_st + ab16;
+        const uint64_t da = d_a0 + (uint64_t)((uint32_t)st * stage16), db = da + ab16;
         if (taps == 3) {
-          ptx::umma_bf16_if(on, tmem_base, da + o0, db, idesc, acc);
+          ptx::umma_bf16_if(on, d_acc, da + o0, db, idesc, acc);
 #pragma unroll
-          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, tmem_base, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
+          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, tmem_base, da + (o1 + 2 * k), db + (b16 + 2 * k), idesc, 1);
+          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o1 + 2 * k), db + (b16 + 2 * k), idesc, 1);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, tmem_base, da + (o2 + 2 * k), db + (2 * b16 + 2 * k), idesc, 1);
+          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o2 + 2 * k), db + (2 * b16 + 2 * k), idesc, 1);
         } else {
-          ptx::umma_bf16_if(on, tmem_base, da + o0, db, idesc, acc);
+          ptx::umma_bf16_if(on, d_acc, da + o0, db, idesc, acc);
 #pragma unroll
-          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, tmem_base, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
+          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
         }
         acc = 1;
         ptx::umma_commit_if(on, &empty[st]);
-        d_st += stage16;
-        if (++st == STAGES) {
-          st = 0;
-          d_st = d_a0;
-          phase ^= 1;
-        }
       }
-      if (on) DC_T(3);
+      if (on && me == 0) DC_T(3);
       ptx::umma_commit_if(on, accum);   // arrives when every UMMA above has finished (also on the failure path)
     }
   } else {
@@ -280,14 +282,14 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // Everything that does not depend on the accumulator is fetched while the main loop runs:
     // per-column constants go to shared memory, the thread's residual row (or, for a left-context
     // row, the carried row) goes to registers.
-    const int et = threadIdx.x - 96;
+    const int et = threadIdx.x - 128;
     if (et < p.BN) {   // BN <= 192 < EPI_THREADS
       s_bias[et] = p.bias[n0 + et];
       s_tau[et] = p.tau != nullptr ? p.tau[n0 + et] : 0.f;
     }
     ptx::pdl_wait();                              // slot table, residual and carry rows are upstream data
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
-    const int half = (warp - 3) >> 2;             // which chunks of the row: chunk index & 1 == half
+    const int half = (warp - 4) >> 2;             // which chunks of the row: chunk index & 1 == half
     const int r = m0 + q * 32 + lane;             // row in slot layout (without GUARD)
     const int slot = r / SLOT_ROWS, rho = r % SLOT_ROWS;
     const bool in_range = slot < p.n_slots;
@@ -321,8 +323,8 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     const bool got = ptx::mbar_wait_relaxed(accum, 0);
     ptx::tc_fence_after();
-    if (threadIdx.x == 96) DC_T(4);
-    if (!got) atomicExch(p.err, 3);
+    if (threadIdx.x == 128) DC_T(4);
+    if (!got) atomicCAS(p.err, 0, 3 | (p.mode << 8));
     const bool slot_ok = in_range && got && *s_fail == 0;
     const bool is_halo = slot_ok && rho < HALO;
     const bool is_chunk = slot_ok && f >= 0 && f < si.T;
@@ -336,6 +338,12 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (c0 >= p.BN) break;
       float acc[16];
       ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
+      if (p.n_issuers == 2) {   // even blocks + odd blocks, always in this order
+        float acc2[16];
+        ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + acc2_off + (uint32_t)c0, acc2);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] += acc2[i];
+      }
       const int n = n0 + c0;
 #pragma unroll
       for (int i = 0; i < 16; ++i) acc[i] += s_bias[c0 + i];
@@ -408,11 +416,11 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (is_chunk || (is_halo && do_halo)) store16(p.out + grow * p.ld + n, va, vb);
       // shift the carry by T frames: [old carry | chunk] -> its last 8 rows
       if (carry_wr) store16(carry + new_row * p.C + n, va, vb);
-      if (threadIdx.x == 96 && kk == 0) DC_T(6);
-      if (threadIdx.x == 96 && kk == 1) DC_T(7);
+      if (threadIdx.x == 128 && kk == 0) DC_T(6);
+      if (threadIdx.x == 128 && kk == 1) DC_T(7);
     }
   }
-  if (threadIdx.x == 96) DC_T(5);
+  if (threadIdx.x == 128) DC_T(5);
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 1) ptx::tmem_dealloc(tmem_base, tmem_cols);
@@ -846,7 +854,8 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, u
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr size_t GEMM_SMEM = 1024 + GEMM_TILE_SMEM + 2 * MAX_STAGES * 8 + 8 + 8 + 2 * MAX_BN * 4 + 64;
+constexpr size_t GEMM_SMEM_EXTRA = 1024 + 2 * MAX_STAGES * 8 + 8 + 8 + 2 * MAX_BN * 4 + 64;   // alignment slack + barriers + constants
+constexpr size_t GEMM_SMEM_MAX = 200 * 1024;
 
 }  // namespace
 
@@ -883,6 +892,8 @@ struct FlowModel {
   Profiler* prof = nullptr;
   // launch plumbing
   bool pdl = true;                       // programmatic dependent launch between the step's kernels
+  bool one_issuer = false;               // experiments: a single UMMA issuer
+  int  wide_stages = 4;                  // 2 or 4 (even, see the stage count rule in enqueue_chunk)
   int  dbg = 0;
   cudaStream_t cap_stream = nullptr;     // used only to capture graphs at create
   std::map<int, GraphEntry> graphs;      // batch size -> captured chunk step
@@ -1048,7 +1059,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   if (e == cudaSuccess) chk(cudaMemcpy(m->wts, hw.data(), wn * sizeof(uint16_t), cudaMemcpyHostToDevice));
   if (e == cudaSuccess) chk(cudaMemcpy(m->fconst, hf.data(), fn * sizeof(float), cudaMemcpyHostToDevice));
   if (e == cudaSuccess)
-    chk(cudaFuncSetAttribute(flow_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM));
+    chk(cudaFuncSetAttribute(flow_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
   if (e == cudaSuccess && cfg.n_attn > 0)
     chk(cudaFuncSetAttribute(flow_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATT_SMEM));
   if (e != cudaSuccess) {
@@ -1087,6 +1098,10 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     m->pdl = !(e && atoi(e));
     const char* d = getenv("DC_GEMM_DBG");
     m->dbg = d ? atoi(d) : 0;
+    const char* oi = getenv("DC_ONE_ISSUER");
+    m->one_issuer = oi && atoi(oi);
+    const char* ws = getenv("DC_GEMM_STAGES");
+    if (ws && (atoi(ws) == 2 || atoi(ws) == 4)) m->wide_stages = atoi(ws);
     const char* g = getenv("DC_NO_GRAPH");
     if (!(g && atoi(g)) && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) == cudaSuccess) {
       // the two batch sizes that matter are captured now, so that no decode call ever builds a graph:
@@ -1142,7 +1157,10 @@ dc_status flow_state_reset(FlowModel*, FlowState* s, cudaStream_t st) {
 int flow_take_device_error(FlowModel* m) {
   int v = 0;
   if (cudaMemcpy(&v, m->d_err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
-  if (v != 0) cudaMemset(m->d_err, 0, sizeof(int));
+  if (v != 0) {
+    cudaMemset(m->d_err, 0, sizeof(int));
+    if (getenv("DC_VERBOSE")) fprintf(stderr, "[dc] device error word 0x%x\n", v);
+  }
   return v;
 }
 
@@ -1211,9 +1229,23 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     p.Rk = m->Rk;
     p.err = m->d_err;
     const int stage_bytes = A_BYTES + p.taps * ((p.BN * 128 + 1023) & ~1023);
-    p.n_stages = std::min(MAX_STAGES, GEMM_TILE_SMEM / stage_bytes);
     p.dbg = m->dbg;
-    launch(lc, flow_gemm_kernel, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), GEMM_SMEM, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
+    // the issuer count fixes the summation order, so it depends on the GEMM's role only, never on the tile
+    // width chosen for the batch size (batched and single-stream results must agree bit for bit);
+    // the QKV and output projections keep one issuer (their wide tiles would not fit two accumulators)
+    p.n_issuers = (p.mode != MODE_QKV && p.mode != MODE_OUT && p.n_kblocks >= 2 && !m->one_issuer) ? 2 : 1;
+    // Stage count.  Two or three stages (<= 88 KB) let two CTAs share an SM, so that the next kernel's
+    // prologue overlaps this kernel's tail.  With two issuers the count must be EVEN: issuer i takes
+    // the reduction blocks kb = i (mod 2), and only with an even ring does every stage always belong
+    // to the same issuer - a parity wait cannot tell "my block has landed" from "the other issuer's
+    // earlier block has landed" on a stage that both use.
+    if (p.n_issuers == 2) {
+      p.n_stages = (p.n_kblocks >= 4 && (4 * stage_bytes <= 104 * 1024 || stage_bytes > 32 * 1024)) ? m->wide_stages : 2;
+    } else {
+      p.n_stages = std::max(1, std::min(std::min(MAX_STAGES, GEMM_TILE_SMEM / stage_bytes), p.n_kblocks));
+    }
+    const size_t smem = GEMM_SMEM_EXTRA + (size_t)p.n_stages * stage_bytes;
+    launch(lc, flow_gemm_kernel, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), smem, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
   };
   auto rmsnorm = [&](const bf16* x) {
     const int warps = n * SLOT_ROWS;
