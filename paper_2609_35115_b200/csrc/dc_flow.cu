@@ -893,6 +893,7 @@ struct FlowModel {
   // launch plumbing
   bool pdl = true;                       // programmatic dependent launch between the step's kernels
   bool one_issuer = false;               // experiments: a single UMMA issuer
+  int  qkv_stages = 4;
   int  wide_stages = 4;                  // 2 or 4 (even, see the stage count rule in enqueue_chunk)
   int  dbg = 0;
   cudaStream_t cap_stream = nullptr;     // used only to capture graphs at create
@@ -1075,7 +1076,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   ok &= make_tmap(&m->tmU, m->U, R, C, A_ROWS);
   ok &= make_tmap(&m->tmO, m->O, R, C, A_ROWS);
   for (int v = 0; v < 3; ++v) {
-    const int bn = 64 >> v, bq = 192 >> v, bo = v == 0 ? mel : 16;
+    const int bn = 64 >> v, bq = 192 >> v, bo = 16;
     ok &= make_tmap(&m->tmWin[v], m->wts + w_in, C, m->Kin, bn);
     ok &= make_tmap(&m->tmWout[v], m->wts + w_out, mel, C, bo);
     m->tmWconv[v].resize(nL);
@@ -1100,6 +1101,8 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     m->dbg = d ? atoi(d) : 0;
     const char* oi = getenv("DC_ONE_ISSUER");
     m->one_issuer = oi && atoi(oi);
+    const char* qs = getenv("DC_QKV_STAGES");
+    if (qs && atoi(qs) >= 2 && atoi(qs) <= 4) m->qkv_stages = atoi(qs);
     const char* ws = getenv("DC_GEMM_STAGES");
     if (ws && (atoi(ws) == 2 || atoi(ws) == 4)) m->wide_stages = atoi(ws);
     const char* g = getenv("DC_NO_GRAPH");
@@ -1220,7 +1223,9 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
   // N-tile variant: the widest whose C-wide GEMMs still give about 96 CTAs, else the narrowest
   int v = 0;
   while (v < 2 && m_tiles * (C / (64 >> v)) < 96) ++v;
-  const int bn = 64 >> v, bq = 192 >> v, bo = v == 0 ? mel : 16;
+  // the output projection always uses 16-column tiles: mel/16 CTAs per row tile instead of one, and a
+  // single Euler-state round trip per epilogue thread
+  const int bn = 64 >> v, bq = 192 >> v, bo = 16;
   auto gemm = [&](const CUtensorMap& tA, const CUtensorMap& tB, GemmParams& p, int N) {
     p.n_slots = n;
     p.slots = m->d_slots;
@@ -1243,6 +1248,8 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       p.n_stages = (p.n_kblocks >= 4 && (4 * stage_bytes <= 104 * 1024 || stage_bytes > 32 * 1024)) ? m->wide_stages : 2;
     } else {
       p.n_stages = std::max(1, std::min(std::min(MAX_STAGES, GEMM_TILE_SMEM / stage_bytes), p.n_kblocks));
+      // the wide QKV tiles fill the GPU with one CTA per SM anyway: a deeper ring hides the load latency
+      if (p.mode == MODE_QKV && stage_bytes > 32 * 1024 && p.n_kblocks >= 4) p.n_stages = m->qkv_stages;
     }
     const size_t smem = GEMM_SMEM_EXTRA + (size_t)p.n_stages * stage_bytes;
     launch(lc, flow_gemm_kernel, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), smem, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
