@@ -520,7 +520,7 @@ constexpr int ATT_TMEM_COLS = 256;      // S (128 columns) + O (64 columns); two
 constexpr int ATT_K_LOADERS = 64;       // warps 2 and 6: Q, then the K blocks
 constexpr int ATT_V_LOADERS = 32;       // warp 7: the V blocks
 constexpr int ATT_Q_BYTES = 64 * 128;   // 64 query rows; the UMMA's rows 64..127 alias the P region
-constexpr int ATT_P_BYTES = 2 * 2 * 64 * 128;       // two P buffers (even / odd blocks) of two 64-key tiles
+constexpr int ATT_P_BYTES = 2 * 64 * 128;
 constexpr int ATT_STAGE_BYTES = 2 * ATT_KB * 128;   // K block + V block
 constexpr size_t ATT_SMEM = 1024 + ATT_Q_BYTES + ATT_P_BYTES + ATT_STAGES * ATT_STAGE_BYTES + 1024;
 constexpr float ATT_RESCALE_LOG2 = 8.0f;
@@ -551,7 +551,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;
-  uint8_t* sP = sQ + ATT_Q_BYTES;                    // buffer j (blocks b = j mod 2) at + 16384 j, its tile t (keys 64 t ..) at + 8192 t
+  uint8_t* sP = sQ + ATT_Q_BYTES;                    // tile t (keys 64 t .. 64 t + 63 of the block) at + 8192 t
   uint8_t* ring = sP + ATT_P_BYTES;
   // K and V have their own two-stage rings: a K stage is free as soon as S of its block has been
   // computed, long before the V stage of the same block (free after P V), so K runs further ahead.
@@ -561,8 +561,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   uint64_t* empty_v = full_v + ATT_STAGES;
   uint64_t* bar_s = empty_v + ATT_STAGES;
   uint64_t* bar_p = bar_s + 1;
-  uint64_t* bar_pv = bar_p + 1;         // [2]: P V of even / odd blocks (a P buffer is reused two blocks later)
-  uint64_t* bar_sfree = bar_pv + 2;     // every softmax thread has copied its S columns to registers
+  uint64_t* bar_pv = bar_p + 1;
+  uint64_t* bar_sfree = bar_pv + 1;     // every softmax thread has copied its S columns to registers
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_sfree + 1);
   float* s_x = reinterpret_cast<float*>(tmem_slot + 2);   // [2][64] exchange between the two column halves
 
@@ -570,7 +570,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   const int slot = blockIdx.x, head = blockIdx.y;
   const int chunks = p.dh >> 3;             // 16-byte chunks per head row
 #ifdef DC_TIMING
-  __shared__ long long a_t[128];
+  __shared__ long long a_t[64];
   const bool atm = blockIdx.x == 3 && blockIdx.y == 2;
   const long long a_start = clock64();
 #define DC_AT(i) do { if (atm) a_t[i] = clock64() - a_start; } while (0)
@@ -587,8 +587,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     }
     ptx::mbar_init(bar_s, 1);
     ptx::mbar_init(bar_p, 128);
-    ptx::mbar_init(&bar_pv[0], 1);
-    ptx::mbar_init(&bar_pv[1], 1);
+    ptx::mbar_init(bar_pv, 1);
     ptx::mbar_init(bar_sfree, 128);
     ptx::fence_barrier_init();
   }
@@ -685,22 +684,16 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
           issue_s(b + 1);
         }
         if (ok && !ptx::mbar_wait(bar_p, b & 1)) { ok = false; atomicExch(p.err, 6); }
-        if (b < 8) DC_AT(72 + b);
         if (ok && !ptx::mbar_wait(&full_v[st], (b / ATT_STAGES) & 1)) { ok = false; atomicExch(p.err, 11); }
         ptx::tc_fence_after();
         const uint64_t dv = ptx::umma_desc_sw128(ptx::smem_u32(ring + st * ATT_STAGE_BYTES + ATT_KB * 128));
         const int valid = L - b * ATT_KB;
         const int ksteps = valid >= ATT_KB ? ATT_KB / 16 : (valid + 15) / 16;
-        const uint64_t dpb = dp + (uint64_t)((b & 1) * (16384 >> 4));
-        // P tile k/4 (8 KB apart), 32-byte K steps; V: 16 key rows = 2 KB per step
-        ptx::umma_bf16(tmem_base + ATT_KB, dpb, dv, idesc_pv, b != 0);
-#pragma unroll
-        for (int k = 1; k < ATT_KB / 16; ++k)
-          if (k < ksteps)
-            ptx::umma_bf16(tmem_base + ATT_KB, dpb + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
-                           idesc_pv, 1);
+        for (int k = 0; k < ksteps; ++k)   // P tile k/4 (8 KB apart), 32-byte K steps; V: 16 key rows = 2 KB per step
+          ptx::umma_bf16(tmem_base + ATT_KB, dp + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
+                         idesc_pv, (b | k) != 0);
         ptx::umma_commit(&empty_v[st]);
-        ptx::umma_commit(&bar_pv[b & 1]);
+        ptx::umma_commit(bar_pv);
         if (b < 8) DC_AT(24 + b);                        // PV(b) issued
       }
     }
@@ -722,7 +715,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       for (int c = 0; c < 4; ++c) ptx::tmem_ld16(lane_addr + (uint32_t)(half * 64 + c * 16), v + 16 * c);
       ptx::tc_fence_before();
       ptx::mbar_arrive(bar_sfree);               // S(b) is in registers: the next block's scores may overwrite it
-      if (tid == 0 && b < 8) DC_AT(48 + b);
       if (valid < 64) {                          // only the last block has padded key columns
 #pragma unroll
         for (int i = 0; i < 64; ++i)
@@ -734,19 +726,15 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       s_x[half * 64 + row] = mx * p.scale_log2e;
       ptx::named_bar_sync(2, 128);
       mx = fmaxf(s_x[row], s_x[64 + row]);
-      if (tid == 0 && b < 8) DC_AT(56 + b);
-      if (b >= 2) {   // this block's P buffer was last read by P V of block b - 2
-        if (ok && !ptx::mbar_wait(&bar_pv[b & 1], ((b >> 1) - 1) & 1)) { ok = false; atomicExch(p.err, 8); }
+      if (b > 0) {   // P V of the previous block must be done: P tile free, O quiescent
+        if (ok && !ptx::mbar_wait(bar_pv, (b - 1) & 1)) { ok = false; atomicExch(p.err, 8); }
+        ptx::tc_fence_after();
       }
       if (b == 0) {
         m_ref = mx;
       } else {
         const bool need = mx > m_ref + ATT_RESCALE_LOG2;
         if (__any_sync(0xffffffffu, need)) {
-          // rare: O is rescaled in place, so P V of the previous block must have finished (P V of this
-          // block cannot have started: it needs the P written below)
-          if (ok && !ptx::mbar_wait(&bar_pv[(b - 1) & 1], ((b - 1) >> 1) & 1)) { ok = false; atomicExch(p.err, 12); }
-          ptx::tc_fence_after();
           const float alpha = need ? exp2f(m_ref - mx) : 1.0f;
           if (need) m_ref = mx;
           lsum *= alpha;
@@ -761,8 +749,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
           }
         }
       }
-      if (tid == 0 && b < 8) DC_AT(64 + b);
-      uint8_t* prow = sP + (b & 1) * 16384 + half * 8192 + row * 128;
+      uint8_t* prow = sP + half * 8192 + row * 128;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         float e[16];
@@ -781,7 +768,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       ptx::mbar_arrive(bar_p);
       if (tid == 0 && b < 8) DC_AT(40 + b);              // P(b) written
     }
-    if (ok && !ptx::mbar_wait(&bar_pv[(nkb - 1) & 1], ((nkb - 1) >> 1) & 1)) { ok = false; atomicExch(p.err, 9); }
+    if (ok && !ptx::mbar_wait(bar_pv, (nkb - 1) & 1)) { ok = false; atomicExch(p.err, 9); }
     ptx::tc_fence_after();
     ptx::named_bar_sync(2, 128);       // every thread is past its last read of s_x
     s_x[half * 64 + row] = lsum;
@@ -818,14 +805,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[40 + i]);
     printf("\n PV_issued:");
     for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[24 + i]);
-    printf("\n sm_ld_done:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[48 + i]);
-    printf("\n sm_max_xchg:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[56 + i]);
-    printf("\n sm_pv_waited:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[64 + i]);
-    printf("\n iss_p_ready:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[72 + i]);
     printf("\n");
   }
 #endif

@@ -13,6 +13,7 @@ def run_gpu_stream(model, feats: np.ndarray, boundaries, stream=None) -> np.ndar
     for c in range(len(boundaries) - 1):
         outs.append(st.decode_chunk(x[boundaries[c]:boundaries[c + 1]].contiguous()).clone())
     torch.cuda.synchronize()
+    assert model.counters()[4] == 0, "a bounded device-side wait timed out"
     if stream is None:
         st.close()
     return torch.cat([o.reshape(-1) if o.dim() == 1 else o for o in outs], dim=0).cpu().numpy()

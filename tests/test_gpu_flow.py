@@ -130,6 +130,7 @@ def test_cfg5_multi_stream_serving_full_size(dc):
         os_ = [outs[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
         dc.decode_batch(m, streams, fs, os_)
     torch.cuda.synchronize()
+    assert m.counters()[4] == 0, "a bounded device-side wait timed out"
     for st in streams:
         st.close()
     got = [o.cpu().numpy() for o in outs]
