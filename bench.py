@@ -154,14 +154,20 @@ def cpu_threads() -> int:
         return os.cpu_count() or 1
 
 
-def time_oracle(cfg, weights, feats, n_chunks: int):
-    """Times the oracle as it stands on n_chunks chunks of one stream; returns seconds."""
+def time_oracle(cfg, weights, feats, budget_s: float = 12.0, min_chunks: int = 8, max_chunks: int = 4000):
+    """Times the oracle as it stands on consecutive chunks of one stream until about budget_s
+    seconds of CPU work are done (the available input chunks are reused cyclically: their values
+    do not change the work).  Returns (chunks, seconds)."""
     from oracle import dc_oracle as orc
     st = orc.make_stream(cfg, weights)
+    avail = feats.shape[0] // cfg.f_chunk
     t0 = time.perf_counter()
-    for c in range(n_chunks):
+    n = 0
+    while n < max_chunks and (n < min_chunks or time.perf_counter() - t0 < budget_s):
+        c = n % avail
         st.decode_chunk(feats[c * cfg.f_chunk:(c + 1) * cfg.f_chunk])
-    return time.perf_counter() - t0
+        n += 1
+    return n, time.perf_counter() - t0
 
 
 def run_reference(args, cfg):
@@ -331,12 +337,10 @@ def main():
     # ---- the oracle on the host cores (rank 0, N = 1 only), bounded sample ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_c = {"cfg5": 40, "cfg3": 40, "cfg2": 40, "cfg4": 200, "cfg1": 8}[cfg.name]
         f = feats_h[:, 0].reshape(-1, cfg.in_dim).numpy()
-        n_c = min(n_c, f.shape[0] // T)
-        dt = time_oracle(cfg, weights, f, n_c)
+        n_c, dt = time_oracle(cfg, weights, f)
         cpu = {"value": n_c * per_chunk / dt, "unit": unit, "cores": cpu_threads(), "kind": "oracle",
-               "sample": f"first {n_c} chunks of stream 0 (carry growing from empty), {dt:.1f} s"}
+               "sample": f"{n_c} consecutive chunks of one stream (carry growing from empty), {dt:.1f} s"}
 
     if rank == 0:
         ws = (S * (cfg.n_steps * cfg.n_attn_layers * 2 * (cfg.kv_cap + T) * cfg.hidden * 2) / 1e6) if cfg.pipeline == "flow" else 0
