@@ -245,11 +245,12 @@ def main():
     feats_h = torch.from_numpy(rng.standard_normal((rounds, S, T, cfg.in_dim), dtype=np.float32))
     feats_d = feats_h.cuda()
     out_d = torch.empty(S, T * cfg.out_per_frame, device="cuda")
+    out_dv = out_d.view(S, T, -1) if cfg.pipeline != "vocoder" else out_d
     batched = cfg.pipeline == "flow" and S > 1
 
     def step(r):
         if batched:
-            dc.decode_batch(model, streams, [feats_d[r, i] for i in range(S)], [out_d[i] for i in range(S)])
+            dc.decode_batch(model, streams, feats_d[r], out_dv)
         else:
             for i in range(S):
                 streams[i].decode_chunk(feats_d[r, i], out=out_d[i])
@@ -283,10 +284,11 @@ def main():
     # ---- end to end through the host-buffer entry points (H2D + decode + D2H + sync per step) ----
     fin = [feats_h[r].pin_memory() for r in range(history + W, rounds)]
     fout = torch.empty(S, T * cfg.out_per_frame).pin_memory()
+    fout_v = fout.view(S, T, -1) if cfg.pipeline != "vocoder" else fout
     e2e_warm = min(3, K)
     def e2e_step(k):
         if batched:
-            dc.decode_batch_host(model, streams, [fin[k][i] for i in range(S)], [fout[i] for i in range(S)])
+            dc.decode_batch_host(model, streams, fin[k], fout_v)
         else:
             for i in range(S):
                 streams[i].decode_chunk_host(fin[k][i], fout[i])

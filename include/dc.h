@@ -156,9 +156,10 @@ dc_status dc_decode_chunk_host(dc_stream* stream, const float* feats_host, int n
                                float* out_host, int* n_out, void* cuda_stream);
 
 /* dc_decode_batch for callers with host buffers: feats_host[i] / out_host[i] are host
- * pointers (pinned memory makes the copies asynchronous).  Copies every stream's chunk to
- * its staging buffer, decodes the batch, copies the results back and synchronises
- * cuda_stream. */
+ * pointers (pageable or pinned).  Gathers the chunks in a pinned buffer owned by the model,
+ * moves them to the device in one transfer, decodes the batch, brings all results back in one
+ * transfer, synchronises cuda_stream and scatters them.  Returns DC_ERR_TIMEOUT (and poisons the
+ * streams) if a bounded device-side wait gave up.  Calls on one model must not overlap. */
 dc_status dc_decode_batch_host(dc_model* model, int n, dc_stream* const* streams,
                                const float* const* feats_host, const int* n_frames,
                                float* const* out_host, void* cuda_stream);

@@ -217,24 +217,41 @@ class Stream:
             self.handle = C.c_void_p()
 
 
-def decode_batch_host(model: Model, streams: Sequence[Stream], feats_host: Sequence, outs_host: Sequence, stream=None):
-    """dc_decode_batch_host: feats_host[i] / outs_host[i] are CPU float32 tensors (ideally pinned)."""
+def _ptr_array(items, n):
+    """Pointers of n chunks: a list of tensors, or one contiguous tensor [n, T, width] (fast path)."""
+    if hasattr(items, "data_ptr"):
+        assert items.is_contiguous() and items.shape[0] == n
+        stride = items.stride(0) * items.element_size()
+        ptrs = items.data_ptr() + stride * np.arange(n, dtype=np.uint64)
+        return (C.c_void_p * n).from_buffer_copy(ptrs.astype(np.uint64).tobytes()), items.shape[1]
+    return (C.c_void_p * n)(*[t.data_ptr() for t in items]), None
+
+
+def _batch_args(model: Model, streams: Sequence[Stream], feats, outs):
     n = len(streams)
-    hs = (C.c_void_p * n)(*[s.handle for s in streams])
-    fp = (C.c_void_p * n)(*[f.data_ptr() for f in feats_host])
-    op = (C.c_void_p * n)(*[o.data_ptr() for o in outs_host])
-    nf = (C.c_int * n)(*[f.shape[0] for f in feats_host])
+    key = tuple(id(s) for s in streams)
+    cache = model.__dict__.setdefault("_handle_cache", {})
+    hs = cache.get(key)
+    if hs is None:
+        hs = cache[key] = (C.c_void_p * n)(*[s.handle for s in streams])
+    fp, T = _ptr_array(feats, n)
+    op, _ = _ptr_array(outs, n)
+    nf = (C.c_int * n)(*([T] * n if T is not None else [f.shape[0] for f in feats]))
+    return n, hs, fp, nf, op
+
+
+def decode_batch_host(model: Model, streams: Sequence[Stream], feats_host, outs_host, stream=None):
+    """dc_decode_batch_host: feats_host / outs_host are lists of CPU float32 tensors, or single contiguous
+    CPU tensors [n_streams, T, width] (one chunk per stream)."""
+    n, hs, fp, nf, op = _batch_args(model, streams, feats_host, outs_host)
     _check(model.lib.dc_decode_batch_host(model.handle, n, hs, fp, nf, op, _cuda_stream_handle(stream)),
            "dc_decode_batch_host")
 
 
-def decode_batch(model: Model, streams: Sequence[Stream], feats: Sequence, outs: Sequence, stream=None):
-    """dc_decode_batch: one chunk for each stream; feats[i] CUDA float32 [T_i, in_dim]."""
-    n = len(streams)
-    hs = (C.c_void_p * n)(*[s.handle for s in streams])
-    fp = (C.c_void_p * n)(*[f.data_ptr() for f in feats])
-    op = (C.c_void_p * n)(*[o.data_ptr() for o in outs])
-    nf = (C.c_int * n)(*[f.shape[0] for f in feats])
+def decode_batch(model: Model, streams: Sequence[Stream], feats, outs, stream=None):
+    """dc_decode_batch: one chunk for each stream; feats / outs are lists of CUDA float32 tensors
+    ([T_i, in_dim] / [T_i, out]) or single contiguous CUDA tensors [n_streams, T, width]."""
+    n, hs, fp, nf, op = _batch_args(model, streams, feats, outs)
     _check(model.lib.dc_decode_batch(model.handle, n, hs, fp, nf, op, _cuda_stream_handle(stream)),
            "dc_decode_batch")
 

@@ -65,7 +65,10 @@ struct dc_model {
   dc_config cfg;
   int       device = 0;
   float*    d_w = nullptr;   // fp32 pipelines: the blob on the device
-  dc::F32Call* d_call = nullptr;   // fp32 pipelines: per-call record read by the captured graphs
+  dc::F32Call* d_call = nullptr;
+  // flow pipeline: staging of dc_decode_batch_host (pinned host + device, max_batch chunks each way)
+  float *h_in = nullptr, *h_out = nullptr, *d_in = nullptr, *d_out = nullptr;
+  int*   h_err = nullptr;   // fp32 pipelines: per-call record read by the captured graphs
   std::vector<F32Layer> layers;
   int       out_per_frame = 0;
   int       in_dim = 0;
@@ -239,6 +242,18 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     st = dc::flow_model_create(*cfg, w, &m->flow);
     m->in_dim = 2 * cfg->mel_dim;
     m->out_per_frame = cfg->mel_dim;
+    if (st == DC_OK) {
+      const size_t ni = (size_t)cfg->max_batch * cfg->f_chunk * m->in_dim, no = (size_t)cfg->max_batch * cfg->f_chunk * m->out_per_frame;
+      cudaError_t e = cudaMallocHost(&m->h_in, ni * sizeof(float));
+      if (e == cudaSuccess) e = cudaMallocHost(&m->h_out, no * sizeof(float));
+      if (e == cudaSuccess) e = cudaMallocHost(&m->h_err, sizeof(int));
+      if (e == cudaSuccess) e = cudaMalloc(&m->d_in, ni * sizeof(float));
+      if (e == cudaSuccess) e = cudaMalloc(&m->d_out, no * sizeof(float));
+      if (e != cudaSuccess) {
+        dc::set_error("staging allocation failed: %s", cudaGetErrorString(e));
+        st = DC_ERR_OOM;
+      }
+    }
   } else {
     build_f32_layers(m);
     cudaError_t e = cudaMalloc(&m->d_w, n_floats * sizeof(float));
@@ -253,6 +268,12 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
   if (st != DC_OK) {
     if (m->d_w) cudaFree(m->d_w);
     if (m->d_call) cudaFree(m->d_call);
+    if (m->flow) dc::flow_model_destroy(m->flow);
+    if (m->h_in) cudaFreeHost(m->h_in);
+    if (m->h_out) cudaFreeHost(m->h_out);
+    if (m->h_err) cudaFreeHost(m->h_err);
+    if (m->d_in) cudaFree(m->d_in);
+    if (m->d_out) cudaFree(m->d_out);
     delete m;
     return st;
   }
@@ -269,6 +290,11 @@ extern "C" dc_status dc_destroy(dc_model* m) {
   if (m->flow) dc::flow_model_destroy(m->flow);
   if (m->d_w) cudaFree(m->d_w);
   if (m->d_call) cudaFree(m->d_call);
+  if (m->h_in) cudaFreeHost(m->h_in);
+  if (m->h_out) cudaFreeHost(m->h_out);
+  if (m->h_err) cudaFreeHost(m->h_err);
+  if (m->d_in) cudaFree(m->d_in);
+  if (m->d_out) cudaFree(m->d_out);
   for (dc_stream* s : m->all_streams) delete s;
   delete m;
   return DC_OK;
@@ -622,34 +648,40 @@ extern "C" dc_status dc_decode_chunk_host(dc_stream* s, const float* feats_host,
 extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* streams, const float* const* feats_host,
                                           const int* n_frames, float* const* out_host, void* cuda_stream) {
   if (!m || !streams || !feats_host || !n_frames || !out_host) return DC_ERR_ARG;
+  if (!m->flow || !m->h_in) {
+    dc::set_error("dc_decode_batch_host serves the flow pipeline only");
+    return DC_ERR_CONFIG;
+  }
   if (n < 1 || n > m->cfg.max_batch) return DC_ERR_ARG;
   cudaStream_t cs = (cudaStream_t)cuda_stream;
+  const size_t in_stride = (size_t)m->cfg.f_chunk * m->in_dim, out_stride = (size_t)m->cfg.f_chunk * m->out_per_frame;
   std::vector<const float*> fin((size_t)n);
   std::vector<float*> fout((size_t)n);
   for (int i = 0; i < n; ++i) {
     dc_status st = admit(streams[i], feats_host[i], n_frames[i], out_host[i]);
     if (st != DC_OK) return st;
-    fin[(size_t)i] = streams[i]->stage_in;
-    fout[(size_t)i] = streams[i]->stage_out;
+    fin[(size_t)i] = m->d_in + (size_t)i * in_stride;
+    fout[(size_t)i] = m->d_out + (size_t)i * out_stride;
   }
+  // one pinned bounce buffer each way: two transfers per step instead of two per stream
   for (int i = 0; i < n; ++i)
-    DC_CUDA(cudaMemcpyAsync(streams[i]->stage_in, feats_host[i], (size_t)n_frames[i] * m->in_dim * sizeof(float),
-                            cudaMemcpyHostToDevice, cs));
+    memcpy(m->h_in + (size_t)i * in_stride, feats_host[i], (size_t)n_frames[i] * m->in_dim * sizeof(float));
+  DC_CUDA(cudaMemcpyAsync(m->d_in, m->h_in, (size_t)n * in_stride * sizeof(float), cudaMemcpyHostToDevice, cs));
   dc_status st = dc_decode_batch(m, n, streams, fin.data(), n_frames, fout.data(), cuda_stream);
   if (st != DC_OK) return st;
-  for (int i = 0; i < n; ++i)
-    DC_CUDA(cudaMemcpyAsync(out_host[i], streams[i]->stage_out, (size_t)n_frames[i] * m->out_per_frame * sizeof(float),
-                            cudaMemcpyDeviceToHost, cs));
+  DC_CUDA(cudaMemcpyAsync(m->h_out, m->d_out, (size_t)n * out_stride * sizeof(float), cudaMemcpyDeviceToHost, cs));
+  DC_CUDA(cudaMemcpyAsync(m->h_err, dc::flow_error_word(m->flow), sizeof(int), cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaStreamSynchronize(cs));
-  {
-    const int code = dc::flow_take_device_error(m->flow);
-    if (code != 0) {
-      m->counters[4]++;
-      for (int i = 0; i < n; ++i) streams[i]->poisoned = true;
-      dc::set_error("device-side wait timed out (code %d)", code);
-      return DC_ERR_TIMEOUT;
-    }
+  if (*m->h_err != 0) {   // a bounded device-side wait gave up: the results are not valid
+    const int code = *m->h_err;
+    dc::flow_take_device_error(m->flow);
+    m->counters[4]++;
+    for (int i = 0; i < n; ++i) streams[i]->poisoned = true;
+    dc::set_error("device-side wait timed out (code %d)", code);
+    return DC_ERR_TIMEOUT;
   }
+  for (int i = 0; i < n; ++i)
+    memcpy(out_host[i], m->h_out + (size_t)i * out_stride, (size_t)n_frames[i] * m->out_per_frame * sizeof(float));
   return DC_OK;
 }
 

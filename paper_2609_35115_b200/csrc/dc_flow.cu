@@ -1157,6 +1157,8 @@ dc_status flow_state_reset(FlowModel*, FlowState* s, cudaStream_t st) {
   return DC_OK;
 }
 
+const int* flow_error_word(const FlowModel* m) { return m->d_err; }
+
 int flow_take_device_error(FlowModel* m) {
   int v = 0;
   if (cudaMemcpy(&v, m->d_err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;

@@ -107,6 +107,7 @@ dc_status flow_state_reset(FlowModel* m, FlowState* s, cudaStream_t st);
 void      flow_state_close(FlowState* s);
 // Reads (and clears) the device-side error word that bounded waits set; synchronous.  0 = no timeout.
 int       flow_take_device_error(FlowModel* m);
+const int* flow_error_word(const FlowModel* m);   // device address of that word
 // One chunk for each of n streams.  Returns the number of kernel launches through *launches.
 dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats_dev,
                       const int* n_frames, float* const* out_dev, cudaStream_t st, int* launches);
