@@ -220,6 +220,14 @@ dc_status dc_stream_carry_info(const dc_stream* stream, uint64_t* out, int max_e
  * [5] kernel launches issued, [6] streams open, [7] reserved. */
 dc_status dc_get_counters(const dc_model* model, uint64_t counters[8]);
 
+/* Self-test of the bounded device-side wait that every pipeline barrier in the kernels uses (the
+ * fail-closed discipline of paper Section 3.3, applied to the device): launches a one-CTA kernel
+ * that waits, for at most max_polls polls (1 .. 1,000,000), on a barrier that nothing ever
+ * completes.  The wait must give up by itself and report it: returns DC_ERR_TIMEOUT when it did
+ * (the expected outcome), DC_OK if the wait claimed success, DC_ERR_CUDA on a launch problem.
+ * Synchronous; the context stays usable afterwards. */
+dc_status dc_selftest_bounded_wait(int max_polls);
+
 const char* dc_status_str(dc_status s);
 
 /* Text of the last CUDA or validation error on the calling thread ("" if none). */

@@ -20,7 +20,8 @@ STATUS = {0: "DC_OK", 1: "DC_ERR_ARG", 2: "DC_ERR_CONFIG", 3: "DC_ERR_FRAMES", 4
 EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_stream_reset",
            "dc_stream_close", "dc_decode_chunk", "dc_decode_batch", "dc_decode_chunk_host",
            "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error",
-           "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end", "dc_conv_stack_noalloc"]
+           "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end", "dc_conv_stack_noalloc",
+           "dc_selftest_bounded_wait"]
 
 
 class dc_config(C.Structure):
@@ -68,6 +69,7 @@ def load_library():
     lib.dc_profile_begin.argtypes = [vp, C.c_int]
     lib.dc_profile_end.argtypes = [vp, cp(C.c_double), cp(C.c_uint64)]
     lib.dc_conv_stack_noalloc.argtypes = [vp, C.c_int, C.c_int, cp(C.c_int), vp, C.c_int, vp, vp]
+    lib.dc_selftest_bounded_wait.argtypes = [C.c_int]
     lib.dc_stream_carry_info.argtypes = [vp, cp(C.c_uint64), C.c_int, cp(C.c_int)]
     lib.dc_get_counters.argtypes = [vp, cp(C.c_uint64)]
     lib.dc_status_str.restype = C.c_char_p
@@ -254,6 +256,11 @@ def decode_batch(model: Model, streams: Sequence[Stream], feats, outs, stream=No
     n, hs, fp, nf, op = _batch_args(model, streams, feats, outs)
     _check(model.lib.dc_decode_batch(model.handle, n, hs, fp, nf, op, _cuda_stream_handle(stream)),
            "dc_decode_batch")
+
+
+def selftest_bounded_wait(max_polls: int = 1000) -> int:
+    """dc_selftest_bounded_wait: returns the dc_status (6 = DC_ERR_TIMEOUT is the expected outcome)."""
+    return load_library().dc_selftest_bounded_wait(max_polls)
 
 
 NOALLOC_SCRATCH_FLOATS = 1 << 19

@@ -731,6 +731,8 @@ extern "C" dc_status dc_get_counters(const dc_model* m, uint64_t counters[8]) {
   return DC_OK;
 }
 
+extern "C" dc_status dc_selftest_bounded_wait(int max_polls) { return dc::flow_selftest_bounded_wait(max_polls); }
+
 extern "C" const char* dc_status_str(dc_status s) {
   switch (s) {
     case DC_OK: return "DC_OK";

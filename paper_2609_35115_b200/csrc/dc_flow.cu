@@ -440,6 +440,18 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
 // ---- small kernels ---------------------------------------------------------------------------
 
+// Waits on a barrier that nothing completes; the bounded wait must return false.  result: 1 = gave
+// up as it should, 2 = claimed success.
+__global__ void bounded_wait_selftest_kernel(uint32_t max_polls, int* result) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    ptx::fence_barrier_init();
+    const bool got = ptx::mbar_wait_limit(&bar, 0, max_polls);
+    *result = got ? 2 : 1;
+  }
+}
+
 __global__ void set_slots_kernel(const SlotSet set, SlotInfo* dst) {
   ptx::pdl_launch();
   const int i = threadIdx.x;
@@ -1158,6 +1170,25 @@ dc_status flow_state_reset(FlowModel*, FlowState* s, cudaStream_t st) {
 }
 
 const int* flow_error_word(const FlowModel* m) { return m->d_err; }
+
+dc_status flow_selftest_bounded_wait(int max_polls) {
+  if (max_polls < 1 || max_polls > 1000000) return DC_ERR_ARG;
+  int* d = nullptr;
+  if (cudaMalloc(reinterpret_cast<void**>(&d), sizeof(int)) != cudaSuccess) return DC_ERR_OOM;
+  int h = 0;
+  cudaError_t e = cudaMemset(d, 0, sizeof(int));
+  if (e == cudaSuccess) {
+    bounded_wait_selftest_kernel<<<1, 32>>>((uint32_t)max_polls, d);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpy(&h, d, sizeof(int), cudaMemcpyDeviceToHost);
+  cudaFree(d);
+  if (e != cudaSuccess) {
+    set_error("bounded-wait self-test failed to run: %s", cudaGetErrorString(e));
+    return DC_ERR_CUDA;
+  }
+  return h == 1 ? DC_ERR_TIMEOUT : (h == 2 ? DC_OK : DC_ERR_CUDA);
+}
 
 int flow_take_device_error(FlowModel* m) {
   int v = 0;

@@ -106,6 +106,7 @@ void      flow_state_buffers(const FlowState* s, DevBuf* out, int max_entries, i
 dc_status flow_state_reset(FlowModel* m, FlowState* s, cudaStream_t st);
 void      flow_state_close(FlowState* s);
 // Reads (and clears) the device-side error word that bounded waits set; synchronous.  0 = no timeout.
+dc_status flow_selftest_bounded_wait(int max_polls);
 int       flow_take_device_error(FlowModel* m);
 const int* flow_error_word(const FlowModel* m);   // device address of that word
 // One chunk for each of n streams.  Returns the number of kernel launches through *launches.

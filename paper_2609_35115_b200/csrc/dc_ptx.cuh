@@ -43,11 +43,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Returns false after kMaxPolls failed polls (each poll blocks in hardware for a
 // short, implementation-defined time), which is orders of magnitude beyond any legitimate wait here.
 constexpr uint32_t kMaxPolls = 4u << 20;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kMaxPolls; ++i)
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, uint32_t max_polls) {
+  for (uint32_t i = 0; i < max_polls; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) { return mbar_wait_limit(bar, parity, kMaxPolls); }
 
 // Same bound, but the waiter sleeps between polls: for the many threads that wait for a whole
 // main loop, so that their polling does not compete with the issuing warps for issue slots and

@@ -163,3 +163,19 @@ def test_host_buffer_entry_point(dc):
     assert gu.rel_err(fout.numpy(), ref) <= TOL_F32
     st.close()
     m.destroy()
+
+
+def test_bounded_device_wait_gives_up_and_reports(dc):
+    """A wait on a barrier that nothing completes runs out after its poll limit and the host reads
+    DC_ERR_TIMEOUT; the context stays usable (a decode call works right after)."""
+    assert dc.selftest_bounded_wait(1000) == 6           # DC_ERR_TIMEOUT: the wait gave up, as it must
+    assert dc.selftest_bounded_wait(0) == 1              # argument check
+    cfg = wl.CONFIGS["cfg1"]
+    w = wl.make_workload(cfg)
+    m = dc.Model(cfg, w.weights)
+    st = m.open_stream()
+    y = st.decode_chunk(torch.from_numpy(w.streams[0].feats[:16]).cuda())
+    torch.cuda.synchronize()
+    assert torch.isfinite(y).all()
+    st.close()
+    m.destroy()
