@@ -15,7 +15,8 @@ namespace dc {
 
 namespace {
 
-constexpr int BK = 16;   // reduction slice
+constexpr int BK = 32;   // reduction slice
+constexpr int KQ = BK / 4;   // 16-byte copies per A-tile row
 
 __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + expf(-z)); }
 
@@ -38,9 +39,9 @@ __device__ __forceinline__ void cp_async16_zfill(void* dst, const void* src, int
 // themselves (step kb belongs to group kb % KS) and their partial tiles are summed through shared
 // memory in a fixed order, so the result does not depend on timing.  The vocoder's early layers
 // have few frames and long reductions: without the split most SMs would hold a single warp.
-// Operands stream through a 4-stage cp.async ring per group (a reduction step is far cheaper than
-// one L2 round trip, so three steps are kept in flight).
-constexpr int F32_STAGES = 4;
+// Operands stream through a 3-stage cp.async ring per group (a reduction step is cheaper than one
+// L2 round trip, so two steps are kept in flight).
+constexpr int F32_STAGES = 3;
 
 template <int BM, int BN>
 struct TapTile {
@@ -74,8 +75,8 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
   const int sh0 = p.shift[0], sh1 = p.shift[1], sh2 = p.shift[2];
   constexpr int NTG = TT::NTG;
   constexpr int TX = BN / 4;              // threads along the channel axis
-  constexpr int NA = BM * 4 / NTG;        // 16-byte copies of the A tile per thread
-  constexpr int NB = BN * 4 / NTG;        // 16-byte copies of the B tile per thread
+  constexpr int NA = BM * KQ / NTG;       // 16-byte copies of the A tile per thread
+  constexpr int NB = BK * BN / 4 / NTG;   // 16-byte copies of the B tile per thread
   constexpr int LDA = TT::LDA;
   extern __shared__ __align__(16) float f32_smem[];
 
@@ -104,8 +105,8 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
 #pragma unroll
   for (int u = 0; u < NA; ++u) {
     const int i = tid + u * NTG;
-    const int row = i >> 2;
-    a_kq[u] = (i & 3) * 4;                                // A tile: BM rows x 16 k
+    const int row = i / KQ;
+    a_kq[u] = (i % KQ) * 4;                               // A tile: BM rows x BK k
     a_ok[u] = m0 + row < T_in;
     a_dst[u] = row * LDA + a_kq[u];
     const long long t = pos_in + m0 + row;
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
 #pragma unroll
   for (int u = 0; u < NB; ++u) {
     const int i = tid + u * NTG;
-    b_k[u] = i / TX;                                      // B tile: 16 k x BN n
+    b_k[u] = i / TX;                                      // B tile: BK k x BN n
     const int nq = (i % TX) * 4;
     b_ok[u] = n0 + nq < C_out;
     b_dst[u] = b_k[u] * BN + nq;
