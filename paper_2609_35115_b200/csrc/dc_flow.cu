@@ -92,6 +92,15 @@ struct GemmParams {
   float        inv_n;
   int          last_step;
   int          mel;
+  // RMS normalisation, folded into the GEMMs around it (Sec. 3.2 block form; the norm has no gain):
+  // (x / rms(x)) W = (x W) / rms(x), so the GEMM that consumes a normalised operand reads x itself
+  // and scales its accumulator rows, and the GEMM that produced x leaves the row sums of squares.
+  // Partial sums are kept per 16-column chunk, [C / 16][ssq_ld], and added in chunk order, so the
+  // statistic does not depend on the tile width chosen for the batch size.
+  float*       ssq_out;         // producer: partial sums of squares of the stored (bf16) output, or null
+  const float* ssq_in;          // consumer (MODE_QKV, MODE_OUT): partial sums of the operand rows
+  long long    ssq_ld;          // rows per chunk plane
+  float        inv_C, eps;
   int*         err;
   int          dbg;
 };
@@ -317,6 +326,16 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
       }
     }
+    // row scale 1 / rms of the normalised operand: chunk partials in ascending order
+    float rs = 1.f;
+    if (p.ssq_in != nullptr) {
+      float ss = 0.f;
+      if (in_range && f >= 0 && f < si.T) {
+        const int n_parts = p.C >> 4;
+        for (int j = 0; j < n_parts; ++j) ss += p.ssq_in[(long long)j * p.ssq_ld + r];
+      }
+      rs = rsqrtf(ss * p.inv_C + p.eps);
+    }
     // constants visible to all epilogue threads; every read of the carry has been performed
     // before any thread below overwrites carry rows
     ptx::named_bar_sync(1, EPI_THREADS);
@@ -346,7 +365,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       const int n = n0 + c0;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) acc[i] += s_bias[c0 + i];
+      for (int i = 0; i < 16; ++i) acc[i] = fmaf(acc[i], rs, s_bias[c0 + i]);
       if (p.mode == MODE_OUT) {
         if (is_chunk) {
           float* xs = p.xstate + (long long)r * p.mel + n;
@@ -414,6 +433,19 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #endif
       // chunk rows store y; left-context rows hand the carried rows to the consumer of `out`
       if (is_chunk || (is_halo && do_halo)) store16(p.out + grow * p.ld + n, va, vb);
+      if (p.ssq_out != nullptr && in_range) {   // sum of squares of the 16 stored values, fixed order
+        float ss = 0.f;
+        if (is_chunk) {
+          const uint32_t w[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+            ss = fmaf(lo, lo, ss);
+            ss = fmaf(hi, hi, ss);
+          }
+        }
+        p.ssq_out[(long long)(n >> 4) * p.ssq_ld + r] = ss;
+      }
       // shift the carry by T frames: [old carry | chunk] -> its last 8 rows
       if (carry_wr) store16(carry + new_row * p.C + n, va, vb);
       if (threadIdx.x == 128 && kk == 0) DC_T(6);
@@ -473,44 +505,6 @@ __global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, 
     ain[(GUARD + r) * ld_ain + mel + c] = __float2bfloat16_rn(mu);
   }
 }
-
-// u = bf16(x * rsqrt(mean(x^2) + eps)), one warp per chunk row.
-__global__ void flow_rmsnorm_kernel(const SlotInfo* slots, int n_slots, const bf16* x, bf16* u, int C, float eps) {
-  ptx::pdl_launch();
-  ptx::pdl_wait();
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  const int slot = warp / SLOT_ROWS, rho = warp % SLOT_ROWS;
-  if (slot >= n_slots) return;
-  const int f = rho - HALO;
-  if (f < 0 || f >= slots[slot].T) return;
-  const long long off = (long long)(GUARD + warp) * C;
-  float ss = 0.f;
-  for (int c = lane * 8; c < C; c += 256) {
-    const uint4 v = *reinterpret_cast<const uint4*>(x + off + c);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float a = __uint_as_float(w[i] << 16), b = __uint_as_float(w[i] & 0xFFFF0000u);
-      ss = fmaf(a, a, ss);
-      ss = fmaf(b, b, ss);
-    }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  const float rs = rsqrtf(ss / (float)C + eps);
-  for (int c = lane * 8; c < C; c += 256) {
-    const uint4 v = *reinterpret_cast<const uint4*>(x + off + c);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t o[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(w[i] << 16) * rs, __uint_as_float(w[i] & 0xFFFF0000u) * rs);
-      o[i] = *reinterpret_cast<const uint32_t*>(&h);
-    }
-    *reinterpret_cast<uint4*>(u + off + c) = make_uint4(o[0], o[1], o[2], o[3]);
-  }
-}
-
 
 // ---- chunk-causal attention with the K/V carry ---------------------------------------------------
 // One CTA per (stream slot, head), two CTAs per SM.  Queries: the T <= 56 chunk frames (rows 0..63
@@ -886,13 +880,14 @@ struct GraphEntry {
 struct FlowModel {
   dc_config cfg;
   int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0;
-  bf16 *Xa = nullptr, *Xb = nullptr, *U = nullptr, *Q = nullptr, *O = nullptr, *Ain = nullptr;
+  bf16 *Xa = nullptr, *Xb = nullptr, *Q = nullptr, *O = nullptr, *Ain = nullptr;
   float* xstate = nullptr;
+  float* ssq = nullptr;      // [C / 16][rows]: per-chunk sums of squares of the rows that feed an RMS norm
   bf16*  wts = nullptr;
   float* fconst = nullptr;   // biases and the timestep-bias table
   SlotInfo* d_slots = nullptr;
   int*   d_err = nullptr;
-  CUtensorMap tmAin, tmXa, tmXb, tmU, tmO;
+  CUtensorMap tmAin, tmXa, tmXb, tmO;
   // weight maps in three tile-width variants v (box rows = N tile): v = 0 wide (64 / 192 / mel), for full
   // batches; v = 1, 2 narrower (32, 16 / 96, 48 / 16), so that a small batch still spreads over many SMs
   CUtensorMap tmWin[3], tmWout[3];
@@ -1062,7 +1057,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   chk(dalloc(m, &m->fconst, fn, false));
   chk(dalloc(m, &m->Xa, R * C));
   chk(dalloc(m, &m->Xb, R * C));
-  chk(dalloc(m, &m->U, R * C));
+  chk(dalloc(m, &m->ssq, (size_t)(C / 16) * m->rows));
   chk(dalloc(m, &m->Q, R * C));
   chk(dalloc(m, &m->O, R * C));
   chk(dalloc(m, &m->Ain, R * m->Kin));
@@ -1085,7 +1080,6 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   ok &= make_tmap(&m->tmAin, m->Ain, R, m->Kin, A_ROWS);
   ok &= make_tmap(&m->tmXa, m->Xa, R, C, A_ROWS);
   ok &= make_tmap(&m->tmXb, m->Xb, R, C, A_ROWS);
-  ok &= make_tmap(&m->tmU, m->U, R, C, A_ROWS);
   ok &= make_tmap(&m->tmO, m->O, R, C, A_ROWS);
   for (int v = 0; v < 3; ++v) {
     const int bn = 64 >> v, bq = 192 >> v, bo = 16;
@@ -1287,10 +1281,10 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     const size_t smem = GEMM_SMEM_EXTRA + (size_t)p.n_stages * stage_bytes;
     launch(lc, flow_gemm_kernel, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), smem, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
   };
-  auto rmsnorm = [&](const bf16* x) {
-    const int warps = n * SLOT_ROWS;
-    launch(lc, flow_rmsnorm_kernel, dim3((warps * 32 + 255) / 256), dim3(256), 0, true, 3, (const SlotInfo*)m->d_slots, n, x, m->U, C,
-           c.rms_eps);
+  // the GEMM whose output feeds an RMS norm leaves the row statistics; the GEMM after the norm applies them
+  auto feeds_norm = [&](GemmParams& p) { p.ssq_out = m->ssq; p.ssq_ld = m->rows; };
+  auto normalised = [&](GemmParams& p) {
+    p.ssq_in = m->ssq; p.ssq_ld = m->rows; p.inv_C = 1.0f / (float)C; p.eps = c.rms_eps;
   };
   auto attention = [&](int step, int layer) {
     AttnParams p{};
@@ -1315,6 +1309,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       p.mode = MODE_INPROJ; p.BN = bn; p.n_kblocks = m->Kin / KBLK; p.taps = 1;
       p.bias = fc + m->o_bin; p.out = X;
       p.halo_off = ((long long)s * c.n_conv + 0) * halo_stride;
+      if (m->cpa == 0) feeds_norm(p);
       gemm(m->tmAin, m->tmWin[v], p, C);
     }
     int l = 0;
@@ -1329,17 +1324,18 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
         p.resid = X; p.out = Y;
         const bool next_is_conv = (j + 1 < m->cpa);
         p.halo_off = next_is_conv ? ((long long)s * c.n_conv + l + 1) * halo_stride : -1;
+        if (!next_is_conv) feeds_norm(p);   // the group's attention norm, or the final norm of a conv-only stack
         gemm(*tX, m->tmWconv[v][l], p, C);
         swap();
       }
       if (c.n_attn > 0) {
-        rmsnorm(X);
         {
           GemmParams p{};
           p.mode = MODE_QKV; p.BN = bq; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bqkv[g]; p.q_out = m->Q; p.halo_off = -1;
           p.kv_off = ((long long)s * c.n_attn + g) * 2 * m->Rk * C;
-          gemm(m->tmU, m->tmWqkv[v][g], p, 3 * C);
+          normalised(p);
+          gemm(*tX, m->tmWqkv[v][g], p, 3 * C);
         }
         attention(s, g);
         {
@@ -1347,19 +1343,20 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
           p.mode = MODE_OPROJ; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bo[g]; p.resid = X; p.out = Y;
           p.halo_off = (l < c.n_conv) ? ((long long)s * c.n_conv + l) * halo_stride : -1;
+          if (g == n_groups - 1 || m->cpa == 0) feeds_norm(p);   // final norm, or the next group's norm
           gemm(m->tmO, m->tmWo[v][g], p, C);
           swap();
         }
       }
     }
-    rmsnorm(X);
     {
       GemmParams p{};
       p.mode = MODE_OUT; p.BN = bo; p.n_kblocks = C / KBLK; p.taps = 1;
       p.bias = fc + m->o_bout; p.halo_off = -1;
       p.xstate = m->xstate; p.ain = m->Ain; p.ld_ain = m->Kin; p.inv_n = 1.0f / c.n_steps;
       p.last_step = (s == c.n_steps - 1); p.mel = mel;
-      gemm(m->tmU, m->tmWout[v], p, mel);
+      normalised(p);
+      gemm(*tX, m->tmWout[v], p, mel);
     }
   }
 }
