@@ -507,25 +507,32 @@ __global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, 
 }
 
 // ---- chunk-causal attention with the K/V carry ---------------------------------------------------
-// One CTA per (stream slot, head), two CTAs per SM.  Queries: the T <= 56 chunk frames (rows 0..63
-// of the 128 UMMA rows; rows 64..127 are never read back).  Keys/values: the kv_len carried frames
+// One CTA per (stream slot, head), two CTAs per SM.  Queries: the T <= 56 chunk frames, held TWICE
+// in the 128 UMMA rows (row 64 + i repeats row i), so that S has a copy of every query row in both
+// halves of tensor memory: a warp can only read the 32 lanes of its own SM sub-partition, and with
+// the copy the softmax work spreads over all four sub-partitions (special-function throughput is
+// what bounds it) instead of the two that own lanes 0..63.  Keys/values: the kv_len carried frames
 // followed by the chunk's own T frames, streamed in place from the stream's ring in blocks of 128
 // keys with 128-bit cp.async loads (the ring may wrap; nothing is compacted or copied in global
 // memory) through a two-stage shared-memory ring.
 //
-// Warp roles (8 warps): warps 0,1,4,5 = softmax (thread = (query row, half of the block's 128 key
-// columns)); warp 3 = UMMA issuer; warps 2,6,7 = K/V/Q loaders.
+// Warp roles (8 warps): warps 0..3 = softmax (thread = (query row, half of the block's 128 key
+// columns); warps 0,1 read lanes 0..63 and own key columns 0..63, warps 2,3 read the copy in lanes
+// 64..127 and own key columns 64..127); warp 4 = UMMA issuer; warps 5,6 = Q and K loaders, warp 7 =
+// V loader.
 // Per key block: S = Q K^T on tcgen05 (accumulator in TMEM) -> the softmax threads read their
 // columns, e = exp2(scale*S - m) with a running reference m that is only raised when the block
 // maximum exceeds it by more than 2^8 (then O and the row sum are rescaled once), row sum from the
-// unrounded e, P = bf16(e) into shared memory -> O += P V on tcgen05 (V is the MN-major operand).
+// unrounded e, P = bf16(e) into shared memory (64 rows; the UMMA's rows 64..127 of P and O are
+// never read back) -> O += P V on tcgen05 (V is the MN-major operand).  O lives in lanes 0..63, so
+// warps 0,1 rescale it and write the result.
 constexpr int ATT_THREADS = 256;
 constexpr int ATT_KB = 128;             // keys per block
 constexpr int ATT_STAGES = 2;
 constexpr int ATT_TMEM_COLS = 256;      // S (128 columns) + O (64 columns); two CTAs share the SM's 512
-constexpr int ATT_K_LOADERS = 64;       // warps 2 and 6: Q, then the K blocks
+constexpr int ATT_K_LOADERS = 64;       // warps 5 and 6: Q, then the K blocks
 constexpr int ATT_V_LOADERS = 32;       // warp 7: the V blocks
-constexpr int ATT_Q_BYTES = 64 * 128;   // 64 query rows; the UMMA's rows 64..127 alias the P region
+constexpr int ATT_Q_BYTES = 128 * 128;  // 64 query rows, twice
 constexpr int ATT_P_BYTES = 2 * 64 * 128;
 constexpr int ATT_STAGE_BYTES = 2 * ATT_KB * 128;   // K block + V block
 constexpr size_t ATT_SMEM = 1024 + ATT_Q_BYTES + ATT_P_BYTES + ATT_STAGES * ATT_STAGE_BYTES + 1024;
@@ -597,7 +604,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     ptx::mbar_init(bar_sfree, 128);
     ptx::fence_barrier_init();
   }
-  if (warp == 3) ptx::tmem_alloc(tmem_slot, ATT_TMEM_COLS);
+  if (warp == 4) ptx::tmem_alloc(tmem_slot, ATT_TMEM_COLS);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -608,7 +615,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   const int T = si.T, L = si.kv_len + T;
   const int nkb = (L + ATT_KB - 1) / ATT_KB;
 
-  if (warp == 2 || warp >= 6) {
+  if (warp >= 5) {
     // ---------------- loaders ----------------
     const bool is_k = warp != 7;
     const int nl = is_k ? ATT_K_LOADERS : ATT_V_LOADERS;
@@ -616,10 +623,10 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
     if (is_k) {
       const bf16* qbase = p.q + (long long)(GUARD + slot * SLOT_ROWS + HALO) * p.ld + head * p.dh;
-      for (int i = lt; i < 64 * 8; i += nl) {
-        const int row = i >> 3, j = i & 7;
+      for (int i = lt; i < 128 * 8; i += nl) {
+        const int row = i >> 3, j = i & 7, qrow = row & 63;   // rows 64.. repeat rows 0..
         uint8_t* dst = sQ + row * 128 + ((j ^ (row & 7)) << 4);
-        if (row < T && j < chunks) cp_async16(dst, qbase + (long long)row * p.ld + j * 8);
+        if (qrow < T && j < chunks) cp_async16(dst, qbase + (long long)qrow * p.ld + j * 8);
         else *reinterpret_cast<uint4*>(dst) = zero;
       }
     }
@@ -660,7 +667,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     ptx::fence_proxy_async_smem();
     ptx::mbar_arrive(&full[(nkb - 1) % ATT_STAGES]);
     if (lt == 0 && is_k && nkb - 1 < 8) DC_AT(8 + nkb - 1);
-  } else if (warp == 3) {
+  } else if (warp == 4) {
     // ---------------- UMMA issuer ----------------
     if (lane == 0) {
       const uint32_t idesc_s = ptx::umma_idesc_bf16(128, ATT_KB, 0, 0);
@@ -695,20 +702,28 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         const uint64_t dv = ptx::umma_desc_sw128(ptx::smem_u32(ring + st * ATT_STAGE_BYTES + ATT_KB * 128));
         const int valid = L - b * ATT_KB;
         const int ksteps = valid >= ATT_KB ? ATT_KB / 16 : (valid + 15) / 16;
-        for (int k = 0; k < ksteps; ++k)   // P tile k/4 (8 KB apart), 32-byte K steps; V: 16 key rows = 2 KB per step
-          ptx::umma_bf16(tmem_base + ATT_KB, dp + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
-                         idesc_pv, (b | k) != 0);
+        // P tile k/4 (8 KB apart), 32-byte K steps; V: 16 key rows = 2 KB per step
+        if (ksteps == ATT_KB / 16) {
+#pragma unroll
+          for (int k = 0; k < ATT_KB / 16; ++k)
+            ptx::umma_bf16(tmem_base + ATT_KB, dp + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
+                           idesc_pv, (b | k) != 0);
+        } else {
+          for (int k = 0; k < ksteps; ++k)
+            ptx::umma_bf16(tmem_base + ATT_KB, dp + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
+                           idesc_pv, (b | k) != 0);
+        }
         ptx::umma_commit(&empty_v[st]);
         ptx::umma_commit(bar_pv);
         if (b < 8) DC_AT(24 + b);                        // PV(b) issued
       }
     }
   } else {
-    // ---------------- softmax: warps 0,1,4,5 ----------------
-    const int quarter = warp & 1;               // TMEM lanes 32*quarter .. (warp % 4 == quarter)
-    const int half = warp >> 2;                 // key columns 64*half .. of each block
+    // ---------------- softmax: warps 0..3 ----------------
+    const int quarter = warp & 1;               // query rows 32*quarter ..
+    const int half = warp >> 1;                 // key columns 64*half .. of each block, read from the row copy in lanes 64*half ..
     const int row = quarter * 32 + lane;        // query row
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);   // the lanes this warp may access
     bool ok = true;
     float m_ref = -INFINITY, lsum = 0.f;
     for (int b = 0; b < nkb; ++b) {
@@ -744,14 +759,15 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
           const float alpha = need ? exp2f(m_ref - mx) : 1.0f;
           if (need) m_ref = mx;
           lsum *= alpha;
-          const int ncol = p.dh >> 1;             // O columns owned by this half
-          for (int c = 0; c < ncol; c += 16) {
-            float o16[16];
-            const uint32_t addr = lane_addr + (uint32_t)(ATT_KB + half * ncol + c);
-            ptx::tmem_ld16(addr, o16);
+          if (half == 0) {                        // O rows 0..63 live in lanes 0..63
+            for (int c = 0; c < p.dh; c += 16) {
+              float o16[16];
+              const uint32_t addr = lane_addr + (uint32_t)(ATT_KB + c);
+              ptx::tmem_ld16(addr, o16);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) o16[i] *= alpha;
-            ptx::tmem_st16(addr, o16);
+              for (int i = 0; i < 16; ++i) o16[i] *= alpha;
+              ptx::tmem_st16(addr, o16);
+            }
           }
         }
       }
@@ -780,11 +796,10 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     s_x[half * 64 + row] = lsum;
     ptx::named_bar_sync(2, 128);
     const float inv = 1.0f / (s_x[row] + s_x[64 + row]);
-    const int ncol = p.dh >> 1;
-    bf16* orow = p.o + (long long)(GUARD + slot * SLOT_ROWS + HALO + row) * p.ld + head * p.dh + half * ncol;
-    for (int c = 0; c < ncol; c += 16) {
+    bf16* orow = p.o + (long long)(GUARD + slot * SLOT_ROWS + HALO + row) * p.ld + head * p.dh;
+    for (int c = 0; c < (half == 0 ? p.dh : 0); c += 16) {
       float o16[16];
-      ptx::tmem_ld16(lane_addr + (uint32_t)(ATT_KB + half * ncol + c), o16);
+      ptx::tmem_ld16(lane_addr + (uint32_t)(ATT_KB + c), o16);
       if (row < T && ok) {
 #pragma unroll
         for (int i = 0; i < 16; ++i) o16[i] *= inv;
@@ -796,7 +811,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   }
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp == 3) ptx::tmem_dealloc(tmem_base, ATT_TMEM_COLS);
+  if (warp == 4) ptx::tmem_dealloc(tmem_base, ATT_TMEM_COLS);
 #ifdef DC_TIMING
   if (atm && tid == 0) {
     printf("ATT nkb %d end %lld\n load_issue:", nkb, clock64() - a_start);
