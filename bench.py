@@ -38,7 +38,7 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 HISTORY_CHUNKS = 12      # untimed stream history so that the K/V carry sits at its cap (steady state)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for that workload)
-NCU_TRAFFIC_BYTES = {"cfg5": 4.01e6,   # conv-mode flow_gemm_kernel, profiles/flow_gemm_kernel_conv_cfg5.md
+NCU_TRAFFIC_BYTES = {"cfg5": 4.03e6,   # conv-mode flow_gemm_kernel, profiles/flow_gemm_kernel_conv_cfg5.md
                      "cfg3": None, "cfg2": None, "cfg4": None, "cfg1": None}
 
 
@@ -59,13 +59,13 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index = index
-        self.rows = []
+        self.rows = []      # (host time of arrival, fields)
         self.proc = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
@@ -76,9 +76,11 @@ class ClockSampler:
         for line in self.proc.stdout:
             parts = [x.strip() for x in line.split(",")]
             if len(parts) >= 7:
-                self.rows.append(parts)
+                self.rows.append((time.perf_counter(), parts))
 
-    def stop(self):
+    def stop(self, windows=None):
+        """windows: {name: (t0, t1)} host-time intervals; the summary uses the samples that arrived
+        inside any of them (a sample describes the ~50 ms before its arrival) and counts them per window."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -86,12 +88,22 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
-        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        counts = {}
+        rows = []
+        for t, parts in self.rows:
+            for name, (t0, t1) in (windows or {"all": (0.0, float("inf"))}).items():
+                if t0 <= t <= t1 + 0.06:
+                    counts[name] = counts.get(name, 0) + 1
+                    rows.append(parts)
+                    break
+        sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in rows if r[1].replace(".", "").isdigit()]
+        pw = [float(r[2]) for r in rows if r[2].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(r[3 + i] == "Active" for r in self.rows)]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i] == "Active" for r in rows)]
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(self.rows)}
+                "power_w": statistics.median(pw) if pw else None, "reasons": reasons, "samples": len(rows),
+                "samples_by_window": counts, "period_ms": 50}
 
 
 def describe(cfg) -> str:
@@ -262,24 +274,59 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    sampler.start()          # nvidia-smi needs a moment before its first sample: start it ahead of the timed region
     for r in range(history + W):
         step(r)
     sync_all()
-    sampler = ClockSampler(local)
-    sampler.start()
     c0 = model.counters()
+    t_timed0 = time.perf_counter()
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
     evs[0].record()
     for k in range(K):
         step(history + W + k)
         evs[k + 1].record()
     torch.cuda.synchronize()
+    t_timed1 = time.perf_counter()
     total_ms = evs[0].elapsed_time(evs[K])
-    clocks = sampler.stop()
     c1 = model.counters()
+    # The timed region of a short run is over before nvidia-smi (50 ms period) has sampled it a few
+    # times: keep the same steps running, untimed, for about a second and sample that load as well.
+    windows = {"timed_region": (t_timed0, t_timed1)}
+    if t_timed1 - t_timed0 < 0.5:
+        t_p0 = time.perf_counter()
+        k = 0
+        while time.perf_counter() - t_p0 < 1.0:
+            step(history + W + (k % K))
+            k += 1
+            if k % 8 == 0:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        windows["same_steps_untimed"] = (t_p0, time.perf_counter())
+    clocks = sampler.stop(windows)
     step_ms = sorted(evs[k].elapsed_time(evs[k + 1]) for k in range(K))
     total_ms = max_over_ranks(total_ms, world)
     value = aggregate_throughput(world, S, K, per_chunk, total_ms * 1e-3)
+
+    # ---- the same step with L2 flushed first (workloads whose working set fits L2 only): a stream paced
+    # at its real-time cadence finds its weights and carries in HBM, not in L2 ----
+    ws_mb = (S * (cfg.n_steps * cfg.n_attn_layers * 2 * (cfg.kv_cap + T) * cfg.hidden * 2) / 1e6) if cfg.pipeline == "flow" else 0.0
+    cold = None
+    if ws_mb <= 126:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        pairs = []
+        for k in range(min(K, 20)):
+            flush.fill_(k & 0xFF)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            step(history + W + k)
+            e1.record()
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        ct = sorted(a.elapsed_time(b) for a, b in pairs)
+        cold = {"p50": 1e3 * ct[len(ct) // 2], "p95": 1e3 * ct[min(len(ct) - 1, int(0.95 * len(ct)))], "steps": len(ct),
+                "flush": "256 MiB written before every step"}
+        del flush
 
     # ---- end to end through the host-buffer entry points (H2D + decode + D2H + sync per step) ----
     fin = [feats_h[r].pin_memory() for r in range(history + W, rounds)]
@@ -345,7 +392,7 @@ def main():
                "sample": f"{n_c} consecutive chunks of one stream (carry growing from empty), {dt:.1f} s"}
 
     if rank == 0:
-        ws = (S * (cfg.n_steps * cfg.n_attn_layers * 2 * (cfg.kv_cap + T) * cfg.hidden * 2) / 1e6) if cfg.pipeline == "flow" else 0
+        ws = ws_mb
         line = {
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -353,10 +400,11 @@ def main():
             "config": {"workload": describe(cfg), "streams_per_gpu": S, "frames_per_chunk": T,
                        "history_chunks": history, "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": (f"K/V carries {ws:.0f} MB > 126 MB L2, streamed from HBM every step" if ws > 126 else
-                              "working set fits L2; inputs differ every step, no flush"),
+                              "working set fits L2: value and latency_us are back-to-back chunks (warm L2), latency_us_cold_l2 flushes L2 before every step"),
                        "inputs": "N(0,1) features, N(0,1/fan_in) weights, seeded"},
             "latency_us": {"p50": 1e3 * step_ms[len(step_ms) // 2], "p95": 1e3 * step_ms[min(len(step_ms) - 1, int(0.95 * len(step_ms)))],
                            "per": "step (one chunk of every stream)"},
+            "latency_us_cold_l2": cold,
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": S * T * cfg.in_dim * 4,
                     "d2h_bytes_per_step": S * T * cfg.out_per_frame * 4, "ms_per_step": 1e3 * e2e_s / K},
             "gpu_launches": int(c1[5] - c0[5]),
