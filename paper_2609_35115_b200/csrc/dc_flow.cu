@@ -44,8 +44,9 @@ constexpr int GEMM_TILE_SMEM = 88 * 1024;    // operand stages per CTA: small en
 constexpr int A_ROWS = TILE_M + HALO;  // the A tile carries 8 extra leading rows so that all taps read it
 constexpr int A_BYTES = A_ROWS * 128;
 constexpr int MAX_BN = 192;
-constexpr int GEMM_THREADS = 384;      // warp 0 TMA (A), warps 1 and 3 UMMA issuers, warp 2 TMA (B), warps 4..11 epilogue
-constexpr int EPI_THREADS = 256;
+constexpr int EPI_GROUPS = 4;           // epilogue warps per TMEM lane quarter: group g owns the 16-column chunks g, g + 4, ...
+constexpr int EPI_THREADS = 128 * EPI_GROUPS;
+constexpr int GEMM_THREADS = 128 + EPI_THREADS;   // warp 0 TMA (A), warps 1 and 3 UMMA issuers, warp 2 TMA (B), the rest epilogue
 constexpr int MAX_SLOTS_PER_SET = 64;
 
 enum GemmMode { MODE_INPROJ = 0, MODE_CONV = 1, MODE_QKV = 2, MODE_OPROJ = 3, MODE_OUT = 4 };
@@ -140,7 +141,7 @@ __device__ __forceinline__ void store16(bf16* p, const uint4& a, const uint4& b)
   *reinterpret_cast<uint4*>(p + 8) = b;
 }
 
-__global__ void __launch_bounds__(GEMM_THREADS, 2)
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
 flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -172,10 +173,15 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #else
 #define DC_T(tag) do {} while (0)
 #endif
-  // second issuer's accumulator sits acc2_off columns after the first
-  const uint32_t acc2_off = p.BN <= 32 ? 32u : 64u;
-  const uint32_t need_cols = p.n_issuers == 2 ? 2u * acc2_off : (uint32_t)p.BN;
-  const uint32_t tmem_cols = need_cols <= 32 ? 32u : (need_cols <= 64 ? 64u : (need_cols <= 128 ? 128u : 256u));
+  // Accumulator: BN columns, or 3 BN for a conv block, whose three taps are the column blocks of ONE
+  // product Z = X [W_0 | W_1 | W_2] (a row shift commutes with the product, so the taps are shifted
+  // and added in the epilogue; a tcgen05.mma costs about 47 cycles however small it is, and one
+  // 128 x 3BN x 16 instruction replaces three 128 x BN x 16 ones).  The second issuer's accumulator
+  // sits acc2_off columns after the first.
+  const uint32_t acc_w = (uint32_t)(p.taps * p.BN);
+  const uint32_t acc2_off = acc_w <= 32 ? 32u : (acc_w <= 64 ? 64u : (acc_w <= 128 ? 128u : 256u));
+  const uint32_t need_cols = p.n_issuers == 2 ? 2u * acc2_off : acc_w;
+  const uint32_t tmem_cols = need_cols <= 32 ? 32u : (need_cols <= 64 ? 64u : (need_cols <= 128 ? 128u : (need_cols <= 256 ? 256u : 512u)));
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
@@ -245,14 +251,15 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int me = warp >> 1;                     // 0 or 1
     if (me < p.n_issuers) {
       const uint32_t on = lane == 0;
-      const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.BN, 0, 0);
-      const int nkb = p.n_kblocks, taps = p.taps, step = p.n_issuers;
+      // the weight tiles of the taps are adjacent in the stage (BN rows of 128 B each, BN a multiple of 8),
+      // so together they are one K-major operand of taps * BN rows
+      const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.taps * p.BN, 0, 0);
+      const int nkb = p.n_kblocks, step = p.n_issuers;
       const uint32_t d_acc = tmem_base + (uint32_t)me * acc2_off;
       // descriptor start addresses are in 16-byte units: +2 per 32-byte K step
       const uint64_t d_a0 = ptx::umma_desc_sw128(ptx::smem_u32(smem));
-      const uint32_t stage16 = stage_bytes >> 4, b16 = b_tile >> 4, ab16 = A_BYTES >> 4;
-      const uint32_t o0 = (uint32_t)(HALO - p.shift[0]) * 8u, o1 = (uint32_t)(HALO - p.shift[1]) * 8u,
-                     o2 = (uint32_t)(HALO - p.shift[2]) * 8u;   // row offset of tap j: rows * 128 B / 16
+      const uint32_t stage16 = stage_bytes >> 4, ab16 = A_BYTES >> 4;
+      const uint32_t o0 = (uint32_t)HALO * 8u;   // the output tile's own rows start 8 rows into the A tile (rows * 128 B / 16)
       uint32_t acc = 0;
       for (int kb = me; kb < nkb; kb += step) {
         const int st = kb % STAGES;
@@ -267,19 +274,9 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (tm && kb < 32 && on) s_k[kb] = clock64() - t_start;
 #endif
         const uint64_t da = d_a0 + (uint64_t)((uint32_t)st * stage16), db = da + ab16;
-        if (taps == 3) {
-          ptx::umma_bf16_if(on, d_acc, da + o0, db, idesc, acc);
+        ptx::umma_bf16_if(on, d_acc, da + o0, db, idesc, acc);
 #pragma unroll
-          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o1 + 2 * k), db + (b16 + 2 * k), idesc, 1);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o2 + 2 * k), db + (2 * b16 + 2 * k), idesc, 1);
-        } else {
-          ptx::umma_bf16_if(on, d_acc, da + o0, db, idesc, acc);
-#pragma unroll
-          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
-        }
+        for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
         acc = 1;
         ptx::umma_commit_if(on, &empty[st]);
       }
@@ -287,7 +284,9 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::umma_commit_if(on, accum);   // arrives when every UMMA above has finished (also on the failure path)
     }
   } else {
-    // ---------------- epilogue: 8 warps; a thread owns one output row and every other 16-column chunk ----------------
+    // ---------------- epilogue: 4 EPI_GROUPS warps; a thread owns one output row and every EPI_GROUPS-th 16-column chunk ----------------
+    // (the epilogue of a tile is a chain of long-latency steps - TMEM load, special functions, stores -
+    // so it is spread over as many warps as there are chunks in the common 64-column tile)
     // Everything that does not depend on the accumulator is fetched while the main loop runs:
     // per-column constants go to shared memory, the thread's residual row (or, for a left-context
     // row, the carried row) goes to registers.
@@ -298,7 +297,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     ptx::pdl_wait();                              // slot table, residual and carry rows are upstream data
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
-    const int half = (warp - 4) >> 2;             // which chunks of the row: chunk index & 1 == half
+    const int cg = (warp - 4) >> 2;               // which chunks of the row: chunk index % EPI_GROUPS == cg
     const int r = m0 + q * 32 + lane;             // row in slot layout (without GUARD)
     const int slot = r / SLOT_ROWS, rho = r % SLOT_ROWS;
     const bool in_range = slot < p.n_slots;
@@ -308,20 +307,22 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const bool has_resid = p.mode == MODE_CONV || p.mode == MODE_OPROJ;
     const long long grow = (long long)(GUARD + r);
     bf16* carry = do_halo && in_range ? si.halo + p.halo_off : nullptr;
-    // pre[2k], pre[2k+1]: the 16 bf16 of this thread's k-th chunk (columns n0 + 16 (2k + half) ..)
-    uint4 pre[4];
+    // pre[2k], pre[2k+1]: the 16 bf16 of this thread's k-th chunk (columns n0 + 16 (EPI_GROUPS k + cg) ..);
+    // the GEMMs with a residual or carried rows have at most 64 columns per tile
+    constexpr int PRE_CHUNKS = 4 / EPI_GROUPS;
+    uint4 pre[2 * PRE_CHUNKS];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) pre[j] = make_uint4(0u, 0u, 0u, 0u);
+    for (int j = 0; j < 2 * PRE_CHUNKS; ++j) pre[j] = make_uint4(0u, 0u, 0u, 0u);
     {
       const bf16* src = nullptr;
       if (in_range && f >= 0 && f < si.T && has_resid) src = p.resid + grow * p.ld + n0;
       else if (in_range && rho < HALO && do_halo) src = carry + rho * p.C + n0;
       if (src != nullptr) {
 #pragma unroll
-        for (int k = 0; k < 2; ++k) {
-          if (16 * (2 * k + half) < p.BN) {
-            pre[2 * k] = *reinterpret_cast<const uint4*>(src + 16 * (2 * k + half));
-            pre[2 * k + 1] = *reinterpret_cast<const uint4*>(src + 16 * (2 * k + half) + 8);
+        for (int k = 0; k < PRE_CHUNKS; ++k) {
+          if (16 * (EPI_GROUPS * k + cg) < p.BN) {
+            pre[2 * k] = *reinterpret_cast<const uint4*>(src + 16 * (EPI_GROUPS * k + cg));
+            pre[2 * k + 1] = *reinterpret_cast<const uint4*>(src + 16 * (EPI_GROUPS * k + cg) + 8);
           }
         }
       }
@@ -351,17 +352,68 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const bool carry_wr = do_halo && (is_halo || is_chunk) && new_row >= 0 && new_row < HALO;
 
 #pragma unroll
-    for (int kk = 0; kk < MAX_BN / 32; ++kk) {
-      const int ch = 2 * kk + half;
+    for (int kk = 0; kk < MAX_BN / (16 * EPI_GROUPS); ++kk) {
+      const int ch = EPI_GROUPS * kk + cg;
       const int c0 = ch * 16;
       if (c0 >= p.BN) break;
       float acc[16];
-      ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
       if (p.n_issuers == 2) {   // even blocks + odd blocks, always in this order
         float acc2[16];
-        ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + acc2_off + (uint32_t)c0, acc2);
+        ptx::tmem_ld16x2(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, tmem_base + ((uint32_t)(q * 32) << 16) + acc2_off + (uint32_t)c0,
+                         acc, acc2);
 #pragma unroll
         for (int i = 0; i < 16; ++i) acc[i] += acc2[i];
+      } else {
+        ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
+      }
+      if (p.taps == 3) {
+        // conv block: acc holds tap 0's product for this row; y[r] = Z_0[r - shift_0] + Z_1[r - shift_1] + Z_2[r].
+        // A row is a TMEM lane, so the shift is a warp shuffle; the first rows of the warps that own
+        // slot rows 32..63 take the last rows of the warp below through shared memory (the operand
+        // stages are idle by now).  Shifts never leave the slot for the rows that are stored (<= 8
+        // left-context rows precede the chunk).
+        float z[16];
+        const uint32_t lanes = tmem_base + ((uint32_t)(q * 32) << 16);
+        if (p.n_issuers == 2) {
+          float t[16];
+          ptx::tmem_ld16x2(lanes + (uint32_t)(p.BN + c0), lanes + acc2_off + (uint32_t)(p.BN + c0), z, t);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) z[i] += t[i];
+        } else {
+          ptx::tmem_ld16(lanes + (uint32_t)(p.BN + c0), z);
+        }
+        float* xch = reinterpret_cast<float*>(smem) + (((cg * 2 + (kk & 1)) * 2 + (q >> 1)) * 8) * 32;   // [8 rows][Z_0 16 | Z_1 16]
+        if (!(q & 1) && lane >= 24) {
+          float* dst = xch + (lane - 24) * 32;
+#pragma unroll
+          for (int i = 0; i < 16; i += 4) {
+            *reinterpret_cast<float4*>(dst + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+            *reinterpret_cast<float4*>(dst + 16 + i) = make_float4(z[i], z[i + 1], z[i + 2], z[i + 3]);
+          }
+        }
+        ptx::named_bar_sync(2 + cg, 128);   // the four warps that own this chunk
+        const int s0 = p.shift[0], s1 = p.shift[1];
+        const bool below = (q & 1) != 0;      // rows 32..63 of a slot: the rows above live in the previous warp
+        const float* src0 = xch + (8 - s0 + lane) * 32;        // row 32 - s0 + lane of the slot = lane 24 + (8 - s0 + lane) of the warp below
+        const float* src1 = xch + (8 - s1 + lane) * 32 + 16;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float a0 = __shfl_up_sync(0xffffffffu, acc[i], (unsigned)s0);
+          float a1 = __shfl_up_sync(0xffffffffu, z[i], (unsigned)s1);
+          if (below && lane < s0) a0 = src0[i];
+          if (below && lane < s1) a1 = src1[i];
+          acc[i] = a0 + a1;
+        }
+        if (p.n_issuers == 2) {
+          float t[16];
+          ptx::tmem_ld16x2(lanes + (uint32_t)(2 * p.BN + c0), lanes + acc2_off + (uint32_t)(2 * p.BN + c0), z, t);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) z[i] += t[i];
+        } else {
+          ptx::tmem_ld16(lanes + (uint32_t)(2 * p.BN + c0), z);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] += z[i];
       }
       const int n = n0 + c0;
 #pragma unroll
@@ -408,7 +460,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         continue;
       }
       // modes with a bf16 activation output: INPROJ, CONV, OPROJ (BN <= 64, so kk < 2)
-      uint4 va = pre[(2 * kk) & 3], vb = pre[(2 * kk + 1) & 3];
+      uint4 va = pre[(2 * kk) % (2 * PRE_CHUNKS)], vb = pre[(2 * kk + 1) % (2 * PRE_CHUNKS)];
       if (!is_halo) {
         if (has_resid) {
           const uint32_t w[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
