@@ -74,6 +74,7 @@ struct GemmParams {
   int          n_stages;        // TMA pipeline depth (<= MAX_STAGES, n_stages * stage bytes <= GEMM_TILE_SMEM)
   int          n_slots;
   int          n_kblocks;       // 64-wide channel blocks of the A matrix (one pipeline stage each)
+  int          wide;            // conv blocks: 1 = the taps are column blocks of one wide UMMA, combined in the epilogue
   int          taps;            // 1, or 3 for the conv blocks (weights: K index = tap * 64 * n_kblocks + channel)
   int          shift[3];        // row shift of tap j (0..8)
   const float* bias;            // [N]
@@ -178,7 +179,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // and added in the epilogue; a tcgen05.mma costs about 47 cycles however small it is, and one
   // 128 x 3BN x 16 instruction replaces three 128 x BN x 16 ones).  The second issuer's accumulator
   // sits acc2_off columns after the first.
-  const uint32_t acc_w = (uint32_t)(p.taps * p.BN);
+  const uint32_t acc_w = (uint32_t)((p.wide ? p.taps : 1) * p.BN);
   const uint32_t acc2_off = acc_w <= 32 ? 32u : (acc_w <= 64 ? 64u : (acc_w <= 128 ? 128u : 256u));
   const uint32_t need_cols = p.n_issuers == 2 ? 2u * acc2_off : acc_w;
   const uint32_t tmem_cols = need_cols <= 32 ? 32u : (need_cols <= 64 ? 64u : (need_cols <= 128 ? 128u : (need_cols <= 256 ? 256u : 512u)));
@@ -254,6 +255,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       // the weight tiles of the taps are adjacent in the stage (BN rows of 128 B each, BN a multiple of 8),
       // so together they are one K-major operand of taps * BN rows
       const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.taps * p.BN, 0, 0);
+      const uint32_t idesc1 = ptx::umma_idesc_bf16(TILE_M, p.BN, 0, 0);
       const int nkb = p.n_kblocks, step = p.n_issuers;
       const uint32_t d_acc = tmem_base + (uint32_t)me * acc2_off;
       // descriptor start addresses are in 16-byte units: +2 per 32-byte K step
@@ -274,9 +276,21 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (tm && kb < 32 && on) s_k[kb] = clock64() - t_start;
 #endif
         const uint64_t da = d_a0 + (uint64_t)((uint32_t)st * stage16), db = da + ab16;
-        ptx::umma_bf16_if(on, d_acc, da + o0, db, idesc, acc);
+        if (p.taps == 3 && !p.wide) {
+          const uint32_t b16 = (uint32_t)p.BN * 8u;
+          const uint32_t t0 = (uint32_t)(HALO - p.shift[0]) * 8u, t1 = (uint32_t)(HALO - p.shift[1]) * 8u;
+          ptx::umma_bf16_if(on, d_acc, da + t0, db, idesc1, acc);
 #pragma unroll
-        for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
+          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (t0 + 2 * k), db + 2 * k, idesc1, 1);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (t1 + 2 * k), db + (b16 + 2 * k), idesc1, 1);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + (2 * b16 + 2 * k), idesc1, 1);
+        } else {
+          ptx::umma_bf16_if(on, d_acc, da + o0, db, idesc, acc);
+#pragma unroll
+          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
+        }
         acc = 1;
         ptx::umma_commit_if(on, &empty[st]);
       }
@@ -366,7 +380,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       } else {
         ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
       }
-      if (p.taps == 3) {
+      if (p.taps == 3 && p.wide) {
         // conv block: acc holds tap 0's product for this row; y[r] = Z_0[r - shift_0] + Z_1[r - shift_1] + Z_2[r].
         // A row is a TMEM lane, so the shift is a warp shuffle; the first rows of the warps that own
         // slot rows 32..63 take the last rows of the warp below through shared memory (the operand
@@ -967,6 +981,7 @@ struct FlowModel {
   // launch plumbing
   bool pdl = true;                       // programmatic dependent launch between the step's kernels
   bool one_issuer = false;               // experiments: a single UMMA issuer
+  bool wide_taps = true;                 // conv blocks: taps as column blocks of one wide UMMA (fixed at create, see flow_model_create)
   int  qkv_stages = 4;
   int  wide_stages = 4;                  // 2 or 4 (even, see the stage count rule in enqueue_chunk)
   int  dbg = 0;
@@ -1172,6 +1187,14 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     m->pdl = !(e && atoi(e));
     const char* d = getenv("DC_GEMM_DBG");
     m->dbg = d ? atoi(d) : 0;
+    // How a conv block's taps are computed is part of the arithmetic (it fixes the order of the fp32
+    // sums), so it is chosen once per model, never per call: batched and single-stream calls of one
+    // model agree bit for bit.  One wide UMMA per reduction step + shift-and-add in the epilogue wins
+    // while tiles are narrow (few streams: the ~47-cycle floor of a tcgen05.mma dominates); three
+    // UMMAs accumulating in place win once a full batch runs 64-column tiles, where the epilogue's
+    // row shifts cost more than the main loop saves.
+    m->wide_taps = ((m->S * SLOT_ROWS + TILE_M - 1) / TILE_M) * (m->C / 64) < 96;
+    if (const char* wt = getenv("DC_WIDE_TAPS")) m->wide_taps = atoi(wt) != 0;   // experiments only
     const char* oi = getenv("DC_ONE_ISSUER");
     m->one_issuer = oi && atoi(oi);
     const char* qs = getenv("DC_QKV_STAGES");
@@ -1385,7 +1408,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       for (int j = 0; j < m->cpa; ++j, ++l) {
         const int d = c.dilations[l];
         GemmParams p{};
-        p.mode = MODE_CONV; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 3;
+        p.mode = MODE_CONV; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 3; p.wide = m->wide_taps ? 1 : 0;
         p.shift[0] = 2 * d; p.shift[1] = d; p.shift[2] = 0;
         p.bias = fc + m->o_bconv[l]; p.tau = fc + m->o_tau + ((size_t)s * c.n_conv + l) * C;
         p.resid = X; p.out = Y;
