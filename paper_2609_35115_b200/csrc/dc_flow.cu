@@ -599,9 +599,18 @@ constexpr int ATT_TMEM_COLS = 256;      // S (128 columns) + O (64 columns); two
 constexpr int ATT_K_LOADERS = 64;       // warps 5 and 6: Q, then the K blocks
 constexpr int ATT_V_LOADERS = 32;       // warp 7: the V blocks
 constexpr int ATT_Q_BYTES = 128 * 128;  // 64 query rows, twice
-constexpr int ATT_P_BYTES = 2 * 64 * 128;
+constexpr int ATT_P_BYTES = 2 * 64 * 128;   // one P buffer: 64 rows x 128 keys; there are two
 constexpr int ATT_STAGE_BYTES = 2 * ATT_KB * 128;   // K block + V block
-constexpr size_t ATT_SMEM = 1024 + ATT_Q_BYTES + ATT_P_BYTES + ATT_STAGES * ATT_STAGE_BYTES + 1024;
+constexpr int ATT_BAR_BYTES = 1024;        // 14 barriers, TMEM slot, softmax exchange (512 B)
+// Two CTAs per SM leave 113 KB each: the tiles take 112 KB, so there is no room for alignment slack.
+// The dynamic shared memory is declared 1024-byte aligned (the swizzled tiles need it) and the kernel
+// checks the address it got.
+#ifdef DC_TIMING
+constexpr size_t ATT_SMEM = 1024 + ATT_Q_BYTES + 2 * ATT_P_BYTES + ATT_STAGES * ATT_STAGE_BYTES + ATT_BAR_BYTES;
+#else
+constexpr size_t ATT_SMEM = ATT_Q_BYTES + 2 * ATT_P_BYTES + ATT_STAGES * ATT_STAGE_BYTES + ATT_BAR_BYTES;
+#endif
+static_assert(ATT_SMEM <= 113 * 1024 + 1024, "two attention CTAs must fit one SM");
 constexpr float ATT_RESCALE_LOG2 = 8.0f;
 
 struct AttnParams {
@@ -627,11 +636,19 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
 }
 
 __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) uint8_t att_smem_raw[];
+#ifdef DC_TIMING
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem_raw) + 1023) & ~(uintptr_t)1023);
+#else
+  uint8_t* smem = att_smem_raw;
+  if ((ptx::smem_u32(smem) & 1023u) != 0u) {   // would corrupt the swizzled tiles: refuse (uniform for the CTA)
+    if (threadIdx.x == 0) atomicExch(p.err, 14);
+    return;
+  }
+#endif
   uint8_t* sQ = smem;
-  uint8_t* sP = sQ + ATT_Q_BYTES;                    // tile t (keys 64 t .. 64 t + 63 of the block) at + 8192 t
-  uint8_t* ring = sP + ATT_P_BYTES;
+  uint8_t* sP = sQ + ATT_Q_BYTES;                    // buffer b & 1 at + ATT_P_BYTES (b & 1); tile t (keys 64 t .. of the block) at + 8192 t
+  uint8_t* ring = sP + 2 * ATT_P_BYTES;
   // K and V have their own two-stage rings: a K stage is free as soon as S of its block has been
   // computed, long before the V stage of the same block (free after P V), so K runs further ahead.
   uint64_t* full_k = reinterpret_cast<uint64_t*>(ring + ATT_STAGES * ATT_STAGE_BYTES);   // [ATT_STAGES] each
@@ -639,9 +656,11 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   uint64_t* full_v = empty_k + ATT_STAGES;
   uint64_t* empty_v = full_v + ATT_STAGES;
   uint64_t* bar_s = empty_v + ATT_STAGES;
-  uint64_t* bar_p = bar_s + 1;
-  uint64_t* bar_pv = bar_p + 1;
-  uint64_t* bar_sfree = bar_pv + 1;     // every softmax thread has copied its S columns to registers
+  // P and "P V done" have one barrier per P buffer (block parity): with a single barrier a waiter
+  // that falls a whole block behind could not tell phase b from phase b + 2.
+  uint64_t* bar_p = bar_s + 1;          // [2]: all softmax threads have written P(b) into buffer b & 1
+  uint64_t* bar_pv = bar_p + 2;         // [2]: P(b) V(b) has been accumulated: buffer b & 1 is free, O holds blocks <= b
+  uint64_t* bar_sfree = bar_pv + 2;     // every softmax thread has copied its S columns to registers
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_sfree + 1);
   float* s_x = reinterpret_cast<float*>(tmem_slot + 2);   // [2][64] exchange between the two column halves
 
@@ -665,8 +684,10 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       ptx::mbar_init(&empty_v[i], 1);
     }
     ptx::mbar_init(bar_s, 1);
-    ptx::mbar_init(bar_p, 128);
-    ptx::mbar_init(bar_pv, 1);
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(&bar_p[i], 128);
+      ptx::mbar_init(&bar_pv[i], 1);
+    }
     ptx::mbar_init(bar_sfree, 128);
     ptx::fence_barrier_init();
   }
@@ -762,7 +783,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
           if (ok && !ptx::mbar_wait(bar_sfree, b & 1)) { ok = false; atomicExch(p.err, 10); }
           issue_s(b + 1);
         }
-        if (ok && !ptx::mbar_wait(bar_p, b & 1)) { ok = false; atomicExch(p.err, 6); }
+        if (ok && !ptx::mbar_wait(&bar_p[b & 1], (b >> 1) & 1)) { ok = false; atomicExch(p.err, 6); }
+        const uint64_t dpb = dp + (uint64_t)((b & 1) * (ATT_P_BYTES >> 4));
         if (ok && !ptx::mbar_wait(&full_v[st], (b / ATT_STAGES) & 1)) { ok = false; atomicExch(p.err, 11); }
         ptx::tc_fence_after();
         const uint64_t dv = ptx::umma_desc_sw128(ptx::smem_u32(ring + st * ATT_STAGE_BYTES + ATT_KB * 128));
@@ -772,15 +794,15 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         if (ksteps == ATT_KB / 16) {
 #pragma unroll
           for (int k = 0; k < ATT_KB / 16; ++k)
-            ptx::umma_bf16(tmem_base + ATT_KB, dp + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
+            ptx::umma_bf16(tmem_base + ATT_KB, dpb + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
                            idesc_pv, (b | k) != 0);
         } else {
           for (int k = 0; k < ksteps; ++k)
-            ptx::umma_bf16(tmem_base + ATT_KB, dp + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
+            ptx::umma_bf16(tmem_base + ATT_KB, dpb + (uint64_t)((k >> 2) * (8192 >> 4) + (k & 3) * 2), dv + (uint64_t)(k * (2048 >> 4)),
                            idesc_pv, (b | k) != 0);
         }
         ptx::umma_commit(&empty_v[st]);
-        ptx::umma_commit(bar_pv);
+        ptx::umma_commit(&bar_pv[b & 1]);
         if (b < 8) DC_AT(24 + b);                        // PV(b) issued
       }
     }
@@ -813,15 +835,15 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       s_x[half * 64 + row] = mx * p.scale_log2e;
       ptx::named_bar_sync(2, 128);
       mx = fmaxf(s_x[row], s_x[64 + row]);
-      if (b > 0) {   // P V of the previous block must be done: P tile free, O quiescent
-        if (ok && !ptx::mbar_wait(bar_pv, (b - 1) & 1)) { ok = false; atomicExch(p.err, 8); }
-        ptx::tc_fence_after();
-      }
+      ptx::named_bar_sync(2, 128);   // all have read: the next block (or the row sums below) may overwrite the exchange
       if (b == 0) {
         m_ref = mx;
       } else {
         const bool need = mx > m_ref + ATT_RESCALE_LOG2;
         if (__any_sync(0xffffffffu, need)) {
+          // O must hold every earlier block and be quiescent before it is rescaled
+          if (ok && !ptx::mbar_wait(&bar_pv[(b - 1) & 1], ((b - 1) >> 1) & 1)) { ok = false; atomicExch(p.err, 8); }
+          ptx::tc_fence_after();
           const float alpha = need ? exp2f(m_ref - mx) : 1.0f;
           if (need) m_ref = mx;
           lsum *= alpha;
@@ -835,9 +857,13 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
               ptx::tmem_st16(addr, o16);
             }
           }
+          ptx::tc_fence_before();
         }
       }
-      uint8_t* prow = sP + half * 8192 + row * 128;
+      if (b >= 2) {   // this block's P buffer was last read by P V of block b - 2
+        if (ok && !ptx::mbar_wait(&bar_pv[b & 1], ((b >> 1) - 1) & 1)) { ok = false; atomicExch(p.err, 15); }
+      }
+      uint8_t* prow = sP + (b & 1) * ATT_P_BYTES + half * 8192 + row * 128;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         float e[16];
@@ -853,12 +879,11 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       }
       ptx::fence_proxy_async_smem();
       ptx::tc_fence_before();
-      ptx::mbar_arrive(bar_p);
+      ptx::mbar_arrive(&bar_p[b & 1]);
       if (tid == 0 && b < 8) DC_AT(40 + b);              // P(b) written
     }
-    if (ok && !ptx::mbar_wait(bar_pv, (nkb - 1) & 1)) { ok = false; atomicExch(p.err, 9); }
+    if (ok && !ptx::mbar_wait(&bar_pv[(nkb - 1) & 1], ((nkb - 1) >> 1) & 1)) { ok = false; atomicExch(p.err, 9); }
     ptx::tc_fence_after();
-    ptx::named_bar_sync(2, 128);       // every thread is past its last read of s_x
     s_x[half * 64 + row] = lsum;
     ptx::named_bar_sync(2, 128);
     const float inv = 1.0f / (s_x[row] + s_x[64 + row]);
