@@ -383,6 +383,56 @@ def main():
         roof["attention_hbm_gbs"] = attention_bytes_per_launch(cfg, S) / a_s / 1e9
         roof["attention_hbm_frac"] = roof["attention_hbm_gbs"] / pk["hbm_gbs"]
 
+    # ---- cost of the two main kernel classes INSIDE the captured graph (flow workloads, N = 1 only) ----
+    # The event-bracketed pass above times direct launches: every bracket adds launch latency and
+    # takes away the overlap between consecutive kernels.  What a class costs in the real step is the
+    # step time with it minus the step time without it: the library can leave a class out of the
+    # graph (environment variable read at dc_create; the outputs are then meaningless, the timing
+    # of everything else is not).
+    if cfg.pipeline == "flow" and world == 1:
+        def step_ms_without(bits: int) -> float:
+            os.environ["DC_GEMM_DBG"] = str(bits)
+            try:
+                m2 = dc.Model(cfg, weights, max_batch=S)
+            finally:
+                os.environ.pop("DC_GEMM_DBG", None)
+            st2 = [m2.open_stream() for _ in range(S)]
+            def step2(r):
+                if batched:
+                    dc.decode_batch(m2, st2, feats_d[r], out_dv)
+                else:
+                    for i in range(S):
+                        st2[i].decode_chunk(feats_d[r, i], out=out_d[i])
+            for r in range(history + W):
+                step2(r)
+            torch.cuda.synchronize()
+            n2 = min(K, 30)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for k in range(n2):
+                step2(history + W + k)
+            b.record()
+            torch.cuda.synchronize()
+            for s2 in st2:
+                s2.close()
+            m2.destroy()
+            return a.elapsed_time(b) / n2
+        full_ms = total_ms / K
+        n_conv_l = kernels.get("gemm_conv", {}).get("launches_per_step", 0)
+        n_att_l = kernels.get("attention", {}).get("launches_per_step", 0)
+        in_graph = {"method": "step time minus the step time of a graph without the class, both over CUDA events"}
+        if n_conv_l:
+            us = 1e3 * (full_ms - step_ms_without(1024)) / n_conv_l
+            in_graph["conv_gemm_us"] = us
+            in_graph["conv_gemm_tflops"] = flops_per_launch(cfg, "gemm_conv", S) / (us * 1e-6) / 1e12
+            in_graph["conv_gemm_frac"] = in_graph["conv_gemm_tflops"] / pk["bf16_tflops_sustained"]
+        if n_att_l:
+            us = 1e3 * (full_ms - step_ms_without(32)) / n_att_l
+            in_graph["attention_us"] = us
+            in_graph["attention_hbm_gbs"] = attention_bytes_per_launch(cfg, S) / (us * 1e-6) / 1e9
+            in_graph["attention_hbm_frac"] = in_graph["attention_hbm_gbs"] / pk["hbm_gbs"]
+        roof["in_graph"] = in_graph
+
     # ---- the oracle on the host cores (rank 0, N = 1 only), bounded sample ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -1440,7 +1440,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
         const bool next_is_conv = (j + 1 < m->cpa);
         p.halo_off = next_is_conv ? ((long long)s * c.n_conv + l + 1) * halo_stride : -1;
         if (!next_is_conv) feeds_norm(p);   // the group's attention norm, or the final norm of a conv-only stack
-        gemm(*tX, m->tmWconv[v][l], p, C);
+        if (!(m->dbg & 1024)) gemm(*tX, m->tmWconv[v][l], p, C);   // bit 1024 (measurement only): without the conv-block kernels
         swap();
       }
       if (c.n_attn > 0) {
@@ -1452,7 +1452,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
           normalised(p);
           gemm(*tX, m->tmWqkv[v][g], p, 3 * C);
         }
-        attention(s, g);
+        if (!(m->dbg & 32)) attention(s, g);    // DC_GEMM_DBG bit 32 (measurement only): the step without its attention kernels
         {
           GemmParams p{};
           p.mode = MODE_OPROJ; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 1;
