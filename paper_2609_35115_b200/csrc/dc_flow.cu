@@ -39,8 +39,7 @@ constexpr int HALO = 8;         // carried frames per (step, conv block); dilati
 constexpr int TILE_M = 128;
 constexpr int KBLK = 64;        // bf16 elements per 128-byte swizzled smem row
 constexpr int MAX_STAGES = 8;
-constexpr int GEMM_TILE_SMEM = 88 * 1024;    // operand stages per CTA: small enough for two CTAs per SM, so that
-                                             // the next kernel's prologue and weight prefetch overlap this one's tail
+constexpr int GEMM_TILE_SMEM = 88 * 1024;    // operand stages of the single-issuer GEMMs (a short reduction needs no deeper ring)
 constexpr int A_ROWS = TILE_M + HALO;  // the A tile carries 8 extra leading rows so that all taps read it
 constexpr int A_BYTES = A_ROWS * 128;
 constexpr int MAX_BN = 192;
@@ -117,16 +116,6 @@ __device__ __forceinline__ float silu_f(float z) {
   return fmaf(h, t, h);
 }
 
-__device__ __forceinline__ void load16_bf16(const bf16* p, float* v) {
-  const uint4 a = *reinterpret_cast<const uint4*>(p);
-  const uint4 b = *reinterpret_cast<const uint4*>(p + 8);
-  const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-  }
-}
 __device__ __forceinline__ void pack16_bf16(const float* v, uint4& a, uint4& b) {
   uint32_t w[8];
 #pragma unroll
@@ -1381,8 +1370,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     // width chosen for the batch size (batched and single-stream results must agree bit for bit);
     // the QKV and output projections keep one issuer (their wide tiles would not fit two accumulators)
     p.n_issuers = (p.mode != MODE_QKV && p.mode != MODE_OUT && p.n_kblocks >= 2 && !m->one_issuer) ? 2 : 1;
-    // Stage count.  Two or three stages (<= 88 KB) let two CTAs share an SM, so that the next kernel's
-    // prologue overlaps this kernel's tail.  With two issuers the count must be EVEN: issuer i takes
+    // Stage count.  With two issuers the count must be EVEN: issuer i takes
     // the reduction blocks kb = i (mod 2), and only with an even ring does every stage always belong
     // to the same issuer - a parity wait cannot tell "my block has landed" from "the other issuer's
     // earlier block has landed" on a stage that both use.
