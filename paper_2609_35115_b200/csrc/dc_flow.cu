@@ -40,7 +40,7 @@ constexpr int TILE_M = 128;
 constexpr int KBLK = 64;        // bf16 elements per 128-byte swizzled smem row
 constexpr int MAX_STAGES = 8;
 constexpr int GEMM_TILE_SMEM = 88 * 1024;    // operand stages of the single-issuer GEMMs (a short reduction needs no deeper ring)
-constexpr int A_ROWS = TILE_M + HALO;  // the A tile carries 8 extra leading rows so that all taps read it
+constexpr int A_ROWS = TILE_M;         // rows of an A box = rows of the output tile (the conv taps are shifted in the epilogue)
 constexpr int A_BYTES = A_ROWS * 128;
 constexpr int MAX_BN = 192;
 constexpr int EPI_GROUPS = 4;           // epilogue warps per TMEM lane quarter: group g owns the 16-column chunks g, g + 4, ...
@@ -73,7 +73,6 @@ struct GemmParams {
   int          n_stages;        // TMA pipeline depth (<= MAX_STAGES, n_stages * stage bytes <= GEMM_TILE_SMEM)
   int          n_slots;
   int          n_kblocks;       // 64-wide channel blocks of the A matrix (one pipeline stage each)
-  int          wide;            // conv blocks: 1 = the taps are column blocks of one wide UMMA, combined in the epilogue
   int          taps;            // 1, or 3 for the conv blocks (weights: K index = tap * 64 * n_kblocks + channel)
   int          shift[3];        // row shift of tap j (0..8)
   const float* bias;            // [N]
@@ -135,9 +134,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  // stage = [A tile 136 x 128 B | one B tile BN x 128 B per tap]; all tile sizes are multiples of
-  // 1024 B.  The A tile starts 8 rows above the output tile: tap j reads it from row 8 - shift[j],
-  // so one load serves all taps.
+  // stage = [A tile 128 x 128 B | one B tile BN x 128 B per tap]; all tile sizes are multiples of
+  // 1024 B.  The weight tiles of a conv block's three taps are adjacent, so that they form one
+  // operand of 3 BN rows.
   const uint32_t b_bytes = (uint32_t)p.BN * 128u;
   const uint32_t b_tile = (b_bytes + 1023u) & ~1023u;
   const uint32_t stage_bytes = (uint32_t)A_BYTES + (uint32_t)p.taps * b_tile;
@@ -168,7 +167,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // and added in the epilogue; a tcgen05.mma costs about 47 cycles however small it is, and one
   // 128 x 3BN x 16 instruction replaces three 128 x BN x 16 ones).  The second issuer's accumulator
   // sits acc2_off columns after the first.
-  const uint32_t acc_w = (uint32_t)((p.wide ? p.taps : 1) * p.BN);
+  const uint32_t acc_w = (uint32_t)(p.taps * p.BN);
   const uint32_t acc2_off = acc_w <= 32 ? 32u : (acc_w <= 64 ? 64u : (acc_w <= 128 ? 128u : 256u));
   const uint32_t need_cols = p.n_issuers == 2 ? 2u * acc2_off : acc_w;
   const uint32_t tmem_cols = need_cols <= 32 ? 32u : (need_cols <= 64 ? 64u : (need_cols <= 128 ? 128u : (need_cols <= 256 ? 256u : 512u)));
@@ -198,7 +197,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const uint32_t on = lane == 0;   // the whole warp runs the loop, lane 0 issues
       const bool is_a = warp == 0;
       const int nkb = p.n_kblocks, taps = p.taps;
-      const int ya = GUARD + m0 - HALO;
+      const int ya = GUARD + m0;
       const uint32_t tx_bytes = is_a ? (uint32_t)A_BYTES : (uint32_t)taps * b_bytes;
       uint8_t* dst = smem + (is_a ? 0 : A_BYTES);
       int st = 0;
@@ -244,13 +243,11 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       // the weight tiles of the taps are adjacent in the stage (BN rows of 128 B each, BN a multiple of 8),
       // so together they are one K-major operand of taps * BN rows
       const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.taps * p.BN, 0, 0);
-      const uint32_t idesc1 = ptx::umma_idesc_bf16(TILE_M, p.BN, 0, 0);
       const int nkb = p.n_kblocks, step = p.n_issuers;
       const uint32_t d_acc = tmem_base + (uint32_t)me * acc2_off;
       // descriptor start addresses are in 16-byte units: +2 per 32-byte K step
       const uint64_t d_a0 = ptx::umma_desc_sw128(ptx::smem_u32(smem));
       const uint32_t stage16 = stage_bytes >> 4, ab16 = A_BYTES >> 4;
-      const uint32_t o0 = (uint32_t)HALO * 8u;   // the output tile's own rows start 8 rows into the A tile (rows * 128 B / 16)
       uint32_t acc = 0;
       for (int kb = me; kb < nkb; kb += step) {
         const int st = kb % STAGES;
@@ -265,21 +262,9 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (tm && kb < 32 && on) s_k[kb] = clock64() - t_start;
 #endif
         const uint64_t da = d_a0 + (uint64_t)((uint32_t)st * stage16), db = da + ab16;
-        if (p.taps == 3 && !p.wide) {
-          const uint32_t b16 = (uint32_t)p.BN * 8u;
-          const uint32_t t0 = (uint32_t)(HALO - p.shift[0]) * 8u, t1 = (uint32_t)(HALO - p.shift[1]) * 8u;
-          ptx::umma_bf16_if(on, d_acc, da + t0, db, idesc1, acc);
+        ptx::umma_bf16_if(on, d_acc, da, db, idesc, acc);
 #pragma unroll
-          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (t0 + 2 * k), db + 2 * k, idesc1, 1);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (t1 + 2 * k), db + (b16 + 2 * k), idesc1, 1);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + (2 * b16 + 2 * k), idesc1, 1);
-        } else {
-          ptx::umma_bf16_if(on, d_acc, da + o0, db, idesc, acc);
-#pragma unroll
-          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + (o0 + 2 * k), db + 2 * k, idesc, 1);
-        }
+        for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + 2 * k, db + 2 * k, idesc, 1);
         acc = 1;
         ptx::umma_commit_if(on, &empty[st]);
       }
@@ -369,12 +354,11 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       } else {
         ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
       }
-      if (p.taps == 3 && p.wide) {
+      if (p.taps == 3) {
         // conv block: acc holds tap 0's product for this row; y[r] = Z_0[r - shift_0] + Z_1[r - shift_1] + Z_2[r].
-        // A row is a TMEM lane, so the shift is a warp shuffle; the first rows of the warps that own
-        // slot rows 32..63 take the last rows of the warp below through shared memory (the operand
-        // stages are idle by now).  Shifts never leave the slot for the rows that are stored (<= 8
-        // left-context rows precede the chunk).
+        // A row is a TMEM lane, which a thread cannot change, so the shifted rows go through shared memory
+        // (the operand stages are idle by now).  Shifts never leave the slot for the rows that are
+        // stored (<= 8 left-context rows precede the chunk).
         float z[16];
         const uint32_t lanes = tmem_base + ((uint32_t)(q * 32) << 16);
         if (p.n_issuers == 2) {
@@ -385,27 +369,24 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         } else {
           ptx::tmem_ld16(lanes + (uint32_t)(p.BN + c0), z);
         }
-        float* xch = reinterpret_cast<float*>(smem) + (((cg * 2 + (kk & 1)) * 2 + (q >> 1)) * 8) * 32;   // [8 rows][Z_0 16 | Z_1 16]
-        if (!(q & 1) && lane >= 24) {
-          float* dst = xch + (lane - 24) * 32;
+        // exchange area of this chunk group: Z_0 then Z_1, each [4 float4 columns][128 rows] (a warp's 32 rows
+        // are 512 contiguous bytes, shifted or not: no bank conflicts); conv tiles have <= 64 columns, so kk = 0
+        float4* xz = reinterpret_cast<float4*>(smem) + cg * (2 * 4 * TILE_M);
+        const int row_t = q * 32 + lane;
 #pragma unroll
-          for (int i = 0; i < 16; i += 4) {
-            *reinterpret_cast<float4*>(dst + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
-            *reinterpret_cast<float4*>(dst + 16 + i) = make_float4(z[i], z[i + 1], z[i + 2], z[i + 3]);
-          }
+        for (int j = 0; j < 4; ++j) {
+          xz[j * TILE_M + row_t] = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+          xz[(4 + j) * TILE_M + row_t] = make_float4(z[4 * j], z[4 * j + 1], z[4 * j + 2], z[4 * j + 3]);
         }
         ptx::named_bar_sync(2 + cg, 128);   // the four warps that own this chunk
-        const int s0 = p.shift[0], s1 = p.shift[1];
-        const bool below = (q & 1) != 0;      // rows 32..63 of a slot: the rows above live in the previous warp
-        const float* src0 = xch + (8 - s0 + lane) * 32;        // row 32 - s0 + lane of the slot = lane 24 + (8 - s0 + lane) of the warp below
-        const float* src1 = xch + (8 - s1 + lane) * 32 + 16;
+        const int r0 = max(row_t - p.shift[0], 0), r1 = max(row_t - p.shift[1], 0);   // (row 0 of a tile is a left-context row)
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float a0 = __shfl_up_sync(0xffffffffu, acc[i], (unsigned)s0);
-          float a1 = __shfl_up_sync(0xffffffffu, z[i], (unsigned)s1);
-          if (below && lane < s0) a0 = src0[i];
-          if (below && lane < s1) a1 = src1[i];
-          acc[i] = a0 + a1;
+        for (int j = 0; j < 4; ++j) {
+          const float4 a0 = xz[j * TILE_M + r0], a1 = xz[(4 + j) * TILE_M + r1];
+          acc[4 * j] = a0.x + a1.x;
+          acc[4 * j + 1] = a0.y + a1.y;
+          acc[4 * j + 2] = a0.z + a1.z;
+          acc[4 * j + 3] = a0.w + a1.w;
         }
         if (p.n_issuers == 2) {
           float t[16];
@@ -995,7 +976,6 @@ struct FlowModel {
   // launch plumbing
   bool pdl = true;                       // programmatic dependent launch between the step's kernels
   bool one_issuer = false;               // experiments: a single UMMA issuer
-  bool wide_taps = true;                 // conv blocks: taps as column blocks of one wide UMMA (fixed at create, see flow_model_create)
   int  qkv_stages = 4;
   int  wide_stages = 4;                  // 2 or 4 (even, see the stage count rule in enqueue_chunk)
   int  dbg = 0;
@@ -1201,14 +1181,6 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     m->pdl = !(e && atoi(e));
     const char* d = getenv("DC_GEMM_DBG");
     m->dbg = d ? atoi(d) : 0;
-    // How a conv block's taps are computed is part of the arithmetic (it fixes the order of the fp32
-    // sums), so it is chosen once per model, never per call: batched and single-stream calls of one
-    // model agree bit for bit.  One wide UMMA per reduction step + shift-and-add in the epilogue wins
-    // while tiles are narrow (few streams: the ~47-cycle floor of a tcgen05.mma dominates); three
-    // UMMAs accumulating in place win once a full batch runs 64-column tiles, where the epilogue's
-    // row shifts cost more than the main loop saves.
-    m->wide_taps = ((m->S * SLOT_ROWS + TILE_M - 1) / TILE_M) * (m->C / 64) < 96;
-    if (const char* wt = getenv("DC_WIDE_TAPS")) m->wide_taps = atoi(wt) != 0;   // experiments only
     const char* oi = getenv("DC_ONE_ISSUER");
     m->one_issuer = oi && atoi(oi);
     const char* qs = getenv("DC_QKV_STAGES");
@@ -1421,7 +1393,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       for (int j = 0; j < m->cpa; ++j, ++l) {
         const int d = c.dilations[l];
         GemmParams p{};
-        p.mode = MODE_CONV; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 3; p.wide = m->wide_taps ? 1 : 0;
+        p.mode = MODE_CONV; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 3;
         p.shift[0] = 2 * d; p.shift[1] = d; p.shift[2] = 0;
         p.bias = fc + m->o_bconv[l]; p.tau = fc + m->o_tau + ((size_t)s * c.n_conv + l) * C;
         p.resid = X; p.out = Y;
