@@ -107,6 +107,9 @@ class ClockSampler:
 
 
 def describe(cfg) -> str:
+    if cfg.pipeline == "token2wav":
+        return (describe(cfg.flow_part()).replace(cfg.name + ".flow", cfg.name) + " -> mel frames on the device -> "
+                + describe(cfg.vocoder_part()).split(": ", 1)[1])
     if cfg.pipeline == "flow":
         return (f"{cfg.name}: {cfg.n_streams} stream(s) x flow decoder C={cfg.hidden}, {len(cfg.dilations)} conv blocks, "
                 f"{cfg.n_attn_layers} attention layers ({cfg.n_heads}x{cfg.head_dim}, KV cap {cfg.kv_cap}), "
@@ -219,12 +222,12 @@ def main():
     ap.add_argument("--steps", type=int, default=60)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg5", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--workload", default="cfg5", choices=sorted(wl.CONFIGS) + sorted(wl.EXTRA_CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--history", type=int, default=None,
                     help="untimed chunks decoded per stream before warm-up (default: enough to fill the K/V carry)")
     args = ap.parse_args()
-    cfg = wl.CONFIGS[args.workload]
+    cfg = wl.CONFIGS.get(args.workload) or wl.EXTRA_CONFIGS[args.workload]
     if args.impl == "reference":
         run_reference(args, cfg)
         return
@@ -246,7 +249,8 @@ def main():
     metric, unit, per_chunk = units_per_chunk(cfg)
     S, T = cfg.n_streams, cfg.f_chunk
     W, K = max(args.warmup, 3), args.steps
-    history = HISTORY_CHUNKS if cfg.pipeline == "flow" else 2
+    has_flow = cfg.pipeline in ("flow", "token2wav")
+    history = HISTORY_CHUNKS if has_flow else 2
     if args.history is not None:
         history = args.history
     rounds = history + W + K
@@ -257,7 +261,7 @@ def main():
     feats_h = torch.from_numpy(rng.standard_normal((rounds, S, T, cfg.in_dim), dtype=np.float32))
     feats_d = feats_h.cuda()
     out_d = torch.empty(S, T * cfg.out_per_frame, device="cuda")
-    out_dv = out_d.view(S, T, -1) if cfg.pipeline != "vocoder" else out_d
+    out_dv = out_d.view(S, T, -1) if cfg.pipeline not in ("vocoder", "token2wav") else out_d
     batched = cfg.pipeline == "flow" and S > 1
 
     def step(r):
@@ -310,7 +314,7 @@ def main():
 
     # ---- the same step with L2 flushed first (workloads whose working set fits L2 only): a stream paced
     # at its real-time cadence finds its weights and carries in HBM, not in L2 ----
-    ws_mb = (S * (cfg.n_steps * cfg.n_attn_layers * 2 * (cfg.kv_cap + T) * cfg.hidden * 2) / 1e6) if cfg.pipeline == "flow" else 0.0
+    ws_mb = (S * (cfg.n_steps * cfg.n_attn_layers * 2 * (cfg.kv_cap + T) * cfg.hidden * 2) / 1e6) if has_flow else 0.0
     cold = None
     if ws_mb <= 126:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -331,7 +335,7 @@ def main():
     # ---- end to end through the host-buffer entry points (H2D + decode + D2H + sync per step) ----
     fin = [feats_h[r].pin_memory() for r in range(history + W, rounds)]
     fout = torch.empty(S, T * cfg.out_per_frame).pin_memory()
-    fout_v = fout.view(S, T, -1) if cfg.pipeline != "vocoder" else fout
+    fout_v = fout.view(S, T, -1) if cfg.pipeline not in ("vocoder", "token2wav") else fout
     e2e_warm = min(3, K)
     def e2e_step(k):
         if batched:
@@ -389,7 +393,7 @@ def main():
     # step time with it minus the step time without it: the library can leave a class out of the
     # graph (environment variable read at dc_create; the outputs are then meaningless, the timing
     # of everything else is not).
-    if cfg.pipeline == "flow" and world == 1:
+    if has_flow and world == 1:
         def step_ms_without(bits: int) -> float:
             os.environ["DC_GEMM_DBG"] = str(bits)
             try:
@@ -446,7 +450,7 @@ def main():
         line = {
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if cfg.precision == "bf16" else "f32", "data": "synthetic",
+            "dtype": ("bf16+f32" if cfg.pipeline == "token2wav" else "bf16" if cfg.precision == "bf16" else "f32"), "data": "synthetic",
             "config": {"workload": describe(cfg), "streams_per_gpu": S, "frames_per_chunk": T,
                        "history_chunks": history, "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": (f"K/V carries {ws:.0f} MB > 126 MB L2, streamed from HBM every step" if ws > 126 else

@@ -36,12 +36,13 @@ import numpy as np
 PIPE_CONV = "conv"
 PIPE_FLOW = "flow"
 PIPE_VOCODER = "vocoder"
+PIPE_TOKEN2WAV = "token2wav"           # flow decoder feeding the vocoder tail inside one decode call
 
 
 @dataclass(frozen=True)
 class DCConfig:
     name: str
-    pipeline: str                       # conv | flow | vocoder
+    pipeline: str                       # conv | flow | vocoder | token2wav
     precision: str                      # f32 | bf16 (fp32 accumulate)
     hidden: int = 0                     # C
     dilations: Tuple[int, ...] = ()     # one per conv block (flow / conv pipelines)
@@ -77,7 +78,7 @@ class DCConfig:
         """Width of one input frame handed to decode_chunk."""
         if self.pipeline == PIPE_CONV:
             return self.hidden
-        if self.pipeline == PIPE_FLOW:
+        if self.pipeline in (PIPE_FLOW, PIPE_TOKEN2WAV):
             return 2 * self.mel_dim      # cols [0,mel) = conditioning mu, [mel,2mel) = noise x0
         return self.mel_dim
 
@@ -95,12 +96,24 @@ class DCConfig:
     def replace(self, **kw) -> "DCConfig":
         return dataclasses.replace(self, **kw)
 
+    # token2wav = the flow decoder (bf16) followed by the vocoder tail (fp32): the two halves as
+    # configurations of their own (weights: the flow blob, then the vocoder blob)
+    def flow_part(self) -> "DCConfig":
+        assert self.pipeline == PIPE_TOKEN2WAV
+        return self.replace(name=self.name + ".flow", pipeline=PIPE_FLOW, precision="bf16")
+
+    def vocoder_part(self) -> "DCConfig":
+        assert self.pipeline == PIPE_TOKEN2WAV
+        return self.replace(name=self.name + ".vocoder", pipeline=PIPE_VOCODER, precision="f32")
+
 
 def blob_layout(cfg: DCConfig) -> List[Tuple[str, Tuple[int, ...], int]]:
     """(name, shape, fan_in) of every tensor of the canonical blob, in order.
     fan_in == 0 marks a bias."""
     out: List[Tuple[str, Tuple[int, ...], int]] = []
     C = cfg.hidden
+    if cfg.pipeline == PIPE_TOKEN2WAV:
+        return blob_layout(cfg.flow_part()) + blob_layout(cfg.vocoder_part())
     if cfg.pipeline == PIPE_CONV:
         for l in range(len(cfg.dilations)):
             out.append((f"conv{l}.W", (3, C, C), 3 * C))
@@ -227,6 +240,26 @@ def tiny_flow(**kw) -> DCConfig:
                     dilations=(1, 2), n_attn_layers=2, n_heads=2, head_dim=32, kv_cap=24,
                     n_steps=3, f_chunk=10, n_chunks=6, seed=11, bias_std=0.1)
     return base.replace(**kw)
+
+
+def token2wav(**kw) -> DCConfig:
+    """cfg3's flow decoder feeding cfg4's vocoder tail: one call turns a 50-frame chunk of
+    [conditioning | noise] into 24,000 PCM samples (the whole decoder step of the method)."""
+    f, v = CONFIGS["cfg3"], CONFIGS["cfg4"]
+    base = f.replace(name="token2wav", pipeline=PIPE_TOKEN2WAV, up_strides=v.up_strides, up_channels=v.up_channels,
+                     res_dilations=v.res_dilations, n_chunks=20, seed=6)
+    return base.replace(**kw)
+
+
+def tiny_token2wav(**kw) -> DCConfig:
+    f = tiny_flow()
+    base = f.replace(name="tiny_token2wav", pipeline=PIPE_TOKEN2WAV, mel_dim=16, up_strides=(3, 2), up_channels=(16, 8, 8),
+                     seed=13)
+    return base.replace(**kw)
+
+
+# beyond the five: the whole decoder step in one call
+EXTRA_CONFIGS: Dict[str, DCConfig] = {"token2wav": token2wav()}
 
 
 def tiny_vocoder(**kw) -> DCConfig:

@@ -54,7 +54,7 @@ typedef enum dc_status {
   DC_ERR_STATE = 7     /* closed or poisoned stream, or streams of different models          */
 } dc_status;
 
-enum { DC_PIPE_CONV = 1, DC_PIPE_FLOW = 2, DC_PIPE_VOCODER = 3 };
+enum { DC_PIPE_CONV = 1, DC_PIPE_FLOW = 2, DC_PIPE_VOCODER = 3, DC_PIPE_TOKEN2WAV = 4 };
 enum { DC_F32 = 0, DC_BF16 = 1 };   /* DC_BF16: bf16 storage and operands, fp32 accumulation */
 
 #define DC_MAX_CONV 32
@@ -67,6 +67,14 @@ enum { DC_F32 = 0, DC_BF16 = 1 };   /* DC_BF16: bf16 storage and operands, fp32 
  *                     n_steps, mel_dim                       (bf16)
  *   DC_PIPE_VOCODER : mel_dim, n_up, up_strides[], up_channels[n_up+1], n_res,
  *                     res_dilations[], n_fft, hop, logmag_clamp   (fp32)
+ *   DC_PIPE_TOKEN2WAV : the fields of DC_PIPE_FLOW and of DC_PIPE_VOCODER (same mel_dim), precision
+ *                     DC_BF16: the whole decoder step of the paper's segment (Section 2.2: flow
+ *                     decoder, then vocoder and inverse STFT) in one call - a chunk of
+ *                     [conditioning | noise] frames in, PCM out; the mel frames in between stay in a
+ *                     device buffer of the stream (bf16 flow decoder, fp32 vocoder tail).  Weights:
+ *                     the flow blob followed by the vocoder blob.  dc_decode_batch serves it too (the
+ *                     flow decoder batched over the streams, the vocoder tail stream by stream);
+ *                     dc_decode_batch_host does not.
  * The flow decoder runs n_conv / n_attn conv blocks, then one attention layer,
  * repeated n_attn times (n_attn = 0: conv blocks only). */
 typedef struct dc_config {

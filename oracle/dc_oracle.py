@@ -462,7 +462,42 @@ class VocoderStream:
 # drivers
 # --------------------------------------------------------------------------------------------
 
+class TokenToWavStream:
+    """The whole decoder step (Sec. 2.2 lists the stages of the segment): the flow decoder's chunk of
+    mel frames, rounded once to float32 as the flow decoder delivers it, is the vocoder tail's input."""
+
+    def __init__(self, cfg, blob, **kw):
+        fc, vc = cfg.flow_part(), cfg.vocoder_part()
+        nf = _blob_floats(fc)
+        self.flow = FlowStream(fc, blob[:nf], **kw)
+        self.voc = VocoderStream(vc, blob[nf:])
+
+    def decode_chunk(self, feats: np.ndarray) -> np.ndarray:
+        mel = self.flow.decode_chunk(feats)
+        return self.voc.decode_chunk(np.asarray(mel, dtype=np.float32))
+
+
+def _blob_floats(cfg) -> int:
+    """Number of floats of a flow configuration's blob (the same tensors that parse_blob takes;
+    the oracle imports nothing from the input generators, so the count is written out here)."""
+    C = cfg.hidden
+    if cfg.pipeline == "flow":
+        m = cfg.mel_dim
+        return (2 * m * C + C + len(cfg.dilations) * (3 * C * C + C + C * C)
+                + cfg.n_attn_layers * (4 * C * C + 4 * C) + C * m + m)
+    raise ValueError(cfg.pipeline)
+
+
+def token2wav_offline(cfg, blob, feats, boundaries) -> np.ndarray:
+    fc, vc = cfg.flow_part(), cfg.vocoder_part()
+    nf = _blob_floats(fc)
+    mel = flow_offline(fc, blob[:nf], feats, boundaries)
+    return vocoder_offline(vc, blob[nf:], np.asarray(mel, dtype=np.float32))
+
+
 def make_stream(cfg, blob, **kw):
+    if cfg.pipeline == "token2wav":
+        return TokenToWavStream(cfg, blob, **kw)
     if cfg.pipeline == "conv":
         return ConvStackStream(cfg, blob)
     if cfg.pipeline == "flow":
@@ -473,6 +508,8 @@ def make_stream(cfg, blob, **kw):
 
 
 def run_offline(cfg, blob, feats, boundaries) -> np.ndarray:
+    if cfg.pipeline == "token2wav":
+        return token2wav_offline(cfg, blob, feats, boundaries)
     if cfg.pipeline == "conv":
         return conv_stack_offline(cfg, blob, feats)
     if cfg.pipeline == "flow":

@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_PKG, "libdc.so")
 _lib = None
 
 DC_MAX_CONV, DC_MAX_UP, DC_MAX_RES = 32, 4, 4
-PIPE = {"conv": 1, "flow": 2, "vocoder": 3}
+PIPE = {"conv": 1, "flow": 2, "vocoder": 3, "token2wav": 4}
 PREC = {"f32": 0, "bf16": 1}
 STATUS = {0: "DC_OK", 1: "DC_ERR_ARG", 2: "DC_ERR_CONFIG", 3: "DC_ERR_FRAMES", 4: "DC_ERR_OOM",
           5: "DC_ERR_CUDA", 6: "DC_ERR_TIMEOUT", 7: "DC_ERR_STATE"}
@@ -95,7 +95,7 @@ def make_config(cfg, max_batch: int = 1) -> dc_config:
         c.dilations[i] = d
     c.n_attn, c.n_heads, c.head_dim, c.kv_cap = cfg.n_attn_layers, cfg.n_heads, cfg.head_dim, cfg.kv_cap
     c.n_steps, c.f_chunk, c.mel_dim = cfg.n_steps, cfg.f_chunk, cfg.mel_dim
-    if cfg.pipeline == "vocoder":
+    if cfg.pipeline in ("vocoder", "token2wav"):
         c.n_up = len(cfg.up_strides)
         for i, s in enumerate(cfg.up_strides):
             c.up_strides[i] = s
@@ -185,7 +185,7 @@ class Stream:
                                       _cuda_stream_handle(stream))
         _check(st, "dc_decode_chunk")
         res = out[: n_out.value]
-        if self.model.cfg.pipeline != "vocoder":
+        if self.model.cfg.pipeline not in ("vocoder", "token2wav"):
             res = res.view(T, -1)
         return res
 

@@ -73,6 +73,9 @@ struct dc_model {
   int       out_per_frame = 0;
   int       in_dim = 0;
   dc::FlowModel* flow = nullptr;
+  // DC_PIPE_TOKEN2WAV: the flow decoder and the vocoder tail as models of their own; this one only chains them
+  dc_model* sub_flow = nullptr;
+  dc_model* sub_voc = nullptr;
   std::atomic<uint64_t> counters[8];
   std::atomic<int> open_streams{0};
   std::mutex mu;
@@ -88,6 +91,9 @@ struct dc_stream {
   std::vector<DevBuf> f32_rings;   // input ring of each fp32 layer
   float*    tails = nullptr;       // [2][12] overlap-add tails (ping-pong)
   dc::FlowState* flow = nullptr;
+  dc_stream* sub_flow = nullptr;   // DC_PIPE_TOKEN2WAV: the two halves' streams and the mel chunk between them
+  dc_stream* sub_voc = nullptr;
+  float*    mel = nullptr;         // [f_chunk][mel_dim] fp32, device
   float*    stage_in = nullptr;    // device staging of dc_decode_chunk_host
   float*    stage_out = nullptr;
   cudaGraph_t     g_graph = nullptr;   // fp32 pipelines: the captured chunk step
@@ -100,12 +106,24 @@ struct dc_stream {
 // configuration
 // ---------------------------------------------------------------------------------------------
 
+static dc_config sub_config(const dc_config& c, int pipeline) {
+  dc_config s = c;
+  s.pipeline = pipeline;
+  s.precision = pipeline == DC_PIPE_FLOW ? DC_BF16 : DC_F32;
+  return s;
+}
+
 static bool config_ok(const dc_config* c, const char** why) {
 #define BAD(msg) do { *why = msg; return false; } while (0)
   if (!c) BAD("null config");
   if (c->size != sizeof(dc_config)) BAD("dc_config.size mismatch");
   if (c->f_chunk < 1 || c->f_chunk > 4096) BAD("f_chunk out of range");
   if (c->max_batch < 1 || c->max_batch > 1024) BAD("max_batch out of range");
+  if (c->pipeline == DC_PIPE_TOKEN2WAV) {
+    if (c->precision != DC_BF16) BAD("token2wav pipeline is bf16 (flow decoder) + fp32 (vocoder tail)");
+    const dc_config f = sub_config(*c, DC_PIPE_FLOW), v = sub_config(*c, DC_PIPE_VOCODER);
+    return config_ok(&f, why) && config_ok(&v, why);
+  }
   if (c->pipeline == DC_PIPE_CONV) {
     if (c->precision != DC_F32) BAD("conv pipeline is fp32");
     if (c->hidden < 4 || c->hidden % 4) BAD("hidden must be a multiple of 4");
@@ -156,6 +174,10 @@ extern "C" size_t dc_weights_count(const dc_config* c) {
   if (!config_ok(c, &why)) return 0;
   size_t n = 0;
   const size_t C = (size_t)c->hidden;
+  if (c->pipeline == DC_PIPE_TOKEN2WAV) {
+    const dc_config f = sub_config(*c, DC_PIPE_FLOW), v = sub_config(*c, DC_PIPE_VOCODER);
+    return dc_weights_count(&f) + dc_weights_count(&v);
+  }
   if (c->pipeline == DC_PIPE_CONV) {
     n = (size_t)c->n_conv * (3 * C * C + C);
   } else if (c->pipeline == DC_PIPE_FLOW) {
@@ -238,7 +260,16 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
   m->device = dev;
   for (auto& c : m->counters) c = 0;
   dc_status st = DC_OK;
-  if (cfg->pipeline == DC_PIPE_FLOW) {
+  if (cfg->pipeline == DC_PIPE_TOKEN2WAV) {
+    const dc_config f = sub_config(*cfg, DC_PIPE_FLOW), v = sub_config(*cfg, DC_PIPE_VOCODER);
+    const size_t nf = dc_weights_count(&f);
+    st = dc_create(w, nf, &f, &m->sub_flow);
+    if (st == DC_OK) st = dc_create(w + nf, n_floats - nf, &v, &m->sub_voc);
+    if (st == DC_OK) {
+      m->in_dim = m->sub_flow->in_dim;
+      m->out_per_frame = m->sub_voc->out_per_frame;
+    }
+  } else if (cfg->pipeline == DC_PIPE_FLOW) {
     st = dc::flow_model_create(*cfg, w, &m->flow);
     m->in_dim = 2 * cfg->mel_dim;
     m->out_per_frame = cfg->mel_dim;
@@ -266,6 +297,8 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     }
   }
   if (st != DC_OK) {
+    if (m->sub_flow) dc_destroy(m->sub_flow);
+    if (m->sub_voc) dc_destroy(m->sub_voc);
     if (m->d_w) cudaFree(m->d_w);
     if (m->d_call) cudaFree(m->d_call);
     if (m->flow) dc::flow_model_destroy(m->flow);
@@ -287,6 +320,8 @@ extern "C" dc_status dc_destroy(dc_model* m) {
     dc::set_error("dc_destroy: %d streams still open", m->open_streams.load());
     return DC_ERR_STATE;
   }
+  if (m->sub_flow) dc_destroy(m->sub_flow);   // their streams were closed with ours
+  if (m->sub_voc) dc_destroy(m->sub_voc);
   if (m->flow) dc::flow_model_destroy(m->flow);
   if (m->d_w) cudaFree(m->d_w);
   if (m->d_call) cudaFree(m->d_call);
@@ -310,6 +345,11 @@ static void free_stream_buffers(dc_stream* s) {
   s->f32_rings.clear();
   if (s->tails) cudaFree(s->tails);
   if (s->flow) dc::flow_state_close(s->flow);
+  if (s->sub_flow) dc_stream_close(s->sub_flow);
+  if (s->sub_voc) dc_stream_close(s->sub_voc);
+  if (s->mel) cudaFree(s->mel);
+  s->sub_flow = s->sub_voc = nullptr;
+  s->mel = nullptr;
   if (s->stage_in) cudaFree(s->stage_in);
   if (s->stage_out) cudaFree(s->stage_out);
   s->tails = nullptr;
@@ -325,7 +365,11 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
   s->model = m;
   cudaError_t e = cudaSuccess;
   dc_status st = DC_OK;
-  if (m->flow) {
+  if (m->sub_flow) {
+    st = dc_stream_open(m->sub_flow, &s->sub_flow);
+    if (st == DC_OK) st = dc_stream_open(m->sub_voc, &s->sub_voc);
+    if (st == DC_OK) e = cudaMalloc(&s->mel, (size_t)m->cfg.f_chunk * m->cfg.mel_dim * sizeof(float));
+  } else if (m->flow) {
     st = dc::flow_state_open(m->flow, &s->flow);
   } else {
     for (const F32Layer& L : m->layers) {
@@ -354,7 +398,7 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
     delete s;
     return st;
   }
-  if (!m->flow) build_f32_graph(s);
+  if (!m->flow && !m->sub_flow) build_f32_graph(s);
   {
     std::lock_guard<std::mutex> lk(m->mu);
     m->all_streams.push_back(s);
@@ -368,7 +412,11 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
 extern "C" dc_status dc_stream_reset(dc_stream* s, void* cuda_stream) {
   if (!s || s->closed) return DC_ERR_STATE;
   cudaStream_t cs = (cudaStream_t)cuda_stream;
-  if (s->flow) {
+  if (s->sub_flow) {
+    dc_status st = dc_stream_reset(s->sub_flow, cuda_stream);
+    if (st == DC_OK) st = dc_stream_reset(s->sub_voc, cuda_stream);
+    if (st != DC_OK) return st;
+  } else if (s->flow) {
     dc_status st = dc::flow_state_reset(s->model->flow, s->flow, cs);
     if (st != DC_OK) return st;
   } else {
@@ -396,7 +444,15 @@ extern "C" dc_status dc_stream_carry_info(const dc_stream* s, uint64_t* out, int
   if (!s || !out || !n_entries || max_entries < 0) return DC_ERR_ARG;
   if (s->closed) return DC_ERR_STATE;
   std::vector<DevBuf> bufs;
-  if (s->flow) {
+  if (s->sub_flow) {   // the carries of both halves, flow decoder first
+    uint64_t tmp[2 * 128];
+    for (const dc_stream* sub : {(const dc_stream*)s->sub_flow, (const dc_stream*)s->sub_voc}) {
+      int n = 0;
+      dc_status st = dc_stream_carry_info(sub, tmp, 128, &n);
+      if (st != DC_OK) return st;
+      for (int i = 0; i < n && i < 128; ++i) bufs.push_back(DevBuf{(void*)(uintptr_t)tmp[2 * i], (size_t)tmp[2 * i + 1]});
+    }
+  } else if (s->flow) {
     bufs.resize(64);
     int n = 0;
     dc::flow_state_buffers(s->flow, bufs.data(), 64, &n);
@@ -558,7 +614,10 @@ extern "C" dc_status dc_decode_chunk(dc_stream* s, const float* feats, int T, fl
   dc_model* m = s->model;
   cudaStream_t cs = (cudaStream_t)cuda_stream;
   int launches = 0;
-  if (m->flow) {
+  if (m->sub_flow) {   // mel frames never leave the device: the flow decoder's output is the vocoder tail's input
+    st = dc_decode_chunk(s->sub_flow, feats, T, s->mel, nullptr, cuda_stream);
+    if (st == DC_OK) st = dc_decode_chunk(s->sub_voc, s->mel, T, out, nullptr, cuda_stream);
+  } else if (m->flow) {
     st = dc::flow_decode(m->flow, 1, &s->flow, &feats, &T, &out, cs, &launches);
   } else {
     st = decode_f32(s, feats, T, out, cs, &launches);
@@ -579,8 +638,8 @@ extern "C" dc_status dc_decode_chunk(dc_stream* s, const float* feats, int T, fl
 extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* streams, const float* const* feats,
                                      const int* n_frames, float* const* out, void* cuda_stream) {
   if (!m || !streams || !feats || !n_frames || !out) return DC_ERR_ARG;
-  if (!m->flow) {
-    dc::set_error("dc_decode_batch serves the flow pipeline only");
+  if (!m->flow && !m->sub_flow) {
+    dc::set_error("dc_decode_batch serves the flow and token2wav pipelines only");
     return DC_ERR_CONFIG;
   }
   if (n < 1 || n > m->cfg.max_batch) {
@@ -605,7 +664,19 @@ extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* strea
     states[(size_t)i] = streams[i]->flow;
   }
   int launches = 0;
-  dc_status st = dc::flow_decode(m->flow, n, states.data(), feats, n_frames, out, (cudaStream_t)cuda_stream, &launches);
+  dc_status st = DC_OK;
+  if (m->sub_flow) {   // flow decoder batched over the streams, then every stream's vocoder tail
+    std::vector<dc_stream*> fs((size_t)n);
+    std::vector<float*> mels((size_t)n);
+    for (int i = 0; i < n; ++i) {
+      fs[(size_t)i] = streams[i]->sub_flow;
+      mels[(size_t)i] = streams[i]->mel;
+    }
+    st = dc_decode_batch(m->sub_flow, n, fs.data(), feats, n_frames, mels.data(), cuda_stream);
+    for (int i = 0; i < n && st == DC_OK; ++i) st = dc_decode_chunk(streams[i]->sub_voc, streams[i]->mel, n_frames[i], out[i], nullptr, cuda_stream);
+  } else {
+    st = dc::flow_decode(m->flow, n, states.data(), feats, n_frames, out, (cudaStream_t)cuda_stream, &launches);
+  }
   m->counters[5] += (uint64_t)launches;
   if (st != DC_OK) {
     for (int i = 0; i < n; ++i) streams[i]->poisoned = true;
@@ -632,8 +703,9 @@ extern "C" dc_status dc_decode_chunk_host(dc_stream* s, const float* feats_host,
   if (st != DC_OK) return st;
   DC_CUDA(cudaMemcpyAsync(out_host, s->stage_out, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaStreamSynchronize(cs));
-  if (m->flow) {
-    const int code = dc::flow_take_device_error(m->flow);
+  dc::FlowModel* fm = m->flow ? m->flow : (m->sub_flow ? m->sub_flow->flow : nullptr);
+  if (fm) {
+    const int code = dc::flow_take_device_error(fm);
     if (code != 0) {   // a bounded device-side wait gave up: the chunk's result is not valid
       m->counters[4]++;
       s->poisoned = true;
@@ -687,6 +759,10 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
 
 extern "C" dc_status dc_profile_begin(dc_model* m, int max_launches) {
   if (!m || max_launches < 1 || max_launches > (1 << 20)) return DC_ERR_ARG;
+  if (m->sub_flow) {
+    dc_status st = dc_profile_begin(m->sub_flow, max_launches);
+    return st == DC_OK ? dc_profile_begin(m->sub_voc, max_launches) : st;
+  }
   dc::Profiler& p = m->prof;
   if (p.on) return DC_ERR_STATE;
   p.ev = new (std::nothrow) cudaEvent_t[2 * (size_t)max_launches];
@@ -702,6 +778,14 @@ extern "C" dc_status dc_profile_begin(dc_model* m, int max_launches) {
 
 extern "C" dc_status dc_profile_end(dc_model* m, double ms[8], uint64_t launches[8]) {
   if (!m || !ms || !launches) return DC_ERR_ARG;
+  if (m->sub_flow) {   // the two halves use disjoint kernel classes
+    double ms2[8];
+    uint64_t l2[8];
+    dc_status st = dc_profile_end(m->sub_flow, ms, launches);
+    if (st == DC_OK) st = dc_profile_end(m->sub_voc, ms2, l2);
+    for (int i = 0; i < 8 && st == DC_OK; ++i) { ms[i] += ms2[i]; launches[i] += l2[i]; }
+    return st;
+  }
   dc::Profiler& p = m->prof;
   if (!p.on) return DC_ERR_STATE;
   p.on = false;
@@ -728,6 +812,13 @@ extern "C" dc_status dc_get_counters(const dc_model* m, uint64_t counters[8]) {
     if (code > 0) const_cast<dc_model*>(m)->counters[4]++;
   }
   for (int i = 0; i < 8; ++i) counters[i] = m->counters[i].load();
+  if (m->sub_flow) {   // kernel launches and device time-outs are counted where they happen
+    uint64_t a[8], b[8];
+    dc_get_counters(m->sub_flow, a);
+    dc_get_counters(m->sub_voc, b);
+    counters[4] += a[4] + b[4];
+    counters[5] += a[5] + b[5];
+  }
   return DC_OK;
 }
 

@@ -388,3 +388,29 @@ def test_paper_memory_ratio_pins():
     assert round(16 * 1000 / (10 * 458), 1) == float(g["rho_standalone"])
     assert round(241.7 / 84.9, 2) == float(g["speedup"])
     assert abs(100 * (1 - 2972 / 4852) - float(g["peak_drop_pct"])) < 0.06   # printed from unrounded data
+
+
+def test_token2wav_chain_streamed_equals_offline_and_is_the_composition():
+    """The whole decoder step (flow decoder feeding the vocoder tail): the chunk loop equals the
+    offline run over the concatenated input (Eq. 4 for the chain), the chain is the composition of
+    the two pinned stages, and the oracle's own count of the flow blob agrees with the layout of
+    the input generators."""
+    cfg = wl.tiny_token2wav(n_chunks=7)
+    bounds = [0, 3, 13, 14, 24, 31, 41, 51]
+    w = wl.make_workload(cfg, boundaries=[bounds])
+    s = w.streams[0]
+    streamed = orc.run_stream(cfg, w.weights, s.feats, s.boundaries)
+    offline = orc.run_offline(cfg, w.weights, s.feats, s.boundaries)
+    assert streamed.shape == (bounds[-1] * cfg.out_per_frame,)
+    assert np.allclose(streamed, offline, rtol=0, atol=1e-9 * np.abs(offline).max())
+    fc, vc = cfg.flow_part(), cfg.vocoder_part()
+    nf = wl.blob_size(fc)
+    assert orc._blob_floats(fc) == nf and nf + wl.blob_size(vc) == w.weights.size
+    mel = orc.flow_offline(fc, w.weights[:nf], s.feats, s.boundaries)
+    assert np.array_equal(offline, orc.vocoder_offline(vc, w.weights[nf:], mel))
+    # one more sample of input changes only later audio (the chain stays causal)
+    f2 = s.feats.copy()
+    f2[40:] += 1.0
+    again = orc.run_offline(cfg, w.weights, f2, s.boundaries)
+    cut = 31 * cfg.out_per_frame          # frames 0..30 belong to chunks that end before frame 40 is seen
+    assert np.array_equal(again[:cut], offline[:cut]) and not np.array_equal(again[cut:], offline[cut:])
