@@ -113,7 +113,8 @@ def describe(cfg) -> str:
     if cfg.pipeline == "flow":
         return (f"{cfg.name}: {cfg.n_streams} stream(s) x flow decoder C={cfg.hidden}, {len(cfg.dilations)} conv blocks, "
                 f"{cfg.n_attn_layers} attention layers ({cfg.n_heads}x{cfg.head_dim}, KV cap {cfg.kv_cap}), "
-                f"{cfg.n_steps} Euler steps, {cfg.f_chunk}-frame chunks, bf16 / fp32 accumulate")
+                f"{cfg.n_steps} Euler steps, {cfg.f_chunk}-frame chunks, bf16 / fp32 accumulate"
+                + (f", classifier-free guidance w={cfg.cfg_scale} (two passes per step)" if cfg.cfg_scale > 0 else ""))
     if cfg.pipeline == "vocoder":
         return (f"{cfg.name}: vocoder tail mel {cfg.mel_dim} -> strides {cfg.up_strides} channels {cfg.up_channels} "
                 f"-> head -> iSTFT n_fft {cfg.n_fft} hop {cfg.hop}, {cfg.f_chunk}-frame chunks, fp32")
@@ -129,7 +130,7 @@ def units_per_chunk(cfg):
 
 def flops_per_launch(cfg, cls: str, n_streams: int) -> float:
     """Algorithmic FLOPs of one launch of a kernel class (valid rows only)."""
-    rows = n_streams * cfg.f_chunk
+    rows = n_streams * cfg.f_chunk * (2 if getattr(cfg, "cfg_scale", 0.0) > 0 else 1)   # guidance: two passes per stream
     C = cfg.hidden
     if cls == "gemm_conv":
         return 2.0 * rows * C * 3 * C
@@ -142,7 +143,8 @@ def flops_per_launch(cfg, cls: str, n_streams: int) -> float:
 def attention_bytes_per_launch(cfg, n_streams: int) -> float:
     """K and V rows of the attended window (bf16) + Q read + O write."""
     L = cfg.kv_cap + cfg.f_chunk
-    return n_streams * (2.0 * L * cfg.hidden * 2 + 2.0 * cfg.f_chunk * cfg.hidden * 2)
+    passes = 2 if getattr(cfg, "cfg_scale", 0.0) > 0 else 1
+    return passes * n_streams * (2.0 * L * cfg.hidden * 2 + 2.0 * cfg.f_chunk * cfg.hidden * 2)
 
 
 def max_over_ranks(value: float, world: int, device: str = "cuda") -> float:

@@ -60,6 +60,7 @@ class DCConfig:
     hop: int = 4
     rms_eps: float = 1e-6
     logmag_clamp: float = math.log(100.0)
+    cfg_scale: float = 0.0              # flow decoder: classifier-free guidance weight w (0 = off, one pass per step)
     # workload (not part of the network)
     n_chunks: int = 1
     n_streams: int = 1
@@ -259,7 +260,11 @@ def tiny_token2wav(**kw) -> DCConfig:
 
 
 # beyond the five: the whole decoder step in one call
-EXTRA_CONFIGS: Dict[str, DCConfig] = {"token2wav": token2wav()}
+EXTRA_CONFIGS: Dict[str, DCConfig] = {
+    "token2wav": token2wav(),
+    # cfg3 with classifier-free guidance (two passes per Euler step, the form the paper measures its flow step in)
+    "cfg3_guided": CONFIGS["cfg3"].replace(name="cfg3_guided", cfg_scale=0.7, seed=7),
+}
 
 
 def tiny_vocoder(**kw) -> DCConfig:

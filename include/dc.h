@@ -98,6 +98,12 @@ typedef struct dc_config {
   float    rms_eps;
   float    logmag_clamp;
   int32_t  max_batch;            /* most streams one dc_decode_batch call may carry (>= 1)   */
+  float    cfg_scale;            /* flow decoder: classifier-free guidance weight w >= 0; 0 = off.  With w > 0 every
+                                  * Euler step evaluates the network twice - with the conditioning and with the
+                                  * conditioning set to zero, each pass with carries of its own - and advances
+                                  * x by ((1 + w) v_cond - w v_uncond) / n_steps (paper Table 1 measures the flow
+                                  * step in this guided, batch x 2 form).  The two passes of a stream are two
+                                  * row blocks of the same GEMM tiles.                            */
 } dc_config;
 
 /* Number of floats of the canonical weight blob for this configuration, 0 if the

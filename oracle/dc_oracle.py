@@ -243,8 +243,9 @@ def flow_offline(cfg, blob, feats: np.ndarray, boundaries: Sequence[int]) -> np.
     assert boundaries[0] == 0 and boundaries[-1] == F
     tau = tau_table(cfg, W)
     plan = _layer_plan(cfg)
-    for s in range(n):
-        h = rb(rb(np.concatenate([x, mu], axis=1)) @ W["in.W"] + W["in.b"])
+
+    def velocity(s, x, cond):
+        h = rb(rb(np.concatenate([x, cond], axis=1)) @ W["in.W"] + W["in.b"])
         for kind, idx, d in plan:
             if kind == "conv":
                 z = causal_conv_k3(h, W[f"conv{idx}.W"], d) + W[f"conv{idx}.b"] + tau[s, idx]
@@ -260,7 +261,15 @@ def flow_offline(cfg, blob, feats: np.ndarray, boundaries: Sequence[int]) -> np.
                     k0 = max(0, lo - cfg.kv_cap)
                     o[lo:hi] = _attend(cfg, q[lo:hi], k[k0:hi], v[k0:hi], rb)
                 h = rb(h + o @ W[f"attn{idx}.Wo"] + W[f"attn{idx}.bo"])
-        vel = rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]
+        return rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]
+
+    w_cfg = getattr(cfg, "cfg_scale", 0.0)
+    for s in range(n):
+        vel = velocity(s, x, mu)
+        if w_cfg > 0:
+            # classifier-free guidance (the flow step of Table 1 is the guided one, batch x 2): a second pass
+            # with the conditioning removed, v = (1 + w) v_cond - w v_uncond
+            vel = (1.0 + w_cfg) * vel - w_cfg * velocity(s, x, np.zeros_like(mu))
         x = x + vel / n
     return x.astype(np.float32)
 
@@ -301,13 +310,17 @@ class FlowStream:
         self.plan = _layer_plan(cfg)
         self.ring = carry == "ring"
         C, n = cfg.hidden, cfg.n_steps
-        self.halo = [[np.zeros((2 * d, C)) for d in cfg.dilations] for _ in range(n)]
-        if self.ring:
-            self.kv = [[KVRing(cfg.kv_cap, cfg.f_chunk, C) for _ in range(cfg.n_attn_layers)]
-                       for _ in range(n)]
-        else:
-            self.kv = [[(np.zeros((0, C)), np.zeros((0, C))) for _ in range(cfg.n_attn_layers)]
-                       for _ in range(n)]
+        self.w_cfg = getattr(cfg, "cfg_scale", 0.0)
+        # with classifier-free guidance the conditional and the unconditional pass each carry a state of their own
+        self.passes = []
+        for _ in range(2 if self.w_cfg > 0 else 1):
+            halo = [[np.zeros((2 * d, C)) for d in cfg.dilations] for _ in range(n)]
+            if self.ring:
+                kv = [[KVRing(cfg.kv_cap, cfg.f_chunk, C) for _ in range(cfg.n_attn_layers)] for _ in range(n)]
+            else:
+                kv = [[(np.zeros((0, C)), np.zeros((0, C))) for _ in range(cfg.n_attn_layers)] for _ in range(n)]
+            self.passes.append((halo, kv))
+        self.halo, self.kv = self.passes[0]
         self.kv_len_seen: List[int] = []
 
     def decode_chunk(self, feats: np.ndarray) -> np.ndarray:
@@ -319,35 +332,43 @@ class FlowStream:
         m, n = cfg.mel_dim, cfg.n_steps
         mu, x = feats[:, :m], feats[:, m:].copy()
         for s in range(n):
-            h = rb(rb(np.concatenate([x, mu], axis=1)) @ W["in.W"] + W["in.b"])
-            for kind, idx, d in self.plan:
-                if kind == "conv":
-                    left = self.halo[s][idx]
-                    self.halo[s][idx] = np.concatenate([left, h], axis=0)[-2 * d:]
-                    z = (causal_conv_k3(h, W[f"conv{idx}.W"], d, left)
-                         + W[f"conv{idx}.b"] + self.tau[s, idx])
-                    h = rb(h + silu(z))
-                else:
-                    u = rb(rmsnorm(h, cfg.rms_eps))
-                    q = rb(u @ W[f"attn{idx}.Wq"] + W[f"attn{idx}.bq"])
-                    k = rb(u @ W[f"attn{idx}.Wk"] + W[f"attn{idx}.bk"])
-                    v = rb(u @ W[f"attn{idx}.Wv"] + W[f"attn{idx}.bv"])
-                    if self.ring:
-                        if s == 0 and idx == 0:
-                            self.kv_len_seen.append(self.kv[s][idx].filled)
-                        k_all, v_all = self.kv[s][idx].append_and_view(k, v)
-                    else:
-                        kc, vc = self.kv[s][idx]
-                        if s == 0 and idx == 0:
-                            self.kv_len_seen.append(kc.shape[0])
-                        k_all = np.concatenate([kc, k], axis=0)
-                        v_all = np.concatenate([vc, v], axis=0)
-                        self.kv[s][idx] = (k_all[-cfg.kv_cap:], v_all[-cfg.kv_cap:])
-                    o = _attend(cfg, q, k_all, v_all, rb)
-                    h = rb(h + o @ W[f"attn{idx}.Wo"] + W[f"attn{idx}.bo"])
-            vel = rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]
+            vel = self._velocity(s, x, mu, 0, rb)
+            if self.w_cfg > 0:
+                vel = (1.0 + self.w_cfg) * vel - self.w_cfg * self._velocity(s, x, np.zeros_like(mu), 1, rb)
             x = x + vel / n
         return x.astype(np.float32)
+
+    def _velocity(self, s, x, cond, p, rb):
+        """One evaluation of the network at Euler step s with pass p's carries (updated in passing)."""
+        cfg, W = self.cfg, self.W
+        halo, kv = self.passes[p]
+        h = rb(rb(np.concatenate([x, cond], axis=1)) @ W["in.W"] + W["in.b"])
+        for kind, idx, d in self.plan:
+            if kind == "conv":
+                left = halo[s][idx]
+                halo[s][idx] = np.concatenate([left, h], axis=0)[-2 * d:]
+                z = (causal_conv_k3(h, W[f"conv{idx}.W"], d, left)
+                     + W[f"conv{idx}.b"] + self.tau[s, idx])
+                h = rb(h + silu(z))
+            else:
+                u = rb(rmsnorm(h, cfg.rms_eps))
+                q = rb(u @ W[f"attn{idx}.Wq"] + W[f"attn{idx}.bq"])
+                k = rb(u @ W[f"attn{idx}.Wk"] + W[f"attn{idx}.bk"])
+                v = rb(u @ W[f"attn{idx}.Wv"] + W[f"attn{idx}.bv"])
+                if self.ring:
+                    if s == 0 and idx == 0 and p == 0:
+                        self.kv_len_seen.append(kv[s][idx].filled)
+                    k_all, v_all = kv[s][idx].append_and_view(k, v)
+                else:
+                    kc, vc = kv[s][idx]
+                    if s == 0 and idx == 0 and p == 0:
+                        self.kv_len_seen.append(kc.shape[0])
+                    k_all = np.concatenate([kc, k], axis=0)
+                    v_all = np.concatenate([vc, v], axis=0)
+                    kv[s][idx] = (k_all[-cfg.kv_cap:], v_all[-cfg.kv_cap:])
+                o = _attend(cfg, q, k_all, v_all, rb)
+                h = rb(h + o @ W[f"attn{idx}.Wo"] + W[f"attn{idx}.bo"])
+        return rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]
 
 
 # --------------------------------------------------------------------------------------------

@@ -32,7 +32,8 @@ class dc_config(C.Structure):
                 ("mel_dim", C.c_int32), ("n_up", C.c_int32), ("up_strides", C.c_int32 * DC_MAX_UP),
                 ("up_channels", C.c_int32 * (DC_MAX_UP + 1)), ("n_res", C.c_int32),
                 ("res_dilations", C.c_int32 * DC_MAX_RES), ("n_fft", C.c_int32), ("hop", C.c_int32),
-                ("rms_eps", C.c_float), ("logmag_clamp", C.c_float), ("max_batch", C.c_int32)]
+                ("rms_eps", C.c_float), ("logmag_clamp", C.c_float), ("max_batch", C.c_int32),
+                ("cfg_scale", C.c_float)]
 
 
 class DCError(RuntimeError):
@@ -107,6 +108,7 @@ def make_config(cfg, max_batch: int = 1) -> dc_config:
         c.n_fft, c.hop = cfg.n_fft, cfg.hop
     c.rms_eps, c.logmag_clamp = cfg.rms_eps, cfg.logmag_clamp
     c.max_batch = max_batch
+    c.cfg_scale = float(getattr(cfg, "cfg_scale", 0.0))
     return c
 
 

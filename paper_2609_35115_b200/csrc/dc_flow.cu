@@ -54,7 +54,7 @@ struct SlotInfo {
   int          T;         // frames presented by this stream in this call
   int          kv_head;   // ring row that receives the chunk's first K/V row
   int          kv_len;    // carried K/V rows attended (<= kv_cap), before this chunk
-  int          pad;
+  int          pass;      // 0: conditional pass (or the only one); 1: the unconditional pass of a guided stream (mu = 0, no output)
   const float* feats;     // [T][2 mel]
   float*       out;       // [T][mel]
   bf16*        halo;      // stream carry: [n_steps][n_conv][8][C]
@@ -92,6 +92,7 @@ struct GemmParams {
   float        inv_n;
   int          last_step;
   int          mel;
+  float        cfg_w;           // MODE_OUT: guidance weight; > 0: the tile's slots are the (conditional, unconditional) passes of one stream
   // RMS normalisation, folded into the GEMMs around it (Sec. 3.2 block form; the norm has no gain):
   // (x / rms(x)) W = (x W) / rms(x), so the GEMM that consumes a normalised operand reads x itself
   // and scales its accumulator rows, and the GEMM that produced x leaves the row sums of squares.
@@ -403,7 +404,28 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
       for (int i = 0; i < 16; ++i) acc[i] = fmaf(acc[i], rs, s_bias[c0 + i]);
       if (p.mode == MODE_OUT) {
-        if (is_chunk) {
+        if (p.cfg_w > 0.f) {
+          // guided step: rows 64.. of the tile are the unconditional pass of the stream in rows 0..63; they hand
+          // their velocity over through shared memory and the conditional rows form (1 + w) v_c - w v_u
+          // (16-column tiles: this chunk group's four warps are the only ones here)
+          float4* xv4 = reinterpret_cast<float4*>(smem);
+          if (q >= 2) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) xv4[j * 64 + (q - 2) * 32 + lane] = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+          }
+          ptx::named_bar_sync(2 + cg, 128);
+          if (q < 2) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float4 u = xv4[j * 64 + q * 32 + lane];
+              acc[4 * j] = fmaf(1.f + p.cfg_w, acc[4 * j], -p.cfg_w * u.x);
+              acc[4 * j + 1] = fmaf(1.f + p.cfg_w, acc[4 * j + 1], -p.cfg_w * u.y);
+              acc[4 * j + 2] = fmaf(1.f + p.cfg_w, acc[4 * j + 2], -p.cfg_w * u.z);
+              acc[4 * j + 3] = fmaf(1.f + p.cfg_w, acc[4 * j + 3], -p.cfg_w * u.w);
+            }
+          }
+        }
+        if (is_chunk && si.pass == 0) {
           float* xs = p.xstate + (long long)r * p.mel + n;
           float xv[16];
 #pragma unroll
@@ -419,6 +441,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           uint4 a, b;
           pack16_bf16(xv, a, b);
           store16(p.ain + grow * p.ld_ain + n, a, b);
+          if (p.cfg_w > 0.f) store16(p.ain + (grow + SLOT_ROWS) * p.ld_ain + n, a, b);   // the unconditional pass starts from the same x
           if (p.last_step) {
             float* o = si.out + (long long)f * p.mel + n;
 #pragma unroll
@@ -534,7 +557,7 @@ __global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, 
   for (int i = threadIdx.x; i < si.T * mel; i += blockDim.x) {
     const int f = i / mel, c = i - f * mel;
     const long long r = (long long)blockIdx.x * SLOT_ROWS + HALO + f;
-    const float mu = si.feats[(long long)f * 2 * mel + c];
+    const float mu = si.pass == 0 ? si.feats[(long long)f * 2 * mel + c] : 0.f;
     const float x0 = si.feats[(long long)f * 2 * mel + mel + c];
     xstate[r * mel + c] = x0;
     ain[(GUARD + r) * ld_ain + c] = __float2bfloat16_rn(x0);
@@ -955,7 +978,9 @@ struct GraphEntry {
 
 struct FlowModel {
   dc_config cfg;
-  int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0;
+  int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0;   // S: slots (streams x passes) of a full batch
+  int n_pass = 1;            // 2 with classifier-free guidance: a stream's conditional and unconditional pass are
+                             // adjacent slots, i.e. the two halves of one row tile
   bf16 *Xa = nullptr, *Xb = nullptr, *Q = nullptr, *O = nullptr, *Ain = nullptr;
   float* xstate = nullptr;
   float* ssq = nullptr;      // [C / 16][rows]: per-chunk sums of squares of the rows that feed an RMS norm
@@ -1031,7 +1056,8 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   m->cfg = cfg;
   const int C = m->C = cfg.hidden, mel = m->mel = cfg.mel_dim;
   m->Kin = ((2 * mel + KBLK - 1) / KBLK) * KBLK;
-  m->S = cfg.max_batch;
+  m->n_pass = cfg.cfg_scale > 0.f ? 2 : 1;
+  m->S = cfg.max_batch * m->n_pass;
   m->rows = ((m->S * SLOT_ROWS + TILE_M - 1) / TILE_M) * TILE_M;
   m->Rk = cfg.kv_cap + cfg.f_chunk;
   m->cpa = cfg.n_attn > 0 ? cfg.n_conv / cfg.n_attn : cfg.n_conv;
@@ -1191,11 +1217,11 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     if (!(g && atoi(g)) && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) == cudaSuccess) {
       // the two batch sizes that matter are captured now, so that no decode call ever builds a graph:
       // a single stream, and the full batch
-      const bool g1 = build_graph(m, 1);
-      const bool gs = m->S > 1 ? build_graph(m, m->S) : g1;
+      const bool g1 = build_graph(m, m->n_pass);   // a single stream
+      const bool gs = m->S > m->n_pass ? build_graph(m, m->S) : g1;
       if (getenv("DC_VERBOSE"))
         fprintf(stderr, "[dc] graphs: n=1 %s, n=%d %s, pdl %d/%d\n", g1 ? "ok" : "none", m->S, gs ? "ok" : "none",
-                g1 ? (int)m->graphs[1].pdl : -1, gs ? (int)m->graphs[m->S].pdl : -1);
+                g1 ? (int)m->graphs[m->n_pass].pdl : -1, gs ? (int)m->graphs[m->S].pdl : -1);
     }
     cudaGetLastError();
   }
@@ -1208,8 +1234,9 @@ dc_status flow_state_open(FlowModel* m, FlowState** out) {
   if (!s) return DC_ERR_OOM;
   s->m = m;
   const dc_config& c = m->cfg;
-  s->halo_bytes = (size_t)c.n_steps * c.n_conv * HALO * m->C * sizeof(bf16);
-  s->kv_bytes = (size_t)c.n_steps * c.n_attn * 2 * m->Rk * m->C * sizeof(bf16);
+  // one set of carries per pass
+  s->halo_bytes = (size_t)m->n_pass * c.n_steps * c.n_conv * HALO * m->C * sizeof(bf16);
+  s->kv_bytes = (size_t)m->n_pass * c.n_steps * c.n_attn * 2 * m->Rk * m->C * sizeof(bf16);
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s->halo), s->halo_bytes);
   if (e == cudaSuccess) e = cudaMemset(s->halo, 0, s->halo_bytes);
   if (e == cudaSuccess && s->kv_bytes) {
@@ -1429,7 +1456,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       p.mode = MODE_OUT; p.BN = bo; p.n_kblocks = C / KBLK; p.taps = 1;
       p.bias = fc + m->o_bout; p.halo_off = -1;
       p.xstate = m->xstate; p.ain = m->Ain; p.ld_ain = m->Kin; p.inv_n = 1.0f / c.n_steps;
-      p.last_step = (s == c.n_steps - 1); p.mel = mel;
+      p.last_step = (s == c.n_steps - 1); p.mel = mel; p.cfg_w = c.cfg_scale;
       normalised(p);
       gemm(*tX, m->tmWout[v], p, mel);
     }
@@ -1489,7 +1516,11 @@ bool build_graph(FlowModel* m, int n) {
 dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats, const int* T,
                       float* const* outp, cudaStream_t st, int* launches) {
   const dc_config& c = m->cfg;
-  // ---- per-call slot table (passed by value through a kernel, so nothing is staged or allocated)
+  // ---- per-call slot table (passed by value through a kernel, so nothing is staged or allocated);
+  // with guidance a stream takes two adjacent slots, one per pass
+  const int n_streams = n;
+  const int np = m->n_pass;
+  n = n_streams * np;                         // slots from here on
   const int n_sets = (n + MAX_SLOTS_PER_SET - 1) / MAX_SLOTS_PER_SET;
   std::vector<SlotSet>& sets = m->sets;   // sized at create
   for (int k = 0; k < n_sets; ++k) {
@@ -1497,16 +1528,17 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
     set.first = k * MAX_SLOTS_PER_SET;
     set.count = n - set.first < MAX_SLOTS_PER_SET ? n - set.first : MAX_SLOTS_PER_SET;
     for (int i = 0; i < set.count; ++i) {
-      FlowState* s = states[set.first + i];
+      const int stream = (set.first + i) / np, pass = (set.first + i) % np;
+      FlowState* s = states[stream];
       SlotInfo& si = set.s[i];
-      si.T = T[set.first + i];
+      si.T = T[stream];
       si.kv_head = (int)(s->frames % m->Rk);
       si.kv_len = (int)(s->frames < c.kv_cap ? s->frames : c.kv_cap);
-      si.pad = 0;
-      si.feats = feats[set.first + i];
-      si.out = outp[set.first + i];
-      si.halo = s->halo;
-      si.kv = s->kv;
+      si.pass = pass;
+      si.feats = feats[stream];
+      si.out = pass == 0 ? outp[stream] : nullptr;
+      si.halo = s->halo + (size_t)pass * (s->halo_bytes / sizeof(bf16) / np);
+      si.kv = s->kv ? s->kv + (size_t)pass * (s->kv_bytes / sizeof(bf16) / np) : nullptr;
     }
   }
   const bool profiling = m->prof != nullptr && m->prof->on;
@@ -1538,7 +1570,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       return DC_ERR_CUDA;
     }
   }
-  for (int i = 0; i < n; ++i) states[i]->frames += T[i];
+  for (int i = 0; i < n_streams; ++i) states[i]->frames += T[i];
   return DC_OK;
 }
 

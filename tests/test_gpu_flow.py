@@ -150,3 +150,42 @@ def test_cfg5_multi_stream_serving_full_size(dc):
         single = gu.run_gpu_stream(m, si.feats[:b[-1]], b)
         assert np.array_equal(single, got[i][:b[-1]])
     m.destroy()
+
+
+# ---- classifier-free guidance: two passes per Euler step, (1 + w) v_cond - w v_uncond ------------------
+
+def test_guided_tiny_ragged(dc):
+    _parity(dc, wl.tiny_flow(cfg_scale=0.7, n_chunks=len(RAGGED) - 1), boundaries=RAGGED)
+
+
+def test_guided_head_dim_64_and_large_weight(dc):
+    _parity(dc, wl.tiny_flow(cfg_scale=2.0, hidden=128, n_heads=2, head_dim=64, n_chunks=5))
+
+
+def test_guided_cfg3_geometry(dc):
+    """cfg3's network with guidance: the two passes fill the 128-row tiles that a single stream half uses."""
+    _parity(dc, wl.CONFIGS["cfg3"].replace(name="cfg3_guided", cfg_scale=0.7, n_chunks=14))
+
+
+def test_guided_batched_equals_single_stream(dc):
+    gu = _gu()
+    cfg = wl.tiny_flow(cfg_scale=0.7, n_chunks=5, n_streams=3)
+    w = wl.make_workload(cfg)
+    m = dc.Model(cfg, w.weights, max_batch=3)
+    single = [gu.run_gpu_stream(m, s.feats, s.boundaries) for s in w.streams]
+    streams = [m.open_stream() for _ in w.streams]
+    feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+    outs = [torch.zeros(s.boundaries[-1], cfg.mel_dim, device="cuda") for s in w.streams]
+    n_rounds = max(len(s.boundaries) - 1 for s in w.streams)
+    for r in range(n_rounds):
+        idx = [i for i, s in enumerate(w.streams) if r < len(s.boundaries) - 1]
+        fs = [feats[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]].contiguous() for i in idx]
+        os_ = [outs[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in idx]
+        dc.decode_batch(m, [streams[i] for i in idx], fs, os_)
+    torch.cuda.synchronize()
+    assert m.counters()[4] == 0
+    for st in streams:
+        st.close()
+    m.destroy()
+    for i in range(len(w.streams)):
+        assert np.array_equal(outs[i].cpu().numpy(), single[i]), f"stream {i}"

@@ -414,3 +414,43 @@ def test_token2wav_chain_streamed_equals_offline_and_is_the_composition():
     again = orc.run_offline(cfg, w.weights, f2, s.boundaries)
     cut = 31 * cfg.out_per_frame          # frames 0..30 belong to chunks that end before frame 40 is seen
     assert np.array_equal(again[:cut], offline[:cut]) and not np.array_equal(again[cut:], offline[cut:])
+
+
+def test_classifier_free_guidance_pins():
+    """Guided flow decoder (two passes per Euler step, v = (1+w) v_cond - w v_uncond):
+    (i) one Euler step is the stated combination of two runs of the (pinned) unguided decoder;
+    (ii) with the conditioning already zero both passes coincide and w drops out;
+    (iii) the chunk loop with per-pass carries equals the offline run (Eq. 4), ring == concat."""
+    w_g = 0.7
+    base = wl.tiny_flow(precision="f32", n_steps=1, n_chunks=4)
+    wk = wl.make_workload(base)
+    s = wk.streams[0]
+    m = base.mel_dim
+    x0 = s.feats[:, m:].astype(np.float64)
+    no_mu = s.feats.copy()
+    no_mu[:, :m] = 0.0
+    x1_c = orc.flow_offline(base, wk.weights, s.feats, s.boundaries).astype(np.float64)
+    x1_u = orc.flow_offline(base, wk.weights, no_mu, s.boundaries).astype(np.float64)
+    want = x0 + (1 + w_g) * (x1_c - x0) - w_g * (x1_u - x0)
+    got = orc.flow_offline(base.replace(cfg_scale=w_g), wk.weights, s.feats, s.boundaries)
+    assert np.allclose(got, want, rtol=0, atol=2e-6 * np.abs(want).max())
+    assert not np.allclose(got, x1_c, atol=1e-3)                    # guidance does something
+    # (ii) several steps, ragged chunks, bf16 mirroring on
+    cfg = wl.tiny_flow(n_chunks=7)
+    bounds = [0, 3, 13, 14, 24, 31, 41, 51]
+    wk = wl.make_workload(cfg, boundaries=[bounds])
+    s = wk.streams[0]
+    no_mu = s.feats.copy()
+    no_mu[:, :cfg.mel_dim] = 0.0
+    plain = orc.run_stream(cfg, wk.weights, no_mu, bounds)
+    for w_try in (0.3, 2.0):
+        guided = orc.run_stream(cfg.replace(cfg_scale=w_try), wk.weights, no_mu, bounds)
+        assert np.allclose(guided, plain, rtol=0, atol=1e-5 * np.abs(plain).max())
+    # (iii)
+    g = cfg.replace(cfg_scale=w_g)
+    off = orc.run_offline(g, wk.weights, s.feats, bounds)
+    st_concat = orc.run_stream(g, wk.weights, s.feats, bounds)
+    st_ring = orc.run_stream(g, wk.weights, s.feats, bounds, carry="ring")
+    assert np.allclose(st_concat, off, rtol=0, atol=1e-9 * np.abs(off).max())
+    assert np.array_equal(st_concat, st_ring)
+    assert not np.allclose(off, orc.run_offline(cfg, wk.weights, s.feats, bounds), atol=1e-3)
