@@ -114,7 +114,8 @@ def describe(cfg) -> str:
         return (f"{cfg.name}: {cfg.n_streams} stream(s) x flow decoder C={cfg.hidden}, {len(cfg.dilations)} conv blocks, "
                 f"{cfg.n_attn_layers} attention layers ({cfg.n_heads}x{cfg.head_dim}, KV cap {cfg.kv_cap}), "
                 f"{cfg.n_steps} Euler steps, {cfg.f_chunk}-frame chunks, bf16 / fp32 accumulate"
-                + (f", classifier-free guidance w={cfg.cfg_scale} (two passes per step)" if cfg.cfg_scale > 0 else ""))
+                + (f", classifier-free guidance w={cfg.cfg_scale} (two passes per step)" if cfg.cfg_scale > 0 else "")
+                + (f", {cfg.f_prompt}-frame prompt kept in the carry" if cfg.f_prompt > 0 else ""))
     if cfg.pipeline == "vocoder":
         return (f"{cfg.name}: vocoder tail mel {cfg.mel_dim} -> strides {cfg.up_strides} channels {cfg.up_channels} "
                 f"-> head -> iSTFT n_fft {cfg.n_fft} hop {cfg.hop}, {cfg.f_chunk}-frame chunks, fp32")
@@ -135,14 +136,14 @@ def flops_per_launch(cfg, cls: str, n_streams: int) -> float:
     if cls == "gemm_conv":
         return 2.0 * rows * C * 3 * C
     if cls == "attention":
-        L = cfg.kv_cap + cfg.f_chunk
+        L = getattr(cfg, "f_prompt", 0) + cfg.kv_cap + cfg.f_chunk
         return 2.0 * 2.0 * rows * L * C
     return 0.0
 
 
 def attention_bytes_per_launch(cfg, n_streams: int) -> float:
     """K and V rows of the attended window (bf16) + Q read + O write."""
-    L = cfg.kv_cap + cfg.f_chunk
+    L = getattr(cfg, "f_prompt", 0) + cfg.kv_cap + cfg.f_chunk
     passes = 2 if getattr(cfg, "cfg_scale", 0.0) > 0 else 1
     return passes * n_streams * (2.0 * L * cfg.hidden * 2 + 2.0 * cfg.f_chunk * cfg.hidden * 2)
 
@@ -316,7 +317,7 @@ def main():
 
     # ---- the same step with L2 flushed first (workloads whose working set fits L2 only): a stream paced
     # at its real-time cadence finds its weights and carries in HBM, not in L2 ----
-    ws_mb = (S * (cfg.n_steps * cfg.n_attn_layers * 2 * (cfg.kv_cap + T) * cfg.hidden * 2) / 1e6) if has_flow else 0.0
+    ws_mb = (S * (cfg.n_steps * cfg.n_attn_layers * 2 * (cfg.f_prompt + cfg.kv_cap + T) * cfg.hidden * 2) / 1e6) if has_flow else 0.0
     cold = None
     if ws_mb <= 126:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")

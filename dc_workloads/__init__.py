@@ -49,7 +49,8 @@ class DCConfig:
     n_attn_layers: int = 0
     n_heads: int = 0
     head_dim: int = 0
-    kv_cap: int = 0                     # W, frames of carried keys/values
+    kv_cap: int = 0                     # W, frames of carried keys/values (the retained history)
+    f_prompt: int = 0                   # the stream's first f_prompt frames are a prompt that is never evicted
     n_steps: int = 0                    # Euler steps per chunk
     f_chunk: int = 50                   # admission bound on frames per call
     mel_dim: int = 80
@@ -264,6 +265,8 @@ EXTRA_CONFIGS: Dict[str, DCConfig] = {
     "token2wav": token2wav(),
     # cfg3 with classifier-free guidance (two passes per Euler step, the form the paper measures its flow step in)
     "cfg3_guided": CONFIGS["cfg3"].replace(name="cfg3_guided", cfg_scale=0.7, seed=7),
+    # cfg3's network with the paper's carry: a 302-frame prompt that is never evicted + 100 retained frames
+    "cfg3_paper_carry": CONFIGS["cfg3"].replace(name="cfg3_paper_carry", f_prompt=302, kv_cap=100, seed=8),
 }
 
 

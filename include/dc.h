@@ -98,6 +98,10 @@ typedef struct dc_config {
   float    rms_eps;
   float    logmag_clamp;
   int32_t  max_batch;            /* most streams one dc_decode_batch call may carry (>= 1)   */
+  int32_t  f_prompt;             /* flow decoder: the stream's first f_prompt frames are a prompt whose keys/values
+                                  * are never evicted; behind them the carry keeps the last kv_cap frames (the
+                                  * paper's f_prompt + f_retained carry, Section 3.1 and Eq. 4).  0: a plain
+                                  * sliding window of kv_cap frames.                              */
   float    cfg_scale;            /* flow decoder: classifier-free guidance weight w >= 0; 0 = off.  With w > 0 every
                                   * Euler step evaluates the network twice - with the conditioning and with the
                                   * conditioning set to zero, each pass with carries of its own - and advances

@@ -227,6 +227,17 @@ def _layer_plan(cfg):
     return plan
 
 
+def attended_frames(cfg, lo: int, hi: int) -> np.ndarray:
+    """Frames whose keys/values the chunk [lo, hi) attends (Sec. 3.1 "Two extents", Eq. 4): the
+    prompt - the stream's first f_prompt frames, never evicted - then the last <= kv_cap frames of
+    history after the prompt, then the chunk itself.  f_prompt = 0: a plain sliding window."""
+    P = getattr(cfg, "f_prompt", 0)
+    prompt = np.arange(0, min(P, hi))                                   # including the prompt frames this chunk brings
+    history = np.arange(max(P, lo - cfg.kv_cap), lo) if lo > P else np.arange(0)   # last <= kv_cap frames after the prompt
+    own = np.arange(max(lo, P), hi)
+    return np.concatenate([prompt, history, own]).astype(np.int64)
+
+
 def flow_offline(cfg, blob, feats: np.ndarray, boundaries: Sequence[int]) -> np.ndarray:
     """Offline causal run over the concatenated input.  feats[:, :mel] is the
     conditioning mu, feats[:, mel:] the initial noise x_0.  For s in 0..n-1:
@@ -258,8 +269,8 @@ def flow_offline(cfg, blob, feats: np.ndarray, boundaries: Sequence[int]) -> np.
                 o = np.zeros_like(q)
                 for c in range(len(boundaries) - 1):
                     lo, hi = boundaries[c], boundaries[c + 1]
-                    k0 = max(0, lo - cfg.kv_cap)
-                    o[lo:hi] = _attend(cfg, q[lo:hi], k[k0:hi], v[k0:hi], rb)
+                    keys = attended_frames(cfg, lo, hi)
+                    o[lo:hi] = _attend(cfg, q[lo:hi], k[keys], v[keys], rb)
                 h = rb(h + o @ W[f"attn{idx}.Wo"] + W[f"attn{idx}.bo"])
         return rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]
 
@@ -289,13 +300,63 @@ class KVRing:
 
     def append_and_view(self, k, v):
         T = k.shape[0]
-        idx = (self.head + np.arange(T)) % self.size
+        idx = (self.head + np.arange(T, dtype=np.int64)) % self.size
         self.k[idx], self.v[idx] = k, v
         L = self.filled + T
-        rows = (self.head + T - L + np.arange(L)) % self.size
+        rows = (self.head + T - L + np.arange(L, dtype=np.int64)) % self.size
         self.head = (self.head + T) % self.size
         self.filled = min(self.cap, L)
         return self.k[rows], self.v[rows]
+
+
+class ConcatCarry:
+    """The stock discipline of Eq. 4's right-hand side: the live cache H is a fresh concatenation,
+    mutable history first (newest frame first: "prepend ordering"), immutable prompt tail last;
+    the carry keeps H[0:kv_cap] and the prompt tail.  The stream's first f_prompt frames are the
+    prompt."""
+
+    def __init__(self, cap: int, f_prompt: int, C: int):
+        self.cap, self.P = cap, f_prompt
+        self.hist_k, self.hist_v = np.zeros((0, C)), np.zeros((0, C))
+        self.prompt_k, self.prompt_v = np.zeros((0, C)), np.zeros((0, C))
+
+    @property
+    def filled(self) -> int:
+        return self.hist_k.shape[0] + self.prompt_k.shape[0]
+
+    def append_and_view(self, k, v, a0: int):
+        tp = min(max(self.P - a0, 0), k.shape[0])          # chunk frames that are prompt frames
+        self.prompt_k = np.concatenate([self.prompt_k, k[:tp]], axis=0)
+        self.prompt_v = np.concatenate([self.prompt_v, v[:tp]], axis=0)
+        live_k = np.concatenate([k[tp:][::-1], self.hist_k], axis=0)
+        live_v = np.concatenate([v[tp:][::-1], self.hist_v], axis=0)
+        H_k = np.concatenate([live_k, self.prompt_k], axis=0)
+        H_v = np.concatenate([live_v, self.prompt_v], axis=0)
+        self.hist_k, self.hist_v = live_k[:self.cap], live_v[:self.cap]   # retention, after the inference that reads H
+        return H_k, H_v
+
+
+class RingCarry:
+    """The in-place discipline (Eq. 4's left-hand side): a prompt buffer of f_prompt rows written
+    once, and a ring of kv_cap + f_chunk rows for the history; nothing is allocated per chunk."""
+
+    def __init__(self, cap: int, f_chunk: int, f_prompt: int, C: int):
+        self.P = f_prompt
+        self.pk, self.pv = np.zeros((f_prompt, C)), np.zeros((f_prompt, C))
+        self.n_prompt = 0
+        self.ring = KVRing(cap, f_chunk, C)
+
+    @property
+    def filled(self) -> int:
+        return self.n_prompt + self.ring.filled
+
+    def append_and_view(self, k, v, a0: int):
+        tp = min(max(self.P - a0, 0), k.shape[0])
+        self.pk[self.n_prompt:self.n_prompt + tp], self.pv[self.n_prompt:self.n_prompt + tp] = k[:tp], v[:tp]
+        self.n_prompt += tp
+        hk, hv = self.ring.append_and_view(k[tp:], v[tp:])
+        return (np.concatenate([self.pk[:self.n_prompt], hk], axis=0),
+                np.concatenate([self.pv[:self.n_prompt], hv], axis=0))
 
 
 class FlowStream:
@@ -315,12 +376,14 @@ class FlowStream:
         self.passes = []
         for _ in range(2 if self.w_cfg > 0 else 1):
             halo = [[np.zeros((2 * d, C)) for d in cfg.dilations] for _ in range(n)]
+            P = getattr(cfg, "f_prompt", 0)
             if self.ring:
-                kv = [[KVRing(cfg.kv_cap, cfg.f_chunk, C) for _ in range(cfg.n_attn_layers)] for _ in range(n)]
+                kv = [[RingCarry(cfg.kv_cap, cfg.f_chunk, P, C) for _ in range(cfg.n_attn_layers)] for _ in range(n)]
             else:
-                kv = [[(np.zeros((0, C)), np.zeros((0, C))) for _ in range(cfg.n_attn_layers)] for _ in range(n)]
+                kv = [[ConcatCarry(cfg.kv_cap, P, C) for _ in range(cfg.n_attn_layers)] for _ in range(n)]
             self.passes.append((halo, kv))
         self.halo, self.kv = self.passes[0]
+        self.frames = 0                      # frames decoded so far = index of the next chunk's first frame
         self.kv_len_seen: List[int] = []
 
     def decode_chunk(self, feats: np.ndarray) -> np.ndarray:
@@ -336,6 +399,7 @@ class FlowStream:
             if self.w_cfg > 0:
                 vel = (1.0 + self.w_cfg) * vel - self.w_cfg * self._velocity(s, x, np.zeros_like(mu), 1, rb)
             x = x + vel / n
+        self.frames += T
         return x.astype(np.float32)
 
     def _velocity(self, s, x, cond, p, rb):
@@ -355,17 +419,9 @@ class FlowStream:
                 q = rb(u @ W[f"attn{idx}.Wq"] + W[f"attn{idx}.bq"])
                 k = rb(u @ W[f"attn{idx}.Wk"] + W[f"attn{idx}.bk"])
                 v = rb(u @ W[f"attn{idx}.Wv"] + W[f"attn{idx}.bv"])
-                if self.ring:
-                    if s == 0 and idx == 0 and p == 0:
-                        self.kv_len_seen.append(kv[s][idx].filled)
-                    k_all, v_all = kv[s][idx].append_and_view(k, v)
-                else:
-                    kc, vc = kv[s][idx]
-                    if s == 0 and idx == 0 and p == 0:
-                        self.kv_len_seen.append(kc.shape[0])
-                    k_all = np.concatenate([kc, k], axis=0)
-                    v_all = np.concatenate([vc, v], axis=0)
-                    kv[s][idx] = (k_all[-cfg.kv_cap:], v_all[-cfg.kv_cap:])
+                if s == 0 and idx == 0 and p == 0:
+                    self.kv_len_seen.append(kv[s][idx].filled)
+                k_all, v_all = kv[s][idx].append_and_view(k, v, self.frames)
                 o = _attend(cfg, q, k_all, v_all, rb)
                 h = rb(h + o @ W[f"attn{idx}.Wo"] + W[f"attn{idx}.bo"])
         return rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]

@@ -33,7 +33,7 @@ class dc_config(C.Structure):
                 ("up_channels", C.c_int32 * (DC_MAX_UP + 1)), ("n_res", C.c_int32),
                 ("res_dilations", C.c_int32 * DC_MAX_RES), ("n_fft", C.c_int32), ("hop", C.c_int32),
                 ("rms_eps", C.c_float), ("logmag_clamp", C.c_float), ("max_batch", C.c_int32),
-                ("cfg_scale", C.c_float)]
+                ("f_prompt", C.c_int32), ("cfg_scale", C.c_float)]
 
 
 class DCError(RuntimeError):
@@ -109,6 +109,7 @@ def make_config(cfg, max_batch: int = 1) -> dc_config:
     c.rms_eps, c.logmag_clamp = cfg.rms_eps, cfg.logmag_clamp
     c.max_batch = max_batch
     c.cfg_scale = float(getattr(cfg, "cfg_scale", 0.0))
+    c.f_prompt = int(getattr(cfg, "f_prompt", 0))
     return c
 
 

@@ -110,7 +110,10 @@ static dc_config sub_config(const dc_config& c, int pipeline) {
   dc_config s = c;
   s.pipeline = pipeline;
   s.precision = pipeline == DC_PIPE_FLOW ? DC_BF16 : DC_F32;
-  if (pipeline != DC_PIPE_FLOW) s.cfg_scale = 0.f;
+  if (pipeline != DC_PIPE_FLOW) {
+    s.cfg_scale = 0.f;
+    s.f_prompt = 0;
+  }
   return s;
 }
 
@@ -121,6 +124,8 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (c->f_chunk < 1 || c->f_chunk > 4096) BAD("f_chunk out of range");
   if (c->max_batch < 1 || c->max_batch > 1024) BAD("max_batch out of range");
   if (!(c->cfg_scale >= 0.f && c->cfg_scale <= 100.f)) BAD("cfg_scale out of range");
+  if (c->f_prompt < 0 || c->f_prompt > 4096) BAD("f_prompt out of range");
+  if (c->f_prompt != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_prompt belongs to the flow decoder");
   if (c->cfg_scale != 0.f && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("cfg_scale belongs to the flow decoder");
   if (c->pipeline == DC_PIPE_TOKEN2WAV) {
     if (c->precision != DC_BF16) BAD("token2wav pipeline is bf16 (flow decoder) + fp32 (vocoder tail)");

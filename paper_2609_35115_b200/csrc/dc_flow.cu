@@ -52,13 +52,15 @@ enum GemmMode { MODE_INPROJ = 0, MODE_CONV = 1, MODE_QKV = 2, MODE_OPROJ = 3, MO
 
 struct SlotInfo {
   int          T;         // frames presented by this stream in this call
-  int          kv_head;   // ring row that receives the chunk's first K/V row
-  int          kv_len;    // carried K/V rows attended (<= kv_cap), before this chunk
+  int          kv_head;   // ring row that receives the chunk's first history (non-prompt) K/V row
+  int          kv_len;    // carried history rows attended (<= kv_cap), before this chunk
   int          pass;      // 0: conditional pass (or the only one); 1: the unconditional pass of a guided stream (mu = 0, no output)
   const float* feats;     // [T][2 mel]
   float*       out;       // [T][mel]
   bf16*        halo;      // stream carry: [n_steps][n_conv][8][C]
-  bf16*        kv;        // stream carry: [n_steps][n_attn][2][Rk][C]
+  bf16*        kv;        // stream carry: [n_steps][n_attn][2][P + Rk][C] (P prompt rows, then the history ring)
+  int          n_prompt0; // prompt rows present before this chunk (<= P); the chunk's first P - n_prompt0 frames join them
+  int          pad;
 };
 
 struct SlotSet {
@@ -85,6 +87,7 @@ struct GemmParams {
   bf16*        q_out;           // MODE_QKV
   long long    kv_off;          // element offset of this (step, layer)'s K ring inside SlotInfo::kv
   int          Rk;              // ring rows
+  int          P;               // prompt rows in front of the ring (0: none)
   int          C;
   float*       xstate;          // MODE_OUT: fp32 Euler state [rows][mel]
   bf16*        ain;             // MODE_OUT: next step's input-projection operand [GUARD+rows][ld_ain]
@@ -290,7 +293,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int r = m0 + q * 32 + lane;             // row in slot layout (without GUARD)
     const int slot = r / SLOT_ROWS, rho = r % SLOT_ROWS;
     const bool in_range = slot < p.n_slots;
-    const SlotInfo si = in_range ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr};
+    const SlotInfo si = in_range ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, 0, 0};
     const int f = rho - HALO;
     const bool do_halo = p.halo_off >= 0;
     const bool has_resid = p.mode == MODE_CONV || p.mode == MODE_OPROJ;
@@ -459,9 +462,17 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (which == 0) {
             store16(p.q_out + grow * p.ld + col, a, b);
           } else {
-            int row = si.kv_head + f;
-            if (row >= p.Rk) row -= p.Rk;
-            store16(si.kv + p.kv_off + (long long)(which - 1) * p.Rk * p.C + (long long)row * p.C + col, a, b);
+            // the chunk's first tp frames complete the prompt, the others go to the history ring behind it
+            const int tp = min(si.T, p.P - si.n_prompt0);
+            int row;
+            if (f < tp) {
+              row = si.n_prompt0 + f;
+            } else {
+              row = si.kv_head + f - tp;
+              if (row >= p.Rk) row -= p.Rk;
+              row += p.P;
+            }
+            store16(si.kv + p.kv_off + (long long)(which - 1) * (p.P + p.Rk) * p.C + (long long)row * p.C + col, a, b);
           }
         }
         continue;
@@ -614,6 +625,7 @@ struct AttnParams {
   int             dh;         // 32 or 64 (smem rows are padded to 64 columns)
   long long       kv_off;     // element offset of this (step, layer)'s K ring inside SlotInfo::kv
   int             Rk, C;
+  int             P;          // prompt rows in front of the ring
   float           scale_log2e;  // log2(e) / sqrt(dh)
   int*            err;
 };
@@ -628,6 +640,9 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(dst)), "l"(src) : "memory");
 }
 
+// PROMPT = false: the carry is a plain window (no prompt rows); a separate instantiation, because this kernel sits at its
+// register limit and the copy loops of its loader warps pace it.
+template <bool PROMPT>
 __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t att_smem_raw[];
 #ifdef DC_TIMING
@@ -692,7 +707,11 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   ptx::pdl_launch();
   ptx::pdl_wait();      // the slot table, Q and the appended K/V rows come from earlier kernels
   const SlotInfo si = p.slots[slot];
-  const int T = si.T, L = si.kv_len + T;
+  // attended keys, in this order: the prompt rows (with the chunk's own prompt frames, already appended), then
+  // the carried history and the chunk's history frames, a circular interval of the ring behind the prompt rows
+  const int T = si.T;
+  const int n_prompt = PROMPT ? si.n_prompt0 + min(T, p.P - si.n_prompt0) : 0;
+  const int L = PROMPT ? n_prompt + si.kv_len + (T - (n_prompt - si.n_prompt0)) : si.kv_len + T;
   const int nkb = (L + ATT_KB - 1) / ATT_KB;
 
   if (warp >= 5) {
@@ -710,7 +729,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         else *reinterpret_cast<uint4*>(dst) = zero;
       }
     }
-    const bf16* src0 = si.kv + p.kv_off + head * p.dh + (is_k ? 0 : (long long)p.Rk * p.C);
+    const bf16* src0 = si.kv + p.kv_off + head * p.dh + (is_k ? 0 : (long long)((PROMPT ? p.P : 0) + p.Rk) * p.C);
     uint64_t* full = is_k ? full_k : full_v;
     uint64_t* empty = is_k ? empty_k : empty_v;
     int start = si.kv_head - si.kv_len;
@@ -730,16 +749,35 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       }
       uint8_t* dstb = ring + st * ATT_STAGE_BYTES + (is_k ? 0 : ATT_KB * 128);
       if (lt == 0 && is_k && b < 8) DC_AT(b);                    // block b load issue starts
-      for (int i = lt; i < ATT_KB * 8; i += nl) {
-        const int row = i >> 3, j = i & 7;
-        const int key = b * ATT_KB + row;
-        const int off = row * 128 + ((j ^ (row & 7)) << 4);
-        if (key < L && j < chunks) {
-          int rr = start + key;
-          if (rr >= p.Rk) rr -= p.Rk;
-          cp_async16(dstb + off, src0 + (long long)rr * p.C + j * 8);
-        } else {
-          *reinterpret_cast<uint4*>(dstb + off) = zero;   // for V: 0 * garbage must not poison O
+      if (!PROMPT) {
+        for (int i = lt; i < ATT_KB * 8; i += nl) {
+          const int row = i >> 3, j = i & 7;
+          const int key = b * ATT_KB + row;
+          const int off = row * 128 + ((j ^ (row & 7)) << 4);
+          if (key < L && j < chunks) {
+            int rr = start + key;
+            if (rr >= p.Rk) rr -= p.Rk;
+            cp_async16(dstb + off, src0 + (long long)rr * p.C + j * 8);
+          } else {
+            *reinterpret_cast<uint4*>(dstb + off) = zero;   // for V: 0 * garbage must not poison O
+          }
+        }
+      } else {
+        for (int i = lt; i < ATT_KB * 8; i += nl) {
+          const int row = i >> 3, j = i & 7;
+          const int key = b * ATT_KB + row;
+          const int off = row * 128 + ((j ^ (row & 7)) << 4);
+          if (key < L && j < chunks) {
+            int rr = key;                            // a prompt row, or ...
+            if (key >= n_prompt) {                   // ... a ring row behind the prompt rows
+              rr = start + key - n_prompt;
+              if (rr >= p.Rk) rr -= p.Rk;
+              rr += p.P;
+            }
+            cp_async16(dstb + off, src0 + (long long)rr * p.C + j * 8);
+          } else {
+            *reinterpret_cast<uint4*>(dstb + off) = zero;
+          }
         }
       }
     }
@@ -979,6 +1017,7 @@ struct GraphEntry {
 struct FlowModel {
   dc_config cfg;
   int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0;   // S: slots (streams x passes) of a full batch
+  int P = 0;                 // prompt rows in front of every K/V ring
   int n_pass = 1;            // 2 with classifier-free guidance: a stream's conditional and unconditional pass are
                              // adjacent slots, i.e. the two halves of one row tile
   bf16 *Xa = nullptr, *Xb = nullptr, *Q = nullptr, *O = nullptr, *Ain = nullptr;
@@ -1060,6 +1099,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   m->S = cfg.max_batch * m->n_pass;
   m->rows = ((m->S * SLOT_ROWS + TILE_M - 1) / TILE_M) * TILE_M;
   m->Rk = cfg.kv_cap + cfg.f_chunk;
+  m->P = cfg.f_prompt;
   m->cpa = cfg.n_attn > 0 ? cfg.n_conv / cfg.n_attn : cfg.n_conv;
   const int nL = cfg.n_conv, nA = cfg.n_attn, nS = cfg.n_steps;
   const size_t R = (size_t)GUARD + m->rows;
@@ -1171,7 +1211,8 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   if (e == cudaSuccess)
     chk(cudaFuncSetAttribute(flow_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
   if (e == cudaSuccess && cfg.n_attn > 0)
-    chk(cudaFuncSetAttribute(flow_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATT_SMEM));
+    chk(cudaFuncSetAttribute(m->P > 0 ? flow_attn_kernel<true> : flow_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)ATT_SMEM));
   if (e != cudaSuccess) {
     set_error("flow model allocation failed: %s", cudaGetErrorString(e));
     flow_model_destroy(m);
@@ -1236,7 +1277,7 @@ dc_status flow_state_open(FlowModel* m, FlowState** out) {
   const dc_config& c = m->cfg;
   // one set of carries per pass
   s->halo_bytes = (size_t)m->n_pass * c.n_steps * c.n_conv * HALO * m->C * sizeof(bf16);
-  s->kv_bytes = (size_t)m->n_pass * c.n_steps * c.n_attn * 2 * m->Rk * m->C * sizeof(bf16);
+  s->kv_bytes = (size_t)m->n_pass * c.n_steps * c.n_attn * 2 * (m->P + m->Rk) * m->C * sizeof(bf16);
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s->halo), s->halo_bytes);
   if (e == cudaSuccess) e = cudaMemset(s->halo, 0, s->halo_bytes);
   if (e == cudaSuccess && s->kv_bytes) {
@@ -1362,6 +1403,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     p.ld = C;
     p.C = C;
     p.Rk = m->Rk;
+    p.P = m->P;
     p.err = m->d_err;
     const int stage_bytes = A_BYTES + p.taps * ((p.BN * 128 + 1023) & ~1023);
     p.dbg = m->dbg;
@@ -1391,11 +1433,11 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
   auto attention = [&](int step, int layer) {
     AttnParams p{};
     p.slots = m->d_slots; p.q = m->Q; p.o = m->O; p.ld = C; p.dh = c.head_dim;
-    p.kv_off = ((long long)step * c.n_attn + layer) * 2 * m->Rk * C;
-    p.Rk = m->Rk; p.C = C;
+    p.kv_off = ((long long)step * c.n_attn + layer) * 2 * (m->P + m->Rk) * C;
+    p.Rk = m->Rk; p.C = C; p.P = m->P;
     p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
     p.err = m->d_err;
-    launch(lc, flow_attn_kernel, dim3(n, c.n_heads), dim3(ATT_THREADS), ATT_SMEM, true, 2, p);
+    launch(lc, m->P > 0 ? flow_attn_kernel<true> : flow_attn_kernel<false>, dim3(n, c.n_heads), dim3(ATT_THREADS), ATT_SMEM, true, 2, p);
   };
   const float* fc = m->fconst;
   const long long halo_stride = (long long)HALO * C;
@@ -1435,7 +1477,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
           GemmParams p{};
           p.mode = MODE_QKV; p.BN = bq; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bqkv[g]; p.q_out = m->Q; p.halo_off = -1;
-          p.kv_off = ((long long)s * c.n_attn + g) * 2 * m->Rk * C;
+          p.kv_off = ((long long)s * c.n_attn + g) * 2 * (m->P + m->Rk) * C;
           normalised(p);
           gemm(*tX, m->tmWqkv[v][g], p, 3 * C);
         }
@@ -1532,8 +1574,11 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       FlowState* s = states[stream];
       SlotInfo& si = set.s[i];
       si.T = T[stream];
-      si.kv_head = (int)(s->frames % m->Rk);
-      si.kv_len = (int)(s->frames < c.kv_cap ? s->frames : c.kv_cap);
+      const long long hist = s->frames > m->P ? s->frames - m->P : 0;   // history frames so far (after the prompt)
+      si.n_prompt0 = (int)(s->frames < m->P ? s->frames : m->P);
+      si.kv_head = (int)(hist % m->Rk);
+      si.kv_len = (int)(hist < c.kv_cap ? hist : c.kv_cap);
+      si.pad = 0;
       si.pass = pass;
       si.feats = feats[stream];
       si.out = pass == 0 ? outp[stream] : nullptr;

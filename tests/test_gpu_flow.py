@@ -189,3 +189,22 @@ def test_guided_batched_equals_single_stream(dc):
     m.destroy()
     for i in range(len(w.streams)):
         assert np.array_equal(outs[i].cpu().numpy(), single[i]), f"stream {i}"
+
+
+# ---- prompt + retained carry: the first f_prompt frames are never evicted, behind them a window of kv_cap frames ----
+
+def test_prompt_carry_tiny_ragged(dc):
+    """A chunk straddles the end of the prompt (frames 14..23, f_prompt = 17); the ring wraps several times."""
+    _parity(dc, wl.tiny_flow(f_prompt=17, n_chunks=len(RAGGED) - 1), boundaries=RAGGED)
+
+
+def test_prompt_carry_with_guidance(dc):
+    _parity(dc, wl.tiny_flow(f_prompt=9, cfg_scale=0.7, n_chunks=len(RAGGED) - 1), boundaries=RAGGED)
+
+
+def test_paper_operating_point_carry(dc):
+    """cfg3's network with the paper's clock quantities: f_prompt = 302, f_retained = 100, 50-frame chunks
+    (attended extents 302 / 352 / 402 once the prompt is in)."""
+    cfg = wl.EXTRA_CONFIGS["cfg3_paper_carry"].replace(n_chunks=13)
+    bounds = [0, 50, 100, 150, 200, 250, 300, 302, 352, 402, 452, 502, 552, 602]
+    _parity(dc, cfg, boundaries=bounds)

@@ -454,3 +454,50 @@ def test_classifier_free_guidance_pins():
     assert np.allclose(st_concat, off, rtol=0, atol=1e-9 * np.abs(off).max())
     assert np.array_equal(st_concat, st_ring)
     assert not np.allclose(off, orc.run_offline(cfg, wk.weights, s.feats, bounds), atol=1e-3)
+
+
+def test_prompt_plus_retained_carry_pins():
+    """Retention policy of the paper's flow decoder (Sec. 3.1 "Two extents", Eq. 4, Eq. 5): the stream's
+    first f_prompt frames are never evicted, behind them a window of f_retained frames.
+    (i) the carried extents of the paper's operating point run through its catalog {302, 352, 402};
+    (ii) stock discipline (concatenate newest-first, truncate) == in-place discipline (prompt buffer +
+    ring) == offline run with the attended sets written out; (iii) a prompt frame still matters far
+    beyond the window, a frame just behind the window does not."""
+    # (i) bookkeeping only: a network as small as possible, the paper's clock quantities
+    cfg = wl.tiny_flow(hidden=64, n_heads=2, head_dim=32, n_steps=1, dilations=(1, 1), n_attn_layers=1,
+                       kv_cap=100, f_prompt=302, f_chunk=50, precision="f32")
+    bounds = [0, 50, 100, 150, 200, 250, 300, 302, 352, 402, 452, 502, 552]     # the prompt, then 50-frame chunks
+    wk = wl.make_workload(cfg.replace(n_chunks=len(bounds) - 1), boundaries=[bounds])
+    s = wk.streams[0]
+    st = orc.FlowStream(cfg, wk.weights, carry="ring")
+    for c in range(len(bounds) - 1):
+        st.decode_chunk(s.feats[bounds[c]:bounds[c + 1]])
+    assert st.kv_len_seen[:7] == [0, 50, 100, 150, 200, 250, 300]
+    assert st.kv_len_seen[7:] == [302, 352, 402, 402, 402]                       # {302, 352, 402}: K = 3 classes
+    envelope = max(st.kv_len_seen) + 56
+    assert envelope == 458
+    # (ii), (iii) on ragged chunks, bf16 mirroring on
+    cfg = wl.tiny_flow(f_prompt=17, n_chunks=9)
+    bounds = [0, 3, 13, 14, 24, 31, 41, 51, 52, 62]
+    wk = wl.make_workload(cfg, boundaries=[bounds])
+    s = wk.streams[0]
+    off = orc.run_offline(cfg, wk.weights, s.feats, bounds)
+    stock = orc.run_stream(cfg, wk.weights, s.feats, bounds)
+    ring = orc.run_stream(cfg, wk.weights, s.feats, bounds, carry="ring")
+    tol = 1e-9 * np.abs(off).max()
+    assert np.allclose(stock, off, rtol=0, atol=tol) and np.allclose(ring, off, rtol=0, atol=tol)
+    assert not np.allclose(off, orc.run_offline(cfg.replace(f_prompt=0), wk.weights, s.feats, bounds), atol=1e-3)
+    # (iii) one attention layer behind local convs, one Euler step: a frame reaches a later chunk only as a key
+    one = wl.tiny_flow(f_prompt=17, n_steps=1, dilations=(1, 1), n_attn_layers=1, n_chunks=9)
+    wk1 = wl.make_workload(one, boundaries=[bounds])
+    s1 = wk1.streams[0]
+    base = orc.run_offline(one, wk1.weights, s1.feats, bounds)
+    f2 = s1.feats.copy()
+    f2[5, :one.mel_dim] += 1.0                              # a prompt frame (5 < 17)
+    assert not np.allclose(orc.run_offline(one, wk1.weights, f2, bounds)[52:], base[52:], atol=1e-4)
+    f3 = s1.feats.copy()
+    f3[20, :one.mel_dim] += 1.0                             # history frame 20: the chunk [52, 62) attends [28, 52) and the prompt
+    assert np.array_equal(orc.run_offline(one, wk1.weights, f3, bounds)[52:], base[52:])
+    no_prompt = one.replace(f_prompt=0)
+    base0 = orc.run_offline(no_prompt, wk1.weights, s1.feats, bounds)
+    assert np.array_equal(orc.run_offline(no_prompt, wk1.weights, f2, bounds)[52:], base0[52:])   # without a prompt frame 5 is gone too
