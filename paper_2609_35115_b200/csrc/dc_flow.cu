@@ -762,7 +762,16 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
             *reinterpret_cast<uint4*>(dstb + off) = zero;   // for V: 0 * garbage must not poison O
           }
         }
+      } else if ((b + 1) * ATT_KB <= n_prompt) {
+        // a block of prompt rows only: row index = key
+        for (int i = lt; i < ATT_KB * 8; i += nl) {
+          const int row = i >> 3, j = i & 7;
+          const int off = row * 128 + ((j ^ (row & 7)) << 4);
+          if (j < chunks) cp_async16(dstb + off, src0 + (long long)(b * ATT_KB + row) * p.C + j * 8);
+          else *reinterpret_cast<uint4*>(dstb + off) = zero;
+        }
       } else {
+        // the block where the prompt rows end and the ring behind them begins (or ring rows only)
         for (int i = lt; i < ATT_KB * 8; i += nl) {
           const int row = i >> 3, j = i & 7;
           const int key = b * ATT_KB + row;
