@@ -115,7 +115,8 @@ def describe(cfg) -> str:
                 f"{cfg.n_attn_layers} attention layers ({cfg.n_heads}x{cfg.head_dim}, KV cap {cfg.kv_cap}), "
                 f"{cfg.n_steps} Euler steps, {cfg.f_chunk}-frame chunks, bf16 / fp32 accumulate"
                 + (f", classifier-free guidance w={cfg.cfg_scale} (two passes per step)" if cfg.cfg_scale > 0 else "")
-                + (f", {cfg.f_prompt}-frame prompt kept in the carry" if cfg.f_prompt > 0 else ""))
+                + (f", {cfg.f_prompt}-frame prompt kept in the carry" if cfg.f_prompt > 0 else "")
+                + (f", {cfg.f_lookahead} look-ahead frames per call" if cfg.f_lookahead > 0 else ""))
     if cfg.pipeline == "vocoder":
         return (f"{cfg.name}: vocoder tail mel {cfg.mel_dim} -> strides {cfg.up_strides} channels {cfg.up_channels} "
                 f"-> head -> iSTFT n_fft {cfg.n_fft} hop {cfg.hop}, {cfg.f_chunk}-frame chunks, fp32")
@@ -143,7 +144,7 @@ def flops_per_launch(cfg, cls: str, n_streams: int) -> float:
 
 def attention_bytes_per_launch(cfg, n_streams: int) -> float:
     """K and V rows of the attended window (bf16) + Q read + O write."""
-    L = getattr(cfg, "f_prompt", 0) + cfg.kv_cap + cfg.f_chunk
+    L = getattr(cfg, "f_prompt", 0) + cfg.kv_cap + cfg.f_chunk + getattr(cfg, "f_lookahead", 0)
     passes = 2 if getattr(cfg, "cfg_scale", 0.0) > 0 else 1
     return passes * n_streams * (2.0 * L * cfg.hidden * 2 + 2.0 * cfg.f_chunk * cfg.hidden * 2)
 
@@ -251,6 +252,7 @@ def main():
 
     metric, unit, per_chunk = units_per_chunk(cfg)
     S, T = cfg.n_streams, cfg.f_chunk
+    Tp = T + getattr(cfg, "f_lookahead", 0)     # frames a call presents; it commits (and is credited with) T
     W, K = max(args.warmup, 3), args.steps
     has_flow = cfg.pipeline in ("flow", "token2wav")
     history = HISTORY_CHUNKS if has_flow else 2
@@ -261,7 +263,7 @@ def main():
     weights = wl.make_weights(cfg, np.random.default_rng(cfg.seed))
     model = dc.Model(cfg, weights, max_batch=S)
     streams = [model.open_stream() for _ in range(S)]
-    feats_h = torch.from_numpy(rng.standard_normal((rounds, S, T, cfg.in_dim), dtype=np.float32))
+    feats_h = torch.from_numpy(rng.standard_normal((rounds, S, Tp, cfg.in_dim), dtype=np.float32))
     feats_d = feats_h.cuda()
     out_d = torch.empty(S, T * cfg.out_per_frame, device="cuda")
     out_dv = out_d.view(S, T, -1) if cfg.pipeline not in ("vocoder", "token2wav") else out_d
@@ -462,7 +464,7 @@ def main():
             "latency_us": {"p50": 1e3 * step_ms[len(step_ms) // 2], "p95": 1e3 * step_ms[min(len(step_ms) - 1, int(0.95 * len(step_ms)))],
                            "per": "step (one chunk of every stream)"},
             "latency_us_cold_l2": cold,
-            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": S * T * cfg.in_dim * 4,
+            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": S * Tp * cfg.in_dim * 4,
                     "d2h_bytes_per_step": S * T * cfg.out_per_frame * 4, "ms_per_step": 1e3 * e2e_s / K},
             "gpu_launches": int(c1[5] - c0[5]),
             "clocks": clocks,

@@ -51,6 +51,7 @@ class DCConfig:
     head_dim: int = 0
     kv_cap: int = 0                     # W, frames of carried keys/values (the retained history)
     f_prompt: int = 0                   # the stream's first f_prompt frames are a prompt that is never evicted
+    f_lookahead: int = 0                # a full call of f_chunk frames also presents this many provisional frames
     n_steps: int = 0                    # Euler steps per chunk
     f_chunk: int = 50                   # admission bound on frames per call
     mel_dim: int = 80
@@ -267,6 +268,8 @@ EXTRA_CONFIGS: Dict[str, DCConfig] = {
     "cfg3_guided": CONFIGS["cfg3"].replace(name="cfg3_guided", cfg_scale=0.7, seed=7),
     # cfg3's network with the paper's carry: a 302-frame prompt that is never evicted + 100 retained frames
     "cfg3_paper_carry": CONFIGS["cfg3"].replace(name="cfg3_paper_carry", f_prompt=302, kv_cap=100, seed=8),
+    # ... and the 6 look-ahead frames of its 56-frame calls: the paper's whole declaration for this decoder
+    "cfg3_paper": CONFIGS["cfg3"].replace(name="cfg3_paper", f_prompt=302, kv_cap=100, f_lookahead=6, seed=9),
 }
 
 

@@ -102,6 +102,13 @@ typedef struct dc_config {
                                   * are never evicted; behind them the carry keeps the last kv_cap frames (the
                                   * paper's f_prompt + f_retained carry, Section 3.1 and Eq. 4).  0: a plain
                                   * sliding window of kv_cap frames.                              */
+  int32_t  f_lookahead;          /* flow decoder: a call may present up to f_chunk + f_lookahead frames; the frames
+                                  * beyond f_chunk are look-ahead (Section 3.1, "Two extents": they sit in the
+                                  * envelope, the call attends them, and they are dropped before the retention
+                                  * policy truncates): the call commits - output, conv left context, K/V carry -
+                                  * its first min(n_frames, f_chunk) frames, reports that count through n_out, and
+                                  * the caller presents the other frames again at the head of its next call.
+                                  * f_chunk + f_lookahead <= 56.                                  */
   float    cfg_scale;            /* flow decoder: classifier-free guidance weight w >= 0; 0 = off.  With w > 0 every
                                   * Euler step evaluates the network twice - with the conditioning and with the
                                   * conditioning set to zero, each pass with carries of its own - and advances

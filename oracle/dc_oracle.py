@@ -291,21 +291,24 @@ class KVRing:
     (Eq. 4's discipline: same values as concatenate-then-truncate, constant
     storage)."""
 
-    def __init__(self, cap: int, f_chunk: int, C: int):
-        self.cap, self.size = cap, cap + f_chunk
+    def __init__(self, cap: int, f_call: int, C: int):
+        self.cap, self.size = cap, cap + f_call
         self.k = np.zeros((self.size, C))
         self.v = np.zeros((self.size, C))
         self.head = 0          # next row to write
         self.filled = 0        # carried rows (<= cap)
 
-    def append_and_view(self, k, v):
+    def append_and_view(self, k, v, n_commit: Optional[int] = None):
+        """Writes the T rows at the head and returns the attended rows; the head only advances by
+        n_commit rows (the others are look-ahead: attended now, overwritten by the next call)."""
         T = k.shape[0]
+        nc = T if n_commit is None else n_commit
         idx = (self.head + np.arange(T, dtype=np.int64)) % self.size
         self.k[idx], self.v[idx] = k, v
         L = self.filled + T
         rows = (self.head + T - L + np.arange(L, dtype=np.int64)) % self.size
-        self.head = (self.head + T) % self.size
-        self.filled = min(self.cap, L)
+        self.head = (self.head + nc) % self.size
+        self.filled = min(self.cap, self.filled + nc)
         return self.k[rows], self.v[rows]
 
 
@@ -324,15 +327,24 @@ class ConcatCarry:
     def filled(self) -> int:
         return self.hist_k.shape[0] + self.prompt_k.shape[0]
 
-    def append_and_view(self, k, v, a0: int):
-        tp = min(max(self.P - a0, 0), k.shape[0])          # chunk frames that are prompt frames
-        self.prompt_k = np.concatenate([self.prompt_k, k[:tp]], axis=0)
-        self.prompt_v = np.concatenate([self.prompt_v, v[:tp]], axis=0)
+    def append_and_view(self, k, v, a0: int, n_commit: Optional[int] = None):
+        """k, v: the call's frames (absolute index a0 ..); only the first n_commit are kept afterwards
+        (look-ahead frames sit in the live cache H but are dropped before truncation)."""
+        T = k.shape[0]
+        nc = T if n_commit is None else n_commit
+        tp = min(max(self.P - a0, 0), T)                    # call frames that are prompt frames
+        live_prompt_k = np.concatenate([self.prompt_k, k[:tp]], axis=0)
+        live_prompt_v = np.concatenate([self.prompt_v, v[:tp]], axis=0)
         live_k = np.concatenate([k[tp:][::-1], self.hist_k], axis=0)
         live_v = np.concatenate([v[tp:][::-1], self.hist_v], axis=0)
-        H_k = np.concatenate([live_k, self.prompt_k], axis=0)
-        H_v = np.concatenate([live_v, self.prompt_v], axis=0)
-        self.hist_k, self.hist_v = live_k[:self.cap], live_v[:self.cap]   # retention, after the inference that reads H
+        H_k = np.concatenate([live_k, live_prompt_k], axis=0)
+        H_v = np.concatenate([live_v, live_prompt_v], axis=0)
+        # retention, after the inference that reads H: drop the look-ahead frames, then truncate
+        tpc = min(tp, nc)
+        self.prompt_k = np.concatenate([self.prompt_k, k[:tpc]], axis=0)
+        self.prompt_v = np.concatenate([self.prompt_v, v[:tpc]], axis=0)
+        drop = (T - tp) - max(nc - tp, 0)                   # look-ahead frames among the history frames (newest first)
+        self.hist_k, self.hist_v = live_k[drop:][:self.cap], live_v[drop:][:self.cap]
         return H_k, H_v
 
 
@@ -350,13 +362,16 @@ class RingCarry:
     def filled(self) -> int:
         return self.n_prompt + self.ring.filled
 
-    def append_and_view(self, k, v, a0: int):
-        tp = min(max(self.P - a0, 0), k.shape[0])
+    def append_and_view(self, k, v, a0: int, n_commit: Optional[int] = None):
+        T = k.shape[0]
+        nc = T if n_commit is None else n_commit
+        tp = min(max(self.P - a0, 0), T)
         self.pk[self.n_prompt:self.n_prompt + tp], self.pv[self.n_prompt:self.n_prompt + tp] = k[:tp], v[:tp]
-        self.n_prompt += tp
-        hk, hv = self.ring.append_and_view(k[tp:], v[tp:])
-        return (np.concatenate([self.pk[:self.n_prompt], hk], axis=0),
-                np.concatenate([self.pv[:self.n_prompt], hv], axis=0))
+        n_live = self.n_prompt + tp                        # look-ahead rows are written too; the next call overwrites them
+        self.n_prompt += min(tp, nc)
+        hk, hv = self.ring.append_and_view(k[tp:], v[tp:], max(nc - tp, 0))
+        return (np.concatenate([self.pk[:n_live], hk], axis=0),
+                np.concatenate([self.pv[:n_live], hv], axis=0))
 
 
 class FlowStream:
@@ -378,7 +393,8 @@ class FlowStream:
             halo = [[np.zeros((2 * d, C)) for d in cfg.dilations] for _ in range(n)]
             P = getattr(cfg, "f_prompt", 0)
             if self.ring:
-                kv = [[RingCarry(cfg.kv_cap, cfg.f_chunk, P, C) for _ in range(cfg.n_attn_layers)] for _ in range(n)]
+                kv = [[RingCarry(cfg.kv_cap, cfg.f_chunk + getattr(cfg, "f_lookahead", 0), P, C)
+                       for _ in range(cfg.n_attn_layers)] for _ in range(n)]
             else:
                 kv = [[ConcatCarry(cfg.kv_cap, P, C) for _ in range(cfg.n_attn_layers)] for _ in range(n)]
             self.passes.append((halo, kv))
@@ -391,7 +407,12 @@ class FlowStream:
         rb = round_bf16 if cfg.precision == "bf16" else (lambda a: a)
         feats = np.asarray(feats, dtype=np.float64)
         T = feats.shape[0]
-        assert 1 <= T <= cfg.f_chunk
+        la = getattr(cfg, "f_lookahead", 0)
+        assert 1 <= T <= cfg.f_chunk + la
+        # Frames beyond f_chunk are look-ahead (Sec. 3.1 "Two extents": they reside in the envelope, are attended
+        # by the call, and are discarded before the retention policy truncates): the call commits the first Tc
+        # frames - output, conv left context and K/V carry - and the caller presents the others again.
+        self.Tc = min(T, cfg.f_chunk)
         m, n = cfg.mel_dim, cfg.n_steps
         mu, x = feats[:, :m], feats[:, m:].copy()
         for s in range(n):
@@ -399,8 +420,8 @@ class FlowStream:
             if self.w_cfg > 0:
                 vel = (1.0 + self.w_cfg) * vel - self.w_cfg * self._velocity(s, x, np.zeros_like(mu), 1, rb)
             x = x + vel / n
-        self.frames += T
-        return x.astype(np.float32)
+        self.frames += self.Tc
+        return x[:self.Tc].astype(np.float32)
 
     def _velocity(self, s, x, cond, p, rb):
         """One evaluation of the network at Euler step s with pass p's carries (updated in passing)."""
@@ -410,7 +431,7 @@ class FlowStream:
         for kind, idx, d in self.plan:
             if kind == "conv":
                 left = halo[s][idx]
-                halo[s][idx] = np.concatenate([left, h], axis=0)[-2 * d:]
+                halo[s][idx] = np.concatenate([left, h[:self.Tc]], axis=0)[-2 * d:]
                 z = (causal_conv_k3(h, W[f"conv{idx}.W"], d, left)
                      + W[f"conv{idx}.b"] + self.tau[s, idx])
                 h = rb(h + silu(z))
@@ -421,7 +442,7 @@ class FlowStream:
                 v = rb(u @ W[f"attn{idx}.Wv"] + W[f"attn{idx}.bv"])
                 if s == 0 and idx == 0 and p == 0:
                     self.kv_len_seen.append(kv[s][idx].filled)
-                k_all, v_all = kv[s][idx].append_and_view(k, v, self.frames)
+                k_all, v_all = kv[s][idx].append_and_view(k, v, self.frames, self.Tc)
                 o = _attend(cfg, q, k_all, v_all, rb)
                 h = rb(h + o @ W[f"attn{idx}.Wo"] + W[f"attn{idx}.bo"])
         return rb(rmsnorm(h, cfg.rms_eps)) @ W["out.W"] + W["out.b"]
@@ -596,6 +617,8 @@ def run_offline(cfg, blob, feats, boundaries) -> np.ndarray:
 
 def run_stream(cfg, blob, feats, boundaries, **kw) -> np.ndarray:
     st = make_stream(cfg, blob, **kw)
-    outs = [st.decode_chunk(feats[boundaries[c]:boundaries[c + 1]])
+    la = getattr(cfg, "f_lookahead", 0)         # a call also presents the next <= la frames, which it does not commit
+    F = boundaries[-1]
+    outs = [st.decode_chunk(feats[boundaries[c]:min(boundaries[c + 1] + (la if boundaries[c + 1] - boundaries[c] == cfg.f_chunk else 0), F)])
             for c in range(len(boundaries) - 1)]
     return np.concatenate(outs, axis=0)

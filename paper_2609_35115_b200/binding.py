@@ -33,7 +33,7 @@ class dc_config(C.Structure):
                 ("up_channels", C.c_int32 * (DC_MAX_UP + 1)), ("n_res", C.c_int32),
                 ("res_dilations", C.c_int32 * DC_MAX_RES), ("n_fft", C.c_int32), ("hop", C.c_int32),
                 ("rms_eps", C.c_float), ("logmag_clamp", C.c_float), ("max_batch", C.c_int32),
-                ("f_prompt", C.c_int32), ("cfg_scale", C.c_float)]
+                ("f_prompt", C.c_int32), ("f_lookahead", C.c_int32), ("cfg_scale", C.c_float)]
 
 
 class DCError(RuntimeError):
@@ -110,6 +110,7 @@ def make_config(cfg, max_batch: int = 1) -> dc_config:
     c.max_batch = max_batch
     c.cfg_scale = float(getattr(cfg, "cfg_scale", 0.0))
     c.f_prompt = int(getattr(cfg, "f_prompt", 0))
+    c.f_lookahead = int(getattr(cfg, "f_lookahead", 0))
     return c
 
 
@@ -189,7 +190,7 @@ class Stream:
         _check(st, "dc_decode_chunk")
         res = out[: n_out.value]
         if self.model.cfg.pipeline not in ("vocoder", "token2wav"):
-            res = res.view(T, -1)
+            res = res.view(-1, self.model.out_per_frame)      # committed frames (fewer than T when the call carried look-ahead frames)
         return res
 
     def decode_chunk_host(self, feats_host, out_host, stream=None) -> int:

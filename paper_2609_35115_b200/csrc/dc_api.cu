@@ -113,6 +113,7 @@ static dc_config sub_config(const dc_config& c, int pipeline) {
   if (pipeline != DC_PIPE_FLOW) {
     s.cfg_scale = 0.f;
     s.f_prompt = 0;
+    s.f_lookahead = 0;
   }
   return s;
 }
@@ -125,6 +126,8 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (c->max_batch < 1 || c->max_batch > 1024) BAD("max_batch out of range");
   if (!(c->cfg_scale >= 0.f && c->cfg_scale <= 100.f)) BAD("cfg_scale out of range");
   if (c->f_prompt < 0 || c->f_prompt > 4096) BAD("f_prompt out of range");
+  if (c->f_lookahead < 0 || c->f_lookahead > 32) BAD("f_lookahead out of range");
+  if (c->f_lookahead != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_lookahead belongs to the flow decoder");
   if (c->f_prompt != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_prompt belongs to the flow decoder");
   if (c->cfg_scale != 0.f && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("cfg_scale belongs to the flow decoder");
   if (c->pipeline == DC_PIPE_TOKEN2WAV) {
@@ -152,7 +155,7 @@ static bool config_ok(const dc_config* c, const char** why) {
     }
     if (c->n_steps < 1 || c->n_steps > 64) BAD("n_steps out of range");
     if (c->mel_dim < 16 || c->mel_dim % 16 || c->mel_dim > 128) BAD("mel_dim must be a multiple of 16, <= 128");
-    if (c->f_chunk > 56) BAD("flow f_chunk must be <= 56");
+    if (c->f_chunk + c->f_lookahead > 56) BAD("flow f_chunk + f_lookahead must be <= 56");
   } else if (c->pipeline == DC_PIPE_VOCODER) {
     if (c->precision != DC_F32) BAD("vocoder pipeline is fp32");
     if (c->mel_dim < 4 || c->mel_dim % 4) BAD("mel_dim must be a multiple of 4");
@@ -282,7 +285,8 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     m->in_dim = 2 * cfg->mel_dim;
     m->out_per_frame = cfg->mel_dim;
     if (st == DC_OK) {
-      const size_t ni = (size_t)cfg->max_batch * cfg->f_chunk * m->in_dim, no = (size_t)cfg->max_batch * cfg->f_chunk * m->out_per_frame;
+      const size_t ni = (size_t)cfg->max_batch * (cfg->f_chunk + cfg->f_lookahead) * m->in_dim,
+                   no = (size_t)cfg->max_batch * cfg->f_chunk * m->out_per_frame;
       cudaError_t e = cudaMallocHost(&m->h_in, ni * sizeof(float));
       if (e == cudaSuccess) e = cudaMallocHost(&m->h_out, no * sizeof(float));
       if (e == cudaSuccess) e = cudaMallocHost(&m->h_err, sizeof(int));
@@ -394,7 +398,7 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
     }
   }
   if (e == cudaSuccess && st == DC_OK) {
-    e = cudaMalloc(&s->stage_in, (size_t)m->cfg.f_chunk * m->in_dim * sizeof(float));
+    e = cudaMalloc(&s->stage_in, (size_t)(m->cfg.f_chunk + m->cfg.f_lookahead) * m->in_dim * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(&s->stage_out, (size_t)m->cfg.f_chunk * m->out_per_frame * sizeof(float));
   }
   if (e != cudaSuccess) {
@@ -608,9 +612,10 @@ static dc_status admit(dc_stream* s, const float* feats, int T, float* out) {
     s->model->counters[3]++;
     return DC_ERR_ARG;
   }
-  if (T < 1 || T > s->model->cfg.f_chunk) {
+  const int f_call = s->model->cfg.f_chunk + s->model->cfg.f_lookahead;   // committed frames are bounded by f_chunk, presented ones by this
+  if (T < 1 || T > f_call) {
     s->model->counters[2]++;
-    dc::set_error("n_frames = %d violates 1 <= n_frames <= f_chunk = %d", T, s->model->cfg.f_chunk);
+    dc::set_error("n_frames = %d violates 1 <= n_frames <= f_chunk + f_lookahead = %d", T, f_call);
     return DC_ERR_FRAMES;
   }
   return DC_OK;
@@ -624,7 +629,7 @@ extern "C" dc_status dc_decode_chunk(dc_stream* s, const float* feats, int T, fl
   int launches = 0;
   if (m->sub_flow) {   // mel frames never leave the device: the flow decoder's output is the vocoder tail's input
     st = dc_decode_chunk(s->sub_flow, feats, T, s->mel, nullptr, cuda_stream);
-    if (st == DC_OK) st = dc_decode_chunk(s->sub_voc, s->mel, T, out, nullptr, cuda_stream);
+    if (st == DC_OK) st = dc_decode_chunk(s->sub_voc, s->mel, T < m->cfg.f_chunk ? T : m->cfg.f_chunk, out, nullptr, cuda_stream);
   } else if (m->flow) {
     st = dc::flow_decode(m->flow, 1, &s->flow, &feats, &T, &out, cs, &launches);
   } else {
@@ -635,11 +640,12 @@ extern "C" dc_status dc_decode_chunk(dc_stream* s, const float* feats, int T, fl
     s->poisoned = true;
     return st;
   }
-  s->frames_total += T;
+  const int Tc = T < m->cfg.f_chunk ? T : m->cfg.f_chunk;   // frames beyond f_chunk were look-ahead: attended, not committed
+  s->frames_total += Tc;
   s->chunks += 1;
   m->counters[0] += 1;
-  m->counters[1] += (uint64_t)T;
-  if (n_out) *n_out = T * m->out_per_frame;
+  m->counters[1] += (uint64_t)Tc;
+  if (n_out) *n_out = Tc * m->out_per_frame;
   return DC_OK;
 }
 
@@ -681,7 +687,9 @@ extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* strea
       mels[(size_t)i] = streams[i]->mel;
     }
     st = dc_decode_batch(m->sub_flow, n, fs.data(), feats, n_frames, mels.data(), cuda_stream);
-    for (int i = 0; i < n && st == DC_OK; ++i) st = dc_decode_chunk(streams[i]->sub_voc, streams[i]->mel, n_frames[i], out[i], nullptr, cuda_stream);
+    for (int i = 0; i < n && st == DC_OK; ++i)
+      st = dc_decode_chunk(streams[i]->sub_voc, streams[i]->mel, n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk, out[i], nullptr,
+                           cuda_stream);
   } else {
     st = dc::flow_decode(m->flow, n, states.data(), feats, n_frames, out, (cudaStream_t)cuda_stream, &launches);
   }
@@ -691,9 +699,10 @@ extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* strea
     return st;
   }
   for (int i = 0; i < n; ++i) {
-    streams[i]->frames_total += n_frames[i];
+    const int Tc = n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk;
+    streams[i]->frames_total += Tc;
     streams[i]->chunks += 1;
-    m->counters[1] += (uint64_t)n_frames[i];
+    m->counters[1] += (uint64_t)Tc;
   }
   m->counters[0] += (uint64_t)n;
   return DC_OK;
@@ -734,7 +743,7 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
   }
   if (n < 1 || n > m->cfg.max_batch) return DC_ERR_ARG;
   cudaStream_t cs = (cudaStream_t)cuda_stream;
-  const size_t in_stride = (size_t)m->cfg.f_chunk * m->in_dim, out_stride = (size_t)m->cfg.f_chunk * m->out_per_frame;
+  const size_t in_stride = (size_t)(m->cfg.f_chunk + m->cfg.f_lookahead) * m->in_dim, out_stride = (size_t)m->cfg.f_chunk * m->out_per_frame;
   std::vector<const float*> fin((size_t)n);
   std::vector<float*> fout((size_t)n);
   for (int i = 0; i < n; ++i) {
@@ -761,7 +770,8 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
     return DC_ERR_TIMEOUT;
   }
   for (int i = 0; i < n; ++i)
-    memcpy(out_host[i], m->h_out + (size_t)i * out_stride, (size_t)n_frames[i] * m->out_per_frame * sizeof(float));
+    memcpy(out_host[i], m->h_out + (size_t)i * out_stride,
+           (size_t)(n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk) * m->out_per_frame * sizeof(float));
   return DC_OK;
 }
 

@@ -60,7 +60,8 @@ struct SlotInfo {
   bf16*        halo;      // stream carry: [n_steps][n_conv][8][C]
   bf16*        kv;        // stream carry: [n_steps][n_attn][2][P + Rk][C] (P prompt rows, then the history ring)
   int          n_prompt0; // prompt rows present before this chunk (<= P); the chunk's first P - n_prompt0 frames join them
-  int          pad;
+  int          Tc;        // committed frames (<= T): the others are look-ahead - computed and attended, but neither output
+                          // nor carried (their K/V rows are written past the ring head and overwritten by the next call)
 };
 
 struct SlotSet {
@@ -340,7 +341,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const bool slot_ok = in_range && got && *s_fail == 0;
     const bool is_halo = slot_ok && rho < HALO;
     const bool is_chunk = slot_ok && f >= 0 && f < si.T;
-    const int new_row = rho - si.T;               // carry row this thread's value moves to
+    const int new_row = rho - si.Tc;              // carry row this thread's value moves to (the carry follows the committed frames)
     const bool carry_wr = do_halo && (is_halo || is_chunk) && new_row >= 0 && new_row < HALO;
 
 #pragma unroll
@@ -445,7 +446,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           pack16_bf16(xv, a, b);
           store16(p.ain + grow * p.ld_ain + n, a, b);
           if (p.cfg_w > 0.f) store16(p.ain + (grow + SLOT_ROWS) * p.ld_ain + n, a, b);   // the unconditional pass starts from the same x
-          if (p.last_step) {
+          if (p.last_step && f < si.Tc) {
             float* o = si.out + (long long)f * p.mel + n;
 #pragma unroll
             for (int i = 0; i < 16; i += 4)
@@ -1107,7 +1108,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   m->n_pass = cfg.cfg_scale > 0.f ? 2 : 1;
   m->S = cfg.max_batch * m->n_pass;
   m->rows = ((m->S * SLOT_ROWS + TILE_M - 1) / TILE_M) * TILE_M;
-  m->Rk = cfg.kv_cap + cfg.f_chunk;
+  m->Rk = cfg.kv_cap + cfg.f_chunk + cfg.f_lookahead;
   m->P = cfg.f_prompt;
   m->cpa = cfg.n_attn > 0 ? cfg.n_conv / cfg.n_attn : cfg.n_conv;
   const int nL = cfg.n_conv, nA = cfg.n_attn, nS = cfg.n_steps;
@@ -1587,7 +1588,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       si.n_prompt0 = (int)(s->frames < m->P ? s->frames : m->P);
       si.kv_head = (int)(hist % m->Rk);
       si.kv_len = (int)(hist < c.kv_cap ? hist : c.kv_cap);
-      si.pad = 0;
+      si.Tc = si.T < c.f_chunk ? si.T : c.f_chunk;
       si.pass = pass;
       si.feats = feats[stream];
       si.out = pass == 0 ? outp[stream] : nullptr;
@@ -1624,7 +1625,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       return DC_ERR_CUDA;
     }
   }
-  for (int i = 0; i < n_streams; ++i) states[i]->frames += T[i];
+  for (int i = 0; i < n_streams; ++i) states[i]->frames += T[i] < c.f_chunk ? T[i] : c.f_chunk;
   return DC_OK;
 }
 

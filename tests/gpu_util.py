@@ -10,8 +10,13 @@ def run_gpu_stream(model, feats: np.ndarray, boundaries, stream=None) -> np.ndar
     st = stream or model.open_stream()
     x = torch.from_numpy(np.ascontiguousarray(feats)).cuda()
     outs = []
+    cfg = model.cfg
+    la = getattr(cfg, "f_lookahead", 0)       # a full call also presents the next <= la frames (not committed)
     for c in range(len(boundaries) - 1):
-        outs.append(st.decode_chunk(x[boundaries[c]:boundaries[c + 1]].contiguous()).clone())
+        lo, hi = boundaries[c], boundaries[c + 1]
+        if la and hi - lo == cfg.f_chunk:
+            hi = min(hi + la, boundaries[-1])
+        outs.append(st.decode_chunk(x[lo:hi].contiguous()).clone())
     torch.cuda.synchronize()
     assert model.counters()[4] == 0, "a bounded device-side wait timed out"
     if stream is None:

@@ -208,3 +208,24 @@ def test_paper_operating_point_carry(dc):
     cfg = wl.EXTRA_CONFIGS["cfg3_paper_carry"].replace(n_chunks=13)
     bounds = [0, 50, 100, 150, 200, 250, 300, 302, 352, 402, 452, 502, 552, 602]
     _parity(dc, cfg, boundaries=bounds)
+
+
+# ---- look-ahead frames: a full call presents f_chunk + f_lookahead frames and commits the first f_chunk ----
+
+LA_BOUNDS = [0, 10, 20, 30, 33, 43, 53, 63, 73, 80]          # f_chunk = 10: full calls (with look-ahead) and partial ones
+
+
+def test_lookahead_tiny(dc):
+    _parity(dc, wl.tiny_flow(f_lookahead=3, n_chunks=len(LA_BOUNDS) - 1), boundaries=LA_BOUNDS)
+
+
+def test_lookahead_with_prompt_and_guidance(dc):
+    _parity(dc, wl.tiny_flow(f_lookahead=3, f_prompt=17, cfg_scale=0.7, n_chunks=len(LA_BOUNDS) - 1), boundaries=LA_BOUNDS)
+
+
+def test_paper_operating_point_full(dc):
+    """The paper's declaration for this decoder: f_prompt = 302, f_retained = 100, f_chunk = 50, f_call = 56
+    (6 look-ahead frames), n_steps = 10 - on cfg3's network; envelope 402 + 56 = 458 attended frames."""
+    cfg = wl.EXTRA_CONFIGS["cfg3_paper"].replace(n_chunks=13)
+    bounds = [0, 50, 100, 150, 200, 250, 300, 302, 352, 402, 452, 502, 552, 602]
+    _parity(dc, cfg, boundaries=bounds)

@@ -501,3 +501,46 @@ def test_prompt_plus_retained_carry_pins():
     no_prompt = one.replace(f_prompt=0)
     base0 = orc.run_offline(no_prompt, wk1.weights, s1.feats, bounds)
     assert np.array_equal(orc.run_offline(no_prompt, wk1.weights, f2, bounds)[52:], base0[52:])   # without a prompt frame 5 is gone too
+
+
+def test_lookahead_frames_pins():
+    """Look-ahead (Sec. 3.1 "Two extents"): a full call presents f_chunk + f_lookahead frames, attends all of
+    them, commits only the first f_chunk.  (i) stock discipline == in-place discipline, with and without a
+    prompt; (ii) a committed chunk sees exactly f_lookahead frames of the future; (iii) the envelope at the
+    paper's clock quantities is 402 + 56 = 458 frames."""
+    bounds = [0, 10, 20, 30, 33, 43, 53, 60]             # f_chunk = 10: full calls and two partial ones
+    for P in (0, 17):
+        cfg = wl.tiny_flow(f_lookahead=3, f_prompt=P, n_chunks=len(bounds) - 1)
+        wk = wl.make_workload(cfg, boundaries=[bounds])
+        s = wk.streams[0]
+        stock = orc.run_stream(cfg, wk.weights, s.feats, bounds)
+        ring = orc.run_stream(cfg, wk.weights, s.feats, bounds, carry="ring")
+        assert stock.shape == (bounds[-1], cfg.mel_dim)
+        assert np.allclose(stock, ring, rtol=0, atol=1e-9 * np.abs(stock).max())
+        plain = orc.run_stream(cfg.replace(f_lookahead=0), wk.weights, s.feats, bounds)
+        assert not np.allclose(stock, plain, atol=1e-3)     # the future frames do something
+    # (ii) one attention layer behind local convs, one Euler step: a later frame reaches a chunk only as a key
+    one = wl.tiny_flow(f_lookahead=3, n_steps=1, dilations=(1, 1), n_attn_layers=1, n_chunks=len(bounds) - 1)
+    wk = wl.make_workload(one, boundaries=[bounds])
+    s = wk.streams[0]
+    base = orc.run_stream(one, wk.weights, s.feats, bounds)
+    near = s.feats.copy()
+    near[22, :one.mel_dim] += 1.0                           # third look-ahead frame of the chunk [10, 20)
+    far = s.feats.copy()
+    far[23, :one.mel_dim] += 1.0                            # first frame beyond its look-ahead
+    assert not np.allclose(orc.run_stream(one, wk.weights, near, bounds)[10:20], base[10:20], atol=1e-4)
+    assert np.array_equal(orc.run_stream(one, wk.weights, far, bounds)[:20], base[:20])
+    # (iii) bookkeeping at the paper's operating point
+    cfg = wl.tiny_flow(hidden=64, n_heads=2, head_dim=32, n_steps=1, dilations=(1, 1), n_attn_layers=1,
+                       kv_cap=100, f_prompt=302, f_chunk=50, f_lookahead=6, precision="f32")
+    pb = [0, 50, 100, 150, 200, 250, 300, 302, 352, 402, 452, 502, 552]
+    wk = wl.make_workload(cfg.replace(n_chunks=len(pb) - 1), boundaries=[pb])
+    st = orc.FlowStream(cfg, wk.weights, carry="ring")
+    attended = []
+    for c in range(len(pb) - 1):
+        full = pb[c + 1] - pb[c] == cfg.f_chunk
+        hi = min(pb[c + 1] + (cfg.f_lookahead if full else 0), pb[-1])
+        st.decode_chunk(wk.streams[0].feats[pb[c]:hi])
+        attended.append(st.kv_len_seen[-1] + (hi - pb[c]))
+    assert st.kv_len_seen[7:] == [302, 352, 402, 402, 402]
+    assert max(attended) == 458
