@@ -234,6 +234,19 @@ dc_status dc_profile_end(dc_model* model, double ms[8], uint64_t launches[8]);
 dc_status dc_conv_stack_noalloc(const float* weights_dev, int hidden, int n_conv, const int* dilations,
                                 const float* x_dev, int n_frames, float* y_dev, void* cuda_stream);
 
+/* Snapshot of a stream's state - every carry buffer and the stream's clocks - in device memory that
+ * the library allocates (the per-session state of paper Section 3.4: sessions share the weights and
+ * the captured graphs, a session is its snapshot).  dc_stream_restore writes a snapshot back IN
+ * PLACE into the carries of `stream` (their addresses do not change), which may be the stream the
+ * snapshot came from - rewinding it - or any other open stream of the same model - moving the
+ * session.  Both enqueue device-to-device copies on cuda_stream; a snapshot may be restored any
+ * number of times and must be released with dc_snapshot_free (before dc_destroy).  Errors:
+ * DC_ERR_STATE for a closed stream or a snapshot of another model, DC_ERR_OOM. */
+typedef struct dc_snapshot dc_snapshot;
+dc_status dc_stream_snapshot(dc_stream* stream, dc_snapshot** out, void* cuda_stream);
+dc_status dc_stream_restore(dc_stream* stream, const dc_snapshot* snapshot, void* cuda_stream);
+dc_status dc_snapshot_free(dc_snapshot* snapshot);
+
 /* Device addresses and byte sizes of the stream's carry buffers, for pointer
  * constancy checks: writes up to max_entries (address, bytes) pairs into out and
  * the number of buffers into n_entries. */

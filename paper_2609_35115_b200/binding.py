@@ -21,7 +21,7 @@ EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_
            "dc_stream_close", "dc_decode_chunk", "dc_decode_batch", "dc_decode_chunk_host",
            "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error",
            "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end", "dc_conv_stack_noalloc",
-           "dc_selftest_bounded_wait"]
+           "dc_selftest_bounded_wait", "dc_stream_snapshot", "dc_stream_restore", "dc_snapshot_free"]
 
 
 class dc_config(C.Structure):
@@ -62,6 +62,9 @@ def load_library():
     lib.dc_destroy.argtypes = [vp]
     lib.dc_stream_open.argtypes = [vp, cp(vp)]
     lib.dc_stream_reset.argtypes = [vp, vp]
+    lib.dc_stream_snapshot.argtypes = [vp, cp(vp), vp]
+    lib.dc_stream_restore.argtypes = [vp, vp, vp]
+    lib.dc_snapshot_free.argtypes = [vp]
     lib.dc_stream_close.argtypes = [vp]
     lib.dc_decode_chunk.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
     lib.dc_decode_batch.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
@@ -124,6 +127,16 @@ def _cuda_stream_handle(stream) -> Optional[int]:
         import torch
         return torch.cuda.current_stream().cuda_stream
     return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+class Snapshot:
+    def __init__(self, lib, handle):
+        self.lib, self.handle = lib, handle
+
+    def free(self):
+        if self.handle:
+            _check(self.lib.dc_snapshot_free(self.handle), "dc_snapshot_free")
+            self.handle = None
 
 
 class Model:
@@ -213,6 +226,16 @@ class Stream:
         n = C.c_int(0)
         _check(self.lib.dc_stream_carry_info(self.handle, buf, 128, C.byref(n)), "dc_stream_carry_info")
         return [(buf[2 * i], buf[2 * i + 1]) for i in range(min(n.value, 128))]
+
+    def snapshot(self, stream=None) -> "Snapshot":
+        """Device-side copy of every carry of the stream plus its clocks (dc_stream_snapshot)."""
+        h = C.c_void_p()
+        _check(self.lib.dc_stream_snapshot(self.handle, C.byref(h), _cuda_stream_handle(stream)), "dc_stream_snapshot")
+        return Snapshot(self.lib, h)
+
+    def restore(self, snap: "Snapshot", stream=None):
+        """Writes a snapshot back in place (of this stream or of another stream of the same model)."""
+        _check(self.lib.dc_stream_restore(self.handle, snap.handle, _cuda_stream_handle(stream)), "dc_stream_restore")
 
     def reset(self, stream=None):
         _check(self.lib.dc_stream_reset(self.handle, _cuda_stream_handle(stream)), "dc_stream_reset")

@@ -482,6 +482,106 @@ extern "C" dc_status dc_stream_carry_info(const dc_stream* s, uint64_t* out, int
 }
 
 // ---------------------------------------------------------------------------------------------
+// snapshots
+// ---------------------------------------------------------------------------------------------
+
+struct dc_snapshot {
+  const dc_model* model = nullptr;
+  void*     data = nullptr;          // the carry buffers, back to back, in dc_stream_carry_info order
+  size_t    bytes = 0;
+  long long frames_total = 0, chunks = 0, flow_frames = 0;
+  dc_snapshot* sub_flow = nullptr;   // DC_PIPE_TOKEN2WAV: the two halves
+  dc_snapshot* sub_voc = nullptr;
+};
+
+static std::vector<DevBuf> carry_buffers(const dc_stream* s) {
+  std::vector<DevBuf> bufs;
+  if (s->flow) {
+    bufs.resize(64);
+    int n = 0;
+    dc::flow_state_buffers(s->flow, bufs.data(), 64, &n);
+    bufs.resize((size_t)n);
+  } else if (!s->sub_flow) {
+    bufs = s->f32_rings;
+    if (s->tails) bufs.push_back(DevBuf{s->tails, 2 * 12 * sizeof(float)});
+  }
+  return bufs;
+}
+
+extern "C" dc_status dc_snapshot_free(dc_snapshot* sn) {
+  if (!sn) return DC_ERR_ARG;
+  if (sn->sub_flow) dc_snapshot_free(sn->sub_flow);
+  if (sn->sub_voc) dc_snapshot_free(sn->sub_voc);
+  if (sn->data) cudaFree(sn->data);
+  delete sn;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_stream_snapshot(dc_stream* s, dc_snapshot** out, void* cuda_stream) {
+  if (!s || !out) return DC_ERR_ARG;
+  *out = nullptr;
+  if (s->closed || s->poisoned) return DC_ERR_STATE;
+  dc_snapshot* sn = new (std::nothrow) dc_snapshot();
+  if (!sn) return DC_ERR_OOM;
+  sn->model = s->model;
+  sn->frames_total = s->frames_total;
+  sn->chunks = s->chunks;
+  dc_status st = DC_OK;
+  if (s->sub_flow) {
+    st = dc_stream_snapshot(s->sub_flow, &sn->sub_flow, cuda_stream);
+    if (st == DC_OK) st = dc_stream_snapshot(s->sub_voc, &sn->sub_voc, cuda_stream);
+  } else {
+    if (s->flow) sn->flow_frames = dc::flow_state_frames(s->flow);
+    const std::vector<DevBuf> bufs = carry_buffers(s);
+    for (const DevBuf& b : bufs) sn->bytes += b.bytes;
+    cudaError_t e = cudaMalloc(&sn->data, sn->bytes ? sn->bytes : 1);
+    size_t off = 0;
+    for (size_t i = 0; i < bufs.size() && e == cudaSuccess; ++i) {
+      e = cudaMemcpyAsync((char*)sn->data + off, bufs[i].p, bufs[i].bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream);
+      off += bufs[i].bytes;
+    }
+    if (e != cudaSuccess) {
+      dc::set_error("dc_stream_snapshot: %s", cudaGetErrorString(e));
+      st = e == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;
+    }
+  }
+  if (st != DC_OK) {
+    dc_snapshot_free(sn);
+    return st;
+  }
+  *out = sn;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_stream_restore(dc_stream* s, const dc_snapshot* sn, void* cuda_stream) {
+  if (!s || !sn) return DC_ERR_ARG;
+  if (s->closed || sn->model != s->model) {
+    dc::set_error("dc_stream_restore: closed stream, or a snapshot of another model");
+    return DC_ERR_STATE;
+  }
+  if (s->sub_flow) {
+    dc_status st = dc_stream_restore(s->sub_flow, sn->sub_flow, cuda_stream);
+    if (st == DC_OK) st = dc_stream_restore(s->sub_voc, sn->sub_voc, cuda_stream);
+    if (st != DC_OK) return st;
+  } else {
+    const std::vector<DevBuf> bufs = carry_buffers(s);
+    size_t total = 0;
+    for (const DevBuf& b : bufs) total += b.bytes;
+    if (total != sn->bytes) return DC_ERR_STATE;
+    size_t off = 0;
+    for (const DevBuf& b : bufs) {   // in place: the carries keep their addresses
+      DC_CUDA(cudaMemcpyAsync(b.p, (const char*)sn->data + off, b.bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream));
+      off += b.bytes;
+    }
+    if (s->flow) dc::flow_state_set_frames(s->flow, sn->flow_frames);
+  }
+  s->frames_total = sn->frames_total;
+  s->chunks = sn->chunks;
+  s->poisoned = false;
+  return DC_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // the chunk step
 // ---------------------------------------------------------------------------------------------
 

@@ -1310,6 +1310,9 @@ void flow_state_buffers(const FlowState* s, DevBuf* out, int max_entries, int* n
   *n = k;
 }
 
+long long flow_state_frames(const FlowState* s) { return s->frames; }
+void flow_state_set_frames(FlowState* s, long long frames) { s->frames = frames; }
+
 dc_status flow_state_reset(FlowModel*, FlowState* s, cudaStream_t st) {
   // base state: zero left context, empty K/V carry (stale ring rows are never attended)
   if (cudaMemsetAsync(s->halo, 0, s->halo_bytes, st) != cudaSuccess) return DC_ERR_CUDA;
