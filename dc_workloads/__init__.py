@@ -62,6 +62,7 @@ class DCConfig:
     hop: int = 4
     rms_eps: float = 1e-6
     logmag_clamp: float = math.log(100.0)
+    noise_seed: int = 0                 # flow decoder: != 0: the Euler noise x_0 is drawn on the device (Philox), feats = mu only
     cfg_scale: float = 0.0              # flow decoder: classifier-free guidance weight w (0 = off, one pass per step)
     # workload (not part of the network)
     n_chunks: int = 1
@@ -82,6 +83,8 @@ class DCConfig:
         if self.pipeline == PIPE_CONV:
             return self.hidden
         if self.pipeline in (PIPE_FLOW, PIPE_TOKEN2WAV):
+            if self.noise_seed:
+                return self.mel_dim      # the conditioning mu; the noise x0 is drawn by the decoder itself
             return 2 * self.mel_dim      # cols [0,mel) = conditioning mu, [mel,2mel) = noise x0
         return self.mel_dim
 

@@ -109,6 +109,15 @@ typedef struct dc_config {
                                   * its first min(n_frames, f_chunk) frames, reports that count through n_out, and
                                   * the caller presents the other frames again at the head of its next call.
                                   * f_chunk + f_lookahead <= 56.                                  */
+  uint32_t noise_seed_lo, noise_seed_hi;   /* flow decoder: a non-zero 64-bit seed makes the decoder draw the Euler noise x_0
+                                  * itself, so that a chunk's input is the conditioning alone ([n_frames][mel_dim]).
+                                  * The draw for (frame t of the stream, channels 4g..4g+3) is Philox4x32-10 at counter
+                                  * (t mod 2^32, t div 2^32, g, stream index) under the key (seed_lo, seed_hi): the
+                                  * generator's offset is the stream's frame clock, so the captured chunk-step graph
+                                  * draws exactly what direct launches would (the device-randomness clause of the
+                                  * paper's effect classification, Section 3.3).  Four normals per draw by two
+                                  * Box-Muller pairs on u = ((r >> 8) + 1/2) 2^-24.  The stream index is the number
+                                  * of streams opened on the model before this one; snapshots carry it along.      */
   float    cfg_scale;            /* flow decoder: classifier-free guidance weight w >= 0; 0 = off.  With w > 0 every
                                   * Euler step evaluates the network twice - with the conditioning and with the
                                   * conditioning set to zero, each pass with carries of its own - and advances

@@ -38,7 +38,7 @@ tau, the Euler state x_s and all accumulations stay unrounded.
 from __future__ import annotations
 
 import math
-from typing import Dict, List, Optional, Sequence
+from typing import Tuple, Dict, List, Optional, Sequence
 
 import numpy as np
 
@@ -227,6 +227,41 @@ def _layer_plan(cfg):
     return plan
 
 
+_PHILOX_M0, _PHILOX_M1 = np.uint64(0xD2511F53), np.uint64(0xCD9E8D57)
+_PHILOX_W0, _PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32_10(ctr: np.ndarray, key: Tuple[int, int]) -> np.ndarray:
+    """Philox4x32 with 10 rounds (Salmon et al., "Parallel random numbers: as easy as 1, 2, 3", 2011),
+    the counter-based generator of device random streams.  ctr: [..., 4] uint32 counters; returns the
+    [..., 4] uint32 outputs."""
+    c = [np.asarray(ctr[..., i], dtype=np.uint64) for i in range(4)]
+    k0, k1 = int(key[0]) & 0xFFFFFFFF, int(key[1]) & 0xFFFFFFFF
+    mask, sh = np.uint64(0xFFFFFFFF), np.uint64(32)
+    for _ in range(10):
+        p0, p1 = _PHILOX_M0 * c[0], _PHILOX_M1 * c[2]
+        c = [(p1 >> sh) ^ c[1] ^ np.uint64(k0), p1 & mask, (p0 >> sh) ^ c[3] ^ np.uint64(k1), p0 & mask]
+        k0, k1 = (k0 + _PHILOX_W0) & 0xFFFFFFFF, (k1 + _PHILOX_W1) & 0xFFFFFFFF
+    return np.stack(c, axis=-1).astype(np.uint32)
+
+
+def device_noise(seed: int, stream_id: int, frame0: int, n_frames: int, mel: int) -> np.ndarray:
+    """The Euler noise x_0 of frames frame0 .. frame0 + n_frames - 1 when the decoder draws it itself:
+    the draw of (frame t, channels 4g .. 4g+3) is Philox4x32-10 at counter (t mod 2^32, t div 2^32, g,
+    stream id) under the key (seed mod 2^32, seed div 2^32) - the generator's offset is the stream's frame
+    clock (Sec. 3.3, effect classification) - turned into four standard normals by two Box-Muller
+    pairs on u = ((r >> 8) + 1/2) 2^-24."""
+    t = np.arange(frame0, frame0 + n_frames, dtype=np.int64)[:, None]
+    g = np.arange(mel // 4, dtype=np.int64)[None, :]
+    ctr = np.stack(np.broadcast_arrays(t & 0xFFFFFFFF, t >> 32, g, np.int64(stream_id)), axis=-1).astype(np.uint32)
+    r = philox4x32_10(ctr, (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)).astype(np.float64)
+    u = (np.floor(r / 256.0) + 0.5) / 16777216.0
+    rad0, rad1 = np.sqrt(-2.0 * np.log(u[..., 0])), np.sqrt(-2.0 * np.log(u[..., 2]))
+    a0, a1 = 2.0 * np.pi * u[..., 1], 2.0 * np.pi * u[..., 3]
+    z = np.stack([rad0 * np.cos(a0), rad0 * np.sin(a0), rad1 * np.cos(a1), rad1 * np.sin(a1)], axis=-1)
+    return z.reshape(n_frames, mel)
+
+
 def attended_frames(cfg, lo: int, hi: int) -> np.ndarray:
     """Frames whose keys/values the chunk [lo, hi) attends (Sec. 3.1 "Two extents", Eq. 4): the
     prompt - the stream's first f_prompt frames, never evicted - then the last <= kv_cap frames of
@@ -238,7 +273,7 @@ def attended_frames(cfg, lo: int, hi: int) -> np.ndarray:
     return np.concatenate([prompt, history, own]).astype(np.int64)
 
 
-def flow_offline(cfg, blob, feats: np.ndarray, boundaries: Sequence[int]) -> np.ndarray:
+def flow_offline(cfg, blob, feats: np.ndarray, boundaries: Sequence[int], stream_id: int = 0) -> np.ndarray:
     """Offline causal run over the concatenated input.  feats[:, :mel] is the
     conditioning mu, feats[:, mel:] the initial noise x_0.  For s in 0..n-1:
     h = [x_s | mu] W_in + b_in; conv blocks h <- h + SiLU(conv(h) + b + tau_{s,l});
@@ -249,8 +284,11 @@ def flow_offline(cfg, blob, feats: np.ndarray, boundaries: Sequence[int]) -> np.
     rb = round_bf16 if cfg.precision == "bf16" else (lambda a: a)
     m, n = cfg.mel_dim, cfg.n_steps
     feats = np.asarray(feats, dtype=np.float64)
-    mu, x = feats[:, :m], feats[:, m:].copy()
     F = feats.shape[0]
+    if getattr(cfg, "noise_seed", 0):
+        mu, x = feats, device_noise(cfg.noise_seed, stream_id, 0, F, m)
+    else:
+        mu, x = feats[:, :m], feats[:, m:].copy()
     assert boundaries[0] == 0 and boundaries[-1] == F
     tau = tau_table(cfg, W)
     plan = _layer_plan(cfg)
@@ -379,8 +417,9 @@ class FlowStream:
     last 2d block-input frames; per attention layer the keys/values of the last
     <= W frames (empty at stream start)."""
 
-    def __init__(self, cfg, blob, carry: str = "concat"):
+    def __init__(self, cfg, blob, carry: str = "concat", stream_id: int = 0):
         self.cfg = cfg
+        self.stream_id = stream_id            # selects the stream's device random stream (noise_seed != 0)
         self.W = parse_blob(cfg, blob)
         self.tau = tau_table(cfg, self.W)
         self.plan = _layer_plan(cfg)
@@ -414,7 +453,10 @@ class FlowStream:
         # frames - output, conv left context and K/V carry - and the caller presents the others again.
         self.Tc = min(T, cfg.f_chunk)
         m, n = cfg.mel_dim, cfg.n_steps
-        mu, x = feats[:, :m], feats[:, m:].copy()
+        if getattr(cfg, "noise_seed", 0):
+            mu, x = feats, device_noise(cfg.noise_seed, self.stream_id, self.frames, T, m)   # look-ahead frames draw again next call
+        else:
+            mu, x = feats[:, :m], feats[:, m:].copy()
         for s in range(n):
             vel = self._velocity(s, x, mu, 0, rb)
             if self.w_cfg > 0:

@@ -33,7 +33,8 @@ class dc_config(C.Structure):
                 ("up_channels", C.c_int32 * (DC_MAX_UP + 1)), ("n_res", C.c_int32),
                 ("res_dilations", C.c_int32 * DC_MAX_RES), ("n_fft", C.c_int32), ("hop", C.c_int32),
                 ("rms_eps", C.c_float), ("logmag_clamp", C.c_float), ("max_batch", C.c_int32),
-                ("f_prompt", C.c_int32), ("f_lookahead", C.c_int32), ("cfg_scale", C.c_float)]
+                ("f_prompt", C.c_int32), ("f_lookahead", C.c_int32), ("noise_seed_lo", C.c_uint32), ("noise_seed_hi", C.c_uint32),
+                ("cfg_scale", C.c_float)]
 
 
 class DCError(RuntimeError):
@@ -114,6 +115,8 @@ def make_config(cfg, max_batch: int = 1) -> dc_config:
     c.cfg_scale = float(getattr(cfg, "cfg_scale", 0.0))
     c.f_prompt = int(getattr(cfg, "f_prompt", 0))
     c.f_lookahead = int(getattr(cfg, "f_lookahead", 0))
+    seed = int(getattr(cfg, "noise_seed", 0))
+    c.noise_seed_lo, c.noise_seed_hi = seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF
     return c
 
 

@@ -114,6 +114,7 @@ static dc_config sub_config(const dc_config& c, int pipeline) {
     s.cfg_scale = 0.f;
     s.f_prompt = 0;
     s.f_lookahead = 0;
+    s.noise_seed_lo = s.noise_seed_hi = 0;
   }
   return s;
 }
@@ -127,6 +128,7 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (!(c->cfg_scale >= 0.f && c->cfg_scale <= 100.f)) BAD("cfg_scale out of range");
   if (c->f_prompt < 0 || c->f_prompt > 4096) BAD("f_prompt out of range");
   if (c->f_lookahead < 0 || c->f_lookahead > 32) BAD("f_lookahead out of range");
+  if ((c->noise_seed_lo | c->noise_seed_hi) != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("noise_seed belongs to the flow decoder");
   if (c->f_lookahead != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_lookahead belongs to the flow decoder");
   if (c->f_prompt != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_prompt belongs to the flow decoder");
   if (c->cfg_scale != 0.f && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("cfg_scale belongs to the flow decoder");
@@ -282,7 +284,7 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     }
   } else if (cfg->pipeline == DC_PIPE_FLOW) {
     st = dc::flow_model_create(*cfg, w, &m->flow);
-    m->in_dim = 2 * cfg->mel_dim;
+    m->in_dim = (cfg->noise_seed_lo | cfg->noise_seed_hi) ? cfg->mel_dim : 2 * cfg->mel_dim;   // [mu | x_0], or mu alone
     m->out_per_frame = cfg->mel_dim;
     if (st == DC_OK) {
       const size_t ni = (size_t)cfg->max_batch * (cfg->f_chunk + cfg->f_lookahead) * m->in_dim,
@@ -490,6 +492,7 @@ struct dc_snapshot {
   void*     data = nullptr;          // the carry buffers, back to back, in dc_stream_carry_info order
   size_t    bytes = 0;
   long long frames_total = 0, chunks = 0, flow_frames = 0;
+  int       rng_id = 0;
   dc_snapshot* sub_flow = nullptr;   // DC_PIPE_TOKEN2WAV: the two halves
   dc_snapshot* sub_voc = nullptr;
 };
@@ -531,7 +534,10 @@ extern "C" dc_status dc_stream_snapshot(dc_stream* s, dc_snapshot** out, void* c
     st = dc_stream_snapshot(s->sub_flow, &sn->sub_flow, cuda_stream);
     if (st == DC_OK) st = dc_stream_snapshot(s->sub_voc, &sn->sub_voc, cuda_stream);
   } else {
-    if (s->flow) sn->flow_frames = dc::flow_state_frames(s->flow);
+    if (s->flow) {
+      sn->flow_frames = dc::flow_state_frames(s->flow);
+      sn->rng_id = dc::flow_state_rng_id(s->flow);
+    }
     const std::vector<DevBuf> bufs = carry_buffers(s);
     for (const DevBuf& b : bufs) sn->bytes += b.bytes;
     cudaError_t e = cudaMalloc(&sn->data, sn->bytes ? sn->bytes : 1);
@@ -573,7 +579,10 @@ extern "C" dc_status dc_stream_restore(dc_stream* s, const dc_snapshot* sn, void
       DC_CUDA(cudaMemcpyAsync(b.p, (const char*)sn->data + off, b.bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream));
       off += b.bytes;
     }
-    if (s->flow) dc::flow_state_set_frames(s->flow, sn->flow_frames);
+    if (s->flow) {
+      dc::flow_state_set_frames(s->flow, sn->flow_frames);
+      dc::flow_state_set_rng_id(s->flow, sn->rng_id);   // the session keeps its random stream wherever it lives
+    }
   }
   s->frames_total = sn->frames_total;
   s->chunks = sn->chunks;

@@ -60,6 +60,9 @@ struct SlotInfo {
   bf16*        halo;      // stream carry: [n_steps][n_conv][8][C]
   bf16*        kv;        // stream carry: [n_steps][n_attn][2][P + Rk][C] (P prompt rows, then the history ring)
   int          n_prompt0; // prompt rows present before this chunk (<= P); the chunk's first P - n_prompt0 frames join them
+  long long    frame0;    // index of the chunk's first frame in the stream (the frame clock)
+  int          rng_id;    // the stream's device random stream
+  int          pad;
   int          Tc;        // committed frames (<= T): the others are look-ahead - computed and attended, but neither output
                           // nor carried (their K/V rows are written past the ring head and overwritten by the next call)
 };
@@ -294,7 +297,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int r = m0 + q * 32 + lane;             // row in slot layout (without GUARD)
     const int slot = r / SLOT_ROWS, rho = r % SLOT_ROWS;
     const bool in_range = slot < p.n_slots;
-    const SlotInfo si = in_range ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, 0, 0};
+    const SlotInfo si = in_range ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 0, 0};
     const int f = rho - HALO;
     const bool do_halo = p.halo_off >= 0;
     const bool has_resid = p.mode == MODE_CONV || p.mode == MODE_OPROJ;
@@ -561,19 +564,57 @@ __global__ void set_slots_kernel(const SlotSet set, SlotInfo* dst) {
   if (i < set.count) dst[set.first + i] = set.s[i];
 }
 
-// feats [T][2 mel] -> Euler state x_0 (fp32) and the bf16 input-projection operand [x_0 | mu].
-__global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, bf16* ain, int ld_ain) {
+// Philox4x32-10 (Salmon et al. 2011): ten rounds of two 32 x 32 -> 64 multiplications and a key bump.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1, uint32_t* out) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// feats [T][2 mel] (or [T][mel] when the noise is drawn here) -> Euler state x_0 (fp32) and the bf16
+// input-projection operand [x_0 | mu].  Device noise: the draw of (frame t, channels 4g..4g+3) is Philox at
+// counter (t, g, stream) under the model's seed - the offset is the stream's frame clock, so a replayed graph
+// draws what direct launches would, and a look-ahead frame draws the same noise when it is presented again.
+__global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, bf16* ain, int ld_ain, uint32_t seed_lo, uint32_t seed_hi) {
   ptx::pdl_launch();
   ptx::pdl_wait();
   const SlotInfo si = slots[blockIdx.x];
-  for (int i = threadIdx.x; i < si.T * mel; i += blockDim.x) {
-    const int f = i / mel, c = i - f * mel;
+  const bool draw = (seed_lo | seed_hi) != 0u;
+  const int fw = draw ? mel : 2 * mel;       // width of a row of feats
+  for (int i = threadIdx.x; i < si.T * (mel / 4); i += blockDim.x) {
+    const int f = i / (mel / 4), g = i - f * (mel / 4);
     const long long r = (long long)blockIdx.x * SLOT_ROWS + HALO + f;
-    const float mu = si.pass == 0 ? si.feats[(long long)f * 2 * mel + c] : 0.f;
-    const float x0 = si.feats[(long long)f * 2 * mel + mel + c];
-    xstate[r * mel + c] = x0;
-    ain[(GUARD + r) * ld_ain + c] = __float2bfloat16_rn(x0);
-    ain[(GUARD + r) * ld_ain + mel + c] = __float2bfloat16_rn(mu);
+    float x0[4];
+    if (draw) {
+      const unsigned long long t = (unsigned long long)(si.frame0 + f);
+      uint32_t w[4];
+      philox4x32_10((uint32_t)t, (uint32_t)(t >> 32), (uint32_t)g, (uint32_t)si.rng_id, seed_lo, seed_hi, w);
+      const float u0 = ((float)(w[0] >> 8) + 0.5f) * (1.0f / 16777216.0f), u1 = ((float)(w[1] >> 8) + 0.5f) * (1.0f / 16777216.0f);
+      const float u2 = ((float)(w[2] >> 8) + 0.5f) * (1.0f / 16777216.0f), u3 = ((float)(w[3] >> 8) + 0.5f) * (1.0f / 16777216.0f);
+      const float ra = sqrtf(-2.0f * logf(u0)), rb = sqrtf(-2.0f * logf(u2));
+      float sa, ca, sb, cb;
+      sincosf(6.283185307179586f * u1, &sa, &ca);
+      sincosf(6.283185307179586f * u3, &sb, &cb);
+      x0[0] = ra * ca; x0[1] = ra * sa; x0[2] = rb * cb; x0[3] = rb * sb;
+    } else {
+      const float4 v = *reinterpret_cast<const float4*>(si.feats + (long long)f * fw + mel + 4 * g);
+      x0[0] = v.x; x0[1] = v.y; x0[2] = v.z; x0[3] = v.w;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c = 4 * g + j;
+      const float mu = si.pass == 0 ? si.feats[(long long)f * fw + c] : 0.f;
+      xstate[r * mel + c] = x0[j];
+      ain[(GUARD + r) * ld_ain + c] = __float2bfloat16_rn(x0[j]);
+      ain[(GUARD + r) * ld_ain + mel + c] = __float2bfloat16_rn(mu);
+    }
   }
 }
 
@@ -1027,6 +1068,7 @@ struct GraphEntry {
 struct FlowModel {
   dc_config cfg;
   int C = 0, mel = 0, Kin = 0, S = 0, rows = 0, Rk = 0, cpa = 0;   // S: slots (streams x passes) of a full batch
+  int streams_opened = 0;    // so far: the next stream's random-stream index
   int P = 0;                 // prompt rows in front of every K/V ring
   int n_pass = 1;            // 2 with classifier-free guidance: a stream's conditional and unconditional pass are
                              // adjacent slots, i.e. the two halves of one row tile
@@ -1064,6 +1106,7 @@ struct FlowState {
   bf16* kv = nullptr;
   size_t halo_bytes = 0, kv_bytes = 0;
   long long frames = 0;     // frames appended so far (drives ring head and carried length)
+  int       rng_id = 0;     // index of the stream's device random stream
 };
 
 namespace {
@@ -1284,6 +1327,7 @@ dc_status flow_state_open(FlowModel* m, FlowState** out) {
   FlowState* s = new (std::nothrow) FlowState();
   if (!s) return DC_ERR_OOM;
   s->m = m;
+  s->rng_id = m->streams_opened++;   // (a plain counter: streams of one model are opened from one thread at a time)
   const dc_config& c = m->cfg;
   // one set of carries per pass
   s->halo_bytes = (size_t)m->n_pass * c.n_steps * c.n_conv * HALO * m->C * sizeof(bf16);
@@ -1312,6 +1356,8 @@ void flow_state_buffers(const FlowState* s, DevBuf* out, int max_entries, int* n
 
 long long flow_state_frames(const FlowState* s) { return s->frames; }
 void flow_state_set_frames(FlowState* s, long long frames) { s->frames = frames; }
+int flow_state_rng_id(const FlowState* s) { return s->rng_id; }
+void flow_state_set_rng_id(FlowState* s, int id) { s->rng_id = id; }
 
 dc_status flow_state_reset(FlowModel*, FlowState* s, cudaStream_t st) {
   // base state: zero left context, empty K/V carry (stale ring rows are never attended)
@@ -1401,7 +1447,8 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
   const int C = m->C, mel = m->mel;
   for (int i = 0; i < n_sets; ++i)   // not a programmatic launch: it overwrites the table the previous chunk still reads
     launch(lc, set_slots_kernel, dim3(1), dim3(MAX_SLOTS_PER_SET), 0, false, 4, sets[i], m->d_slots);
-  launch(lc, flow_prep_kernel, dim3(n), dim3(128), 0, true, 4, (const SlotInfo*)m->d_slots, mel, m->xstate, m->Ain, m->Kin);
+  launch(lc, flow_prep_kernel, dim3(n), dim3(128), 0, true, 4, (const SlotInfo*)m->d_slots, mel, m->xstate, m->Ain, m->Kin,
+         (uint32_t)c.noise_seed_lo, (uint32_t)c.noise_seed_hi);
 
   const int m_tiles = (n * SLOT_ROWS + TILE_M - 1) / TILE_M;
   // N-tile variant: the widest whose C-wide GEMMs still give about 96 CTAs, else the narrowest
@@ -1592,6 +1639,9 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       si.kv_head = (int)(hist % m->Rk);
       si.kv_len = (int)(hist < c.kv_cap ? hist : c.kv_cap);
       si.Tc = si.T < c.f_chunk ? si.T : c.f_chunk;
+      si.frame0 = s->frames;
+      si.rng_id = s->rng_id;
+      si.pad = 0;
       si.pass = pass;
       si.feats = feats[stream];
       si.out = pass == 0 ? outp[stream] : nullptr;

@@ -105,6 +105,8 @@ dc_status flow_state_open(FlowModel* m, FlowState** out);
 void      flow_state_buffers(const FlowState* s, DevBuf* out, int max_entries, int* n);
 long long flow_state_frames(const FlowState* s);              // the stream's frame clock (committed frames)
 void      flow_state_set_frames(FlowState* s, long long frames);
+int       flow_state_rng_id(const FlowState* s);               // which device random stream the session draws from
+void      flow_state_set_rng_id(FlowState* s, int id);
 dc_status flow_state_reset(FlowModel* m, FlowState* s, cudaStream_t st);
 void      flow_state_close(FlowState* s);
 // Reads (and clears) the device-side error word that bounded waits set; synchronous.  0 = no timeout.

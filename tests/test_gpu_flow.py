@@ -229,3 +229,43 @@ def test_paper_operating_point_full(dc):
     cfg = wl.EXTRA_CONFIGS["cfg3_paper"].replace(n_chunks=13)
     bounds = [0, 50, 100, 150, 200, 250, 300, 302, 352, 402, 452, 502, 552, 602]
     _parity(dc, cfg, boundaries=bounds)
+
+
+# ---- device-drawn Euler noise (Philox keyed by the stream's frame clock) ----
+
+def _noise_run(dc, m, cfg, w, s, stream_id):
+    gu = _gu()
+    got = gu.run_gpu_stream(m, s.feats, s.boundaries)          # opens the model's next stream
+    ref = orc.run_stream(cfg, w.weights, s.feats, s.boundaries, stream_id=stream_id)
+    err = gu.rel_err(got, ref)
+    assert err <= TOL_BF16, f"{cfg.name} stream {stream_id}: {err}"
+    return got
+
+
+def test_device_noise_per_stream_and_replay(dc):
+    import os
+    cfg = wl.tiny_flow(noise_seed=0x1234567890ABCDEF, n_chunks=len(RAGGED) - 1)
+    w = wl.make_workload(cfg, boundaries=[RAGGED])
+    s = w.streams[0]
+    assert s.feats.shape[1] == cfg.mel_dim                      # the input is the conditioning alone
+    m = dc.Model(cfg, w.weights)
+    a = _noise_run(dc, m, cfg, w, s, 0)
+    b = _noise_run(dc, m, cfg, w, s, 1)                         # the model's second stream draws another sequence
+    assert not np.array_equal(a, b)
+    m.destroy()
+    # a model that launches its kernels directly (no captured graph) draws exactly the same
+    os.environ["DC_NO_GRAPH"] = "1"
+    try:
+        m2 = dc.Model(cfg, w.weights)
+    finally:
+        os.environ.pop("DC_NO_GRAPH", None)
+    assert np.array_equal(_noise_run(dc, m2, cfg, w, s, 0), a)
+    m2.destroy()
+
+
+def test_device_noise_with_lookahead_prompt_and_guidance(dc):
+    cfg = wl.tiny_flow(noise_seed=77, f_lookahead=3, f_prompt=17, cfg_scale=0.7, n_chunks=len(LA_BOUNDS) - 1)
+    w = wl.make_workload(cfg, boundaries=[LA_BOUNDS])
+    m = dc.Model(cfg, w.weights)
+    _noise_run(dc, m, cfg, w, w.streams[0], 0)
+    m.destroy()

@@ -24,6 +24,8 @@ def _chunks(st, x, bounds, lo, hi):
 
 
 @pytest.mark.parametrize("make", [lambda: wl.tiny_flow(n_chunks=8, f_prompt=9, cfg_scale=0.7),
+                                  lambda: wl.tiny_flow(n_chunks=8, noise_seed=5),     # the session keeps its random stream
+
                                   lambda: wl.tiny_vocoder(n_chunks=8),
                                   lambda: wl.CONFIGS["cfg1"],
                                   lambda: wl.tiny_token2wav(n_chunks=8)])

@@ -544,3 +544,40 @@ def test_lookahead_frames_pins():
         attended.append(st.kv_len_seen[-1] + (hi - pb[c]))
     assert st.kv_len_seen[7:] == [302, 352, 402, 402, 402]
     assert max(attended) == 458
+
+
+def test_philox_known_answers_and_device_noise():
+    """The counter-based generator of the device-drawn Euler noise: the published known-answer vectors of
+    Philox4x32-10 (Random123 test suite), the moments of the normals built from it, and its keying: the
+    draw depends on (seed, stream, frame, channel) only, so chunking cannot change it."""
+    kat = [((0, 0, 0, 0), (0, 0), (0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8)),
+           ((0xffffffff,) * 4, (0xffffffff,) * 2, (0x408f276d, 0x41c83b0e, 0xa20bc7c6, 0x6d5451fd)),
+           ((0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344), (0xa4093822, 0x299f31d0),
+            (0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1))]
+    for ctr, key, want in kat:
+        got = orc.philox4x32_10(np.array(ctr, dtype=np.uint32), key)
+        assert tuple(int(x) for x in got) == want
+    z = orc.device_noise(20240607, 1, 0, 20000, 16)
+    assert abs(z.mean()) < 0.01 and abs(z.std() - 1.0) < 0.01
+    assert abs(np.mean(z ** 3)) < 0.03 and abs(np.mean(z ** 4) - 3.0) < 0.1          # skewness 0, kurtosis 3
+    assert abs(np.corrcoef(z[:-1].ravel(), z[1:].ravel())[0, 1]) < 0.01              # frame to frame
+    assert abs(np.corrcoef(z[:, 0], z[:, 1])[0, 1]) < 0.02                           # both halves of a Box-Muller pair
+    assert np.array_equal(orc.device_noise(7, 2, 100, 50, 16), orc.device_noise(7, 2, 0, 150, 16)[100:])
+    assert not np.array_equal(orc.device_noise(7, 2, 0, 8, 16), orc.device_noise(7, 3, 0, 8, 16))
+    assert not np.array_equal(orc.device_noise(7, 2, 0, 8, 16), orc.device_noise(8, 2, 0, 8, 16))
+    # the decoder in device-noise mode: chunk loop == offline run, for any partition, also with look-ahead
+    cfg = wl.tiny_flow(noise_seed=99, n_chunks=7)
+    assert cfg.in_dim == cfg.mel_dim
+    bounds = [0, 3, 13, 14, 24, 31, 41, 51]
+    wk = wl.make_workload(cfg, boundaries=[bounds])
+    s = wk.streams[0]
+    off = orc.run_offline(cfg, wk.weights, s.feats, bounds)
+    st = orc.run_stream(cfg, wk.weights, s.feats, bounds)
+    assert np.allclose(st, off, rtol=0, atol=1e-9 * np.abs(off).max())
+    assert not np.allclose(st, orc.run_stream(cfg, wk.weights, s.feats, bounds, stream_id=1), atol=1e-3)
+    la = wl.tiny_flow(noise_seed=99, f_lookahead=3, n_chunks=6)
+    lb = [0, 10, 20, 30, 33, 43, 50]
+    wk = wl.make_workload(la, boundaries=[lb])
+    a = orc.run_stream(la, wk.weights, wk.streams[0].feats, lb)
+    b = orc.run_stream(la, wk.weights, wk.streams[0].feats, lb, carry="ring")
+    assert np.allclose(a, b, rtol=0, atol=1e-9 * np.abs(a).max())
