@@ -38,7 +38,7 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 HISTORY_CHUNKS = 12      # untimed stream history so that the K/V carry sits at its cap (steady state)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for that workload)
-NCU_TRAFFIC_BYTES = {"cfg5": 4.03e6,   # conv-mode flow_gemm_kernel, profiles/flow_gemm_kernel_conv_cfg5.md
+NCU_TRAFFIC_BYTES = {"cfg5": 4.00e6,   # conv-mode flow_gemm_kernel, profiles/flow_gemm_kernel_conv_cfg5.md
                      "cfg3": None, "cfg2": None, "cfg4": None, "cfg1": None}
 
 

@@ -162,13 +162,15 @@ dc_status dc_stream_reset(dc_stream* stream, void* cuda_stream);
 dc_status dc_stream_close(dc_stream* stream);
 
 /* One chunk of one stream.
- *   feats_dev : device fp32 [n_frames][F_in]; F_in = hidden (conv), 2*mel_dim (flow:
- *               cols [0,mel) conditioning, [mel,2 mel) initial noise), mel_dim (vocoder)
- *   out_dev   : device fp32; conv: [n_frames][hidden]; flow: [n_frames][mel_dim];
- *               vocoder: n_frames * prod(up_strides) * hop PCM samples
+ *   feats_dev : device fp32 [n_frames][F_in]; F_in = hidden (conv), 2*mel_dim (flow and token2wav:
+ *               cols [0,mel) conditioning, [mel,2 mel) initial noise; mel_dim - the conditioning
+ *               alone - when the model draws the noise itself, see noise_seed), mel_dim (vocoder)
+ *   out_dev   : device fp32; conv: [n_frames][hidden]; flow: [committed frames][mel_dim];
+ *               vocoder and token2wav: committed frames * prod(up_strides) * hop PCM samples
  *   n_out     : host pointer (may be NULL) receiving the number of floats written
- * Fails with DC_ERR_FRAMES unless 1 <= n_frames <= f_chunk; a failed call leaves
- * the stream untouched.  Allocates nothing. */
+ * Fails with DC_ERR_FRAMES unless 1 <= n_frames <= f_chunk + f_lookahead; a failed call leaves
+ * the stream untouched.  The call commits min(n_frames, f_chunk) frames (see f_lookahead; all of
+ * them when f_lookahead = 0).  Allocates nothing. */
 dc_status dc_decode_chunk(dc_stream* stream, const float* feats_dev, int n_frames,
                           float* out_dev, int* n_out, void* cuda_stream);
 
@@ -177,7 +179,8 @@ dc_status dc_decode_chunk(dc_stream* stream, const float* feats_dev, int n_frame
  * out_dev[i].  feats_dev, n_frames and out_dev are HOST arrays (of device
  * pointers / ints).  Results are bitwise identical to n single dc_decode_chunk
  * calls.  (Multi-session serving over shared weights with per-session state:
- * paper Section 3.4, last paragraph, and Section 4.3 "Serving capacity".)  Flow pipeline only. */
+ * paper Section 3.4, last paragraph, and Section 4.3 "Serving capacity".)  Flow and token2wav
+ * pipelines. */
 dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
                           const float* const* feats_dev, const int* n_frames,
                           float* const* out_dev, void* cuda_stream);
@@ -204,7 +207,8 @@ dc_status dc_decode_batch_host(dc_model* model, int n, dc_stream* const* streams
  * bracketed by CUDA events on the launching stream (this slows the step down: never report
  * throughput from a profiled pass).  dc_profile_end synchronises the device and returns, per
  * class, the summed milliseconds and the launch count.  Classes: 0 conv GEMM, 1 other GEMMs
- * (input/QKV/output projections), 2 attention, 3 RMS norm, 4 slot table + input prep,
+ * (input/QKV/output projections), 2 attention, 3 unused (the RMS norm is folded into the GEMMs),
+ * 4 slot table + input prep,
  * 5 fp32 tap convolution, 6 fp32 head + inverse STFT.
  * max_launches bounds the event pool allocated by dc_profile_begin. */
 dc_status dc_profile_begin(dc_model* model, int max_launches);
