@@ -185,6 +185,23 @@ dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
                           const float* const* feats_dev, const int* n_frames,
                           float* const* out_dev, void* cuda_stream);
 
+/* Offline decoding of one stream whose remaining input is all there: the n_frames frames are cut
+ * into consecutive chunks of f_chunk frames (the last one shorter), each attending its f_lookahead
+ * following frames where they exist, and decoded as a WAVEFRONT: chunk j runs Euler step s of the
+ * flow decoder (Section 3.1's per-chunk loop) in pass j + s of the network, so that n_steps chunks
+ * are in flight at once, one per step, as the slots of one launch.  Chunk j's step s needs only the
+ * step-s carries that chunk j-1 left one pass earlier, so the result - and the stream's carries
+ * afterwards - are bitwise those of the same chunks given to dc_decode_chunk one by one.
+ *   feats_dev : device fp32 [n_frames][F_in] (as for dc_decode_chunk)
+ *   out_dev   : device fp32; flow: [n_frames][mel_dim]; token2wav: n_frames * out_per_frame samples
+ *   n_out     : host pointer (may be NULL) receiving the number of floats written
+ * Flow and token2wav pipelines; the model must have been created with max_batch >= n_steps
+ * (DC_ERR_ARG otherwise, stream untouched).  The token2wav composite keeps the call's mel frames
+ * in a device buffer owned by the stream, which this call (re)allocates when n_frames exceeds
+ * every earlier call's; the flow pipeline allocates nothing. */
+dc_status dc_decode_wavefront(dc_stream* stream, const float* feats_dev, long long n_frames,
+                              float* out_dev, long long* n_out, void* cuda_stream);
+
 /* Convenience for callers with host buffers: copies feats_host to the device,
  * decodes, copies the result back and synchronises cuda_stream.  Uses staging
  * buffers owned by the stream (allocated at dc_stream_open).  Returns DC_ERR_TIMEOUT

@@ -21,7 +21,8 @@ EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_
            "dc_stream_close", "dc_decode_chunk", "dc_decode_batch", "dc_decode_chunk_host",
            "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error",
            "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end", "dc_conv_stack_noalloc",
-           "dc_selftest_bounded_wait", "dc_stream_snapshot", "dc_stream_restore", "dc_snapshot_free"]
+           "dc_selftest_bounded_wait", "dc_stream_snapshot", "dc_stream_restore", "dc_snapshot_free",
+           "dc_decode_wavefront"]
 
 
 class dc_config(C.Structure):
@@ -69,6 +70,7 @@ def load_library():
     lib.dc_stream_close.argtypes = [vp]
     lib.dc_decode_chunk.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
     lib.dc_decode_batch.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
+    lib.dc_decode_wavefront.argtypes = [vp, vp, C.c_longlong, vp, cp(C.c_longlong), vp]
     lib.dc_decode_chunk_host.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
     lib.dc_decode_batch_host.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
     lib.dc_profile_begin.argtypes = [vp, C.c_int]
@@ -207,6 +209,23 @@ class Stream:
         res = out[: n_out.value]
         if self.model.cfg.pipeline not in ("vocoder", "token2wav"):
             res = res.view(-1, self.model.out_per_frame)      # committed frames (fewer than T when the call carried look-ahead frames)
+        return res
+
+    def decode_wavefront(self, feats, out=None, stream=None):
+        """dc_decode_wavefront: feats is a CUDA float32 tensor [n_frames, in_dim] holding all the stream's
+        remaining input; returns what the chunk-by-chunk calls would have returned, concatenated."""
+        import torch
+        assert feats.is_cuda and feats.dtype == torch.float32 and feats.is_contiguous()
+        n = feats.shape[0]
+        if out is None:
+            out = torch.empty(n * self.model.out_per_frame, device=feats.device, dtype=torch.float32)
+        n_out = C.c_longlong(0)
+        st = self.lib.dc_decode_wavefront(self.handle, feats.data_ptr(), n, out.data_ptr(), C.byref(n_out),
+                                          _cuda_stream_handle(stream))
+        _check(st, "dc_decode_wavefront")
+        res = out[: n_out.value]
+        if self.model.cfg.pipeline not in ("vocoder", "token2wav"):
+            res = res.view(-1, self.model.out_per_frame)
         return res
 
     def decode_chunk_host(self, feats_host, out_host, stream=None) -> int:

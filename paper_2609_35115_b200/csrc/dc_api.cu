@@ -94,6 +94,8 @@ struct dc_stream {
   dc_stream* sub_flow = nullptr;   // DC_PIPE_TOKEN2WAV: the two halves' streams and the mel chunk between them
   dc_stream* sub_voc = nullptr;
   float*    mel = nullptr;         // [f_chunk][mel_dim] fp32, device
+  float*    wave_mel = nullptr;    // dc_decode_wavefront of the composite: all mel frames of one call (grown on demand)
+  long long wave_mel_frames = 0;
   float*    stage_in = nullptr;    // device staging of dc_decode_chunk_host
   float*    stage_out = nullptr;
   cudaGraph_t     g_graph = nullptr;   // fp32 pipelines: the captured chunk step
@@ -362,6 +364,8 @@ static void free_stream_buffers(dc_stream* s) {
   if (s->sub_flow) dc_stream_close(s->sub_flow);
   if (s->sub_voc) dc_stream_close(s->sub_voc);
   if (s->mel) cudaFree(s->mel);
+  if (s->wave_mel) cudaFree(s->wave_mel);
+  s->wave_mel = nullptr;
   s->sub_flow = s->sub_voc = nullptr;
   s->mel = nullptr;
   if (s->stage_in) cudaFree(s->stage_in);
@@ -755,6 +759,66 @@ extern "C" dc_status dc_decode_chunk(dc_stream* s, const float* feats, int T, fl
   m->counters[0] += 1;
   m->counters[1] += (uint64_t)Tc;
   if (n_out) *n_out = Tc * m->out_per_frame;
+  return DC_OK;
+}
+
+extern "C" dc_status dc_decode_wavefront(dc_stream* s, const float* feats, long long n_frames, float* out, long long* n_out,
+                                         void* cuda_stream) {
+  if (!s) return DC_ERR_ARG;
+  if (s->closed || s->poisoned) return DC_ERR_STATE;
+  dc_model* m = s->model;
+  if (!feats || !out || n_frames < 1) {
+    m->counters[3]++;
+    return DC_ERR_ARG;
+  }
+  if (!m->flow && !m->sub_flow) {
+    dc::set_error("dc_decode_wavefront serves the flow and token2wav pipelines only");
+    return DC_ERR_CONFIG;
+  }
+  cudaStream_t cs = (cudaStream_t)cuda_stream;
+  const int fc = m->cfg.f_chunk;
+  const long long n_chunks = (n_frames + fc - 1) / fc;
+  dc_status st = DC_OK;
+  if (m->sub_flow) {
+    // the flow decoder's wavefront leaves every mel frame of the call on the device, then the vocoder
+    // tail (whose chunk step has no Euler loop to pipeline) consumes them chunk by chunk
+    if (s->wave_mel_frames < n_frames) {
+      if (s->wave_mel) cudaFree(s->wave_mel);
+      s->wave_mel = nullptr;
+      s->wave_mel_frames = 0;
+      if (cudaMalloc(&s->wave_mel, (size_t)n_frames * m->cfg.mel_dim * sizeof(float)) != cudaSuccess) {
+        cudaGetLastError();
+        return DC_ERR_OOM;
+      }
+      s->wave_mel_frames = n_frames;
+    }
+    st = dc_decode_wavefront(s->sub_flow, feats, n_frames, s->wave_mel, nullptr, cuda_stream);
+    for (long long j = 0; j < n_chunks && st == DC_OK; ++j) {
+      const int T = (int)(n_frames - j * fc < fc ? n_frames - j * fc : fc);
+      st = dc_decode_chunk(s->sub_voc, s->wave_mel + j * fc * m->cfg.mel_dim, T, out + j * fc * m->out_per_frame, nullptr, cuda_stream);
+    }
+    if (st != DC_OK) {
+      s->poisoned = true;
+      return st;
+    }
+  } else {
+    int launches = 0;
+    st = dc::flow_decode_wave(m->flow, s->flow, feats, m->in_dim, n_frames, out, cs, &launches);
+    m->counters[5] += (uint64_t)launches;
+    if (st == DC_ERR_ARG) {   // refused before anything ran (max_batch < n_steps): the stream is untouched
+      m->counters[3]++;
+      return st;
+    }
+    if (st != DC_OK) {
+      s->poisoned = true;
+      return st;
+    }
+  }
+  s->frames_total += n_frames;
+  s->chunks += n_chunks;
+  m->counters[0] += (uint64_t)n_chunks;
+  m->counters[1] += (uint64_t)n_frames;
+  if (n_out) *n_out = n_frames * m->out_per_frame;
   return DC_OK;
 }
 

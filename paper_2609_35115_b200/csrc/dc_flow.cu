@@ -60,12 +60,17 @@ struct SlotInfo {
   bf16*        halo;      // stream carry: [n_steps][n_conv][8][C]
   bf16*        kv;        // stream carry: [n_steps][n_attn][2][P + Rk][C] (P prompt rows, then the history ring)
   int          n_prompt0; // prompt rows present before this chunk (<= P); the chunk's first P - n_prompt0 frames join them
-  long long    frame0;    // index of the chunk's first frame in the stream (the frame clock)
-  int          rng_id;    // the stream's device random stream
-  int          pad;
   int          Tc;        // committed frames (<= T): the others are look-ahead - computed and attended, but neither output
                           // nor carried (their K/V rows are written past the ring head and overwritten by the next call)
+  long long    frame0;    // index of the chunk's first frame in the stream (the frame clock)
+  int          rng_id;    // the stream's device random stream
+  // Wavefront decoding (several chunks of one stream in flight, each at an Euler step of its own): the slot's step
+  // is folded into its halo / kv pointers by the host; what remains per slot is the timestep-bias row and two flags.
+  int          tau_off;   // float offset of the slot's Euler step inside the timestep-bias table (0 when the launch's own step applies)
+  int          flags;     // SLOT_FIRST: the prep kernel loads x_0 and mu; SLOT_LAST: the output projection also writes `out`
+  int          pad;
 };
+constexpr int SLOT_FIRST = 1, SLOT_LAST = 2;
 
 struct SlotSet {
   int      first, count;
@@ -287,17 +292,18 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // per-column constants go to shared memory, the thread's residual row (or, for a left-context
     // row, the carried row) goes to registers.
     const int et = threadIdx.x - 128;
-    if (et < p.BN) {   // BN <= 192 < EPI_THREADS
-      s_bias[et] = p.bias[n0 + et];
-      s_tau[et] = p.tau != nullptr ? p.tau[n0 + et] : 0.f;
-    }
+    if (et < p.BN) s_bias[et] = p.bias[n0 + et];   // BN <= 192 < EPI_THREADS
     ptx::pdl_wait();                              // slot table, residual and carry rows are upstream data
+    if (p.tau != nullptr && et < 2 * p.BN) {      // conv blocks (BN <= 64): the timestep bias of each of the tile's two slots
+      const int sl = et / p.BN, c = et - sl * p.BN, ts = m0 / SLOT_ROWS + sl;
+      s_tau[sl * 64 + c] = ts < p.n_slots ? p.tau[p.slots[ts].tau_off + n0 + c] : 0.f;
+    }
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int cg = (warp - 4) >> 2;               // which chunks of the row: chunk index % EPI_GROUPS == cg
     const int r = m0 + q * 32 + lane;             // row in slot layout (without GUARD)
     const int slot = r / SLOT_ROWS, rho = r % SLOT_ROWS;
-    const bool in_range = slot < p.n_slots;
-    const SlotInfo si = in_range ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 0, 0};
+    const SlotInfo si = slot < p.n_slots ? p.slots[slot] : SlotInfo{0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, 0, 0, 0, 0, 0, 0, 0};
+    const bool in_range = si.T > 0;               // (a slot without frames - a hole in a wavefront - is left alone)
     const int f = rho - HALO;
     const bool do_halo = p.halo_off >= 0;
     const bool has_resid = p.mode == MODE_CONV || p.mode == MODE_OPROJ;
@@ -342,6 +348,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (threadIdx.x == 128) DC_T(4);
     if (!got) atomicCAS(p.err, 0, 3 | (p.mode << 8));
     const bool slot_ok = in_range && got && *s_fail == 0;
+    const float* tau_s = s_tau + ((q >> 1) & 1) * 64;   // rows 64.. of the tile are its second slot
     const bool is_halo = slot_ok && rho < HALO;
     const bool is_chunk = slot_ok && f >= 0 && f < si.T;
     const int new_row = rho - si.Tc;              // carry row this thread's value moves to (the carry follows the committed frames)
@@ -449,7 +456,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           pack16_bf16(xv, a, b);
           store16(p.ain + grow * p.ld_ain + n, a, b);
           if (p.cfg_w > 0.f) store16(p.ain + (grow + SLOT_ROWS) * p.ld_ain + n, a, b);   // the unconditional pass starts from the same x
-          if (p.last_step && f < si.Tc) {
+          if ((p.last_step || (si.flags & SLOT_LAST)) && f < si.Tc) {
             float* o = si.out + (long long)f * p.mel + n;
 #pragma unroll
             for (int i = 0; i < 16; i += 4)
@@ -489,8 +496,8 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (p.mode == MODE_CONV && !(p.dbg & 16)) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-              acc[2 * i] = __uint_as_float(w[i] << 16) + silu_f(acc[2 * i] + s_tau[c0 + 2 * i]);
-              acc[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u) + silu_f(acc[2 * i + 1] + s_tau[c0 + 2 * i + 1]);
+              acc[2 * i] = __uint_as_float(w[i] << 16) + silu_f(acc[2 * i] + tau_s[c0 + 2 * i]);
+              acc[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u) + silu_f(acc[2 * i + 1] + tau_s[c0 + 2 * i + 1]);
             }
           } else {
 #pragma unroll
@@ -586,6 +593,7 @@ __global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, 
   ptx::pdl_launch();
   ptx::pdl_wait();
   const SlotInfo si = slots[blockIdx.x];
+  if (!(si.flags & SLOT_FIRST)) return;      // (wavefront: this slot's chunk is past its first Euler step)
   const bool draw = (seed_lo | seed_hi) != 0u;
   const int fw = draw ? mel : 2 * mel;       // width of a row of feats
   for (int i = threadIdx.x; i < si.T * (mel / 4); i += blockDim.x) {
@@ -756,7 +764,9 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   const int L = PROMPT ? n_prompt + si.kv_len + (T - (n_prompt - si.n_prompt0)) : si.kv_len + T;
   const int nkb = (L + ATT_KB - 1) / ATT_KB;
 
-  if (warp >= 5) {
+  if (T == 0) {
+    // a slot without frames (a hole in a wavefront): nothing to do but to release tensor memory below
+  } else if (warp >= 5) {
     // ---------------- loaders ----------------
     const bool is_k = warp != 7;
     const int nl = is_k ? ATT_K_LOADERS : ATT_V_LOADERS;
@@ -1128,7 +1138,7 @@ void pack_wt(std::vector<uint16_t>& dst, size_t off, const float* W, int K, int 
 }  // namespace
 
 namespace {
-bool build_graph(FlowModel* m, int n);
+bool build_graph(FlowModel* m, int n, bool tick = false);
 }
 
 void flow_model_destroy(FlowModel* m) {
@@ -1442,7 +1452,9 @@ void launch(LaunchCtx& lc, void (*kernel)(KArgs...), dim3 grid, dim3 block, size
 
 // Issues every kernel of one chunk step for n slots (the slot table is uploaded by the first
 // kernel(s) from `sets`).
-void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchCtx& lc) {
+// tick = false: the n slots' chunks, all Euler steps.  tick = true: ONE pass of the network, every slot at the Euler step
+// that its slot-table entry encodes (wavefront decoding: the slots are consecutive chunks of one stream).
+void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchCtx& lc, bool tick = false) {
   const dc_config& c = m->cfg;
   const int C = m->C, mel = m->mel;
   for (int i = 0; i < n_sets; ++i)   // not a programmatic launch: it overwrites the table the previous chunk still reads
@@ -1502,7 +1514,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
   const float* fc = m->fconst;
   const long long halo_stride = (long long)HALO * C;
 
-  for (int s = 0; s < c.n_steps; ++s) {
+  for (int s = 0; s < (tick ? 1 : c.n_steps); ++s) {
     bf16* X = m->Xa;                 // current residual stream
     bf16* Y = m->Xb;
     const CUtensorMap* tX = &m->tmXa;
@@ -1558,7 +1570,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       p.mode = MODE_OUT; p.BN = bo; p.n_kblocks = C / KBLK; p.taps = 1;
       p.bias = fc + m->o_bout; p.halo_off = -1;
       p.xstate = m->xstate; p.ain = m->Ain; p.ld_ain = m->Kin; p.inv_n = 1.0f / c.n_steps;
-      p.last_step = (s == c.n_steps - 1); p.mel = mel; p.cfg_w = c.cfg_scale;
+      p.last_step = (!tick && s == c.n_steps - 1); p.mel = mel; p.cfg_w = c.cfg_scale;
       normalised(p);
       gemm(*tX, m->tmWout[v], p, mel);
     }
@@ -1567,7 +1579,8 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
 
 // One captured graph per batch size: the whole chunk step becomes a single graph launch; only the
 // slot-table node's by-value argument changes from call to call.
-bool build_graph(FlowModel* m, int n) {
+// Graphs are keyed by the slot count; tick graphs (one pass of the network, wavefront decoding) by its negative.
+bool build_graph(FlowModel* m, int n, bool tick) {
   if (n > MAX_SLOTS_PER_SET || m->cap_stream == nullptr) return false;
   for (int use_pdl = m->pdl ? 1 : 0; use_pdl >= 0; --use_pdl) {
     SlotSet dummy{};
@@ -1579,7 +1592,7 @@ bool build_graph(FlowModel* m, int n) {
       return false;
     }
     LaunchCtx lc{m->cap_stream, use_pdl != 0, nullptr};
-    enqueue_chunk(m, n, &dummy, 1, lc);
+    enqueue_chunk(m, n, &dummy, 1, lc, tick);
     cudaError_t e = cudaStreamEndCapture(m->cap_stream, &graph);
     if (e != cudaSuccess || lc.err != cudaSuccess || graph == nullptr) {
       cudaGetLastError();
@@ -1607,7 +1620,7 @@ bool build_graph(FlowModel* m, int n) {
     ge.graph = graph;
     ge.launches = lc.launches;
     ge.pdl = use_pdl != 0;
-    m->graphs[n] = ge;
+    m->graphs[tick ? -n : n] = ge;
     return true;
   }
   return false;
@@ -1641,6 +1654,8 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       si.Tc = si.T < c.f_chunk ? si.T : c.f_chunk;
       si.frame0 = s->frames;
       si.rng_id = s->rng_id;
+      si.tau_off = 0;
+      si.flags = SLOT_FIRST;
       si.pad = 0;
       si.pass = pass;
       si.feats = feats[stream];
@@ -1681,5 +1696,88 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
   for (int i = 0; i < n_streams; ++i) states[i]->frames += T[i] < c.f_chunk ? T[i] : c.f_chunk;
   return DC_OK;
 }
+
+// Wavefront decoding of ONE stream whose input is all there: chunk j runs its Euler step s in tick j + s,
+// so a tick is one pass of the network over n_steps consecutive chunks, each at its own step.  Chunk j at
+// step s needs the step-s carries that chunk j-1 left one tick earlier, and chunks that share a tick use the
+// carries of different steps, so every tick is free of read/write conflicts.  A chunk keeps slot
+// (j mod n_steps) for its n_steps ticks (its Euler state lives there); slots of chunks not yet started or already
+// finished are holes (T = 0).  The arithmetic of a slot never depends on what the other slots hold, so the
+// result equals chunk-by-chunk decoding bit for bit.
+dc_status flow_decode_wave(FlowModel* m, FlowState* s, const float* feats, int in_dim, long long n_frames, float* out,
+                           cudaStream_t st, int* launches) {
+  const dc_config& c = m->cfg;
+  const int np = m->n_pass, K = c.n_steps;
+  const int n = K * np;                                   // slots of a tick
+  if (n > m->S || n > MAX_SLOTS_PER_SET) {
+    set_error("wavefront decoding keeps n_steps = %d chunks in flight: max_batch must be >= n_steps", K);
+    return DC_ERR_ARG;
+  }
+  const long long n_chunks = (n_frames + c.f_chunk - 1) / c.f_chunk;
+  const bool profiling = m->prof != nullptr && m->prof->on;
+  auto it = m->graphs.find(-n);
+  if (it == m->graphs.end() && !profiling && build_graph(m, n, true)) it = m->graphs.find(-n);
+  const long long frames0 = s->frames;
+  const size_t halo_pass = s->halo_bytes / sizeof(bf16) / np, kv_pass = s->kv_bytes / sizeof(bf16) / np;
+  const size_t halo_step = (size_t)c.n_conv * HALO * m->C, kv_step = (size_t)c.n_attn * 2 * (m->P + m->Rk) * m->C;
+  SlotSet& set = m->sets[0];
+  for (long long t = 0; t < n_chunks + K - 1; ++t) {
+    set.first = 0;
+    set.count = n;
+    for (int i = 0; i < n; ++i) {
+      SlotInfo& si = set.s[i];
+      si = SlotInfo{};
+      const int ring = i / np, pass = i % np;
+      // the chunk that owns ring slot `ring` in tick t: the largest j <= t with j = ring (mod K)
+      const long long j = t - (((t - ring) % K) + K) % K;
+      const long long step = t - j;
+      if (j < 0 || j >= n_chunks || step >= K) continue;                  // hole
+      const long long f0 = j * c.f_chunk, left = n_frames - f0;
+      const long long frames = frames0 + f0;
+      si.T = (int)(left < c.f_chunk + c.f_lookahead ? left : c.f_chunk + c.f_lookahead);
+      si.Tc = si.T < c.f_chunk ? si.T : c.f_chunk;
+      const long long hist = frames > m->P ? frames - m->P : 0;
+      si.n_prompt0 = (int)(frames < m->P ? frames : m->P);
+      si.kv_head = (int)(hist % m->Rk);
+      si.kv_len = (int)(hist < c.kv_cap ? hist : c.kv_cap);
+      si.frame0 = frames;
+      si.rng_id = s->rng_id;
+      si.tau_off = (int)(step * c.n_conv * m->C);
+      si.flags = (step == 0 ? SLOT_FIRST : 0) | (step == K - 1 ? SLOT_LAST : 0);
+      si.pass = pass;
+      si.feats = feats + f0 * in_dim;
+      si.out = pass == 0 ? out + f0 * m->mel : nullptr;
+      si.halo = s->halo + (size_t)pass * halo_pass + (size_t)step * halo_step;
+      si.kv = s->kv ? s->kv + (size_t)pass * kv_pass + (size_t)step * kv_step : nullptr;
+    }
+    if (!profiling && it != m->graphs.end()) {
+      GraphEntry& ge = it->second;
+      void* args[2] = {&set, &m->d_slots};
+      cudaKernelNodeParams kp{};
+      kp.func = (void*)set_slots_kernel;
+      kp.gridDim = dim3(1);
+      kp.blockDim = dim3(MAX_SLOTS_PER_SET);
+      kp.kernelParams = args;
+      cudaError_t e = cudaGraphExecKernelNodeSetParams(ge.exec, ge.set_node, &kp);
+      if (e == cudaSuccess) e = cudaGraphLaunch(ge.exec, st);
+      if (e != cudaSuccess) {
+        set_error("wavefront graph launch failed: %s", cudaGetErrorString(e));
+        return DC_ERR_CUDA;
+      }
+      *launches += ge.launches;
+    } else {
+      LaunchCtx lc{st, m->pdl && !profiling, m->prof};
+      enqueue_chunk(m, n, &set, 1, lc, true);
+      *launches += lc.launches;
+      if (lc.err != cudaSuccess || cudaGetLastError() != cudaSuccess) {
+        set_error("wavefront launch failed: %s", cudaGetErrorString(lc.err));
+        return DC_ERR_CUDA;
+      }
+    }
+  }
+  s->frames = frames0 + n_frames;
+  return DC_OK;
+}
+
 
 }  // namespace dc
