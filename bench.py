@@ -358,6 +358,35 @@ def main():
     e2e_s = max_over_ranks(e2e_s, world)
     e2e_value = aggregate_throughput(world, S, K, per_chunk, e2e_s)
 
+    # ---- offline decoding of the same single stream as a wavefront (n_steps chunks in flight, one per
+    # Euler step; same bytes as the chunk-by-chunk calls): what the step costs when the input is all there ----
+    wave = None
+    if has_flow and S == 1 and world == 1:
+        n_wc = 200
+        mw = dc.Model(cfg, weights, max_batch=cfg.n_steps)
+        sw = mw.open_stream()
+        fw = torch.from_numpy(rng.standard_normal((n_wc * T, cfg.in_dim), dtype=np.float32)).cuda()
+        ow = torch.empty(n_wc * T * cfg.out_per_frame, device="cuda")
+        for _ in range(3):
+            sw.decode_wavefront(fw, out=ow)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        cw0 = mw.counters()
+        a.record()
+        n_calls = 3
+        for _ in range(n_calls):
+            sw.decode_wavefront(fw, out=ow)
+        b.record()
+        torch.cuda.synchronize()
+        cw1 = mw.counters()
+        ms_w = a.elapsed_time(b) / n_calls
+        wave = {"value": n_wc * per_chunk / (ms_w * 1e-3), "unit": unit, "ms_per_chunk": ms_w / n_wc,
+                "chunks_per_call": n_wc, "chunks_in_flight": cfg.n_steps, "calls_timed": n_calls,
+                "gpu_launches_per_call": int(cw1[5] - cw0[5]) // n_calls,
+                "note": "dc_decode_wavefront on one stream, input resident in HBM; includes the ramp-up and ramp-down passes"}
+        sw.close()
+        mw.destroy()
+
     # ---- per-kernel-class device time (separate profiled pass; events between launches slow the step) ----
     pk, how = peaks()
     nprof = min(K, 3)
@@ -464,6 +493,7 @@ def main():
             "latency_us": {"p50": 1e3 * step_ms[len(step_ms) // 2], "p95": 1e3 * step_ms[min(len(step_ms) - 1, int(0.95 * len(step_ms)))],
                            "per": "step (one chunk of every stream)"},
             "latency_us_cold_l2": cold,
+            "wavefront": wave,
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": S * Tp * cfg.in_dim * 4,
                     "d2h_bytes_per_step": S * T * cfg.out_per_frame * 4, "ms_per_step": 1e3 * e2e_s / K},
             "gpu_launches": int(c1[5] - c0[5]),

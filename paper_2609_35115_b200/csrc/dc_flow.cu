@@ -1102,6 +1102,8 @@ struct FlowModel {
   // launch plumbing
   bool pdl = true;                       // programmatic dependent launch between the step's kernels
   bool one_issuer = false;               // experiments: a single UMMA issuer
+  int  n_sm = 148;                       // SMs of the device (read at create)
+  int  force_v = -1;                     // experiments: N-tile variant forced (0: 64, 1: 32, 2: 16 columns)
   int  qkv_stages = 4;
   int  wide_stages = 4;                  // 2 or 4 (even, see the stage count rule in enqueue_chunk)
   int  dbg = 0;
@@ -1311,6 +1313,11 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     m->pdl = !(e && atoi(e));
     const char* d = getenv("DC_GEMM_DBG");
     m->dbg = d ? atoi(d) : 0;
+    const char* fv = getenv("DC_TILE_V");
+    m->force_v = (fv && fv[0] && atoi(fv) >= 0 && atoi(fv) <= 2) ? atoi(fv) : -1;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      m->n_sm = sms;
     const char* oi = getenv("DC_ONE_ISSUER");
     m->one_issuer = oi && atoi(oi);
     const char* qs = getenv("DC_QKV_STAGES");
@@ -1463,9 +1470,12 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
          (uint32_t)c.noise_seed_lo, (uint32_t)c.noise_seed_hi);
 
   const int m_tiles = (n * SLOT_ROWS + TILE_M - 1) / TILE_M;
-  // N-tile variant: the widest whose C-wide GEMMs still give about 96 CTAs, else the narrowest
-  int v = 0;
-  while (v < 2 && m_tiles * (C / (64 >> v)) < 96) ++v;
+  // N-tile variant: the narrowest whose C-wide GEMMs still fit ONE wave (a GEMM CTA has an SM to itself);
+  // a second, part-filled wave costs more than wider tiles do (measured with 5 and 10 row tiles: 160 CTAs
+  // of 16 columns 0.26 ms per pass, 80 CTAs of 32 columns 0.20 ms)
+  int v = 2;
+  while (v > 0 && m_tiles * (C / (64 >> v)) > m->n_sm) --v;
+  if (m->force_v >= 0) v = m->force_v;
   // the output projection always uses 16-column tiles: mel/16 CTAs per row tile instead of one, and a
   // single Euler-state round trip per epilogue thread
   const int bn = 64 >> v, bq = 192 >> v, bo = 16;
