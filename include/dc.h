@@ -198,7 +198,11 @@ dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
  * Flow and token2wav pipelines; the model must have been created with max_batch >= n_steps
  * (DC_ERR_ARG otherwise, stream untouched).  The token2wav composite keeps the call's mel frames
  * in a device buffer owned by the stream, which this call (re)allocates when n_frames exceeds
- * every earlier call's; the flow pipeline allocates nothing. */
+ * every earlier call's; the flow pipeline allocates nothing.  The composite's vocoder tail has no
+ * Euler loop to pipeline: chunk j's tail is enqueued, behind an event, on a CUDA stream owned by
+ * the dc_stream as soon as the pass that finishes chunk j is, so it runs beside the flow decoder's
+ * later passes; cuda_stream is made to wait for the last tail before the call returns, so work the
+ * caller enqueues afterwards on cuda_stream sees the complete output. */
 dc_status dc_decode_wavefront(dc_stream* stream, const float* feats_dev, long long n_frames,
                               float* out_dev, long long* n_out, void* cuda_stream);
 

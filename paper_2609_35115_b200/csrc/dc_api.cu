@@ -96,6 +96,8 @@ struct dc_stream {
   float*    mel = nullptr;         // [f_chunk][mel_dim] fp32, device
   float*    wave_mel = nullptr;    // dc_decode_wavefront of the composite: all mel frames of one call (grown on demand)
   long long wave_mel_frames = 0;
+  cudaStream_t wave_side = nullptr;   // the vocoder tail of a wavefront call runs here, beside the flow decoder's passes
+  cudaEvent_t  wave_ev = nullptr;
   float*    stage_in = nullptr;    // device staging of dc_decode_chunk_host
   float*    stage_out = nullptr;
   cudaGraph_t     g_graph = nullptr;   // fp32 pipelines: the captured chunk step
@@ -366,6 +368,10 @@ static void free_stream_buffers(dc_stream* s) {
   if (s->mel) cudaFree(s->mel);
   if (s->wave_mel) cudaFree(s->wave_mel);
   s->wave_mel = nullptr;
+  if (s->wave_side) cudaStreamDestroy(s->wave_side);
+  if (s->wave_ev) cudaEventDestroy(s->wave_ev);
+  s->wave_side = nullptr;
+  s->wave_ev = nullptr;
   s->sub_flow = s->sub_voc = nullptr;
   s->mel = nullptr;
   if (s->stage_in) cudaFree(s->stage_in);
@@ -762,6 +768,58 @@ extern "C" dc_status dc_decode_chunk(dc_stream* s, const float* feats, int T, fl
   return DC_OK;
 }
 
+// The flow pipeline's part of dc_decode_wavefront, with the stream's bookkeeping.
+static dc_status wave_flow(dc_stream* s, const float* feats, long long n_frames, float* out, cudaStream_t cs,
+                           void (*on_chunk)(void*, long long), void* ctx) {
+  dc_model* m = s->model;
+  int launches = 0;
+  dc_status st = dc::flow_decode_wave(m->flow, s->flow, feats, m->in_dim, n_frames, out, cs, &launches, on_chunk, ctx);
+  m->counters[5] += (uint64_t)launches;
+  if (st == DC_ERR_ARG) {   // refused before anything ran (max_batch < n_steps): the stream is untouched
+    m->counters[3]++;
+    return st;
+  }
+  if (st != DC_OK) {
+    s->poisoned = true;
+    return st;
+  }
+  const long long n_chunks = (n_frames + m->cfg.f_chunk - 1) / m->cfg.f_chunk;
+  s->frames_total += n_frames;
+  s->chunks += n_chunks;
+  m->counters[0] += (uint64_t)n_chunks;
+  m->counters[1] += (uint64_t)n_frames;
+  return DC_OK;
+}
+
+namespace {
+// Host-side hook of the composite's wavefront: as soon as the pass that finishes chunk j is enqueued, the
+// vocoder tail of chunk j is enqueued on the side stream behind an event, so that it runs beside the flow
+// decoder's next passes (which leave most SMs idle) instead of after them.
+struct WaveTail {
+  dc_stream*   s;
+  cudaStream_t main_st, side;
+  float*       out;
+  long long    n_frames;
+  dc_status    st = DC_OK;
+};
+
+void wave_tail_chunk(void* ctx, long long j) {
+  WaveTail* w = static_cast<WaveTail*>(ctx);
+  if (w->st != DC_OK) return;
+  dc_stream* s = w->s;
+  dc_model* m = s->model;
+  const int fc = m->cfg.f_chunk;
+  const int T = (int)(w->n_frames - j * fc < fc ? w->n_frames - j * fc : fc);
+  if (w->side != w->main_st) {
+    if (cudaEventRecord(s->wave_ev, w->main_st) != cudaSuccess || cudaStreamWaitEvent(w->side, s->wave_ev, 0) != cudaSuccess) {
+      w->st = DC_ERR_CUDA;
+      return;
+    }
+  }
+  w->st = dc_decode_chunk(s->sub_voc, s->wave_mel + j * fc * m->cfg.mel_dim, T, w->out + j * fc * m->out_per_frame, nullptr, (void*)w->side);
+}
+}  // namespace
+
 extern "C" dc_status dc_decode_wavefront(dc_stream* s, const float* feats, long long n_frames, float* out, long long* n_out,
                                          void* cuda_stream) {
   if (!s) return DC_ERR_ARG;
@@ -780,8 +838,12 @@ extern "C" dc_status dc_decode_wavefront(dc_stream* s, const float* feats, long 
   const long long n_chunks = (n_frames + fc - 1) / fc;
   dc_status st = DC_OK;
   if (m->sub_flow) {
-    // the flow decoder's wavefront leaves every mel frame of the call on the device, then the vocoder
-    // tail (whose chunk step has no Euler loop to pipeline) consumes them chunk by chunk
+    if (m->cfg.max_batch < m->cfg.n_steps) {
+      m->counters[3]++;
+      dc::set_error("wavefront decoding keeps n_steps = %d chunks in flight: max_batch must be >= n_steps", m->cfg.n_steps);
+      return DC_ERR_ARG;
+    }
+    // the call's mel frames stay on the device, in a buffer of the stream
     if (s->wave_mel_frames < n_frames) {
       if (s->wave_mel) cudaFree(s->wave_mel);
       s->wave_mel = nullptr;
@@ -792,32 +854,32 @@ extern "C" dc_status dc_decode_wavefront(dc_stream* s, const float* feats, long 
       }
       s->wave_mel_frames = n_frames;
     }
-    st = dc_decode_wavefront(s->sub_flow, feats, n_frames, s->wave_mel, nullptr, cuda_stream);
-    for (long long j = 0; j < n_chunks && st == DC_OK; ++j) {
-      const int T = (int)(n_frames - j * fc < fc ? n_frames - j * fc : fc);
-      st = dc_decode_chunk(s->sub_voc, s->wave_mel + j * fc * m->cfg.mel_dim, T, out + j * fc * m->out_per_frame, nullptr, cuda_stream);
+    if (!s->wave_side) {
+      if (cudaStreamCreateWithFlags(&s->wave_side, cudaStreamNonBlocking) != cudaSuccess ||
+          cudaEventCreateWithFlags(&s->wave_ev, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        return DC_ERR_CUDA;
+      }
+    }
+    // while profiling, everything stays on the caller's stream (the event brackets assume one stream)
+    WaveTail w{s, cs, (m->sub_voc->prof.on || m->sub_flow->prof.on) ? cs : s->wave_side, out, n_frames};
+    st = wave_flow(s->sub_flow, feats, n_frames, s->wave_mel, cs, wave_tail_chunk, &w);
+    if (st == DC_OK) st = w.st;
+    if (st == DC_OK && w.side != cs) {   // the caller's stream continues only after the last vocoder chunk
+      if (cudaEventRecord(s->wave_ev, w.side) != cudaSuccess || cudaStreamWaitEvent(cs, s->wave_ev, 0) != cudaSuccess) st = DC_ERR_CUDA;
     }
     if (st != DC_OK) {
       s->poisoned = true;
       return st;
     }
+    s->frames_total += n_frames;
+    s->chunks += n_chunks;
+    m->counters[0] += (uint64_t)n_chunks;
+    m->counters[1] += (uint64_t)n_frames;
   } else {
-    int launches = 0;
-    st = dc::flow_decode_wave(m->flow, s->flow, feats, m->in_dim, n_frames, out, cs, &launches);
-    m->counters[5] += (uint64_t)launches;
-    if (st == DC_ERR_ARG) {   // refused before anything ran (max_batch < n_steps): the stream is untouched
-      m->counters[3]++;
-      return st;
-    }
-    if (st != DC_OK) {
-      s->poisoned = true;
-      return st;
-    }
+    st = wave_flow(s, feats, n_frames, out, cs, nullptr, nullptr);
+    if (st != DC_OK) return st;
   }
-  s->frames_total += n_frames;
-  s->chunks += n_chunks;
-  m->counters[0] += (uint64_t)n_chunks;
-  m->counters[1] += (uint64_t)n_frames;
   if (n_out) *n_out = n_frames * m->out_per_frame;
   return DC_OK;
 }

@@ -1715,7 +1715,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
 // finished are holes (T = 0).  The arithmetic of a slot never depends on what the other slots hold, so the
 // result equals chunk-by-chunk decoding bit for bit.
 dc_status flow_decode_wave(FlowModel* m, FlowState* s, const float* feats, int in_dim, long long n_frames, float* out,
-                           cudaStream_t st, int* launches) {
+                           cudaStream_t st, int* launches, void (*on_chunk)(void*, long long), void* hook_ctx) {
   const dc_config& c = m->cfg;
   const int np = m->n_pass, K = c.n_steps;
   const int n = K * np;                                   // slots of a tick
@@ -1784,6 +1784,7 @@ dc_status flow_decode_wave(FlowModel* m, FlowState* s, const float* feats, int i
         return DC_ERR_CUDA;
       }
     }
+    if (on_chunk && t >= K - 1) on_chunk(hook_ctx, t - (K - 1));   // that chunk's last Euler step is now enqueued
   }
   s->frames = frames0 + n_frames;
   return DC_OK;
