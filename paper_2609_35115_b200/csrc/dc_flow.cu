@@ -95,6 +95,8 @@ struct GemmParams {
   long long    halo_off;        // element offset of the next conv's carry inside SlotInfo::halo, or -1
   bf16*        q_out;           // MODE_QKV
   long long    kv_off;          // element offset of this (step, layer)'s K ring inside SlotInfo::kv
+  int          kv_rs, kv_hs;    // K/V planes: elements between a head's consecutive rows / between heads
+  int          dh_shift;        // log2(head_dim)
   int          Rk;              // ring rows
   int          P;               // prompt rows in front of the ring (0: none)
   int          C;
@@ -483,7 +485,8 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               if (row >= p.Rk) row -= p.Rk;
               row += p.P;
             }
-            store16(si.kv + p.kv_off + (long long)(which - 1) * (p.P + p.Rk) * p.C + (long long)row * p.C + col, a, b);
+            const int hh = col >> p.dh_shift, wi = col - (hh << p.dh_shift);
+            store16(si.kv + p.kv_off + (long long)(which - 1) * (p.P + p.Rk) * p.C + (long long)hh * p.kv_hs + (long long)row * p.kv_rs + wi, a, b);
           }
         }
         continue;
@@ -674,6 +677,7 @@ struct AttnParams {
   int             ld;
   int             dh;         // 32 or 64 (smem rows are padded to 64 columns)
   long long       kv_off;     // element offset of this (step, layer)'s K ring inside SlotInfo::kv
+  int             kv_rs, kv_hs;   // K/V planes: elements between a head's consecutive rows / between heads
   int             Rk, C;
   int             P;          // prompt rows in front of the ring
   float           scale_log2e;  // log2(e) / sqrt(dh)
@@ -755,7 +759,11 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   ptx::pdl_launch();
-  ptx::pdl_wait();      // the slot table, Q and the appended K/V rows come from earlier kernels
+  // Q and the chunk's appended K/V rows come from the kernel before this one.  The slot table and the CARRIED K/V
+  // rows do not (the table is written by the first kernel of the step, which has completed before any projection
+  // starts; carried rows by earlier steps), so the loader warps fetch the leading all-carried key blocks first
+  // and wait afterwards.
+  if (warp < 5) ptx::pdl_wait();
   const SlotInfo si = p.slots[slot];
   // attended keys, in this order: the prompt rows (with the chunk's own prompt frames, already appended), then
   // the carried history and the chunk's history frames, a circular interval of the ring behind the prompt rows
@@ -772,35 +780,14 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     const int nl = is_k ? ATT_K_LOADERS : ATT_V_LOADERS;
     const int lt = (warp == 6 ? 32 : 0) + lane;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-    if (is_k) {
-      const bf16* qbase = p.q + (long long)(GUARD + slot * SLOT_ROWS + HALO) * p.ld + head * p.dh;
-      for (int i = lt; i < 128 * 8; i += nl) {
-        const int row = i >> 3, j = i & 7, qrow = row & 63;   // rows 64.. repeat rows 0..
-        uint8_t* dst = sQ + row * 128 + ((j ^ (row & 7)) << 4);
-        if (qrow < T && j < chunks) cp_async16(dst, qbase + (long long)qrow * p.ld + j * 8);
-        else *reinterpret_cast<uint4*>(dst) = zero;
-      }
-    }
-    const bf16* src0 = si.kv + p.kv_off + head * p.dh + (is_k ? 0 : (long long)((PROMPT ? p.P : 0) + p.Rk) * p.C);
+    const bf16* src0 = si.kv + p.kv_off + (long long)head * p.kv_hs + (is_k ? 0 : (long long)((PROMPT ? p.P : 0) + p.Rk) * p.C);
+    const int rs = p.kv_rs;
     uint64_t* full = is_k ? full_k : full_v;
     uint64_t* empty = is_k ? empty_k : empty_v;
     int start = si.kv_head - si.kv_len;
     if (start < 0) start += p.Rk;
-    bool ok = true;
-    for (int b = 0; b < nkb; ++b) {
-      const int st = b % ATT_STAGES;
-      if (b >= 1) {   // the previous block has been issued a whole iteration ago: publish it
-        asm volatile("cp.async.wait_all;" ::: "memory");
-        ptx::fence_proxy_async_smem();
-        ptx::mbar_arrive(&full[(b - 1) % ATT_STAGES]);
-        if (lt == 0 && is_k && b - 1 < 8) DC_AT(8 + b - 1);     // block b-1 landed
-      }
-      if (b >= ATT_STAGES && ok && !ptx::mbar_wait_relaxed(&empty[st], ((b / ATT_STAGES) - 1) & 1)) {
-        ok = false;
-        atomicExch(p.err, 4);
-      }
-      uint8_t* dstb = ring + st * ATT_STAGE_BYTES + (is_k ? 0 : ATT_KB * 128);
-      if (lt == 0 && is_k && b < 8) DC_AT(b);                    // block b load issue starts
+    auto issue_block = [&](int b) {
+      uint8_t* dstb = ring + (b % ATT_STAGES) * ATT_STAGE_BYTES + (is_k ? 0 : ATT_KB * 128);
       if (!PROMPT) {
         for (int i = lt; i < ATT_KB * 8; i += nl) {
           const int row = i >> 3, j = i & 7;
@@ -809,7 +796,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
           if (key < L && j < chunks) {
             int rr = start + key;
             if (rr >= p.Rk) rr -= p.Rk;
-            cp_async16(dstb + off, src0 + (long long)rr * p.C + j * 8);
+            cp_async16(dstb + off, src0 + (long long)rr * rs + j * 8);
           } else {
             *reinterpret_cast<uint4*>(dstb + off) = zero;   // for V: 0 * garbage must not poison O
           }
@@ -819,7 +806,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         for (int i = lt; i < ATT_KB * 8; i += nl) {
           const int row = i >> 3, j = i & 7;
           const int off = row * 128 + ((j ^ (row & 7)) << 4);
-          if (j < chunks) cp_async16(dstb + off, src0 + (long long)(b * ATT_KB + row) * p.C + j * 8);
+          if (j < chunks) cp_async16(dstb + off, src0 + (long long)(b * ATT_KB + row) * rs + j * 8);
           else *reinterpret_cast<uint4*>(dstb + off) = zero;
         }
       } else {
@@ -835,12 +822,44 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
               if (rr >= p.Rk) rr -= p.Rk;
               rr += p.P;
             }
-            cp_async16(dstb + off, src0 + (long long)rr * p.C + j * 8);
+            cp_async16(dstb + off, src0 + (long long)rr * rs + j * 8);
           } else {
             *reinterpret_cast<uint4*>(dstb + off) = zero;
           }
         }
       }
+    };
+    // keys [0, carried) were appended by earlier steps: the prompt rows already there, and - once the prompt is
+    // complete - the retained history behind them
+    const int carried = PROMPT ? (n_prompt == si.n_prompt0 ? n_prompt + si.kv_len : si.n_prompt0) : si.kv_len;
+    const int n_early = min(min(carried / ATT_KB, ATT_STAGES), nkb);
+    for (int b = 0; b < n_early; ++b) issue_block(b);
+    ptx::pdl_wait();
+    if (is_k) {
+      const bf16* qbase = p.q + (long long)(GUARD + slot * SLOT_ROWS + HALO) * p.ld + head * p.dh;
+      for (int i = lt; i < 128 * 8; i += nl) {
+        const int row = i >> 3, j = i & 7, qrow = row & 63;   // rows 64.. repeat rows 0..
+        uint8_t* dst = sQ + row * 128 + ((j ^ (row & 7)) << 4);
+        if (qrow < T && j < chunks) cp_async16(dst, qbase + (long long)qrow * p.ld + j * 8);
+        else *reinterpret_cast<uint4*>(dst) = zero;
+      }
+    }
+    bool ok = true;
+    for (int b = 0; b < nkb; ++b) {
+      const int st = b % ATT_STAGES;
+      if (b >= 1) {   // the previous block has been issued a whole iteration ago: publish it (block 0 together with Q)
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        ptx::fence_proxy_async_smem();
+        ptx::mbar_arrive(&full[(b - 1) % ATT_STAGES]);
+        if (lt == 0 && is_k && b - 1 < 8) DC_AT(8 + b - 1);     // block b-1 landed
+      }
+      if (b < n_early) continue;                                // already in flight
+      if (b >= ATT_STAGES && ok && !ptx::mbar_wait_relaxed(&empty[st], ((b / ATT_STAGES) - 1) & 1)) {
+        ok = false;
+        atomicExch(p.err, 4);
+      }
+      if (lt == 0 && is_k && b < 8) DC_AT(b);                    // block b load issue starts
+      issue_block(b);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     ptx::fence_proxy_async_smem();
@@ -1102,6 +1121,7 @@ struct FlowModel {
   // launch plumbing
   bool pdl = true;                       // programmatic dependent launch between the step's kernels
   bool one_issuer = false;               // experiments: a single UMMA issuer
+  int  kv_rs = 0, kv_hs = 0, dh_shift = 0;   // K/V plane layout (see GemmParams)
   int  n_sm = 148;                       // SMs of the device (read at create)
   int  force_v = -1;                     // experiments: N-tile variant forced (0: 64, 1: 32, 2: 16 columns)
   int  qkv_stages = 4;
@@ -1313,6 +1333,13 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     m->pdl = !(e && atoi(e));
     const char* d = getenv("DC_GEMM_DBG");
     m->dbg = d ? atoi(d) : 0;
+    {
+      const char* hm = getenv("DC_KV_ROWMAJOR");   // experiments: rows of all heads interleaved
+      const bool head_major = !(hm && atoi(hm)) && m->cfg.head_dim > 0;
+      m->dh_shift = m->cfg.head_dim == 64 ? 6 : 5;
+      m->kv_rs = head_major ? m->cfg.head_dim : m->C;
+      m->kv_hs = head_major ? (m->P + m->Rk) * m->cfg.head_dim : m->cfg.head_dim;
+    }
     const char* fv = getenv("DC_TILE_V");
     m->force_v = (fv && fv[0] && atoi(fv) >= 0 && atoi(fv) <= 2) ? atoi(fv) : -1;
     int dev = 0, sms = 0;
@@ -1517,6 +1544,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     p.slots = m->d_slots; p.q = m->Q; p.o = m->O; p.ld = C; p.dh = c.head_dim;
     p.kv_off = ((long long)step * c.n_attn + layer) * 2 * (m->P + m->Rk) * C;
     p.Rk = m->Rk; p.C = C; p.P = m->P;
+    p.kv_rs = m->kv_rs; p.kv_hs = m->kv_hs;
     p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
     p.err = m->d_err;
     launch(lc, m->P > 0 ? flow_attn_kernel<true> : flow_attn_kernel<false>, dim3(n, c.n_heads), dim3(ATT_THREADS), ATT_SMEM, true, 2, p);
@@ -1560,6 +1588,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
           p.mode = MODE_QKV; p.BN = bq; p.n_kblocks = C / KBLK; p.taps = 1;
           p.bias = fc + m->o_bqkv[g]; p.q_out = m->Q; p.halo_off = -1;
           p.kv_off = ((long long)s * c.n_attn + g) * 2 * (m->P + m->Rk) * C;
+          p.kv_rs = m->kv_rs; p.kv_hs = m->kv_hs; p.dh_shift = m->dh_shift;
           normalised(p);
           gemm(*tX, m->tmWqkv[v][g], p, 3 * C);
         }
