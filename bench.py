@@ -267,7 +267,8 @@ def main():
     feats_d = feats_h.cuda()
     out_d = torch.empty(S, T * cfg.out_per_frame, device="cuda")
     out_dv = out_d.view(S, T, -1) if cfg.pipeline not in ("vocoder", "token2wav") else out_d
-    batched = cfg.pipeline == "flow" and S > 1
+    batched = cfg.pipeline in ("flow", "token2wav") and S > 1
+    batched_host = cfg.pipeline == "flow" and S > 1     # the host-buffer batch call serves the flow pipeline only
 
     def step(r):
         if batched:
@@ -343,7 +344,7 @@ def main():
     fout_v = fout.view(S, T, -1) if cfg.pipeline not in ("vocoder", "token2wav") else fout
     e2e_warm = min(3, K)
     def e2e_step(k):
-        if batched:
+        if batched_host:
             dc.decode_batch_host(model, streams, fin[k], fout_v)
         else:
             for i in range(S):

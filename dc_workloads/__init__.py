@@ -267,6 +267,8 @@ def tiny_token2wav(**kw) -> DCConfig:
 # beyond the five: the whole decoder step in one call
 EXTRA_CONFIGS: Dict[str, DCConfig] = {
     "token2wav": token2wav(),
+    # ... for 32 concurrent streams (cfg5's serving shape with the vocoder tail behind every stream)
+    "token2wav_serving": token2wav(name="token2wav_serving", n_streams=32, n_chunks=100, seed=10),
     # cfg3 with classifier-free guidance (two passes per Euler step, the form the paper measures its flow step in)
     "cfg3_guided": CONFIGS["cfg3"].replace(name="cfg3_guided", cfg_scale=0.7, seed=7),
     # cfg3's network with the paper's carry: a 302-frame prompt that is never evicted + 100 retained frames

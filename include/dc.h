@@ -180,7 +180,9 @@ dc_status dc_decode_chunk(dc_stream* stream, const float* feats_dev, int n_frame
  * pointers / ints).  Results are bitwise identical to n single dc_decode_chunk
  * calls.  (Multi-session serving over shared weights with per-session state:
  * paper Section 3.4, last paragraph, and Section 4.3 "Serving capacity".)  Flow and token2wav
- * pipelines. */
+ * pipelines.  The token2wav composite batches the flow decoder and then runs the streams' vocoder
+ * tails side by side on CUDA streams owned by the model, forked behind the flow decoder on
+ * cuda_stream and joined back into it before the call returns. */
 dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
                           const float* const* feats_dev, const int* n_frames,
                           float* const* out_dev, void* cuda_stream);

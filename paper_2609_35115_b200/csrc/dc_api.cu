@@ -65,7 +65,6 @@ struct dc_model {
   dc_config cfg;
   int       device = 0;
   float*    d_w = nullptr;   // fp32 pipelines: the blob on the device
-  dc::F32Call* d_call = nullptr;
   // flow pipeline: staging of dc_decode_batch_host (pinned host + device, max_batch chunks each way)
   float *h_in = nullptr, *h_out = nullptr, *d_in = nullptr, *d_out = nullptr;
   int*   h_err = nullptr;   // fp32 pipelines: per-call record read by the captured graphs
@@ -76,12 +75,25 @@ struct dc_model {
   // DC_PIPE_TOKEN2WAV: the flow decoder and the vocoder tail as models of their own; this one only chains them
   dc_model* sub_flow = nullptr;
   dc_model* sub_voc = nullptr;
+  // ... and CUDA streams of its own on which dc_decode_batch runs the streams' vocoder tails side by side
+  std::vector<cudaStream_t> tail_streams;
+  std::vector<cudaEvent_t>  tail_done;
+  cudaEvent_t               tail_fork = nullptr;
   std::atomic<uint64_t> counters[8];
   std::atomic<int> open_streams{0};
   std::mutex mu;
   dc::Profiler prof;
   std::vector<dc_stream*> all_streams;   // host structs live until dc_destroy, so a closed handle stays detectable
 };
+
+static void free_tail_streams(dc_model* m) {
+  for (cudaStream_t t : m->tail_streams) cudaStreamDestroy(t);
+  for (cudaEvent_t e : m->tail_done) cudaEventDestroy(e);
+  if (m->tail_fork) cudaEventDestroy(m->tail_fork);
+  m->tail_streams.clear();
+  m->tail_done.clear();
+  m->tail_fork = nullptr;
+}
 
 struct dc_stream {
   dc_model* model = nullptr;
@@ -90,6 +102,8 @@ struct dc_stream {
   long long chunks = 0;
   std::vector<DevBuf> f32_rings;   // input ring of each fp32 layer
   float*    tails = nullptr;       // [2][12] overlap-add tails (ping-pong)
+  dc::F32Call* d_call = nullptr;   // fp32 pipelines: per-call record read by this stream's captured graph (streams of one
+                                   // model may decode at the same time on different CUDA streams)
   dc::FlowState* flow = nullptr;
   dc_stream* sub_flow = nullptr;   // DC_PIPE_TOKEN2WAV: the two halves' streams and the mel chunk between them
   dc_stream* sub_voc = nullptr;
@@ -285,6 +299,24 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     if (st == DC_OK) {
       m->in_dim = m->sub_flow->in_dim;
       m->out_per_frame = m->sub_voc->out_per_frame;
+      // a vocoder chunk step fills a fraction of the GPU (12 short kernels on small grids): up to 8 of a batch's
+      // tails run at the same time
+      const char* nts = getenv("DC_TAIL_STREAMS");   // experiments: 0 or 1 = the tails one after another on the caller's stream
+      const int want = nts ? atoi(nts) : 8;
+      const int n_side = cfg->max_batch < want ? cfg->max_batch : (want > 32 ? 32 : want);
+      bool ok = n_side < 2 || cudaEventCreateWithFlags(&m->tail_fork, cudaEventDisableTiming) == cudaSuccess;
+      for (int i = 0; ok && n_side >= 2 && i < n_side; ++i) {
+        cudaStream_t cs2 = nullptr;
+        cudaEvent_t ev = nullptr;
+        ok = cudaStreamCreateWithFlags(&cs2, cudaStreamNonBlocking) == cudaSuccess;
+        if (ok) m->tail_streams.push_back(cs2);
+        ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
+        if (ev) m->tail_done.push_back(ev);
+      }
+      if (!ok) {
+        dc::set_error("stream / event creation failed");
+        st = DC_ERR_CUDA;
+      }
     }
   } else if (cfg->pipeline == DC_PIPE_FLOW) {
     st = dc::flow_model_create(*cfg, w, &m->flow);
@@ -308,7 +340,6 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     cudaError_t e = cudaMalloc(&m->d_w, n_floats * sizeof(float));
     if (e == cudaSuccess) e = cudaMemcpy(m->d_w, w, n_floats * sizeof(float), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = dc::prepare_f32_constants();
-    if (e == cudaSuccess) e = cudaMalloc(&m->d_call, sizeof(dc::F32Call));
     if (e != cudaSuccess) {
       dc::set_error("weight upload failed: %s", cudaGetErrorString(e));
       st = e == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;
@@ -317,8 +348,8 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
   if (st != DC_OK) {
     if (m->sub_flow) dc_destroy(m->sub_flow);
     if (m->sub_voc) dc_destroy(m->sub_voc);
+    free_tail_streams(m);
     if (m->d_w) cudaFree(m->d_w);
-    if (m->d_call) cudaFree(m->d_call);
     if (m->flow) dc::flow_model_destroy(m->flow);
     if (m->h_in) cudaFreeHost(m->h_in);
     if (m->h_out) cudaFreeHost(m->h_out);
@@ -340,9 +371,9 @@ extern "C" dc_status dc_destroy(dc_model* m) {
   }
   if (m->sub_flow) dc_destroy(m->sub_flow);   // their streams were closed with ours
   if (m->sub_voc) dc_destroy(m->sub_voc);
+  free_tail_streams(m);
   if (m->flow) dc::flow_model_destroy(m->flow);
   if (m->d_w) cudaFree(m->d_w);
-  if (m->d_call) cudaFree(m->d_call);
   if (m->h_in) cudaFreeHost(m->h_in);
   if (m->h_out) cudaFreeHost(m->h_out);
   if (m->h_err) cudaFreeHost(m->h_err);
@@ -362,6 +393,8 @@ static void free_stream_buffers(dc_stream* s) {
     if (b.p) cudaFree(b.p);
   s->f32_rings.clear();
   if (s->tails) cudaFree(s->tails);
+  if (s->d_call) cudaFree(s->d_call);
+  s->d_call = nullptr;
   if (s->flow) dc::flow_state_close(s->flow);
   if (s->sub_flow) dc_stream_close(s->sub_flow);
   if (s->sub_voc) dc_stream_close(s->sub_voc);
@@ -404,6 +437,7 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
       e = cudaMemset(b.p, 0, b.bytes);
       if (e != cudaSuccess) break;
     }
+    if (e == cudaSuccess) e = cudaMalloc(&s->d_call, sizeof(dc::F32Call));
     if (e == cudaSuccess && m->cfg.pipeline == DC_PIPE_VOCODER) {
       e = cudaMalloc(&s->tails, 2 * 12 * sizeof(float));
       if (e == cudaSuccess) e = cudaMemset(s->tails, 0, 2 * 12 * sizeof(float));
@@ -621,7 +655,7 @@ static void enqueue_f32(dc_stream* s, bool use_call, const float* feats, int T, 
       h.in_ring = ring; h.in_mask = L.ring_cap - 1; h.C = L.C_in;
       h.W = m->d_w + L.w_off; h.bias = m->d_w + L.b_off; h.clamp = m->cfg.logmag_clamp;
       if (use_call) {
-        h.call = m->d_call; h.rate_in = L.rate_in; h.tails = s->tails;
+        h.call = s->d_call; h.rate_in = L.rate_in; h.tails = s->tails;
       } else {
         h.pos = pos; h.T = Tin;
         h.tail_in = s->tails + 12 * (s->chunks & 1);
@@ -635,7 +669,7 @@ static void enqueue_f32(dc_stream* s, bool use_call, const float* feats, int T, 
       p.in_ring = ring; p.in_mask = L.ring_cap - 1; p.C_in = L.C_in;
       p.first_layer = l == 0; p.last_layer = l + 1 == nL; p.rate_in = L.rate_in;
       if (use_call) {
-        p.call = m->d_call;
+        p.call = s->d_call;
       } else {
         p.pos_in = pos; p.T_in = Tin;
         if (l == 0) p.in_direct = feats;
@@ -674,7 +708,7 @@ static void build_f32_graph(dc_stream* s) {
   cudaGraph_t graph = nullptr;
   if (cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
     dc::F32Call dummy{};
-    dc::launch_set_f32_call(dummy, m->d_call, cap);
+    dc::launch_set_f32_call(dummy, s->d_call, cap);
     int n = 1;
     enqueue_f32(s, true, nullptr, 0, nullptr, cap, pdl, &n);
     if (cudaStreamEndCapture(cap, &graph) == cudaSuccess && graph != nullptr) {
@@ -707,7 +741,7 @@ static dc_status decode_f32(dc_stream* s, const float* feats, int T, float* out,
   dc_model* m = s->model;
   if (s->g_exec != nullptr && !m->prof.on) {
     dc::F32Call v{s->frames_total, T, (int)(s->chunks & 1), feats, out};
-    dc::F32Call* dst = m->d_call;
+    dc::F32Call* dst = s->d_call;
     void* args[2] = {&v, &dst};
     cudaKernelNodeParams kp{};
     kp.func = const_cast<void*>(dc::set_f32_call_func());
@@ -922,9 +956,23 @@ extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* strea
       mels[(size_t)i] = streams[i]->mel;
     }
     st = dc_decode_batch(m->sub_flow, n, fs.data(), feats, n_frames, mels.data(), cuda_stream);
-    for (int i = 0; i < n && st == DC_OK; ++i)
-      st = dc_decode_chunk(streams[i]->sub_voc, streams[i]->mel, n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk, out[i], nullptr,
-                           cuda_stream);
+    // the tails are independent of one another: spread over the model's side streams, behind the flow
+    // decoder, and joined back into the caller's stream (all on cuda_stream while profiling: the event
+    // brackets assume one stream)
+    cudaStream_t cs = (cudaStream_t)cuda_stream;
+    const int n_side = (n >= 2 && !m->sub_voc->prof.on && !m->sub_flow->prof.on) ? (int)m->tail_streams.size() : 0;
+    if (st == DC_OK && n_side > 0 && cudaEventRecord(m->tail_fork, cs) != cudaSuccess) st = DC_ERR_CUDA;
+    for (int i = 0; i < n && st == DC_OK; ++i) {
+      cudaStream_t ts = n_side > 0 ? m->tail_streams[(size_t)(i % n_side)] : cs;
+      if (n_side > 0 && i < n_side && cudaStreamWaitEvent(ts, m->tail_fork, 0) != cudaSuccess) st = DC_ERR_CUDA;
+      if (st == DC_OK)
+        st = dc_decode_chunk(streams[i]->sub_voc, streams[i]->mel, n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk, out[i],
+                             nullptr, (void*)ts);
+    }
+    for (int k = 0; k < n_side && k < n && st == DC_OK; ++k)
+      if (cudaEventRecord(m->tail_done[(size_t)k], m->tail_streams[(size_t)k]) != cudaSuccess ||
+          cudaStreamWaitEvent(cs, m->tail_done[(size_t)k], 0) != cudaSuccess)
+        st = DC_ERR_CUDA;
   } else {
     st = dc::flow_decode(m->flow, n, states.data(), feats, n_frames, out, (cudaStream_t)cuda_stream, &launches);
   }

@@ -179,3 +179,30 @@ def test_bounded_device_wait_gives_up_and_reports(dc):
     assert torch.isfinite(y).all()
     st.close()
     m.destroy()
+
+
+def test_streams_of_one_model_on_different_cuda_streams(dc):
+    """Each stream's captured chunk step reads a call record of its own, so two streams of one model may
+    decode at the same time on different CUDA streams."""
+    import torch
+    from tests import gpu_util as gu
+    cfg = wl.tiny_vocoder(n_chunks=6, n_streams=2)
+    w = wl.make_workload(cfg)
+    m = dc.Model(cfg, w.weights)
+    ref = [gu.run_gpu_stream(m, s.feats, s.boundaries) for s in w.streams]
+    sts = [m.open_stream() for _ in w.streams]
+    cs = [torch.cuda.Stream() for _ in w.streams]
+    xs = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+    outs = [[], []]
+    torch.cuda.synchronize()
+    n_rounds = max(len(s.boundaries) - 1 for s in w.streams)
+    for r in range(n_rounds):
+        for i, s in enumerate(w.streams):
+            if r < len(s.boundaries) - 1:
+                outs[i].append(sts[i].decode_chunk(xs[i][s.boundaries[r]:s.boundaries[r + 1]].contiguous(), stream=cs[i]))
+    torch.cuda.synchronize()
+    for i in range(2):
+        got = torch.cat(outs[i]).cpu().numpy()
+        assert np.array_equal(got, ref[i]), f"stream {i}"
+        sts[i].close()
+    m.destroy()

@@ -97,11 +97,14 @@ def test_chain_equals_the_two_models_by_hand(dc):
     assert np.array_equal(pcm, by_hand)
 
 
-def test_batched_chain_equals_single_stream(dc):
-    cfg = wl.tiny_token2wav(n_chunks=4, n_streams=3)
+@pytest.mark.parametrize("n_streams", [3, 11])
+def test_batched_chain_equals_single_stream(dc, n_streams):
+    """The batch call runs the streams' vocoder tails side by side on CUDA streams of the model (8 at most:
+    with 11 streams some side streams carry two tails); every stream's bytes are those of its own calls."""
+    cfg = wl.tiny_token2wav(n_chunks=4, n_streams=n_streams)
     w = wl.make_workload(cfg)
     gu = _gu()
-    m = dc.Model(cfg, w.weights, max_batch=3)
+    m = dc.Model(cfg, w.weights, max_batch=n_streams)
     single = [gu.run_gpu_stream(m, s.feats, s.boundaries) for s in w.streams]
     streams = [m.open_stream() for _ in w.streams]
     feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
