@@ -387,6 +387,28 @@ def main():
                 "note": "dc_decode_wavefront on one stream, input resident in HBM; includes the ramp-up and ramp-down passes"}
         sw.close()
         mw.destroy()
+        # ... and of several streams at once (dc_decode_wavefront_batch): every pass carries n_steps chunks of each
+        n_pass = 2 if getattr(cfg, "cfg_scale", 0.0) > 0 else 1
+        n_ws = min(3, 64 // (cfg.n_steps * n_pass))
+        if n_ws >= 2:
+            mb = dc.Model(cfg, weights, max_batch=n_ws * cfg.n_steps)
+            sb = [mb.open_stream() for _ in range(n_ws)]
+            fb = [torch.from_numpy(rng.standard_normal((n_wc * T, cfg.in_dim), dtype=np.float32)).cuda() for _ in range(n_ws)]
+            ob = [torch.empty(n_wc * T * cfg.out_per_frame, device="cuda") for _ in range(n_ws)]
+            for _ in range(2):
+                dc.decode_wavefront_batch(mb, sb, fb, ob)
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(n_calls):
+                dc.decode_wavefront_batch(mb, sb, fb, ob)
+            b.record()
+            torch.cuda.synchronize()
+            ms_b = a.elapsed_time(b) / n_calls
+            wave["batch"] = {"streams": n_ws, "value": n_ws * n_wc * per_chunk / (ms_b * 1e-3), "unit": unit,
+                             "ms_per_pass": ms_b / (n_wc + cfg.n_steps - 1), "chunks_per_stream": n_wc}
+            for s_ in sb:
+                s_.close()
+            mb.destroy()
 
     # ---- per-kernel-class device time (separate profiled pass; events between launches slow the step) ----
     pk, how = peaks()

@@ -208,6 +208,17 @@ dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
 dc_status dc_decode_wavefront(dc_stream* stream, const float* feats_dev, long long n_frames,
                               float* out_dev, long long* n_out, void* cuda_stream);
 
+/* dc_decode_wavefront for n distinct streams of one model at once: every pass of the network then
+ * carries n_steps chunks of each stream (n * n_steps slots; needs max_batch >= n * n_steps and
+ * n * n_steps * (2 with guidance) <= 64, DC_ERR_ARG otherwise with the streams untouched).
+ * feats_dev, n_frames, out_dev are HOST arrays as for dc_decode_batch; streams may have different
+ * lengths (a stream that has finished leaves holes in the later passes).  Results are bitwise those
+ * of n dc_decode_wavefront calls, hence of chunk-by-chunk decoding.  The single-stream pass is
+ * captured as a graph at dc_create; another stream count captures its pass at its first call. */
+dc_status dc_decode_wavefront_batch(dc_model* model, int n, dc_stream* const* streams,
+                                    const float* const* feats_dev, const long long* n_frames,
+                                    float* const* out_dev, void* cuda_stream);
+
 /* Convenience for callers with host buffers: copies feats_host to the device,
  * decodes, copies the result back and synchronises cuda_stream.  Uses staging
  * buffers owned by the stream (allocated at dc_stream_open).  Returns DC_ERR_TIMEOUT

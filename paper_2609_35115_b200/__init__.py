@@ -4,5 +4,5 @@ Argument marshalling only: every step of the decoder runs inside the CUDA
 library.  torch is used for device memory and streams.  There is no fallback:
 if the library is missing or no sm_100 device is present, calls raise.
 """
-from .binding import (DCError, NOALLOC_SCRATCH_FLOATS, conv_stack_noalloc, Model, Stream, decode_batch, decode_batch_host, library_path, load_library,  # noqa: F401
+from .binding import (DCError, NOALLOC_SCRATCH_FLOATS, conv_stack_noalloc, Model, Stream, decode_batch, decode_batch_host, decode_wavefront_batch, library_path, load_library,  # noqa: F401
                       make_config, selftest_bounded_wait, STATUS)

@@ -22,7 +22,7 @@ EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_
            "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error",
            "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end", "dc_conv_stack_noalloc",
            "dc_selftest_bounded_wait", "dc_stream_snapshot", "dc_stream_restore", "dc_snapshot_free",
-           "dc_decode_wavefront"]
+           "dc_decode_wavefront", "dc_decode_wavefront_batch"]
 
 
 class dc_config(C.Structure):
@@ -71,6 +71,7 @@ def load_library():
     lib.dc_decode_chunk.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
     lib.dc_decode_batch.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
     lib.dc_decode_wavefront.argtypes = [vp, vp, C.c_longlong, vp, cp(C.c_longlong), vp]
+    lib.dc_decode_wavefront_batch.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_longlong), cp(vp), vp]
     lib.dc_decode_chunk_host.argtypes = [vp, vp, C.c_int, vp, cp(C.c_int), vp]
     lib.dc_decode_batch_host.argtypes = [vp, C.c_int, cp(vp), cp(vp), cp(C.c_int), cp(vp), vp]
     lib.dc_profile_begin.argtypes = [vp, C.c_int]
@@ -305,6 +306,26 @@ def decode_batch(model: Model, streams: Sequence[Stream], feats, outs, stream=No
     n, hs, fp, nf, op = _batch_args(model, streams, feats, outs)
     _check(model.lib.dc_decode_batch(model.handle, n, hs, fp, nf, op, _cuda_stream_handle(stream)),
            "dc_decode_batch")
+
+
+def decode_wavefront_batch(model: Model, streams: Sequence[Stream], feats, outs=None, stream=None):
+    """dc_decode_wavefront_batch: feats[i] is a CUDA float32 tensor [n_frames_i, in_dim] with all of stream i's
+    remaining input; returns the list of outputs (allocated here unless given)."""
+    import torch
+    n = len(streams)
+    if outs is None:
+        outs = [torch.empty(f.shape[0] * model.out_per_frame, device=f.device, dtype=torch.float32) for f in feats]
+    for f in feats:
+        assert f.is_cuda and f.dtype == torch.float32 and f.is_contiguous()
+    hs = (C.c_void_p * n)(*[s.handle for s in streams])
+    fp = (C.c_void_p * n)(*[f.data_ptr() for f in feats])
+    nf = (C.c_longlong * n)(*[f.shape[0] for f in feats])
+    op = (C.c_void_p * n)(*[o.data_ptr() for o in outs])
+    _check(model.lib.dc_decode_wavefront_batch(model.handle, n, hs, fp, nf, op, _cuda_stream_handle(stream)),
+           "dc_decode_wavefront_batch")
+    if model.cfg.pipeline not in ("vocoder", "token2wav"):
+        outs = [o.view(-1, model.out_per_frame) for o in outs]
+    return outs
 
 
 def selftest_bounded_wait(max_polls: int = 1000) -> int:

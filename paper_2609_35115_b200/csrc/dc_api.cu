@@ -802,120 +802,135 @@ extern "C" dc_status dc_decode_chunk(dc_stream* s, const float* feats, int T, fl
   return DC_OK;
 }
 
-// The flow pipeline's part of dc_decode_wavefront, with the stream's bookkeeping.
-static dc_status wave_flow(dc_stream* s, const float* feats, long long n_frames, float* out, cudaStream_t cs,
-                           void (*on_chunk)(void*, long long), void* ctx) {
+namespace {
+// Host-side hook of the composite's wavefront: as soon as the pass that finishes chunk j of a stream is
+// enqueued, the vocoder tail of that chunk is enqueued on the stream's side stream behind an event, so that it
+// runs beside the flow decoder's next passes (which leave most SMs idle) instead of after them.
+struct WaveTail {
+  dc_stream* const* streams;
+  cudaStream_t      main_st;
+  bool              side;          // false while profiling: everything on the caller's stream
+  float* const*     out;
+  const long long*  n_frames;
+  dc_status         st = DC_OK;
+};
+
+void wave_tail_chunk(void* ctx, int i, long long j) {
+  WaveTail* w = static_cast<WaveTail*>(ctx);
+  if (w->st != DC_OK) return;
+  dc_stream* s = w->streams[i];
   dc_model* m = s->model;
+  const int fc = m->cfg.f_chunk;
+  const int T = (int)(w->n_frames[i] - j * fc < fc ? w->n_frames[i] - j * fc : fc);
+  cudaStream_t ts = w->side ? s->wave_side : w->main_st;
+  if (w->side && (cudaEventRecord(s->wave_ev, w->main_st) != cudaSuccess || cudaStreamWaitEvent(ts, s->wave_ev, 0) != cudaSuccess)) {
+    w->st = DC_ERR_CUDA;
+    return;
+  }
+  w->st = dc_decode_chunk(s->sub_voc, s->wave_mel + j * fc * m->cfg.mel_dim, T, w->out[i] + j * fc * m->out_per_frame, nullptr, (void*)ts);
+}
+}  // namespace
+
+extern "C" dc_status dc_decode_wavefront_batch(dc_model* m, int n, dc_stream* const* streams, const float* const* feats,
+                                               const long long* n_frames, float* const* out, void* cuda_stream) {
+  if (!m || !streams || !feats || !n_frames || !out) return DC_ERR_ARG;
+  if (!m->flow && !m->sub_flow) {
+    dc::set_error("wavefront decoding serves the flow and token2wav pipelines only");
+    return DC_ERR_CONFIG;
+  }
+  if (n < 1 || (long long)n * m->cfg.n_steps > m->cfg.max_batch) {
+    m->counters[3]++;
+    dc::set_error("wavefront decoding keeps n_steps = %d chunks per stream in flight: %d streams need max_batch >= %d", m->cfg.n_steps, n,
+                  n * m->cfg.n_steps);
+    return DC_ERR_ARG;
+  }
+  for (int i = 0; i < n; ++i) {
+    dc_stream* s = streams[i];
+    if (!s) return DC_ERR_ARG;
+    if (s->closed || s->poisoned || s->model != m) return DC_ERR_STATE;
+    if (!feats[i] || !out[i] || n_frames[i] < 1) {
+      m->counters[3]++;
+      return DC_ERR_ARG;
+    }
+    for (int j = 0; j < i; ++j)
+      if (streams[j] == s) {
+        m->counters[3]++;
+        dc::set_error("stream %d appears twice in the batch", i);
+        return DC_ERR_ARG;
+      }
+  }
+  cudaStream_t cs = (cudaStream_t)cuda_stream;
+  const int fc = m->cfg.f_chunk;
+  dc_model* fm = m->sub_flow ? m->sub_flow : m;
+  std::vector<dc::FlowState*> states((size_t)n);
+  std::vector<float*> mels((size_t)n);
+  for (int i = 0; i < n; ++i) states[(size_t)i] = m->sub_flow ? streams[i]->sub_flow->flow : streams[i]->flow;
+  dc_status st = DC_OK;
   int launches = 0;
-  dc_status st = dc::flow_decode_wave(m->flow, s->flow, feats, m->in_dim, n_frames, out, cs, &launches, on_chunk, ctx);
-  m->counters[5] += (uint64_t)launches;
-  if (st == DC_ERR_ARG) {   // refused before anything ran (max_batch < n_steps): the stream is untouched
+  if (m->sub_flow) {
+    // each stream's mel frames stay on the device, in a buffer of the stream; its vocoder tails run on a
+    // CUDA stream of its own
+    for (int i = 0; i < n; ++i) {
+      dc_stream* s = streams[i];
+      if (s->wave_mel_frames < n_frames[i]) {
+        if (s->wave_mel) cudaFree(s->wave_mel);
+        s->wave_mel = nullptr;
+        s->wave_mel_frames = 0;
+        if (cudaMalloc(&s->wave_mel, (size_t)n_frames[i] * m->cfg.mel_dim * sizeof(float)) != cudaSuccess) {
+          cudaGetLastError();
+          return DC_ERR_OOM;
+        }
+        s->wave_mel_frames = n_frames[i];
+      }
+      if (!s->wave_side && (cudaStreamCreateWithFlags(&s->wave_side, cudaStreamNonBlocking) != cudaSuccess ||
+                            cudaEventCreateWithFlags(&s->wave_ev, cudaEventDisableTiming) != cudaSuccess)) {
+        cudaGetLastError();
+        return DC_ERR_CUDA;
+      }
+      mels[(size_t)i] = s->wave_mel;
+    }
+    WaveTail w{streams, cs, !(m->sub_voc->prof.on || m->sub_flow->prof.on), out, n_frames};
+    st = dc::flow_decode_wave(fm->flow, n, states.data(), feats, fm->in_dim, n_frames, mels.data(), cs, &launches, wave_tail_chunk, &w);
+    if (st == DC_OK) st = w.st;
+    for (int i = 0; i < n && st == DC_OK && w.side; ++i)   // the caller's stream continues only after every stream's last tail
+      if (cudaEventRecord(streams[i]->wave_ev, streams[i]->wave_side) != cudaSuccess ||
+          cudaStreamWaitEvent(cs, streams[i]->wave_ev, 0) != cudaSuccess)
+        st = DC_ERR_CUDA;
+  } else {
+    st = dc::flow_decode_wave(fm->flow, n, states.data(), feats, fm->in_dim, n_frames, out, cs, &launches, nullptr, nullptr);
+  }
+  fm->counters[5] += (uint64_t)launches;
+  if (st == DC_ERR_ARG) {   // refused before anything ran: the streams are untouched
     m->counters[3]++;
     return st;
   }
   if (st != DC_OK) {
-    s->poisoned = true;
+    for (int i = 0; i < n; ++i) {
+      streams[i]->poisoned = true;
+      if (m->sub_flow) streams[i]->sub_flow->poisoned = true;
+    }
     return st;
   }
-  const long long n_chunks = (n_frames + m->cfg.f_chunk - 1) / m->cfg.f_chunk;
-  s->frames_total += n_frames;
-  s->chunks += n_chunks;
-  m->counters[0] += (uint64_t)n_chunks;
-  m->counters[1] += (uint64_t)n_frames;
-  return DC_OK;
-}
-
-namespace {
-// Host-side hook of the composite's wavefront: as soon as the pass that finishes chunk j is enqueued, the
-// vocoder tail of chunk j is enqueued on the side stream behind an event, so that it runs beside the flow
-// decoder's next passes (which leave most SMs idle) instead of after them.
-struct WaveTail {
-  dc_stream*   s;
-  cudaStream_t main_st, side;
-  float*       out;
-  long long    n_frames;
-  dc_status    st = DC_OK;
-};
-
-void wave_tail_chunk(void* ctx, long long j) {
-  WaveTail* w = static_cast<WaveTail*>(ctx);
-  if (w->st != DC_OK) return;
-  dc_stream* s = w->s;
-  dc_model* m = s->model;
-  const int fc = m->cfg.f_chunk;
-  const int T = (int)(w->n_frames - j * fc < fc ? w->n_frames - j * fc : fc);
-  if (w->side != w->main_st) {
-    if (cudaEventRecord(s->wave_ev, w->main_st) != cudaSuccess || cudaStreamWaitEvent(w->side, s->wave_ev, 0) != cudaSuccess) {
-      w->st = DC_ERR_CUDA;
-      return;
+  for (int i = 0; i < n; ++i) {
+    const long long n_chunks = (n_frames[i] + fc - 1) / fc;
+    for (dc_stream* s : {streams[i], m->sub_flow ? streams[i]->sub_flow : (dc_stream*)nullptr}) {
+      if (!s) continue;
+      s->frames_total += n_frames[i];
+      s->chunks += n_chunks;
+      s->model->counters[0] += (uint64_t)n_chunks;
+      s->model->counters[1] += (uint64_t)n_frames[i];
     }
   }
-  w->st = dc_decode_chunk(s->sub_voc, s->wave_mel + j * fc * m->cfg.mel_dim, T, w->out + j * fc * m->out_per_frame, nullptr, (void*)w->side);
+  return DC_OK;
 }
-}  // namespace
 
 extern "C" dc_status dc_decode_wavefront(dc_stream* s, const float* feats, long long n_frames, float* out, long long* n_out,
                                          void* cuda_stream) {
   if (!s) return DC_ERR_ARG;
   if (s->closed || s->poisoned) return DC_ERR_STATE;
-  dc_model* m = s->model;
-  if (!feats || !out || n_frames < 1) {
-    m->counters[3]++;
-    return DC_ERR_ARG;
-  }
-  if (!m->flow && !m->sub_flow) {
-    dc::set_error("dc_decode_wavefront serves the flow and token2wav pipelines only");
-    return DC_ERR_CONFIG;
-  }
-  cudaStream_t cs = (cudaStream_t)cuda_stream;
-  const int fc = m->cfg.f_chunk;
-  const long long n_chunks = (n_frames + fc - 1) / fc;
-  dc_status st = DC_OK;
-  if (m->sub_flow) {
-    if (m->cfg.max_batch < m->cfg.n_steps) {
-      m->counters[3]++;
-      dc::set_error("wavefront decoding keeps n_steps = %d chunks in flight: max_batch must be >= n_steps", m->cfg.n_steps);
-      return DC_ERR_ARG;
-    }
-    // the call's mel frames stay on the device, in a buffer of the stream
-    if (s->wave_mel_frames < n_frames) {
-      if (s->wave_mel) cudaFree(s->wave_mel);
-      s->wave_mel = nullptr;
-      s->wave_mel_frames = 0;
-      if (cudaMalloc(&s->wave_mel, (size_t)n_frames * m->cfg.mel_dim * sizeof(float)) != cudaSuccess) {
-        cudaGetLastError();
-        return DC_ERR_OOM;
-      }
-      s->wave_mel_frames = n_frames;
-    }
-    if (!s->wave_side) {
-      if (cudaStreamCreateWithFlags(&s->wave_side, cudaStreamNonBlocking) != cudaSuccess ||
-          cudaEventCreateWithFlags(&s->wave_ev, cudaEventDisableTiming) != cudaSuccess) {
-        cudaGetLastError();
-        return DC_ERR_CUDA;
-      }
-    }
-    // while profiling, everything stays on the caller's stream (the event brackets assume one stream)
-    WaveTail w{s, cs, (m->sub_voc->prof.on || m->sub_flow->prof.on) ? cs : s->wave_side, out, n_frames};
-    st = wave_flow(s->sub_flow, feats, n_frames, s->wave_mel, cs, wave_tail_chunk, &w);
-    if (st == DC_OK) st = w.st;
-    if (st == DC_OK && w.side != cs) {   // the caller's stream continues only after the last vocoder chunk
-      if (cudaEventRecord(s->wave_ev, w.side) != cudaSuccess || cudaStreamWaitEvent(cs, s->wave_ev, 0) != cudaSuccess) st = DC_ERR_CUDA;
-    }
-    if (st != DC_OK) {
-      s->poisoned = true;
-      return st;
-    }
-    s->frames_total += n_frames;
-    s->chunks += n_chunks;
-    m->counters[0] += (uint64_t)n_chunks;
-    m->counters[1] += (uint64_t)n_frames;
-  } else {
-    st = wave_flow(s, feats, n_frames, out, cs, nullptr, nullptr);
-    if (st != DC_OK) return st;
-  }
-  if (n_out) *n_out = n_frames * m->out_per_frame;
-  return DC_OK;
+  dc_status st = dc_decode_wavefront_batch(s->model, 1, &s, &feats, &n_frames, &out, cuda_stream);
+  if (st == DC_OK && n_out) *n_out = n_frames * s->model->out_per_frame;
+  return st;
 }
 
 extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* streams, const float* const* feats,

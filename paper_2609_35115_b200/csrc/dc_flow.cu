@@ -1357,6 +1357,9 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
       // a single stream, and the full batch
       const bool g1 = build_graph(m, m->n_pass);   // a single stream
       const bool gs = m->S > m->n_pass ? build_graph(m, m->S) : g1;
+      // ... and one pass of the network over n_steps chunks (wavefront decoding), where the model has room for it
+      const int n_wave = cfg.n_steps * m->n_pass;
+      if (n_wave <= m->S && n_wave <= MAX_SLOTS_PER_SET) build_graph(m, n_wave, true);
       if (getenv("DC_VERBOSE"))
         fprintf(stderr, "[dc] graphs: n=1 %s, n=%d %s, pdl %d/%d\n", g1 ? "ok" : "none", m->S, gs ? "ok" : "none",
                 g1 ? (int)m->graphs[m->n_pass].pdl : -1, gs ? (int)m->graphs[m->S].pdl : -1);
@@ -1736,43 +1739,49 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
   return DC_OK;
 }
 
-// Wavefront decoding of ONE stream whose input is all there: chunk j runs its Euler step s in tick j + s,
-// so a tick is one pass of the network over n_steps consecutive chunks, each at its own step.  Chunk j at
-// step s needs the step-s carries that chunk j-1 left one tick earlier, and chunks that share a tick use the
-// carries of different steps, so every tick is free of read/write conflicts.  A chunk keeps slot
-// (j mod n_steps) for its n_steps ticks (its Euler state lives there); slots of chunks not yet started or already
-// finished are holes (T = 0).  The arithmetic of a slot never depends on what the other slots hold, so the
-// result equals chunk-by-chunk decoding bit for bit.
-dc_status flow_decode_wave(FlowModel* m, FlowState* s, const float* feats, int in_dim, long long n_frames, float* out,
-                           cudaStream_t st, int* launches, void (*on_chunk)(void*, long long), void* hook_ctx) {
+// Wavefront decoding of streams whose input is all there: chunk j of a stream runs its Euler step s in tick
+// j + s, so a tick is one pass of the network over n_steps consecutive chunks of every stream, each at its own
+// step.  Chunk j at step s needs the step-s carries that chunk j-1 left one tick earlier, and chunks that share a
+// tick use the carries of different steps, so every tick is free of read/write conflicts.  A chunk keeps slot
+// (j mod n_steps) of its stream's slots for its n_steps ticks (its Euler state lives there); slots of chunks not
+// yet started or already finished are holes (T = 0).  The arithmetic of a slot never depends on what the other
+// slots hold, so the result equals chunk-by-chunk decoding bit for bit.
+dc_status flow_decode_wave(FlowModel* m, int n_streams, FlowState* const* states, const float* const* feats, int in_dim,
+                           const long long* n_frames, float* const* outs, cudaStream_t st, int* launches,
+                           void (*on_chunk)(void*, int, long long), void* hook_ctx) {
   const dc_config& c = m->cfg;
   const int np = m->n_pass, K = c.n_steps;
-  const int n = K * np;                                   // slots of a tick
-  if (n > m->S || n > MAX_SLOTS_PER_SET) {
-    set_error("wavefront decoding keeps n_steps = %d chunks in flight: max_batch must be >= n_steps", K);
+  const int n = n_streams * K * np;                       // slots of a tick
+  if (n_streams < 1 || n > m->S || n > MAX_SLOTS_PER_SET) {
+    set_error("wavefront decoding keeps n_steps = %d chunks per stream in flight: %d streams need max_batch >= %d (and at most %d slots)",
+              K, n_streams, n_streams * K, MAX_SLOTS_PER_SET);
     return DC_ERR_ARG;
   }
-  const long long n_chunks = (n_frames + c.f_chunk - 1) / c.f_chunk;
+  long long max_chunks = 0;
+  for (int i = 0; i < n_streams; ++i) {
+    const long long nc = (n_frames[i] + c.f_chunk - 1) / c.f_chunk;
+    if (nc > max_chunks) max_chunks = nc;
+  }
   const bool profiling = m->prof != nullptr && m->prof->on;
-  auto it = m->graphs.find(-n);
+  auto it = m->graphs.find(-n);   // one stream: captured at create; other stream counts: at their first call
   if (it == m->graphs.end() && !profiling && build_graph(m, n, true)) it = m->graphs.find(-n);
-  const long long frames0 = s->frames;
-  const size_t halo_pass = s->halo_bytes / sizeof(bf16) / np, kv_pass = s->kv_bytes / sizeof(bf16) / np;
   const size_t halo_step = (size_t)c.n_conv * HALO * m->C, kv_step = (size_t)c.n_attn * 2 * (m->P + m->Rk) * m->C;
   SlotSet& set = m->sets[0];
-  for (long long t = 0; t < n_chunks + K - 1; ++t) {
+  for (long long t = 0; t < max_chunks + K - 1; ++t) {
     set.first = 0;
     set.count = n;
     for (int i = 0; i < n; ++i) {
       SlotInfo& si = set.s[i];
       si = SlotInfo{};
-      const int ring = i / np, pass = i % np;
+      const int stream = i / (K * np), ring = (i / np) % K, pass = i % np;
+      const FlowState* s = states[stream];
+      const long long n_chunks = (n_frames[stream] + c.f_chunk - 1) / c.f_chunk;
       // the chunk that owns ring slot `ring` in tick t: the largest j <= t with j = ring (mod K)
       const long long j = t - (((t - ring) % K) + K) % K;
       const long long step = t - j;
       if (j < 0 || j >= n_chunks || step >= K) continue;                  // hole
-      const long long f0 = j * c.f_chunk, left = n_frames - f0;
-      const long long frames = frames0 + f0;
+      const long long f0 = j * c.f_chunk, left = n_frames[stream] - f0;
+      const long long frames = s->frames + f0;
       si.T = (int)(left < c.f_chunk + c.f_lookahead ? left : c.f_chunk + c.f_lookahead);
       si.Tc = si.T < c.f_chunk ? si.T : c.f_chunk;
       const long long hist = frames > m->P ? frames - m->P : 0;
@@ -1784,10 +1793,10 @@ dc_status flow_decode_wave(FlowModel* m, FlowState* s, const float* feats, int i
       si.tau_off = (int)(step * c.n_conv * m->C);
       si.flags = (step == 0 ? SLOT_FIRST : 0) | (step == K - 1 ? SLOT_LAST : 0);
       si.pass = pass;
-      si.feats = feats + f0 * in_dim;
-      si.out = pass == 0 ? out + f0 * m->mel : nullptr;
-      si.halo = s->halo + (size_t)pass * halo_pass + (size_t)step * halo_step;
-      si.kv = s->kv ? s->kv + (size_t)pass * kv_pass + (size_t)step * kv_step : nullptr;
+      si.feats = feats[stream] + f0 * in_dim;
+      si.out = pass == 0 ? outs[stream] + f0 * m->mel : nullptr;
+      si.halo = s->halo + (size_t)pass * (s->halo_bytes / sizeof(bf16) / np) + (size_t)step * halo_step;
+      si.kv = s->kv ? s->kv + (size_t)pass * (s->kv_bytes / sizeof(bf16) / np) + (size_t)step * kv_step : nullptr;
     }
     if (!profiling && it != m->graphs.end()) {
       GraphEntry& ge = it->second;
@@ -1813,9 +1822,11 @@ dc_status flow_decode_wave(FlowModel* m, FlowState* s, const float* feats, int i
         return DC_ERR_CUDA;
       }
     }
-    if (on_chunk && t >= K - 1) on_chunk(hook_ctx, t - (K - 1));   // that chunk's last Euler step is now enqueued
+    if (on_chunk && t >= K - 1)   // the last Euler step of every stream's chunk t - (K - 1) is now enqueued
+      for (int i = 0; i < n_streams; ++i)
+        if (t - (K - 1) < (n_frames[i] + c.f_chunk - 1) / c.f_chunk) on_chunk(hook_ctx, i, t - (K - 1));
   }
-  s->frames = frames0 + n_frames;
+  for (int i = 0; i < n_streams; ++i) states[i]->frames += n_frames[i];
   return DC_OK;
 }
 

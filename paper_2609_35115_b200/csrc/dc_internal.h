@@ -116,12 +116,13 @@ const int* flow_error_word(const FlowModel* m);   // device address of that word
 // One chunk for each of n streams.  Returns the number of kernel launches through *launches.
 dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats_dev,
                       const int* n_frames, float* const* out_dev, cudaStream_t st, int* launches);
-// All of one stream's remaining input at once, n_steps chunks in flight (one per Euler step); same bytes as
-// chunk-by-chunk decoding.  feats rows are in_dim floats wide; out receives n_frames mel rows.  on_chunk (may be
-// null) is called on the host with (hook_ctx, j) right after the pass that finishes chunk j has been enqueued.
-dc_status flow_decode_wave(FlowModel* m, FlowState* s, const float* feats_dev, int in_dim, long long n_frames,
-                           float* out_dev, cudaStream_t st, int* launches, void (*on_chunk)(void*, long long) = nullptr,
-                           void* hook_ctx = nullptr);
+// All of the remaining input of n_streams streams at once, n_steps chunks per stream in flight (one per Euler
+// step); same bytes as chunk-by-chunk decoding.  feats rows are in_dim floats wide; outs[i] receives n_frames[i]
+// mel rows.  on_chunk (may be null) is called on the host with (hook_ctx, stream index, j) right after the pass that
+// finishes chunk j of that stream has been enqueued.
+dc_status flow_decode_wave(FlowModel* m, int n_streams, FlowState* const* states, const float* const* feats_dev, int in_dim,
+                           const long long* n_frames, float* const* outs_dev, cudaStream_t st, int* launches,
+                           void (*on_chunk)(void*, int, long long) = nullptr, void* hook_ctx = nullptr);
 
 // Event-bracketed launches while profiling is on (see dc_profile_begin in dc.h).
 struct Profiler {

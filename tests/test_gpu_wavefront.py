@@ -160,3 +160,46 @@ def test_wavefront_needs_room_for_n_steps_chunks(dc):
     st.close()
     m.destroy()
     assert np.array_equal(got, ref)
+
+
+def _batch_case(dc, cfg, lengths, tok2wav=False):
+    """Several streams of different lengths decoded by one dc_decode_wavefront_batch call, each against its own
+    chunk-by-chunk run."""
+    gu = _gu()
+    bounds = [_uniform(n, cfg.f_chunk) for n in lengths]
+    cfgn = cfg.replace(n_streams=len(lengths), n_chunks=max(len(b) for b in bounds) - 1)
+    w = wl.make_workload(cfgn, boundaries=bounds)
+    m = dc.Model(cfgn, w.weights, max_batch=len(lengths) * cfg.n_steps)
+    refs = [gu.run_gpu_stream(m, s.feats[:n], b) for s, n, b in zip(w.streams, lengths, bounds)]
+    sts = [m.open_stream() for _ in lengths]
+    xs = [torch.from_numpy(np.ascontiguousarray(s.feats[:n])).cuda() for s, n in zip(w.streams, lengths)]
+    outs = dc.decode_wavefront_batch(m, sts, xs)
+    torch.cuda.synchronize()
+    assert m.counters()[4] == 0
+    for i, (o, r) in enumerate(zip(outs, refs)):
+        assert np.array_equal(o.cpu().numpy(), r), f"{cfg.name}: stream {i}"
+    # one stream too many for the model's slots: refused, nothing touched
+    if not tok2wav:
+        extra = m.open_stream()
+        with pytest.raises(dc.DCError):
+            dc.decode_wavefront_batch(m, sts + [extra], xs + [xs[0]])
+        extra.close()
+    for st in sts:
+        st.close()
+    m.destroy()
+
+
+def test_wavefront_batch_of_streams(dc):
+    _batch_case(dc, wl.tiny_flow(), [87, 34, 120])
+
+
+def test_wavefront_batch_guided_prompt_lookahead(dc):
+    _batch_case(dc, wl.tiny_flow(f_lookahead=3, f_prompt=17, cfg_scale=0.7), [63, 87])
+
+
+def test_wavefront_batch_token2wav(dc):
+    _batch_case(dc, wl.tiny_token2wav(), [87, 34, 55], tok2wav=True)
+
+
+def test_wavefront_batch_cfg3_size(dc):
+    _batch_case(dc, wl.CONFIGS["cfg3"], [12 * 50, 9 * 50 + 20, 14 * 50 + 7])
