@@ -431,7 +431,8 @@ def main():
         roof = {"kernel": "flow_attn_kernel", "bound": "hbm", "achieved": by / avg_s / 1e9, "peak": pk["hbm_gbs"],
                 "unit": "GB/s", "peak_kind": f"copy bandwidth, {how}"}
     elif dom == "tapconv_f32":
-        fl_chunk = {"cfg4": 1.73e9, "cfg1": 0.79e6}.get(cfg.name, 0.0)
+        # per stream-chunk; the token2wav workloads carry cfg4's vocoder tail behind every stream
+        fl_chunk = S * (1.73e9 if cfg.pipeline in ("vocoder", "token2wav") else 0.79e6)
         roof = {"kernel": "tapconv_f32_kernel", "bound": "alu", "achieved": fl_chunk / (1e-3 * ms[dom] / nprof) / 1e12,
                 "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s", "peak_kind": "FP32 FFMA, derived: 148 SM x 128 x 2 x 1.965 GHz"}
     else:
