@@ -221,15 +221,21 @@ dc_status dc_decode_wavefront_batch(dc_model* model, int n, dc_stream* const* st
 
 /* Convenience for callers with host buffers: copies feats_host to the device,
  * decodes, copies the result back and synchronises cuda_stream.  Uses staging
- * buffers owned by the stream (allocated at dc_stream_open).  Returns DC_ERR_TIMEOUT
- * (and poisons the stream until dc_stream_reset) if a bounded device-side wait gave up. */
+ * buffers owned by the stream (allocated at dc_stream_open).  Flow pipeline: a caller buffer that
+ * is page-locked (cudaHostAlloc / cudaHostRegister, checked per call) is not staged at all - the
+ * kernels read the chunk from it and write the mel rows into it across the bus.  Returns
+ * DC_ERR_TIMEOUT (and poisons the stream until dc_stream_reset) if a bounded device-side wait
+ * gave up. */
 dc_status dc_decode_chunk_host(dc_stream* stream, const float* feats_host, int n_frames,
                                float* out_host, int* n_out, void* cuda_stream);
 
 /* dc_decode_batch for callers with host buffers: feats_host[i] / out_host[i] are host
- * pointers (pageable or pinned).  Gathers the chunks in a pinned buffer owned by the model,
- * moves them to the device in one transfer, decodes the batch, brings all results back in one
- * transfer, synchronises cuda_stream and scatters them.  Returns DC_ERR_TIMEOUT (and poisons the
+ * pointers (pageable or pinned).  If every input (every output) buffer is page-locked, the
+ * kernels read the chunks from (write the results into) the caller's buffers directly, with no
+ * staging copy and no copy-engine transfer on that side.  Otherwise the call gathers the chunks
+ * in a pinned buffer owned by the model, moves them to the device in one transfer, decodes the
+ * batch, brings all results back in one transfer and scatters them.  Either way it synchronises
+ * cuda_stream before it returns.  Returns DC_ERR_TIMEOUT (and poisons the
  * streams) if a bounded device-side wait gave up.  Calls on one model must not overlap. */
 dc_status dc_decode_batch_host(dc_model* model, int n, dc_stream* const* streams,
                                const float* const* feats_host, const int* n_frames,

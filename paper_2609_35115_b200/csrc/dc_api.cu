@@ -67,7 +67,8 @@ struct dc_model {
   float*    d_w = nullptr;   // fp32 pipelines: the blob on the device
   // flow pipeline: staging of dc_decode_batch_host (pinned host + device, max_batch chunks each way)
   float *h_in = nullptr, *h_out = nullptr, *d_in = nullptr, *d_out = nullptr;
-  int*   h_err = nullptr;   // fp32 pipelines: per-call record read by the captured graphs
+  bool   zero_copy = true;   // dc_decode_batch_host: kernels access page-locked caller buffers directly
+  int*   h_err = nullptr;   // pinned: the device error word, read back by the host-buffer calls
   std::vector<F32Layer> layers;
   int       out_per_frame = 0;
   int       in_dim = 0;
@@ -328,6 +329,10 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
       cudaError_t e = cudaMallocHost(&m->h_in, ni * sizeof(float));
       if (e == cudaSuccess) e = cudaMallocHost(&m->h_out, no * sizeof(float));
       if (e == cudaSuccess) e = cudaMallocHost(&m->h_err, sizeof(int));
+      {
+        const char* z = getenv("DC_NO_ZEROCOPY");   // experiments: always stage through the bounce buffers
+        m->zero_copy = !(z && atoi(z));
+      }
       if (e == cudaSuccess) e = cudaMalloc(&m->d_in, ni * sizeof(float));
       if (e == cudaSuccess) e = cudaMalloc(&m->d_out, no * sizeof(float));
       if (e != cudaSuccess) {
@@ -1012,21 +1017,32 @@ extern "C" dc_status dc_decode_chunk_host(dc_stream* s, const float* feats_host,
   if (st != DC_OK) return st;
   dc_model* m = s->model;
   cudaStream_t cs = (cudaStream_t)cuda_stream;
-  DC_CUDA(cudaMemcpyAsync(s->stage_in, feats_host, (size_t)T * m->in_dim * sizeof(float), cudaMemcpyHostToDevice, cs));
+  // flow pipeline: page-locked caller buffers are read / written by the kernels themselves (see dc_decode_batch_host)
+  const float* fin = s->stage_in;
+  float* fout = s->stage_out;
+  if (m->flow && m->zero_copy) {
+    cudaPointerAttributes a{};
+    if (cudaPointerGetAttributes(&a, feats_host) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr)
+      fin = static_cast<const float*>(a.devicePointer);
+    if (cudaPointerGetAttributes(&a, out_host) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr)
+      fout = static_cast<float*>(a.devicePointer);
+    cudaGetLastError();
+  }
+  if (fin == s->stage_in)
+    DC_CUDA(cudaMemcpyAsync(s->stage_in, feats_host, (size_t)T * m->in_dim * sizeof(float), cudaMemcpyHostToDevice, cs));
   int n = 0;
-  st = dc_decode_chunk(s, s->stage_in, T, s->stage_out, &n, cuda_stream);
+  st = dc_decode_chunk(s, fin, T, fout, &n, cuda_stream);
   if (st != DC_OK) return st;
-  DC_CUDA(cudaMemcpyAsync(out_host, s->stage_out, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, cs));
+  if (fout == s->stage_out) DC_CUDA(cudaMemcpyAsync(out_host, s->stage_out, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, cs));
+  dc_model* fmod = m->flow ? m : m->sub_flow;   // the model that owns the flow decoder, if any
+  if (fmod && fmod->h_err) DC_CUDA(cudaMemcpyAsync(fmod->h_err, dc::flow_error_word(fmod->flow), sizeof(int), cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaStreamSynchronize(cs));
-  dc::FlowModel* fm = m->flow ? m->flow : (m->sub_flow ? m->sub_flow->flow : nullptr);
-  if (fm) {
-    const int code = dc::flow_take_device_error(fm);
-    if (code != 0) {   // a bounded device-side wait gave up: the chunk's result is not valid
-      m->counters[4]++;
-      s->poisoned = true;
-      dc::set_error("device-side wait timed out (code %d)", code);
-      return DC_ERR_TIMEOUT;
-    }
+  if (fmod && fmod->h_err && *fmod->h_err != 0) {   // a bounded device-side wait gave up: the chunk's result is not valid
+    const int code = dc::flow_take_device_error(fmod->flow);   // reads and clears the word
+    m->counters[4]++;
+    s->poisoned = true;
+    dc::set_error("device-side wait timed out (code %d)", code);
+    return DC_ERR_TIMEOUT;
   }
   if (n_out) *n_out = n;
   return DC_OK;
@@ -1050,13 +1066,41 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
     fin[(size_t)i] = m->d_in + (size_t)i * in_stride;
     fout[(size_t)i] = m->d_out + (size_t)i * out_stride;
   }
-  // one pinned bounce buffer each way: two transfers per step instead of two per stream
-  for (int i = 0; i < n; ++i)
-    memcpy(m->h_in + (size_t)i * in_stride, feats_host[i], (size_t)n_frames[i] * m->in_dim * sizeof(float));
-  DC_CUDA(cudaMemcpyAsync(m->d_in, m->h_in, (size_t)n * in_stride * sizeof(float), cudaMemcpyHostToDevice, cs));
+  // Page-locked caller buffers are read and written by the kernels themselves (the input-preparation kernel
+  // pulls the chunks over the bus, the last output-projection epilogue pushes the mel rows back): no staging
+  // copy and no copy-engine operation on either side.  Pageable buffers go through one pinned bounce buffer
+  // each way: two transfers per step instead of two per stream.
+  bool in_direct = m->zero_copy, out_direct = m->zero_copy;
+  for (int i = 0; i < n && (in_direct || out_direct); ++i) {
+    cudaPointerAttributes a{};
+    if (in_direct) {
+      if (cudaPointerGetAttributes(&a, feats_host[i]) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr) {
+        fin[(size_t)i] = static_cast<const float*>(a.devicePointer);
+      } else {
+        in_direct = false;
+      }
+    }
+    if (out_direct) {
+      if (cudaPointerGetAttributes(&a, out_host[i]) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr) {
+        fout[(size_t)i] = static_cast<float*>(a.devicePointer);
+      } else {
+        out_direct = false;
+      }
+    }
+  }
+  cudaGetLastError();
+  if (!in_direct) {
+    for (int i = 0; i < n; ++i) {
+      fin[(size_t)i] = m->d_in + (size_t)i * in_stride;
+      memcpy(m->h_in + (size_t)i * in_stride, feats_host[i], (size_t)n_frames[i] * m->in_dim * sizeof(float));
+    }
+    DC_CUDA(cudaMemcpyAsync(m->d_in, m->h_in, (size_t)n * in_stride * sizeof(float), cudaMemcpyHostToDevice, cs));
+  }
+  if (!out_direct)
+    for (int i = 0; i < n; ++i) fout[(size_t)i] = m->d_out + (size_t)i * out_stride;
   dc_status st = dc_decode_batch(m, n, streams, fin.data(), n_frames, fout.data(), cuda_stream);
   if (st != DC_OK) return st;
-  DC_CUDA(cudaMemcpyAsync(m->h_out, m->d_out, (size_t)n * out_stride * sizeof(float), cudaMemcpyDeviceToHost, cs));
+  if (!out_direct) DC_CUDA(cudaMemcpyAsync(m->h_out, m->d_out, (size_t)n * out_stride * sizeof(float), cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaMemcpyAsync(m->h_err, dc::flow_error_word(m->flow), sizeof(int), cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaStreamSynchronize(cs));
   if (*m->h_err != 0) {   // a bounded device-side wait gave up: the results are not valid
@@ -1067,9 +1111,10 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
     dc::set_error("device-side wait timed out (code %d)", code);
     return DC_ERR_TIMEOUT;
   }
-  for (int i = 0; i < n; ++i)
-    memcpy(out_host[i], m->h_out + (size_t)i * out_stride,
-           (size_t)(n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk) * m->out_per_frame * sizeof(float));
+  if (!out_direct)
+    for (int i = 0; i < n; ++i)
+      memcpy(out_host[i], m->h_out + (size_t)i * out_stride,
+             (size_t)(n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk) * m->out_per_frame * sizeof(float));
   return DC_OK;
 }
 

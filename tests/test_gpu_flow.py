@@ -269,3 +269,57 @@ def test_device_noise_with_lookahead_prompt_and_guidance(dc):
     m = dc.Model(cfg, w.weights)
     _noise_run(dc, m, cfg, w, w.streams[0], 0)
     m.destroy()
+
+
+# ---- host-buffer batch call: page-locked caller buffers are accessed by the kernels directly, pageable ones
+# ---- go through the model's bounce buffers; the bytes are those of the device-buffer call either way ----
+
+@pytest.mark.parametrize("pinned_in,pinned_out", [(True, True), (False, False), (True, False), (False, True)])
+def test_batch_host_pinned_and_pageable(dc, pinned_in, pinned_out):
+    cfg = wl.tiny_flow(n_streams=3, n_chunks=5)
+    w = wl.make_workload(cfg)
+    gu = _gu()
+    m = dc.Model(cfg, w.weights, max_batch=3)
+    single = [gu.run_gpu_stream(m, s.feats, s.boundaries) for s in w.streams]
+    streams = [m.open_stream() for _ in w.streams]
+    outs = [[] for _ in w.streams]
+    n_rounds = max(len(s.boundaries) - 1 for s in w.streams)
+    for r in range(n_rounds):
+        idx = [i for i, s in enumerate(w.streams) if r < len(s.boundaries) - 1]
+        fs, os_ = [], []
+        for i in idx:
+            b = w.streams[i].boundaries
+            f = torch.from_numpy(np.ascontiguousarray(w.streams[i].feats[b[r]:b[r + 1]]))
+            o = torch.full((b[r + 1] - b[r], cfg.mel_dim), float("nan"))
+            fs.append(f.pin_memory() if pinned_in else f)
+            os_.append(o.pin_memory() if pinned_out else o)
+        dc.decode_batch_host(m, [streams[i] for i in idx], fs, os_)     # returns after the results are in place
+        for i, o in zip(idx, os_):
+            outs[i].append(o.clone())
+    assert m.counters()[4] == 0
+    for st in streams:
+        st.close()
+    m.destroy()
+    for i in range(len(w.streams)):
+        assert np.array_equal(torch.cat(outs[i]).numpy(), single[i]), f"stream {i}"
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_chunk_host_pinned_and_pageable(dc, pinned):
+    cfg = wl.tiny_flow(n_chunks=5)
+    w = wl.make_workload(cfg)
+    s = w.streams[0]
+    m = dc.Model(cfg, w.weights)
+    ref = _gu().run_gpu_stream(m, s.feats, s.boundaries)
+    st = m.open_stream()
+    fin = torch.from_numpy(s.feats)
+    fout = torch.full((s.feats.shape[0], cfg.mel_dim), float("nan"))
+    if pinned:
+        fin, fout = fin.pin_memory(), fout.pin_memory()
+    for c in range(len(s.boundaries) - 1):
+        lo, hi = s.boundaries[c], s.boundaries[c + 1]
+        n = st.decode_chunk_host(fin[lo:hi], fout[lo:hi])
+        assert n == (hi - lo) * cfg.mel_dim
+    st.close()
+    m.destroy()
+    assert np.array_equal(fout.numpy(), ref)
