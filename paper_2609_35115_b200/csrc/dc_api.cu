@@ -709,7 +709,7 @@ static void build_f32_graph(dc_stream* s) {
   if (cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return; }
   // programmatic dependent launch is left off here: measured on the vocoder tail it made the step
   // slower (0.200 ms vs 0.169 ms per chunk), the kernels are too short to gain from early prologues
-  const bool pdl = getenv("DC_F32_PDL") && atoi(getenv("DC_F32_PDL"));
+  const bool pdl = false;
   cudaGraph_t graph = nullptr;
   if (cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
     dc::F32Call dummy{};

@@ -1120,12 +1120,8 @@ struct FlowModel {
   Profiler* prof = nullptr;
   // launch plumbing
   bool pdl = true;                       // programmatic dependent launch between the step's kernels
-  bool one_issuer = false;               // experiments: a single UMMA issuer
   int  kv_rs = 0, kv_hs = 0, dh_shift = 0;   // K/V plane layout (see GemmParams)
   int  n_sm = 148;                       // SMs of the device (read at create)
-  int  force_v = -1;                     // experiments: N-tile variant forced (0: 64, 1: 32, 2: 16 columns)
-  int  qkv_stages = 4;
-  int  wide_stages = 4;                  // 2 or 4 (even, see the stage count rule in enqueue_chunk)
   int  dbg = 0;
   cudaStream_t cap_stream = nullptr;     // used only to capture graphs at create
   std::map<int, GraphEntry> graphs;      // batch size -> captured chunk step
@@ -1333,24 +1329,13 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     m->pdl = !(e && atoi(e));
     const char* d = getenv("DC_GEMM_DBG");
     m->dbg = d ? atoi(d) : 0;
-    {
-      const char* hm = getenv("DC_KV_ROWMAJOR");   // experiments: rows of all heads interleaved
-      const bool head_major = !(hm && atoi(hm)) && m->cfg.head_dim > 0;
-      m->dh_shift = m->cfg.head_dim == 64 ? 6 : 5;
-      m->kv_rs = head_major ? m->cfg.head_dim : m->C;
-      m->kv_hs = head_major ? (m->P + m->Rk) * m->cfg.head_dim : m->cfg.head_dim;
-    }
-    const char* fv = getenv("DC_TILE_V");
-    m->force_v = (fv && fv[0] && atoi(fv) >= 0 && atoi(fv) <= 2) ? atoi(fv) : -1;
+    // K/V planes are head-major: the rows one attention CTA streams are contiguous
+    m->dh_shift = m->cfg.head_dim == 64 ? 6 : 5;
+    m->kv_rs = m->cfg.head_dim;
+    m->kv_hs = (m->P + m->Rk) * m->cfg.head_dim;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
       m->n_sm = sms;
-    const char* oi = getenv("DC_ONE_ISSUER");
-    m->one_issuer = oi && atoi(oi);
-    const char* qs = getenv("DC_QKV_STAGES");
-    if (qs && atoi(qs) >= 2 && atoi(qs) <= 4) m->qkv_stages = atoi(qs);
-    const char* ws = getenv("DC_GEMM_STAGES");
-    if (ws && (atoi(ws) == 2 || atoi(ws) == 4)) m->wide_stages = atoi(ws);
     const char* g = getenv("DC_NO_GRAPH");
     if (!(g && atoi(g)) && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) == cudaSuccess) {
       // the two batch sizes that matter are captured now, so that no decode call ever builds a graph:
@@ -1505,7 +1490,6 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
   // of 16 columns 0.26 ms per pass, 80 CTAs of 32 columns 0.20 ms)
   int v = 2;
   while (v > 0 && m_tiles * (C / (64 >> v)) > m->n_sm) --v;
-  if (m->force_v >= 0) v = m->force_v;
   // the output projection always uses 16-column tiles: mel/16 CTAs per row tile instead of one, and a
   // single Euler-state round trip per epilogue thread
   const int bn = 64 >> v, bq = 192 >> v, bo = 16;
@@ -1522,17 +1506,17 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     // the issuer count fixes the summation order, so it depends on the GEMM's role only, never on the tile
     // width chosen for the batch size (batched and single-stream results must agree bit for bit);
     // the QKV and output projections keep one issuer (their wide tiles would not fit two accumulators)
-    p.n_issuers = (p.mode != MODE_QKV && p.mode != MODE_OUT && p.n_kblocks >= 2 && !m->one_issuer) ? 2 : 1;
+    p.n_issuers = (p.mode != MODE_QKV && p.mode != MODE_OUT && p.n_kblocks >= 2) ? 2 : 1;
     // Stage count.  With two issuers the count must be EVEN: issuer i takes
     // the reduction blocks kb = i (mod 2), and only with an even ring does every stage always belong
     // to the same issuer - a parity wait cannot tell "my block has landed" from "the other issuer's
     // earlier block has landed" on a stage that both use.
     if (p.n_issuers == 2) {
-      p.n_stages = (p.n_kblocks >= 4 && (4 * stage_bytes <= 104 * 1024 || stage_bytes > 32 * 1024)) ? m->wide_stages : 2;
+      p.n_stages = (p.n_kblocks >= 4 && (4 * stage_bytes <= 104 * 1024 || stage_bytes > 32 * 1024)) ? 4 : 2;
     } else {
       p.n_stages = std::max(1, std::min(std::min(MAX_STAGES, GEMM_TILE_SMEM / stage_bytes), p.n_kblocks));
       // the wide QKV tiles fill the GPU with one CTA per SM anyway: a deeper ring hides the load latency
-      if (p.mode == MODE_QKV && stage_bytes > 32 * 1024 && p.n_kblocks >= 4) p.n_stages = m->qkv_stages;
+      if (p.mode == MODE_QKV && stage_bytes > 32 * 1024 && p.n_kblocks >= 4) p.n_stages = 4;
     }
     const size_t smem = GEMM_SMEM_EXTRA + (size_t)p.n_stages * stage_bytes;
     launch(lc, flow_gemm_kernel, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), smem, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
