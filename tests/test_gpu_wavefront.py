@@ -203,3 +203,35 @@ def test_wavefront_batch_token2wav(dc):
 
 def test_wavefront_batch_cfg3_size(dc):
     _batch_case(dc, wl.CONFIGS["cfg3"], [12 * 50, 9 * 50 + 20, 14 * 50 + 7])
+
+
+def test_wavefront_direct_launches_equal_graph(dc):
+    """The wavefront pass as direct launches (a model without graphs, and a profiled call) gives the bytes of
+    the captured pass."""
+    import os
+    gu = _gu()
+    cfg = wl.tiny_flow(f_prompt=17, cfg_scale=0.7)
+    bounds = _uniform(87, cfg.f_chunk)
+    w = wl.make_workload(cfg.replace(n_chunks=len(bounds) - 1), boundaries=[bounds])
+    x = torch.from_numpy(w.streams[0].feats).cuda().contiguous()
+    m = dc.Model(cfg, w.weights, max_batch=cfg.n_steps)
+    st = m.open_stream()
+    ref = st.decode_wavefront(x).cpu().numpy()
+    st.reset()
+    m.profile_begin(4096)
+    got_prof = st.decode_wavefront(x).cpu().numpy()
+    ms, nl = m.profile_end()
+    assert sum(nl.values()) > 0
+    st.close()
+    m.destroy()
+    os.environ["DC_NO_GRAPH"] = "1"
+    try:
+        m2 = dc.Model(cfg, w.weights, max_batch=cfg.n_steps)
+    finally:
+        os.environ.pop("DC_NO_GRAPH", None)
+    st2 = m2.open_stream()
+    got_direct = st2.decode_wavefront(x).cpu().numpy()
+    assert m2.counters()[4] == 0
+    st2.close()
+    m2.destroy()
+    assert np.array_equal(got_prof, ref) and np.array_equal(got_direct, ref)
