@@ -730,7 +730,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   const int slot = blockIdx.x, head = blockIdx.y;
   const int chunks = p.dh >> 3;             // 16-byte chunks per head row
 #ifdef DC_TIMING
-  __shared__ long long a_t[64];
+  long long* a_t = reinterpret_cast<long long*>(s_x + 128);   // 48 stamps in the spare bytes of the barrier area (keeps 2 CTAs per SM)
   const bool atm = blockIdx.x == 3 && blockIdx.y == 2;
   const long long a_start = clock64();
 #define DC_AT(i) do { if (atm) a_t[i] = clock64() - a_start; } while (0)
