@@ -235,3 +235,47 @@ def test_wavefront_direct_launches_equal_graph(dc):
     st2.close()
     m2.destroy()
     assert np.array_equal(got_prof, ref) and np.array_equal(got_direct, ref)
+
+
+def test_wavefront_refusals_leave_the_streams_untouched(dc):
+    """Argument errors of the wavefront calls are refused before anything runs."""
+    gu = _gu()
+    cfg = wl.tiny_flow()
+    w = wl.make_workload(cfg)
+    s = w.streams[0]
+    m = dc.Model(cfg, w.weights, max_batch=2 * cfg.n_steps)
+    other = dc.Model(cfg, w.weights, max_batch=cfg.n_steps)
+    a, b, foreign = m.open_stream(), m.open_stream(), other.open_stream()
+    x = torch.from_numpy(s.feats).cuda().contiguous()
+    with pytest.raises(dc.DCError):                       # the same stream twice
+        dc.decode_wavefront_batch(m, [a, a], [x, x])
+    with pytest.raises(dc.DCError):                       # a stream of another model
+        dc.decode_wavefront_batch(m, [a, foreign], [x, x])
+    with pytest.raises(dc.DCError):                       # no frames
+        dc.decode_wavefront_batch(m, [a], [x[:0].contiguous()])
+    closed = m.open_stream()
+    closed.close()
+    with pytest.raises(dc.DCError):                       # a closed stream
+        dc.decode_wavefront_batch(m, [closed], [x])
+    # a vocoder model has no Euler loop to pipeline
+    vcfg = wl.tiny_vocoder()
+    vw = wl.make_workload(vcfg)
+    vm = dc.Model(vcfg, vw.weights)
+    vs = vm.open_stream()
+    with pytest.raises(dc.DCError):
+        vs.decode_wavefront(torch.from_numpy(vw.streams[0].feats).cuda().contiguous())
+    vs.close()
+    vm.destroy()
+    # after all the refusals the two streams decode from their base state
+    ref = gu.run_gpu_stream(m, s.feats, s.boundaries)
+    got = dc.decode_wavefront_batch(m, [a, b], [x, x])
+    torch.cuda.synchronize()
+    assert m.counters()[4] == 0
+    # (uniform chunks of the default workload: the wavefront cuts the same boundaries)
+    assert s.boundaries == _uniform(s.boundaries[-1], cfg.f_chunk)
+    for o in got:
+        assert np.array_equal(o.cpu().numpy(), ref)
+    for st in (a, b, foreign):
+        st.close()
+    m.destroy()
+    other.destroy()
