@@ -142,6 +142,21 @@ def flops_per_launch(cfg, cls: str, n_streams: int) -> float:
     return 0.0
 
 
+def flow_step_work(cfg, n_streams: int):
+    """Algorithmic FLOPs and HBM bytes of one whole chunk step of a flow decoder (all Euler steps, valid rows)."""
+    rows = n_streams * cfg.f_chunk * (2 if getattr(cfg, "cfg_scale", 0.0) > 0 else 1)
+    C, mel = cfg.hidden, cfg.mel_dim
+    n_conv, n_attn = len(cfg.dilations), cfg.n_attn_layers
+    per_step = (2.0 * rows * 2 * mel * C                       # input projection
+                + n_conv * 2.0 * rows * C * 3 * C              # conv blocks
+                + n_attn * (2.0 * rows * C * 3 * C             # QKV projection
+                            + flops_per_launch(cfg, "attention", n_streams)
+                            + 2.0 * rows * C * C)              # attention output projection
+                + 2.0 * rows * C * mel)                        # output projection
+    by = cfg.n_steps * n_attn * attention_bytes_per_launch(cfg, n_streams)   # the K/V sweeps; weights and activations live in L2
+    return cfg.n_steps * per_step, by
+
+
 def attention_bytes_per_launch(cfg, n_streams: int) -> float:
     """K and V rows of the attended window (bf16) + Q read + O write."""
     L = getattr(cfg, "f_prompt", 0) + cfg.kv_cap + cfg.f_chunk + getattr(cfg, "f_lookahead", 0)
@@ -494,6 +509,12 @@ def main():
             in_graph["attention_hbm_gbs"] = attention_bytes_per_launch(cfg, S) / (us * 1e-6) / 1e9
             in_graph["attention_hbm_frac"] = in_graph["attention_hbm_gbs"] / pk["hbm_gbs"]
         roof["in_graph"] = in_graph
+        # the whole step against the two rooflines (the paper's stage bound, Eq. 1: max of the compute time and
+        # the memory time), next to the per-kernel figures above
+        fl_step, by_step = flow_step_work(cfg, S)   # (token2wav workloads: the flow decoder's part of the work only)
+        t_floor = max(fl_step / (pk["bf16_tflops_sustained"] * 1e12), by_step / (pk["hbm_gbs"] * 1e9))
+        roof["step"] = {"flops": fl_step, "hbm_bytes": by_step, "floor_us": 1e6 * t_floor,
+                        "measured_us": 1e3 * full_ms, "frac": t_floor / (1e-3 * full_ms)}
 
     # ---- the oracle on the host cores (rank 0, N = 1 only), bounded sample ----
     cpu = None
