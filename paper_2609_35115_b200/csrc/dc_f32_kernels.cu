@@ -253,14 +253,20 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
 
 // ---------------------------------------------------------------------------------------------
 
-constexpr int HT = 64;          // threads per CTA of the head kernel
-constexpr int HF = HT - 3;      // new frames per CTA; the first 3 threads recompute the overlap
+constexpr int HFR = 64;         // frames per CTA of the head kernel: 3 recomputed frames of overlap + 61 new ones
+constexpr int HF = HFR - 3;     // new frames per CTA
+constexpr int HQ = 4;           // threads per frame: each reduces a quarter of the channels, then a quarter of the DFT outputs
+constexpr int HT = HFR * HQ;    // threads per CTA
 constexpr int NFFT = 16, NB = 9, NH = 18, HOP = 4, TAIL = NFFT - HOP;
 
 __constant__ float c_cos16[16];  // cos(2 pi j / 16)
 __constant__ float c_sin16[16];
 __constant__ float c_hann16[16];
 
+// One thread per frame left a 3 x C x 18 reduction (3,456 dependent multiply-adds at C = 64) on two warps per CTA:
+// 23 us for 6,000 frames.  Four adjacent lanes share a frame: lane q reduces the channels c = q (mod 4) blocks of
+// four, the partial sums are added across the four lanes in a fixed butterfly (every lane ends with the same
+// bits), and lane q then produces DFT outputs 4q .. 4q + 3 of the frame.
 __global__ void __launch_bounds__(HT) head_istft_f32_kernel(const HeadIstftF32 p_in) {
   extern __shared__ __align__(16) float smem[];
   ptx::pdl_launch();
@@ -276,78 +282,91 @@ __global__ void __launch_bounds__(HT) head_istft_f32_kernel(const HeadIstftF32 p
   }
   if ((int)blockIdx.x * HF >= p.T) return;
   float* Ws = smem;                              // [3*C][NH]
-  float* g = smem + 3 * p.C * NH;                // [HT][NFFT] windowed frame signals
+  float* g = smem + 3 * p.C * NH;                // [HFR][NFFT] windowed frame signals
   const int tid = threadIdx.x;
   for (int i = tid; i < 3 * p.C * NH; i += HT) Ws[i] = p.W[i];
   __syncthreads();
 
-  const int f_local = blockIdx.x * HF + tid - 3;  // frame index within the chunk (may be < 0)
-  const bool is_new = tid >= 3 && f_local < p.T;
+  const int fr = tid / HQ, q = tid % HQ;          // frame slot of the CTA, quarter
+  const int f_local = blockIdx.x * HF + fr - 3;   // frame index within the chunk (may be < 0)
   const bool compute = f_local >= 0 && f_local < p.T;   // frames of earlier chunks come from the tail
-  float gv[NFFT];
+  // (all four lanes of a frame take the same branch, and a warp holds whole frames: the shuffles below are
+  // executed by complete groups)
+  float z[NH];
 #pragma unroll
-  for (int k = 0; k < NFFT; ++k) gv[k] = 0.f;
+  for (int o = 0; o < NH; ++o) z[o] = 0.f;
   if (compute) {
-    float z[NH];
-#pragma unroll
-    for (int o = 0; o < NH; ++o) z[o] = p.bias[o];
     const long long t = p.pos + f_local;
     for (int tap = 0; tap < 3; ++tap) {
       const float* x = p.in_ring + (long long)((int)((t - (2 - tap)) & (long long)p.in_mask)) * p.C;
       const float* w = Ws + tap * p.C * NH;
-      for (int c = 0; c < p.C; c += 4) {
+      for (int c = 4 * q; c < p.C; c += 4 * HQ) {
         const float4 xv = *reinterpret_cast<const float4*>(x + c);
         const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
+        for (int u = 0; u < 4; ++u)
 #pragma unroll
-          for (int o = 0; o < NH; ++o) z[o] = fmaf(xs[q], w[(c + q) * NH + o], z[o]);
+          for (int o = 0; o < NH; ++o) z[o] = fmaf(xs[u], w[(c + u) * NH + o], z[o]);
       }
     }
+  }
+#pragma unroll
+  for (int o = 0; o < NH; ++o) {
+    z[o] += __shfl_xor_sync(0xffffffffu, z[o], 1);
+    z[o] += __shfl_xor_sync(0xffffffffu, z[o], 2);
+  }
+  float gv[NFFT / HQ];
+#pragma unroll
+  for (int k = 0; k < NFFT / HQ; ++k) gv[k] = 0.f;
+  if (compute) {
     float re[NB], im[NB];
 #pragma unroll
     for (int f = 0; f < NB; ++f) {
-      const float mag = expf(fminf(z[f], p.clamp));
-      float s, c;
-      sincosf(z[NB + f], &s, &c);
-      re[f] = mag * c;
-      im[f] = mag * s;
+      const float mag = expf(fminf(z[f] + p.bias[f], p.clamp));
+      float sn, cs;
+      sincosf(z[NB + f] + p.bias[NB + f], &sn, &cs);
+      re[f] = mag * cs;
+      im[f] = mag * sn;
     }
 #pragma unroll
-    for (int k = 0; k < NFFT; ++k) {
+    for (int kk = 0; kk < NFFT / HQ; ++kk) {
+      const int k = q * (NFFT / HQ) + kk;
       float a = re[0] + ((k & 1) ? -re[NB - 1] : re[NB - 1]);
 #pragma unroll
       for (int f = 1; f < NB - 1; ++f) {
         const int j = (f * k) & 15;
         a += 2.0f * (re[f] * c_cos16[j] - im[f] * c_sin16[j]);
       }
-      gv[k] = c_hann16[k] * a * (1.0f / NFFT);
+      gv[kk] = c_hann16[k] * a * (1.0f / NFFT);
     }
   }
 #pragma unroll
-  for (int k = 0; k < NFFT; ++k) g[tid * NFFT + k] = gv[k];
+  for (int kk = 0; kk < NFFT / HQ; ++kk) g[fr * NFFT + q * (NFFT / HQ) + kk] = gv[kk];
   __syncthreads();
 
-  if (is_new) {
+  // overlap-add: one thread per new frame
+  const int fo = tid;                              // frame slot
+  const int fo_local = blockIdx.x * HF + fo - 3;
+  if (tid < HFR && fo >= 3 && fo_local < p.T) {
     const float inv_norm = 1.0f / 1.5f;   // sum of the four overlapping squared Hann windows
     float out[HOP];
 #pragma unroll
     for (int j = 0; j < HOP; ++j) {
       // sample 4 f + j: contributions of frames f, f-1, f-2, f-3 at offsets j, 4+j, 8+j, 12+j;
       // the part that frames of earlier chunks contribute is the carried tail
-      float a = (f_local < 3 && 4 * f_local + j < TAIL) ? p.tail_in[4 * f_local + j] : 0.f;
+      float a = (fo_local < 3 && 4 * fo_local + j < TAIL) ? p.tail_in[4 * fo_local + j] : 0.f;
 #pragma unroll
-      for (int i = 3; i >= 0; --i) a += g[(tid - i) * NFFT + 4 * i + j];
+      for (int i = 3; i >= 0; --i) a += g[(fo - i) * NFFT + 4 * i + j];
       out[j] = a * inv_norm;
     }
-    *reinterpret_cast<float4*>(p.pcm + 4ll * f_local) = make_float4(out[0], out[1], out[2], out[3]);
-    if (f_local == p.T - 1) {
+    *reinterpret_cast<float4*>(p.pcm + 4ll * fo_local) = make_float4(out[0], out[1], out[2], out[3]);
+    if (fo_local == p.T - 1) {
       // tail for the next chunk: samples 4T + q, q in [0,12), from the last three frames
-      for (int q = 0; q < TAIL; ++q) {
+      for (int qq = 0; qq < TAIL; ++qq) {
         float a = 0.f;
         for (int i = 2; i >= 0; --i)
-          if (4 * (i + 1) + q < NFFT) a += g[(tid - i) * NFFT + 4 * (i + 1) + q];
-        p.tail_out[q] = a;
+          if (4 * (i + 1) + qq < NFFT) a += g[(fo - i) * NFFT + 4 * (i + 1) + qq];
+        p.tail_out[qq] = a;
       }
     }
   }
@@ -432,7 +451,7 @@ cudaError_t prepare_f32_constants() {
 
 void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st, int T_grid, bool pdl) {
   if (T_grid < 0) T_grid = p.T;
-  const size_t smem = (size_t)(3 * p.C * NH + HT * NFFT) * sizeof(float);
+  const size_t smem = (size_t)(3 * p.C * NH + HFR * NFFT) * sizeof(float);
   const int grid = (T_grid + HF - 1) / HF;
   launch_ex(head_istft_f32_kernel, dim3(grid), dim3(HT), smem, st, pdl, p);
 }
