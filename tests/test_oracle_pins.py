@@ -581,3 +581,135 @@ def test_philox_known_answers_and_device_noise():
     a = orc.run_stream(la, wk.weights, wk.streams[0].feats, lb)
     b = orc.run_stream(la, wk.weights, wk.streams[0].feats, lb, carry="ring")
     assert np.allclose(a, b, rtol=0, atol=1e-9 * np.abs(a).max())
+
+
+# ---------------------------------------------------------------- vocoder tail as a whole / normal draw
+
+def torch_vocoder_reference(cfg, blob, mel):
+    """Independent library formulation (float64 torch ops) of the whole vocoder tail: conv1d with
+    left padding for the entry conv, the residual blocks and the head, conv_transpose1d with the
+    trailing `stride` samples dropped, F.silu, torch.polar + torch.fft.irfft for the frame
+    synthesis and an explicit overlap-add loop; it walks the weight blob on its own."""
+    Wd, pos = {}, 0
+    for nm, shape, _ in wl.blob_layout(cfg):
+        n = int(np.prod(shape))
+        Wd[nm] = torch.from_numpy(blob[pos:pos + n].astype(np.float64).reshape(shape))
+        pos += n
+    assert pos == blob.size
+
+    def conv3(x, Wn, bn, d):                     # x [C_in, T] -> [C_out, T], causal, taps 2d / d / 0 frames back
+        wt = Wd[Wn].permute(2, 1, 0).contiguous()            # [C_out, C_in, k], k index 2 = current frame
+        return F.conv1d(F.pad(x[None], (2 * d, 0)), wt, Wd[bn], dilation=d)[0]
+
+    a = conv3(torch.from_numpy(np.asarray(mel, np.float64)).T.contiguous(), "pre.W", "pre.b", 1)
+    for q, s in enumerate(cfg.up_strides):
+        wt = Wd[f"up{q}.Wt"].permute(1, 2, 0).contiguous()   # [C_in, C_out, k]
+        a = F.conv_transpose1d(a[None], wt, Wd[f"up{q}.bt"], stride=s)[0][:, :a.shape[1] * s]
+        for r, d in enumerate(cfg.res_dilations):
+            a = a + F.silu(conv3(a, f"up{q}.res{r}.W", f"up{q}.res{r}.b", d))
+    z = conv3(F.silu(a), "head.W", "head.b", 1).T            # [M, n_fft + 2]
+    nb = cfg.n_fft // 2 + 1
+    logmag = torch.clamp(z[:, :nb], max=cfg.logmag_clamp)
+    X = torch.polar(torch.exp(logmag), z[:, nb:].contiguous())
+    xi = torch.fft.irfft(X, n=cfg.n_fft, dim=1)
+    win = torch.hann_window(cfg.n_fft, periodic=True, dtype=torch.float64)
+    M = xi.shape[0]
+    acc = torch.zeros(cfg.hop * M + cfg.n_fft, dtype=torch.float64)
+    env = torch.zeros_like(acc)
+    for m in range(M):
+        acc[cfg.hop * m: cfg.hop * m + cfg.n_fft] += win * xi[m]
+        env[cfg.hop * m: cfg.hop * m + cfg.n_fft] += win * win
+    steady = float(env[cfg.n_fft: cfg.hop * M].mean()) if cfg.hop * M > cfg.n_fft else 1.5
+    return (acc[:cfg.hop * M] / steady).numpy()
+
+
+def _vocoder_case():
+    cfg = wl.tiny_vocoder(bias_std=0.3)
+    w = wl.make_workload(cfg, boundaries=[[0, 5, 10, 15, 20]])
+    return cfg, w.weights, w.streams[0].feats
+
+
+def test_vocoder_offline_matches_library_formulation():
+    """The vocoder tail as a composition: entry conv (no activation) -> (transposed conv -> residual
+    blocks) per stage -> SiLU -> head -> frame synthesis -> overlap-add, against torch's own ops."""
+    cfg, blob, mel = _vocoder_case()
+    assert np.abs(blob[-(cfg.n_fft + 2):]).max() > 0          # biases are not zero in this case
+    mine = orc.vocoder_offline(cfg, blob, mel).astype(np.float64)
+    ref = torch_vocoder_reference(cfg, blob, mel)
+    rms = np.sqrt((ref ** 2).mean())
+    assert mine.shape == ref.shape
+    assert np.abs(mine - ref).max() <= 2e-7 * max(rms, np.abs(ref).max())     # float32 output rounding only
+    # at full precision: the oracle's stages chained by hand, without the float32 output rounding
+    W = orc.parse_blob(cfg, blob)
+    a = orc.causal_conv_k3(mel.astype(np.float64), W["pre.W"], 1) + W["pre.b"]
+    for q, s in enumerate(cfg.up_strides):
+        a = orc.conv_transpose_causal(a, W[f"up{q}.Wt"], W[f"up{q}.bt"], s)
+        for r, d in enumerate(cfg.res_dilations):
+            a = a + orc.silu(orc.causal_conv_k3(a, W[f"up{q}.res{r}.W"], d) + W[f"up{q}.res{r}.b"])
+    z = orc.causal_conv_k3(orc.silu(a), W["head.W"], 1) + W["head.b"]
+    pcm, _ = orc.overlap_add(orc.frame_signal(z, cfg.n_fft, cfg.logmag_clamp), cfg.n_fft, cfg.hop)
+    assert np.abs(pcm - ref).max() <= 1e-9 * max(rms, np.abs(ref).max())
+    assert np.array_equal(pcm.astype(np.float32), orc.vocoder_offline(cfg, blob, mel))
+
+
+@pytest.mark.parametrize("mistake", ["no_silu_before_head", "no_residual_skip", "silu_after_pre", "taps_reversed"])
+def test_vocoder_library_formulation_catches_plausible_mistakes(mistake, monkeypatch):
+    """The pin above has teeth: each of these one-line mistakes in the chain moves the output far
+    beyond the pin's tolerance."""
+    cfg, blob, mel = _vocoder_case()
+    ref = torch_vocoder_reference(cfg, blob, mel)
+    rms = np.sqrt((ref ** 2).mean())
+    silu, conv = orc.silu, orc.causal_conv_k3
+    calls = {"silu": 0, "conv": 0}
+    n_res = len(cfg.up_strides) * len(cfg.res_dilations)
+
+    def silu_m(z):
+        calls["silu"] += 1
+        if mistake == "no_silu_before_head" and calls["silu"] == n_res + 1:
+            return z
+        if mistake == "no_residual_skip" and calls["silu"] == 2:
+            return silu(z) - silu_m.last_in                    # cancels the skip of the second block
+        return silu(z)
+
+    def conv_m(x, W, d, left=None):
+        calls["conv"] += 1
+        silu_m.last_in = x
+        if mistake == "taps_reversed" and calls["conv"] == 2:
+            W = W[::-1]
+        y = conv(x, W, d, left)
+        if mistake == "silu_after_pre" and calls["conv"] == 1:
+            return silu(y)                                     # bias added after, close enough to the mistake
+        return y
+
+    monkeypatch.setattr(orc, "silu", silu_m)
+    monkeypatch.setattr(orc, "causal_conv_k3", conv_m)
+    wrong = orc.vocoder_offline(cfg, blob, mel).astype(np.float64)
+    assert np.abs(wrong - ref).max() > 1e-3 * rms
+
+
+def test_device_noise_single_values_by_hand():
+    """Two frames of the normal draw computed here from the pinned generator words: the uniform
+    map u = ((r >> 8) + 1/2) 2^-24, the pairing (u0, u1) / (u2, u3) and cos before sin."""
+    seed, sid, mel = 0x1234567890, 5, 8
+    got = orc.device_noise(seed, sid, 41, 2, mel)
+    assert got.shape == (2, mel)
+    for i, t in enumerate((41, 42)):
+        for g in range(mel // 4):
+            words = orc.philox4x32_10(np.array([t, 0, g, sid], dtype=np.uint32), (seed & 0xFFFFFFFF, seed >> 32))
+            u = [((int(r) >> 8) + 0.5) * 2.0 ** -24 for r in words]
+            want = [math.sqrt(-2.0 * math.log(u[0])) * math.cos(2.0 * math.pi * u[1]),
+                    math.sqrt(-2.0 * math.log(u[0])) * math.sin(2.0 * math.pi * u[1]),
+                    math.sqrt(-2.0 * math.log(u[2])) * math.cos(2.0 * math.pi * u[3]),
+                    math.sqrt(-2.0 * math.log(u[2])) * math.sin(2.0 * math.pi * u[3])]
+            assert np.allclose(got[i, 4 * g: 4 * g + 4], want, rtol=0, atol=1e-12)
+    # the known-answer counter (0,0,0,0) under key (0,0): the first frame, first channel group of stream 0, seed 0
+    r = [0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8]
+    u = [((x >> 8) + 0.5) / 16777216.0 for x in r]
+    z0 = orc.device_noise(0, 0, 0, 1, 4)[0]
+    assert math.isclose(z0[0], math.sqrt(-2 * math.log(u[0])) * math.cos(2 * math.pi * u[1]), abs_tol=1e-12)
+    assert math.isclose(z0[3], math.sqrt(-2 * math.log(u[2])) * math.sin(2 * math.pi * u[3]), abs_tol=1e-12)
+    # a frame clock beyond 2^32 moves into the second counter word
+    big = orc.device_noise(3, 1, (1 << 32) + 7, 1, 4)[0]
+    w = orc.philox4x32_10(np.array([7, 1, 0, 1], dtype=np.uint32), (3, 0))
+    assert math.isclose(big[0], math.sqrt(-2 * math.log(((int(w[0]) >> 8) + 0.5) / 2 ** 24))
+                        * math.cos(2 * math.pi * ((int(w[1]) >> 8) + 0.5) / 2 ** 24), abs_tol=1e-12)
