@@ -379,7 +379,7 @@ def main():
     wave = None
     if has_flow and S == 1 and world == 1:
         n_wc = 200
-        mw = dc.Model(cfg, weights, max_batch=cfg.n_steps)
+        mw = dc.Model(cfg, weights, max_batch=cfg.n_steps, max_wave_frames=n_wc * T if cfg.pipeline == "token2wav" else 0)
         sw = mw.open_stream()
         fw = torch.from_numpy(rng.standard_normal((n_wc * T, cfg.in_dim), dtype=np.float32)).cuda()
         ow = torch.empty(n_wc * T * cfg.out_per_frame, device="cuda")
@@ -406,7 +406,7 @@ def main():
         n_pass = 2 if getattr(cfg, "cfg_scale", 0.0) > 0 else 1
         n_ws = min(3, 64 // (cfg.n_steps * n_pass))
         if n_ws >= 2:
-            mb = dc.Model(cfg, weights, max_batch=n_ws * cfg.n_steps)
+            mb = dc.Model(cfg, weights, max_batch=n_ws * cfg.n_steps, max_wave_frames=n_wc * T if cfg.pipeline == "token2wav" else 0)
             sb = [mb.open_stream() for _ in range(n_ws)]
             fb = [torch.from_numpy(rng.standard_normal((n_wc * T, cfg.in_dim), dtype=np.float32)).cuda() for _ in range(n_ws)]
             ob = [torch.empty(n_wc * T * cfg.out_per_frame, device="cuda") for _ in range(n_ws)]
@@ -464,15 +464,11 @@ def main():
     # The event-bracketed pass above times direct launches: every bracket adds launch latency and
     # takes away the overlap between consecutive kernels.  What a class costs in the real step is the
     # step time with it minus the step time without it: the library can leave a class out of the
-    # graph (environment variable read at dc_create; the outputs are then meaningless, the timing
+    # graph (a measurement-only option of dc_create; the outputs are then meaningless, the timing
     # of everything else is not).
     if has_flow and world == 1:
         def step_ms_without(bits: int) -> float:
-            os.environ["DC_GEMM_DBG"] = str(bits)
-            try:
-                m2 = dc.Model(cfg, weights, max_batch=S)
-            finally:
-                os.environ.pop("DC_GEMM_DBG", None)
+            m2 = dc.Model(cfg, weights, max_batch=S, options=bits)
             st2 = [m2.open_stream() for _ in range(S)]
             def step2(r):
                 if batched:
@@ -499,12 +495,12 @@ def main():
         n_att_l = kernels.get("attention", {}).get("launches_per_step", 0)
         in_graph = {"method": "step time minus the step time of a graph without the class, both over CUDA events"}
         if n_conv_l:
-            us = 1e3 * (full_ms - step_ms_without(1024)) / n_conv_l
+            us = 1e3 * (full_ms - step_ms_without(dc.OPT_SKIP_CONV_GEMM)) / n_conv_l
             in_graph["conv_gemm_us"] = us
             in_graph["conv_gemm_tflops"] = flops_per_launch(cfg, "gemm_conv", S) / (us * 1e-6) / 1e12
             in_graph["conv_gemm_frac"] = in_graph["conv_gemm_tflops"] / pk["bf16_tflops_sustained"]
         if n_att_l:
-            us = 1e3 * (full_ms - step_ms_without(32)) / n_att_l
+            us = 1e3 * (full_ms - step_ms_without(dc.OPT_SKIP_ATTENTION)) / n_att_l
             in_graph["attention_us"] = us
             in_graph["attention_hbm_gbs"] = attention_bytes_per_launch(cfg, S) / (us * 1e-6) / 1e9
             in_graph["attention_hbm_frac"] = in_graph["attention_hbm_gbs"] / pk["hbm_gbs"]

@@ -18,6 +18,13 @@
  *   - "dev" pointers are device pointers valid on the model's device, "host"
  *     pointers are ordinary host pointers.  The library never takes ownership
  *     of a caller buffer.
+ *   - Alignment: every device pointer to floats that a caller passes (feats_dev,
+ *     out_dev, weights_dev, x_dev, y_dev, and each element of the host arrays of
+ *     device pointers) must be 16-byte aligned - the kernels access them with
+ *     16-byte loads and stores; a misaligned pointer is refused with DC_ERR_ARG
+ *     before anything is launched.  Host buffers (the *_host calls) need only
+ *     float alignment: a page-locked buffer is accessed directly by the kernels
+ *     when it is 16-byte aligned and staged otherwise.
  *   - Every function returns a dc_status; nothing throws or aborts.  Argument
  *     and admission checks run before any state is touched (fail closed, paper
  *     Section 3.3 admission clauses; the admission predicate is
@@ -56,6 +63,19 @@ typedef enum dc_status {
 
 enum { DC_PIPE_CONV = 1, DC_PIPE_FLOW = 2, DC_PIPE_VOCODER = 3, DC_PIPE_TOKEN2WAV = 4 };
 enum { DC_F32 = 0, DC_BF16 = 1 };   /* DC_BF16: bf16 storage and operands, fp32 accumulation */
+
+/* dc_config.options: switches for tests and measurements.  None of the first four changes a result
+ * byte.  (There is no configuration by environment variable.) */
+enum {
+  DC_OPT_NO_GRAPH     = 1,        /* decode calls issue their kernels one by one instead of one captured graph  */
+  DC_OPT_NO_PDL       = 2,        /* no programmatic dependent launch between the kernels of a step             */
+  DC_OPT_NO_ZEROCOPY  = 4,        /* the *_host calls always stage, also for page-locked caller buffers         */
+  DC_OPT_SERIAL_TAILS = 8,        /* token2wav dc_decode_batch: the vocoder tails one after another             */
+  /* MEASUREMENT ONLY - the outputs of such a model are meaningless: the step without the kernels of
+   * one class, so that step-time differences give that class's cost inside the captured graph. */
+  DC_OPT_SKIP_CONV_GEMM = 1 << 16,
+  DC_OPT_SKIP_ATTENTION = 1 << 17
+};
 
 #define DC_MAX_CONV 32
 #define DC_MAX_UP 4
@@ -124,6 +144,12 @@ typedef struct dc_config {
                                   * x by ((1 + w) v_cond - w v_uncond) / n_steps (paper Table 1 measures the flow
                                   * step in this guided, batch x 2 form).  The two passes of a stream are two
                                   * row blocks of the same GEMM tiles.                            */
+  int32_t  max_wave_frames;      /* token2wav pipeline: the most frames one dc_decode_wavefront call may carry per
+                                  * stream.  dc_stream_open allocates the buffer that holds a wavefront call's mel
+                                  * frames ([max_wave_frames][mel_dim] fp32) and the side stream its vocoder tails run
+                                  * on, so that no decode call allocates; 0 = wavefront calls on this model are
+                                  * refused.  Must be 0 for the other pipelines (their wavefront needs no buffer). */
+  uint32_t options;              /* DC_OPT_* bits, 0 for normal use                           */
 } dc_config;
 
 /* Number of floats of the canonical weight blob for this configuration, 0 if the
@@ -146,7 +172,8 @@ size_t dc_weights_count(const dc_config* cfg);
  * constants: paper Section 3.1, "constant has a trivial clock".) */
 dc_status dc_create(const float* weights_host, size_t n_floats, const dc_config* cfg, dc_model** out);
 
-/* Frees a model.  All its streams must be closed first (else DC_ERR_STATE). */
+/* Frees a model: the shared binding of Section 3.4 (weights, constant tables, captured graphs) goes
+ * when the last session has gone.  All its streams must be closed first (else DC_ERR_STATE). */
 dc_status dc_destroy(dc_model* model);
 
 /* Allocates and zeroes every carry of one stream (conv left context per (step,
@@ -159,6 +186,8 @@ dc_status dc_stream_open(dc_model* model, dc_stream** out);
  * existing buffers, on cuda_stream; addresses do not change (Section 3.2). */
 dc_status dc_stream_reset(dc_stream* stream, void* cuda_stream);
 
+/* Ends the stream and frees its carries (the per-session state of Section 3.4 ends with the session);
+ * the handle stays recognisable as closed (DC_ERR_STATE) until dc_destroy. */
 dc_status dc_stream_close(dc_stream* stream);
 
 /* One chunk of one stream.
@@ -179,7 +208,11 @@ dc_status dc_decode_chunk(dc_stream* stream, const float* feats_dev, int n_frame
  * out_dev[i].  feats_dev, n_frames and out_dev are HOST arrays (of device
  * pointers / ints).  Results are bitwise identical to n single dc_decode_chunk
  * calls.  (Multi-session serving over shared weights with per-session state:
- * paper Section 3.4, last paragraph, and Section 4.3 "Serving capacity".)  Flow and token2wav
+ * paper Section 3.4, last paragraph, and Section 4.3 "Serving capacity".)  Every admitted call is ONE
+ * CUDA graph launch: the chunk step is captured once per batch size - for 1 and max_batch streams at
+ * dc_create, for any other n at the first call that carries n streams (that one call also pays the
+ * capture; the graphs form the finite catalog of Section 3.3, Eq. 5) - and only the slot table
+ * passed by value changes from call to call.  Flow and token2wav
  * pipelines.  The token2wav composite batches the flow decoder and then runs the streams' vocoder
  * tails side by side on CUDA streams owned by the model, forked behind the flow decoder on
  * cuda_stream and joined back into it before the call returns. */
@@ -199,8 +232,9 @@ dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
  *   n_out     : host pointer (may be NULL) receiving the number of floats written
  * Flow and token2wav pipelines; the model must have been created with max_batch >= n_steps
  * (DC_ERR_ARG otherwise, stream untouched).  The token2wav composite keeps the call's mel frames
- * in a device buffer owned by the stream, which this call (re)allocates when n_frames exceeds
- * every earlier call's; the flow pipeline allocates nothing.  The composite's vocoder tail has no
+ * in a device buffer owned by the stream and sized at dc_stream_open from dc_config.max_wave_frames;
+ * a call with more frames than that is refused with DC_ERR_ARG, the stream untouched.  Like every
+ * decode call, this one allocates nothing.  The composite's vocoder tail has no
  * Euler loop to pipeline: chunk j's tail is enqueued, behind an event, on a CUDA stream owned by
  * the dc_stream as soon as the pass that finishes chunk j is, so it runs beside the flow decoder's
  * later passes; cuda_stream is made to wait for the last tail before the call returns, so work the
@@ -300,15 +334,18 @@ dc_status dc_stream_snapshot(dc_stream* stream, dc_snapshot** out, void* cuda_st
 dc_status dc_stream_restore(dc_stream* stream, const dc_snapshot* snapshot, void* cuda_stream);
 dc_status dc_snapshot_free(dc_snapshot* snapshot);
 
-/* Device addresses and byte sizes of the stream's carry buffers, for pointer
- * constancy checks: writes up to max_entries (address, bytes) pairs into out and
+/* Device addresses and byte sizes of the stream's carry buffers, for checks of the pointer
+ * constancy that Section 3.2 (Eq. 4) demands over the stream's lifetime: writes up to max_entries (address, bytes) pairs into out and
  * the number of buffers into n_entries. */
 dc_status dc_stream_carry_info(const dc_stream* stream, uint64_t* out, int max_entries, int* n_entries);
 
 /* counters[0] chunks decoded, [1] frames decoded, [2] calls rejected (DC_ERR_FRAMES),
  * [3] calls rejected (other argument/state errors), [4] device timeouts (this call reads the
  * device-side error word synchronously, so it also reports timeouts of asynchronous decode calls),
- * [5] kernel launches issued, [6] streams open, [7] reserved. */
+ * [5] kernel launches issued (kernel nodes of graph launches included), [6] streams open,
+ * [7] CUDA graph launches issued by decode calls (one per chunk step - the paper's one launch
+ * per chunk, Section 3.3 "Granularity", Eq. 6; rejected calls by reason: Section 3.3's counted
+ * refusal reasons). */
 dc_status dc_get_counters(const dc_model* model, uint64_t counters[8]);
 
 /* Self-test of the bounded device-side wait that every pipeline barrier in the kernels uses (the

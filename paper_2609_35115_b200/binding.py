@@ -35,7 +35,7 @@ class dc_config(C.Structure):
                 ("res_dilations", C.c_int32 * DC_MAX_RES), ("n_fft", C.c_int32), ("hop", C.c_int32),
                 ("rms_eps", C.c_float), ("logmag_clamp", C.c_float), ("max_batch", C.c_int32),
                 ("f_prompt", C.c_int32), ("f_lookahead", C.c_int32), ("noise_seed_lo", C.c_uint32), ("noise_seed_hi", C.c_uint32),
-                ("cfg_scale", C.c_float)]
+                ("cfg_scale", C.c_float), ("max_wave_frames", C.c_int32), ("options", C.c_uint32)]
 
 
 class DCError(RuntimeError):
@@ -91,7 +91,11 @@ def load_library():
     return lib
 
 
-def make_config(cfg, max_batch: int = 1) -> dc_config:
+OPT_NO_GRAPH, OPT_NO_PDL, OPT_NO_ZEROCOPY, OPT_SERIAL_TAILS = 1, 2, 4, 8
+OPT_SKIP_CONV_GEMM, OPT_SKIP_ATTENTION = 1 << 16, 1 << 17     # measurement only: outputs are meaningless
+
+
+def make_config(cfg, max_batch: int = 1, max_wave_frames: int = 0, options: int = 0) -> dc_config:
     """dc_workloads.DCConfig (or any object with the same attributes) -> dc_config."""
     c = dc_config()
     c.size = C.sizeof(dc_config)
@@ -115,6 +119,8 @@ def make_config(cfg, max_batch: int = 1) -> dc_config:
         c.n_fft, c.hop = cfg.n_fft, cfg.hop
     c.rms_eps, c.logmag_clamp = cfg.rms_eps, cfg.logmag_clamp
     c.max_batch = max_batch
+    c.max_wave_frames = max_wave_frames
+    c.options = options
     c.cfg_scale = float(getattr(cfg, "cfg_scale", 0.0))
     c.f_prompt = int(getattr(cfg, "f_prompt", 0))
     c.f_lookahead = int(getattr(cfg, "f_lookahead", 0))
@@ -148,10 +154,10 @@ class Snapshot:
 class Model:
     """dc_create / dc_destroy."""
 
-    def __init__(self, cfg, weights: np.ndarray, max_batch: int = 1):
+    def __init__(self, cfg, weights: np.ndarray, max_batch: int = 1, max_wave_frames: int = 0, options: int = 0):
         self.lib = load_library()
         self.cfg = cfg
-        self.c_cfg = make_config(cfg, max_batch)
+        self.c_cfg = make_config(cfg, max_batch, max_wave_frames, options)
         w = np.ascontiguousarray(weights, dtype=np.float32)
         self.handle = C.c_void_p()
         _check(self.lib.dc_create(w.ctypes.data, w.size, C.byref(self.c_cfg), C.byref(self.handle)), "dc_create")

@@ -29,8 +29,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
     cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB,
            *[os.path.join(CSRC, s) for s in SOURCES]]
-    extra = os.environ.get("DC_NVCC_FLAGS", "").split()   # experiments only, e.g. -DDC_STAGES=6
-    cmd[1:1] = extra
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     res = subprocess.run(cmd, capture_output=True, text=True)

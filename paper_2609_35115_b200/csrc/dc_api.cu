@@ -109,7 +109,7 @@ struct dc_stream {
   dc_stream* sub_flow = nullptr;   // DC_PIPE_TOKEN2WAV: the two halves' streams and the mel chunk between them
   dc_stream* sub_voc = nullptr;
   float*    mel = nullptr;         // [f_chunk][mel_dim] fp32, device
-  float*    wave_mel = nullptr;    // dc_decode_wavefront of the composite: all mel frames of one call (grown on demand)
+  float*    wave_mel = nullptr;    // dc_decode_wavefront of the composite: all mel frames of one call (max_wave_frames rows, sized at open)
   long long wave_mel_frames = 0;
   cudaStream_t wave_side = nullptr;   // the vocoder tail of a wavefront call runs here, beside the flow decoder's passes
   cudaEvent_t  wave_ev = nullptr;
@@ -129,6 +129,7 @@ static dc_config sub_config(const dc_config& c, int pipeline) {
   dc_config s = c;
   s.pipeline = pipeline;
   s.precision = pipeline == DC_PIPE_FLOW ? DC_BF16 : DC_F32;
+  s.max_wave_frames = 0;   // the mel buffer of a wavefront call belongs to the composite
   if (pipeline != DC_PIPE_FLOW) {
     s.cfg_scale = 0.f;
     s.f_prompt = 0;
@@ -151,6 +152,11 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (c->f_lookahead != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_lookahead belongs to the flow decoder");
   if (c->f_prompt != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_prompt belongs to the flow decoder");
   if (c->cfg_scale != 0.f && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("cfg_scale belongs to the flow decoder");
+  if (c->options & ~(uint32_t)(DC_OPT_NO_GRAPH | DC_OPT_NO_PDL | DC_OPT_NO_ZEROCOPY | DC_OPT_SERIAL_TAILS | DC_OPT_SKIP_CONV_GEMM |
+                               DC_OPT_SKIP_ATTENTION))
+    BAD("unknown option bit");
+  if (c->max_wave_frames < 0 || c->max_wave_frames > (1 << 24)) BAD("max_wave_frames out of range");
+  if (c->max_wave_frames != 0 && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("max_wave_frames belongs to the token2wav pipeline");
   if (c->pipeline == DC_PIPE_TOKEN2WAV) {
     if (c->precision != DC_BF16) BAD("token2wav pipeline is bf16 (flow decoder) + fp32 (vocoder tail)");
     const dc_config f = sub_config(*c, DC_PIPE_FLOW), v = sub_config(*c, DC_PIPE_VOCODER);
@@ -302,9 +308,8 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
       m->out_per_frame = m->sub_voc->out_per_frame;
       // a vocoder chunk step fills a fraction of the GPU (12 short kernels on small grids): up to 8 of a batch's
       // tails run at the same time
-      const char* nts = getenv("DC_TAIL_STREAMS");   // experiments: 0 or 1 = the tails one after another on the caller's stream
-      const int want = nts ? atoi(nts) : 8;
-      const int n_side = cfg->max_batch < want ? cfg->max_batch : (want > 32 ? 32 : want);
+      const int want = (cfg->options & DC_OPT_SERIAL_TAILS) ? 1 : 8;
+      const int n_side = cfg->max_batch < want ? cfg->max_batch : want;
       bool ok = n_side < 2 || cudaEventCreateWithFlags(&m->tail_fork, cudaEventDisableTiming) == cudaSuccess;
       for (int i = 0; ok && n_side >= 2 && i < n_side; ++i) {
         cudaStream_t cs2 = nullptr;
@@ -329,10 +334,7 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
       cudaError_t e = cudaMallocHost(&m->h_in, ni * sizeof(float));
       if (e == cudaSuccess) e = cudaMallocHost(&m->h_out, no * sizeof(float));
       if (e == cudaSuccess) e = cudaMallocHost(&m->h_err, sizeof(int));
-      {
-        const char* z = getenv("DC_NO_ZEROCOPY");   // experiments: always stage through the bounce buffers
-        m->zero_copy = !(z && atoi(z));
-      }
+      m->zero_copy = !(cfg->options & DC_OPT_NO_ZEROCOPY);
       if (e == cudaSuccess) e = cudaMalloc(&m->d_in, ni * sizeof(float));
       if (e == cudaSuccess) e = cudaMalloc(&m->d_out, no * sizeof(float));
       if (e != cudaSuccess) {
@@ -431,6 +433,14 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
     st = dc_stream_open(m->sub_flow, &s->sub_flow);
     if (st == DC_OK) st = dc_stream_open(m->sub_voc, &s->sub_voc);
     if (st == DC_OK) e = cudaMalloc(&s->mel, (size_t)m->cfg.f_chunk * m->cfg.mel_dim * sizeof(float));
+    if (st == DC_OK && e == cudaSuccess && m->cfg.max_wave_frames > 0) {
+      // wavefront calls keep a whole call's mel frames on the device and run the vocoder tails on a side stream:
+      // both are set up here, so that no decode call allocates or creates anything
+      e = cudaMalloc(&s->wave_mel, (size_t)m->cfg.max_wave_frames * m->cfg.mel_dim * sizeof(float));
+      if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->wave_side, cudaStreamNonBlocking);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->wave_ev, cudaEventDisableTiming);
+      if (e == cudaSuccess) s->wave_mel_frames = m->cfg.max_wave_frames;
+    }
   } else if (m->flow) {
     st = dc::flow_state_open(m->flow, &s->flow);
   } else {
@@ -704,7 +714,7 @@ static void enqueue_f32(dc_stream* s, bool use_call, const float* feats, int T, 
 // Captures the stream's chunk step once (at dc_stream_open): afterwards a chunk is one graph launch.
 static void build_f32_graph(dc_stream* s) {
   dc_model* m = s->model;
-  if (getenv("DC_NO_GRAPH") && atoi(getenv("DC_NO_GRAPH"))) return;
+  if (m->cfg.options & DC_OPT_NO_GRAPH) return;
   cudaStream_t cap = nullptr;
   if (cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return; }
   // programmatic dependent launch is left off here: measured on the vocoder tail it made the step
@@ -756,6 +766,7 @@ static dc_status decode_f32(dc_stream* s, const float* feats, int T, float* out,
     DC_CUDA(cudaGraphExecKernelNodeSetParams(s->g_exec, s->g_set_node, &kp));
     DC_CUDA(cudaGraphLaunch(s->g_exec, cs));
     *launches += s->g_launches;
+    m->counters[7]++;
     return DC_OK;
   }
   enqueue_f32(s, false, feats, T, out, cs, false, launches);
@@ -763,11 +774,21 @@ static dc_status decode_f32(dc_stream* s, const float* feats, int T, float* out,
   return DC_OK;
 }
 
-static dc_status admit(dc_stream* s, const float* feats, int T, float* out) {
+// The kernels read the caller's chunk and write its output with 16-byte accesses.
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// device_ptrs: feats / out are what the kernels will dereference (device pointers, or the device alias of a
+// page-locked host buffer), so they must be 16-byte aligned; host buffers that are staged need no alignment.
+static dc_status admit(dc_stream* s, const float* feats, int T, float* out, bool device_ptrs = true) {
   if (!s) return DC_ERR_ARG;
   if (s->closed || s->poisoned) return DC_ERR_STATE;
   if (!feats || !out) {
     s->model->counters[3]++;
+    return DC_ERR_ARG;
+  }
+  if (device_ptrs && (!aligned16(feats) || !aligned16(out))) {
+    s->model->counters[3]++;
+    dc::set_error("feats (%p) and out (%p) must be 16-byte aligned device pointers", (const void*)feats, (const void*)out);
     return DC_ERR_ARG;
   }
   const int f_call = s->model->cfg.f_chunk + s->model->cfg.f_lookahead;   // committed frames are bounded by f_chunk, presented ones by this
@@ -857,6 +878,16 @@ extern "C" dc_status dc_decode_wavefront_batch(dc_model* m, int n, dc_stream* co
       m->counters[3]++;
       return DC_ERR_ARG;
     }
+    if (!aligned16(feats[i]) || !aligned16(out[i])) {
+      m->counters[3]++;
+      dc::set_error("feats[%d] (%p) and out[%d] (%p) must be 16-byte aligned device pointers", i, (const void*)feats[i], i, (const void*)out[i]);
+      return DC_ERR_ARG;
+    }
+    if (m->sub_flow && n_frames[i] > s->wave_mel_frames) {
+      m->counters[3]++;
+      dc::set_error("wavefront call of %lld frames on a token2wav stream opened with max_wave_frames = %lld", n_frames[i], s->wave_mel_frames);
+      return DC_ERR_ARG;
+    }
     for (int j = 0; j < i; ++j)
       if (streams[j] == s) {
         m->counters[3]++;
@@ -877,21 +908,6 @@ extern "C" dc_status dc_decode_wavefront_batch(dc_model* m, int n, dc_stream* co
     // CUDA stream of its own
     for (int i = 0; i < n; ++i) {
       dc_stream* s = streams[i];
-      if (s->wave_mel_frames < n_frames[i]) {
-        if (s->wave_mel) cudaFree(s->wave_mel);
-        s->wave_mel = nullptr;
-        s->wave_mel_frames = 0;
-        if (cudaMalloc(&s->wave_mel, (size_t)n_frames[i] * m->cfg.mel_dim * sizeof(float)) != cudaSuccess) {
-          cudaGetLastError();
-          return DC_ERR_OOM;
-        }
-        s->wave_mel_frames = n_frames[i];
-      }
-      if (!s->wave_side && (cudaStreamCreateWithFlags(&s->wave_side, cudaStreamNonBlocking) != cudaSuccess ||
-                            cudaEventCreateWithFlags(&s->wave_ev, cudaEventDisableTiming) != cudaSuccess)) {
-        cudaGetLastError();
-        return DC_ERR_CUDA;
-      }
       mels[(size_t)i] = s->wave_mel;
     }
     WaveTail w{streams, cs, !(m->sub_voc->prof.on || m->sub_flow->prof.on), out, n_frames};
@@ -1013,18 +1029,21 @@ extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* strea
 
 extern "C" dc_status dc_decode_chunk_host(dc_stream* s, const float* feats_host, int T, float* out_host, int* n_out,
                                           void* cuda_stream) {
-  dc_status st = admit(s, feats_host, T, out_host);
+  dc_status st = admit(s, feats_host, T, out_host, false);
   if (st != DC_OK) return st;
   dc_model* m = s->model;
   cudaStream_t cs = (cudaStream_t)cuda_stream;
-  // flow pipeline: page-locked caller buffers are read / written by the kernels themselves (see dc_decode_batch_host)
+  // flow pipeline: page-locked, 16-byte aligned caller buffers are read / written by the kernels themselves
+  // (see dc_decode_batch_host); any other buffer is staged
   const float* fin = s->stage_in;
   float* fout = s->stage_out;
   if (m->flow && m->zero_copy) {
     cudaPointerAttributes a{};
-    if (cudaPointerGetAttributes(&a, feats_host) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr)
+    if (cudaPointerGetAttributes(&a, feats_host) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr &&
+        aligned16(a.devicePointer))
       fin = static_cast<const float*>(a.devicePointer);
-    if (cudaPointerGetAttributes(&a, out_host) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr)
+    if (cudaPointerGetAttributes(&a, out_host) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr &&
+        aligned16(a.devicePointer))
       fout = static_cast<float*>(a.devicePointer);
     cudaGetLastError();
   }
@@ -1061,7 +1080,7 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
   std::vector<const float*> fin((size_t)n);
   std::vector<float*> fout((size_t)n);
   for (int i = 0; i < n; ++i) {
-    dc_status st = admit(streams[i], feats_host[i], n_frames[i], out_host[i]);
+    dc_status st = admit(streams[i], feats_host[i], n_frames[i], out_host[i], false);
     if (st != DC_OK) return st;
     fin[(size_t)i] = m->d_in + (size_t)i * in_stride;
     fout[(size_t)i] = m->d_out + (size_t)i * out_stride;
@@ -1074,14 +1093,16 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
   for (int i = 0; i < n && (in_direct || out_direct); ++i) {
     cudaPointerAttributes a{};
     if (in_direct) {
-      if (cudaPointerGetAttributes(&a, feats_host[i]) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr) {
+      if (cudaPointerGetAttributes(&a, feats_host[i]) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr &&
+          aligned16(a.devicePointer)) {
         fin[(size_t)i] = static_cast<const float*>(a.devicePointer);
       } else {
         in_direct = false;
       }
     }
     if (out_direct) {
-      if (cudaPointerGetAttributes(&a, out_host[i]) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr) {
+      if (cudaPointerGetAttributes(&a, out_host[i]) == cudaSuccess && a.type == cudaMemoryTypeHost && a.devicePointer != nullptr &&
+          aligned16(a.devicePointer)) {
         fout[(size_t)i] = static_cast<float*>(a.devicePointer);
       } else {
         out_direct = false;
@@ -1173,12 +1194,14 @@ extern "C" dc_status dc_get_counters(const dc_model* m, uint64_t counters[8]) {
     if (code > 0) const_cast<dc_model*>(m)->counters[4]++;
   }
   for (int i = 0; i < 8; ++i) counters[i] = m->counters[i].load();
-  if (m->sub_flow) {   // kernel launches and device time-outs are counted where they happen
+  if (m->flow) counters[7] += dc::flow_graph_launches(m->flow);
+  if (m->sub_flow) {   // kernel launches, graph launches and device time-outs are counted where they happen
     uint64_t a[8], b[8];
     dc_get_counters(m->sub_flow, a);
     dc_get_counters(m->sub_voc, b);
     counters[4] += a[4] + b[4];
     counters[5] += a[5] + b[5];
+    counters[7] += a[7] + b[7];
   }
   return DC_OK;
 }

@@ -151,17 +151,9 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
     asm volatile("cp.async.commit_group;" ::: "memory");   // an (empty) group per step keeps the count uniform
   };
 
-#ifdef DC_TIMING
-  __shared__ long long f_t[40];
-  const bool ftm = blockIdx.x == 0 && blockIdx.y == 1 && blockIdx.z == 0 && threadIdx.x == 0;
-  const long long f0 = clock64();
-#endif
 #pragma unroll
   for (int s = 0; s < F32_STAGES - 1; ++s) issue(s);
   for (int s = 0; s < my_steps; ++s) {
-#ifdef DC_TIMING
-    if (ftm && s < 32) f_t[s] = clock64() - f0;
-#endif
     asm volatile("cp.async.wait_group %0;" ::"n"(F32_STAGES - 2) : "memory");   // step s has landed
     asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "r"(NTG) : "memory");       // for the whole group; step s-1's buffer is free
     issue(s + F32_STAGES - 1);
@@ -186,13 +178,6 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
     }
   }
 
-#ifdef DC_TIMING
-  if (ftm) {
-    printf("F32 grid (%d,%d,%d) KS %d steps %d loop_end %lld:", gridDim.x, gridDim.y, gridDim.z, KS, my_steps, clock64() - f0);
-    for (int i = 0; i < my_steps && i < 32; ++i) printf(" %lld", f_t[i]);
-    printf("\n");
-  }
-#endif
   if (KS > 1) {
     // fixed-order sum of the groups' partial tiles: group g parks its tile in its own (now idle)
     // operand ring, group 0 adds them in the order 1, 2, ...
@@ -498,6 +483,10 @@ extern "C" dc_status dc_conv_stack_noalloc(const float* weights_dev, int hidden,
                                            const float* x_dev, int n_frames, float* y_dev, void* cuda_stream) {
   if (!weights_dev || !dilations || !x_dev || !y_dev) {
     dc::set_error("dc_conv_stack_noalloc: null pointer argument");
+    return DC_ERR_ARG;
+  }
+  if (((reinterpret_cast<uintptr_t>(weights_dev) | reinterpret_cast<uintptr_t>(x_dev) | reinterpret_cast<uintptr_t>(y_dev)) & 15u) != 0) {
+    dc::set_error("dc_conv_stack_noalloc: weights_dev, x_dev and y_dev must be 16-byte aligned (the kernels use 16-byte accesses)");
     return DC_ERR_ARG;
   }
   if (hidden < 4 || hidden % 4 || n_conv < 1 || n_conv > DC_MAX_CONV || n_frames < 1) {

@@ -117,7 +117,6 @@ struct GemmParams {
   long long    ssq_ld;          // rows per chunk plane
   float        inv_C, eps;
   int*         err;
-  int          dbg;
 };
 
 // SiLU(z) = z * sigmoid(z) = 0.5 z (1 + tanh(z / 2)): one MUFU op per element instead of two (exp + reciprocal);
@@ -166,17 +165,6 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * TILE_M, n0 = blockIdx.y * p.BN;
-#ifdef DC_TIMING
-  const bool tm = blockIdx.x == 0 && blockIdx.y == 1 && p.mode == MODE_CONV;
-  long long t_start = 0;
-  if (tm) t_start = clock64();
-  __shared__ long long s_t[8];
-  __shared__ long long s_k[32];
-  __shared__ long long s_p[32];
-#define DC_T(idx) do { if (tm) s_t[idx] = clock64() - t_start; } while (0)
-#else
-#define DC_T(tag) do {} while (0)
-#endif
   // Accumulator: BN columns, or 3 BN for a conv block, whose three taps are the column blocks of ONE
   // product Z = X [W_0 | W_1 | W_2] (a row shift commutes with the product, so the taps are shifted
   // and added in the epilogue; a tcgen05.mma costs about 47 cycles however small it is, and one
@@ -201,7 +189,6 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (threadIdx.x == 0) DC_T(0);
   ptx::pdl_launch();   // the next kernel may start its prologue and its weight prefetch now
 
   if (warp == 0 || warp == 2) {
@@ -225,9 +212,6 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           *s_fail = 1;
           break;
         }
-#ifdef DC_TIMING
-        if (tm && kb < 32 && is_a && on) s_p[kb] = clock64() - t_start;
-#endif
         ptx::mbar_expect_tx_if(on, &full[st], tx_bytes);
         if (is_a) {
           ptx::tma_load_2d_if(on, dst, &tmA, x, ya, &full[st]);
@@ -246,7 +230,6 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           phase ^= 1;
         }
       }
-      if (is_a && on) DC_T(1);
     }
   } else if (warp == 1 || warp == 3) {
     // UMMA issuers.  A single thread spends about 100 cycles per tcgen05.mma it issues, more than a
@@ -272,10 +255,6 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           break;
         }
         ptx::tc_fence_after();
-        if (kb == 0 && on) DC_T(2);
-#ifdef DC_TIMING
-        if (tm && kb < 32 && on) s_k[kb] = clock64() - t_start;
-#endif
         const uint64_t da = d_a0 + (uint64_t)((uint32_t)st * stage16), db = da + ab16;
         ptx::umma_bf16_if(on, d_acc, da, db, idesc, acc);
 #pragma unroll
@@ -283,7 +262,6 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         acc = 1;
         ptx::umma_commit_if(on, &empty[st]);
       }
-      if (on && me == 0) DC_T(3);
       ptx::umma_commit_if(on, accum);   // arrives when every UMMA above has finished (also on the failure path)
     }
   } else {
@@ -347,7 +325,6 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     const bool got = ptx::mbar_wait_relaxed(accum, 0);
     ptx::tc_fence_after();
-    if (threadIdx.x == 128) DC_T(4);
     if (!got) atomicCAS(p.err, 0, 3 | (p.mode << 8));
     const bool slot_ok = in_range && got && *s_fail == 0;
     const float* tau_s = s_tau + ((q >> 1) & 1) * 64;   // rows 64.. of the tile are its second slot
@@ -496,7 +473,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!is_halo) {
         if (has_resid) {
           const uint32_t w[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
-          if (p.mode == MODE_CONV && !(p.dbg & 16)) {
+          if (p.mode == MODE_CONV) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               acc[2 * i] = __uint_as_float(w[i] << 16) + silu_f(acc[2 * i] + tau_s[c0 + 2 * i]);
@@ -512,9 +489,6 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         pack16_bf16(acc, va, vb);
       }
-#ifdef DC_TIMING
-      if (p.dbg & 8) continue;
-#endif
       // chunk rows store y; left-context rows hand the carried rows to the consumer of `out`
       if (is_chunk || (is_halo && do_halo)) store16(p.out + grow * p.ld + n, va, vb);
       if (p.ssq_out != nullptr && in_range) {   // sum of squares of the 16 stored values, fixed order
@@ -532,26 +506,11 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       // shift the carry by T frames: [old carry | chunk] -> its last 8 rows
       if (carry_wr) store16(carry + new_row * p.C + n, va, vb);
-      if (threadIdx.x == 128 && kk == 0) DC_T(6);
-      if (threadIdx.x == 128 && kk == 1) DC_T(7);
     }
   }
-  if (threadIdx.x == 128) DC_T(5);
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 1) ptx::tmem_dealloc(tmem_base, tmem_cols);
-#ifdef DC_TIMING
-  if (tm && threadIdx.x == 0)
-    printf("T setup %lld tma_issued %lld first_full %lld mma_issued %lld accum_ready %lld ch0 %lld ch1 %lld epi_done %lld end %lld\n", s_t[0], s_t[1],
-           s_t[2], s_t[3], s_t[4], s_t[6], s_t[7], s_t[5], clock64() - t_start);
-  if (tm && threadIdx.x == 0) {
-    printf("K full:");
-    for (int i = 0; i < p.n_kblocks && i < 32; ++i) printf(" %lld", s_k[i]);
-    printf("\nK prod:");
-    for (int i = 0; i < p.n_kblocks && i < 32; ++i) printf(" %lld", s_p[i]);
-    printf("\n");
-  }
-#endif
 }
 
 // ---- small kernels ---------------------------------------------------------------------------
@@ -662,11 +621,7 @@ constexpr int ATT_BAR_BYTES = 1024;        // 14 barriers, TMEM slot, softmax ex
 // Two CTAs per SM leave 113 KB each: the tiles take 112 KB, so there is no room for alignment slack.
 // The dynamic shared memory is declared 1024-byte aligned (the swizzled tiles need it) and the kernel
 // checks the address it got.
-#ifdef DC_TIMING
-constexpr size_t ATT_SMEM = 1024 + ATT_Q_BYTES + 2 * ATT_P_BYTES + ATT_STAGES * ATT_STAGE_BYTES + ATT_BAR_BYTES;
-#else
 constexpr size_t ATT_SMEM = ATT_Q_BYTES + 2 * ATT_P_BYTES + ATT_STAGES * ATT_STAGE_BYTES + ATT_BAR_BYTES;
-#endif
 static_assert(ATT_SMEM <= 113 * 1024 + 1024, "two attention CTAs must fit one SM");
 constexpr float ATT_RESCALE_LOG2 = 8.0f;
 
@@ -699,15 +654,11 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
 template <bool PROMPT>
 __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t att_smem_raw[];
-#ifdef DC_TIMING
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem_raw) + 1023) & ~(uintptr_t)1023);
-#else
   uint8_t* smem = att_smem_raw;
   if ((ptx::smem_u32(smem) & 1023u) != 0u) {   // would corrupt the swizzled tiles: refuse (uniform for the CTA)
     if (threadIdx.x == 0) atomicExch(p.err, 14);
     return;
   }
-#endif
   uint8_t* sQ = smem;
   uint8_t* sP = sQ + ATT_Q_BYTES;                    // buffer b & 1 at + ATT_P_BYTES (b & 1); tile t (keys 64 t .. of the block) at + 8192 t
   uint8_t* ring = sP + 2 * ATT_P_BYTES;
@@ -729,14 +680,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int slot = blockIdx.x, head = blockIdx.y;
   const int chunks = p.dh >> 3;             // 16-byte chunks per head row
-#ifdef DC_TIMING
-  long long* a_t = reinterpret_cast<long long*>(s_x + 128);   // 48 stamps in the spare bytes of the barrier area (keeps 2 CTAs per SM)
-  const bool atm = blockIdx.x == 3 && blockIdx.y == 2;
-  const long long a_start = clock64();
-#define DC_AT(i) do { if (atm) a_t[i] = clock64() - a_start; } while (0)
-#else
-#define DC_AT(i) do {} while (0)
-#endif
 
   if (tid == 0) {
     for (int i = 0; i < ATT_STAGES; ++i) {
@@ -851,20 +794,17 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         asm volatile("cp.async.wait_all;" ::: "memory");
         ptx::fence_proxy_async_smem();
         ptx::mbar_arrive(&full[(b - 1) % ATT_STAGES]);
-        if (lt == 0 && is_k && b - 1 < 8) DC_AT(8 + b - 1);     // block b-1 landed
       }
       if (b < n_early) continue;                                // already in flight
       if (b >= ATT_STAGES && ok && !ptx::mbar_wait_relaxed(&empty[st], ((b / ATT_STAGES) - 1) & 1)) {
         ok = false;
         atomicExch(p.err, 4);
       }
-      if (lt == 0 && is_k && b < 8) DC_AT(b);                    // block b load issue starts
       issue_block(b);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
     ptx::fence_proxy_async_smem();
     ptx::mbar_arrive(&full[(nkb - 1) % ATT_STAGES]);
-    if (lt == 0 && is_k && nkb - 1 < 8) DC_AT(8 + nkb - 1);
   } else if (warp == 4) {
     // ---------------- UMMA issuer ----------------
     if (lane == 0) {
@@ -885,7 +825,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         for (int k = 0; k < 4; ++k) ptx::umma_bf16(tmem_base, dq + 2 * k, dk + 2 * k, idesc_s, k != 0);
         ptx::umma_commit(bar_s);
         ptx::umma_commit(&empty_k[st]);                  // the K stage is free once S(b) has been computed
-        if (b < 8) DC_AT(16 + b);                        // S(b) issued
       };
       issue_s(0);
       for (int b = 0; b < nkb; ++b) {
@@ -914,7 +853,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         }
         ptx::umma_commit(&empty_v[st]);
         ptx::umma_commit(&bar_pv[b & 1]);
-        if (b < 8) DC_AT(24 + b);                        // PV(b) issued
       }
     }
   } else {
@@ -928,7 +866,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     for (int b = 0; b < nkb; ++b) {
       if (ok && !ptx::mbar_wait(bar_s, b & 1)) { ok = false; atomicExch(p.err, 7); }
       ptx::tc_fence_after();
-      if (tid == 0 && b < 8) DC_AT(32 + b);              // S(b) ready
       const int valid = L - b * ATT_KB - half * 64;   // columns of this half that are real keys
       float v[64];
 #pragma unroll
@@ -991,7 +928,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       ptx::fence_proxy_async_smem();
       ptx::tc_fence_before();
       ptx::mbar_arrive(&bar_p[b & 1]);
-      if (tid == 0 && b < 8) DC_AT(40 + b);              // P(b) written
     }
     if (ok && !ptx::mbar_wait(&bar_pv[(nkb - 1) & 1], ((nkb - 1) >> 1) & 1)) { ok = false; atomicExch(p.err, 9); }
     ptx::tc_fence_after();
@@ -1014,23 +950,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 4) ptx::tmem_dealloc(tmem_base, ATT_TMEM_COLS);
-#ifdef DC_TIMING
-  if (atm && tid == 0) {
-    printf("ATT nkb %d end %lld\n load_issue:", nkb, clock64() - a_start);
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[i]);
-    printf("\n landed:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[8 + i]);
-    printf("\n S_issued:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[16 + i]);
-    printf("\n S_ready:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[32 + i]);
-    printf("\n P_written:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[40 + i]);
-    printf("\n PV_issued:");
-    for (int i = 0; i < nkb; ++i) printf(" %lld", a_t[24 + i]);
-    printf("\n");
-  }
-#endif
 }
 
 // ---- host helpers ----------------------------------------------------------------------------
@@ -1122,9 +1041,9 @@ struct FlowModel {
   bool pdl = true;                       // programmatic dependent launch between the step's kernels
   int  kv_rs = 0, kv_hs = 0, dh_shift = 0;   // K/V plane layout (see GemmParams)
   int  n_sm = 148;                       // SMs of the device (read at create)
-  int  dbg = 0;
   cudaStream_t cap_stream = nullptr;     // used only to capture graphs at create
   std::map<int, GraphEntry> graphs;      // batch size -> captured chunk step
+  uint64_t graph_launches = 0;           // graph launches issued by decode calls
   std::vector<SlotSet> sets;
 };
 
@@ -1325,10 +1244,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   }
   m->sets.resize((size_t)(m->S + MAX_SLOTS_PER_SET - 1) / MAX_SLOTS_PER_SET);
   {
-    const char* e = getenv("DC_NO_PDL");        // experiments only
-    m->pdl = !(e && atoi(e));
-    const char* d = getenv("DC_GEMM_DBG");
-    m->dbg = d ? atoi(d) : 0;
+    m->pdl = !(cfg.options & DC_OPT_NO_PDL);
     // K/V planes are head-major: the rows one attention CTA streams are contiguous
     m->dh_shift = m->cfg.head_dim == 64 ? 6 : 5;
     m->kv_rs = m->cfg.head_dim;
@@ -1336,8 +1252,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
       m->n_sm = sms;
-    const char* g = getenv("DC_NO_GRAPH");
-    if (!(g && atoi(g)) && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) == cudaSuccess) {
+    if (!(cfg.options & DC_OPT_NO_GRAPH) && cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking) == cudaSuccess) {
       // the two batch sizes that matter are captured now, so that no decode call ever builds a graph:
       // a single stream, and the full batch
       const bool g1 = build_graph(m, m->n_pass);   // a single stream
@@ -1345,9 +1260,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
       // ... and one pass of the network over n_steps chunks (wavefront decoding), where the model has room for it
       const int n_wave = cfg.n_steps * m->n_pass;
       if (n_wave <= m->S && n_wave <= MAX_SLOTS_PER_SET) build_graph(m, n_wave, true);
-      if (getenv("DC_VERBOSE"))
-        fprintf(stderr, "[dc] graphs: n=1 %s, n=%d %s, pdl %d/%d\n", g1 ? "ok" : "none", m->S, gs ? "ok" : "none",
-                g1 ? (int)m->graphs[m->n_pass].pdl : -1, gs ? (int)m->graphs[m->S].pdl : -1);
+      (void)gs;
     }
     cudaGetLastError();
   }
@@ -1399,6 +1312,7 @@ dc_status flow_state_reset(FlowModel*, FlowState* s, cudaStream_t st) {
 }
 
 const int* flow_error_word(const FlowModel* m) { return m->d_err; }
+uint64_t flow_graph_launches(const FlowModel* m) { return m->graph_launches; }
 
 dc_status flow_selftest_bounded_wait(int max_polls) {
   if (max_polls < 1 || max_polls > 1000000) return DC_ERR_ARG;
@@ -1424,7 +1338,6 @@ int flow_take_device_error(FlowModel* m) {
   if (cudaMemcpy(&v, m->d_err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
   if (v != 0) {
     cudaMemset(m->d_err, 0, sizeof(int));
-    if (getenv("DC_VERBOSE")) fprintf(stderr, "[dc] device error word 0x%x\n", v);
   }
   return v;
 }
@@ -1502,7 +1415,6 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     p.P = m->P;
     p.err = m->d_err;
     const int stage_bytes = A_BYTES + p.taps * ((p.BN * 128 + 1023) & ~1023);
-    p.dbg = m->dbg;
     // the issuer count fixes the summation order, so it depends on the GEMM's role only, never on the tile
     // width chosen for the batch size (batched and single-stream results must agree bit for bit);
     // the QKV and output projections keep one issuer (their wide tiles would not fit two accumulators)
@@ -1566,7 +1478,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
         const bool next_is_conv = (j + 1 < m->cpa);
         p.halo_off = next_is_conv ? ((long long)s * c.n_conv + l + 1) * halo_stride : -1;
         if (!next_is_conv) feeds_norm(p);   // the group's attention norm, or the final norm of a conv-only stack
-        if (!(m->dbg & 1024)) gemm(*tX, m->tmWconv[v][l], p, C);   // bit 1024 (measurement only): without the conv-block kernels
+        if (!(c.options & DC_OPT_SKIP_CONV_GEMM)) gemm(*tX, m->tmWconv[v][l], p, C);   // (measurement only: the step without this class)
         swap();
       }
       if (c.n_attn > 0) {
@@ -1579,7 +1491,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
           normalised(p);
           gemm(*tX, m->tmWqkv[v][g], p, 3 * C);
         }
-        if (!(m->dbg & 32)) attention(s, g);    // DC_GEMM_DBG bit 32 (measurement only): the step without its attention kernels
+        if (!(c.options & DC_OPT_SKIP_ATTENTION)) attention(s, g);   // (measurement only: the step without this class)
         {
           GemmParams p{};
           p.mode = MODE_OPROJ; p.BN = bn; p.n_kblocks = C / KBLK; p.taps = 1;
@@ -1692,6 +1604,9 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
   }
   const bool profiling = m->prof != nullptr && m->prof->on;
   auto it = m->graphs.find(n);
+  // a batch size met for the first time captures its chunk step now (one graph per size, kept for the model's
+  // lifetime: the finite catalog of launch shapes), so that every admitted call is one graph launch
+  if (it == m->graphs.end() && !profiling && build_graph(m, n)) it = m->graphs.find(n);
   if (!profiling && it != m->graphs.end()) {
     // one launch for the whole chunk step
     GraphEntry& ge = it->second;
@@ -1710,6 +1625,7 @@ dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float
       return DC_ERR_CUDA;
     }
     *launches += ge.launches;
+    ++m->graph_launches;
   } else {
     LaunchCtx lc{st, m->pdl && !profiling, m->prof};
     enqueue_chunk(m, n, sets.data(), n_sets, lc);
@@ -1797,6 +1713,7 @@ dc_status flow_decode_wave(FlowModel* m, int n_streams, FlowState* const* states
         return DC_ERR_CUDA;
       }
       *launches += ge.launches;
+      ++m->graph_launches;
     } else {
       LaunchCtx lc{st, m->pdl && !profiling, m->prof};
       enqueue_chunk(m, n, &set, 1, lc, true);

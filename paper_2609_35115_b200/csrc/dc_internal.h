@@ -113,6 +113,7 @@ void      flow_state_close(FlowState* s);
 dc_status flow_selftest_bounded_wait(int max_polls);
 int       flow_take_device_error(FlowModel* m);
 const int* flow_error_word(const FlowModel* m);   // device address of that word
+uint64_t  flow_graph_launches(const FlowModel* m);   // graph launches issued by decode calls so far
 // One chunk for each of n streams.  Returns the number of kernel launches through *launches.
 dc_status flow_decode(FlowModel* m, int n, FlowState* const* states, const float* const* feats_dev,
                       const int* n_frames, float* const* out_dev, cudaStream_t st, int* launches);

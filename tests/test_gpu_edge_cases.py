@@ -98,3 +98,71 @@ def test_conv_stream_large_dilation(dc):
 def test_vocoder_without_residual_blocks_and_big_stride(dc):
     cfg = wl.tiny_vocoder(name="edge_voc", up_strides=(16,), up_channels=(8, 12), res_dilations=(), f_chunk=7, seed=36)
     _check(dc, cfg, [0, 7, 8, 15, 16, 23], TOL_F32)
+
+
+def test_misaligned_device_pointers_are_refused_before_any_launch(dc):
+    """The kernels access the caller's chunk, output and weights with 16-byte loads and stores; a pointer
+    that is not 16-byte aligned is refused with DC_ERR_ARG before anything is launched (the check is on
+    the host, so nothing here reaches the device), and the stream stays usable and untouched."""
+    lib = dc.load_library()
+    for cfg in (wl.CONFIGS["cfg1"], wl.tiny_flow(), wl.tiny_vocoder()):
+        w = wl.make_workload(cfg)
+        s = w.streams[0]
+        m = dc.Model(cfg, w.weights, max_batch=cfg.n_steps if cfg.pipeline == "flow" else 1)
+        st = m.open_stream()
+        T = s.boundaries[1]
+        x = torch.from_numpy(s.feats[:T]).cuda()
+        y = torch.zeros(T * cfg.out_per_frame + 8, device="cuda")
+        before = m.counters()
+        assert st.decode_raw(x.data_ptr() + 4, T - 1, y.data_ptr()) == 1
+        assert "16-byte aligned" in lib.dc_last_error().decode()
+        assert st.decode_raw(x.data_ptr(), T, y.data_ptr() + 8) == 1
+        after = m.counters()
+        assert after[3] == before[3] + 2 and after[5] == before[5] and after[0] == before[0]
+        if cfg.pipeline == "flow":
+            with pytest.raises(dc.DCError):
+                dc.decode_batch(m, [st], [x.view(-1)[1:1 + (T - 1) * cfg.in_dim].view(T - 1, cfg.in_dim)],
+                                [y[:(T - 1) * cfg.out_per_frame].view(T - 1, -1)])
+            with pytest.raises(dc.DCError):
+                dc.decode_wavefront_batch(m, [st], [x], [y[1:1 + T * cfg.out_per_frame]])
+            assert m.counters()[5] == before[5]
+        # the refused calls left the stream as it was: the chunk decodes as the first chunk of a fresh stream
+        got = st.decode_chunk(x).clone().reshape(-1).cpu().numpy()
+        ref = orc.run_stream(cfg, w.weights, s.feats[:T], [0, T]).reshape(-1)
+        assert _gu().rel_err(got, ref) <= (TOL_F32 if cfg.precision == "f32" else TOL_BF16)
+        st.close()
+        m.destroy()
+    # the allocation-free entry point checks its three device pointers the same way
+    C = 64
+    wts = torch.zeros(3 * C * C + C + 4, device="cuda")
+    xs = torch.zeros(8 * C + 4, device="cuda")
+    ys = torch.zeros(8 * C + 4, device="cuda")
+    assert dc.conv_stack_noalloc(wts[1:], C, (1,), xs[:8 * C].view(8, C), ys[:8 * C].view(8, C)) == 1
+    assert "16-byte aligned" in lib.dc_last_error().decode()
+    assert dc.conv_stack_noalloc(wts, C, (1,), xs[1:1 + 8 * C].view(8, C), ys[:8 * C].view(8, C)) == 1
+    assert dc.conv_stack_noalloc(wts, C, (1,), xs[:8 * C].view(8, C), ys[3:3 + 8 * C].view(8, C)) == 1
+    assert dc.conv_stack_noalloc(wts, C, (1,), xs[:8 * C].view(8, C), ys[:8 * C].view(8, C)) == 0
+    torch.cuda.synchronize()
+
+
+def test_host_entry_point_stages_a_misaligned_pinned_buffer(dc):
+    """A page-locked host buffer at an odd float offset cannot be read by the kernels directly; the host
+    entry points fall back to their staging copy and give the same bytes."""
+    cfg = wl.tiny_flow()
+    w = wl.make_workload(cfg)
+    s = w.streams[0]
+    T = s.boundaries[1]
+    m = dc.Model(cfg, w.weights)
+    pin_in = torch.zeros(T * cfg.in_dim + 4).pin_memory()
+    pin_out = torch.zeros(T * cfg.mel_dim + 4).pin_memory()
+    outs = []
+    for off in (0, 1):
+        st = m.open_stream()
+        fi = pin_in[off:off + T * cfg.in_dim].view(T, cfg.in_dim)
+        fo = pin_out[off:off + T * cfg.mel_dim].view(T, cfg.mel_dim)
+        fi.copy_(torch.from_numpy(s.feats[:T]))
+        assert st.decode_chunk_host(fi, fo) == T * cfg.mel_dim
+        outs.append(fo.clone().numpy())
+        st.close()
+    m.destroy()
+    assert np.array_equal(outs[0], outs[1])

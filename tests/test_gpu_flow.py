@@ -62,8 +62,10 @@ def test_cfg2_small_flow_decoder(dc):
 
 
 def test_cfg3_token2wav_sized_flow_decoder(dc):
-    # 30 chunks: passes the K/V cap (512 frames after 11 chunks) and wraps the 562-row ring
-    _parity(dc, wl.CONFIGS["cfg3"].replace(n_chunks=30))
+    # the whole configuration, 100 chunks: passes the K/V cap (512 frames after 11 chunks) and wraps the
+    # 562-row ring several times; _parity also asserts that a second full run gives the same bytes
+    assert wl.CONFIGS["cfg3"].n_chunks == 100
+    _parity(dc, wl.CONFIGS["cfg3"])
 
 
 def test_batched_streams_match_oracle_and_single_stream_bytes(dc):
@@ -122,27 +124,32 @@ def test_cfg5_multi_stream_serving_full_size(dc):
     S = cfg.n_streams
     assert len({s.boundaries[1] for s in w.streams}) > 8          # offsets really are staggered
     m = dc.Model(cfg, w.weights, max_batch=S)
-    streams = [m.open_stream() for _ in range(S)]
     feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
-    outs = [torch.empty(s.feats.shape[0], cfg.mel_dim, device="cuda") for s in w.streams]
-    for r in range(cfg.n_chunks):
-        fs = [feats[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
-        os_ = [outs[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
-        dc.decode_batch(m, streams, fs, os_)
-    torch.cuda.synchronize()
-    assert m.counters()[4] == 0, "a bounded device-side wait timed out"
-    for st in streams:
-        st.close()
-    got = [o.cpu().numpy() for o in outs]
+
+    def full_run():
+        streams = [m.open_stream() for _ in range(S)]
+        outs = [torch.empty(s.feats.shape[0], cfg.mel_dim, device="cuda") for s in w.streams]
+        for r in range(cfg.n_chunks):
+            fs = [feats[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
+            os_ = [outs[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
+            dc.decode_batch(m, streams, fs, os_)
+        torch.cuda.synchronize()
+        assert m.counters()[4] == 0, "a bounded device-side wait timed out"
+        for st in streams:
+            st.close()
+        return [o.cpu().numpy() for o in outs]
+
+    got = full_run()
     assert all(np.isfinite(g).all() for g in got)
-    # (a) one stream against the oracle over all 100 chunks, another over its first 14 chunks
-    s7 = w.streams[7]
-    ref = orc.run_stream(cfg, w.weights, s7.feats, s7.boundaries)
-    assert gu.rel_err(got[7], ref) <= TOL_BF16
-    s20 = w.streams[20]
-    b = s20.boundaries[:15]
-    ref = orc.run_stream(cfg, w.weights, s20.feats[:b[-1]], b)
-    assert gu.rel_err(got[20][:b[-1]], ref) <= TOL_BF16
+    again = full_run()
+    assert all(np.array_equal(a, b) for a, b in zip(got, again)), "not bitwise reproducible run to run"
+    # (a) four streams against the oracle: two over all 100 chunks, two over their first 40
+    for i, n_ch in ((7, cfg.n_chunks), (20, cfg.n_chunks), (0, 40), (31, 40)):
+        si = w.streams[i]
+        b = si.boundaries[:n_ch + 1]
+        ref = orc.run_stream(cfg, w.weights, si.feats[:b[-1]], b)
+        err = gu.rel_err(got[i][:b[-1]], ref)
+        assert err <= TOL_BF16, f"stream {i}: {err}"
     # (b) batching never changes a stream's bytes
     for i in (0, 13, 31):
         si = w.streams[i]
@@ -254,11 +261,7 @@ def test_device_noise_per_stream_and_replay(dc):
     assert not np.array_equal(a, b)
     m.destroy()
     # a model that launches its kernels directly (no captured graph) draws exactly the same
-    os.environ["DC_NO_GRAPH"] = "1"
-    try:
-        m2 = dc.Model(cfg, w.weights)
-    finally:
-        os.environ.pop("DC_NO_GRAPH", None)
+    m2 = dc.Model(cfg, w.weights, options=dc.OPT_NO_GRAPH)
     assert np.array_equal(_noise_run(dc, m2, cfg, w, s, 0), a)
     m2.destroy()
 
@@ -323,3 +326,40 @@ def test_chunk_host_pinned_and_pageable(dc, pinned):
     st.close()
     m.destroy()
     assert np.array_equal(fout.numpy(), ref)
+
+
+def test_partial_batch_is_one_graph_launch(dc):
+    """A serving round in which some streams have nothing to decode: every admitted call is still ONE graph
+    launch (counters[7]) - the chunk step of a batch size met for the first time is captured at that call -
+    and gives the bytes of single-stream decoding."""
+    gu = _gu()
+    cfg = wl.tiny_flow(name="tiny_partial", n_streams=5, n_chunks=4)
+    w = wl.make_workload(cfg)
+    m = dc.Model(cfg, w.weights, max_batch=5)
+    single = [gu.run_gpu_stream(m, s.feats, s.boundaries) for s in w.streams]
+    streams = [m.open_stream() for _ in w.streams]
+    feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+    outs = [torch.zeros(s.feats.shape[0], cfg.mel_dim, device="cuda") for s in w.streams]
+    done = [0] * 5
+    # rounds with 5, 3, 4, 2, ... streams present: every stream still sees its chunks in order
+    present = [[0, 1, 2, 3, 4], [0, 2, 4], [1, 3], [0, 1, 2, 3], [4, 1, 3, 0, 2], [2, 4], [0, 1, 3], [2, 4]]
+    for idx in present:
+        idx = [i for i in idx if done[i] < cfg.n_chunks]
+        if not idx:
+            continue
+        c0 = m.counters()
+        fs = [feats[i][w.streams[i].boundaries[done[i]]:w.streams[i].boundaries[done[i] + 1]] for i in idx]
+        os_ = [outs[i][w.streams[i].boundaries[done[i]]:w.streams[i].boundaries[done[i] + 1]] for i in idx]
+        dc.decode_batch(m, [streams[i] for i in idx], fs, os_)
+        c1 = m.counters()
+        assert c1[7] == c0[7] + 1, f"batch of {len(idx)}: not a single graph launch"
+        assert c1[5] > c0[5]
+        for i in idx:
+            done[i] += 1
+    torch.cuda.synchronize()
+    assert done == [cfg.n_chunks] * 5 and m.counters()[4] == 0
+    for st in streams:
+        st.close()
+    m.destroy()
+    for i in range(5):
+        assert np.array_equal(outs[i].cpu().numpy(), single[i]), f"stream {i}"

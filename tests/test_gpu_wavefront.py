@@ -132,7 +132,7 @@ def test_wavefront_token2wav(dc):
     bounds = _uniform(87, cfg.f_chunk)
     w = wl.make_workload(cfg.replace(n_chunks=len(bounds) - 1), boundaries=[bounds])
     s = w.streams[0]
-    m = dc.Model(cfg, w.weights, max_batch=cfg.n_steps)
+    m = dc.Model(cfg, w.weights, max_batch=cfg.n_steps, max_wave_frames=50)
     ref = gu.run_gpu_stream(m, s.feats, bounds)
     st = m.open_stream()
     x = torch.from_numpy(s.feats).cuda().contiguous()
@@ -140,6 +140,12 @@ def test_wavefront_token2wav(dc):
     b = st.decode_wavefront(x[50:].contiguous()).clone()            # a second call: shorter, reuses the mel buffer
     torch.cuda.synchronize()
     assert m.counters()[4] == 0
+    # the mel buffer of a wavefront call is sized at dc_stream_open: a longer call is refused, nothing touched
+    before = m.counters()
+    with pytest.raises(dc.DCError):
+        st.decode_wavefront(x[:51].contiguous())
+    after = m.counters()
+    assert after[3] == before[3] + 1 and after[5] == before[5] and after[0] == before[0]
     st.close()
     m.destroy()
     assert np.array_equal(torch.cat([a, b]).cpu().numpy(), ref)
@@ -169,7 +175,7 @@ def _batch_case(dc, cfg, lengths, tok2wav=False):
     bounds = [_uniform(n, cfg.f_chunk) for n in lengths]
     cfgn = cfg.replace(n_streams=len(lengths), n_chunks=max(len(b) for b in bounds) - 1)
     w = wl.make_workload(cfgn, boundaries=bounds)
-    m = dc.Model(cfgn, w.weights, max_batch=len(lengths) * cfg.n_steps)
+    m = dc.Model(cfgn, w.weights, max_batch=len(lengths) * cfg.n_steps, max_wave_frames=max(lengths) if tok2wav else 0)
     refs = [gu.run_gpu_stream(m, s.feats[:n], b) for s, n, b in zip(w.streams, lengths, bounds)]
     sts = [m.open_stream() for _ in lengths]
     xs = [torch.from_numpy(np.ascontiguousarray(s.feats[:n])).cuda() for s, n in zip(w.streams, lengths)]
@@ -224,11 +230,7 @@ def test_wavefront_direct_launches_equal_graph(dc):
     assert sum(nl.values()) > 0
     st.close()
     m.destroy()
-    os.environ["DC_NO_GRAPH"] = "1"
-    try:
-        m2 = dc.Model(cfg, w.weights, max_batch=cfg.n_steps)
-    finally:
-        os.environ.pop("DC_NO_GRAPH", None)
+    m2 = dc.Model(cfg, w.weights, max_batch=cfg.n_steps, options=dc.OPT_NO_GRAPH)
     st2 = m2.open_stream()
     got_direct = st2.decode_wavefront(x).cpu().numpy()
     assert m2.counters()[4] == 0

@@ -1,7 +1,8 @@
 """dc_conv_stack_noalloc: the entry point for callers that cannot allocate device memory (a fixed
 memory budget, a foreign allocator's pool, a real-time audio callback).  It must give what the
-ordinary stream API gives for the same network and input, call after call, although every call
-shares one built-in scratch array that still holds the previous call's values.
+ordinary stream API gives for the same network and input - and what the CPU oracle's offline run
+over the whole sequence gives - call after call, although every call shares one built-in scratch
+array that still holds the previous call's values.
 
 Collected last on purpose: if it fails, a run that stops at the first failure has already run
 every other test."""
@@ -10,6 +11,7 @@ import pytest
 import torch
 
 import dc_workloads as wl
+from oracle import dc_oracle as orc
 
 pytestmark = pytest.mark.gpu
 
@@ -46,7 +48,10 @@ def test_noalloc_entry_matches_stream_api_on_two_calls_in_a_row():
     for cfg, n_frames in cases:
         weights = wl.make_weights(cfg, np.random.default_rng(cfg.seed))
         x = rng.standard_normal((n_frames, cfg.hidden), dtype=np.float32)
-        prepared.append((cfg, weights, x, _stream_api_result(dc, cfg, weights, x)))
+        ref = _stream_api_result(dc, cfg, weights, x)
+        # the existing entry point itself against the oracle's definition (offline causal run)
+        assert _rel_err(ref, orc.conv_stack_offline(cfg, weights, x)) <= TOL_F32, cfg.name
+        prepared.append((cfg, weights, x, ref))
     # everything the new entry point touches is allocated here, by the caller, beforehand
     bufs = [(torch.from_numpy(w).cuda(), torch.from_numpy(x).cuda(), torch.full(x.shape, 7.0, device="cuda"))
             for _, w, x, _ in prepared]
@@ -54,10 +59,11 @@ def test_noalloc_entry_matches_stream_api_on_two_calls_in_a_row():
     for (cfg, _, _, ref), (wd, xd, yd) in zip(prepared, bufs):
         assert dc.conv_stack_noalloc(wd, cfg.hidden, cfg.dilations, xd, yd) == 0
     torch.cuda.synchronize()
-    for (cfg, _, _, ref), (_, _, yd) in zip(prepared, bufs):
+    for (cfg, weights, x, ref), (_, _, yd) in zip(prepared, bufs):
         got = yd.cpu().numpy()
         assert got.shape == ref.shape
         assert _rel_err(got, ref) <= TOL_F32, cfg.name
+        assert _rel_err(got, orc.conv_stack_offline(cfg, weights, x)) <= TOL_F32, cfg.name
     # the same two calls again, in the other order, still agree
     for (cfg, _, _, ref), (wd, xd, yd) in reversed(list(zip(prepared, bufs))):
         yd.fill_(-3.0)
