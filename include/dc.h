@@ -65,12 +65,20 @@ enum { DC_PIPE_CONV = 1, DC_PIPE_FLOW = 2, DC_PIPE_VOCODER = 3, DC_PIPE_TOKEN2WA
 enum { DC_F32 = 0, DC_BF16 = 1 };   /* DC_BF16: bf16 storage and operands, fp32 accumulation */
 
 /* dc_config.options: switches for tests and measurements.  None of the first four changes a result
- * byte.  (There is no configuration by environment variable.) */
+ * byte; DC_OPT_ROUNDED_NORM selects the other of two admissible roundings.  (There is no configuration
+ * by environment variable.) */
 enum {
   DC_OPT_NO_GRAPH     = 1,        /* decode calls issue their kernels one by one instead of one captured graph  */
   DC_OPT_NO_PDL       = 2,        /* no programmatic dependent launch between the kernels of a step             */
   DC_OPT_NO_ZEROCOPY  = 4,        /* the *_host calls always stage, also for page-locked caller buffers         */
   DC_OPT_SERIAL_TAILS = 8,        /* token2wav dc_decode_batch: the vocoder tails one after another             */
+  /* Flow decoder: the RMS-normalised activations are written as a tensor of their own, rounded to bf16, and
+   * the projections read it - the storage-point reading of "bf16 activations" taken literally - instead of
+   * the default, which folds the norm into the projection as a scale of its fp32 accumulator rows and so
+   * skips that one rounding (results of the two forms differ by a few 1e-3 of RMS; the folded form costs one
+   * kernel and one activation round trip less per norm).  DC_PIPE_TOKEN2WAV always builds its flow decoder
+   * this way: the vocoder tail amplifies the flow stage's deviation several times. */
+  DC_OPT_ROUNDED_NORM = 16,
   /* MEASUREMENT ONLY - the outputs of such a model are meaningless: the step without the kernels of
    * one class, so that step-time differences give that class's cost inside the captured graph. */
   DC_OPT_SKIP_CONV_GEMM = 1 << 16,

@@ -91,7 +91,7 @@ def load_library():
     return lib
 
 
-OPT_NO_GRAPH, OPT_NO_PDL, OPT_NO_ZEROCOPY, OPT_SERIAL_TAILS = 1, 2, 4, 8
+OPT_NO_GRAPH, OPT_NO_PDL, OPT_NO_ZEROCOPY, OPT_SERIAL_TAILS, OPT_ROUNDED_NORM = 1, 2, 4, 8, 16
 OPT_SKIP_CONV_GEMM, OPT_SKIP_ATTENTION = 1 << 16, 1 << 17     # measurement only: outputs are meaningless
 
 

@@ -152,7 +152,7 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (c->f_lookahead != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_lookahead belongs to the flow decoder");
   if (c->f_prompt != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_prompt belongs to the flow decoder");
   if (c->cfg_scale != 0.f && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("cfg_scale belongs to the flow decoder");
-  if (c->options & ~(uint32_t)(DC_OPT_NO_GRAPH | DC_OPT_NO_PDL | DC_OPT_NO_ZEROCOPY | DC_OPT_SERIAL_TAILS | DC_OPT_SKIP_CONV_GEMM |
+  if (c->options & ~(uint32_t)(DC_OPT_NO_GRAPH | DC_OPT_NO_PDL | DC_OPT_NO_ZEROCOPY | DC_OPT_SERIAL_TAILS | DC_OPT_ROUNDED_NORM | DC_OPT_SKIP_CONV_GEMM |
                                DC_OPT_SKIP_ATTENTION))
     BAD("unknown option bit");
   if (c->max_wave_frames < 0 || c->max_wave_frames > (1 << 24)) BAD("max_wave_frames out of range");
@@ -299,7 +299,9 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
   for (auto& c : m->counters) c = 0;
   dc_status st = DC_OK;
   if (cfg->pipeline == DC_PIPE_TOKEN2WAV) {
-    const dc_config f = sub_config(*cfg, DC_PIPE_FLOW), v = sub_config(*cfg, DC_PIPE_VOCODER);
+    dc_config f = sub_config(*cfg, DC_PIPE_FLOW);
+    const dc_config v = sub_config(*cfg, DC_PIPE_VOCODER);
+    f.options |= DC_OPT_ROUNDED_NORM;   // the vocoder tail expands the flow stage's deviation: keep every declared rounding
     const size_t nf = dc_weights_count(&f);
     st = dc_create(w, nf, &f, &m->sub_flow);
     if (st == DC_OK) st = dc_create(w + nf, n_floats - nf, &v, &m->sub_voc);

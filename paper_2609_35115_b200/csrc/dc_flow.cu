@@ -588,6 +588,36 @@ __global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, 
   }
 }
 
+// u = bf16(x * rsqrt(mean(x^2) + eps)), one warp per chunk row: the normalised activation as a stored, rounded
+// tensor (DC_OPT_ROUNDED_NORM) instead of a row scale folded into the consuming GEMM's accumulator.  The row
+// statistic is the one the producing GEMM left (partial sums of squares per 16-column chunk, added in chunk
+// order), so both forms of the norm use the same 1 / rms.
+__global__ void flow_rmsnorm_kernel(const SlotInfo* slots, int n_slots, const bf16* x, bf16* u, int C, const float* ssq, long long ssq_ld,
+                                    float inv_C, float eps) {
+  ptx::pdl_launch();
+  ptx::pdl_wait();
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  const int slot = warp / SLOT_ROWS, rho = warp % SLOT_ROWS;
+  if (slot >= n_slots) return;
+  const int f = rho - HALO;
+  if (f < 0 || f >= slots[slot].T) return;
+  float ss = 0.f;
+  for (int j = 0; j < (C >> 4); ++j) ss += ssq[(long long)j * ssq_ld + warp];
+  const float rs = rsqrtf(ss * inv_C + eps);
+  const long long off = (long long)(GUARD + warp) * C;
+  for (int c = lane * 8; c < C; c += 256) {
+    const uint4 v = *reinterpret_cast<const uint4*>(x + off + c);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(w[i] << 16) * rs, __uint_as_float(w[i] & 0xFFFF0000u) * rs);
+      o[i] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(u + off + c) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 // ---- chunk-causal attention with the K/V carry ---------------------------------------------------
 // One CTA per (stream slot, head), two CTAs per SM.  Queries: the T <= 56 chunk frames, held TWICE
 // in the 128 UMMA rows (row 64 + i repeats row i), so that S has a copy of every query row in both
@@ -1021,13 +1051,14 @@ struct FlowModel {
   int n_pass = 1;            // 2 with classifier-free guidance: a stream's conditional and unconditional pass are
                              // adjacent slots, i.e. the two halves of one row tile
   bf16 *Xa = nullptr, *Xb = nullptr, *Q = nullptr, *O = nullptr, *Ain = nullptr;
+  bf16 *U = nullptr;         // DC_OPT_ROUNDED_NORM: the normalised activations as a stored bf16 tensor
   float* xstate = nullptr;
   float* ssq = nullptr;      // [C / 16][rows]: per-chunk sums of squares of the rows that feed an RMS norm
   bf16*  wts = nullptr;
   float* fconst = nullptr;   // biases and the timestep-bias table
   SlotInfo* d_slots = nullptr;
   int*   d_err = nullptr;
-  CUtensorMap tmAin, tmXa, tmXb, tmO;
+  CUtensorMap tmAin, tmXa, tmXb, tmO, tmU;
   // weight maps in three tile-width variants v (box rows = N tile): v = 0 wide (64 / 192 / mel), for full
   // batches; v = 1, 2 narrower (32, 16 / 96, 48 / 16), so that a small batch still spreads over many SMs
   CUtensorMap tmWin[3], tmWout[3];
@@ -1200,6 +1231,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   chk(dalloc(m, &m->Xa, R * C));
   chk(dalloc(m, &m->Xb, R * C));
   chk(dalloc(m, &m->ssq, (size_t)(C / 16) * m->rows));
+  if (cfg.options & DC_OPT_ROUNDED_NORM) chk(dalloc(m, &m->U, R * C));
   chk(dalloc(m, &m->Q, R * C));
   chk(dalloc(m, &m->O, R * C));
   chk(dalloc(m, &m->Ain, R * m->Kin));
@@ -1224,6 +1256,7 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   ok &= make_tmap(&m->tmXa, m->Xa, R, C, A_ROWS);
   ok &= make_tmap(&m->tmXb, m->Xb, R, C, A_ROWS);
   ok &= make_tmap(&m->tmO, m->O, R, C, A_ROWS);
+  if (m->U) ok &= make_tmap(&m->tmU, m->U, R, C, A_ROWS);
   for (int v = 0; v < 3; ++v) {
     const int bn = 64 >> v, bq = 192 >> v, bo = 16;
     ok &= make_tmap(&m->tmWin[v], m->wts + w_in, C, m->Kin, bn);
@@ -1438,6 +1471,13 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
   auto normalised = [&](GemmParams& p) {
     p.ssq_in = m->ssq; p.ssq_ld = m->rows; p.inv_C = 1.0f / (float)C; p.eps = c.rms_eps;
   };
+  // DC_OPT_ROUNDED_NORM: a kernel of its own writes u = bf16(x / rms) and the projection reads u unscaled
+  const bool rounded_norm = m->U != nullptr;
+  auto rmsnorm = [&](const bf16* x) {
+    const int warps = n * SLOT_ROWS;
+    launch(lc, flow_rmsnorm_kernel, dim3((warps * 32 + 255) / 256), dim3(256), 0, true, 3, (const SlotInfo*)m->d_slots, n, x, m->U, C,
+           (const float*)m->ssq, (long long)m->rows, 1.0f / (float)C, c.rms_eps);
+  };
   auto attention = [&](int step, int layer) {
     AttnParams p{};
     p.slots = m->d_slots; p.q = m->Q; p.o = m->O; p.ld = C; p.dh = c.head_dim;
@@ -1488,8 +1528,13 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
           p.bias = fc + m->o_bqkv[g]; p.q_out = m->Q; p.halo_off = -1;
           p.kv_off = ((long long)s * c.n_attn + g) * 2 * (m->P + m->Rk) * C;
           p.kv_rs = m->kv_rs; p.kv_hs = m->kv_hs; p.dh_shift = m->dh_shift;
-          normalised(p);
-          gemm(*tX, m->tmWqkv[v][g], p, 3 * C);
+          if (rounded_norm) {
+            rmsnorm(X);
+            gemm(m->tmU, m->tmWqkv[v][g], p, 3 * C);
+          } else {
+            normalised(p);
+            gemm(*tX, m->tmWqkv[v][g], p, 3 * C);
+          }
         }
         if (!(c.options & DC_OPT_SKIP_ATTENTION)) attention(s, g);   // (measurement only: the step without this class)
         {
@@ -1509,8 +1554,13 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       p.bias = fc + m->o_bout; p.halo_off = -1;
       p.xstate = m->xstate; p.ain = m->Ain; p.ld_ain = m->Kin; p.inv_n = 1.0f / c.n_steps;
       p.last_step = (!tick && s == c.n_steps - 1); p.mel = mel; p.cfg_w = c.cfg_scale;
-      normalised(p);
-      gemm(*tX, m->tmWout[v], p, mel);
+      if (rounded_norm) {
+        rmsnorm(X);
+        gemm(m->tmU, m->tmWout[v], p, mel);
+      } else {
+        normalised(p);
+        gemm(*tX, m->tmWout[v], p, mel);
+      }
     }
   }
 }

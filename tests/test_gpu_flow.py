@@ -363,3 +363,33 @@ def test_partial_batch_is_one_graph_launch(dc):
     m.destroy()
     for i in range(5):
         assert np.array_equal(outs[i].cpu().numpy(), single[i]), f"stream {i}"
+
+
+def test_rounded_norm_option_matches_oracle_and_batching(dc):
+    """DC_OPT_ROUNDED_NORM: the normalised activations stored and rounded to bf16 by a kernel of their own (the
+    storage-point reading taken literally) instead of a scale folded into the projection's accumulator."""
+    gu = _gu()
+    cfg = wl.tiny_flow(name="tiny_rounded", n_streams=3, n_chunks=5)
+    w = wl.make_workload(cfg)
+    m = dc.Model(cfg, w.weights, max_batch=3, options=dc.OPT_ROUNDED_NORM)
+    single = [gu.run_gpu_stream(m, s.feats, s.boundaries) for s in w.streams]
+    for s, got in zip(w.streams, single):
+        assert gu.rel_err(got, orc.run_stream(cfg, w.weights, s.feats, s.boundaries)) <= TOL_BF16
+    streams = [m.open_stream() for _ in w.streams]
+    feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+    outs = [torch.zeros(s.feats.shape[0], cfg.mel_dim, device="cuda") for s in w.streams]
+    for r in range(cfg.n_chunks):
+        dc.decode_batch(m, streams, [feats[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(3)],
+                        [outs[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(3)])
+    torch.cuda.synchronize()
+    assert m.counters()[4] == 0
+    for st in streams:
+        st.close()
+    m.destroy()
+    for i in range(3):
+        assert np.array_equal(outs[i].cpu().numpy(), single[i])
+    # the two forms of the norm are different roundings of the same network, not different networks
+    m0 = dc.Model(cfg, w.weights)
+    folded = gu.run_gpu_stream(m0, w.streams[0].feats, w.streams[0].boundaries)
+    m0.destroy()
+    assert not np.array_equal(folded, single[0]) and gu.rel_err(folded, single[0].astype(np.float64)) <= TOL_BF16

@@ -2,11 +2,17 @@
 dc_decode_chunk, the mel frames staying on the device), through the C ABI.
 
 The vocoder tail is a strongly expanding map (exp of the log-magnitude channels): in the oracle
-itself, mel frames that differ by 7e-3 of their RMS give PCM that differs by 4e-2.  The parity of
-the chain is therefore stated stage by stage, on the data each stage really sees:
+itself, mel frames that differ by 4e-3 of their RMS give PCM that differs by about 3e-2.  The
+parity of the chain is therefore stated stage by stage, on the data each stage really sees:
   * the flow stage's mel frames against the oracle's flow decoder        (bf16 bar, 2e-2),
   * the PCM against the ORACLE's vocoder tail applied to the GPU's mel   (fp32 bar, 1e-4),
-and the distance of the PCM to the oracle's end-to-end chain is reported and loosely bounded."""
+and the distance of the PCM to the oracle's end-to-end chain is bounded by E2E_BOUND, the tightest
+round value that held on every case measured (2.7e-2 at full size, 2.9e-2 and 3.4e-2 on the tiny
+cases) with the flow stage keeping every declared bf16 rounding (the composite builds its flow
+decoder with the rounded RMS norm; with the folded norm the same cases gave 3.2e-2 to 4.6e-2).
+The 2e-2 bar of the bf16 pipelines is NOT met end to end: the flow stage sits 4e-3 from the oracle
+- fp32 accumulation against the oracle's float64 flips individual bf16 roundings - and the tail
+multiplies that by 6 to 7."""
 import numpy as np
 import pytest
 import torch
@@ -18,6 +24,7 @@ pytestmark = pytest.mark.gpu
 
 TOL_BF16 = 2e-2
 TOL_F32 = 1e-4
+E2E_BOUND = 4e-2
 RAGGED = [0, 3, 13, 14, 24, 31, 41, 51, 52, 62, 72, 80]
 
 
@@ -33,7 +40,7 @@ def _gu():
     return gpu_util
 
 
-def _stagewise(dc, cfg, boundaries=None, e2e_bound=0.1):
+def _stagewise(dc, cfg, boundaries=None, e2e_bound=E2E_BOUND):
     gu = _gu()
     w = wl.make_workload(cfg, boundaries=[boundaries] if boundaries else None)
     s = w.streams[0]
@@ -47,7 +54,7 @@ def _stagewise(dc, cfg, boundaries=None, e2e_bound=0.1):
     assert np.array_equal(pcm, pcm2), "reruns differ"
     assert pcm.shape == (s.boundaries[-1] * cfg.out_per_frame,) and np.isfinite(pcm).all()
     # the flow stage alone, same weights: its output is what the chain hands to the vocoder tail
-    mf = dc.Model(fc, w.weights[:nf])
+    mf = dc.Model(fc, w.weights[:nf], options=dc.OPT_ROUNDED_NORM)     # as the composite builds it
     mel = gu.run_gpu_stream(mf, s.feats, s.boundaries)
     mf.destroy()
     ref_mel = orc.run_stream(fc, w.weights[:nf], s.feats, s.boundaries)
@@ -57,7 +64,7 @@ def _stagewise(dc, cfg, boundaries=None, e2e_bound=0.1):
     ref_pcm_stage = orc.run_stream(vc, w.weights[nf:], mel, s.boundaries)
     e_voc = gu.rel_err(pcm, ref_pcm_stage)
     assert e_voc <= TOL_F32, f"vocoder stage: {e_voc}"
-    # end to end against the oracle's chain: reported, bounded loosely (see the module docstring)
+    # end to end against the oracle's chain (see the module docstring)
     ref = orc.run_stream(cfg, w.weights, s.feats, s.boundaries)
     e_all = gu.rel_err(pcm, ref)
     print(f"{cfg.name}: flow stage {e_mel:.2e}, vocoder stage {e_voc:.2e}, end to end {e_all:.2e}")
@@ -84,7 +91,7 @@ def test_chain_equals_the_two_models_by_hand(dc):
     m = dc.Model(cfg, w.weights)
     pcm = gu.run_gpu_stream(m, s.feats, s.boundaries)
     m.destroy()
-    mf, mv = dc.Model(cfg.flow_part(), w.weights[:nf]), dc.Model(cfg.vocoder_part(), w.weights[nf:])
+    mf, mv = dc.Model(cfg.flow_part(), w.weights[:nf], options=dc.OPT_ROUNDED_NORM), dc.Model(cfg.vocoder_part(), w.weights[nf:])
     sf, sv = mf.open_stream(), mv.open_stream()
     x = torch.from_numpy(s.feats).cuda()
     outs = []
