@@ -36,9 +36,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # FP32 FFMA peak of the part: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (no measured figure exists)
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 HISTORY_CHUNKS = 12      # untimed stream history so that the K/V carry sits at its cap (steady state)
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until a capture exists for that workload)
-NCU_TRAFFIC_BYTES = {"cfg5": 4.00e6,   # conv-mode flow_gemm_kernel, profiles/flow_gemm_kernel_conv_cfg5.md
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from an ncu capture of
+# this command (a figure of a capture, not read in the run; None until a capture exists for that workload)
+NCU_TRAFFIC_BYTES = {"cfg5": 4.00e6,   # conv-mode flow_gemm_kernel
                      "cfg3": None, "cfg2": None, "cfg4": None, "cfg1": None}
 
 
@@ -277,20 +277,29 @@ def main():
     rng = np.random.default_rng(cfg.seed + 1000 * rank)
     weights = wl.make_weights(cfg, np.random.default_rng(cfg.seed))
     model = dc.Model(cfg, weights, max_batch=S)
-    streams = [model.open_stream() for _ in range(S)]
     feats_h = torch.from_numpy(rng.standard_normal((rounds, S, Tp, cfg.in_dim), dtype=np.float32))
     feats_d = feats_h.cuda()
-    out_d = torch.empty(S, T * cfg.out_per_frame, device="cuda")
-    out_dv = out_d.view(S, T, -1) if cfg.pipeline not in ("vocoder", "token2wav") else out_d
+    out_all = torch.empty(K, S, T * cfg.out_per_frame, device="cuda")     # every timed step's output, hashed after the run
+    out_d = out_all[0]
+    as_rows = cfg.pipeline not in ("vocoder", "token2wav")
+    out_dv = out_d.view(S, T, -1) if as_rows else out_d
     batched = cfg.pipeline in ("flow", "token2wav") and S > 1
     batched_host = cfg.pipeline == "flow" and S > 1     # the host-buffer batch call serves the flow pipeline only
+    # multi-stream serving: the streams' chunk boundaries are staggered by seeded offsets in [0, f_chunk) - stream i's
+    # first chunk has o_i frames (a full chunk if o_i = 0), every later one f_chunk
+    offsets = np.random.default_rng(cfg.seed).integers(0, T, S) if (batched and S > 1) else np.zeros(S, dtype=np.int64)
+    streams = []
 
-    def step(r):
-        if batched:
-            dc.decode_batch(model, streams, feats_d[r], out_dv)
+    def step(r, out=None):
+        o = out_d if out is None else out
+        if batched and r == 0 and offsets.any():
+            t0 = [int(x) if x > 0 else T for x in offsets]
+            dc.decode_batch(model, streams, [feats_d[0, i, :t0[i]] for i in range(S)], [o[i, :t0[i] * cfg.out_per_frame] for i in range(S)])
+        elif batched:
+            dc.decode_batch(model, streams, feats_d[r], o.view(S, T, -1) if as_rows else o)
         else:
             for i in range(S):
-                streams[i].decode_chunk(feats_d[r, i], out=out_d[i])
+                streams[i].decode_chunk(feats_d[r, i], out=o[i])
 
     def sync_all():
         torch.cuda.synchronize()
@@ -299,39 +308,57 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    def timed_run():
+        """Freshly opened streams, history + warm-up, then exactly K timed steps.  Returns per-step events' times,
+        the total, the launch count and a hash of every timed step's output."""
+        import hashlib
+        for s_ in streams:
+            s_.close()
+        streams[:] = [model.open_stream() for _ in range(S)]
+        for r in range(history + W):
+            step(r)
+        sync_all()
+        c0 = model.counters()
+        t_host0 = time.perf_counter()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+        evs[0].record()
+        for k in range(K):
+            step(history + W + k, out_all[k])
+            evs[k + 1].record()
+        torch.cuda.synchronize()
+        t_host1 = time.perf_counter()
+        c1 = model.counters()
+        digest = hashlib.sha256(out_all.cpu().numpy().tobytes()).hexdigest()
+        return {"total_ms": evs[0].elapsed_time(evs[K]), "step_ms": sorted(evs[k].elapsed_time(evs[k + 1]) for k in range(K)),
+                "launches": int(c1[5] - c0[5]), "graph_launches": int(c1[7] - c0[7]), "hash": digest, "host": (t_host0, t_host1)}
+
     sampler = ClockSampler(local)
     sampler.start()          # nvidia-smi needs a moment before its first sample: start it ahead of the timed region
-    for r in range(history + W):
-        step(r)
-    sync_all()
-    c0 = model.counters()
-    t_timed0 = time.perf_counter()
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
-    evs[0].record()
-    for k in range(K):
-        step(history + W + k)
-        evs[k + 1].record()
-    torch.cuda.synchronize()
-    t_timed1 = time.perf_counter()
-    total_ms = evs[0].elapsed_time(evs[K])
-    c1 = model.counters()
+    n_rep = 5
+    runs = [timed_run() for _ in range(n_rep)]
+    if len({r_["hash"] for r_ in runs}) != 1:
+        raise SystemExit("bench: the outputs of repeated runs differ (the decoder step must be byte-reproducible)")
+    runs_sorted = sorted(runs, key=lambda r_: r_["total_ms"])
+    med = runs_sorted[n_rep // 2]
+    total_ms, step_ms = med["total_ms"], med["step_ms"]
+    c_launches, c_graphs = med["launches"], med["graph_launches"]
     # The timed region of a short run is over before nvidia-smi (50 ms period) has sampled it a few
     # times: keep the same steps running, untimed, for about a second and sample that load as well.
-    windows = {"timed_region": (t_timed0, t_timed1)}
-    if t_timed1 - t_timed0 < 0.5:
-        t_p0 = time.perf_counter()
-        k = 0
-        while time.perf_counter() - t_p0 < 1.0:
-            step(history + W + (k % K))
-            k += 1
-            if k % 8 == 0:
-                torch.cuda.synchronize()
-        torch.cuda.synchronize()
-        windows["same_steps_untimed"] = (t_p0, time.perf_counter())
+    windows = {f"timed_region_{i}": r_["host"] for i, r_ in enumerate(runs)}
+    t_p0 = time.perf_counter()
+    k = 0
+    while time.perf_counter() - t_p0 < 1.0:
+        step(history + W + (k % K))
+        k += 1
+        if k % 8 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    windows["same_steps_untimed"] = (t_p0, time.perf_counter())
     clocks = sampler.stop(windows)
-    step_ms = sorted(evs[k].elapsed_time(evs[k + 1]) for k in range(K))
     total_ms = max_over_ranks(total_ms, world)
     value = aggregate_throughput(world, S, K, per_chunk, total_ms * 1e-3)
+    repeats = {"runs": n_rep, "ms_per_step": [r_["total_ms"] / K for r_ in runs], "reported": "median run",
+               "fresh_streams_per_run": True, "outputs_sha256_identical": True, "sha256": med["hash"][:16]}
 
     # ---- the same step with L2 flushed first (workloads whose working set fits L2 only): a stream paced
     # at its real-time cadence finds its weights and carries in HBM, not in L2 ----
@@ -427,6 +454,11 @@ def main():
 
     # ---- per-kernel-class device time (separate profiled pass; events between launches slow the step) ----
     pk, how = peaks()
+    # Tensor peak to divide by: the burst figure (a GEMM timed alone at full clock) when this run's SM clock sat at
+    # its maximum, the sustained one (seconds of GEMM under the power cap) when it did not; the other is printed beside it.
+    at_max = bool(clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] >= 0.97 * clocks["sm_max_mhz"])
+    tensor_peak = pk["bf16_tflops"] if at_max else pk["bf16_tflops_sustained"]
+    tensor_kind = f"bf16 {'burst (SM clock at max during the run)' if at_max else 'sustained'}, {how}"
     nprof = min(K, 3)
     model.profile_begin(1 << 15)
     for k in range(nprof):
@@ -440,7 +472,8 @@ def main():
     if dom in ("gemm_conv",):
         fl = flops_per_launch(cfg, dom, S)
         roof = {"kernel": "flow_gemm_kernel (conv blocks)", "bound": "tensor", "achieved": fl / avg_s / 1e12,
-                "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "peak_kind": f"bf16 sustained, {how}"}
+                "peak": tensor_peak, "unit": "TFLOP/s", "peak_kind": tensor_kind,
+                "frac_of_sustained_peak": fl / avg_s / 1e12 / pk["bf16_tflops_sustained"]}
     elif dom == "attention":
         by = attention_bytes_per_launch(cfg, S)
         roof = {"kernel": "flow_attn_kernel", "bound": "hbm", "achieved": by / avg_s / 1e9, "peak": pk["hbm_gbs"],
@@ -498,7 +531,8 @@ def main():
             us = 1e3 * (full_ms - step_ms_without(dc.OPT_SKIP_CONV_GEMM)) / n_conv_l
             in_graph["conv_gemm_us"] = us
             in_graph["conv_gemm_tflops"] = flops_per_launch(cfg, "gemm_conv", S) / (us * 1e-6) / 1e12
-            in_graph["conv_gemm_frac"] = in_graph["conv_gemm_tflops"] / pk["bf16_tflops_sustained"]
+            in_graph["conv_gemm_frac"] = in_graph["conv_gemm_tflops"] / tensor_peak
+            in_graph["conv_gemm_frac_of_sustained_peak"] = in_graph["conv_gemm_tflops"] / pk["bf16_tflops_sustained"]
         if n_att_l:
             us = 1e3 * (full_ms - step_ms_without(dc.OPT_SKIP_ATTENTION)) / n_att_l
             in_graph["attention_us"] = us
@@ -508,9 +542,14 @@ def main():
         # the whole step against the two rooflines (the paper's stage bound, Eq. 1: max of the compute time and
         # the memory time), next to the per-kernel figures above
         fl_step, by_step = flow_step_work(cfg, S)   # (token2wav workloads: the flow decoder's part of the work only)
-        t_floor = max(fl_step / (pk["bf16_tflops_sustained"] * 1e12), by_step / (pk["hbm_gbs"] * 1e9))
+        t_floor = max(fl_step / (tensor_peak * 1e12), by_step / (pk["hbm_gbs"] * 1e9))
         roof["step"] = {"flops": fl_step, "hbm_bytes": by_step, "floor_us": 1e6 * t_floor,
                         "measured_us": 1e3 * full_ms, "frac": t_floor / (1e-3 * full_ms)}
+        # the stage-latency floor: the same graph with kernels that return at once (same nodes, same launch attributes)
+        empty_ms = step_ms_without(dc.OPT_EMPTY_KERNELS)
+        n_nodes = c_launches // K
+        roof["t_sync"] = {"empty_step_us": 1e3 * empty_ms, "graph_nodes": n_nodes, "t_sync_us": 1e3 * empty_ms / max(n_nodes, 1),
+                          "method": "the step's graph with GEMM and attention kernels that return at once"}
 
     # ---- the oracle on the host cores (rank 0, N = 1 only), bounded sample ----
     cpu = None
@@ -530,14 +569,18 @@ def main():
                        "history_chunks": history, "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": (f"K/V carries {ws:.0f} MB > 126 MB L2, streamed from HBM every step" if ws > 126 else
                               "working set fits L2: value and latency_us are back-to-back chunks (warm L2), latency_us_cold_l2 flushes L2 before every step"),
-                       "inputs": "N(0,1) features, N(0,1/fan_in) weights, seeded"},
+                       "inputs": "N(0,1) features, N(0,1/fan_in) weights, seeded"
+                                 + ("; stream i's first chunk has a seeded o_i in [0, f_chunk) frames (staggered chunk boundaries)" if offsets.any() else ""),
+                       "protocol": f"{n_rep} runs of history + warm-up + K timed steps, each on freshly opened streams; outputs hashed, median run reported"},
             "latency_us": {"p50": 1e3 * step_ms[len(step_ms) // 2], "p95": 1e3 * step_ms[min(len(step_ms) - 1, int(0.95 * len(step_ms)))],
                            "per": "step (one chunk of every stream)"},
             "latency_us_cold_l2": cold,
             "wavefront": wave,
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": S * Tp * cfg.in_dim * 4,
                     "d2h_bytes_per_step": S * T * cfg.out_per_frame * 4, "ms_per_step": 1e3 * e2e_s / K},
-            "gpu_launches": int(c1[5] - c0[5]),
+            "gpu_launches": c_launches,
+            "graph_launches": c_graphs,
+            "repeats": repeats,
             "clocks": clocks,
             "roofline": roof,
             "kernels": kernels,

@@ -82,7 +82,11 @@ enum {
   /* MEASUREMENT ONLY - the outputs of such a model are meaningless: the step without the kernels of
    * one class, so that step-time differences give that class's cost inside the captured graph. */
   DC_OPT_SKIP_CONV_GEMM = 1 << 16,
-  DC_OPT_SKIP_ATTENTION = 1 << 17
+  DC_OPT_SKIP_ATTENTION = 1 << 17,
+  /* ... and the step whose GEMM and attention kernels return at once: same graph, same node count,
+   * same launch attributes; its time divided by the node count is the cost of a bare stage boundary
+   * (the t_sync of the stage-latency floor n_stages x t_sync; paper Section 2.2, T_o = sum t_k + G_o). */
+  DC_OPT_EMPTY_KERNELS  = 1 << 18
 };
 
 #define DC_MAX_CONV 32

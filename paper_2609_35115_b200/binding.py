@@ -92,7 +92,7 @@ def load_library():
 
 
 OPT_NO_GRAPH, OPT_NO_PDL, OPT_NO_ZEROCOPY, OPT_SERIAL_TAILS, OPT_ROUNDED_NORM = 1, 2, 4, 8, 16
-OPT_SKIP_CONV_GEMM, OPT_SKIP_ATTENTION = 1 << 16, 1 << 17     # measurement only: outputs are meaningless
+OPT_SKIP_CONV_GEMM, OPT_SKIP_ATTENTION, OPT_EMPTY_KERNELS = 1 << 16, 1 << 17, 1 << 18     # measurement only: outputs are meaningless
 
 
 def make_config(cfg, max_batch: int = 1, max_wave_frames: int = 0, options: int = 0) -> dc_config:

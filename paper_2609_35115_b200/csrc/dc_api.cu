@@ -153,7 +153,7 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (c->f_prompt != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_prompt belongs to the flow decoder");
   if (c->cfg_scale != 0.f && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("cfg_scale belongs to the flow decoder");
   if (c->options & ~(uint32_t)(DC_OPT_NO_GRAPH | DC_OPT_NO_PDL | DC_OPT_NO_ZEROCOPY | DC_OPT_SERIAL_TAILS | DC_OPT_ROUNDED_NORM | DC_OPT_SKIP_CONV_GEMM |
-                               DC_OPT_SKIP_ATTENTION))
+                               DC_OPT_SKIP_ATTENTION | DC_OPT_EMPTY_KERNELS))
     BAD("unknown option bit");
   if (c->max_wave_frames < 0 || c->max_wave_frames > (1 << 24)) BAD("max_wave_frames out of range");
   if (c->max_wave_frames != 0 && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("max_wave_frames belongs to the token2wav pipeline");

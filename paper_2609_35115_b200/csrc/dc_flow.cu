@@ -117,6 +117,7 @@ struct GemmParams {
   long long    ssq_ld;          // rows per chunk plane
   float        inv_C, eps;
   int*         err;
+  int          empty;           // measurement only: the kernel returns at once (the cost of the bare stage boundary)
 };
 
 // SiLU(z) = z * sigmoid(z) = 0.5 z (1 + tanh(z / 2)): one MUFU op per element instead of two (exp + reciprocal);
@@ -147,6 +148,11 @@ __device__ __forceinline__ void store16(bf16* p, const uint4& a, const uint4& b)
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
+  if (p.empty) {
+    ptx::pdl_launch();
+    ptx::pdl_wait();
+    return;
+  }
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   // stage = [A tile 128 x 128 B | one B tile BN x 128 B per tap]; all tile sizes are multiples of
   // 1024 B.  The weight tiles of a conv block's three taps are adjacent, so that they form one
@@ -667,6 +673,7 @@ struct AttnParams {
   int             P;          // prompt rows in front of the ring
   float           scale_log2e;  // log2(e) / sqrt(dh)
   int*            err;
+  int             empty;      // measurement only: the kernel returns at once (the cost of the bare stage boundary)
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -685,6 +692,11 @@ template <bool PROMPT>
 __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t att_smem_raw[];
   uint8_t* smem = att_smem_raw;
+  if (p.empty) {
+    ptx::pdl_launch();
+    ptx::pdl_wait();
+    return;
+  }
   if ((ptx::smem_u32(smem) & 1023u) != 0u) {   // would corrupt the swizzled tiles: refuse (uniform for the CTA)
     if (threadIdx.x == 0) atomicExch(p.err, 14);
     return;
@@ -1447,6 +1459,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     p.Rk = m->Rk;
     p.P = m->P;
     p.err = m->d_err;
+    p.empty = (c.options & DC_OPT_EMPTY_KERNELS) ? 1 : 0;
     const int stage_bytes = A_BYTES + p.taps * ((p.BN * 128 + 1023) & ~1023);
     // the issuer count fixes the summation order, so it depends on the GEMM's role only, never on the tile
     // width chosen for the batch size (batched and single-stream results must agree bit for bit);
@@ -1486,6 +1499,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     p.kv_rs = m->kv_rs; p.kv_hs = m->kv_hs;
     p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
     p.err = m->d_err;
+    p.empty = (c.options & DC_OPT_EMPTY_KERNELS) ? 1 : 0;
     launch(lc, m->P > 0 ? flow_attn_kernel<true> : flow_attn_kernel<false>, dim3(n, c.n_heads), dim3(ATT_THREADS), ATT_SMEM, true, 2, p);
   };
   const float* fc = m->fconst;
