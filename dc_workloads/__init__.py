@@ -64,6 +64,8 @@ class DCConfig:
     logmag_clamp: float = math.log(100.0)
     noise_seed: int = 0                 # flow decoder: != 0: the Euler noise x_0 is drawn on the device (Philox), feats = mu only
     cfg_scale: float = 0.0              # flow decoder: classifier-free guidance weight w (0 = off, one pass per step)
+    excitation_std: float = 0.0         # vocoder: > 0: Gaussian excitation of this standard deviation, drawn on the device, added
+    excitation_seed: int = 0            # ... after the last transposed conv (its generator key; must be != 0 then)
     # workload (not part of the network)
     n_chunks: int = 1
     n_streams: int = 1

@@ -262,6 +262,24 @@ def device_noise(seed: int, stream_id: int, frame0: int, n_frames: int, mel: int
     return z.reshape(n_frames, mel)
 
 
+def excitation_noise(seed: int, stream_id: int, t0: int, n: int, C: int) -> np.ndarray:
+    """The vocoder's random excitation (the device-random source of Sec. 3.1 / Sec. 3.3 effect classification,
+    clause (iii): admitted because its generator offset is a function of the call clock).  Rows are frames
+    t0 .. t0 + n - 1 at the rate of the last upsampling stage, counted from the stream start; the draw of
+    (frame t, channels 4g .. 4g+3) is Philox4x32-10 at counter (t mod 2^32, t div 2^32, g, 2^31 + stream id) -
+    the high bit keeps these draws apart from the flow decoder's noise under the same key - under the key
+    (seed mod 2^32, seed div 2^32), turned into four standard normals exactly as in device_noise."""
+    t = np.arange(t0, t0 + n, dtype=np.int64)[:, None]
+    g = np.arange(C // 4, dtype=np.int64)[None, :]
+    ctr = np.stack(np.broadcast_arrays(t & 0xFFFFFFFF, t >> 32, g, np.int64((1 << 31) + stream_id)), axis=-1).astype(np.uint32)
+    r = philox4x32_10(ctr, (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)).astype(np.float64)
+    u = (np.floor(r / 256.0) + 0.5) / 16777216.0
+    rad0, rad1 = np.sqrt(-2.0 * np.log(u[..., 0])), np.sqrt(-2.0 * np.log(u[..., 2]))
+    a0, a1 = 2.0 * np.pi * u[..., 1], 2.0 * np.pi * u[..., 3]
+    z = np.stack([rad0 * np.cos(a0), rad0 * np.sin(a0), rad1 * np.cos(a1), rad1 * np.sin(a1)], axis=-1)
+    return z.reshape(n, C)
+
+
 def attended_frames(cfg, lo: int, hi: int) -> np.ndarray:
     """Frames whose keys/values the chunk [lo, hi) attends (Sec. 3.1 "Two extents", Eq. 4): the
     prompt - the stream's first f_prompt frames, never evicted - then the last <= kv_cap frames of
@@ -548,11 +566,15 @@ def overlap_add(xi: np.ndarray, n_fft: int, hop: int, tail: Optional[np.ndarray]
     return acc[:hop * M] / ola_norm(n_fft, hop), acc[hop * M:]
 
 
-def vocoder_offline(cfg, blob, mel: np.ndarray) -> np.ndarray:
+def vocoder_offline(cfg, blob, mel: np.ndarray, stream_id: int = 0) -> np.ndarray:
+    """The vocoder tail over a whole sequence.  With cfg.excitation_std > 0 the output of the LAST transposed
+    conv (before that stage's residual blocks) receives excitation_std * excitation_noise."""
     W = parse_blob(cfg, blob)
     a = causal_conv_k3(np.asarray(mel, dtype=np.float64), W["pre.W"], 1) + W["pre.b"]
     for q, s in enumerate(cfg.up_strides):
         a = conv_transpose_causal(a, W[f"up{q}.Wt"], W[f"up{q}.bt"], s)
+        if q == len(cfg.up_strides) - 1 and getattr(cfg, "excitation_std", 0.0) > 0.0:
+            a = a + cfg.excitation_std * excitation_noise(cfg.excitation_seed, stream_id, 0, a.shape[0], a.shape[1])
         for r, d in enumerate(cfg.res_dilations):
             a = a + silu(causal_conv_k3(a, W[f"up{q}.res{r}.W"], d) + W[f"up{q}.res{r}.b"])
     z = causal_conv_k3(silu(a), W["head.W"], 1) + W["head.b"]
@@ -566,9 +588,11 @@ class VocoderStream:
     of each transposed conv, last 2d input frames of each residual block, last 2
     frames before the head, and the n_fft - hop overlap-add partial sums."""
 
-    def __init__(self, cfg, blob):
+    def __init__(self, cfg, blob, stream_id: int = 0):
         self.cfg = cfg
         self.W = parse_blob(cfg, blob)
+        self.stream_id = stream_id
+        self.t_exc = 0                 # frames emitted so far at the last stage's rate: the excitation's clock
         ch = cfg.up_channels
         self.c_pre = np.zeros((2, cfg.mel_dim))
         self.c_up = [np.zeros((1, ch[q])) for q in range(len(cfg.up_strides))]
@@ -586,6 +610,9 @@ class VocoderStream:
         for q, s in enumerate(cfg.up_strides):
             prev, self.c_up[q] = self.c_up[q], a[-1:].copy()
             a = conv_transpose_causal(a, W[f"up{q}.Wt"], W[f"up{q}.bt"], s, prev)
+            if q == len(cfg.up_strides) - 1 and getattr(cfg, "excitation_std", 0.0) > 0.0:
+                a = a + cfg.excitation_std * excitation_noise(cfg.excitation_seed, self.stream_id, self.t_exc, a.shape[0], a.shape[1])
+                self.t_exc += a.shape[0]
             for r, d in enumerate(cfg.res_dilations):
                 left = self.c_res[q][r]
                 self.c_res[q][r] = np.concatenate([left, a], axis=0)[-2 * d:]
@@ -610,7 +637,7 @@ class TokenToWavStream:
         fc, vc = cfg.flow_part(), cfg.vocoder_part()
         nf = _blob_floats(fc)
         self.flow = FlowStream(fc, blob[:nf], **kw)
-        self.voc = VocoderStream(vc, blob[nf:])
+        self.voc = VocoderStream(vc, blob[nf:], stream_id=kw.get("stream_id", 0))
 
     def decode_chunk(self, feats: np.ndarray) -> np.ndarray:
         mel = self.flow.decode_chunk(feats)
@@ -628,11 +655,11 @@ def _blob_floats(cfg) -> int:
     raise ValueError(cfg.pipeline)
 
 
-def token2wav_offline(cfg, blob, feats, boundaries) -> np.ndarray:
+def token2wav_offline(cfg, blob, feats, boundaries, stream_id: int = 0) -> np.ndarray:
     fc, vc = cfg.flow_part(), cfg.vocoder_part()
     nf = _blob_floats(fc)
-    mel = flow_offline(fc, blob[:nf], feats, boundaries)
-    return vocoder_offline(vc, blob[nf:], np.asarray(mel, dtype=np.float32))
+    mel = flow_offline(fc, blob[:nf], feats, boundaries, stream_id)
+    return vocoder_offline(vc, blob[nf:], np.asarray(mel, dtype=np.float32), stream_id)
 
 
 def make_stream(cfg, blob, **kw):
@@ -643,18 +670,18 @@ def make_stream(cfg, blob, **kw):
     if cfg.pipeline == "flow":
         return FlowStream(cfg, blob, **kw)
     if cfg.pipeline == "vocoder":
-        return VocoderStream(cfg, blob)
+        return VocoderStream(cfg, blob, stream_id=kw.get("stream_id", 0))
     raise ValueError(cfg.pipeline)
 
 
-def run_offline(cfg, blob, feats, boundaries) -> np.ndarray:
+def run_offline(cfg, blob, feats, boundaries, stream_id: int = 0) -> np.ndarray:
     if cfg.pipeline == "token2wav":
-        return token2wav_offline(cfg, blob, feats, boundaries)
+        return token2wav_offline(cfg, blob, feats, boundaries, stream_id)
     if cfg.pipeline == "conv":
         return conv_stack_offline(cfg, blob, feats)
     if cfg.pipeline == "flow":
-        return flow_offline(cfg, blob, feats, boundaries)
-    return vocoder_offline(cfg, blob, feats)
+        return flow_offline(cfg, blob, feats, boundaries, stream_id)
+    return vocoder_offline(cfg, blob, feats, stream_id)
 
 
 def run_stream(cfg, blob, feats, boundaries, **kw) -> np.ndarray:

@@ -585,7 +585,7 @@ def test_philox_known_answers_and_device_noise():
 
 # ---------------------------------------------------------------- vocoder tail as a whole / normal draw
 
-def torch_vocoder_reference(cfg, blob, mel):
+def torch_vocoder_reference(cfg, blob, mel, excitation=None):
     """Independent library formulation (float64 torch ops) of the whole vocoder tail: conv1d with
     left padding for the entry conv, the residual blocks and the head, conv_transpose1d with the
     trailing `stride` samples dropped, F.silu, torch.polar + torch.fft.irfft for the frame
@@ -605,6 +605,8 @@ def torch_vocoder_reference(cfg, blob, mel):
     for q, s in enumerate(cfg.up_strides):
         wt = Wd[f"up{q}.Wt"].permute(1, 2, 0).contiguous()   # [C_in, C_out, k]
         a = F.conv_transpose1d(a[None], wt, Wd[f"up{q}.bt"], stride=s)[0][:, :a.shape[1] * s]
+        if excitation is not None and q == len(cfg.up_strides) - 1:
+            a = a + torch.from_numpy(excitation).T          # [frames at the last stage's rate, C] -> [C, frames]
         for r, d in enumerate(cfg.res_dilations):
             a = a + F.silu(conv3(a, f"up{q}.res{r}.W", f"up{q}.res{r}.b", d))
     z = conv3(F.silu(a), "head.W", "head.b", 1).T            # [M, n_fft + 2]
@@ -713,3 +715,45 @@ def test_device_noise_single_values_by_hand():
     w = orc.philox4x32_10(np.array([7, 1, 0, 1], dtype=np.uint32), (3, 0))
     assert math.isclose(big[0], math.sqrt(-2 * math.log(((int(w[0]) >> 8) + 0.5) / 2 ** 24))
                         * math.cos(2 * math.pi * ((int(w[1]) >> 8) + 0.5) / 2 ** 24), abs_tol=1e-12)
+
+
+def _normals_by_hand(words):
+    u = [((int(r) >> 8) + 0.5) * 2.0 ** -24 for r in words]
+    return [math.sqrt(-2.0 * math.log(u[0])) * math.cos(2.0 * math.pi * u[1]), math.sqrt(-2.0 * math.log(u[0])) * math.sin(2.0 * math.pi * u[1]),
+            math.sqrt(-2.0 * math.log(u[2])) * math.cos(2.0 * math.pi * u[3]), math.sqrt(-2.0 * math.log(u[2])) * math.sin(2.0 * math.pi * u[3])]
+
+
+def test_vocoder_excitation_pins():
+    """The vocoder's random excitation (device randomness admitted through the call clock): single values by hand
+    from the pinned generator words, keying, where it enters the chain, and chunking invariance."""
+    seed, sid, C = 0xABCDEF0123, 3, 8
+    z = orc.excitation_noise(seed, sid, 1000, 3, C)
+    for i, t in enumerate((1000, 1001, 1002)):
+        for g in range(C // 4):
+            words = orc.philox4x32_10(np.array([t, 0, g, (1 << 31) + sid], dtype=np.uint32), (seed & 0xFFFFFFFF, seed >> 32))
+            assert np.allclose(z[i, 4 * g:4 * g + 4], _normals_by_hand(words), rtol=0, atol=1e-12)
+    # its draws never coincide with the flow decoder's noise of the same key, stream, frame and channel group
+    assert not np.allclose(orc.excitation_noise(7, 2, 0, 4, 8), orc.device_noise(7, 2, 0, 4, 8))
+    big = orc.excitation_noise(9, 0, 1 << 20, 20000, 8)
+    assert abs(big.mean()) < 0.01 and abs(big.std() - 1.0) < 0.01 and abs(np.mean(big ** 4) - 3.0) < 0.1
+    # where it enters: after the last transposed conv, before that stage's residual blocks (independent torch chain)
+    cfg = wl.tiny_vocoder(bias_std=0.3, excitation_std=0.25, excitation_seed=seed)
+    w = wl.make_workload(cfg, boundaries=[[0, 5, 10, 15, 20]])
+    mel = w.streams[0].feats
+    rate = int(np.prod(cfg.up_strides))
+    exc = cfg.excitation_std * np.array([[v for g in range(cfg.up_channels[-1] // 4)
+                                          for v in _normals_by_hand(orc.philox4x32_10(np.array([t, 0, g, (1 << 31) + sid], dtype=np.uint32),
+                                                                                      (seed & 0xFFFFFFFF, seed >> 32)))]
+                                         for t in range(20 * rate)])
+    ref = torch_vocoder_reference(cfg, w.weights, mel, excitation=exc)
+    mine = orc.vocoder_offline(cfg, w.weights, mel, stream_id=sid).astype(np.float64)
+    rms = np.sqrt((ref ** 2).mean())
+    assert np.abs(mine - ref).max() <= 2e-7 * max(rms, np.abs(ref).max())
+    quiet = orc.vocoder_offline(cfg.replace(excitation_std=0.0), w.weights, mel).astype(np.float64)
+    assert np.abs(mine - quiet).max() > 1e-2 * rms                     # the source is audible
+    assert np.array_equal(quiet, orc.vocoder_offline(wl.tiny_vocoder(bias_std=0.3), w.weights, mel))
+    # chunking cannot change the draw: the generator's offset is the stream's clock at the last stage's rate
+    for bnd in ([0, 1, 2, 7, 8, 13, 18, 20], [0, 5, 10, 15, 20]):
+        st = orc.run_stream(cfg, w.weights, mel, bnd, stream_id=sid)
+        assert np.abs(st - mine).max() <= 1e-6 * rms
+    assert np.abs(orc.run_stream(cfg, w.weights, mel, [0, 5, 10, 15, 20], stream_id=sid + 1) - mine).max() > 1e-3 * rms
