@@ -108,11 +108,12 @@ class DCConfig:
     # configurations of their own (weights: the flow blob, then the vocoder blob)
     def flow_part(self) -> "DCConfig":
         assert self.pipeline == PIPE_TOKEN2WAV
-        return self.replace(name=self.name + ".flow", pipeline=PIPE_FLOW, precision="bf16")
+        return self.replace(name=self.name + ".flow", pipeline=PIPE_FLOW, precision="bf16", excitation_std=0.0, excitation_seed=0)
 
     def vocoder_part(self) -> "DCConfig":
         assert self.pipeline == PIPE_TOKEN2WAV
-        return self.replace(name=self.name + ".vocoder", pipeline=PIPE_VOCODER, precision="f32")
+        return self.replace(name=self.name + ".vocoder", pipeline=PIPE_VOCODER, precision="f32", noise_seed=0, cfg_scale=0.0,
+                            f_prompt=0, f_lookahead=0)
 
 
 def blob_layout(cfg: DCConfig) -> List[Tuple[str, Tuple[int, ...], int]]:

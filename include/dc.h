@@ -162,6 +162,17 @@ typedef struct dc_config {
                                   * on, so that no decode call allocates; 0 = wavefront calls on this model are
                                   * refused.  Must be 0 for the other pipelines (their wavefront needs no buffer). */
   uint32_t options;              /* DC_OPT_* bits, 0 for normal use                           */
+  float    excitation_std;       /* vocoder tail (and token2wav): > 0 adds a random excitation drawn on the device - the
+                                  * vocoder's source signal, the paper's own instance of device randomness (Section
+                                  * 3.1 "device random stream"; Section 3.3, effect classification: admitted because the
+                                  * generator's offset is a function of the call clock).  The output of the LAST
+                                  * transposed conv, before that stage's residual blocks, receives
+                                  * excitation_std * N(0,1): the draw of (frame t at that layer's output rate, counted
+                                  * from the stream start, channels 4g..4g+3) is Philox4x32-10 at counter
+                                  * (t mod 2^32, t div 2^32, g, 2^31 + stream index) under the key below, four
+                                  * normals per draw as for noise_seed.  Chunking, graph replay and snapshots cannot
+                                  * change the draw.  0: no excitation (the five benchmark configurations).       */
+  uint32_t excitation_seed_lo, excitation_seed_hi;   /* its key; non-zero when excitation_std > 0                */
 } dc_config;
 
 /* Number of floats of the canonical weight blob for this configuration, 0 if the

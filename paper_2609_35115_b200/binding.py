@@ -35,7 +35,8 @@ class dc_config(C.Structure):
                 ("res_dilations", C.c_int32 * DC_MAX_RES), ("n_fft", C.c_int32), ("hop", C.c_int32),
                 ("rms_eps", C.c_float), ("logmag_clamp", C.c_float), ("max_batch", C.c_int32),
                 ("f_prompt", C.c_int32), ("f_lookahead", C.c_int32), ("noise_seed_lo", C.c_uint32), ("noise_seed_hi", C.c_uint32),
-                ("cfg_scale", C.c_float), ("max_wave_frames", C.c_int32), ("options", C.c_uint32)]
+                ("cfg_scale", C.c_float), ("max_wave_frames", C.c_int32), ("options", C.c_uint32),
+                ("excitation_std", C.c_float), ("excitation_seed_lo", C.c_uint32), ("excitation_seed_hi", C.c_uint32)]
 
 
 class DCError(RuntimeError):
@@ -121,6 +122,9 @@ def make_config(cfg, max_batch: int = 1, max_wave_frames: int = 0, options: int 
     c.max_batch = max_batch
     c.max_wave_frames = max_wave_frames
     c.options = options
+    c.excitation_std = float(getattr(cfg, "excitation_std", 0.0))
+    eseed = int(getattr(cfg, "excitation_seed", 0))
+    c.excitation_seed_lo, c.excitation_seed_hi = eseed & 0xFFFFFFFF, (eseed >> 32) & 0xFFFFFFFF
     c.cfg_scale = float(getattr(cfg, "cfg_scale", 0.0))
     c.f_prompt = int(getattr(cfg, "f_prompt", 0))
     c.f_lookahead = int(getattr(cfg, "f_lookahead", 0))

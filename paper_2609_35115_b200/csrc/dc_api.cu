@@ -54,6 +54,7 @@ struct F32Layer {
   int    residual_silu, post_silu;
   size_t w_off, b_off;  // float offsets in the blob
   int    ring_cap;    // rows of its input ring
+  int    excite;      // the random excitation is added to this layer's output
 };
 
 }  // namespace dc
@@ -82,6 +83,7 @@ struct dc_model {
   cudaEvent_t               tail_fork = nullptr;
   std::atomic<uint64_t> counters[8];
   std::atomic<int> open_streams{0};
+  int    streams_opened = 0;   // so far: the next fp32 stream's random-stream index (streams of a model are opened one at a time)
   std::mutex mu;
   dc::Profiler prof;
   std::vector<dc_stream*> all_streams;   // host structs live until dc_destroy, so a closed handle stays detectable
@@ -101,6 +103,7 @@ struct dc_stream {
   bool      closed = false, poisoned = false;
   long long frames_total = 0;
   long long chunks = 0;
+  int       rng_id = 0;            // fp32 pipelines: which device random stream the session draws from (vocoder excitation)
   std::vector<DevBuf> f32_rings;   // input ring of each fp32 layer
   float*    tails = nullptr;       // [2][12] overlap-add tails (ping-pong)
   dc::F32Call* d_call = nullptr;   // fp32 pipelines: per-call record read by this stream's captured graph (streams of one
@@ -130,6 +133,10 @@ static dc_config sub_config(const dc_config& c, int pipeline) {
   s.pipeline = pipeline;
   s.precision = pipeline == DC_PIPE_FLOW ? DC_BF16 : DC_F32;
   s.max_wave_frames = 0;   // the mel buffer of a wavefront call belongs to the composite
+  if (pipeline == DC_PIPE_FLOW) {
+    s.excitation_std = 0.f;
+    s.excitation_seed_lo = s.excitation_seed_hi = 0;
+  }
   if (pipeline != DC_PIPE_FLOW) {
     s.cfg_scale = 0.f;
     s.f_prompt = 0;
@@ -155,6 +162,9 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (c->options & ~(uint32_t)(DC_OPT_NO_GRAPH | DC_OPT_NO_PDL | DC_OPT_NO_ZEROCOPY | DC_OPT_SERIAL_TAILS | DC_OPT_ROUNDED_NORM | DC_OPT_SKIP_CONV_GEMM |
                                DC_OPT_SKIP_ATTENTION | DC_OPT_EMPTY_KERNELS))
     BAD("unknown option bit");
+  if (!(c->excitation_std >= 0.f && c->excitation_std <= 1e6f)) BAD("excitation_std out of range");
+  if (c->excitation_std > 0.f && c->pipeline != DC_PIPE_VOCODER && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("excitation_std belongs to the vocoder tail");
+  if (c->excitation_std > 0.f && (c->excitation_seed_lo | c->excitation_seed_hi) == 0) BAD("excitation_std > 0 needs a non-zero excitation seed");
   if (c->max_wave_frames < 0 || c->max_wave_frames > (1 << 24)) BAD("max_wave_frames out of range");
   if (c->max_wave_frames != 0 && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("max_wave_frames belongs to the token2wav pipeline");
   if (c->pipeline == DC_PIPE_TOKEN2WAV) {
@@ -255,6 +265,7 @@ static void build_f32_layers(dc_model* m) {
     for (int q = 0; q < c.n_up; ++q) {
       const int ci = c.up_channels[q], co = c.up_channels[q + 1], s = c.up_strides[q];
       add(1, ci, co, 1, s, rate, 1, 0, (size_t)2 * s * ci * co);
+      if (q == c.n_up - 1 && c.excitation_std > 0.f) m->layers.back().excite = 1;
       rate *= s;
       for (int r = 0; r < c.n_res; ++r)
         add(0, co, co, c.res_dilations[r], 1, rate, 2 * c.res_dilations[r], 1, (size_t)3 * co * co);
@@ -446,6 +457,7 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
   } else if (m->flow) {
     st = dc::flow_state_open(m->flow, &s->flow);
   } else {
+    s->rng_id = m->streams_opened++;
     for (const F32Layer& L : m->layers) {
       DevBuf b{nullptr, (size_t)L.ring_cap * L.C_in * sizeof(float)};
       e = cudaMalloc(&b.p, b.bytes);
@@ -598,6 +610,8 @@ extern "C" dc_status dc_stream_snapshot(dc_stream* s, dc_snapshot** out, void* c
     if (s->flow) {
       sn->flow_frames = dc::flow_state_frames(s->flow);
       sn->rng_id = dc::flow_state_rng_id(s->flow);
+    } else {
+      sn->rng_id = s->rng_id;
     }
     const std::vector<DevBuf> bufs = carry_buffers(s);
     for (const DevBuf& b : bufs) sn->bytes += b.bytes;
@@ -643,6 +657,8 @@ extern "C" dc_status dc_stream_restore(dc_stream* s, const dc_snapshot* sn, void
     if (s->flow) {
       dc::flow_state_set_frames(s->flow, sn->flow_frames);
       dc::flow_state_set_rng_id(s->flow, sn->rng_id);   // the session keeps its random stream wherever it lives
+    } else {
+      s->rng_id = sn->rng_id;
     }
   }
   s->frames_total = sn->frames_total;
@@ -701,6 +717,10 @@ static void enqueue_f32(dc_stream* s, bool use_call, const float* feats, int T, 
       }
       p.W = m->d_w + L.w_off; p.bias = m->d_w + L.b_off; p.C_out = L.C_out;
       p.residual_silu = L.residual_silu; p.post_silu = L.post_silu;
+      if (L.excite) {
+        p.exc_std = m->cfg.excitation_std; p.exc_seed_lo = m->cfg.excitation_seed_lo; p.exc_seed_hi = m->cfg.excitation_seed_hi;
+        p.exc_rng_id = s->rng_id;
+      }
       if (l + 1 < nL) {
         p.out_ring = (float*)s->f32_rings[l + 1].p; p.out_mask = m->layers[l + 1].ring_cap - 1;
       } else if (!use_call) {
@@ -757,7 +777,7 @@ static void build_f32_graph(dc_stream* s) {
 static dc_status decode_f32(dc_stream* s, const float* feats, int T, float* out, cudaStream_t cs, int* launches) {
   dc_model* m = s->model;
   if (s->g_exec != nullptr && !m->prof.on) {
-    dc::F32Call v{s->frames_total, T, (int)(s->chunks & 1), feats, out};
+    dc::F32Call v{s->frames_total, T, (int)(s->chunks & 1), feats, out, s->rng_id};
     dc::F32Call* dst = s->d_call;
     void* args[2] = {&v, &dst};
     cudaKernelNodeParams kp{};

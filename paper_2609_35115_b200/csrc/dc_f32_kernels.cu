@@ -4,6 +4,7 @@
 // out single-pass TF32, so these run on the FP32 pipe.
 #include "dc_internal.h"
 #include "dc_ptx.cuh"
+#include "dc_rng.cuh"
 
 #include <math.h>
 #include <stdio.h>
@@ -61,8 +62,10 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
   long long pos_in = p.pos_in, pos_out = p.pos_out;
   const float* in_direct = p.in_direct;
   float* out_direct = p.out_direct;
+  int exc_rng_id = p.exc_rng_id;
   if (p.call != nullptr) {
     const F32Call c = *p.call;
+    exc_rng_id = c.rng_id;
     T_in = c.T * p.rate_in;
     pos_in = c.frames * p.rate_in;
     pos_out = pos_in * p.n_phase;
@@ -215,6 +218,14 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
       }
       if (p.post_silu) v = make_float4(silu_f(v.x), silu_f(v.y), silu_f(v.z), silu_f(v.w));
       const long long t_out = (long long)p.n_phase * t_in + phase;
+      if (p.exc_std != 0.f) {   // the stream's clock at this layer's output rate is the generator's offset
+        uint32_t w[4];
+        float z[4];
+        philox4x32_10((uint32_t)(unsigned long long)t_out, (uint32_t)((unsigned long long)t_out >> 32), (uint32_t)(n >> 2),
+                      0x80000000u + (uint32_t)exc_rng_id, p.exc_seed_lo, p.exc_seed_hi, w);
+        normals4(w, z);
+        v.x = fmaf(p.exc_std, z[0], v.x); v.y = fmaf(p.exc_std, z[1], v.y); v.z = fmaf(p.exc_std, z[2], v.z); v.w = fmaf(p.exc_std, z[3], v.w);
+      }
       float* dst = (out_direct != nullptr)
                        ? out_direct + (t_out - pos_out) * C_out + n
                        : p.out_ring + (long long)((int)(t_out & (long long)p.out_mask)) * C_out + n;

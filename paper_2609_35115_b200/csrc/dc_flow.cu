@@ -26,6 +26,7 @@
 
 #include "dc_internal.h"
 #include "dc_ptx.cuh"
+#include "dc_rng.cuh"
 
 namespace dc {
 
@@ -539,20 +540,6 @@ __global__ void set_slots_kernel(const SlotSet set, SlotInfo* dst) {
   if (i < set.count) dst[set.first + i] = set.s[i];
 }
 
-// Philox4x32-10 (Salmon et al. 2011): ten rounds of two 32 x 32 -> 64 multiplications and a key bump.
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1, uint32_t* out) {
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
-    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
-  }
-  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
-}
-
 // feats [T][2 mel] (or [T][mel] when the noise is drawn here) -> Euler state x_0 (fp32) and the bf16
 // input-projection operand [x_0 | mu].  Device noise: the draw of (frame t, channels 4g..4g+3) is Philox at
 // counter (t, g, stream) under the model's seed - the offset is the stream's frame clock, so a replayed graph
@@ -572,13 +559,7 @@ __global__ void flow_prep_kernel(const SlotInfo* slots, int mel, float* xstate, 
       const unsigned long long t = (unsigned long long)(si.frame0 + f);
       uint32_t w[4];
       philox4x32_10((uint32_t)t, (uint32_t)(t >> 32), (uint32_t)g, (uint32_t)si.rng_id, seed_lo, seed_hi, w);
-      const float u0 = ((float)(w[0] >> 8) + 0.5f) * (1.0f / 16777216.0f), u1 = ((float)(w[1] >> 8) + 0.5f) * (1.0f / 16777216.0f);
-      const float u2 = ((float)(w[2] >> 8) + 0.5f) * (1.0f / 16777216.0f), u3 = ((float)(w[3] >> 8) + 0.5f) * (1.0f / 16777216.0f);
-      const float ra = sqrtf(-2.0f * logf(u0)), rb = sqrtf(-2.0f * logf(u2));
-      float sa, ca, sb, cb;
-      sincosf(6.283185307179586f * u1, &sa, &ca);
-      sincosf(6.283185307179586f * u3, &sb, &cb);
-      x0[0] = ra * ca; x0[1] = ra * sa; x0[2] = rb * cb; x0[3] = rb * sb;
+      normals4(w, x0);
     } else {
       const float4 v = *reinterpret_cast<const float4*>(si.feats + (long long)f * fw + mel + 4 * g);
       x0[0] = v.x; x0[1] = v.y; x0[2] = v.z; x0[3] = v.w;

@@ -26,6 +26,7 @@ struct F32Call {
   int          parity;     // which overlap-add tail buffer holds the previous call's tail
   const float* feats;      // caller's chunk
   float*       out;        // caller's output
+  int          rng_id;     // the stream's device random stream (vocoder excitation)
 };
 
 struct TapConvF32 {
@@ -54,6 +55,11 @@ struct TapConvF32 {
   long long    pos_out;
   float*       save_ring;     // if set: copy the last save_rows rows of in_direct into the input ring
   int          save_rows;
+  // Random excitation added to this layer's output (vocoder: the last transposed conv): exc_std * N(0,1), the draw of
+  // (output frame t, channels 4g..4g+3) being Philox4x32-10 at counter (t lo, t hi, g, 2^31 + rng id) under the seed.
+  float        exc_std;       // 0: none
+  uint32_t     exc_seed_lo, exc_seed_hi;
+  int          exc_rng_id;    // by value, or from *call
 };
 
 // T_grid: frames the grid is sized for (p.T_in, or the largest T_in when p.call is set).

@@ -206,3 +206,59 @@ def test_streams_of_one_model_on_different_cuda_streams(dc):
         assert np.array_equal(got, ref[i]), f"stream {i}"
         sts[i].close()
     m.destroy()
+
+
+# ---- the vocoder's random excitation: drawn on the device, keyed by the stream and its output-frame clock ----
+
+EXC = dict(excitation_std=0.25, excitation_seed=0xABCDEF0123)
+
+
+def test_vocoder_excitation_matches_oracle_for_any_chunking_and_stream(dc):
+    gu = _util()
+    cfg = wl.tiny_vocoder(bias_std=0.3, **EXC)
+    bnd = [0, 1, 2, 7, 8, 13, 18, 20]
+    w = wl.make_workload(cfg, boundaries=[bnd])
+    s = w.streams[0]
+    m = dc.Model(cfg, w.weights)
+    quiet = orc.vocoder_offline(cfg.replace(excitation_std=0.0), w.weights, s.feats)
+    outs = []
+    for sid, b in enumerate((bnd, [0, 5, 10, 15, 20], bnd)):       # the model's streams 0, 1, 2 draw different sequences
+        ref = orc.vocoder_offline(cfg, w.weights, s.feats, stream_id=sid)
+        st = m.open_stream()
+        got = gu.run_gpu_stream(m, s.feats, b, stream=st)
+        assert gu.rel_err(got, ref) <= TOL_F32, f"stream {sid}"
+        assert gu.rel_err(got, quiet) > 1e-2                        # the source is really there
+        outs.append(got)
+        if sid == 2:                                                # a reset restarts the stream's clock: same draw again
+            st.reset()
+            assert np.array_equal(gu.run_gpu_stream(m, s.feats, b, stream=st), got)
+        st.close()
+    assert not np.array_equal(outs[0], outs[2])
+    m.destroy()
+    # direct launches draw what the captured chunk step draws
+    m2 = dc.Model(cfg, w.weights, options=dc.OPT_NO_GRAPH)
+    assert np.array_equal(gu.run_gpu_stream(m2, s.feats, bnd), outs[0])
+    m2.destroy()
+
+
+def test_vocoder_excitation_cfg4_geometry(dc):
+    """cfg4's network with the excitation on: 6 chunks of 50 frames (6,000 excitation frames of 64 channels each)."""
+    gu = _util()
+    cfg = wl.CONFIGS["cfg4"].replace(name="cfg4_excited", n_chunks=6, **EXC)
+    w = wl.make_workload(cfg)
+    s = w.streams[0]
+    ref = orc.run_stream(cfg, w.weights, s.feats, s.boundaries)
+    m = dc.Model(cfg, w.weights)
+    got = gu.run_gpu_stream(m, s.feats, s.boundaries)
+    m.destroy()
+    assert gu.rel_err(got, ref) <= TOL_F32
+
+
+def test_excitation_needs_a_seed_and_a_vocoder(dc):
+    cfg = wl.tiny_vocoder(excitation_std=0.2)                       # no seed
+    w = wl.make_workload(cfg)
+    with pytest.raises(dc.DCError):
+        dc.Model(cfg, w.weights)
+    c1 = wl.CONFIGS["cfg1"].replace(excitation_std=0.2, excitation_seed=3)
+    with pytest.raises(dc.DCError):
+        dc.Model(c1, wl.make_workload(c1).weights)

@@ -27,6 +27,7 @@ def _chunks(st, x, bounds, lo, hi):
                                   lambda: wl.tiny_flow(n_chunks=8, noise_seed=5),     # the session keeps its random stream
 
                                   lambda: wl.tiny_vocoder(n_chunks=8),
+                                  lambda: wl.tiny_vocoder(n_chunks=8, excitation_std=0.3, excitation_seed=77),   # ... and its excitation clock
                                   lambda: wl.CONFIGS["cfg1"],
                                   lambda: wl.tiny_token2wav(n_chunks=8)])
 def test_rewind_and_move(dc, make):
