@@ -71,7 +71,7 @@ enum {
   DC_OPT_NO_GRAPH     = 1,        /* decode calls issue their kernels one by one instead of one captured graph  */
   DC_OPT_NO_PDL       = 2,        /* no programmatic dependent launch between the kernels of a step             */
   DC_OPT_NO_ZEROCOPY  = 4,        /* the *_host calls always stage, also for page-locked caller buffers         */
-  DC_OPT_SERIAL_TAILS = 8,        /* token2wav dc_decode_batch: the vocoder tails one after another             */
+  DC_OPT_SERIAL_TAILS = 8,        /* token2wav dc_decode_batch: the vocoder tails stream by stream, not batched */
   /* Flow decoder: the RMS-normalised activations are written as a tensor of their own, rounded to bf16, and
    * the projections read it - the storage-point reading of "bf16 activations" taken literally - instead of
    * the default, which folds the norm into the projection as a scale of its fp32 accumulator rows and so
@@ -104,9 +104,8 @@ enum {
  *                     decoder, then vocoder and inverse STFT) in one call - a chunk of
  *                     [conditioning | noise] frames in, PCM out; the mel frames in between stay in a
  *                     device buffer of the stream (bf16 flow decoder, fp32 vocoder tail).  Weights:
- *                     the flow blob followed by the vocoder blob.  dc_decode_batch serves it too (the
- *                     flow decoder batched over the streams, the vocoder tail stream by stream);
- *                     dc_decode_batch_host does not.
+ *                     the flow blob followed by the vocoder blob.  dc_decode_batch serves it too (max_batch
+ *                     <= 64); dc_decode_batch_host does not.
  * The flow decoder runs n_conv / n_attn conv blocks, then one attention layer,
  * repeated n_attn times (n_attn = 0: conv blocks only). */
 typedef struct dc_config {
@@ -235,10 +234,11 @@ dc_status dc_decode_chunk(dc_stream* stream, const float* feats_dev, int n_frame
  * CUDA graph launch: the chunk step is captured once per batch size - for 1 and max_batch streams at
  * dc_create, for any other n at the first call that carries n streams (that one call also pays the
  * capture; the graphs form the finite catalog of Section 3.3, Eq. 5) - and only the slot table
- * passed by value changes from call to call.  Flow and token2wav
- * pipelines.  The token2wav composite batches the flow decoder and then runs the streams' vocoder
- * tails side by side on CUDA streams owned by the model, forked behind the flow decoder on
- * cuda_stream and joined back into it before the call returns. */
+ * passed by value changes from call to call.  All four pipelines: the fp32 pipelines run every layer
+ * once for the whole batch (a slot of the batch is a plane of the layer's grid, with the tiles and the
+ * reduction split of the single-stream step; at most 64 streams), and the token2wav composite batches
+ * the flow decoder and then the vocoder tails in the same way - a serving round of n sessions is two
+ * graph launches. */
 dc_status dc_decode_batch(dc_model* model, int n, dc_stream* const* streams,
                           const float* const* feats_dev, const int* n_frames,
                           float* const* out_dev, void* cuda_stream);

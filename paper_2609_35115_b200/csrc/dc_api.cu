@@ -77,10 +77,13 @@ struct dc_model {
   // DC_PIPE_TOKEN2WAV: the flow decoder and the vocoder tail as models of their own; this one only chains them
   dc_model* sub_flow = nullptr;
   dc_model* sub_voc = nullptr;
-  // ... and CUDA streams of its own on which dc_decode_batch runs the streams' vocoder tails side by side
-  std::vector<cudaStream_t> tail_streams;
-  std::vector<cudaEvent_t>  tail_done;
-  cudaEvent_t               tail_fork = nullptr;
+  // fp32 pipelines: dc_decode_batch runs every layer ONCE for all the streams of the batch (slot = grid plane); the slot
+  // records live here and are rewritten per call by the first node of the captured batch step
+  dc::F32Batch*   d_batch = nullptr;
+  cudaGraph_t     gb_graph = nullptr;
+  cudaGraphExec_t gb_exec = nullptr;
+  cudaGraphNode_t gb_set_node = nullptr;
+  int             gb_launches = 0;
   std::atomic<uint64_t> counters[8];
   std::atomic<int> open_streams{0};
   int    streams_opened = 0;   // so far: the next fp32 stream's random-stream index (streams of a model are opened one at a time)
@@ -89,13 +92,13 @@ struct dc_model {
   std::vector<dc_stream*> all_streams;   // host structs live until dc_destroy, so a closed handle stays detectable
 };
 
-static void free_tail_streams(dc_model* m) {
-  for (cudaStream_t t : m->tail_streams) cudaStreamDestroy(t);
-  for (cudaEvent_t e : m->tail_done) cudaEventDestroy(e);
-  if (m->tail_fork) cudaEventDestroy(m->tail_fork);
-  m->tail_streams.clear();
-  m->tail_done.clear();
-  m->tail_fork = nullptr;
+static void free_batch_graph(dc_model* m) {
+  if (m->gb_exec) cudaGraphExecDestroy(m->gb_exec);
+  if (m->gb_graph) cudaGraphDestroy(m->gb_graph);
+  if (m->d_batch) cudaFree(m->d_batch);
+  m->gb_exec = nullptr;
+  m->gb_graph = nullptr;
+  m->d_batch = nullptr;
 }
 
 struct dc_stream {
@@ -106,6 +109,7 @@ struct dc_stream {
   int       rng_id = 0;            // fp32 pipelines: which device random stream the session draws from (vocoder excitation)
   std::vector<DevBuf> f32_rings;   // input ring of each fp32 layer
   float*    tails = nullptr;       // [2][12] overlap-add tails (ping-pong)
+  dc::F32StreamPtrs* d_ptrs = nullptr;   // fp32 pipelines: the addresses of this stream's rings and tails, for batched launches
   dc::F32Call* d_call = nullptr;   // fp32 pipelines: per-call record read by this stream's captured graph (streams of one
                                    // model may decode at the same time on different CUDA streams)
   dc::FlowState* flow = nullptr;
@@ -172,6 +176,7 @@ static bool config_ok(const dc_config* c, const char** why) {
     const dc_config f = sub_config(*c, DC_PIPE_FLOW), v = sub_config(*c, DC_PIPE_VOCODER);
     return config_ok(&f, why) && config_ok(&v, why);
   }
+  if ((c->pipeline == DC_PIPE_CONV || c->pipeline == DC_PIPE_VOCODER) && c->max_batch > dc::F32_MAX_BATCH) BAD("fp32 pipelines batch at most 64 streams");
   if (c->pipeline == DC_PIPE_CONV) {
     if (c->precision != DC_F32) BAD("conv pipeline is fp32");
     if (c->hidden < 4 || c->hidden % 4) BAD("hidden must be a multiple of 4");
@@ -278,6 +283,7 @@ static void build_f32_layers(dc_model* m) {
 }
 
 static void build_f32_graph(dc_stream* s);
+static void build_f32_batch_graph(dc_model* m);
 
 // ---------------------------------------------------------------------------------------------
 // lifetime
@@ -319,23 +325,6 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     if (st == DC_OK) {
       m->in_dim = m->sub_flow->in_dim;
       m->out_per_frame = m->sub_voc->out_per_frame;
-      // a vocoder chunk step fills a fraction of the GPU (12 short kernels on small grids): up to 8 of a batch's
-      // tails run at the same time
-      const int want = (cfg->options & DC_OPT_SERIAL_TAILS) ? 1 : 8;
-      const int n_side = cfg->max_batch < want ? cfg->max_batch : want;
-      bool ok = n_side < 2 || cudaEventCreateWithFlags(&m->tail_fork, cudaEventDisableTiming) == cudaSuccess;
-      for (int i = 0; ok && n_side >= 2 && i < n_side; ++i) {
-        cudaStream_t cs2 = nullptr;
-        cudaEvent_t ev = nullptr;
-        ok = cudaStreamCreateWithFlags(&cs2, cudaStreamNonBlocking) == cudaSuccess;
-        if (ok) m->tail_streams.push_back(cs2);
-        ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
-        if (ev) m->tail_done.push_back(ev);
-      }
-      if (!ok) {
-        dc::set_error("stream / event creation failed");
-        st = DC_ERR_CUDA;
-      }
     }
   } else if (cfg->pipeline == DC_PIPE_FLOW) {
     st = dc::flow_model_create(*cfg, w, &m->flow);
@@ -360,15 +349,20 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     cudaError_t e = cudaMalloc(&m->d_w, n_floats * sizeof(float));
     if (e == cudaSuccess) e = cudaMemcpy(m->d_w, w, n_floats * sizeof(float), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = dc::prepare_f32_constants();
+    if (e == cudaSuccess && cfg->max_batch > 1) {
+      e = cudaMalloc(&m->d_batch, sizeof(dc::F32Batch));
+      if (e == cudaSuccess) e = cudaMemset(m->d_batch, 0, sizeof(dc::F32Batch));
+    }
     if (e != cudaSuccess) {
       dc::set_error("weight upload failed: %s", cudaGetErrorString(e));
       st = e == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;
     }
+    if (st == DC_OK && m->d_batch) build_f32_batch_graph(m);
   }
   if (st != DC_OK) {
     if (m->sub_flow) dc_destroy(m->sub_flow);
     if (m->sub_voc) dc_destroy(m->sub_voc);
-    free_tail_streams(m);
+    free_batch_graph(m);
     if (m->d_w) cudaFree(m->d_w);
     if (m->flow) dc::flow_model_destroy(m->flow);
     if (m->h_in) cudaFreeHost(m->h_in);
@@ -391,7 +385,7 @@ extern "C" dc_status dc_destroy(dc_model* m) {
   }
   if (m->sub_flow) dc_destroy(m->sub_flow);   // their streams were closed with ours
   if (m->sub_voc) dc_destroy(m->sub_voc);
-  free_tail_streams(m);
+  free_batch_graph(m);
   if (m->flow) dc::flow_model_destroy(m->flow);
   if (m->d_w) cudaFree(m->d_w);
   if (m->h_in) cudaFreeHost(m->h_in);
@@ -415,6 +409,8 @@ static void free_stream_buffers(dc_stream* s) {
   if (s->tails) cudaFree(s->tails);
   if (s->d_call) cudaFree(s->d_call);
   s->d_call = nullptr;
+  if (s->d_ptrs) cudaFree(s->d_ptrs);
+  s->d_ptrs = nullptr;
   if (s->flow) dc::flow_state_close(s->flow);
   if (s->sub_flow) dc_stream_close(s->sub_flow);
   if (s->sub_voc) dc_stream_close(s->sub_voc);
@@ -470,6 +466,13 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
     if (e == cudaSuccess && m->cfg.pipeline == DC_PIPE_VOCODER) {
       e = cudaMalloc(&s->tails, 2 * 12 * sizeof(float));
       if (e == cudaSuccess) e = cudaMemset(s->tails, 0, 2 * 12 * sizeof(float));
+    }
+    if (e == cudaSuccess) {
+      dc::F32StreamPtrs hp{};
+      for (size_t l = 0; l < s->f32_rings.size() && l < (size_t)dc::F32_MAX_LAYERS; ++l) hp.ring[l] = (float*)s->f32_rings[l].p;
+      hp.tails = s->tails;
+      e = cudaMalloc(&s->d_ptrs, sizeof(hp));
+      if (e == cudaSuccess) e = cudaMemcpy(s->d_ptrs, &hp, sizeof(hp), cudaMemcpyHostToDevice);
     }
   }
   if (e == cudaSuccess && st == DC_OK) {
@@ -774,6 +777,115 @@ static void build_f32_graph(dc_stream* s) {
   cudaStreamDestroy(cap);
 }
 
+// The layers of one fp32 chunk step for up to max_batch streams at once: every layer is ONE launch whose grid planes
+// are the slots of the batch record (stream, frames, pointers); per slot the tiles, the reduction split and the
+// arithmetic are those of the single-stream step, so a stream's bytes do not depend on who shares its launch.
+static void enqueue_f32_batch(dc_model* m, cudaStream_t cs, int* launches) {
+  const int nL = (int)m->layers.size(), nb = m->cfg.max_batch;
+  for (int l = 0; l < nL; ++l) {
+    const F32Layer& L = m->layers[l];
+    const int Tgrid = m->cfg.f_chunk * L.rate_in;
+    if (L.kind == 2) {
+      dc::HeadIstftF32 h{};
+      h.batch = m->d_batch; h.layer = l; h.rate_in = L.rate_in;
+      h.in_mask = L.ring_cap - 1; h.C = L.C_in;
+      h.W = m->d_w + L.w_off; h.bias = m->d_w + L.b_off; h.clamp = m->cfg.logmag_clamp;
+      dc::ProfScope ps(&m->prof, 6, cs);
+      dc::launch_head_istft_f32(h, cs, Tgrid, false, nb);
+    } else {
+      dc::TapConvF32 p{};
+      p.batch = m->d_batch; p.layer = l;
+      p.in_mask = L.ring_cap - 1; p.C_in = L.C_in;
+      p.first_layer = l == 0; p.last_layer = l + 1 == nL; p.rate_in = L.rate_in;
+      if (l == 0) p.save_rows = L.halo;
+      if (L.kind == 0) {
+        p.n_taps = 3; p.shift[0] = 2 * L.dil; p.shift[1] = L.dil; p.shift[2] = 0; p.n_phase = 1;
+        p.w_tap_stride = (long long)L.C_in * L.C_out; p.w_phase_stride = 0;
+      } else {
+        p.n_taps = 2; p.shift[0] = 0; p.shift[1] = 1; p.shift[2] = 0; p.n_phase = L.stride;
+        p.w_tap_stride = (long long)L.stride * L.C_in * L.C_out; p.w_phase_stride = (long long)L.C_in * L.C_out;
+      }
+      p.W = m->d_w + L.w_off; p.bias = m->d_w + L.b_off; p.C_out = L.C_out;
+      p.residual_silu = L.residual_silu; p.post_silu = L.post_silu;
+      if (L.excite) {
+        p.exc_std = m->cfg.excitation_std; p.exc_seed_lo = m->cfg.excitation_seed_lo; p.exc_seed_hi = m->cfg.excitation_seed_hi;
+      }
+      if (l + 1 < nL) p.out_mask = m->layers[l + 1].ring_cap - 1;
+      dc::ProfScope ps(&m->prof, 5, cs);
+      dc::launch_tapconv_f32(p, cs, Tgrid, false, nb);
+    }
+    ++*launches;
+  }
+}
+
+// Captured once per model (at dc_create): the batch step is one graph launch, only the slot records change.
+static void build_f32_batch_graph(dc_model* m) {
+  if (m->cfg.options & DC_OPT_NO_GRAPH) return;
+  cudaStream_t cap = nullptr;
+  if (cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return; }
+  cudaGraph_t graph = nullptr;
+  if (cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+    static const dc::F32Batch empty{};
+    dc::launch_set_f32_batch(empty, m->d_batch, cap);
+    int n = 1;
+    enqueue_f32_batch(m, cap, &n);
+    if (cudaStreamEndCapture(cap, &graph) == cudaSuccess && graph != nullptr) {
+      size_t n_nodes = 0;
+      cudaGraphGetNodes(graph, nullptr, &n_nodes);
+      std::vector<cudaGraphNode_t> nodes(n_nodes);
+      cudaGraphGetNodes(graph, nodes.data(), &n_nodes);
+      for (cudaGraphNode_t nd : nodes) {
+        cudaGraphNodeType ty;
+        cudaKernelNodeParams kp{};
+        if (cudaGraphNodeGetType(nd, &ty) == cudaSuccess && ty == cudaGraphNodeTypeKernel &&
+            cudaGraphKernelNodeGetParams(nd, &kp) == cudaSuccess && kp.func == dc::set_f32_batch_func())
+          m->gb_set_node = nd;
+      }
+      if (m->gb_set_node != nullptr && cudaGraphInstantiate(&m->gb_exec, graph, 0) == cudaSuccess) {
+        m->gb_graph = graph;
+        m->gb_launches = n;
+        graph = nullptr;
+      } else {
+        m->gb_exec = nullptr;
+      }
+    }
+  }
+  cudaGetLastError();
+  if (graph) cudaGraphDestroy(graph);
+  cudaStreamDestroy(cap);
+}
+
+// One chunk for each of n streams of an fp32 model (admitted by the caller).
+static dc_status decode_f32_batch(dc_model* m, int n, dc_stream* const* streams, const float* const* feats, const int* T, float* const* out,
+                                  cudaStream_t cs, int* launches) {
+  dc::F32Batch hb{};
+  hb.n = n;
+  for (int i = 0; i < n; ++i) {
+    dc_stream* s = streams[i];
+    hb.s[i].call = dc::F32Call{s->frames_total, T[i], (int)(s->chunks & 1), feats[i], out[i], s->rng_id};
+    hb.s[i].ptrs = s->d_ptrs;
+  }
+  if (m->gb_exec != nullptr && !m->prof.on) {
+    dc::F32Batch* dst = m->d_batch;
+    void* args[2] = {&hb, &dst};
+    cudaKernelNodeParams kp{};
+    kp.func = const_cast<void*>(dc::set_f32_batch_func());
+    kp.gridDim = dim3(1);
+    kp.blockDim = dim3(dc::F32_MAX_BATCH);
+    kp.kernelParams = args;
+    DC_CUDA(cudaGraphExecKernelNodeSetParams(m->gb_exec, m->gb_set_node, &kp));
+    DC_CUDA(cudaGraphLaunch(m->gb_exec, cs));
+    *launches += m->gb_launches;
+    m->counters[7]++;
+    return DC_OK;
+  }
+  dc::launch_set_f32_batch(hb, m->d_batch, cs);
+  ++*launches;
+  enqueue_f32_batch(m, cs, launches);
+  DC_CUDA(cudaGetLastError());
+  return DC_OK;
+}
+
 static dc_status decode_f32(dc_stream* s, const float* feats, int T, float* out, cudaStream_t cs, int* launches) {
   dc_model* m = s->model;
   if (s->g_exec != nullptr && !m->prof.on) {
@@ -979,10 +1091,6 @@ extern "C" dc_status dc_decode_wavefront(dc_stream* s, const float* feats, long 
 extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* streams, const float* const* feats,
                                      const int* n_frames, float* const* out, void* cuda_stream) {
   if (!m || !streams || !feats || !n_frames || !out) return DC_ERR_ARG;
-  if (!m->flow && !m->sub_flow) {
-    dc::set_error("dc_decode_batch serves the flow and token2wav pipelines only");
-    return DC_ERR_CONFIG;
-  }
   if (n < 1 || n > m->cfg.max_batch) {
     m->counters[3]++;
     dc::set_error("batch of %d streams, max_batch = %d", n, m->cfg.max_batch);
@@ -1014,25 +1122,27 @@ extern "C" dc_status dc_decode_batch(dc_model* m, int n, dc_stream* const* strea
       mels[(size_t)i] = streams[i]->mel;
     }
     st = dc_decode_batch(m->sub_flow, n, fs.data(), feats, n_frames, mels.data(), cuda_stream);
-    // the tails are independent of one another: spread over the model's side streams, behind the flow
-    // decoder, and joined back into the caller's stream (all on cuda_stream while profiling: the event
-    // brackets assume one stream)
-    cudaStream_t cs = (cudaStream_t)cuda_stream;
-    const int n_side = (n >= 2 && !m->sub_voc->prof.on && !m->sub_flow->prof.on) ? (int)m->tail_streams.size() : 0;
-    if (st == DC_OK && n_side > 0 && cudaEventRecord(m->tail_fork, cs) != cudaSuccess) st = DC_ERR_CUDA;
-    for (int i = 0; i < n && st == DC_OK; ++i) {
-      cudaStream_t ts = n_side > 0 ? m->tail_streams[(size_t)(i % n_side)] : cs;
-      if (n_side > 0 && i < n_side && cudaStreamWaitEvent(ts, m->tail_fork, 0) != cudaSuccess) st = DC_ERR_CUDA;
-      if (st == DC_OK)
-        st = dc_decode_chunk(streams[i]->sub_voc, streams[i]->mel, n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk, out[i],
-                             nullptr, (void*)ts);
+    // ... then the vocoder tails of all the streams, every layer one launch over the batch (n = 1, or
+    // DC_OPT_SERIAL_TAILS: stream by stream, one captured step each)
+    if (st == DC_OK) {
+      std::vector<dc_stream*> vs((size_t)n);
+      std::vector<int> tc((size_t)n);
+      for (int i = 0; i < n; ++i) {
+        vs[(size_t)i] = streams[i]->sub_voc;
+        tc[(size_t)i] = n_frames[i] < m->cfg.f_chunk ? n_frames[i] : m->cfg.f_chunk;
+      }
+      if (n >= 2 && !(m->cfg.options & DC_OPT_SERIAL_TAILS)) {
+        st = dc_decode_batch(m->sub_voc, n, vs.data(), mels.data(), tc.data(), out, cuda_stream);
+      } else {
+        for (int i = 0; i < n && st == DC_OK; ++i) st = dc_decode_chunk(vs[(size_t)i], mels[(size_t)i], tc[(size_t)i], out[i], nullptr, cuda_stream);
+      }
     }
-    for (int k = 0; k < n_side && k < n && st == DC_OK; ++k)
-      if (cudaEventRecord(m->tail_done[(size_t)k], m->tail_streams[(size_t)k]) != cudaSuccess ||
-          cudaStreamWaitEvent(cs, m->tail_done[(size_t)k], 0) != cudaSuccess)
-        st = DC_ERR_CUDA;
-  } else {
+  } else if (m->flow) {
     st = dc::flow_decode(m->flow, n, states.data(), feats, n_frames, out, (cudaStream_t)cuda_stream, &launches);
+  } else if (m->d_batch == nullptr) {   // an fp32 model created with max_batch = 1
+    st = decode_f32(streams[0], feats[0], n_frames[0], out[0], (cudaStream_t)cuda_stream, &launches);
+  } else {
+    st = decode_f32_batch(m, n, streams, feats, n_frames, out, (cudaStream_t)cuda_stream, &launches);
   }
   m->counters[5] += (uint64_t)launches;
   if (st != DC_OK) {

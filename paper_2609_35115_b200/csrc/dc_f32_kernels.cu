@@ -63,8 +63,23 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
   const float* in_direct = p.in_direct;
   float* out_direct = p.out_direct;
   int exc_rng_id = p.exc_rng_id;
-  if (p.call != nullptr) {
-    const F32Call c = *p.call;
+  const float* in_ring = p.in_ring;
+  float* out_ring = p.out_ring;
+  float* save_ring = p.save_ring;
+  int phase = blockIdx.z;
+  const F32Call* callp = p.call;
+  if (p.batch != nullptr) {
+    const int slot = blockIdx.z / p.n_phase;
+    phase = blockIdx.z - slot * p.n_phase;
+    if (slot >= p.batch->n) return;
+    const F32BatchSlot& bs = p.batch->s[slot];
+    callp = &bs.call;
+    in_ring = bs.ptrs->ring[p.layer];
+    out_ring = p.last_layer ? nullptr : bs.ptrs->ring[p.layer + 1];
+    save_ring = p.first_layer ? bs.ptrs->ring[p.layer] : nullptr;
+  }
+  if (callp != nullptr) {
+    const F32Call c = *callp;
     exc_rng_id = c.rng_id;
     T_in = c.T * p.rate_in;
     pos_in = c.frames * p.rate_in;
@@ -73,7 +88,6 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
     out_direct = p.last_layer ? c.out : nullptr;
   }
   if ((int)blockIdx.x * BM >= T_in) return;   // the grid is sized for the longest chunk
-  const float* in_ring = p.in_ring;
   const int in_mask = p.in_mask, C_in = p.C_in, C_out = p.C_out;
   const int sh0 = p.shift[0], sh1 = p.shift[1], sh2 = p.shift[2];
   constexpr int NTG = TT::NTG;
@@ -87,7 +101,7 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
   const int tid = threadIdx.x - grp * NTG;
   float* gbase = f32_smem + grp * TT::GROUP_FLOATS;
   const int tx = tid % TX, ty = tid / TX;
-  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, phase = blockIdx.z;
+  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
   const float* Wp = p.W + (long long)phase * p.w_phase_stride;
 
   const int kb_per_tap = (C_in + BK - 1) / BK;
@@ -228,7 +242,7 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
       }
       float* dst = (out_direct != nullptr)
                        ? out_direct + (t_out - pos_out) * C_out + n
-                       : p.out_ring + (long long)((int)(t_out & (long long)p.out_mask)) * C_out + n;
+                       : out_ring + (long long)((int)(t_out & (long long)p.out_mask)) * C_out + n;
       *reinterpret_cast<float4*>(dst) = v;
     }
   }
@@ -236,13 +250,13 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
   // Carry update of the first layer: its left context for the next chunk is the tail of the
   // caller's chunk, written into ring rows that no CTA of this launch reads (distinct logical
   // frames map to distinct rows because the ring holds f_chunk + halo frames).
-  if (p.save_ring != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+  if (save_ring != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && phase == 0) {
     const int first = T_in > p.save_rows ? T_in - p.save_rows : 0;
     const int c4 = C_in >> 2;
     for (int i = tid; i < (T_in - first) * c4; i += NTG) {
       const int r = first + i / c4, c = (i - (i / c4) * c4) * 4;
       const float4 v = *reinterpret_cast<const float4*>(in_direct + (long long)r * C_in + c);
-      *reinterpret_cast<float4*>(p.save_ring + (long long)((int)((pos_in + r) & (long long)in_mask)) * C_in + c) = v;
+      *reinterpret_cast<float4*>(save_ring + (long long)((int)((pos_in + r) & (long long)in_mask)) * C_in + c) = v;
     }
   }
 }
@@ -268,6 +282,13 @@ __global__ void __launch_bounds__(HT) head_istft_f32_kernel(const HeadIstftF32 p
   ptx::pdl_launch();
   ptx::pdl_wait();
   HeadIstftF32 p = p_in;
+  if (p.batch != nullptr) {
+    if ((int)blockIdx.y >= p.batch->n) return;
+    const F32BatchSlot& bs = p.batch->s[blockIdx.y];
+    p.call = &bs.call;
+    p.in_ring = bs.ptrs->ring[p.layer];
+    p.tails = bs.ptrs->tails;
+  }
   if (p.call != nullptr) {
     const F32Call c = *p.call;
     p.T = c.T * p.rate_in;
@@ -376,6 +397,14 @@ __global__ void set_f32_call_kernel(const F32Call v, F32Call* dst) {
   if (threadIdx.x == 0) *dst = v;
 }
 
+__global__ void set_f32_batch_kernel(const __grid_constant__ F32Batch v, F32Batch* dst) {
+  if (threadIdx.x == 0) {
+    dst->n = v.n;
+    dst->pad = 0;
+  }
+  if ((int)threadIdx.x < v.n) dst->s[threadIdx.x] = v.s[threadIdx.x];
+}
+
 template <typename... KArgs, typename... Args>
 void launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl, Args&&... args) {
   cudaLaunchConfig_t cfg{};
@@ -394,7 +423,7 @@ void launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cud
 }
 
 template <int BM, int BN>
-void launch_tile(const TapConvF32& p, int KS, int T_grid, cudaStream_t st, bool pdl) {
+void launch_tile(const TapConvF32& p, int KS, int T_grid, cudaStream_t st, bool pdl, int n_batch) {
   using TT = TapTile<BM, BN>;
   static bool attr_set[64] = {false};
   int dev = 0;
@@ -404,7 +433,7 @@ void launch_tile(const TapConvF32& p, int KS, int T_grid, cudaStream_t st, bool 
     cudaFuncSetAttribute(tapconv_f32_kernel<BM, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, want > 227 * 1024 ? 227 * 1024 : want);
     attr_set[dev] = true;
   }
-  dim3 grid((T_grid + BM - 1) / BM, (p.C_out + BN - 1) / BN, p.n_phase);
+  dim3 grid((T_grid + BM - 1) / BM, (p.C_out + BN - 1) / BN, p.n_phase * (n_batch > 0 ? n_batch : 1));
   launch_ex(tapconv_f32_kernel<BM, BN>, grid, dim3(KS * TT::NTG), (size_t)KS * TT::GROUP_FLOATS * sizeof(float), st, pdl, p, KS);
 }
 }  // namespace
@@ -415,19 +444,24 @@ void launch_set_f32_call(const F32Call& v, F32Call* dst, cudaStream_t st) {
   set_f32_call_kernel<<<1, 32, 0, st>>>(v, dst);
 }
 
-void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st, int T_grid, bool pdl) {
+void launch_set_f32_batch(const F32Batch& v, F32Batch* dst, cudaStream_t st) {
+  set_f32_batch_kernel<<<1, F32_MAX_BATCH, 0, st>>>(v, dst);
+}
+const void* set_f32_batch_func() { return (const void*)set_f32_batch_kernel; }
+
+void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st, int T_grid, bool pdl, int n_batch) {
   if (T_grid < 0) T_grid = p.T_in;
   const int nkb = p.n_taps * ((p.C_in + BK - 1) / BK);
   const long long ctas64 = (long long)((T_grid + 63) / 64) * ((p.C_out + 63) / 64) * p.n_phase;
   if (ctas64 >= 296) {
-    launch_tile<64, 64>(p, 1, T_grid, st, pdl);
+    launch_tile<64, 64>(p, 1, T_grid, st, pdl, n_batch);
   } else {
     // few tiles: small tiles, and split the reduction inside the CTA until the GPU holds about
     // 1200 warps (8 per SM), keeping at least 4 steps per group; at most 8 groups (512 threads)
     const long long ctas32 = (long long)((T_grid + 31) / 32) * ((p.C_out + 31) / 32) * p.n_phase;
     int KS = 1;
     while (KS < 8 && ctas32 * 2 * KS < 1200 && nkb / (2 * KS) >= 4) KS *= 2;
-    launch_tile<32, 32>(p, KS, T_grid, st, pdl);
+    launch_tile<32, 32>(p, KS, T_grid, st, pdl, n_batch);
   }
 }
 
@@ -445,11 +479,11 @@ cudaError_t prepare_f32_constants() {
   return e;
 }
 
-void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st, int T_grid, bool pdl) {
+void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st, int T_grid, bool pdl, int n_batch) {
   if (T_grid < 0) T_grid = p.T;
   const size_t smem = (size_t)(3 * p.C * NH + HFR * NFFT) * sizeof(float);
   const int grid = (T_grid + HF - 1) / HF;
-  launch_ex(head_istft_f32_kernel, dim3(grid), dim3(HT), smem, st, pdl, p);
+  launch_ex(head_istft_f32_kernel, dim3(grid, n_batch > 0 ? n_batch : 1), dim3(HT), smem, st, pdl, p);
 }
 
 }  // namespace dc

@@ -29,7 +29,28 @@ struct F32Call {
   int          rng_id;     // the stream's device random stream (vocoder excitation)
 };
 
+// Several streams of one fp32 model in ONE launch of every layer (multi-session serving): a record per slot in
+// device memory, rewritten per call by a setter kernel (its by-value argument), and - because every stream has
+// rings of its own - a per-stream table of ring addresses written once at dc_stream_open.  Slot i of the batch
+// is grid plane i of every layer kernel; the arithmetic of a slot is exactly that of a single-stream call.
+constexpr int F32_MAX_LAYERS = 24;
+constexpr int F32_MAX_BATCH = 64;
+struct F32StreamPtrs {
+  float* ring[F32_MAX_LAYERS];   // input ring of each layer
+  float* tails;                  // [2][12] overlap-add tails
+};
+struct F32BatchSlot {
+  F32Call              call;
+  const F32StreamPtrs* ptrs;
+};
+struct F32Batch {
+  int          n, pad;
+  F32BatchSlot s[F32_MAX_BATCH];
+};
+
 struct TapConvF32 {
+  const F32Batch* batch;   // if set: slot = blockIdx.z / n_phase; per-call values and ring addresses come from batch->s[slot]
+  int          layer;      // ... ring[layer] is this layer's input ring, ring[layer + 1] its output ring
   const F32Call* call;     // if set: T_in, pos_in, pos_out, in_direct, out_direct come from *call
   int          rate_in;    // ... scaled by this layer's frames per chunk frame
   int          first_layer, last_layer;
@@ -63,13 +84,19 @@ struct TapConvF32 {
 };
 
 // T_grid: frames the grid is sized for (p.T_in, or the largest T_in when p.call is set).
-void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st, int T_grid = -1, bool pdl = false);
+// n_batch > 0: the launch carries that many slots (p.batch set); tile shape and reduction split are those of the
+// single-stream launch of the same layer, so that a slot's result has the single-stream bytes.
+void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st, int T_grid = -1, bool pdl = false, int n_batch = 0);
 void launch_set_f32_call(const F32Call& v, F32Call* dst, cudaStream_t st);
 const void* set_f32_call_func();
+void launch_set_f32_batch(const F32Batch& v, F32Batch* dst, cudaStream_t st);
+const void* set_f32_batch_func();
 
 // Head conv (k = 3, input already SiLU-activated) + magnitude/phase -> inverse real DFT (n_fft = 16)
 // -> synthesis window -> overlap-add (hop 4) with the 12-sample tail carried across chunks.
 struct HeadIstftF32 {
+  const F32Batch* batch;      // if set: slot = blockIdx.y; per-call values, ring and tails come from batch->s[slot]
+  int          layer;
   const F32Call* call;        // if set: pos, T, tails and pcm come from *call
   int          rate_in;
   float*       tails;         // [2][12] ping-pong pair (used with call)
@@ -86,7 +113,7 @@ struct HeadIstftF32 {
   float*       pcm;           // [4*T]
 };
 
-void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st, int T_grid = -1, bool pdl = false);
+void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st, int T_grid = -1, bool pdl = false, int n_batch = 0);
 
 // Uploads the constant tables of the head kernel (DFT twiddles, periodic Hann window) to the
 // current device.  Synchronous; called from dc_create, never from a decode call.

@@ -262,3 +262,59 @@ def test_excitation_needs_a_seed_and_a_vocoder(dc):
     c1 = wl.CONFIGS["cfg1"].replace(excitation_std=0.2, excitation_seed=3)
     with pytest.raises(dc.DCError):
         dc.Model(c1, wl.make_workload(c1).weights)
+
+
+# ---- multi-stream batching of the fp32 pipelines: every layer one launch for all the streams of the batch ----
+
+@pytest.mark.parametrize("make", [lambda: wl.tiny_vocoder(n_streams=5, n_chunks=6, bias_std=0.2, **EXC),
+                                  lambda: wl.CONFIGS["cfg1"].replace(name="cfg1_batch", n_streams=3, bias_std=0.2),
+                                  lambda: wl.CONFIGS["cfg4"].replace(name="cfg4_batch", n_streams=4, n_chunks=3)])
+def test_f32_batched_streams_equal_single_stream_bytes_and_oracle(dc, make):
+    gu = _util()
+    cfg = make()
+    S = cfg.n_streams
+    bounds = None
+    if cfg.f_chunk <= 16:      # ragged and different per stream (a stream that has run out of chunks sits a round out)
+        F = cfg.f_chunk * cfg.n_chunks
+        rng = np.random.default_rng(3)
+        bounds = []
+        for _ in range(S):
+            b = [0]
+            while b[-1] < F:
+                b.append(min(F, b[-1] + int(rng.integers(1, cfg.f_chunk + 1))))
+            bounds.append(b)
+    w = wl.make_workload(cfg, boundaries=bounds)
+    # single-stream runs on a model of their own, so that stream i is that model's i-th stream here too
+    m1 = dc.Model(cfg, w.weights)
+    single = []
+    for s in w.streams:
+        st = m1.open_stream()
+        single.append(gu.run_gpu_stream(m1, s.feats, s.boundaries, stream=st))
+        st.close()
+    m1.destroy()
+    m = dc.Model(cfg, w.weights, max_batch=S)
+    streams = [m.open_stream() for _ in range(S)]
+    feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+    outs = [torch.zeros(s.boundaries[-1] * cfg.out_per_frame, device="cuda") for s in w.streams]
+    opf = cfg.out_per_frame
+    c0 = m.counters()
+    rounds = max(len(s.boundaries) - 1 for s in w.streams)
+    calls = 0
+    for r in range(rounds):
+        idx = [i for i, s in enumerate(w.streams) if r < len(s.boundaries) - 1]
+        fs = [feats[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in idx]
+        os_ = [outs[i][w.streams[i].boundaries[r] * opf:w.streams[i].boundaries[r + 1] * opf] for i in idx]
+        dc.decode_batch(m, [streams[i] for i in idx], fs, os_)
+        calls += 1
+    torch.cuda.synchronize()
+    c1 = m.counters()
+    assert c1[7] - c0[7] == calls                         # one graph launch per round, whoever is present
+    for st in streams:
+        st.close()
+    m.destroy()
+    for i, s in enumerate(w.streams):
+        got = outs[i].cpu().numpy().reshape(single[i].shape)
+        assert np.array_equal(got, single[i]), f"{cfg.name}: stream {i} differs from its single-stream bytes"
+        if i < 2:
+            ref = orc.run_stream(cfg, w.weights, s.feats, s.boundaries, stream_id=i)
+            assert gu.rel_err(got, ref) <= TOL_F32
