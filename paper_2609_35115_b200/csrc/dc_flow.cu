@@ -5,13 +5,16 @@
 // row GUARD + 64 i, whose rows 0..7 hold the conv left context (the last 8 block-input frames of
 // the previous chunk, copied in from the stream's carry by the producing epilogue) and rows
 // 8..8+T-1 the T <= 56 frames of the chunk.  A tap of a dilated conv is then a plain row shift
-// of the whole matrix, so the k = 3 conv is three accumulating UMMA passes whose A tiles are TMA
-// boxes at row offsets -2d, -d, 0.  One CTA computes a 128 x BN output tile (two slots).
+// of the whole matrix.  One CTA computes a 128 x BN output tile (two slots).
 //
-// GEMM kernel: warp 0 = TMA producer, warp 1 = UMMA issuer (accumulator in tensor memory),
-// warps 2..5 = epilogue (one TMEM lane = one output row per thread).  The epilogues fuse bias,
-// timestep bias, SiLU, residual, the carry update of the next conv block, the in-place append of
-// K/V rows to the stream's ring, and the Euler update.
+// GEMM kernel (640 threads, one CTA per SM): warp 0 = TMA producer of the A tiles, warp 2 = TMA
+// producer of the weight tiles, warps 1 and 3 = UMMA issuers (even / odd reduction blocks into
+// accumulators of their own in tensor memory), warps 4..19 = epilogue (one TMEM lane = one output
+// row per thread, one 16-column chunk in four).  The three taps of a conv block are the column
+// blocks of ONE 128 x 3BN x 16 UMMA per reduction step; the epilogue shifts the tap products by
+// rows through shared memory and adds them.  The epilogues fuse bias, timestep bias, SiLU,
+// residual, the carry update of the next conv block, the row statistics of the RMS norm, the
+// in-place append of K/V rows to the stream's ring, and the Euler update.
 #include <cuda.h>
 #include <math.h>
 #include <stdio.h>
