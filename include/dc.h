@@ -79,6 +79,11 @@ enum {
    * kernel and one activation round trip less per norm).  DC_PIPE_TOKEN2WAV always builds its flow decoder
    * this way: the vocoder tail amplifies the flow stage's deviation several times. */
   DC_OPT_ROUNDED_NORM = 16,
+  /* Debug aid (the stand-in for a memory checker): every device buffer of a stream opened on this model is
+   * allocated with 256 bytes of a known pattern in front of it and behind it; dc_stream_check_guards reads the
+   * patterns back.  An index error in a kernel that writes just outside a carry is then reported instead of
+   * silently corrupting a neighbour. */
+  DC_OPT_GUARD_ZONES = 32,
   /* MEASUREMENT ONLY - the outputs of such a model are meaningless: the step without the kernels of
    * one class, so that step-time differences give that class's cost inside the captured graph. */
   DC_OPT_SKIP_CONV_GEMM = 1 << 16,
@@ -370,6 +375,18 @@ dc_status dc_stream_carry_info(const dc_stream* stream, uint64_t* out, int max_e
  * per chunk, Section 3.3 "Granularity", Eq. 6; rejected calls by reason: Section 3.3's counted
  * refusal reasons). */
 dc_status dc_get_counters(const dc_model* model, uint64_t counters[8]);
+
+/* Checks the guard zones around every device buffer of the stream (carries, rings, tails, staging; a model created
+ * with DC_OPT_GUARD_ZONES - otherwise there is nothing to check and the call returns DC_OK).  Synchronises the
+ * device.  DC_OK if every pattern is intact, DC_ERR_STATE if not (*n_damaged, which may be NULL, receives the number of
+ * overwritten zones).  (Fail-closed discipline, paper Section 3.3, applied to the library's own memory.) */
+dc_status dc_stream_check_guards(dc_stream* stream, int* n_damaged);
+
+/* Host-side fault injection for tests (the paper has no counterpart): the nth device allocation that the calling
+ * thread makes through this library from now on fails as if the device were out of memory, without touching the
+ * device (nth = 1: the next one; 0 disarms).  dc_create and dc_stream_open must then return DC_ERR_OOM with
+ * everything they had allocated released. */
+dc_status dc_test_fail_allocation(int nth);
 
 /* Self-test of the bounded device-side wait that every pipeline barrier in the kernels uses (the
  * fail-closed discipline of paper Section 3.3, applied to the device): launches a one-CTA kernel

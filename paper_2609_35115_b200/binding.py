@@ -22,7 +22,7 @@ EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_
            "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error",
            "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end", "dc_conv_stack_noalloc",
            "dc_selftest_bounded_wait", "dc_stream_snapshot", "dc_stream_restore", "dc_snapshot_free",
-           "dc_decode_wavefront", "dc_decode_wavefront_batch"]
+           "dc_decode_wavefront", "dc_decode_wavefront_batch", "dc_stream_check_guards", "dc_test_fail_allocation"]
 
 
 class dc_config(C.Structure):
@@ -79,6 +79,8 @@ def load_library():
     lib.dc_profile_end.argtypes = [vp, cp(C.c_double), cp(C.c_uint64)]
     lib.dc_conv_stack_noalloc.argtypes = [vp, C.c_int, C.c_int, cp(C.c_int), vp, C.c_int, vp, vp]
     lib.dc_selftest_bounded_wait.argtypes = [C.c_int]
+    lib.dc_stream_check_guards.argtypes = [vp, cp(C.c_int)]
+    lib.dc_test_fail_allocation.argtypes = [C.c_int]
     lib.dc_stream_carry_info.argtypes = [vp, cp(C.c_uint64), C.c_int, cp(C.c_int)]
     lib.dc_get_counters.argtypes = [vp, cp(C.c_uint64)]
     lib.dc_status_str.restype = C.c_char_p
@@ -92,7 +94,7 @@ def load_library():
     return lib
 
 
-OPT_NO_GRAPH, OPT_NO_PDL, OPT_NO_ZEROCOPY, OPT_SERIAL_TAILS, OPT_ROUNDED_NORM = 1, 2, 4, 8, 16
+OPT_NO_GRAPH, OPT_NO_PDL, OPT_NO_ZEROCOPY, OPT_SERIAL_TAILS, OPT_ROUNDED_NORM, OPT_GUARD_ZONES = 1, 2, 4, 8, 16, 32
 OPT_SKIP_CONV_GEMM, OPT_SKIP_ATTENTION, OPT_EMPTY_KERNELS = 1 << 16, 1 << 17, 1 << 18     # measurement only: outputs are meaningless
 
 
@@ -270,6 +272,14 @@ class Stream:
         """Writes a snapshot back in place (of this stream or of another stream of the same model)."""
         _check(self.lib.dc_stream_restore(self.handle, snap.handle, _cuda_stream_handle(stream)), "dc_stream_restore")
 
+    def check_guards(self) -> int:
+        """dc_stream_check_guards: returns the number of damaged guard zones (0 = intact); raises on other errors."""
+        n = C.c_int(0)
+        st = self.lib.dc_stream_check_guards(self.handle, C.byref(n))
+        if st not in (0, 7):
+            _check(st, "dc_stream_check_guards")
+        return n.value
+
     def reset(self, stream=None):
         _check(self.lib.dc_stream_reset(self.handle, _cuda_stream_handle(stream)), "dc_stream_reset")
 
@@ -336,6 +346,11 @@ def decode_wavefront_batch(model: Model, streams: Sequence[Stream], feats, outs=
     if model.cfg.pipeline not in ("vocoder", "token2wav"):
         outs = [o.view(-1, model.out_per_frame) for o in outs]
     return outs
+
+
+def fail_allocation(nth: int) -> None:
+    """dc_test_fail_allocation: the nth device allocation of the calling thread from now on fails (0 disarms)."""
+    _check(load_library().dc_test_fail_allocation(nth), "dc_test_fail_allocation")
 
 
 def selftest_bounded_wait(max_polls: int = 1000) -> int:

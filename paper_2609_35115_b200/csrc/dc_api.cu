@@ -11,6 +11,7 @@
 #include <mutex>
 #include <new>
 #include <string>
+#include <map>
 #include <vector>
 
 #include "dc_internal.h"
@@ -26,6 +27,76 @@ void set_error(const char* fmt, ...) {
   vsnprintf(buf, sizeof(buf), fmt, ap);
   va_end(ap);
   g_last_error = buf;
+}
+
+// ---- device allocation shim (see dc_internal.h) ---------------------------------------------------------------
+namespace {
+constexpr size_t   kGuardBytes = 256;
+constexpr int      kGuardByte = 0xC5;
+struct GuardInfo { void* base; size_t bytes; };
+std::mutex g_guard_mu;
+std::map<void*, GuardInfo> g_guarded;          // user pointer -> allocation with guard zones
+thread_local int  g_fail_countdown = 0;         // > 0: the allocation that brings it to 0 fails
+thread_local bool g_guard_mode = false;
+}  // namespace
+
+cudaError_t dev_alloc(void** p, size_t bytes) {
+  *p = nullptr;
+  if (g_fail_countdown > 0 && --g_fail_countdown == 0) return cudaErrorMemoryAllocation;   // injected: the device is not touched
+  if (!g_guard_mode) return cudaMalloc(p, bytes);
+  void* base = nullptr;
+  cudaError_t e = cudaMalloc(&base, bytes + 2 * kGuardBytes);
+  if (e != cudaSuccess) return e;
+  char* user = static_cast<char*>(base) + kGuardBytes;
+  e = cudaMemset(base, kGuardByte, kGuardBytes);
+  if (e == cudaSuccess) e = cudaMemset(user + bytes, kGuardByte, kGuardBytes);
+  if (e != cudaSuccess) {
+    cudaFree(base);
+    return e;
+  }
+  {
+    std::lock_guard<std::mutex> lk(g_guard_mu);
+    g_guarded[user] = GuardInfo{base, bytes};
+  }
+  *p = user;
+  return cudaSuccess;
+}
+
+void dev_free(void* p) {
+  if (!p) return;
+  {
+    std::lock_guard<std::mutex> lk(g_guard_mu);
+    auto it = g_guarded.find(p);
+    if (it != g_guarded.end()) {
+      p = it->second.base;
+      g_guarded.erase(it);
+    }
+  }
+  cudaFree(p);
+}
+
+// Reads the guard zones of one allocation back; returns the number of zones (0..2) whose pattern changed, or -1 on a
+// CUDA error.  An allocation without guard zones counts as intact.
+static int damaged_guards(const void* user) {
+  GuardInfo gi{};
+  {
+    std::lock_guard<std::mutex> lk(g_guard_mu);
+    auto it = g_guarded.find(const_cast<void*>(user));
+    if (it == g_guarded.end()) return 0;
+    gi = it->second;
+  }
+  unsigned char h[2 * kGuardBytes];
+  if (cudaMemcpy(h, gi.base, kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(h + kGuardBytes, static_cast<const char*>(user) + gi.bytes, kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return -1;
+  int bad = 0;
+  for (int z = 0; z < 2; ++z)
+    for (size_t i = 0; i < kGuardBytes; ++i)
+      if (h[z * kGuardBytes + i] != kGuardByte) {
+        ++bad;
+        break;
+      }
+  return bad;
 }
 
 #define DC_CUDA(expr)                                                                    \
@@ -95,7 +166,7 @@ struct dc_model {
 static void free_batch_graph(dc_model* m) {
   if (m->gb_exec) cudaGraphExecDestroy(m->gb_exec);
   if (m->gb_graph) cudaGraphDestroy(m->gb_graph);
-  if (m->d_batch) cudaFree(m->d_batch);
+  if (m->d_batch) dc::dev_free(m->d_batch);
   m->gb_exec = nullptr;
   m->gb_graph = nullptr;
   m->d_batch = nullptr;
@@ -164,7 +235,7 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (c->f_prompt != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_prompt belongs to the flow decoder");
   if (c->cfg_scale != 0.f && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("cfg_scale belongs to the flow decoder");
   if (c->options & ~(uint32_t)(DC_OPT_NO_GRAPH | DC_OPT_NO_PDL | DC_OPT_NO_ZEROCOPY | DC_OPT_SERIAL_TAILS | DC_OPT_ROUNDED_NORM | DC_OPT_SKIP_CONV_GEMM |
-                               DC_OPT_SKIP_ATTENTION | DC_OPT_EMPTY_KERNELS))
+                               DC_OPT_SKIP_ATTENTION | DC_OPT_EMPTY_KERNELS | DC_OPT_GUARD_ZONES))
     BAD("unknown option bit");
   if (!(c->excitation_std >= 0.f && c->excitation_std <= 1e6f)) BAD("excitation_std out of range");
   if (c->excitation_std > 0.f && c->pipeline != DC_PIPE_VOCODER && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("excitation_std belongs to the vocoder tail");
@@ -337,8 +408,8 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
       if (e == cudaSuccess) e = cudaMallocHost(&m->h_out, no * sizeof(float));
       if (e == cudaSuccess) e = cudaMallocHost(&m->h_err, sizeof(int));
       m->zero_copy = !(cfg->options & DC_OPT_NO_ZEROCOPY);
-      if (e == cudaSuccess) e = cudaMalloc(&m->d_in, ni * sizeof(float));
-      if (e == cudaSuccess) e = cudaMalloc(&m->d_out, no * sizeof(float));
+      if (e == cudaSuccess) e = dc::dev_alloc(&m->d_in, ni * sizeof(float));
+      if (e == cudaSuccess) e = dc::dev_alloc(&m->d_out, no * sizeof(float));
       if (e != cudaSuccess) {
         dc::set_error("staging allocation failed: %s", cudaGetErrorString(e));
         st = DC_ERR_OOM;
@@ -346,11 +417,11 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     }
   } else {
     build_f32_layers(m);
-    cudaError_t e = cudaMalloc(&m->d_w, n_floats * sizeof(float));
+    cudaError_t e = dc::dev_alloc(&m->d_w, n_floats * sizeof(float));
     if (e == cudaSuccess) e = cudaMemcpy(m->d_w, w, n_floats * sizeof(float), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = dc::prepare_f32_constants();
     if (e == cudaSuccess && cfg->max_batch > 1) {
-      e = cudaMalloc(&m->d_batch, sizeof(dc::F32Batch));
+      e = dc::dev_alloc(&m->d_batch, sizeof(dc::F32Batch));
       if (e == cudaSuccess) e = cudaMemset(m->d_batch, 0, sizeof(dc::F32Batch));
     }
     if (e != cudaSuccess) {
@@ -363,13 +434,13 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     if (m->sub_flow) dc_destroy(m->sub_flow);
     if (m->sub_voc) dc_destroy(m->sub_voc);
     free_batch_graph(m);
-    if (m->d_w) cudaFree(m->d_w);
+    if (m->d_w) dc::dev_free(m->d_w);
     if (m->flow) dc::flow_model_destroy(m->flow);
     if (m->h_in) cudaFreeHost(m->h_in);
     if (m->h_out) cudaFreeHost(m->h_out);
     if (m->h_err) cudaFreeHost(m->h_err);
-    if (m->d_in) cudaFree(m->d_in);
-    if (m->d_out) cudaFree(m->d_out);
+    if (m->d_in) dc::dev_free(m->d_in);
+    if (m->d_out) dc::dev_free(m->d_out);
     delete m;
     return st;
   }
@@ -387,12 +458,12 @@ extern "C" dc_status dc_destroy(dc_model* m) {
   if (m->sub_voc) dc_destroy(m->sub_voc);
   free_batch_graph(m);
   if (m->flow) dc::flow_model_destroy(m->flow);
-  if (m->d_w) cudaFree(m->d_w);
+  if (m->d_w) dc::dev_free(m->d_w);
   if (m->h_in) cudaFreeHost(m->h_in);
   if (m->h_out) cudaFreeHost(m->h_out);
   if (m->h_err) cudaFreeHost(m->h_err);
-  if (m->d_in) cudaFree(m->d_in);
-  if (m->d_out) cudaFree(m->d_out);
+  if (m->d_in) dc::dev_free(m->d_in);
+  if (m->d_out) dc::dev_free(m->d_out);
   for (dc_stream* s : m->all_streams) delete s;
   delete m;
   return DC_OK;
@@ -404,18 +475,18 @@ static void free_stream_buffers(dc_stream* s) {
   s->g_exec = nullptr;
   s->g_graph = nullptr;
   for (auto& b : s->f32_rings)
-    if (b.p) cudaFree(b.p);
+    if (b.p) dc::dev_free(b.p);
   s->f32_rings.clear();
-  if (s->tails) cudaFree(s->tails);
-  if (s->d_call) cudaFree(s->d_call);
+  if (s->tails) dc::dev_free(s->tails);
+  if (s->d_call) dc::dev_free(s->d_call);
   s->d_call = nullptr;
-  if (s->d_ptrs) cudaFree(s->d_ptrs);
+  if (s->d_ptrs) dc::dev_free(s->d_ptrs);
   s->d_ptrs = nullptr;
   if (s->flow) dc::flow_state_close(s->flow);
   if (s->sub_flow) dc_stream_close(s->sub_flow);
   if (s->sub_voc) dc_stream_close(s->sub_voc);
-  if (s->mel) cudaFree(s->mel);
-  if (s->wave_mel) cudaFree(s->wave_mel);
+  if (s->mel) dc::dev_free(s->mel);
+  if (s->wave_mel) dc::dev_free(s->wave_mel);
   s->wave_mel = nullptr;
   if (s->wave_side) cudaStreamDestroy(s->wave_side);
   if (s->wave_ev) cudaEventDestroy(s->wave_ev);
@@ -423,8 +494,8 @@ static void free_stream_buffers(dc_stream* s) {
   s->wave_ev = nullptr;
   s->sub_flow = s->sub_voc = nullptr;
   s->mel = nullptr;
-  if (s->stage_in) cudaFree(s->stage_in);
-  if (s->stage_out) cudaFree(s->stage_out);
+  if (s->stage_in) dc::dev_free(s->stage_in);
+  if (s->stage_out) dc::dev_free(s->stage_out);
   s->tails = nullptr;
   s->flow = nullptr;
   s->stage_in = s->stage_out = nullptr;
@@ -438,14 +509,19 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
   s->model = m;
   cudaError_t e = cudaSuccess;
   dc_status st = DC_OK;
+  struct GuardScope {   // every device buffer of a stream gets guard zones when the model asks for them
+    bool prev;
+    explicit GuardScope(bool on) : prev(dc::g_guard_mode) { dc::g_guard_mode = prev || on; }
+    ~GuardScope() { dc::g_guard_mode = prev; }
+  } guard_scope((m->cfg.options & DC_OPT_GUARD_ZONES) != 0);
   if (m->sub_flow) {
     st = dc_stream_open(m->sub_flow, &s->sub_flow);
     if (st == DC_OK) st = dc_stream_open(m->sub_voc, &s->sub_voc);
-    if (st == DC_OK) e = cudaMalloc(&s->mel, (size_t)m->cfg.f_chunk * m->cfg.mel_dim * sizeof(float));
+    if (st == DC_OK) e = dc::dev_alloc(&s->mel, (size_t)m->cfg.f_chunk * m->cfg.mel_dim * sizeof(float));
     if (st == DC_OK && e == cudaSuccess && m->cfg.max_wave_frames > 0) {
       // wavefront calls keep a whole call's mel frames on the device and run the vocoder tails on a side stream:
       // both are set up here, so that no decode call allocates or creates anything
-      e = cudaMalloc(&s->wave_mel, (size_t)m->cfg.max_wave_frames * m->cfg.mel_dim * sizeof(float));
+      e = dc::dev_alloc(&s->wave_mel, (size_t)m->cfg.max_wave_frames * m->cfg.mel_dim * sizeof(float));
       if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->wave_side, cudaStreamNonBlocking);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->wave_ev, cudaEventDisableTiming);
       if (e == cudaSuccess) s->wave_mel_frames = m->cfg.max_wave_frames;
@@ -456,28 +532,28 @@ extern "C" dc_status dc_stream_open(dc_model* m, dc_stream** out) {
     s->rng_id = m->streams_opened++;
     for (const F32Layer& L : m->layers) {
       DevBuf b{nullptr, (size_t)L.ring_cap * L.C_in * sizeof(float)};
-      e = cudaMalloc(&b.p, b.bytes);
+      e = dc::dev_alloc(&b.p, b.bytes);
       if (e != cudaSuccess) break;
       s->f32_rings.push_back(b);
       e = cudaMemset(b.p, 0, b.bytes);
       if (e != cudaSuccess) break;
     }
-    if (e == cudaSuccess) e = cudaMalloc(&s->d_call, sizeof(dc::F32Call));
+    if (e == cudaSuccess) e = dc::dev_alloc(&s->d_call, sizeof(dc::F32Call));
     if (e == cudaSuccess && m->cfg.pipeline == DC_PIPE_VOCODER) {
-      e = cudaMalloc(&s->tails, 2 * 12 * sizeof(float));
+      e = dc::dev_alloc(&s->tails, 2 * 12 * sizeof(float));
       if (e == cudaSuccess) e = cudaMemset(s->tails, 0, 2 * 12 * sizeof(float));
     }
     if (e == cudaSuccess) {
       dc::F32StreamPtrs hp{};
       for (size_t l = 0; l < s->f32_rings.size() && l < (size_t)dc::F32_MAX_LAYERS; ++l) hp.ring[l] = (float*)s->f32_rings[l].p;
       hp.tails = s->tails;
-      e = cudaMalloc(&s->d_ptrs, sizeof(hp));
+      e = dc::dev_alloc(&s->d_ptrs, sizeof(hp));
       if (e == cudaSuccess) e = cudaMemcpy(s->d_ptrs, &hp, sizeof(hp), cudaMemcpyHostToDevice);
     }
   }
   if (e == cudaSuccess && st == DC_OK) {
-    e = cudaMalloc(&s->stage_in, (size_t)(m->cfg.f_chunk + m->cfg.f_lookahead) * m->in_dim * sizeof(float));
-    if (e == cudaSuccess) e = cudaMalloc(&s->stage_out, (size_t)m->cfg.f_chunk * m->out_per_frame * sizeof(float));
+    e = dc::dev_alloc(&s->stage_in, (size_t)(m->cfg.f_chunk + m->cfg.f_lookahead) * m->in_dim * sizeof(float));
+    if (e == cudaSuccess) e = dc::dev_alloc(&s->stage_out, (size_t)m->cfg.f_chunk * m->out_per_frame * sizeof(float));
   }
   if (e != cudaSuccess) {
     dc::set_error("stream allocation failed: %s", cudaGetErrorString(e));
@@ -591,7 +667,7 @@ extern "C" dc_status dc_snapshot_free(dc_snapshot* sn) {
   if (!sn) return DC_ERR_ARG;
   if (sn->sub_flow) dc_snapshot_free(sn->sub_flow);
   if (sn->sub_voc) dc_snapshot_free(sn->sub_voc);
-  if (sn->data) cudaFree(sn->data);
+  if (sn->data) dc::dev_free(sn->data);
   delete sn;
   return DC_OK;
 }
@@ -618,7 +694,7 @@ extern "C" dc_status dc_stream_snapshot(dc_stream* s, dc_snapshot** out, void* c
     }
     const std::vector<DevBuf> bufs = carry_buffers(s);
     for (const DevBuf& b : bufs) sn->bytes += b.bytes;
-    cudaError_t e = cudaMalloc(&sn->data, sn->bytes ? sn->bytes : 1);
+    cudaError_t e = dc::dev_alloc(&sn->data, sn->bytes ? sn->bytes : 1);
     size_t off = 0;
     for (size_t i = 0; i < bufs.size() && e == cudaSuccess; ++i) {
       e = cudaMemcpyAsync((char*)sn->data + off, bufs[i].p, bufs[i].bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream);
@@ -1335,6 +1411,41 @@ extern "C" dc_status dc_get_counters(const dc_model* m, uint64_t counters[8]) {
     counters[5] += a[5] + b[5];
     counters[7] += a[7] + b[7];
   }
+  return DC_OK;
+}
+
+extern "C" dc_status dc_stream_check_guards(dc_stream* s, int* n_damaged) {
+  if (!s) return DC_ERR_ARG;
+  if (s->closed) return DC_ERR_STATE;
+  if (n_damaged) *n_damaged = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return DC_ERR_CUDA;
+  int total = 0;
+  std::vector<dc_stream*> parts = {s};
+  if (s->sub_flow) parts.push_back(s->sub_flow);
+  if (s->sub_voc) parts.push_back(s->sub_voc);
+  for (dc_stream* q : parts) {
+    std::vector<const void*> bufs;
+    for (const DevBuf& b : carry_buffers(q)) bufs.push_back(b.p);
+    for (const void* extra : {(const void*)q->mel, (const void*)q->wave_mel, (const void*)q->stage_in, (const void*)q->stage_out,
+                              (const void*)q->d_call, (const void*)q->d_ptrs})
+      if (extra) bufs.push_back(extra);
+    for (const void* b : bufs) {
+      const int bad = dc::damaged_guards(b);
+      if (bad < 0) return DC_ERR_CUDA;
+      total += bad;
+    }
+  }
+  if (n_damaged) *n_damaged = total;
+  if (total > 0) {
+    dc::set_error("%d guard zone(s) around the stream's device buffers were overwritten", total);
+    return DC_ERR_STATE;
+  }
+  return DC_OK;
+}
+
+extern "C" dc_status dc_test_fail_allocation(int nth) {
+  if (nth < 0) return DC_ERR_ARG;
+  dc::g_fail_countdown = nth;
   return DC_OK;
 }
 

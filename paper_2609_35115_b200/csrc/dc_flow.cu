@@ -1087,7 +1087,7 @@ namespace {
 
 template <typename T>
 cudaError_t dalloc(FlowModel* m, T** p, size_t n, bool zero = true) {
-  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T));
+  cudaError_t e = dev_alloc(p, n * sizeof(T));
   if (e != cudaSuccess) return e;
   m->allocs.push_back(*p);
   return zero ? cudaMemset(*p, 0, n * sizeof(T)) : cudaSuccess;
@@ -1112,7 +1112,7 @@ void flow_model_destroy(FlowModel* m) {
     if (kv.second.graph) cudaGraphDestroy(kv.second.graph);
   }
   if (m->cap_stream) cudaStreamDestroy(m->cap_stream);
-  for (void* p : m->allocs) cudaFree(p);
+  for (void* p : m->allocs) dev_free(p);
   delete m;
 }
 
@@ -1306,10 +1306,10 @@ dc_status flow_state_open(FlowModel* m, FlowState** out) {
   // one set of carries per pass
   s->halo_bytes = (size_t)m->n_pass * c.n_steps * c.n_conv * HALO * m->C * sizeof(bf16);
   s->kv_bytes = (size_t)m->n_pass * c.n_steps * c.n_attn * 2 * (m->P + m->Rk) * m->C * sizeof(bf16);
-  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&s->halo), s->halo_bytes);
+  cudaError_t e = dev_alloc(&s->halo, s->halo_bytes);
   if (e == cudaSuccess) e = cudaMemset(s->halo, 0, s->halo_bytes);
   if (e == cudaSuccess && s->kv_bytes) {
-    e = cudaMalloc(reinterpret_cast<void**>(&s->kv), s->kv_bytes);
+    e = dev_alloc(&s->kv, s->kv_bytes);
     if (e == cudaSuccess) e = cudaMemset(s->kv, 0, s->kv_bytes);
   }
   if (e != cudaSuccess) {
@@ -1346,7 +1346,7 @@ uint64_t flow_graph_launches(const FlowModel* m) { return m->graph_launches; }
 dc_status flow_selftest_bounded_wait(int max_polls) {
   if (max_polls < 1 || max_polls > 1000000) return DC_ERR_ARG;
   int* d = nullptr;
-  if (cudaMalloc(reinterpret_cast<void**>(&d), sizeof(int)) != cudaSuccess) return DC_ERR_OOM;
+  if (dev_alloc(&d, sizeof(int)) != cudaSuccess) return DC_ERR_OOM;
   int h = 0;
   cudaError_t e = cudaMemset(d, 0, sizeof(int));
   if (e == cudaSuccess) {
@@ -1354,7 +1354,7 @@ dc_status flow_selftest_bounded_wait(int max_polls) {
     e = cudaGetLastError();
   }
   if (e == cudaSuccess) e = cudaMemcpy(&h, d, sizeof(int), cudaMemcpyDeviceToHost);
-  cudaFree(d);
+  dev_free(d);
   if (e != cudaSuccess) {
     set_error("bounded-wait self-test failed to run: %s", cudaGetErrorString(e));
     return DC_ERR_CUDA;
@@ -1373,8 +1373,8 @@ int flow_take_device_error(FlowModel* m) {
 
 void flow_state_close(FlowState* s) {
   if (!s) return;
-  if (s->halo) cudaFree(s->halo);
-  if (s->kv) cudaFree(s->kv);
+  if (s->halo) dev_free(s->halo);
+  if (s->kv) dev_free(s->kv);
   delete s;
 }
 

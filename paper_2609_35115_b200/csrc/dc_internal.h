@@ -132,6 +132,16 @@ struct FlowState;    // carries of one stream
 
 void set_error(const char* fmt, ...);
 
+// Every device allocation of the library goes through this pair (dc_api.cu).  Two test facilities hang off it, both
+// host-side: an injected allocation failure (dc_test_fail_allocation: the n-th allocation made by the calling thread
+// from now on reports cudaErrorMemoryAllocation without touching the device) and guard zones (while guard mode is on
+// for the calling thread - dc_stream_open of a model created with DC_OPT_GUARD_ZONES - an allocation gets 256 bytes
+// of a known pattern in front of and behind it, which dc_stream_check_guards reads back).
+cudaError_t dev_alloc(void** p, size_t bytes);
+void        dev_free(void* p);
+template <typename T>
+inline cudaError_t dev_alloc(T** p, size_t bytes) { return dev_alloc(reinterpret_cast<void**>(p), bytes); }
+
 dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** out);
 void      flow_model_destroy(FlowModel* m);
 dc_status flow_state_open(FlowModel* m, FlowState** out);
