@@ -286,7 +286,7 @@ def main():
     as_rows = cfg.pipeline not in ("vocoder", "token2wav")
     out_dv = out_d.view(S, T, -1) if as_rows else out_d
     batched = cfg.pipeline in ("flow", "token2wav") and S > 1
-    batched_host = cfg.pipeline == "flow" and S > 1     # the host-buffer batch call serves the flow pipeline only
+    batched_host = batched                              # dc_decode_batch_host: one call per step for all the streams
     # multi-stream serving: the streams' chunk boundaries are staggered by seeded offsets in [0, f_chunk) - stream i's
     # first chunk has o_i frames (a full chunk if o_i = 0), every later one f_chunk
     offsets = np.random.default_rng(cfg.seed).integers(0, T, S) if (batched and S > 1) else np.zeros(S, dtype=np.int64)

@@ -109,8 +109,8 @@ enum {
  *                     decoder, then vocoder and inverse STFT) in one call - a chunk of
  *                     [conditioning | noise] frames in, PCM out; the mel frames in between stay in a
  *                     device buffer of the stream (bf16 flow decoder, fp32 vocoder tail).  Weights:
- *                     the flow blob followed by the vocoder blob.  dc_decode_batch serves it too (max_batch
- *                     <= 64); dc_decode_batch_host does not.
+ *                     the flow blob followed by the vocoder blob.  dc_decode_batch and dc_decode_batch_host
+ *                     serve it too (max_batch <= 64).
  * The flow decoder runs n_conv / n_attn conv blocks, then one attention layer,
  * repeated n_attn times (n_attn = 0: conv blocks only). */
 typedef struct dc_config {
@@ -291,8 +291,8 @@ dc_status dc_decode_wavefront_batch(dc_model* model, int n, dc_stream* const* st
 dc_status dc_decode_chunk_host(dc_stream* stream, const float* feats_host, int n_frames,
                                float* out_host, int* n_out, void* cuda_stream);
 
-/* dc_decode_batch for callers with host buffers: feats_host[i] / out_host[i] are host
- * pointers (pageable or pinned).  If every input (every output) buffer is page-locked, the
+/* dc_decode_batch for callers with host buffers, all four pipelines: feats_host[i] / out_host[i] are host
+ * pointers (pageable or pinned).  Flow pipeline: if every input (every output) buffer is page-locked, the
  * kernels read the chunks from (write the results into) the caller's buffers directly, with no
  * staging copy and no copy-engine transfer on that side.  Otherwise the call gathers the chunks
  * in a pinned buffer owned by the model, moves them to the device in one transfer, decodes the

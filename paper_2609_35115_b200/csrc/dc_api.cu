@@ -430,6 +430,21 @@ extern "C" dc_status dc_create(const float* w, size_t n_floats, const dc_config*
     }
     if (st == DC_OK && m->d_batch) build_f32_batch_graph(m);
   }
+  if (st == DC_OK && !m->flow && m->h_in == nullptr) {
+    // bounce buffers of dc_decode_batch_host for the pipelines whose kernels do not read host memory themselves
+    // (pinned host + device, max_batch chunks each way), sized once here
+    const size_t ni = (size_t)cfg->max_batch * (cfg->f_chunk + cfg->f_lookahead) * m->in_dim,
+                 no = (size_t)cfg->max_batch * cfg->f_chunk * m->out_per_frame;
+    cudaError_t e = cudaMallocHost(&m->h_in, ni * sizeof(float));
+    if (e == cudaSuccess) e = cudaMallocHost(&m->h_out, no * sizeof(float));
+    if (e == cudaSuccess) e = dc::dev_alloc(&m->d_in, ni * sizeof(float));
+    if (e == cudaSuccess) e = dc::dev_alloc(&m->d_out, no * sizeof(float));
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      dc::set_error("staging allocation failed: %s", cudaGetErrorString(e));
+      st = DC_ERR_OOM;
+    }
+  }
   if (st != DC_OK) {
     if (m->sub_flow) dc_destroy(m->sub_flow);
     if (m->sub_voc) dc_destroy(m->sub_voc);
@@ -1278,12 +1293,13 @@ extern "C" dc_status dc_decode_chunk_host(dc_stream* s, const float* feats_host,
 extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* streams, const float* const* feats_host,
                                           const int* n_frames, float* const* out_host, void* cuda_stream) {
   if (!m || !streams || !feats_host || !n_frames || !out_host) return DC_ERR_ARG;
-  if (!m->flow || !m->h_in) {
-    dc::set_error("dc_decode_batch_host serves the flow pipeline only");
+  if (!m->h_in) {
+    dc::set_error("dc_decode_batch_host: the model has no staging buffers");
     return DC_ERR_CONFIG;
   }
   if (n < 1 || n > m->cfg.max_batch) return DC_ERR_ARG;
   cudaStream_t cs = (cudaStream_t)cuda_stream;
+  dc_model* fmod = m->flow ? m : m->sub_flow;   // the model that owns a flow decoder (and its device error word), if any
   const size_t in_stride = (size_t)(m->cfg.f_chunk + m->cfg.f_lookahead) * m->in_dim, out_stride = (size_t)m->cfg.f_chunk * m->out_per_frame;
   std::vector<const float*> fin((size_t)n);
   std::vector<float*> fout((size_t)n);
@@ -1297,7 +1313,8 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
   // pulls the chunks over the bus, the last output-projection epilogue pushes the mel rows back): no staging
   // copy and no copy-engine operation on either side.  Pageable buffers go through one pinned bounce buffer
   // each way: two transfers per step instead of two per stream.
-  bool in_direct = m->zero_copy, out_direct = m->zero_copy;
+  // (flow pipeline only: its kernels are the ones that can address host memory)
+  bool in_direct = m->flow && m->zero_copy, out_direct = m->flow && m->zero_copy;
   for (int i = 0; i < n && (in_direct || out_direct); ++i) {
     cudaPointerAttributes a{};
     if (in_direct) {
@@ -1330,11 +1347,11 @@ extern "C" dc_status dc_decode_batch_host(dc_model* m, int n, dc_stream* const* 
   dc_status st = dc_decode_batch(m, n, streams, fin.data(), n_frames, fout.data(), cuda_stream);
   if (st != DC_OK) return st;
   if (!out_direct) DC_CUDA(cudaMemcpyAsync(m->h_out, m->d_out, (size_t)n * out_stride * sizeof(float), cudaMemcpyDeviceToHost, cs));
-  DC_CUDA(cudaMemcpyAsync(m->h_err, dc::flow_error_word(m->flow), sizeof(int), cudaMemcpyDeviceToHost, cs));
+  if (fmod) DC_CUDA(cudaMemcpyAsync(fmod->h_err, dc::flow_error_word(fmod->flow), sizeof(int), cudaMemcpyDeviceToHost, cs));
   DC_CUDA(cudaStreamSynchronize(cs));
-  if (*m->h_err != 0) {   // a bounded device-side wait gave up: the results are not valid
-    const int code = *m->h_err;
-    dc::flow_take_device_error(m->flow);
+  if (fmod && *fmod->h_err != 0) {   // a bounded device-side wait gave up: the results are not valid
+    const int code = *fmod->h_err;
+    dc::flow_take_device_error(fmod->flow);
     m->counters[4]++;
     for (int i = 0; i < n; ++i) streams[i]->poisoned = true;
     dc::set_error("device-side wait timed out (code %d)", code);

@@ -155,3 +155,42 @@ def test_chain_with_device_randomness_in_both_stages(dc):
     """The whole decoder step drawing its own randomness: the flow decoder's Euler noise and the vocoder's
     excitation, both Philox streams keyed by the session and its clocks; stage-wise parity as above."""
     _stagewise(dc, wl.tiny_token2wav(n_chunks=len(RAGGED) - 1, noise_seed=41, excitation_std=0.2, excitation_seed=43), boundaries=RAGGED)
+
+
+@pytest.mark.parametrize("make", [lambda: wl.tiny_token2wav(n_chunks=4, n_streams=3), lambda: wl.tiny_vocoder(n_chunks=4, n_streams=3)])
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_batch_call_serves_the_fp32_and_composite_pipelines(dc, make, pinned):
+    """dc_decode_batch_host for the pipelines that stage through the model's bounce buffers: same bytes as the
+    device-pointer batch call, with page-locked and with pageable caller buffers."""
+    cfg = make()
+    w = wl.make_workload(cfg)
+    S = cfg.n_streams
+    m = dc.Model(cfg, w.weights, max_batch=S)
+    opf = cfg.out_per_frame
+
+    def run(host):
+        streams = [m.open_stream() for _ in range(S)]
+        outs = []
+        for r in range(cfg.n_chunks):
+            lo, hi = w.streams[0].boundaries[r], w.streams[0].boundaries[r + 1]
+            if host:
+                fin = [torch.from_numpy(np.ascontiguousarray(s.feats[lo:hi])) for s in w.streams]
+                fout = [torch.zeros((hi - lo) * opf) for _ in range(S)]
+                if pinned:
+                    fin, fout = [t.pin_memory() for t in fin], [t.pin_memory() for t in fout]
+                dc.decode_batch_host(m, streams, fin, fout)
+                outs.append(np.stack([t.numpy().copy() for t in fout]))
+            else:
+                fin = [torch.from_numpy(np.ascontiguousarray(s.feats[lo:hi])).cuda() for s in w.streams]
+                fout = [torch.zeros((hi - lo) * opf, device="cuda") for _ in range(S)]
+                dc.decode_batch(m, streams, fin, fout)
+                torch.cuda.synchronize()
+                outs.append(np.stack([t.cpu().numpy() for t in fout]))
+        for st in streams:
+            st.close()
+        return np.concatenate(outs, axis=1)
+
+    a, b = run(False), run(True)
+    assert m.counters()[4] == 0
+    m.destroy()
+    assert np.isfinite(a).all() and np.array_equal(a, b)
