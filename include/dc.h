@@ -376,6 +376,12 @@ dc_status dc_stream_carry_info(const dc_stream* stream, uint64_t* out, int max_e
  * refusal reasons). */
 dc_status dc_get_counters(const dc_model* model, uint64_t counters[8]);
 
+/* Measures the FP32 fused multiply-add throughput of the current device (TFLOP/s) with a register-only kernel of
+ * independent FMA chains: the denominator of the fp32 pipelines' roofline fractions (the paper's measurement model,
+ * Section 2.2, Eq. 1, needs a peak P for the pipe a stage runs on; for the FP32 pipe no measured figure is supplied,
+ * so the library measures it).  Synchronous, a few milliseconds; allocates and frees a small device buffer. */
+dc_status dc_measure_fp32_peak(double* tflops);
+
 /* Checks the guard zones around every device buffer of the stream (carries, rings, tails, staging; a model created
  * with DC_OPT_GUARD_ZONES - otherwise there is nothing to check and the call returns DC_OK).  Synchronises the
  * device.  DC_OK if every pattern is intact, DC_ERR_STATE if not (*n_damaged, which may be NULL, receives the number of

@@ -22,7 +22,7 @@ EXPORTS = ["dc_weights_count", "dc_create", "dc_destroy", "dc_stream_open", "dc_
            "dc_stream_carry_info", "dc_get_counters", "dc_status_str", "dc_last_error",
            "dc_decode_batch_host", "dc_profile_begin", "dc_profile_end", "dc_conv_stack_noalloc",
            "dc_selftest_bounded_wait", "dc_stream_snapshot", "dc_stream_restore", "dc_snapshot_free",
-           "dc_decode_wavefront", "dc_decode_wavefront_batch", "dc_stream_check_guards", "dc_test_fail_allocation"]
+           "dc_decode_wavefront", "dc_decode_wavefront_batch", "dc_stream_check_guards", "dc_test_fail_allocation", "dc_measure_fp32_peak"]
 
 
 class dc_config(C.Structure):
@@ -81,6 +81,7 @@ def load_library():
     lib.dc_selftest_bounded_wait.argtypes = [C.c_int]
     lib.dc_stream_check_guards.argtypes = [vp, cp(C.c_int)]
     lib.dc_test_fail_allocation.argtypes = [C.c_int]
+    lib.dc_measure_fp32_peak.argtypes = [cp(C.c_double)]
     lib.dc_stream_carry_info.argtypes = [vp, cp(C.c_uint64), C.c_int, cp(C.c_int)]
     lib.dc_get_counters.argtypes = [vp, cp(C.c_uint64)]
     lib.dc_status_str.restype = C.c_char_p
@@ -346,6 +347,13 @@ def decode_wavefront_batch(model: Model, streams: Sequence[Stream], feats, outs=
     if model.cfg.pipeline not in ("vocoder", "token2wav"):
         outs = [o.view(-1, model.out_per_frame) for o in outs]
     return outs
+
+
+def measure_fp32_peak() -> float:
+    """dc_measure_fp32_peak: measured FP32 multiply-add throughput of the current device in TFLOP/s."""
+    v = C.c_double(0.0)
+    _check(load_library().dc_measure_fp32_peak(C.byref(v)), "dc_measure_fp32_peak")
+    return v.value
 
 
 def fail_allocation(nth: int) -> None:

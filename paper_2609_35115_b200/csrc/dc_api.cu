@@ -1460,6 +1460,17 @@ extern "C" dc_status dc_stream_check_guards(dc_stream* s, int* n_damaged) {
   return DC_OK;
 }
 
+extern "C" dc_status dc_measure_fp32_peak(double* tflops) {
+  if (!tflops) return DC_ERR_ARG;
+  *tflops = 0.0;
+  cudaError_t e = dc::measure_fp32_peak(tflops);
+  if (e != cudaSuccess) {
+    dc::set_error("dc_measure_fp32_peak: %s", cudaGetErrorString(e));
+    return e == cudaErrorMemoryAllocation ? DC_ERR_OOM : DC_ERR_CUDA;
+  }
+  return DC_OK;
+}
+
 extern "C" dc_status dc_test_fail_allocation(int nth) {
   if (nth < 0) return DC_ERR_ARG;
   dc::g_fail_countdown = nth;

@@ -465,6 +465,51 @@ void launch_tapconv_f32(const TapConvF32& p, cudaStream_t st, int T_grid, bool p
   }
 }
 
+// ---- FP32 multiply-add peak, measured -----------------------------------------------------------------------
+// Sixteen independent fused multiply-add chains per thread, 1,024 threads per SM-filling CTA pair: nothing but the FP32
+// pipe limits it.  The result is written so that the compiler keeps the arithmetic.
+__global__ void __launch_bounds__(512) fp32_peak_kernel(float* out, int iters, float a, float b) {
+  float x[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) x[i] = (float)(threadIdx.x + i);
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[i] = fmaf(x[i], a, b);
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) s += x[i];
+  if (s == 123.456f) out[blockIdx.x * blockDim.x + threadIdx.x] = s;   // (practically never: the store only keeps the loop alive)
+}
+
+cudaError_t measure_fp32_peak(double* tflops) {
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  float* d = nullptr;
+  const int ctas = sms * 4, iters = 1 << 14;
+  if (e == cudaSuccess) e = cudaMalloc(&d, (size_t)ctas * 512 * sizeof(float));
+  cudaEvent_t a = nullptr, b = nullptr;
+  if (e == cudaSuccess) e = cudaEventCreate(&a);
+  if (e == cudaSuccess) e = cudaEventCreate(&b);
+  double best = 0.0;
+  for (int rep = 0; rep < 5 && e == cudaSuccess; ++rep) {   // the first repetitions also warm the clocks up
+    cudaEventRecord(a);
+    fp32_peak_kernel<<<ctas, 512>>>(d, iters, 0.999f, 0.001f);
+    cudaEventRecord(b);
+    e = cudaEventSynchronize(b);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+    const double fl = 2.0 * 16.0 * iters * 512.0 * ctas;
+    if (e == cudaSuccess && ms > 0.f && fl / (ms * 1e-3) / 1e12 > best) best = fl / (ms * 1e-3) / 1e12;
+  }
+  if (a) cudaEventDestroy(a);
+  if (b) cudaEventDestroy(b);
+  if (d) cudaFree(d);
+  *tflops = best;
+  return e;
+}
+
 cudaError_t prepare_f32_constants() {
   float c[16], s[16], w[16];
   for (int j = 0; j < 16; ++j) {

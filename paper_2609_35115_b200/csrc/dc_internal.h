@@ -118,6 +118,8 @@ void launch_head_istft_f32(const HeadIstftF32& p, cudaStream_t st, int T_grid = 
 // Uploads the constant tables of the head kernel (DFT twiddles, periodic Hann window) to the
 // current device.  Synchronous; called from dc_create, never from a decode call.
 cudaError_t prepare_f32_constants();
+// Measured FP32 fused multiply-add throughput of the current device (TFLOP/s; a few milliseconds of device time).
+cudaError_t measure_fp32_peak(double* tflops);
 
 // ---------------------------------------------------------------------------------------------
 // bf16 flow decoder (dc_flow.cu)
