@@ -119,3 +119,46 @@ def test_injected_allocation_failures_unwind_cleanly(dc, make):
     a = gu.run_gpu_stream(m, s.feats, s.boundaries)
     m.destroy()
     assert np.isfinite(a).all()
+
+
+@pytest.mark.parametrize("make", [lambda: wl.tiny_flow(n_streams=5, n_chunks=6, cfg_scale=0.7),
+                                  lambda: wl.tiny_vocoder(n_streams=5, n_chunks=6, excitation_std=0.2, excitation_seed=5),
+                                  lambda: wl.tiny_token2wav(n_streams=3, n_chunks=6)])
+def test_no_batched_or_wavefront_kernel_writes_outside_a_stream_buffer(dc, make):
+    """The multi-stream launches (slot tables, batched fp32 layers) and the wavefront passes under guard zones."""
+    cfg = make()
+    w = wl.make_workload(cfg)
+    S = cfg.n_streams
+    is_flow = cfg.pipeline in ("flow", "token2wav")
+    F = w.streams[0].feats.shape[0]
+    m = dc.Model(cfg, w.weights, max_batch=max(S, cfg.n_steps if is_flow else 1), max_wave_frames=F if cfg.pipeline == "token2wav" else 0,
+                 options=dc.OPT_GUARD_ZONES)
+    streams = [m.open_stream() for _ in range(S)]
+    feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+    opf = cfg.out_per_frame
+    outs = [torch.zeros(F * opf, device="cuda") for _ in range(S)]
+    for r in range(cfg.n_chunks):
+        idx = [i for i in range(S) if (i + r) % 4 != 3]            # a different subset of the streams every round
+        # (streams that sit a round out fall behind; give every present stream ITS next chunk)
+        fs, os_ = [], []
+        for i in idx:
+            k = getattr(streams[i], "_next", 0)
+            lo, hi = w.streams[i].boundaries[k], w.streams[i].boundaries[k + 1]
+            fs.append(feats[i][lo:hi])
+            os_.append(outs[i][lo * opf:hi * opf])
+            streams[i]._next = k + 1
+        dc.decode_batch(m, [streams[i] for i in idx], fs, os_)
+    torch.cuda.synchronize()
+    assert all(st.check_guards() == 0 for st in streams)
+    if is_flow:                                                     # ... and one wavefront call over a stream's remaining input
+        st = streams[0]
+        k = st._next
+        lo = w.streams[0].boundaries[k]
+        if lo < F:
+            st.decode_wavefront(feats[0][lo:].contiguous())
+            torch.cuda.synchronize()
+            assert st.check_guards() == 0
+    assert m.counters()[4] == 0
+    for st in streams:
+        st.close()
+    m.destroy()
