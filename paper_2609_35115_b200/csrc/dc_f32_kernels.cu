@@ -180,7 +180,9 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
     for (int k4 = 0; k4 < BK; k4 += 4) {
       float4 a[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4*>(As + (ty * 4 + i) * LDA + k4);
+      // (a thread's four rows are ty, ty + BM/4, ...: the four consecutive ty of a warp then read rows LDA = 36 words
+      // apart, i.e. four different bank quads - with rows 4 ty + i two of them would share their banks)
+      for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4*>(As + (ty + (BM / 4) * i) * LDA + k4);
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) {
         const float4 b = *reinterpret_cast<const float4*>(Bs + (k4 + kk) * BN + tx * 4);
@@ -222,7 +224,7 @@ __global__ void __launch_bounds__(512) tapconv_f32_kernel(const TapConvF32 p, co
     const float4 bias = *reinterpret_cast<const float4*>(p.bias + n);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const int row = m0 + ty * 4 + i;
+      const int row = m0 + ty + (BM / 4) * i;
       if (row >= T_in) continue;
       const long long t_in = pos_in + row;
       float4 v = make_float4(acc[i][0] + bias.x, acc[i][1] + bias.y, acc[i][2] + bias.z, acc[i][3] + bias.w);
