@@ -246,6 +246,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--repeats", type=int, default=5,
                     help="runs of history + warm-up + K timed steps, each on freshly opened streams (median reported; 1 for profiler captures)")
+    ap.add_argument("--cta-pairs", action="store_true",
+                    help="flow decoder: conv and QKV GEMMs of full batches on pairs of SMs (DC_OPT_CTA_PAIRS; same bytes, measured slower)")
     ap.add_argument("--history", type=int, default=None,
                     help="untimed chunks decoded per stream before warm-up (default: enough to fill the K/V carry)")
     args = ap.parse_args()
@@ -279,7 +281,8 @@ def main():
     rounds = history + W + K
     rng = np.random.default_rng(cfg.seed + 1000 * rank)
     weights = wl.make_weights(cfg, np.random.default_rng(cfg.seed))
-    model = dc.Model(cfg, weights, max_batch=S)
+    base_options = dc.OPT_CTA_PAIRS if args.cta_pairs else 0
+    model = dc.Model(cfg, weights, max_batch=S, options=base_options)
     feats_h = torch.from_numpy(rng.standard_normal((rounds, S, Tp, cfg.in_dim), dtype=np.float32))
     feats_d = feats_h.cuda()
     out_all = torch.empty(K, S, T * cfg.out_per_frame, device="cuda")     # every timed step's output, hashed after the run
@@ -472,9 +475,9 @@ def main():
                for k in ms if nl[k]}
     dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
     avg_s = 1e-3 * ms[dom] / nl[dom]
-    if dom in ("gemm_conv",):
-        fl = flops_per_launch(cfg, dom, S)
-        roof = {"kernel": "flow_gemm_kernel (conv blocks)", "bound": "tensor", "achieved": fl / avg_s / 1e12,
+    if dom in ("gemm_conv", "gemm_pair"):   # (a paired launch is a conv block or a QKV projection: the same FLOPs)
+        fl = flops_per_launch(cfg, "gemm_conv", S)
+        roof = {"kernel": "flow_gemm_kernel (conv blocks)" if dom == "gemm_conv" else "flow_gemm_kernel<PAIR> (conv blocks and QKV projections on CTA pairs)", "bound": "tensor", "achieved": fl / avg_s / 1e12,
                 "peak": tensor_peak, "unit": "TFLOP/s", "peak_kind": tensor_kind,
                 "frac_of_sustained_peak": fl / avg_s / 1e12 / pk["bf16_tflops_sustained"]}
     elif dom == "attention":
@@ -506,7 +509,7 @@ def main():
     # of everything else is not).
     if has_flow and world == 1:
         def step_ms_without(bits: int) -> float:
-            m2 = dc.Model(cfg, weights, max_batch=S, options=bits)
+            m2 = dc.Model(cfg, weights, max_batch=S, options=bits | base_options)
             st2 = [m2.open_stream() for _ in range(S)]
             def step2(r):
                 if batched:
@@ -574,7 +577,7 @@ def main():
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": ("bf16+f32" if cfg.pipeline == "token2wav" else "bf16" if cfg.precision == "bf16" else "f32"), "data": "synthetic",
             "config": {"workload": describe(cfg), "streams_per_gpu": S, "frames_per_chunk": T,
-                       "history_chunks": history, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                       "history_chunks": history, "cta_pairs": bool(args.cta_pairs), "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": (f"K/V carries {ws:.0f} MB > 126 MB L2, streamed from HBM every step" if ws > 126 else
                               "working set fits L2: value and latency_us are back-to-back chunks (warm L2), latency_us_cold_l2 flushes L2 before every step"),
                        "inputs": "N(0,1) features, N(0,1/fan_in) weights, seeded"

@@ -64,7 +64,7 @@ typedef enum dc_status {
 enum { DC_PIPE_CONV = 1, DC_PIPE_FLOW = 2, DC_PIPE_VOCODER = 3, DC_PIPE_TOKEN2WAV = 4 };
 enum { DC_F32 = 0, DC_BF16 = 1 };   /* DC_BF16: bf16 storage and operands, fp32 accumulation */
 
-/* dc_config.options: switches for tests and measurements.  None of the first four changes a result
+/* dc_config.options: switches for tests and measurements.  None of the first four (nor DC_OPT_CTA_PAIRS) changes a result
  * byte; DC_OPT_ROUNDED_NORM selects the other of two admissible roundings.  (There is no configuration
  * by environment variable.) */
 enum {
@@ -84,6 +84,12 @@ enum {
    * patterns back.  An index error in a kernel that writes just outside a carry is then reported instead of
    * silently corrupting a neighbour. */
   DC_OPT_GUARD_ZONES = 32,
+  /* Flow decoder: full batches run the conv and QKV GEMMs of two adjacent row tiles as ONE 256-row product on
+   * a pair of SMs (tcgen05 cta_group::2; each CTA stages half of the weight tile).  The results are the same
+   * bytes either way.  Off by default: on this part the pair's fixed costs (cluster barrier before the odd
+   * CTA's first copy, pair allocation of tensor memory) exceed what the shorter main loop saves for the
+   * 7-microsecond kernels of this decoder. */
+  DC_OPT_CTA_PAIRS = 64,
   /* MEASUREMENT ONLY - the outputs of such a model are meaningless: the step without the kernels of
    * one class, so that step-time differences give that class's cost inside the captured graph. */
   DC_OPT_SKIP_CONV_GEMM = 1 << 16,
@@ -311,7 +317,8 @@ dc_status dc_decode_batch_host(dc_model* model, int n, dc_stream* const* streams
  * class, the summed milliseconds and the launch count.  Classes: 0 conv GEMM, 1 other GEMMs
  * (input/QKV/output projections), 2 attention, 3 unused (the RMS norm is folded into the GEMMs),
  * 4 slot table + input prep,
- * 5 fp32 tap convolution, 6 fp32 head + inverse STFT.
+ * 5 fp32 tap convolution, 6 fp32 head + inverse STFT, 7 conv / QKV GEMMs launched as CTA pairs
+ * (DC_OPT_CTA_PAIRS; they then do not count in classes 0 and 1).
  * max_launches bounds the event pool allocated by dc_profile_begin. */
 dc_status dc_profile_begin(dc_model* model, int max_launches);
 dc_status dc_profile_end(dc_model* model, double ms[8], uint64_t launches[8]);

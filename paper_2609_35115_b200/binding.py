@@ -96,6 +96,7 @@ def load_library():
 
 
 OPT_NO_GRAPH, OPT_NO_PDL, OPT_NO_ZEROCOPY, OPT_SERIAL_TAILS, OPT_ROUNDED_NORM, OPT_GUARD_ZONES = 1, 2, 4, 8, 16, 32
+OPT_CTA_PAIRS = 64
 OPT_SKIP_CONV_GEMM, OPT_SKIP_ATTENTION, OPT_EMPTY_KERNELS = 1 << 16, 1 << 17, 1 << 18     # measurement only: outputs are meaningless
 
 
@@ -190,7 +191,7 @@ class Model:
         ms = (C.c_double * 8)()
         n = (C.c_uint64 * 8)()
         _check(self.lib.dc_profile_end(self.handle, ms, n), "dc_profile_end")
-        names = ["gemm_conv", "gemm_proj", "attention", "rmsnorm", "prep", "tapconv_f32", "head_istft_f32"]
+        names = ["gemm_conv", "gemm_proj", "attention", "rmsnorm", "prep", "tapconv_f32", "head_istft_f32", "gemm_pair"]
         return ({k: ms[i] for i, k in enumerate(names)}, {k: n[i] for i, k in enumerate(names)})
 
     def destroy(self):

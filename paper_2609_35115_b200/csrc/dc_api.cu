@@ -235,7 +235,7 @@ static bool config_ok(const dc_config* c, const char** why) {
   if (c->f_prompt != 0 && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("f_prompt belongs to the flow decoder");
   if (c->cfg_scale != 0.f && c->pipeline != DC_PIPE_FLOW && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("cfg_scale belongs to the flow decoder");
   if (c->options & ~(uint32_t)(DC_OPT_NO_GRAPH | DC_OPT_NO_PDL | DC_OPT_NO_ZEROCOPY | DC_OPT_SERIAL_TAILS | DC_OPT_ROUNDED_NORM | DC_OPT_SKIP_CONV_GEMM |
-                               DC_OPT_SKIP_ATTENTION | DC_OPT_EMPTY_KERNELS | DC_OPT_GUARD_ZONES))
+                               DC_OPT_SKIP_ATTENTION | DC_OPT_EMPTY_KERNELS | DC_OPT_GUARD_ZONES | DC_OPT_CTA_PAIRS))
     BAD("unknown option bit");
   if (!(c->excitation_std >= 0.f && c->excitation_std <= 1e6f)) BAD("excitation_std out of range");
   if (c->excitation_std > 0.f && c->pipeline != DC_PIPE_VOCODER && c->pipeline != DC_PIPE_TOKEN2WAV) BAD("excitation_std belongs to the vocoder tail");

@@ -149,6 +149,17 @@ __device__ __forceinline__ void store16(bf16* p, const uint4& a, const uint4& b)
   *reinterpret_cast<uint4*>(p + 8) = b;
 }
 
+// PAIR: the CTAs of two adjacent row tiles (a cluster of two along x, one TPC) run ONE 256-row UMMA per
+// reduction step.  Each stages its own activation rows and only HALF of the weight tile (tmB then has boxes
+// of BN / 2 rows), so a CTA draws 28 KB instead of 40 KB per reduction block from L2 and the whole weight
+// panel of a C = 512 layer fits its shared memory ahead of the activations.  The even CTA issues for both;
+// accumulators, epilogue and summation order are those of the single-CTA form, so the results are the same bits.
+// Measured on the 32-stream serving workload: the main loop of a conv block drops from 3.9 k to 3.3 k cycles
+// (400 per reduction block, the tensor pipe's own rate), but the odd CTA may not copy before the cluster barrier
+// has told it that the even CTA's barriers exist, and that barrier, with the pair allocation of tensor memory,
+// puts the first full stage 0.4 to 1.6 microseconds later - more than the loop saves in a 7-microsecond kernel.
+// Hence an option (DC_OPT_CTA_PAIRS), off by default.
+template <bool PAIR>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -161,7 +172,8 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // stage = [A tile 128 x 128 B | one B tile BN x 128 B per tap]; all tile sizes are multiples of
   // 1024 B.  The weight tiles of a conv block's three taps are adjacent, so that they form one
   // operand of 3 BN rows.
-  const uint32_t b_bytes = (uint32_t)p.BN * 128u;
+  // (PAIR: a "tile" is one of the CTA's `taps` units of BN / 2 weight rows; BN is then a multiple of 16)
+  const uint32_t b_bytes = PAIR ? (uint32_t)p.BN * 64u : (uint32_t)p.BN * 128u;
   const uint32_t b_tile = (b_bytes + 1023u) & ~1023u;
   const uint32_t stage_bytes = (uint32_t)A_BYTES + (uint32_t)p.taps * b_tile;
   const int STAGES = p.n_stages;
@@ -175,6 +187,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * TILE_M, n0 = blockIdx.y * p.BN;
+  const uint32_t pair_rank = PAIR ? ptx::cluster_ctarank() : 0u;   // 0: issues the UMMAs and owns the "full" barriers
   // Accumulator: BN columns, or 3 BN for a conv block, whose three taps are the column blocks of ONE
   // product Z = X [W_0 | W_1 | W_2] (a row shift commutes with the product, so the taps are shifted
   // and added in the epilogue; a tcgen05.mma costs about 47 cycles however small it is, and one
@@ -194,7 +207,15 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     *s_fail = 0;
     ptx::fence_barrier_init();
   }
-  if (warp == 1) ptx::tmem_alloc(tmem_slot, tmem_cols);
+  if (warp == 1) {
+    if (PAIR) ptx::tmem_alloc_pair(tmem_slot, tmem_cols);
+    else ptx::tmem_alloc(tmem_slot, tmem_cols);
+  }
+  // PAIR: the CTAs signal each other's barriers and the even one writes both accumulators, so each must know
+  // that the other's barriers and tensor memory exist.  Every thread arrives at the cluster barrier here
+  // (thread 0 after the initialisation, warp 1 after the allocation) and waits only where it first depends
+  // on the partner, which keeps most of the barrier's latency off the path to the first copy.
+  if (PAIR) ptx::cluster_arrive();
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -210,11 +231,24 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const bool is_a = warp == 0;
       const int nkb = p.n_kblocks, taps = p.taps;
       const int ya = GUARD + m0;
-      const uint32_t tx_bytes = is_a ? (uint32_t)A_BYTES : (uint32_t)taps * b_bytes;
+      // PAIR: the even CTA's barrier counts the bytes of both CTAs' copies; the odd CTA only issues its own
+      const uint32_t tx_bytes = (is_a ? (uint32_t)A_BYTES : (uint32_t)taps * b_bytes) * (PAIR ? 2u : 1u);
       uint8_t* dst = smem + (is_a ? 0 : A_BYTES);
+      // PAIR: this CTA's j-th weight unit is unit u = taps * rank + j of the 2 * taps half-tiles: tap u / 2, half u % 2
+      int ux[3] = {0, 0, 0}, uy[3] = {0, 0, 0};
+      if (PAIR) {
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+          const int u = taps * (int)pair_rank + j;
+          ux[j] = (u >> 1) * nkb * KBLK;
+          uy[j] = n0 + (u & 1) * (p.BN >> 1);
+        }
+      }
+      const uint32_t full0 = PAIR ? ptx::map_to_cta(ptx::smem_u32(&full[0]), 0u) : 0u;
       int st = 0;
       uint32_t phase = 1;          // parity of the "empty" phase to wait for (first pass: no wait)
       int x = 0;
+      if (PAIR && pair_rank != 0) ptx::cluster_wait();   // this CTA's copies count on its partner's barriers
       if (is_a) ptx::pdl_wait();   // activations come from the previous kernel; weights do not
       for (int kb = 0; kb < nkb; ++kb) {
         if (kb >= STAGES && !ptx::mbar_wait(&empty[st], phase)) {
@@ -222,10 +256,23 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           *s_fail = 1;
           break;
         }
-        ptx::mbar_expect_tx_if(on, &full[st], tx_bytes);
-        if (is_a) {
+        if (PAIR) {
+          ptx::mbar_expect_tx_if(on && pair_rank == 0, &full[st], tx_bytes);
+          const uint32_t bar = full0 + (uint32_t)st * 8u;
+          if (is_a) {
+            ptx::tma_load_2d_pair_if(on, dst, &tmA, x, ya, bar);
+          } else {
+            ptx::tma_load_2d_pair_if(on, dst, &tmB, x + ux[0], uy[0], bar);
+            if (taps == 3) {
+              ptx::tma_load_2d_pair_if(on, dst + b_tile, &tmB, x + ux[1], uy[1], bar);
+              ptx::tma_load_2d_pair_if(on, dst + 2 * b_tile, &tmB, x + ux[2], uy[2], bar);
+            }
+          }
+        } else if (is_a) {
+          ptx::mbar_expect_tx_if(on, &full[st], tx_bytes);
           ptx::tma_load_2d_if(on, dst, &tmA, x, ya, &full[st]);
         } else {
+          ptx::mbar_expect_tx_if(on, &full[st], tx_bytes);
           ptx::tma_load_2d_if(on, dst, &tmB, x, n0, &full[st]);
           if (taps == 3) {
             ptx::tma_load_2d_if(on, dst + b_tile, &tmB, x + nkb * KBLK, n0, &full[st]);
@@ -246,17 +293,20 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // narrow UMMA takes to execute, so two warps issue alternate reduction blocks into accumulators
     // of their own; the epilogue adds the two in a fixed order.
     const int me = warp >> 1;                     // 0 or 1
-    if (me < p.n_issuers) {
+    if (me < p.n_issuers && pair_rank == 0) {
       const uint32_t on = lane == 0;
       // the weight tiles of the taps are adjacent in the stage (BN rows of 128 B each, BN a multiple of 8),
       // so together they are one K-major operand of taps * BN rows
-      const uint32_t idesc = ptx::umma_idesc_bf16(TILE_M, p.taps * p.BN, 0, 0);
+      const uint32_t idesc = ptx::umma_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, p.taps * p.BN, 0, 0);
+      // PAIR: every completion is reported to both CTAs (their producers and epilogues wait on barriers of their own)
+      const uint32_t empty_mine = ptx::smem_u32(&empty[0]), empty_peer = PAIR ? ptx::map_to_cta(empty_mine, 1u) : 0u;
       const int nkb = p.n_kblocks, step = p.n_issuers;
       const uint32_t d_acc = tmem_base + (uint32_t)me * acc2_off;
       // descriptor start addresses are in 16-byte units: +2 per 32-byte K step
       const uint64_t d_a0 = ptx::umma_desc_sw128(ptx::smem_u32(smem));
       const uint32_t stage16 = stage_bytes >> 4, ab16 = A_BYTES >> 4;
       uint32_t acc = 0;
+      if (PAIR) ptx::cluster_wait();   // the partner's tensor memory and barriers
       for (int kb = me; kb < nkb; kb += step) {
         const int st = kb % STAGES;
         if (!ptx::mbar_wait(&full[st], (uint32_t)(kb / STAGES) & 1u)) {
@@ -266,13 +316,27 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         ptx::tc_fence_after();
         const uint64_t da = d_a0 + (uint64_t)((uint32_t)st * stage16), db = da + ab16;
-        ptx::umma_bf16_if(on, d_acc, da, db, idesc, acc);
+        if (PAIR) {
+          ptx::umma_bf16_pair_if(on, d_acc, da, db, idesc, acc);
 #pragma unroll
-        for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + 2 * k, db + 2 * k, idesc, 1);
+          for (int k = 1; k < 4; ++k) ptx::umma_bf16_pair_if(on, d_acc, da + 2 * k, db + 2 * k, idesc, 1);
+          ptx::umma_commit_pair_if(on, empty_mine + (uint32_t)st * 8u);
+          ptx::umma_commit_pair_if(on, empty_peer + (uint32_t)st * 8u);
+        } else {
+          ptx::umma_bf16_if(on, d_acc, da, db, idesc, acc);
+#pragma unroll
+          for (int k = 1; k < 4; ++k) ptx::umma_bf16_if(on, d_acc, da + 2 * k, db + 2 * k, idesc, 1);
+          ptx::umma_commit_if(on, &empty[st]);
+        }
         acc = 1;
-        ptx::umma_commit_if(on, &empty[st]);
       }
-      ptx::umma_commit_if(on, accum);   // arrives when every UMMA above has finished (also on the failure path)
+      // arrives when every UMMA above has finished (also on the failure path)
+      if (PAIR) {
+        ptx::umma_commit_pair_if(on, ptx::smem_u32(accum));
+        ptx::umma_commit_pair_if(on, ptx::map_to_cta(ptx::smem_u32(accum), 1u));
+      } else {
+        ptx::umma_commit_if(on, accum);
+      }
     }
   } else {
     // ---------------- epilogue: 4 EPI_GROUPS warps; a thread owns one output row and every EPI_GROUPS-th 16-column chunk ----------------
@@ -334,6 +398,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     ptx::named_bar_sync(1, EPI_THREADS);
 
     const bool got = ptx::mbar_wait_relaxed(accum, 0);
+    if (PAIR) ptx::cluster_wait();   // (long complete; a thread waits once between its two arrivals)
     ptx::tc_fence_after();
     if (!got) atomicCAS(p.err, 0, 3 | (p.mode << 8));
     const bool slot_ok = in_range && got && *s_fail == 0;
@@ -343,6 +408,10 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int new_row = rho - si.Tc;              // carry row this thread's value moves to (the carry follows the committed frames)
     const bool carry_wr = do_halo && (is_halo || is_chunk) && new_row >= 0 && new_row < HALO;
 
+    // PAIR: tensor memory is freed for both CTAs at once, so each thread reports its LAST accumulator load
+    // to the cluster barrier as soon as it has happened; the barrier's latency (about 1500 cycles) then runs
+    // under the arithmetic and the stores that follow, and the freeing warp finds it complete.
+    const int last_kk = (p.BN - 16 * cg - 1) / (16 * EPI_GROUPS);   // (BN > 16 cg for every chunk group of a paired GEMM)
 #pragma unroll
     for (int kk = 0; kk < MAX_BN / (16 * EPI_GROUPS); ++kk) {
       const int ch = EPI_GROUPS * kk + cg;
@@ -402,6 +471,10 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
 #pragma unroll
         for (int i = 0; i < 16; ++i) acc[i] += z[i];
+      }
+      if (PAIR && kk == last_kk) {
+        ptx::tc_fence_before();
+        ptx::cluster_arrive();
       }
       const int n = n0 + c0;
 #pragma unroll
@@ -518,9 +591,24 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (carry_wr) store16(carry + new_row * p.C + n, va, vb);
     }
   }
-  ptx::tc_fence_before();
-  __syncthreads();
-  if (warp == 1) ptx::tmem_dealloc(tmem_base, tmem_cols);
+  if (PAIR) {
+    // Nothing of a CTA is touched by its partner after its own waits have returned (its copies count on the
+    // even CTA's barriers, which that CTA waits for; the UMMAs that read its shared memory are complete when
+    // its accumulator barrier fires), so a CTA may leave as soon as tensor memory can be freed: when every
+    // thread of the pair has arrived, the epilogue threads having done so after their last accumulator load.
+    // (warps that have not waited on the first phase yet do so now)
+    if (warp < 4 && !(((warp & 1) == 0 && pair_rank != 0) || ((warp & 1) == 1 && (warp >> 1) < p.n_issuers && pair_rank == 0))) ptx::cluster_wait();
+    if (warp < 4) ptx::cluster_arrive();
+    if (warp == 1) {
+      ptx::cluster_wait();
+      ptx::tc_fence_after();
+      ptx::tmem_dealloc_pair(tmem_base, tmem_cols);
+    }
+  } else {
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) ptx::tmem_dealloc(tmem_base, tmem_cols);
+  }
 }
 
 // ---- small kernels ---------------------------------------------------------------------------
@@ -1024,6 +1112,7 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, u
 
 constexpr size_t GEMM_SMEM_EXTRA = 1024 + 2 * MAX_STAGES * 8 + 8 + 8 + 2 * MAX_BN * 4 + 64;   // alignment slack + barriers + constants
 constexpr size_t GEMM_SMEM_MAX = 200 * 1024;
+constexpr size_t GEMM_SMEM_MAX_PAIR = 227 * 1024;   // the opt-in limit of the device: eight 28 KB stages of a CTA pair
 
 }  // namespace
 
@@ -1237,7 +1326,9 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   if (e == cudaSuccess) chk(cudaMemcpy(m->wts, hw.data(), wn * sizeof(uint16_t), cudaMemcpyHostToDevice));
   if (e == cudaSuccess) chk(cudaMemcpy(m->fconst, hf.data(), fn * sizeof(float), cudaMemcpyHostToDevice));
   if (e == cudaSuccess)
-    chk(cudaFuncSetAttribute(flow_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
+    chk(cudaFuncSetAttribute(flow_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
+  if (e == cudaSuccess)
+    chk(cudaFuncSetAttribute(flow_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX_PAIR));
   if (e == cudaSuccess && cfg.n_attn > 0)
     chk(cudaFuncSetAttribute(m->P > 0 ? flow_attn_kernel<true> : flow_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)ATT_SMEM));
@@ -1392,6 +1483,7 @@ struct LaunchCtx {
   Profiler*    prof;
   int          launches = 0;
   cudaError_t  err = cudaSuccess;
+  int          cluster_x = 1;   // > 1: the next launch is a cluster launch of that many CTAs along x
 };
 
 template <typename... KArgs, typename... Args>
@@ -1402,12 +1494,20 @@ void launch(LaunchCtx& lc, void (*kernel)(KArgs...), dim3 grid, dim3 block, size
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = lc.st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
+  cfg.attrs = attr;
   if (lc.pdl && pdl_ok) {
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+    ++cfg.numAttrs;
+  }
+  if (lc.cluster_x > 1) {   // set by the caller for this one launch
+    attr[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
+    attr[cfg.numAttrs].val.clusterDim.x = (unsigned)lc.cluster_x;
+    attr[cfg.numAttrs].val.clusterDim.y = 1;
+    attr[cfg.numAttrs].val.clusterDim.z = 1;
+    ++cfg.numAttrs;
+    lc.cluster_x = 1;
   }
   cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
   if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
@@ -1435,7 +1535,10 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
   // the output projection always uses 16-column tiles: mel/16 CTAs per row tile instead of one, and a
   // single Euler-state round trip per epilogue thread
   const int bn = 64 >> v, bq = 192 >> v, bo = 16;
-  auto gemm = [&](const CUtensorMap& tA, const CUtensorMap& tB, GemmParams& p, int N) {
+  // CTA pairs (DC_OPT_CTA_PAIRS): full batches only (the widest tiles, an even number of row tiles), and only the
+  // GEMMs whose weight tile is a large part of a stage; tBh is the same weight matrix with boxes of BN / 2 rows
+  const bool pairs_ok = v == 0 && m_tiles % 2 == 0 && (c.options & DC_OPT_CTA_PAIRS);
+  auto gemm = [&](const CUtensorMap& tA, const CUtensorMap& tB, GemmParams& p, int N, const CUtensorMap* tBh = nullptr) {
     p.n_slots = n;
     p.slots = m->d_slots;
     p.ld = C;
@@ -1460,8 +1563,22 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       // the wide QKV tiles fill the GPU with one CTA per SM anyway: a deeper ring hides the load latency
       if (p.mode == MODE_QKV && stage_bytes > 32 * 1024 && p.n_kblocks >= 4) p.n_stages = 4;
     }
+    if (pairs_ok && tBh != nullptr) {
+      const int pair_stage = A_BYTES + p.taps * (p.BN * 64);
+      int ns = p.n_kblocks < MAX_STAGES ? p.n_kblocks : MAX_STAGES;
+      while (ns > 1 && GEMM_SMEM_EXTRA + (size_t)ns * pair_stage > GEMM_SMEM_MAX_PAIR) --ns;
+      if (p.n_issuers == 2) ns &= ~1;
+      // the conv epilogue exchanges shifted rows through 64 KB of the (by then idle) ring
+      if (ns >= 2 && (size_t)ns * pair_stage >= 64 * 1024) {
+        p.n_stages = ns;
+        lc.cluster_x = 2;
+        launch(lc, flow_gemm_kernel<true>, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), GEMM_SMEM_EXTRA + (size_t)ns * pair_stage, true,
+               7, tA, *tBh, p);
+        return;
+      }
+    }
     const size_t smem = GEMM_SMEM_EXTRA + (size_t)p.n_stages * stage_bytes;
-    launch(lc, flow_gemm_kernel, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), smem, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
+    launch(lc, flow_gemm_kernel<false>, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), smem, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
   };
   // the GEMM whose output feeds an RMS norm leaves the row statistics; the GEMM after the norm applies them
   auto feeds_norm = [&](GemmParams& p) { p.ssq_out = m->ssq; p.ssq_ld = m->rows; };
@@ -1516,7 +1633,7 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
         const bool next_is_conv = (j + 1 < m->cpa);
         p.halo_off = next_is_conv ? ((long long)s * c.n_conv + l + 1) * halo_stride : -1;
         if (!next_is_conv) feeds_norm(p);   // the group's attention norm, or the final norm of a conv-only stack
-        if (!(c.options & DC_OPT_SKIP_CONV_GEMM)) gemm(*tX, m->tmWconv[v][l], p, C);   // (measurement only: the step without this class)
+        if (!(c.options & DC_OPT_SKIP_CONV_GEMM)) gemm(*tX, m->tmWconv[v][l], p, C, &m->tmWconv[1][l]);   // (measurement only: the step without this class)
         swap();
       }
       if (c.n_attn > 0) {
@@ -1528,10 +1645,10 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
           p.kv_rs = m->kv_rs; p.kv_hs = m->kv_hs; p.dh_shift = m->dh_shift;
           if (rounded_norm) {
             rmsnorm(X);
-            gemm(m->tmU, m->tmWqkv[v][g], p, 3 * C);
+            gemm(m->tmU, m->tmWqkv[v][g], p, 3 * C, &m->tmWqkv[1][g]);
           } else {
             normalised(p);
-            gemm(*tX, m->tmWqkv[v][g], p, 3 * C);
+            gemm(*tX, m->tmWqkv[v][g], p, 3 * C, &m->tmWqkv[1][g]);
           }
         }
         if (!(c.options & DC_OPT_SKIP_ATTENTION)) attention(s, g);   // (measurement only: the step without this class)

@@ -220,6 +220,65 @@ __device__ __forceinline__ void umma_commit_if(uint32_t on, uint64_t* bar) {
       : "memory");
 }
 
+// ---- CTA pairs (cta_group::2) --------------------------------------------------------------------
+// Two CTAs of a cluster, on the two SMs of one TPC, execute one UMMA of 256 rows: each supplies its own
+// 128 rows of A and HALF of the B rows (same shared-memory offsets in both), and each receives the
+// accumulator of its own 128 rows, all N columns, in its own tensor memory.  Only the CTA of even
+// cluster rank issues; barriers of the other are reached through shared::cluster addresses.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in the CTA of cluster rank `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+// The hardware barrier over every thread of the cluster (not a spin on memory: it cannot outlive the CTAs),
+// in its two halves, for a thread that has something to do in between - or nothing to wait for: a thread
+// may arrive and exit, the barrier waits only for threads that have not exited.  A thread waits exactly
+// once between two arrivals.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+// both CTAs of the pair execute these with the same warp and the same shared-memory slot offset
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* slot, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// tile load whose completion bytes are counted on a barrier given as a shared::cluster address (the
+// issuing CTA's own or its pair partner's); the data lands in the issuing CTA's shared memory
+__device__ __forceinline__ void tma_load_2d_pair_if(uint32_t on, void* dst, const CUtensorMap* m, int x, int y, uint32_t bar_cluster) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n"
+      "@q cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n}\n"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(bar_cluster), "r"(on)
+      : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B over the pair; M = 256 in the instruction descriptor
+__device__ __forceinline__ void umma_bf16_pair_if(uint32_t on, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t accumulate) {
+  const uint32_t z = 0;   // no output lane is disabled
+  asm volatile(
+      "{\n.reg .pred p, q;\nsetp.ne.b32 p, %4, 0;\nsetp.ne.b32 q, %5, 0;\n"
+      "@q tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%6, %6, %6, %6, %6, %6, %6, %6}, p;\n}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(on), "r"(z)
+      : "memory");
+}
+// the barrier at a shared::cluster address receives one arrival once every pair UMMA issued so far
+// by this thread has completed
+__device__ __forceinline__ void umma_commit_pair_if(uint32_t on, uint32_t bar_cluster) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
+      "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}\n" ::"r"(bar_cluster),
+      "r"(on)
+      : "memory");
+}
+
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }

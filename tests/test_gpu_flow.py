@@ -393,3 +393,56 @@ def test_rounded_norm_option_matches_oracle_and_batching(dc):
     folded = gu.run_gpu_stream(m0, w.streams[0].feats, w.streams[0].boundaries)
     m0.destroy()
     assert not np.array_equal(folded, single[0]) and gu.rel_err(folded, single[0].astype(np.float64)) <= TOL_BF16
+
+
+def test_cta_pairs_option_same_bytes_as_single_ctas(dc):
+    """DC_OPT_CTA_PAIRS: the conv and QKV GEMMs of a full batch as 256-row products on pairs of SMs
+    (tcgen05 cta_group::2, each CTA staging half of the weight tile).  Same accumulators, same summation
+    order: the bytes must be those of the default single-CTA launches, ragged chunks and carried state
+    included; the profile classes prove that the paired kernels are what ran."""
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS["cfg5"], name="cfg5_pairs", n_streams=24, n_chunks=6)
+    w = wl.make_workload(cfg)
+    S = cfg.n_streams
+    feats = [torch.from_numpy(s.feats).cuda() for s in w.streams]
+
+    def run(options, profiled_round=None):
+        m = dc.Model(cfg, w.weights, max_batch=S, options=options)
+        streams = [m.open_stream() for _ in range(S)]
+        outs = [torch.zeros(s.feats.shape[0], cfg.mel_dim, device="cuda") for s in w.streams]
+        launches = None
+        for r in range(cfg.n_chunks):
+            fs = [feats[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
+            os_ = [outs[i][w.streams[i].boundaries[r]:w.streams[i].boundaries[r + 1]] for i in range(S)]
+            if r == profiled_round:
+                m.profile_begin()
+            dc.decode_batch(m, streams, fs, os_)
+            if r == profiled_round:
+                launches = m.profile_end()[1]
+        torch.cuda.synchronize()
+        assert m.counters()[4] == 0, "a bounded device-side wait timed out"
+        for st in streams:
+            st.close()
+        m.destroy()
+        return [o.cpu().numpy() for o in outs], launches
+
+    base, n_base = run(0, profiled_round=2)
+    pairs, n_pairs = run(dc.OPT_CTA_PAIRS, profiled_round=2)
+    per_step = len(cfg.dilations) + cfg.n_attn_layers
+    assert n_base["gemm_pair"] == 0 and n_pairs["gemm_pair"] == cfg.n_steps * per_step
+    assert n_pairs["gemm_conv"] == 0
+    assert all(np.isfinite(p).all() for p in pairs)
+    for i in range(S):
+        assert np.array_equal(base[i], pairs[i]), f"stream {i}"
+    # ... and a batch with an odd number of row tiles falls back to single CTAs
+    cfg_odd = dataclasses.replace(cfg, name="cfg5_pairs_odd", n_streams=22)
+    m = dc.Model(cfg_odd, w.weights, max_batch=22, options=dc.OPT_CTA_PAIRS)
+    streams = [m.open_stream() for _ in range(22)]
+    outs = [torch.zeros(50, cfg.mel_dim, device="cuda") for _ in range(22)]
+    m.profile_begin()
+    dc.decode_batch(m, streams, [feats[i][:50] for i in range(22)], outs)
+    n_odd = m.profile_end()[1]
+    assert n_odd["gemm_pair"] == 0 and n_odd["gemm_conv"] == cfg.n_steps * len(cfg.dilations)
+    for st in streams:
+        st.close()
+    m.destroy()
