@@ -159,10 +159,15 @@ __device__ __forceinline__ void store16(bf16* p, const uint4& a, const uint4& b)
 // has told it that the even CTA's barriers exist, and that barrier, with the pair allocation of tensor memory,
 // puts the first full stage 0.4 to 1.6 microseconds later - more than the loop saves in a 7-microsecond kernel.
 // Hence an option (DC_OPT_CTA_PAIRS), off by default.
-template <bool PAIR>
+template <bool PAIR, int MODE_T>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
+  // MODE_T >= 0: a kernel specialised for one role, so that the other roles' epilogues and the slot fields only they
+  // use cost neither registers nor instructions
+  const int mode = MODE_T >= 0 ? MODE_T : p.mode;
+  const int n_taps = MODE_T == MODE_CONV ? 3 : (MODE_T >= 0 ? 1 : p.taps);
+  const int n_iss = MODE_T == MODE_CONV ? 2 : p.n_issuers;
   if (p.empty) {
     ptx::pdl_launch();
     ptx::pdl_wait();
@@ -175,7 +180,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // (PAIR: a "tile" is one of the CTA's `taps` units of BN / 2 weight rows; BN is then a multiple of 16)
   const uint32_t b_bytes = PAIR ? (uint32_t)p.BN * 64u : (uint32_t)p.BN * 128u;
   const uint32_t b_tile = (b_bytes + 1023u) & ~1023u;
-  const uint32_t stage_bytes = (uint32_t)A_BYTES + (uint32_t)p.taps * b_tile;
+  const uint32_t stage_bytes = (uint32_t)A_BYTES + (uint32_t)n_taps * b_tile;
   const int STAGES = p.n_stages;
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * stage_bytes);
   uint64_t* empty = full + MAX_STAGES;
@@ -193,9 +198,9 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // and added in the epilogue; a tcgen05.mma costs about 47 cycles however small it is, and one
   // 128 x 3BN x 16 instruction replaces three 128 x BN x 16 ones).  The second issuer's accumulator
   // sits acc2_off columns after the first.
-  const uint32_t acc_w = (uint32_t)(p.taps * p.BN);
+  const uint32_t acc_w = (uint32_t)(n_taps * p.BN);
   const uint32_t acc2_off = acc_w <= 32 ? 32u : (acc_w <= 64 ? 64u : (acc_w <= 128 ? 128u : 256u));
-  const uint32_t need_cols = p.n_issuers == 2 ? 2u * acc2_off : acc_w;
+  const uint32_t need_cols = n_iss == 2 ? 2u * acc2_off : acc_w;
   const uint32_t tmem_cols = need_cols <= 32 ? 32u : (need_cols <= 64 ? 64u : (need_cols <= 128 ? 128u : (need_cols <= 256 ? 256u : 512u)));
 
   if (threadIdx.x == 0) {
@@ -203,7 +208,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ptx::mbar_init(&full[i], 2);   // one arrival per producer thread
       ptx::mbar_init(&empty[i], 1);
     }
-    ptx::mbar_init(accum, (uint32_t)p.n_issuers);
+    ptx::mbar_init(accum, (uint32_t)n_iss);
     *s_fail = 0;
     ptx::fence_barrier_init();
   }
@@ -229,7 +234,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     {
       const uint32_t on = lane == 0;   // the whole warp runs the loop, lane 0 issues
       const bool is_a = warp == 0;
-      const int nkb = p.n_kblocks, taps = p.taps;
+      const int nkb = p.n_kblocks, taps = n_taps;
       const int ya = GUARD + m0;
       // PAIR: the even CTA's barrier counts the bytes of both CTAs' copies; the odd CTA only issues its own
       const uint32_t tx_bytes = (is_a ? (uint32_t)A_BYTES : (uint32_t)taps * b_bytes) * (PAIR ? 2u : 1u);
@@ -252,7 +257,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (is_a) ptx::pdl_wait();   // activations come from the previous kernel; weights do not
       for (int kb = 0; kb < nkb; ++kb) {
         if (kb >= STAGES && !ptx::mbar_wait(&empty[st], phase)) {
-          atomicCAS(p.err, 0, 1 | (is_a ? 0 : 0x10) | (p.mode << 8) | (kb << 12) | ((int)blockIdx.x << 20));
+          atomicCAS(p.err, 0, 1 | (is_a ? 0 : 0x10) | (mode << 8) | (kb << 12) | ((int)blockIdx.x << 20));
           *s_fail = 1;
           break;
         }
@@ -293,14 +298,14 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // narrow UMMA takes to execute, so two warps issue alternate reduction blocks into accumulators
     // of their own; the epilogue adds the two in a fixed order.
     const int me = warp >> 1;                     // 0 or 1
-    if (me < p.n_issuers && pair_rank == 0) {
+    if (me < n_iss && pair_rank == 0) {
       const uint32_t on = lane == 0;
       // the weight tiles of the taps are adjacent in the stage (BN rows of 128 B each, BN a multiple of 8),
       // so together they are one K-major operand of taps * BN rows
-      const uint32_t idesc = ptx::umma_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, p.taps * p.BN, 0, 0);
+      const uint32_t idesc = ptx::umma_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, n_taps * p.BN, 0, 0);
       // PAIR: every completion is reported to both CTAs (their producers and epilogues wait on barriers of their own)
       const uint32_t empty_mine = ptx::smem_u32(&empty[0]), empty_peer = PAIR ? ptx::map_to_cta(empty_mine, 1u) : 0u;
-      const int nkb = p.n_kblocks, step = p.n_issuers;
+      const int nkb = p.n_kblocks, step = n_iss;
       const uint32_t d_acc = tmem_base + (uint32_t)me * acc2_off;
       // descriptor start addresses are in 16-byte units: +2 per 32-byte K step
       const uint64_t d_a0 = ptx::umma_desc_sw128(ptx::smem_u32(smem));
@@ -310,7 +315,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       for (int kb = me; kb < nkb; kb += step) {
         const int st = kb % STAGES;
         if (!ptx::mbar_wait(&full[st], (uint32_t)(kb / STAGES) & 1u)) {
-          atomicCAS(p.err, 0, 2 | (me << 4) | (p.mode << 8) | (kb << 12) | ((int)blockIdx.x << 20));
+          atomicCAS(p.err, 0, 2 | (me << 4) | (mode << 8) | (kb << 12) | ((int)blockIdx.x << 20));
           *s_fail = 1;
           break;
         }
@@ -360,7 +365,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const bool in_range = si.T > 0;               // (a slot without frames - a hole in a wavefront - is left alone)
     const int f = rho - HALO;
     const bool do_halo = p.halo_off >= 0;
-    const bool has_resid = p.mode == MODE_CONV || p.mode == MODE_OPROJ;
+    const bool has_resid = mode == MODE_CONV || mode == MODE_OPROJ;
     const long long grow = (long long)(GUARD + r);
     bf16* carry = do_halo && in_range ? si.halo + p.halo_off : nullptr;
     // pre[2k], pre[2k+1]: the 16 bf16 of this thread's k-th chunk (columns n0 + 16 (EPI_GROUPS k + cg) ..);
@@ -400,7 +405,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const bool got = ptx::mbar_wait_relaxed(accum, 0);
     if (PAIR) ptx::cluster_wait();   // (long complete; a thread waits once between its two arrivals)
     ptx::tc_fence_after();
-    if (!got) atomicCAS(p.err, 0, 3 | (p.mode << 8));
+    if (!got) atomicCAS(p.err, 0, 3 | (mode << 8));
     const bool slot_ok = in_range && got && *s_fail == 0;
     const float* tau_s = s_tau + ((q >> 1) & 1) * 64;   // rows 64.. of the tile are its second slot
     const bool is_halo = slot_ok && rho < HALO;
@@ -418,7 +423,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int c0 = ch * 16;
       if (c0 >= p.BN) break;
       float acc[16];
-      if (p.n_issuers == 2) {   // even blocks + odd blocks, always in this order
+      if (n_iss == 2) {   // even blocks + odd blocks, always in this order
         float acc2[16];
         ptx::tmem_ld16x2(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, tmem_base + ((uint32_t)(q * 32) << 16) + acc2_off + (uint32_t)c0,
                          acc, acc2);
@@ -427,14 +432,14 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       } else {
         ptx::tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, acc);
       }
-      if (p.taps == 3) {
+      if (n_taps == 3) {
         // conv block: acc holds tap 0's product for this row; y[r] = Z_0[r - shift_0] + Z_1[r - shift_1] + Z_2[r].
         // A row is a TMEM lane, which a thread cannot change, so the shifted rows go through shared memory
         // (the operand stages are idle by now).  Shifts never leave the slot for the rows that are
         // stored (<= 8 left-context rows precede the chunk).
         float z[16];
         const uint32_t lanes = tmem_base + ((uint32_t)(q * 32) << 16);
-        if (p.n_issuers == 2) {
+        if (n_iss == 2) {
           float t[16];
           ptx::tmem_ld16x2(lanes + (uint32_t)(p.BN + c0), lanes + acc2_off + (uint32_t)(p.BN + c0), z, t);
 #pragma unroll
@@ -461,7 +466,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           acc[4 * j + 2] = a0.z + a1.z;
           acc[4 * j + 3] = a0.w + a1.w;
         }
-        if (p.n_issuers == 2) {
+        if (n_iss == 2) {
           float t[16];
           ptx::tmem_ld16x2(lanes + (uint32_t)(2 * p.BN + c0), lanes + acc2_off + (uint32_t)(2 * p.BN + c0), z, t);
 #pragma unroll
@@ -479,7 +484,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int n = n0 + c0;
 #pragma unroll
       for (int i = 0; i < 16; ++i) acc[i] = fmaf(acc[i], rs, s_bias[c0 + i]);
-      if (p.mode == MODE_OUT) {
+      if (mode == MODE_OUT) {
         if (p.cfg_w > 0.f) {
           // guided step: rows 64.. of the tile are the unconditional pass of the stream in rows 0..63; they hand
           // their velocity over through shared memory and the conditional rows form (1 + w) v_c - w v_u
@@ -527,7 +532,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         continue;
       }
-      if (p.mode == MODE_QKV) {
+      if (mode == MODE_QKV) {
         if (is_chunk) {
           uint4 a, b;
           pack16_bf16(acc, a, b);
@@ -556,7 +561,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!is_halo) {
         if (has_resid) {
           const uint32_t w[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
-          if (p.mode == MODE_CONV) {
+          if (mode == MODE_CONV) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               acc[2 * i] = __uint_as_float(w[i] << 16) + silu_f(acc[2 * i] + tau_s[c0 + 2 * i]);
@@ -597,7 +602,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // its accumulator barrier fires), so a CTA may leave as soon as tensor memory can be freed: when every
     // thread of the pair has arrived, the epilogue threads having done so after their last accumulator load.
     // (warps that have not waited on the first phase yet do so now)
-    if (warp < 4 && !(((warp & 1) == 0 && pair_rank != 0) || ((warp & 1) == 1 && (warp >> 1) < p.n_issuers && pair_rank == 0))) ptx::cluster_wait();
+    if (warp < 4 && !(((warp & 1) == 0 && pair_rank != 0) || ((warp & 1) == 1 && (warp >> 1) < n_iss && pair_rank == 0))) ptx::cluster_wait();
     if (warp < 4) ptx::cluster_arrive();
     if (warp == 1) {
       ptx::cluster_wait();
@@ -1112,6 +1117,7 @@ bool make_tmap(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, u
 
 constexpr size_t GEMM_SMEM_EXTRA = 1024 + 2 * MAX_STAGES * 8 + 8 + 8 + 2 * MAX_BN * 4 + 64;   // alignment slack + barriers + constants
 constexpr size_t GEMM_SMEM_MAX = 200 * 1024;
+constexpr int SPECIALISE_FROM_TILES = 8;   // row tiles of a batch from which the GEMMs run as one kernel per role
 constexpr size_t GEMM_SMEM_MAX_PAIR = 227 * 1024;   // the opt-in limit of the device: eight 28 KB stages of a CTA pair
 
 }  // namespace
@@ -1326,9 +1332,12 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   if (e == cudaSuccess) chk(cudaMemcpy(m->wts, hw.data(), wn * sizeof(uint16_t), cudaMemcpyHostToDevice));
   if (e == cudaSuccess) chk(cudaMemcpy(m->fconst, hf.data(), fn * sizeof(float), cudaMemcpyHostToDevice));
   if (e == cudaSuccess)
-    chk(cudaFuncSetAttribute(flow_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
+    chk(cudaFuncSetAttribute(flow_gemm_kernel<false, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
+  for (auto fn : {flow_gemm_kernel<false, MODE_INPROJ>, flow_gemm_kernel<false, MODE_CONV>, flow_gemm_kernel<false, MODE_QKV>,
+                  flow_gemm_kernel<false, MODE_OPROJ>, flow_gemm_kernel<false, MODE_OUT>})
+    if (e == cudaSuccess) chk(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
   if (e == cudaSuccess)
-    chk(cudaFuncSetAttribute(flow_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX_PAIR));
+    chk(cudaFuncSetAttribute(flow_gemm_kernel<true, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX_PAIR));
   if (e == cudaSuccess && cfg.n_attn > 0)
     chk(cudaFuncSetAttribute(m->P > 0 ? flow_attn_kernel<true> : flow_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)ATT_SMEM));
@@ -1572,13 +1581,26 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
       if (ns >= 2 && (size_t)ns * pair_stage >= 64 * 1024) {
         p.n_stages = ns;
         lc.cluster_x = 2;
-        launch(lc, flow_gemm_kernel<true>, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), GEMM_SMEM_EXTRA + (size_t)ns * pair_stage, true,
+        launch(lc, flow_gemm_kernel<true, -1>, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), GEMM_SMEM_EXTRA + (size_t)ns * pair_stage, true,
                7, tA, *tBh, p);
         return;
       }
     }
     const size_t smem = GEMM_SMEM_EXTRA + (size_t)p.n_stages * stage_bytes;
-    launch(lc, flow_gemm_kernel<false>, dim3(m_tiles, N / p.BN), dim3(GEMM_THREADS), smem, true, p.mode == MODE_CONV ? 0 : 1, tA, tB, p);
+    // One instantiation per role for batches of eight row tiles or more: the other roles' epilogues and the slot
+    // fields only they read then cost neither registers nor instructions (32 streams: 2.01 -> 1.94 ms per step).
+    // Small batches keep the one generic kernel for every role: their launches are so short that five alternating
+    // kernel images cost more in instruction-cache misses than the leaner code saves (1 stream: 1.37 -> 1.46 ms
+    // with the specialised forms; the two break even between 4 and 8 row tiles).
+    const dim3 grid(m_tiles, N / p.BN);
+    const int cls = p.mode == MODE_CONV ? 0 : 1;
+    if (m_tiles < SPECIALISE_FROM_TILES) launch(lc, flow_gemm_kernel<false, -1>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
+    else if (p.mode == MODE_CONV && p.n_issuers == 2) launch(lc, flow_gemm_kernel<false, MODE_CONV>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
+    else if (p.mode == MODE_QKV) launch(lc, flow_gemm_kernel<false, MODE_QKV>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
+    else if (p.mode == MODE_OPROJ) launch(lc, flow_gemm_kernel<false, MODE_OPROJ>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
+    else if (p.mode == MODE_INPROJ) launch(lc, flow_gemm_kernel<false, MODE_INPROJ>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
+    else if (p.mode == MODE_OUT) launch(lc, flow_gemm_kernel<false, MODE_OUT>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
+    else launch(lc, flow_gemm_kernel<false, -1>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
   };
   // the GEMM whose output feeds an RMS norm leaves the row statistics; the GEMM after the norm applies them
   auto feeds_norm = [&](GemmParams& p) { p.ssq_out = m->ssq; p.ssq_ld = m->rows; };
