@@ -159,7 +159,7 @@ __device__ __forceinline__ void store16(bf16* p, const uint4& a, const uint4& b)
 // has told it that the even CTA's barriers exist, and that barrier, with the pair allocation of tensor memory,
 // puts the first full stage 0.4 to 1.6 microseconds later - more than the loop saves in a 7-microsecond kernel.
 // Hence an option (DC_OPT_CTA_PAIRS), off by default.
-template <bool PAIR, int MODE_T>
+template <bool PAIR, int MODE_T, int BN_T = 0>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -168,6 +168,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int mode = MODE_T >= 0 ? MODE_T : p.mode;
   const int n_taps = MODE_T == MODE_CONV ? 3 : (MODE_T >= 0 ? 1 : p.taps);
   const int n_iss = MODE_T == MODE_CONV ? 2 : p.n_issuers;
+  const int BN = BN_T > 0 ? BN_T : p.BN;   // BN_T > 0: the tile width known at compile time (the chunk loop of the epilogue unrolls away)
   if (p.empty) {
     ptx::pdl_launch();
     ptx::pdl_wait();
@@ -178,7 +179,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // 1024 B.  The weight tiles of a conv block's three taps are adjacent, so that they form one
   // operand of 3 BN rows.
   // (PAIR: a "tile" is one of the CTA's `taps` units of BN / 2 weight rows; BN is then a multiple of 16)
-  const uint32_t b_bytes = PAIR ? (uint32_t)p.BN * 64u : (uint32_t)p.BN * 128u;
+  const uint32_t b_bytes = PAIR ? (uint32_t)BN * 64u : (uint32_t)BN * 128u;
   const uint32_t b_tile = (b_bytes + 1023u) & ~1023u;
   const uint32_t stage_bytes = (uint32_t)A_BYTES + (uint32_t)n_taps * b_tile;
   const int STAGES = p.n_stages;
@@ -191,14 +192,14 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   float* s_tau = s_bias + MAX_BN;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * TILE_M, n0 = blockIdx.y * p.BN;
+  const int m0 = blockIdx.x * TILE_M, n0 = blockIdx.y * BN;
   const uint32_t pair_rank = PAIR ? ptx::cluster_ctarank() : 0u;   // 0: issues the UMMAs and owns the "full" barriers
   // Accumulator: BN columns, or 3 BN for a conv block, whose three taps are the column blocks of ONE
   // product Z = X [W_0 | W_1 | W_2] (a row shift commutes with the product, so the taps are shifted
   // and added in the epilogue; a tcgen05.mma costs about 47 cycles however small it is, and one
   // 128 x 3BN x 16 instruction replaces three 128 x BN x 16 ones).  The second issuer's accumulator
   // sits acc2_off columns after the first.
-  const uint32_t acc_w = (uint32_t)(n_taps * p.BN);
+  const uint32_t acc_w = (uint32_t)(n_taps * BN);
   const uint32_t acc2_off = acc_w <= 32 ? 32u : (acc_w <= 64 ? 64u : (acc_w <= 128 ? 128u : 256u));
   const uint32_t need_cols = n_iss == 2 ? 2u * acc2_off : acc_w;
   const uint32_t tmem_cols = need_cols <= 32 ? 32u : (need_cols <= 64 ? 64u : (need_cols <= 128 ? 128u : (need_cols <= 256 ? 256u : 512u)));
@@ -246,7 +247,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int j = 0; j < 3; ++j) {
           const int u = taps * (int)pair_rank + j;
           ux[j] = (u >> 1) * nkb * KBLK;
-          uy[j] = n0 + (u & 1) * (p.BN >> 1);
+          uy[j] = n0 + (u & 1) * (BN >> 1);
         }
       }
       const uint32_t full0 = PAIR ? ptx::map_to_cta(ptx::smem_u32(&full[0]), 0u) : 0u;
@@ -302,7 +303,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const uint32_t on = lane == 0;
       // the weight tiles of the taps are adjacent in the stage (BN rows of 128 B each, BN a multiple of 8),
       // so together they are one K-major operand of taps * BN rows
-      const uint32_t idesc = ptx::umma_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, n_taps * p.BN, 0, 0);
+      const uint32_t idesc = ptx::umma_idesc_bf16(PAIR ? 2 * TILE_M : TILE_M, n_taps * BN, 0, 0);
       // PAIR: every completion is reported to both CTAs (their producers and epilogues wait on barriers of their own)
       const uint32_t empty_mine = ptx::smem_u32(&empty[0]), empty_peer = PAIR ? ptx::map_to_cta(empty_mine, 1u) : 0u;
       const int nkb = p.n_kblocks, step = n_iss;
@@ -351,10 +352,10 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // per-column constants go to shared memory, the thread's residual row (or, for a left-context
     // row, the carried row) goes to registers.
     const int et = threadIdx.x - 128;
-    if (et < p.BN) s_bias[et] = p.bias[n0 + et];   // BN <= 192 < EPI_THREADS
+    if (et < BN) s_bias[et] = p.bias[n0 + et];   // BN <= 192 < EPI_THREADS
     ptx::pdl_wait();                              // slot table, residual and carry rows are upstream data
-    if (p.tau != nullptr && et < 2 * p.BN) {      // conv blocks (BN <= 64): the timestep bias of each of the tile's two slots
-      const int sl = et / p.BN, c = et - sl * p.BN, ts = m0 / SLOT_ROWS + sl;
+    if (p.tau != nullptr && et < 2 * BN) {      // conv blocks (BN <= 64): the timestep bias of each of the tile's two slots
+      const int sl = et / BN, c = et - sl * BN, ts = m0 / SLOT_ROWS + sl;
       s_tau[sl * 64 + c] = ts < p.n_slots ? p.tau[p.slots[ts].tau_off + n0 + c] : 0.f;
     }
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
@@ -381,7 +382,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (src != nullptr) {
 #pragma unroll
         for (int k = 0; k < PRE_CHUNKS; ++k) {
-          if (16 * (EPI_GROUPS * k + cg) < p.BN) {
+          if (16 * (EPI_GROUPS * k + cg) < BN) {
             pre[2 * k] = *reinterpret_cast<const uint4*>(src + 16 * (EPI_GROUPS * k + cg));
             pre[2 * k + 1] = *reinterpret_cast<const uint4*>(src + 16 * (EPI_GROUPS * k + cg) + 8);
           }
@@ -416,12 +417,12 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // PAIR: tensor memory is freed for both CTAs at once, so each thread reports its LAST accumulator load
     // to the cluster barrier as soon as it has happened; the barrier's latency (about 1500 cycles) then runs
     // under the arithmetic and the stores that follow, and the freeing warp finds it complete.
-    const int last_kk = (p.BN - 16 * cg - 1) / (16 * EPI_GROUPS);   // (BN > 16 cg for every chunk group of a paired GEMM)
+    const int last_kk = (BN - 16 * cg - 1) / (16 * EPI_GROUPS);   // (BN > 16 cg for every chunk group of a paired GEMM)
 #pragma unroll
     for (int kk = 0; kk < MAX_BN / (16 * EPI_GROUPS); ++kk) {
       const int ch = EPI_GROUPS * kk + cg;
       const int c0 = ch * 16;
-      if (c0 >= p.BN) break;
+      if (c0 >= BN) break;
       float acc[16];
       if (n_iss == 2) {   // even blocks + odd blocks, always in this order
         float acc2[16];
@@ -441,11 +442,11 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t lanes = tmem_base + ((uint32_t)(q * 32) << 16);
         if (n_iss == 2) {
           float t[16];
-          ptx::tmem_ld16x2(lanes + (uint32_t)(p.BN + c0), lanes + acc2_off + (uint32_t)(p.BN + c0), z, t);
+          ptx::tmem_ld16x2(lanes + (uint32_t)(BN + c0), lanes + acc2_off + (uint32_t)(BN + c0), z, t);
 #pragma unroll
           for (int i = 0; i < 16; ++i) z[i] += t[i];
         } else {
-          ptx::tmem_ld16(lanes + (uint32_t)(p.BN + c0), z);
+          ptx::tmem_ld16(lanes + (uint32_t)(BN + c0), z);
         }
         // exchange area of this chunk group: Z_0 then Z_1, each [4 float4 columns][128 rows] (a warp's 32 rows
         // are 512 contiguous bytes, shifted or not: no bank conflicts); conv tiles have <= 64 columns, so kk = 0
@@ -468,11 +469,11 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         if (n_iss == 2) {
           float t[16];
-          ptx::tmem_ld16x2(lanes + (uint32_t)(2 * p.BN + c0), lanes + acc2_off + (uint32_t)(2 * p.BN + c0), z, t);
+          ptx::tmem_ld16x2(lanes + (uint32_t)(2 * BN + c0), lanes + acc2_off + (uint32_t)(2 * BN + c0), z, t);
 #pragma unroll
           for (int i = 0; i < 16; ++i) z[i] += t[i];
         } else {
-          ptx::tmem_ld16(lanes + (uint32_t)(2 * p.BN + c0), z);
+          ptx::tmem_ld16(lanes + (uint32_t)(2 * BN + c0), z);
         }
 #pragma unroll
         for (int i = 0; i < 16; ++i) acc[i] += z[i];
@@ -1333,8 +1334,9 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   if (e == cudaSuccess) chk(cudaMemcpy(m->fconst, hf.data(), fn * sizeof(float), cudaMemcpyHostToDevice));
   if (e == cudaSuccess)
     chk(cudaFuncSetAttribute(flow_gemm_kernel<false, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
-  for (auto fn : {flow_gemm_kernel<false, MODE_INPROJ>, flow_gemm_kernel<false, MODE_CONV>, flow_gemm_kernel<false, MODE_QKV>,
-                  flow_gemm_kernel<false, MODE_OPROJ>, flow_gemm_kernel<false, MODE_OUT>})
+  for (auto fn : {flow_gemm_kernel<false, MODE_INPROJ>, flow_gemm_kernel<false, MODE_CONV>, flow_gemm_kernel<false, MODE_CONV, 64>,
+                  flow_gemm_kernel<false, MODE_QKV>, flow_gemm_kernel<false, MODE_OPROJ>,
+                  flow_gemm_kernel<false, MODE_OUT>})
     if (e == cudaSuccess) chk(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX));
   if (e == cudaSuccess)
     chk(cudaFuncSetAttribute(flow_gemm_kernel<true, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX_PAIR));
@@ -1595,6 +1597,11 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     const dim3 grid(m_tiles, N / p.BN);
     const int cls = p.mode == MODE_CONV ? 0 : 1;
     if (m_tiles < SPECIALISE_FROM_TILES) launch(lc, flow_gemm_kernel<false, -1>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
+    // (a conv block's widest tile, that of a full batch, also has its width fixed at compile time - the epilogue's chunk
+    // loop unrolls away: 1.94 -> 1.91 ms per step; the same for the other roles, or a second conv image per kind of
+    // tail - carried rows / row statistics - measured nothing or cost what another kernel image costs)
+    else if (p.mode == MODE_CONV && p.n_issuers == 2 && p.BN == 64)
+      launch(lc, flow_gemm_kernel<false, MODE_CONV, 64>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
     else if (p.mode == MODE_CONV && p.n_issuers == 2) launch(lc, flow_gemm_kernel<false, MODE_CONV>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
     else if (p.mode == MODE_QKV) launch(lc, flow_gemm_kernel<false, MODE_QKV>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
     else if (p.mode == MODE_OPROJ) launch(lc, flow_gemm_kernel<false, MODE_OPROJ>, grid, dim3(GEMM_THREADS), smem, true, cls, tA, tB, p);
