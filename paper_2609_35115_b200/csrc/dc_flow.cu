@@ -418,7 +418,10 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // to the cluster barrier as soon as it has happened; the barrier's latency (about 1500 cycles) then runs
     // under the arithmetic and the stores that follow, and the freeing warp finds it complete.
     const int last_kk = (BN - 16 * cg - 1) / (16 * EPI_GROUPS);   // (BN > 16 cg for every chunk group of a paired GEMM)
-#pragma unroll
+    // (in the generic kernel, the one of small batches, the loop stays a loop: three unrolled copies of the epilogue
+    // body are code that has to come through the instruction cache at every one of their short launches - cfg3 1.371 ->
+    // 1.359 ms per chunk; the kernels of a role keep them: a QKV thread overlaps its three chunks, 1.911 against 1.926)
+#pragma unroll(MODE_T >= 0 ? MAX_BN / (16 * EPI_GROUPS) : 1)
     for (int kk = 0; kk < MAX_BN / (16 * EPI_GROUPS); ++kk) {
       const int ch = EPI_GROUPS * kk + cg;
       const int c0 = ch * 16;
