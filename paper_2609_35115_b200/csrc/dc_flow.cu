@@ -559,7 +559,7 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (is_chunk) {
           uint4 a, b;
           pack16_bf16(acc, a, b);
-          const int which = n / p.C, col = n - which * p.C;
+          const int which = (n >= p.C) + (n >= 2 * p.C), col = n - which * p.C;   // 0: Q, 1: K, 2: V (no division)
           if (which == 0) {
             store16(p.q_out + grow * p.ld + col, a, b);
           } else {
