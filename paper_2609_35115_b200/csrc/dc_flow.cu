@@ -574,7 +574,13 @@ flow_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               row += p.P;
             }
             const int hh = col >> p.dh_shift, wi = col - (hh << p.dh_shift);
-            store16(si.kv + p.kv_off + (long long)(which - 1) * (p.P + p.Rk) * p.C + (long long)hh * p.kv_hs + (long long)row * p.kv_rs + wi, a, b);
+            // head_dim 64: a K / V row is stored with its 16-byte chunks in the order of the swizzled shared-memory row
+            // that the attention kernel copies it to, chunk c at position c ^ (row & 7).  The two chunks of this
+            // thread stay inside their 32 bytes, swapped for odd rows.
+            const int wp = p.dh_shift == 6 ? ((((wi >> 3) ^ (row & 7)) & ~1) << 3) : wi;
+            const bool swap = p.dh_shift == 6 && (row & 1);
+            store16(si.kv + p.kv_off + (long long)(which - 1) * (p.P + p.Rk) * p.C + (long long)hh * p.kv_hs + (long long)row * p.kv_rs + wp,
+                    swap ? b : a, swap ? a : b);
           }
         }
         continue;
@@ -788,7 +794,14 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
 
 // PROMPT = false: the carry is a plain window (no prompt rows); a separate instantiation, because this kernel sits at its
 // register limit and the copy loops of its loader warps pace it.
-template <bool PROMPT>
+// BULK (no prompt rows, head_dim 64): a head's K / V rows are 128 contiguous bytes each, stored with their 16-byte
+// chunks already in the order of the swizzled shared-memory row they will occupy (chunk c of plane row r at
+// position c ^ (r & 7)), and the ring is walked from the 8-row boundary below the attended interval, so that a block
+// of 128 keys is one flat span of 16 KB (two at the ring's wrap) with shared-memory row == plane row (mod 8): ONE thread
+// fetches it with one or two untiled bulk copies that complete on the stage's barrier.  The up to seven keys in front
+// of the interval are masked like the padding behind it.  Without BULK the loader warps copy 16 bytes per thread and
+// instruction (about 2,800 cycles of issue per block and warp).
+template <bool PROMPT, bool BULK>
 __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t att_smem_raw[];
   uint8_t* smem = att_smem_raw;
@@ -816,7 +829,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   uint64_t* bar_p = bar_s + 1;          // [2]: all softmax threads have written P(b) into buffer b & 1
   uint64_t* bar_pv = bar_p + 2;         // [2]: P(b) V(b) has been accumulated: buffer b & 1 is free, O holds blocks <= b
   uint64_t* bar_sfree = bar_pv + 2;     // every softmax thread has copied its S columns to registers
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_sfree + 1);
+  uint64_t* bar_q = bar_sfree + 1;      // BULK: Q has landed (without BULK it is published with the first K block)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_sfree + 2);
   float* s_x = reinterpret_cast<float*>(tmem_slot + 2);   // [2][64] exchange between the two column halves
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -825,9 +839,9 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
 
   if (tid == 0) {
     for (int i = 0; i < ATT_STAGES; ++i) {
-      ptx::mbar_init(&full_k[i], ATT_K_LOADERS);
+      ptx::mbar_init(&full_k[i], BULK ? 1 : ATT_K_LOADERS);
       ptx::mbar_init(&empty_k[i], 1);
-      ptx::mbar_init(&full_v[i], ATT_V_LOADERS);
+      ptx::mbar_init(&full_v[i], BULK ? 1 : ATT_V_LOADERS);
       ptx::mbar_init(&empty_v[i], 1);
     }
     ptx::mbar_init(bar_s, 1);
@@ -836,6 +850,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
       ptx::mbar_init(&bar_pv[i], 1);
     }
     ptx::mbar_init(bar_sfree, 128);
+    ptx::mbar_init(bar_q, ATT_K_LOADERS);
     ptx::fence_barrier_init();
   }
   if (warp == 4) ptx::tmem_alloc(tmem_slot, ATT_TMEM_COLS);
@@ -854,11 +869,68 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
   // the carried history and the chunk's history frames, a circular interval of the ring behind the prompt rows
   const int T = si.T;
   const int n_prompt = PROMPT ? si.n_prompt0 + min(T, p.P - si.n_prompt0) : 0;
-  const int L = PROMPT ? n_prompt + si.kv_len + (T - (n_prompt - si.n_prompt0)) : si.kv_len + T;
+  const int L0 = PROMPT ? n_prompt + si.kv_len + (T - (n_prompt - si.n_prompt0)) : si.kv_len + T;
+  int ring_start = si.kv_head - si.kv_len;      // ring row of the oldest attended history frame
+  if (ring_start < 0) ring_start += p.Rk;
+  const int phi = BULK ? (ring_start & 7) : 0;  // BULK: keys 0 .. phi - 1 are the rows between the 8-row boundary and the interval
+  const int L = L0 + phi;
   const int nkb = (L + ATT_KB - 1) / ATT_KB;
 
   if (T == 0) {
     // a slot without frames (a hole in a wavefront): nothing to do but to release tensor memory below
+  } else if (BULK && warp >= 5) {
+    // ---------------- loaders, bulk copies: lane 0 of warp 5 fetches the K blocks, lane 0 of warp 7 the V blocks;
+    // warps 5 and 6 copy Q (64 rows of the projection's output, each held twice) ----------------
+    const bool is_k = warp != 7;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    const bf16* src0 = si.kv + p.kv_off + (long long)head * p.kv_hs + (is_k ? 0 : (long long)p.Rk * p.C);
+    uint64_t* full = is_k ? full_k : full_v;
+    uint64_t* empty = is_k ? empty_k : empty_v;
+    const int row0 = ring_start - phi;                     // a multiple of 8 (the ring has a multiple of 8 rows)
+    const int n_early = min(min((si.kv_len + phi) / ATT_KB, ATT_STAGES), nkb);   // blocks of carried rows only (< nkb: the chunk's rows come last)
+    bool ok = true;
+    auto fetch = [&](int b) {                               // warps 5 and 7, all lanes (lane 0 issues)
+      const int st = b % ATT_STAGES;
+      if (b >= ATT_STAGES && ok && !ptx::mbar_wait_relaxed(&empty[st], ((b / ATT_STAGES) - 1) & 1)) {
+        ok = false;
+        atomicExch(p.err, 4);
+      }
+      uint8_t* dstb = ring + st * ATT_STAGE_BYTES + (is_k ? 0 : ATT_KB * 128);
+      const int n = min(ATT_KB, L - b * ATT_KB);            // key rows of this block
+      if (!is_k && n < ATT_KB) {
+        // the P V product reads whole 16-row steps: the rows behind the last key must be finite (their weights are 0)
+        const int n16 = min(ATT_KB, (n + 15) & ~15);
+        for (int i = lane; i < (n16 - n) * 8; i += 32) *reinterpret_cast<uint4*>(dstb + n * 128 + i * 16) = zero;
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+      }
+      if (lane == 0) {
+        int rr = row0 + b * ATT_KB;
+        while (rr >= p.Rk) rr -= p.Rk;
+        const int n1 = min(n, p.Rk - rr);
+        ptx::mbar_expect_tx(&full[st], (uint32_t)n * 128u);
+        ptx::bulk_load(dstb, src0 + (long long)rr * 64, (uint32_t)n1 * 128u, &full[st]);
+        if (n1 < n) ptx::bulk_load(dstb + n1 * 128, src0, (uint32_t)(n - n1) * 128u, &full[st]);
+      }
+    };
+    if (warp != 6)
+      for (int b = 0; b < n_early; ++b) fetch(b);           // (b < ATT_STAGES: no stage to wait for)
+    ptx::pdl_wait();                                        // Q and the chunk's own K / V rows are the projection's output
+    if (is_k) {
+      const int lt = (warp == 6 ? 32 : 0) + lane;
+      const bf16* qbase = p.q + (long long)(GUARD + slot * SLOT_ROWS + HALO) * p.ld + head * 64;
+      for (int i = lt; i < 128 * 8; i += ATT_K_LOADERS) {
+        const int row = i >> 3, j = i & 7, qrow = row & 63;   // rows 64.. repeat rows 0..
+        uint8_t* dst = sQ + row * 128 + ((j ^ (row & 7)) << 4);
+        if (qrow < T) cp_async16(dst, qbase + (long long)qrow * p.ld + j * 8);
+        else *reinterpret_cast<uint4*>(dst) = zero;
+      }
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      ptx::fence_proxy_async_smem();
+      ptx::mbar_arrive(bar_q);
+    }
+    if (warp != 6)
+      for (int b = n_early; b < nkb; ++b) fetch(b);
   } else if (warp >= 5) {
     // ---------------- loaders ----------------
     const bool is_k = warp != 7;
@@ -869,8 +941,9 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
     const int rs = p.kv_rs;
     uint64_t* full = is_k ? full_k : full_v;
     uint64_t* empty = is_k ? empty_k : empty_v;
-    int start = si.kv_head - si.kv_len;
-    if (start < 0) start += p.Rk;
+    const int start = ring_start;
+    // head_dim 64: chunk j of plane row rr is stored at position j ^ (rr & 7) (see BULK); head_dim 32 rows are stored plainly
+    const int perm = p.dh == 64 ? 7 : 0;
     auto issue_block = [&](int b) {
       uint8_t* dstb = ring + (b % ATT_STAGES) * ATT_STAGE_BYTES + (is_k ? 0 : ATT_KB * 128);
       if (!PROMPT) {
@@ -881,7 +954,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
           if (key < L && j < chunks) {
             int rr = start + key;
             if (rr >= p.Rk) rr -= p.Rk;
-            cp_async16(dstb + off, src0 + (long long)rr * rs + j * 8);
+            cp_async16(dstb + off, src0 + (long long)rr * rs + ((j ^ (rr & perm)) << 3));
           } else {
             *reinterpret_cast<uint4*>(dstb + off) = zero;   // for V: 0 * garbage must not poison O
           }
@@ -891,7 +964,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         for (int i = lt; i < ATT_KB * 8; i += nl) {
           const int row = i >> 3, j = i & 7;
           const int off = row * 128 + ((j ^ (row & 7)) << 4);
-          if (j < chunks) cp_async16(dstb + off, src0 + (long long)(b * ATT_KB + row) * rs + j * 8);
+          if (j < chunks) cp_async16(dstb + off, src0 + (long long)(b * ATT_KB + row) * rs + ((j ^ (row & perm)) << 3));
           else *reinterpret_cast<uint4*>(dstb + off) = zero;
         }
       } else {
@@ -907,7 +980,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
               if (rr >= p.Rk) rr -= p.Rk;
               rr += p.P;
             }
-            cp_async16(dstb + off, src0 + (long long)rr * rs + j * 8);
+            cp_async16(dstb + off, src0 + (long long)rr * rs + ((j ^ (rr & perm)) << 3));
           } else {
             *reinterpret_cast<uint4*>(dstb + off) = zero;
           }
@@ -968,6 +1041,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
         ptx::umma_commit(bar_s);
         ptx::umma_commit(&empty_k[st]);                  // the K stage is free once S(b) has been computed
       };
+      if (BULK && !ptx::mbar_wait(bar_q, 0)) { ok = false; atomicExch(p.err, 12); }
       issue_s(0);
       for (int b = 0; b < nkb; ++b) {
         const int st = b % ATT_STAGES;
@@ -1018,6 +1092,11 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) flow_attn_kernel(const AttnPar
 #pragma unroll
         for (int i = 0; i < 64; ++i)
           if (i >= valid) v[i] = -INFINITY;
+      }
+      if (BULK && b == 0 && half == 0) {         // the rows between the 8-row boundary and the attended interval
+#pragma unroll
+        for (int i = 0; i < 7; ++i)
+          if (i < phi) v[i] = -INFINITY;
       }
       float mx = -INFINITY;
 #pragma unroll
@@ -1243,7 +1322,9 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   m->n_pass = cfg.cfg_scale > 0.f ? 2 : 1;
   m->S = cfg.max_batch * m->n_pass;
   m->rows = ((m->S * SLOT_ROWS + TILE_M - 1) / TILE_M) * TILE_M;
-  m->Rk = cfg.kv_cap + cfg.f_chunk + cfg.f_lookahead;
+  // (a multiple of 8 rows: the attention kernel walks the ring in whole 8-row groups of its swizzled tiles; the extra
+  // rows only delay the overwriting of frames that are no longer attended)
+  m->Rk = (cfg.kv_cap + cfg.f_chunk + cfg.f_lookahead + 7) & ~7;
   m->P = cfg.f_prompt;
   m->cpa = cfg.n_attn > 0 ? cfg.n_conv / cfg.n_attn : cfg.n_conv;
   const int nL = cfg.n_conv, nA = cfg.n_attn, nS = cfg.n_steps;
@@ -1363,8 +1444,8 @@ dc_status flow_model_create(const dc_config& cfg, const float* w, FlowModel** ou
   if (e == cudaSuccess)
     chk(cudaFuncSetAttribute(flow_gemm_kernel<true, -1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM_MAX_PAIR));
   if (e == cudaSuccess && cfg.n_attn > 0)
-    chk(cudaFuncSetAttribute(m->P > 0 ? flow_attn_kernel<true> : flow_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)ATT_SMEM));
+    chk(cudaFuncSetAttribute(m->P > 0 ? flow_attn_kernel<true, false> : (cfg.head_dim == 64 ? flow_attn_kernel<false, true> : flow_attn_kernel<false, false>),
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATT_SMEM));
   if (e != cudaSuccess) {
     set_error("flow model allocation failed: %s", cudaGetErrorString(e));
     flow_model_destroy(m);
@@ -1652,7 +1733,8 @@ void enqueue_chunk(FlowModel* m, int n, const SlotSet* sets, int n_sets, LaunchC
     p.scale_log2e = (float)(1.4426950408889634 / sqrt((double)c.head_dim));
     p.err = m->d_err;
     p.empty = (c.options & DC_OPT_EMPTY_KERNELS) ? 1 : 0;
-    launch(lc, m->P > 0 ? flow_attn_kernel<true> : flow_attn_kernel<false>, dim3(n, c.n_heads), dim3(ATT_THREADS), ATT_SMEM, true, 2, p);
+    launch(lc, m->P > 0 ? flow_attn_kernel<true, false> : (c.head_dim == 64 ? flow_attn_kernel<false, true> : flow_attn_kernel<false, false>),
+           dim3(n, c.n_heads), dim3(ATT_THREADS), ATT_SMEM, true, 2, p);
   };
   const float* fc = m->fconst;
   const long long halo_stride = (long long)HALO * C;

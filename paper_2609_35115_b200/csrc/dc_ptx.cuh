@@ -93,6 +93,14 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* m, int
       : "memory");
 }
 
+// Untiled bulk copy global -> shared (no tensor map): `bytes` (a multiple of 16) from a 16-byte aligned source to a
+// 16-byte aligned destination in this CTA's shared memory; completion counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+               "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
 // ---- tensor memory ----------------------------------------------------------------------------
 // Allocates `ncols` (power of two >= 32) TMEM columns; the base address lands in *slot (shared).
 // Must be executed by one full warp.
