@@ -45,6 +45,20 @@ def test_flow_max_chunk_and_cap_shorter_than_chunk(dc):
     _check(dc, cfg, [0, 56, 57, 113, 120, 176, 177, 178, 234], TOL_BF16)
 
 
+def test_flow_bulk_loader_small_ring_ragged(dc):
+    # head_dim 64 without prompt rows takes the attention kernel's bulk-copy loader: a ring of 64 rows (cap 8 + chunk
+    # 56) wraps inside almost every key block, the attended interval starts at every offset from its 8-row boundary
+    # (single frames included), and the one key block is always partial (zero-filled V rows behind the last key)
+    cfg = wl.tiny_flow(name="edge_bulk_cap8", hidden=128, n_heads=2, head_dim=64, kv_cap=8, f_chunk=56, mel_dim=16,
+                       dilations=(2, 4), n_attn_layers=2, n_steps=2, seed=35)
+    _check(dc, cfg, [0, 56, 57, 58, 61, 117, 120, 127, 183, 184, 191, 247, 250], TOL_BF16)
+    # ... and a carry of 200 frames: two key blocks, the second one partial, interval offsets 0..7 by single-frame steps
+    cfg = wl.tiny_flow(name="edge_bulk_cap200", hidden=64, n_heads=1, head_dim=64, kv_cap=200, f_chunk=50,
+                       dilations=(1,), n_attn_layers=1, n_steps=1, seed=36)
+    bnd = [0, 50, 100, 150, 200, 250] + [251 + i for i in range(9)] + [309, 359, 360, 410]
+    _check(dc, cfg, bnd, TOL_BF16)
+
+
 def test_flow_long_carry_many_key_blocks(dc):
     # kv_cap 700: up to 6 key blocks per query, ring of 750 rows wrapped once
     cfg = wl.tiny_flow(name="edge_cap700", hidden=64, n_heads=1, head_dim=64, kv_cap=700, f_chunk=50,
